@@ -1,0 +1,399 @@
+// LogQuant CPU oracle  --  TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+//
+// A plain, slow, single-pass C++17 restatement of what the decode-time hot path of
+// LogQuant computes.  It exists so that the CUDA library can be checked element by
+// element; only the test-suite, the smoke check and the benchmark's CPU-baseline leg
+// may call it.  It shares no code, header, table or helper with the CUDA library.
+//
+// What each part follows (paper = "LogQuant: Log-Distributed 2-Bit Quantization of
+// KV Cache", arXiv 2503.19950):
+//   * filter        : Algorithm 1 (AppendToken) with Python slice semantics, Sec. 2.5.
+//   * quantiser     : the paper only names "INT2", group size G and the "Key-per-channel
+//                     strategy" (Sec. 2.5 Implementation, Sec. 3.1 Settings).  The reading
+//                     taken here is asymmetric min/max quantisation:
+//                         zero  = min(group)                         (a bf16 value, exact)
+//                         scale = bf16_rne((max - min) / 3)          (fp32 IEEE ops)
+//                         code  = clamp(rint((x - zero) / scale), 0, 3), all 0 if scale == 0
+//                         x^    = zero + code * scale
+//                     keys: one group = G consecutive evicted tokens of one channel;
+//                     values: one group = G consecutive channels of one token.
+//   * packer        : 4 codes per byte, channel 4j+i in bits [2i+1:2i] of byte j.
+//   * attention     : Eq. 2 with the 1/sqrt(d) scale of the appendix (passed in as
+//                     sm_scale), float64, one pass with max subtraction, over the union
+//                     of the full-precision list and the dequantised store.  Eq. 3
+//                     (position-agnostic attention) is what allows the union to be
+//                     visited in any order.
+//
+// Parity status: filter, quantiser, packer and attention are pinned by tests that do
+// not go through this file's own formulas (hand simulation of Algorithm 1, closed
+// forms, a hand-worked quantiser example, library softmax attention, brute force).
+// Parity with the paper's own numbers is UNPINNED: the paper prints no worked numeric
+// example and delegates its quantiser to a library it does not describe.
+//
+// Build:  g++ -O2 -std=c++17 -ffp-contract=off -fPIC -shared -pthread
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <thread>
+#include <vector>
+
+namespace {
+
+// ---- bf16 <-> fp32 (bit manipulation; finite inputs) -------------------------------
+float bf16_to_f32(uint16_t h) {
+  uint32_t u = static_cast<uint32_t>(h) << 16;
+  float f;
+  std::memcpy(&f, &u, sizeof f);
+  return f;
+}
+
+uint16_t f32_to_bf16_rne(float f) {
+  uint32_t u;
+  std::memcpy(&u, &f, sizeof u);
+  uint32_t lsb = (u >> 16) & 1u;
+  u += 0x7FFFu + lsb;  // round to nearest, ties to even
+  return static_cast<uint16_t>(u >> 16);
+}
+
+// ---- quantiser: one group of n values, read with a stride --------------------------
+// All arithmetic is IEEE binary32 with one rounding per operation (the file is built
+// with -ffp-contract=off so no multiply-add is ever contracted).
+void quantize_group(const uint16_t* x, int n, int64_t stride, uint16_t* scale_out,
+                    uint16_t* zero_out, uint8_t* codes, int64_t code_stride) {
+  float mn = bf16_to_f32(x[0]);
+  float mx = mn;
+  for (int i = 1; i < n; ++i) {
+    float v = bf16_to_f32(x[i * stride]);
+    if (v < mn) mn = v;
+    if (v > mx) mx = v;
+  }
+  volatile float range = mx - mn;
+  volatile float third = range / 3.0f;
+  uint16_t sb = f32_to_bf16_rne(third);
+  float scale = bf16_to_f32(sb);
+  *scale_out = sb;
+  *zero_out = f32_to_bf16_rne(mn);  // mn is a bf16 value already: conversion is exact
+  for (int i = 0; i < n; ++i) {
+    uint8_t c = 0;
+    if (scale != 0.0f) {
+      volatile float d = bf16_to_f32(x[i * stride]) - mn;
+      volatile float q = d / scale;
+      float r = std::nearbyintf(q);  // default rounding mode: ties to even
+      if (r < 0.0f) r = 0.0f;
+      if (r > 3.0f) r = 3.0f;
+      c = static_cast<uint8_t>(r);
+    }
+    codes[i * code_stride] = c;
+  }
+}
+
+double dequant(uint16_t scale, uint16_t zero, uint8_t code) {
+  return static_cast<double>(bf16_to_f32(zero)) +
+         static_cast<double>(code) * static_cast<double>(bf16_to_f32(scale));
+}
+
+// ---- the cache ---------------------------------------------------------------------
+struct Head {  // one (batch row, kv head)
+  std::vector<uint16_t> fp_k, fp_v;      // [len(A)][D], rows in the order of list A
+  std::vector<uint8_t> k_codes, v_codes;  // [nq][D], one code per byte (unpacked)
+  std::vector<uint16_t> k_scale, k_zero;  // [nq/G][D]
+  std::vector<uint16_t> v_scale, v_zero;  // [nq][D/G]
+};
+
+struct Cache {
+  int B, Hq, Hkv, D, W, G;
+  int64_t n_seen = 0, n_events = 0;
+  std::vector<int64_t> A;  // ids of the tokens kept at original precision, age order
+  std::vector<int64_t> Q;  // ids of the quantised tokens, store order
+  std::vector<Head> heads;  // [B*Hkv]
+};
+
+// One window-overflow event (Algorithm 1, the else-branch): the entries at odd positions
+// of A[0:2W] leave the list, in age order; A becomes A[0:2W:2] ++ A[2W:3W].
+void overflow_event(Cache& c) {
+  const int W = c.W, D = c.D, G = c.G;
+  std::vector<int64_t> evict_pos, keep_pos;
+  for (int i = 0; i < 2 * W; ++i) (i % 2 ? evict_pos : keep_pos).push_back(i);
+  for (int i = 2 * W; i < 3 * W; ++i) keep_pos.push_back(i);
+  for (auto& h : c.heads) {
+    // gather the W leaving rows, in eviction order
+    std::vector<uint16_t> ek(static_cast<size_t>(W) * D), ev(static_cast<size_t>(W) * D);
+    for (int e = 0; e < W; ++e) {
+      std::memcpy(&ek[static_cast<size_t>(e) * D], &h.fp_k[evict_pos[e] * D], D * 2);
+      std::memcpy(&ev[static_cast<size_t>(e) * D], &h.fp_v[evict_pos[e] * D], D * 2);
+    }
+    const size_t nq0 = h.k_codes.size() / D;
+    h.k_codes.resize((nq0 + W) * D);
+    h.v_codes.resize((nq0 + W) * D);
+    h.k_scale.resize((nq0 + W) / G * D);
+    h.k_zero.resize((nq0 + W) / G * D);
+    h.v_scale.resize((nq0 + W) * (D / G));
+    h.v_zero.resize((nq0 + W) * (D / G));
+    // keys: group = G consecutive evicted tokens of one channel
+    for (int blk = 0; blk < W / G; ++blk)
+      for (int d = 0; d < D; ++d) {
+        size_t grp = (nq0 / G + blk) * D + d;
+        quantize_group(&ek[static_cast<size_t>(blk) * G * D + d], G, D, &h.k_scale[grp],
+                       &h.k_zero[grp], &h.k_codes[(nq0 + static_cast<size_t>(blk) * G) * D + d], D);
+      }
+    // values: group = G consecutive channels of one token
+    for (int e = 0; e < W; ++e)
+      for (int g = 0; g < D / G; ++g) {
+        size_t grp = (nq0 + e) * (D / G) + g;
+        quantize_group(&ev[static_cast<size_t>(e) * D + g * G], G, 1, &h.v_scale[grp],
+                       &h.v_zero[grp], &h.v_codes[(nq0 + e) * D + g * G], 1);
+      }
+    // shrink the full-precision rows to the kept positions
+    std::vector<uint16_t> nk(keep_pos.size() * D), nv(keep_pos.size() * D);
+    for (size_t i = 0; i < keep_pos.size(); ++i) {
+      std::memcpy(&nk[i * D], &h.fp_k[keep_pos[i] * D], D * 2);
+      std::memcpy(&nv[i * D], &h.fp_v[keep_pos[i] * D], D * 2);
+    }
+    h.fp_k.swap(nk);
+    h.fp_v.swap(nv);
+  }
+  std::vector<int64_t> nA;
+  for (auto p : evict_pos) c.Q.push_back(c.A[p]);
+  for (auto p : keep_pos) nA.push_back(c.A[p]);
+  c.A.swap(nA);
+  c.n_events++;
+}
+
+// Dense softmax attention of one query over n tokens, float64 (Eq. 2 with sm_scale).
+void attention_dense(const double* q, const double* K, const double* V, int64_t n, int D,
+                     double sm_scale, double* out) {
+  std::vector<double> s(n);
+  double m = -INFINITY;
+  for (int64_t t = 0; t < n; ++t) {
+    double acc = 0.0;
+    for (int d = 0; d < D; ++d) acc += q[d] * K[t * D + d];
+    s[t] = acc * sm_scale;
+    if (s[t] > m) m = s[t];
+  }
+  double l = 0.0;
+  for (int64_t t = 0; t < n; ++t) {
+    s[t] = std::exp(s[t] - m);
+    l += s[t];
+  }
+  for (int d = 0; d < D; ++d) out[d] = 0.0;
+  for (int64_t t = 0; t < n; ++t) {
+    double p = s[t] / l;
+    for (int d = 0; d < D; ++d) out[d] += p * V[t * D + d];
+  }
+}
+
+// All tokens of one head as float64 rows: first the full-precision list (order of A),
+// then the quantised store (order of Q), dequantised.
+void dense_rows(const Cache& c, const Head& h, std::vector<double>& K, std::vector<double>& V) {
+  const int D = c.D, G = c.G;
+  const size_t nf = c.A.size(), nq = c.Q.size();
+  K.resize((nf + nq) * D);
+  V.resize((nf + nq) * D);
+  for (size_t i = 0; i < nf * D; ++i) {
+    K[i] = bf16_to_f32(h.fp_k[i]);
+    V[i] = bf16_to_f32(h.fp_v[i]);
+  }
+  for (size_t t = 0; t < nq; ++t)
+    for (int d = 0; d < D; ++d) {
+      size_t kg = (t / G) * D + d;
+      size_t vg = t * (D / G) + d / G;
+      K[(nf + t) * D + d] = dequant(h.k_scale[kg], h.k_zero[kg], h.k_codes[t * D + d]);
+      V[(nf + t) * D + d] = dequant(h.v_scale[vg], h.v_zero[vg], h.v_codes[t * D + d]);
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+// ---- stand-alone pieces --------------------------------------------------------------
+// Algorithm 1 on token ids 0..N-1.  kept/quant must hold 3W and N entries; returns the
+// number of events and writes the two lengths.
+int64_t lqo_filter(int W, int64_t N, int64_t* kept, int64_t* n_kept, int64_t* quant, int64_t* n_quant) {
+  std::vector<int64_t> A, Q;
+  int64_t events = 0;
+  for (int64_t t = 0; t < N; ++t) {
+    if (static_cast<int64_t>(A.size()) < 3 * static_cast<int64_t>(W)) {
+      A.push_back(t);
+    } else {
+      std::vector<int64_t> nA;
+      for (int i = 0; i < 2 * W; i += 2) nA.push_back(A[i]);
+      for (int i = 1; i < 2 * W; i += 2) Q.push_back(A[i]);
+      for (int i = 2 * W; i < 3 * W; ++i) nA.push_back(A[i]);
+      nA.push_back(t);
+      A.swap(nA);
+      events++;
+    }
+  }
+  std::copy(A.begin(), A.end(), kept);
+  std::copy(Q.begin(), Q.end(), quant);
+  *n_kept = static_cast<int64_t>(A.size());
+  *n_quant = static_cast<int64_t>(Q.size());
+  return events;
+}
+
+void lqo_quantize_group(const uint16_t* x, int n, uint16_t* scale, uint16_t* zero, uint8_t* codes) {
+  quantize_group(x, n, 1, scale, zero, codes, 1);
+}
+
+double lqo_dequant(uint16_t scale, uint16_t zero, uint8_t code) { return dequant(scale, zero, code); }
+
+// 4 codes per byte: code of element 4j+i in bits [2i+1:2i] of byte j.  n % 4 == 0.
+void lqo_pack2(const uint8_t* codes, int64_t n, uint8_t* bytes) {
+  for (int64_t j = 0; j < n / 4; ++j) {
+    uint8_t b = 0;
+    for (int i = 0; i < 4; ++i) b |= static_cast<uint8_t>((codes[4 * j + i] & 3u) << (2 * i));
+    bytes[j] = b;
+  }
+}
+
+void lqo_unpack2(const uint8_t* bytes, int64_t n, uint8_t* codes) {
+  for (int64_t j = 0; j < n / 4; ++j)
+    for (int i = 0; i < 4; ++i) codes[4 * j + i] = (bytes[j] >> (2 * i)) & 3u;
+}
+
+uint16_t lqo_f32_to_bf16(float f) { return f32_to_bf16_rne(f); }
+float lqo_bf16_to_f32(uint16_t h) { return bf16_to_f32(h); }
+
+void lqo_attention_dense(const double* q, const double* K, const double* V, int64_t n, int D,
+                         double sm_scale, double* out) {
+  attention_dense(q, K, V, n, D, sm_scale, out);
+}
+
+// Partial softmax state of one segment: m = max score, l = sum exp(s - m),
+// o = sum exp(s - m) * v (not normalised).  n may be 0 (m = -inf, l = 0, o = 0).
+void lqo_attention_partial(const double* q, const double* K, const double* V, int64_t n, int D,
+                           double sm_scale, double* m_out, double* l_out, double* o) {
+  double m = -INFINITY;
+  std::vector<double> s(n);
+  for (int64_t t = 0; t < n; ++t) {
+    double acc = 0.0;
+    for (int d = 0; d < D; ++d) acc += q[d] * K[t * D + d];
+    s[t] = acc * sm_scale;
+    if (s[t] > m) m = s[t];
+  }
+  double l = 0.0;
+  for (int d = 0; d < D; ++d) o[d] = 0.0;
+  for (int64_t t = 0; t < n; ++t) {
+    double p = std::exp(s[t] - m);
+    l += p;
+    for (int d = 0; d < D; ++d) o[d] += p * V[t * D + d];
+  }
+  *m_out = m;
+  *l_out = l;
+}
+
+// Merge of S partial states: m = max m_s, l = sum l_s e^{m_s-m}, out = sum o_s e^{m_s-m} / l.
+void lqo_attention_merge(const double* m, const double* l, const double* o, int S, int D, double* out) {
+  double mm = -INFINITY;
+  for (int s = 0; s < S; ++s) mm = std::max(mm, m[s]);
+  double ll = 0.0;
+  for (int d = 0; d < D; ++d) out[d] = 0.0;
+  for (int s = 0; s < S; ++s) {
+    if (l[s] == 0.0) continue;
+    double w = std::exp(m[s] - mm);
+    ll += l[s] * w;
+    for (int d = 0; d < D; ++d) out[d] += o[s * D + d] * w;
+  }
+  for (int d = 0; d < D; ++d) out[d] /= ll;
+}
+
+// ---- the cache object ------------------------------------------------------------------
+void* lqo_create(int B, int Hq, int Hkv, int D, int W, int G) {
+  if (B < 1 || Hkv < 1 || Hq % Hkv || D < 1 || W < 1 || G < 1 || W % G || D % G || D % 4) return nullptr;
+  Cache* c = new Cache;
+  c->B = B; c->Hq = Hq; c->Hkv = Hkv; c->D = D; c->W = W; c->G = G;
+  c->heads.resize(static_cast<size_t>(B) * Hkv);
+  return c;
+}
+
+void lqo_destroy(void* p) { delete static_cast<Cache*>(p); }
+
+// k, v: [B][Hkv][n][D] bf16 bit patterns.  A prompt of n tokens is n single appends.
+void lqo_append(void* p, const uint16_t* k, const uint16_t* v, int n) {
+  Cache& c = *static_cast<Cache*>(p);
+  for (int t = 0; t < n; ++t) {
+    if (static_cast<int64_t>(c.A.size()) >= 3 * static_cast<int64_t>(c.W)) overflow_event(c);
+    for (int b = 0; b < c.B; ++b)
+      for (int h = 0; h < c.Hkv; ++h) {
+        Head& hd = c.heads[static_cast<size_t>(b) * c.Hkv + h];
+        const size_t off = ((static_cast<size_t>(b) * c.Hkv + h) * n + t) * c.D;
+        hd.fp_k.insert(hd.fp_k.end(), k + off, k + off + c.D);
+        hd.fp_v.insert(hd.fp_v.end(), v + off, v + off + c.D);
+      }
+    c.A.push_back(c.n_seen++);
+  }
+}
+
+int64_t lqo_n_seen(void* p) { return static_cast<Cache*>(p)->n_seen; }
+int64_t lqo_n_fp(void* p) { return static_cast<int64_t>(static_cast<Cache*>(p)->A.size()); }
+int64_t lqo_n_quant(void* p) { return static_cast<int64_t>(static_cast<Cache*>(p)->Q.size()); }
+int64_t lqo_n_events(void* p) { return static_cast<Cache*>(p)->n_events; }
+
+// Canonical image.  kept_ids ascending (list A is in age order, hence ascending);
+// quant_ids in store order; codes packed 4 per byte; scale/zero as bf16 bit patterns;
+// fp rows in kept_ids order.  Any pointer may be null to skip that array.
+void lqo_export(void* p, int32_t* kept_ids, int32_t* quant_ids, uint8_t* k_codes, uint8_t* v_codes,
+                uint16_t* k_scale, uint16_t* k_zero, uint16_t* v_scale, uint16_t* v_zero,
+                uint16_t* fp_k, uint16_t* fp_v) {
+  Cache& c = *static_cast<Cache*>(p);
+  const size_t nf = c.A.size(), nq = c.Q.size(), D = c.D, G = c.G;
+  if (kept_ids) for (size_t i = 0; i < nf; ++i) kept_ids[i] = static_cast<int32_t>(c.A[i]);
+  if (quant_ids) for (size_t i = 0; i < nq; ++i) quant_ids[i] = static_cast<int32_t>(c.Q[i]);
+  for (size_t hh = 0; hh < c.heads.size(); ++hh) {
+    const Head& h = c.heads[hh];
+    if (k_codes) lqo_pack2(h.k_codes.data(), nq * D, k_codes + hh * nq * D / 4);
+    if (v_codes) lqo_pack2(h.v_codes.data(), nq * D, v_codes + hh * nq * D / 4);
+    if (k_scale) std::copy(h.k_scale.begin(), h.k_scale.end(), k_scale + hh * (nq / G) * D);
+    if (k_zero) std::copy(h.k_zero.begin(), h.k_zero.end(), k_zero + hh * (nq / G) * D);
+    if (v_scale) std::copy(h.v_scale.begin(), h.v_scale.end(), v_scale + hh * nq * (D / G));
+    if (v_zero) std::copy(h.v_zero.begin(), h.v_zero.end(), v_zero + hh * nq * (D / G));
+    if (fp_k) std::copy(h.fp_k.begin(), h.fp_k.end(), fp_k + hh * nf * D);
+    if (fp_v) std::copy(h.fp_v.begin(), h.fp_v.end(), fp_v + hh * nf * D);
+  }
+}
+
+// Every token of head (b, kv) as float64 rows: the full-precision list then the
+// dequantised store.  K, V: [(n_fp + n_quant)][D].
+void lqo_dense_rows(void* p, int b, int kv, double* K, double* V) {
+  Cache& c = *static_cast<Cache*>(p);
+  std::vector<double> k, v;
+  dense_rows(c, c.heads[static_cast<size_t>(b) * c.Hkv + kv], k, v);
+  std::copy(k.begin(), k.end(), K);
+  std::copy(v.begin(), v.end(), V);
+}
+
+// Decode attention of one query token per (b, query head) over the whole mixed cache.
+// q: [B][Hq][D] bf16 bits; out: [B][Hq][D] float64.  Query head h reads KV head
+// h / (Hq/Hkv).  n_threads > 1 spreads (b, kv head) pairs over std::threads.
+void lqo_attention(void* p, const uint16_t* q, double sm_scale, double* out, int n_threads) {
+  Cache& c = *static_cast<Cache*>(p);
+  const int r = c.Hq / c.Hkv, D = c.D;
+  const int n_pairs = c.B * c.Hkv;
+  auto work = [&](int first, int step) {
+    std::vector<double> K, V, qd(D);
+    for (int pair = first; pair < n_pairs; pair += step) {
+      const int b = pair / c.Hkv, kv = pair % c.Hkv;
+      dense_rows(c, c.heads[pair], K, V);
+      const int64_t n = static_cast<int64_t>(K.size()) / D;
+      for (int j = 0; j < r; ++j) {
+        const size_t qo = (static_cast<size_t>(b) * c.Hq + kv * r + j) * D;
+        for (int d = 0; d < D; ++d) qd[d] = bf16_to_f32(q[qo + d]);
+        attention_dense(qd.data(), K.data(), V.data(), n, D, sm_scale, out + qo);
+      }
+    }
+  };
+  if (n_threads <= 1) {
+    work(0, 1);
+  } else {
+    std::vector<std::thread> th;
+    for (int i = 0; i < n_threads; ++i) th.emplace_back(work, i, n_threads);
+    for (auto& t : th) t.join();
+  }
+}
+
+unsigned lqo_hardware_threads() { return std::thread::hardware_concurrency(); }
+
+}  // extern "C"

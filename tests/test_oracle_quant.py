@@ -1,0 +1,151 @@
+"""Pins for the oracle's 2-bit quantiser and packer."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from helpers import bf16_bits_to_f64, f32_to_bf16_bits
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden", "quant_worked_example.txt")
+
+
+def _gold():
+    out = []
+    for line in open(GOLD):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        vals, sz, codes, bts = [s.split() for s in line.split("|")]
+        out.append(([float(v) for v in vals], float(sz[0]), float(sz[1]), [int(c) for c in codes],
+                    [int(b, 16) for b in bts]))
+    return out
+
+
+@pytest.mark.parametrize("vals,scale,zero,codes,packed", _gold())
+def test_worked_examples(vals, scale, zero, codes, packed):
+    x = f32_to_bf16_bits(np.array(vals, np.float32))
+    assert np.array_equal(bf16_bits_to_f64(x), np.array(vals))  # the fixture is bf16-exact
+    s, z, c = oracle.quantize_group(x)
+    assert oracle.bf16_to_f32(s) == scale and oracle.bf16_to_f32(z) == zero
+    assert c.tolist() == codes
+    assert oracle.pack2(c).tolist() == packed
+
+
+def test_pack_unpack_all_bytes():
+    allb = np.arange(256, dtype=np.uint8)
+    codes = oracle.unpack2(allb)
+    assert codes.max() == 3
+    assert np.array_equal(oracle.pack2(codes), allb)
+    # bit layout: element 4j+i in bits [2i+1:2i] of byte j
+    for i in range(4):
+        c = np.zeros(8, np.uint8)
+        c[4 + i] = 3
+        assert oracle.pack2(c).tolist() == [0, 3 << (2 * i)]
+
+
+@pytest.mark.parametrize("n", [32, 64])
+@pytest.mark.parametrize("spread", [1.0, 10.0, 1e-3, 300.0])
+def test_round_trip_bound_and_order(n, spread):
+    rng = np.random.default_rng(1234 + n)
+    for trial in range(200):
+        x = f32_to_bf16_bits((rng.standard_normal(n) * spread + rng.standard_normal() * spread).astype(np.float32))
+        s, z, c = oracle.quantize_group(x)
+        xv = bf16_bits_to_f64(x)
+        sv, zv = oracle.bf16_to_f32(s), oracle.bf16_to_f32(z)
+        assert zv == xv.min()
+        assert abs(sv - (xv.max() - xv.min()) / 3) <= 2.0 ** -8 * sv  # scale is (max-min)/3 to bf16 precision
+        xh = np.array([oracle.dequant(s, z, int(ci)) for ci in c])
+        assert np.all(np.abs(xv - xh) <= sv / 2 * (1 + 1e-6) + 3 * sv * 2.0 ** -8)
+        assert np.array_equal(xh, zv + c.astype(np.float64) * sv)
+        assert c[np.argmin(xv)] == 0 and c[np.argmax(xv)] == 3
+        order = np.argsort(xv, kind="stable")
+        assert np.all(np.diff(c[order].astype(int)) >= 0)  # codes are monotone in x
+
+
+def test_half_scale_bound_when_scale_is_exact():
+    # When (max-min)/3 is exactly a bf16 value the bound |x - x^| <= scale/2 holds with no slack.
+    rng = np.random.default_rng(7)
+    worst = 0.0
+    for trial in range(300):
+        s = 2.0 ** rng.integers(-6, 4)
+        a = float(rng.integers(-8, 8)) * s
+        x = a + rng.uniform(0, 3 * s, 32)
+        x[0], x[1] = a, a + 3 * s
+        xb = f32_to_bf16_bits(x.astype(np.float32))
+        xv = bf16_bits_to_f64(xb)
+        sb, zb, c = oracle.quantize_group(xb)
+        assert oracle.bf16_to_f32(sb) == s and oracle.bf16_to_f32(zb) == a
+        err = np.abs(xv - (a + c * s))
+        worst = max(worst, float(err.max() / s))
+        assert np.all(err <= s / 2)
+    assert worst > 0.4  # the bound is tight
+
+
+def test_lattice_groups_round_trip_exactly():
+    rng = np.random.default_rng(3)
+    for trial in range(100):
+        s = 2.0 ** rng.integers(-5, 5)
+        a = float(rng.integers(-16, 16)) * s
+        k = rng.integers(0, 4, 32)
+        k[:2] = [0, 3]
+        x = f32_to_bf16_bits((a + k * s).astype(np.float32))
+        sb, zb, c = oracle.quantize_group(x)
+        assert np.array_equal(c, k.astype(np.uint8))
+        assert oracle.bf16_to_f32(sb) == s and oracle.bf16_to_f32(zb) == a
+
+
+def test_constant_group():
+    x = f32_to_bf16_bits(np.full(64, 1.2345, np.float32))
+    s, z, c = oracle.quantize_group(x)
+    assert s == 0 and not c.any() and oracle.dequant(s, z, 0) == bf16_bits_to_f64(x)[0]
+
+
+def test_cache_grouping_matches_vectorised_numpy():
+    """Keys: groups run down G evicted tokens per channel; values: across G channels per token.
+    The groups are re-formed here with numpy reshapes from the literal Algorithm 1 eviction order."""
+    from helpers import alg1_python, bf16_bits_to_f32
+    B, Hq, Hkv, D, W, G = 2, 4, 2, 128, 32, 32
+    N = 3 * W + W + 1  # two events
+    rng = np.random.default_rng(11)
+    k = f32_to_bf16_bits(rng.standard_normal((B, Hkv, N, D)).astype(np.float32))
+    v = f32_to_bf16_bits(rng.standard_normal((B, Hkv, N, D)).astype(np.float32))
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G)
+    oc.append(k, v)
+    img = oc.export()
+    A, Q = alg1_python(W, N)
+    assert img["kept_ids"].tolist() == A and img["quant_ids"].tolist() == Q
+    assert np.array_equal(img["fp_k"], k[:, :, A, :]) and np.array_equal(img["fp_v"], v[:, :, A, :])
+
+    def quant(x, axis):  # x fp32, group along `axis`; fp32 arithmetic like the quantiser's reading
+        mn, mx = x.min(axis, keepdims=True), x.max(axis, keepdims=True)
+        sc = bf16_bits_to_f32(f32_to_bf16_bits(((mx - mn) / np.float32(3.0)).astype(np.float32)))
+        with np.errstate(divide="ignore", invalid="ignore"):
+            c = np.clip(np.rint((x - mn) / sc), 0, 3)
+        c = np.where(sc == 0, 0, c).astype(np.uint8)
+        return c, f32_to_bf16_bits(sc), f32_to_bf16_bits(mn)
+
+    kq = bf16_bits_to_f32(k[:, :, Q, :]).reshape(B, Hkv, len(Q) // G, G, D)
+    c, s, z = quant(kq, 3)
+    assert np.array_equal(oracle.unpack2(img["k_codes"]).reshape(kq.shape), c)
+    assert np.array_equal(img["k_scale"], s[:, :, :, 0, :]) and np.array_equal(img["k_zero"], z[:, :, :, 0, :])
+    vq = bf16_bits_to_f32(v[:, :, Q, :]).reshape(B, Hkv, len(Q), D // G, G)
+    c, s, z = quant(vq, 4)
+    assert np.array_equal(oracle.unpack2(img["v_codes"]).reshape(vq.shape), c)
+    assert np.array_equal(img["v_scale"], s[..., 0]) and np.array_equal(img["v_zero"], z[..., 0])
+
+
+def test_export_sizes_match_byte_formulas():
+    B, Hq, Hkv, D, W, G = 1, 8, 2, 128, 128, 32
+    rng = np.random.default_rng(5)
+    N = 1024
+    k = f32_to_bf16_bits(rng.standard_normal((B, Hkv, N, D)).astype(np.float32))
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G)
+    oc.append(k, k)
+    assert (oc.n_quant, oc.n_fp, oc.n_events) == (640, 384, 5)
+    oc.append(k[:, :, :1], k[:, :, :1])
+    assert (oc.n_quant, oc.n_fp, oc.n_events) == (768, 257, 6)
+    img = oc.export()
+    per_tok = sum(img[n].nbytes for n in ("k_codes", "v_codes", "k_scale", "k_zero", "v_scale", "v_zero"))
+    assert per_tok == B * Hkv * oc.n_quant * 96  # 96 B per quantised token per KV head at G = 32
+    assert img["fp_k"].nbytes + img["fp_v"].nbytes == B * Hkv * oc.n_fp * 512
