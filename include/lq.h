@@ -1,0 +1,174 @@
+/*
+ * logquant -- decode-time hot path of LogQuant (arXiv 2503.19950) for NVIDIA B200 (sm_100a).
+ *
+ * A mixed KV cache per (layer, batch row, KV head):
+ *   - a full-precision (bf16) store holding at most 3W tokens, maintained by the log-based
+ *     filter of the paper's Algorithm 1 (Sec. 2.5), and
+ *   - a 2-bit store that receives the W tokens the filter removes at every window overflow,
+ *     quantised with asymmetric min/max groups of G values: keys grouped per channel over G
+ *     consecutive removed tokens ("Key-per-channel strategy", Sec. 2.5), values grouped per
+ *     token over G consecutive channels, scale and zero stored as bf16.
+ * Decode attention (Eq. 2, with the 1/sqrt(d) of the appendix) runs directly on both stores,
+ * dequantising in registers; the two stores and the split-K partitions are visited in an
+ * arbitrary order and merged with an online-softmax (m, l) reduction, which Eq. 3
+ * (position-agnostic attention, Sec. 2.4) permits.
+ *
+ * Conventions for every call
+ *   - Pointers named k, v, q, out are DEVICE pointers unless the name ends in _host.  They are
+ *     borrowed: they must stay valid until `stream` has executed the call's work.
+ *   - Layout of k, v: [batch, kv_head, token, head_dim] contiguous bf16.  q, out:
+ *     [batch, q_head, head_dim].  Query head h reads KV head h / (n_q_heads / n_kv_heads).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Calls enqueue work and return without synchronising (lq_export and the *_host entry
+ *     points synchronise).  Argument and state errors are detected on the host and leave the
+ *     cache unchanged; every length is a function of the number of appended tokens, so the
+ *     host never has to read one back from the device.
+ *   - No call throws, aborts or traps.  One cache must not be used from two threads at once.
+ *   - There is no CPU implementation: without a CUDA device lq_cache_create fails, except for
+ *     the bookkeeping-only mode device == LQ_DEVICE_NONE in which the compute calls return
+ *     LQ_ERR_UNSUPPORTED.
+ */
+#ifndef LQ_H_
+#define LQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lq_cache lq_cache_t; /* opaque; owns every device byte it allocates */
+
+typedef enum {
+  LQ_OK = 0,
+  LQ_ERR_INVALID_ARG = 1, /* null pointer, index out of range, empty cache for attention        */
+  LQ_ERR_UNSUPPORTED = 2, /* configuration outside what the kernels implement                   */
+  LQ_ERR_OOM = 3,         /* device allocation failed                                           */
+  LQ_ERR_WINDOW_FULL = 4, /* lq_append would exceed 3W full-precision tokens (auto_compress=0)  */
+  LQ_ERR_NOT_FULL = 5,    /* lq_compress on a layer that holds fewer than 3W full-precision tokens */
+  LQ_ERR_CAPACITY = 6,    /* max_tokens would be exceeded                                       */
+  LQ_ERR_CUDA = 7         /* a CUDA runtime call or a kernel launch failed                      */
+} lq_status_t;
+
+#define LQ_DEVICE_NONE (-1)
+
+/* decode-attention kernel selection */
+#define LQ_KERNEL_AUTO 0   /* the tensor-core kernel                                             */
+#define LQ_KERNEL_SCALAR 1 /* plain fp32 FMA kernel (slow; kept as an independent cross-check)   */
+#define LQ_KERNEL_MMA 2    /* mma.sync tensor-core kernel with bulk-copy staging                 */
+
+typedef struct {
+  int32_t n_layers;      /* independent stacked layer caches, >= 1                               */
+  int32_t batch;         /* B: sequences; all share one length                                   */
+  int32_t n_q_heads;     /* Hq; Hq % Hkv == 0 and Hq / Hkv <= 8                                  */
+  int32_t n_kv_heads;    /* Hkv                                                                  */
+  int32_t head_dim;      /* D; only 128 is implemented                                           */
+  int32_t window;        /* W of Algorithm 1; W % G == 0, W <= 512                               */
+  int32_t group;         /* G: quantisation group size, 32 or 64                                 */
+  int32_t bits;          /* 2                                                                    */
+  int64_t max_tokens;    /* capacity per sequence (tokens ever appended)                         */
+  int32_t auto_compress; /* 1: lq_append runs the overflow step itself when the window is full   */
+  int32_t device;        /* CUDA device ordinal, or LQ_DEVICE_NONE for bookkeeping only          */
+  int32_t kernel;        /* LQ_KERNEL_*                                                          */
+  int32_t n_splits;      /* split-K partitions per (batch row, KV head); 0 = chosen by the library */
+} lq_config_t;
+
+typedef struct {
+  int64_t n_seen;   /* tokens appended so far                                                    */
+  int64_t n_fp;     /* tokens in the full-precision store (2W < n_fp <= 3W after the first event) */
+  int64_t n_quant;  /* tokens in the 2-bit store (a multiple of W)                               */
+  int64_t n_events; /* window overflows processed                                                */
+  int64_t bytes_device;        /* device bytes owned by the whole cache (all layers + workspace) */
+  int64_t bytes_decode_step;   /* algorithmic bytes one lq_decode_attn on this layer has to read:
+                                  B*Hkv*(n_quant*bytes_quant_per_token + n_fp*4*D); q/out excluded */
+  int64_t bytes_quant_per_token; /* per KV head: codes + amortised scale/zero (96 at G=32, 80 at G=64) */
+  int32_t n_splits;            /* split-K partitions the next lq_decode_attn would use           */
+  int32_t reserved;
+} lq_info_t;
+
+/*
+ * Canonical image of one layer (host buffers supplied by the caller; a null member is skipped).
+ * Sizes use n_fp, n_quant from lq_cache_info.  This is the format parity is judged on; the
+ * device-side layout is private.
+ *   kept_ids  [n_fp]    int32, ascending: ids (append order, from 0) of the full-precision tokens
+ *   quant_ids [n_quant] int32, in store order: event order, then age order inside an event
+ *   k_codes, v_codes [B][Hkv][n_quant][D/4] uint8: channel 4j+i of a token in bits [2i+1:2i] of byte j
+ *   k_scale, k_zero  [B][Hkv][n_quant/G][D] uint16 (bf16 bit patterns)
+ *   v_scale, v_zero  [B][Hkv][n_quant][D/G] uint16
+ *   fp_k, fp_v       [B][Hkv][n_fp][D] uint16, rows in kept_ids order
+ */
+typedef struct {
+  int32_t* kept_ids;
+  int32_t* quant_ids;
+  uint8_t* k_codes;
+  uint8_t* v_codes;
+  uint16_t* k_scale;
+  uint16_t* k_zero;
+  uint16_t* v_scale;
+  uint16_t* v_zero;
+  uint16_t* fp_k;
+  uint16_t* fp_v;
+} lq_image_t;
+
+/* Create a cache.  Validates the configuration (LQ_ERR_INVALID_ARG / LQ_ERR_UNSUPPORTED),
+ * selects cfg->device and allocates both stores and the split-K workspace with cudaMalloc
+ * (LQ_ERR_OOM).  *out is written only on success.  (Problem statement: window W of Sec. 2.5,
+ * group size G and INT2 of Sec. 3.1.) */
+lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out);
+
+/* Free the cache and its device memory.  NULL is a no-op.  The caller must have synchronised
+ * every stream that still has work of this cache in flight. */
+lq_status_t lq_destroy(lq_cache_t* cache);
+
+/* Append n_tokens new tokens (Algorithm 1, the "length(A) < 3W" branch) to one layer.
+ * k, v: device, bf16, [B, Hkv, n_tokens, D].  A prompt of n tokens is equivalent to n single
+ * appends.  auto_compress = 0: LQ_ERR_WINDOW_FULL if the tokens do not fit below 3W (nothing is
+ * appended).  auto_compress = 1: the call is split into fill-to-3W / overflow step / continue. */
+lq_status_t lq_append(lq_cache_t* cache, int32_t layer, const void* k, const void* v,
+                      int32_t n_tokens, void* stream);
+
+/* Window-overflow step (Algorithm 1, else-branch; Fig. 5): of the 3W full-precision tokens in
+ * age order A, the W tokens A[1], A[3], ..., A[2W-1] are 2-bit quantised (keys per channel over
+ * blocks of G of these tokens in age order, values per token over blocks of G channels; group
+ * min/max by warp-shuffle reductions), bit-packed and appended to the 2-bit store; A[0:2W:2] and
+ * A[2W:3W] stay.  layer = -1 processes every layer that is full (others are skipped);
+ * a single layer that is not full gives LQ_ERR_NOT_FULL. */
+lq_status_t lq_compress(lq_cache_t* cache, int32_t layer, void* stream);
+
+/* One-token decode attention over the whole mixed cache of one layer (Eq. 2; order of the two
+ * stores and of the split-K partitions is free by Eq. 3).  q: device bf16 [B, Hq, D];
+ * sm_scale <= 0 selects 1/sqrt(D); out: device [B, Hq, D], out_dtype 0 = fp32, 1 = bf16.
+ * Accumulation is fp32.  An empty cache gives LQ_ERR_INVALID_ARG. */
+lq_status_t lq_decode_attn(lq_cache_t* cache, int32_t layer, const void* q, float sm_scale,
+                           void* out, int32_t out_dtype, void* stream);
+
+/* One decode step of one layer with HOST buffers: copies k_host, v_host ([B,Hkv,1,D] bf16) and
+ * q_host ([B,Hq,D] bf16) to the device, appends (running the overflow step first when the window
+ * is full, whatever auto_compress says), runs decode attention and copies the fp32 result to
+ * out_host ([B,Hq,D]).  Synchronises `stream` before returning.  Pinned host memory is
+ * recommended. */
+lq_status_t lq_decode_step_host(lq_cache_t* cache, int32_t layer, const void* k_host,
+                                const void* v_host, const void* q_host, float sm_scale,
+                                float* out_host, void* stream);
+
+/* Introspection (not on the hot path). */
+lq_status_t lq_cache_info(const lq_cache_t* cache, int32_t layer, lq_info_t* info);
+
+/* Copy the canonical image of one layer into the caller's HOST buffers.  Synchronises the device. */
+lq_status_t lq_export(const lq_cache_t* cache, int32_t layer, lq_image_t* image_host);
+
+/* Host-side bookkeeping only (works in LQ_DEVICE_NONE mode): ids of the tokens the next
+ * lq_compress on `layer` would remove, in removal order (W entries; LQ_ERR_NOT_FULL if the
+ * layer holds fewer than 3W full-precision tokens). */
+lq_status_t lq_next_evicted_ids(const lq_cache_t* cache, int32_t layer, int32_t* ids_host);
+
+const char* lq_status_str(lq_status_t status);
+
+/* Sticky description of the last CUDA error seen by this cache ("" if none). */
+const char* lq_last_error(const lq_cache_t* cache);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LQ_H_ */

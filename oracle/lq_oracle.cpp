@@ -11,7 +11,7 @@
 //   * quantiser     : the paper only names "INT2", group size G and the "Key-per-channel
 //                     strategy" (Sec. 2.5 Implementation, Sec. 3.1 Settings).  The reading
 //                     taken here is asymmetric min/max quantisation:
-//                         zero  = min(group)                         (a bf16 value, exact)
+//                         zero  = min(group)                         (a bf16 value, exact; -0 -> +0)
 //                         scale = bf16_rne((max - min) / 3)          (fp32 IEEE ops)
 //                         code  = clamp(rint((x - zero) / scale), 0, 3), all 0 if scale == 0
 //                         x^    = zero + code * scale
@@ -69,6 +69,8 @@ void quantize_group(const uint16_t* x, int n, int64_t stride, uint16_t* scale_ou
     if (v < mn) mn = v;
     if (v > mx) mx = v;
   }
+  mn = mn + 0.0f;  // a zero-valued min or max is taken as +0 (the sign of zero is not information)
+  mx = mx + 0.0f;
   volatile float range = mx - mn;
   volatile float third = range / 3.0f;
   uint16_t sb = f32_to_bf16_rne(third);

@@ -1,0 +1,10 @@
+"""LogQuant decode hot path for B200 (sm_100a): thin ctypes binding over the C-ABI library.
+
+Every step of the path runs in the CUDA kernels of ``liblogquant.so``; this package only marshals
+arguments.  PyTorch is used by callers for device memory and streams.
+"""
+from .binding import (LQ_DEVICE_NONE, LQ_KERNEL_AUTO, LQ_KERNEL_MMA, LQ_KERNEL_SCALAR, LogQuantCache,
+                      LogQuantError, exported_symbols, load_library)
+
+__all__ = ["LogQuantCache", "LogQuantError", "load_library", "exported_symbols", "LQ_DEVICE_NONE",
+           "LQ_KERNEL_AUTO", "LQ_KERNEL_SCALAR", "LQ_KERNEL_MMA"]

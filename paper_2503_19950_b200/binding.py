@@ -1,0 +1,175 @@
+"""ctypes binding with the same names as include/lq.h (argument marshalling only)."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "liblogquant.so")
+
+LQ_DEVICE_NONE = -1
+LQ_KERNEL_AUTO, LQ_KERNEL_SCALAR, LQ_KERNEL_MMA = 0, 1, 2
+LQ_OK, LQ_ERR_INVALID_ARG, LQ_ERR_UNSUPPORTED, LQ_ERR_OOM, LQ_ERR_WINDOW_FULL, LQ_ERR_NOT_FULL, \
+    LQ_ERR_CAPACITY, LQ_ERR_CUDA = range(8)
+
+
+class lq_config_t(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("batch", C.c_int32), ("n_q_heads", C.c_int32),
+                ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("window", C.c_int32),
+                ("group", C.c_int32), ("bits", C.c_int32), ("max_tokens", C.c_int64),
+                ("auto_compress", C.c_int32), ("device", C.c_int32), ("kernel", C.c_int32),
+                ("n_splits", C.c_int32)]
+
+
+class lq_info_t(C.Structure):
+    _fields_ = [("n_seen", C.c_int64), ("n_fp", C.c_int64), ("n_quant", C.c_int64), ("n_events", C.c_int64),
+                ("bytes_device", C.c_int64), ("bytes_decode_step", C.c_int64),
+                ("bytes_quant_per_token", C.c_int64), ("n_splits", C.c_int32), ("reserved", C.c_int32)]
+
+
+class lq_image_t(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("kept_ids", "quant_ids", "k_codes", "v_codes", "k_scale", "k_zero",
+                                          "v_scale", "v_zero", "fp_k", "fp_v")]
+
+
+SYMBOLS = ["lq_cache_create", "lq_destroy", "lq_append", "lq_compress", "lq_decode_attn",
+           "lq_decode_step_host", "lq_cache_info", "lq_export", "lq_next_evicted_ids", "lq_status_str",
+           "lq_last_error"]
+
+_lib = None
+
+
+class LogQuantError(RuntimeError):
+    def __init__(self, status, msg):
+        super().__init__(msg)
+        self.status = status
+
+
+def load_library():
+    """Load liblogquant.so.  There is no fallback: a missing library is an error."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(f"{_LIB_PATH} is missing: run `python -m paper_2503_19950_b200.build` "
+                              "(there is no CPU or PyTorch fallback for the LogQuant kernels)")
+        L = C.CDLL(_LIB_PATH)
+        vp, i32 = C.c_void_p, C.c_int32
+        L.lq_cache_create.argtypes = [C.POINTER(lq_config_t), C.POINTER(vp)]
+        L.lq_destroy.argtypes = [vp]
+        L.lq_append.argtypes = [vp, i32, vp, vp, i32, vp]
+        L.lq_compress.argtypes = [vp, i32, vp]
+        L.lq_decode_attn.argtypes = [vp, i32, vp, C.c_float, vp, i32, vp]
+        L.lq_decode_step_host.argtypes = [vp, i32, vp, vp, vp, C.c_float, vp, vp]
+        L.lq_cache_info.argtypes = [vp, i32, C.POINTER(lq_info_t)]
+        L.lq_export.argtypes = [vp, i32, C.POINTER(lq_image_t)]
+        L.lq_next_evicted_ids.argtypes = [vp, i32, vp]
+        L.lq_status_str.argtypes = [i32]
+        L.lq_status_str.restype = C.c_char_p
+        L.lq_last_error.argtypes = [vp]
+        L.lq_last_error.restype = C.c_char_p
+        for s in SYMBOLS:
+            if getattr(L, s).restype is C.c_int:
+                getattr(L, s).restype = i32
+        _lib = L
+    return _lib
+
+
+def exported_symbols():
+    L = load_library()
+    return [s for s in SYMBOLS if hasattr(L, s)]
+
+
+def _ptr(x):
+    """Device/host address of a torch tensor, numpy array, int or None."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if isinstance(x, np.ndarray):
+        return x.ctypes.data
+    return x.data_ptr()  # torch tensor
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream if torch.cuda.is_available() else None
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+class LogQuantCache:
+    """Owner of one lq_cache_t.  Methods mirror the C entry points one to one."""
+
+    def __init__(self, n_layers, batch, n_q_heads, n_kv_heads, window, group, max_tokens, head_dim=128, bits=2,
+                 auto_compress=True, device=0, kernel=LQ_KERNEL_AUTO, n_splits=0):
+        self._lib = load_library()
+        self.cfg = lq_config_t(n_layers, batch, n_q_heads, n_kv_heads, head_dim, window, group, bits, max_tokens,
+                               int(auto_compress), device, kernel, n_splits)
+        self._h = C.c_void_p()
+        self._check(self._lib.lq_cache_create(C.byref(self.cfg), C.byref(self._h)), create=True)
+
+    def _check(self, status, create=False):
+        if status != LQ_OK:
+            msg = self._lib.lq_status_str(status).decode()
+            if not create and status == LQ_ERR_CUDA:
+                msg += ": " + self._lib.lq_last_error(self._h).decode()
+            raise LogQuantError(status, msg)
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.lq_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the five calls -----------------------------------------------------------------
+    def append(self, layer, k, v, n_tokens=None, stream=None):
+        if n_tokens is None:
+            n_tokens = k.shape[2]
+        self._check(self._lib.lq_append(self._h, layer, _ptr(k), _ptr(v), n_tokens,
+                                        None if self.cfg.device < 0 else _stream(stream)))
+
+    def compress(self, layer=-1, stream=None):
+        self._check(self._lib.lq_compress(self._h, layer, None if self.cfg.device < 0 else _stream(stream)))
+
+    def decode_attn(self, layer, q, out, sm_scale=0.0, stream=None):
+        import torch
+        out_dtype = 1 if out.dtype == torch.bfloat16 else 0
+        self._check(self._lib.lq_decode_attn(self._h, layer, _ptr(q), sm_scale, _ptr(out), out_dtype,
+                                             _stream(stream)))
+
+    def decode_step_host(self, layer, k_host, v_host, q_host, out_host, sm_scale=0.0, stream=None):
+        self._check(self._lib.lq_decode_step_host(self._h, layer, _ptr(k_host), _ptr(v_host), _ptr(q_host),
+                                                  sm_scale, _ptr(out_host), _stream(stream)))
+
+    # -- introspection --------------------------------------------------------------------
+    def info(self, layer=0) -> lq_info_t:
+        info = lq_info_t()
+        self._check(self._lib.lq_cache_info(self._h, layer, C.byref(info)))
+        return info
+
+    def next_evicted_ids(self, layer=0) -> np.ndarray:
+        ids = np.zeros(self.cfg.window, np.int32)
+        self._check(self._lib.lq_next_evicted_ids(self._h, layer, ids.ctypes.data))
+        return ids
+
+    def export(self, layer=0, ids_only=False) -> dict:
+        """Canonical image of one layer as numpy arrays (see include/lq.h)."""
+        c, inf = self.cfg, self.info(layer)
+        B, H, D, G, nf, nq = c.batch, c.n_kv_heads, c.head_dim, c.group, inf.n_fp, inf.n_quant
+        img = dict(kept_ids=np.zeros(nf, np.int32), quant_ids=np.zeros(nq, np.int32))
+        if not ids_only:
+            img.update(
+                k_codes=np.zeros((B, H, nq, D // 4), np.uint8), v_codes=np.zeros((B, H, nq, D // 4), np.uint8),
+                k_scale=np.zeros((B, H, nq // G, D), np.uint16), k_zero=np.zeros((B, H, nq // G, D), np.uint16),
+                v_scale=np.zeros((B, H, nq, D // G), np.uint16), v_zero=np.zeros((B, H, nq, D // G), np.uint16),
+                fp_k=np.zeros((B, H, nf, D), np.uint16), fp_v=np.zeros((B, H, nf, D), np.uint16))
+        st = lq_image_t(**{k: (v.ctypes.data if v.size else None) for k, v in img.items()})
+        self._check(self._lib.lq_export(self._h, layer, C.byref(st)))
+        return img

@@ -1,0 +1,456 @@
+// C-ABI of the library (include/lq.h) and the host-side state machine.
+//
+// The log-based filter of Algorithm 1 is data-independent: which tokens stay at full precision,
+// which W leave at each overflow and every store length are functions of the number of appended
+// tokens only.  The host therefore mirrors the filter exactly (token ids, age order, physical
+// slots) and hands the kernels plain slot lists and lengths; nothing is ever read back.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/lq.h"
+#include "lq_kernels.cuh"
+
+using namespace lq;
+
+namespace {
+
+struct LayerState {
+  int64_t n_seen = 0, n_events = 0, n_quant = 0;
+  int n_fp = 0;
+  std::vector<int32_t> age_slot;    // age order (oldest first) -> physical fp slot; size n_fp
+  std::vector<int32_t> slot_token;  // physical fp slot -> token id; size 3W
+  std::vector<int32_t> quant_ids;   // token ids in 2-bit store order
+};
+
+}  // namespace
+
+struct lq_cache {
+  lq_config_t cfg;
+  CacheView cv;
+  std::vector<LayerState> layers;
+  bool dry = false;
+  int sm_count = 148;
+  int max_splits = 1;
+  int64_t bytes_device = 0;
+  float* part_o = nullptr;
+  float* part_ml = nullptr;
+  int* status = nullptr;
+  // staging for the host-buffer entry point
+  void* stage_k = nullptr;
+  void* stage_v = nullptr;
+  void* stage_q = nullptr;
+  float* stage_out = nullptr;
+  std::string last_error;
+};
+
+namespace {
+
+lq_status_t cuda_fail(lq_cache* c, cudaError_t e, const char* what) {
+  char buf[256];
+  std::snprintf(buf, sizeof buf, "%s: %s", what, cudaGetErrorString(e));
+  if (c) c->last_error = buf;
+  return LQ_ERR_CUDA;
+}
+
+bool dev_alloc(lq_cache* c, void** p, int64_t bytes) {
+  if (cudaMalloc(p, static_cast<size_t>(bytes)) != cudaSuccess) {
+    cudaGetLastError();
+    *p = nullptr;
+    return false;
+  }
+  c->bytes_device += bytes;
+  return true;
+}
+
+void free_all(lq_cache* c) {
+  if (!c->dry) {
+    cudaFree(c->cv.quant);
+    cudaFree(c->cv.fp);
+    cudaFree(c->part_o);
+    cudaFree(c->part_ml);
+    cudaFree(c->status);
+    cudaFree(c->stage_k);
+    cudaFree(c->stage_v);
+    cudaFree(c->stage_q);
+    cudaFree(c->stage_out);
+  }
+}
+
+int ratio(const lq_cache* c) { return c->cfg.n_q_heads / c->cfg.n_kv_heads; }
+
+// slots and ids of the tokens the next overflow removes: A[1], A[3], ..., A[2W-1] in age order
+void next_evicted(const lq_cache* c, const LayerState& L, EvictList* ev, int32_t* ids) {
+  const int W = c->cfg.window;
+  for (int e = 0; e < W; ++e) {
+    const int slot = L.age_slot[2 * e + 1];
+    if (ev) ev->slot[e] = static_cast<uint16_t>(slot);
+    if (ids) ids[e] = L.slot_token[slot];
+  }
+}
+
+// host bookkeeping of one overflow event (device work is launched separately)
+void apply_event(const lq_cache* c, LayerState& L) {
+  const int W = c->cfg.window;
+  std::vector<int32_t> na;
+  na.reserve(3 * W);
+  for (int i = 0; i < 2 * W; i += 2) na.push_back(L.age_slot[i]);
+  for (int e = 0; e < W; ++e) {
+    const int hole = L.age_slot[2 * e + 1];
+    L.quant_ids.push_back(L.slot_token[hole]);
+    // the row of slot 2W+e (age position 2W+e) is moved into the hole
+    L.slot_token[hole] = L.slot_token[2 * W + e];
+    na.push_back(hole);
+  }
+  L.age_slot.swap(na);
+  L.n_fp = 2 * W;
+  L.n_quant += W;
+  L.n_events++;
+}
+
+lq_status_t run_events(lq_cache* c, const std::vector<int>& full_layers, cudaStream_t st) {
+  // group layers whose removal lists coincide into one launch
+  std::vector<char> done(full_layers.size(), 0);
+  for (size_t i = 0; i < full_layers.size(); ++i) {
+    if (done[i]) continue;
+    LayerState& Li = c->layers[full_layers[i]];
+    EvictList ev;
+    std::memset(&ev, 0, sizeof ev);
+    next_evicted(c, Li, &ev, nullptr);
+    LayerList ll;
+    ll.n = 0;
+    std::vector<int> members;
+    for (size_t k = i; k < full_layers.size() && ll.n < 128; ++k) {
+      if (done[k]) continue;
+      LayerState& Lk = c->layers[full_layers[k]];
+      if (Lk.n_quant != Li.n_quant) continue;
+      EvictList ek;
+      std::memset(&ek, 0, sizeof ek);
+      next_evicted(c, Lk, &ek, nullptr);
+      if (std::memcmp(&ek, &ev, sizeof ev) != 0) continue;
+      ll.layer[ll.n++] = static_cast<uint8_t>(full_layers[k]);
+      members.push_back(static_cast<int>(k));
+    }
+    if (!c->dry) {
+      cudaError_t e = launch_compress(c->cv, ll, ev, Li.n_quant / c->cfg.group, st);
+      if (e != cudaSuccess) return cuda_fail(c, e, "lq_compress_kernel");
+    }
+    for (int k : members) {
+      done[k] = 1;
+      apply_event(c, c->layers[full_layers[k]]);
+    }
+  }
+  return LQ_OK;
+}
+
+int choose_splits(const lq_cache* c, const LayerState& L) {
+  if (c->cfg.n_splits > 0) return std::min(c->cfg.n_splits, c->max_splits);
+  const int pairs = c->cfg.batch * c->cfg.n_kv_heads;
+  const int64_t T = L.n_fp + L.n_quant;
+  int64_t s = (4LL * c->sm_count + pairs - 1) / pairs;
+  s = std::min<int64_t>(s, (T + 127) / 128);
+  s = std::max<int64_t>(1, std::min<int64_t>(s, c->max_splits));
+  return static_cast<int>(s);
+}
+
+bool use_mma(const lq_cache* c) { return c->cfg.kernel == LQ_KERNEL_MMA; }  // TEMP until the MMA kernel lands
+
+}  // namespace
+
+extern "C" {
+
+const char* lq_status_str(lq_status_t s) {
+  switch (s) {
+    case LQ_OK: return "ok";
+    case LQ_ERR_INVALID_ARG: return "invalid argument";
+    case LQ_ERR_UNSUPPORTED: return "unsupported configuration";
+    case LQ_ERR_OOM: return "out of device memory";
+    case LQ_ERR_WINDOW_FULL: return "full-precision window is full";
+    case LQ_ERR_NOT_FULL: return "full-precision window is not full";
+    case LQ_ERR_CAPACITY: return "max_tokens exceeded";
+    case LQ_ERR_CUDA: return "CUDA error";
+  }
+  return "unknown status";
+}
+
+const char* lq_last_error(const lq_cache_t* c) { return c ? c->last_error.c_str() : ""; }
+
+lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
+  if (!cfg || !out) return LQ_ERR_INVALID_ARG;
+  if (cfg->n_layers < 1 || cfg->batch < 1 || cfg->n_q_heads < 1 || cfg->n_kv_heads < 1 ||
+      cfg->window < 1 || cfg->group < 1 || cfg->max_tokens < 1 || cfg->n_splits < 0)
+    return LQ_ERR_INVALID_ARG;
+  if (cfg->n_q_heads % cfg->n_kv_heads) return LQ_ERR_INVALID_ARG;
+  if (cfg->head_dim != kD || cfg->bits != 2) return LQ_ERR_UNSUPPORTED;
+  if (cfg->group != 32 && cfg->group != 64) return LQ_ERR_UNSUPPORTED;
+  if (cfg->window % cfg->group || cfg->window > kMaxW) return LQ_ERR_UNSUPPORTED;
+  if (cfg->n_q_heads / cfg->n_kv_heads > kMaxRatio || cfg->n_layers > 128) return LQ_ERR_UNSUPPORTED;
+  if (cfg->kernel < LQ_KERNEL_AUTO || cfg->kernel > LQ_KERNEL_MMA) return LQ_ERR_INVALID_ARG;
+
+  lq_cache* c = new (std::nothrow) lq_cache;
+  if (!c) return LQ_ERR_OOM;
+  c->cfg = *cfg;
+  c->dry = cfg->device == LQ_DEVICE_NONE;
+  const int W = cfg->window, G = cfg->group;
+  const int64_t pairs = static_cast<int64_t>(cfg->batch) * cfg->n_kv_heads;
+  CacheView& cv = c->cv;
+  std::memset(&cv, 0, sizeof cv);
+  cv.B = cfg->batch; cv.Hq = cfg->n_q_heads; cv.Hkv = cfg->n_kv_heads; cv.G = G; cv.W = W;
+  cv.quant_tiles_cap = (cfg->max_tokens + G - 1) / G;
+  cv.quant_head_stride = cv.quant_tiles_cap * quant_tile_bytes(G);
+  cv.quant_layer_stride = cv.quant_head_stride * pairs;
+  cv.fp_head_stride = static_cast<int64_t>(3 * W / kFpTileSlots) * kFpTileBytes;
+  cv.fp_layer_stride = cv.fp_head_stride * pairs;
+  c->layers.resize(cfg->n_layers);
+  for (auto& L : c->layers) L.slot_token.assign(3 * W, -1);
+
+  if (!c->dry) {
+    cudaError_t e = cudaSetDevice(cfg->device);
+    if (e != cudaSuccess) { delete c; cudaGetLastError(); return LQ_ERR_CUDA; }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, cfg->device) == cudaSuccess) c->sm_count = prop.multiProcessorCount;
+    c->max_splits = cfg->n_splits > 0
+                        ? cfg->n_splits
+                        : static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(512, (8LL * c->sm_count + pairs - 1) / pairs)));
+    const int r = ratio(c);
+    bool ok = dev_alloc(c, reinterpret_cast<void**>(&cv.quant), cv.quant_layer_stride * cfg->n_layers) &&
+              dev_alloc(c, reinterpret_cast<void**>(&cv.fp), cv.fp_layer_stride * cfg->n_layers) &&
+              dev_alloc(c, reinterpret_cast<void**>(&c->part_o), pairs * c->max_splits * r * kD * 4) &&
+              dev_alloc(c, reinterpret_cast<void**>(&c->part_ml), pairs * c->max_splits * r * 2 * 4) &&
+              dev_alloc(c, reinterpret_cast<void**>(&c->status), 256) &&
+              dev_alloc(c, &c->stage_k, pairs * kD * 2) && dev_alloc(c, &c->stage_v, pairs * kD * 2) &&
+              dev_alloc(c, &c->stage_q, static_cast<int64_t>(cfg->batch) * cfg->n_q_heads * kD * 2) &&
+              dev_alloc(c, reinterpret_cast<void**>(&c->stage_out),
+                        static_cast<int64_t>(cfg->batch) * cfg->n_q_heads * kD * 4);
+    if (ok) ok = cudaMemset(c->status, 0, 256) == cudaSuccess;
+    // the fp store must never hold non-finite garbage in unused slots of a partly filled tile
+    if (ok) ok = cudaMemset(cv.fp, 0, static_cast<size_t>(cv.fp_layer_stride) * cfg->n_layers) == cudaSuccess;
+    if (!ok) {
+      free_all(c);
+      delete c;
+      cudaGetLastError();
+      return LQ_ERR_OOM;
+    }
+  } else {
+    c->max_splits = std::max(1, cfg->n_splits);
+  }
+  *out = c;
+  return LQ_OK;
+}
+
+lq_status_t lq_destroy(lq_cache_t* c) {
+  if (!c) return LQ_OK;
+  free_all(c);
+  delete c;
+  return LQ_OK;
+}
+
+lq_status_t lq_append(lq_cache_t* c, int32_t layer, const void* k, const void* v, int32_t n, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || n < 0) return LQ_ERR_INVALID_ARG;
+  if (!c->dry && (!k || !v)) return LQ_ERR_INVALID_ARG;
+  if (!c->dry && ((reinterpret_cast<uintptr_t>(k) | reinterpret_cast<uintptr_t>(v)) & 15)) return LQ_ERR_INVALID_ARG;
+  LayerState& L = c->layers[layer];
+  const int W = c->cfg.window;
+  if (L.n_seen + n > c->cfg.max_tokens) return LQ_ERR_CAPACITY;
+  if (!c->cfg.auto_compress && L.n_fp + n > 3 * W) return LQ_ERR_WINDOW_FULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int done = 0;
+  while (done < n) {
+    if (L.n_fp == 3 * W) {
+      lq_status_t s = run_events(c, std::vector<int>{layer}, st);
+      if (s != LQ_OK) return s;
+    }
+    const int take = std::min(n - done, 3 * W - L.n_fp);
+    if (!c->dry) {
+      cudaError_t e = launch_append(c->cv, layer, k, v, n, done, take, L.n_fp, st);
+      if (e != cudaSuccess) return cuda_fail(c, e, "lq_append_kernel");
+    }
+    for (int t = 0; t < take; ++t) {
+      L.age_slot.push_back(L.n_fp + t);
+      L.slot_token[L.n_fp + t] = static_cast<int32_t>(L.n_seen + t);
+    }
+    L.n_fp += take;
+    L.n_seen += take;
+    done += take;
+  }
+  return LQ_OK;
+}
+
+lq_status_t lq_compress(lq_cache_t* c, int32_t layer, void* stream) {
+  if (!c || layer < -1 || layer >= c->cfg.n_layers) return LQ_ERR_INVALID_ARG;
+  const int W = c->cfg.window;
+  std::vector<int> full;
+  if (layer >= 0) {
+    if (c->layers[layer].n_fp != 3 * W) return LQ_ERR_NOT_FULL;
+    full.push_back(layer);
+  } else {
+    for (int i = 0; i < c->cfg.n_layers; ++i)
+      if (c->layers[i].n_fp == 3 * W) full.push_back(i);
+  }
+  if (full.empty()) return LQ_OK;
+  return run_events(c, full, static_cast<cudaStream_t>(stream));
+}
+
+lq_status_t lq_decode_attn(lq_cache_t* c, int32_t layer, const void* q, float sm_scale, void* out,
+                           int32_t out_dtype, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || (out_dtype != 0 && out_dtype != 1)) return LQ_ERR_INVALID_ARG;
+  if (c->dry) return LQ_ERR_UNSUPPORTED;
+  if (!q || !out) return LQ_ERR_INVALID_ARG;
+  LayerState& L = c->layers[layer];
+  if (L.n_fp + L.n_quant == 0) return LQ_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  DecodeArgs a;
+  a.cv = c->cv;
+  a.layer = layer;
+  a.n_fp = L.n_fp;
+  a.n_quant = L.n_quant;
+  if (!(sm_scale > 0.f)) sm_scale = 1.0f / std::sqrt(static_cast<float>(kD));
+  a.scale_log2 = sm_scale * 1.4426950408889634f;
+  a.q = q;
+  a.part_o = c->part_o;
+  a.part_ml = c->part_ml;
+  a.out = out;
+  a.out_bf16 = out_dtype;
+  a.status = c->status;
+  cudaError_t e;
+  if (use_mma(c)) {
+    a.S = c->cfg.n_splits > 0 ? std::min(c->cfg.n_splits, c->max_splits)
+                              : std::min(c->max_splits, decode_mma_max_splits(c->cv, L.n_fp, L.n_quant, c->sm_count));
+    e = launch_decode_mma(a, st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "lq_decode_mma_kernel");
+  } else {
+    a.S = choose_splits(c, L);
+    e = launch_decode_scalar(a, st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "lq_decode_scalar_kernel");
+  }
+  e = launch_merge(a, st);
+  if (e != cudaSuccess) return cuda_fail(c, e, "lq_merge_kernel");
+  return LQ_OK;
+}
+
+lq_status_t lq_decode_step_host(lq_cache_t* c, int32_t layer, const void* k_host, const void* v_host,
+                                const void* q_host, float sm_scale, float* out_host, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers) return LQ_ERR_INVALID_ARG;
+  if (c->dry) return LQ_ERR_UNSUPPORTED;
+  if (!k_host || !v_host || !q_host || !out_host) return LQ_ERR_INVALID_ARG;
+  LayerState& L = c->layers[layer];
+  if (L.n_seen + 1 > c->cfg.max_tokens) return LQ_ERR_CAPACITY;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t kvb = static_cast<size_t>(c->cfg.batch) * c->cfg.n_kv_heads * kD * 2;
+  const size_t qb = static_cast<size_t>(c->cfg.batch) * c->cfg.n_q_heads * kD * 2;
+  cudaError_t e;
+  if ((e = cudaMemcpyAsync(c->stage_k, k_host, kvb, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(c->stage_v, v_host, kvb, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(c->stage_q, q_host, qb, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+    return cuda_fail(c, e, "host-to-device copy");
+  if (L.n_fp == 3 * c->cfg.window) {
+    lq_status_t s = run_events(c, std::vector<int>{layer}, st);
+    if (s != LQ_OK) return s;
+  }
+  lq_status_t s = lq_append(c, layer, c->stage_k, c->stage_v, 1, stream);
+  if (s != LQ_OK) return s;
+  s = lq_decode_attn(c, layer, c->stage_q, sm_scale, c->stage_out, 0, stream);
+  if (s != LQ_OK) return s;
+  if ((e = cudaMemcpyAsync(out_host, c->stage_out, qb * 2, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+    return cuda_fail(c, e, "device-to-host copy");
+  if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(c, e, "cudaStreamSynchronize");
+  return LQ_OK;
+}
+
+lq_status_t lq_cache_info(const lq_cache_t* c, int32_t layer, lq_info_t* info) {
+  if (!c || !info || layer < 0 || layer >= c->cfg.n_layers) return LQ_ERR_INVALID_ARG;
+  const LayerState& L = c->layers[layer];
+  std::memset(info, 0, sizeof *info);
+  info->n_seen = L.n_seen;
+  info->n_fp = L.n_fp;
+  info->n_quant = L.n_quant;
+  info->n_events = L.n_events;
+  info->bytes_device = c->bytes_device;
+  info->bytes_quant_per_token = quant_tile_bytes(c->cfg.group) / c->cfg.group;
+  info->bytes_decode_step = static_cast<int64_t>(c->cfg.batch) * c->cfg.n_kv_heads *
+                            (L.n_quant * info->bytes_quant_per_token + static_cast<int64_t>(L.n_fp) * 4 * kD);
+  if (c->dry || L.n_fp + L.n_quant == 0)
+    info->n_splits = 0;
+  else if (use_mma(c))
+    info->n_splits = c->cfg.n_splits > 0 ? std::min(c->cfg.n_splits, c->max_splits)
+                                         : std::min(c->max_splits, decode_mma_max_splits(c->cv, L.n_fp, L.n_quant, c->sm_count));
+  else
+    info->n_splits = choose_splits(c, L);
+  return LQ_OK;
+}
+
+lq_status_t lq_next_evicted_ids(const lq_cache_t* c, int32_t layer, int32_t* ids) {
+  if (!c || !ids || layer < 0 || layer >= c->cfg.n_layers) return LQ_ERR_INVALID_ARG;
+  const LayerState& L = c->layers[layer];
+  if (L.n_fp != 3 * c->cfg.window) return LQ_ERR_NOT_FULL;
+  next_evicted(c, L, nullptr, ids);
+  return LQ_OK;
+}
+
+lq_status_t lq_export(const lq_cache_t* cc, int32_t layer, lq_image_t* img) {
+  lq_cache* c = const_cast<lq_cache*>(cc);
+  if (!c || !img || layer < 0 || layer >= c->cfg.n_layers) return LQ_ERR_INVALID_ARG;
+  const LayerState& L = c->layers[layer];
+  // kept ids ascending, with the slot each lives in
+  std::vector<std::pair<int32_t, int32_t>> kept;  // (token id, slot)
+  for (int i = 0; i < L.n_fp; ++i) kept.emplace_back(L.slot_token[L.age_slot[i]], L.age_slot[i]);
+  std::sort(kept.begin(), kept.end());
+  if (img->kept_ids) for (int i = 0; i < L.n_fp; ++i) img->kept_ids[i] = kept[i].first;
+  if (img->quant_ids) std::copy(L.quant_ids.begin(), L.quant_ids.end(), img->quant_ids);
+  const bool want_dev = img->k_codes || img->v_codes || img->k_scale || img->k_zero || img->v_scale ||
+                        img->v_zero || img->fp_k || img->fp_v;
+  if (!want_dev) return LQ_OK;
+  if (c->dry) return LQ_ERR_UNSUPPORTED;
+
+  const int64_t pairs = static_cast<int64_t>(c->cfg.batch) * c->cfg.n_kv_heads;
+  const int G = c->cfg.group;
+  const int64_t nq = L.n_quant, nf = L.n_fp;
+  const int64_t sz_codes = pairs * nq * (kD / 4);
+  const int64_t sz_kp = pairs * (nq / G) * kD * 2;
+  const int64_t sz_vp = pairs * nq * (kD / G) * 2;
+  const int64_t sz_fp = pairs * nf * kD * 2;
+  struct Buf { void* host; int64_t bytes; void* dev; };
+  Buf bufs[8] = {{img->k_codes, sz_codes, nullptr}, {img->v_codes, sz_codes, nullptr},
+                 {img->k_scale, sz_kp, nullptr},    {img->k_zero, sz_kp, nullptr},
+                 {img->v_scale, sz_vp, nullptr},    {img->v_zero, sz_vp, nullptr},
+                 {img->fp_k, sz_fp, nullptr},       {img->fp_v, sz_fp, nullptr}};
+  int* slots_dev = nullptr;
+  lq_status_t status = LQ_OK;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(c, e, "cudaDeviceSynchronize");
+  for (auto& b : bufs)
+    if (b.host && b.bytes > 0 && cudaMalloc(&b.dev, static_cast<size_t>(b.bytes)) != cudaSuccess) status = LQ_ERR_OOM;
+  if (status == LQ_OK && nf > 0) {
+    std::vector<int> slots(nf);
+    for (int i = 0; i < nf; ++i) slots[i] = kept[i].second;
+    if (cudaMalloc(&slots_dev, nf * sizeof(int)) != cudaSuccess) status = LQ_ERR_OOM;
+    else cudaMemcpy(slots_dev, slots.data(), nf * sizeof(int), cudaMemcpyHostToDevice);
+  }
+  if (status == LQ_OK) {
+    e = launch_export(c->cv, layer, static_cast<int>(nf), nq, slots_dev,
+                      static_cast<uint8_t*>(bufs[0].dev), static_cast<uint8_t*>(bufs[1].dev),
+                      static_cast<uint16_t*>(bufs[2].dev), static_cast<uint16_t*>(bufs[3].dev),
+                      static_cast<uint16_t*>(bufs[4].dev), static_cast<uint16_t*>(bufs[5].dev),
+                      static_cast<uint16_t*>(bufs[6].dev), static_cast<uint16_t*>(bufs[7].dev), nullptr);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) status = cuda_fail(c, e, "export kernels");
+  }
+  if (status == LQ_OK)
+    for (auto& b : bufs)
+      if (b.dev) {
+        e = cudaMemcpy(b.host, b.dev, static_cast<size_t>(b.bytes), cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) { status = cuda_fail(c, e, "export copy"); break; }
+      }
+  for (auto& b : bufs) cudaFree(b.dev);
+  cudaFree(slots_dev);
+  if (status == LQ_ERR_OOM) cudaGetLastError();
+  return status;
+}
+
+}  // extern "C"

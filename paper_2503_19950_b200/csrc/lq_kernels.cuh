@@ -1,0 +1,71 @@
+// Launchers of the CUDA kernels behind the C-ABI (host-callable; defined in the .cu files).
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+
+#include "lq_layout.cuh"
+
+namespace lq {
+
+// Geometry and base pointers shared by every kernel.
+struct CacheView {
+  int B, Hq, Hkv, G, W;
+  int64_t quant_tiles_cap;    // capacity in tiles per (layer, b, kv)
+  int64_t quant_head_stride;  // bytes between (b, kv) heads of the 2-bit store
+  int64_t quant_layer_stride;
+  int64_t fp_head_stride;     // bytes between (b, kv) heads of the fp store (3W/16 fp tiles)
+  int64_t fp_layer_stride;
+  uint8_t* quant;  // 2-bit store base
+  uint8_t* fp;     // full-precision store base
+};
+
+struct EvictList {
+  uint16_t slot[kMaxW];  // physical fp slots of the W removed tokens, in removal order
+};
+
+struct LayerList {
+  int n;
+  uint8_t layer[128];
+};
+
+// K1: write n_tokens new rows into fp slots [slot0, slot0 + n_tokens) of one layer.
+// k, v: [B, Hkv, n_src_tokens, D] bf16; tokens [src0, src0 + n_tokens) of them are written.
+cudaError_t launch_append(const CacheView& cv, int layer, const void* k, const void* v,
+                          int n_src_tokens, int src0, int n_tokens, int slot0, cudaStream_t st);
+
+// K2: overflow step for the listed layers (all of them in the same state): quantise + pack the W
+// rows of `ev` into quant tiles [tile0, tile0 + W/G), then move rows 2W+e into slot ev.slot[e].
+cudaError_t launch_compress(const CacheView& cv, const LayerList& layers, const EvictList& ev,
+                            int64_t tile0, cudaStream_t st);
+
+// Canonical export of one layer into device buffers (any pointer may be null).
+// slot_of_rank[i] = fp slot of the i-th kept id (ascending ids); device array of n_fp ints.
+cudaError_t launch_export(const CacheView& cv, int layer, int n_fp, int64_t n_quant,
+                          const int* slot_of_rank_dev, uint8_t* k_codes, uint8_t* v_codes,
+                          uint16_t* k_scale, uint16_t* k_zero, uint16_t* v_scale, uint16_t* v_zero,
+                          uint16_t* fp_k, uint16_t* fp_v, cudaStream_t st);
+
+// Split-K partial state: for partition s of head pair p = b*Hkv + kv and query head j of the
+// group (j < r): o[128] unnormalised, m (in log2 units), l.
+//   part_o : [(p*S + s)*r + j][128] float,  part_ml : [(p*S + s)*r + j][2] float
+struct DecodeArgs {
+  CacheView cv;
+  int layer;
+  int n_fp;
+  int64_t n_quant;
+  int S;  // partitions per (b, kv)
+  float scale_log2;  // sm_scale * log2(e)
+  const void* q;     // [B, Hq, D] bf16
+  float* part_o;
+  float* part_ml;
+  void* out;
+  int out_bf16;
+  int* status;  // device word; kernels OR error bits into it (bounded waits that gave up)
+};
+
+cudaError_t launch_decode_scalar(const DecodeArgs& a, cudaStream_t st);
+cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st);
+int decode_mma_max_splits(const CacheView& cv, int n_fp, int64_t n_quant, int sm_count);
+cudaError_t launch_merge(const DecodeArgs& a, cudaStream_t st);
+
+}  // namespace lq

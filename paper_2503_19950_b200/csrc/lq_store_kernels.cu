@@ -1,0 +1,293 @@
+// Kernels that write and read back the two stores: append (K1), window-overflow step (K2:
+// quantise + bit-pack + back-fill) and the canonical export.  Layout: lq_layout.cuh.
+#include <cuda_bf16.h>
+
+#include "lq_kernels.cuh"
+
+namespace lq {
+
+// ---------------------------------------------------------------------------------------
+// K1  append: Algorithm 1, branch length(A) < 3W -- the new rows go to the next free slots.
+// One thread per 16-byte chunk of a K or V row.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+lq_append_kernel(CacheView cv, int layer, const uint4* __restrict__ k, const uint4* __restrict__ v,
+                 int n_src, int src0, int n, int slot0) {
+  const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int64_t total = static_cast<int64_t>(cv.B) * cv.Hkv * n * 32;
+  if (idx >= total) return;
+  const int c = static_cast<int>(idx & 15);
+  const int which = static_cast<int>((idx >> 4) & 1);
+  const int64_t row = idx >> 5;
+  const int t = static_cast<int>(row % n);
+  const int64_t pair = row / n;
+  const uint4* src = (which ? v : k) + ((pair * n_src + src0 + t) * 16 + c);
+  uint8_t* base = cv.fp + layer * cv.fp_layer_stride + pair * cv.fp_head_stride;
+  const int64_t off = fp_chunk_off(slot0 + t, c) + (which ? kFpTileVOffset : 0);
+  *reinterpret_cast<uint4*>(base + off) = *src;
+}
+
+cudaError_t launch_append(const CacheView& cv, int layer, const void* k, const void* v, int n_src,
+                          int src0, int n, int slot0, cudaStream_t st) {
+  const int64_t total = static_cast<int64_t>(cv.B) * cv.Hkv * n * 32;
+  const int blocks = static_cast<int>((total + 255) / 256);
+  lq_append_kernel<<<blocks, 256, 0, st>>>(cv, layer, static_cast<const uint4*>(k),
+                                           static_cast<const uint4*>(v), n_src, src0, n, slot0);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// K2  window-overflow step (Algorithm 1, else-branch).
+//
+// One CTA per (key group tau of the event, (b, kv) head, layer).  It
+//   1. gathers the G removed rows of its group (K and V) into shared memory,
+//   2. back-fills the G holes with the rows of slots 2W + tau*G + e (the newest window), so the
+//      valid slots stay the dense prefix [0, 2W) -- legal because the order of the cache is free
+//      (Eq. 3) -- and only this CTA ever touches these 2G slots,
+//   3. quantises: keys per channel down the G tokens (one thread per channel), values per token
+//      across G channels (one warp per token, group min/max by __shfl_xor_sync),
+//   4. packs the codes into the fragment order of the tile and stores the tile.
+//
+// Quantiser arithmetic (IEEE binary32, one rounding per operation, ties to even):
+//   zero = min, scale = bf16(fdiv(fsub(max, min), 3)), code = clamp(rint(fdiv(fsub(x, min), scale)), 0, 3),
+//   all codes 0 when scale == 0.  A zero-valued min or max is taken as +0.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b) {
+  return __uint_as_float(static_cast<uint32_t>(b) << 16);
+}
+
+__device__ __forceinline__ uint32_t quant_code(float x, float mn, float scale) {
+  if (scale == 0.0f) return 0u;
+  float q = __fdiv_rn(__fsub_rn(x, mn), scale);
+  float r = rintf(q);
+  r = fminf(fmaxf(r, 0.0f), 3.0f);
+  return static_cast<uint32_t>(r);
+}
+
+__device__ __forceinline__ void group_params(float mn, float mx, uint16_t& scale_bits,
+                                             uint16_t& zero_bits, float& mn_c, float& scale) {
+  mn_c = __fadd_rn(mn, 0.0f);  // -0 -> +0
+  float mxc = __fadd_rn(mx, 0.0f);
+  float third = __fdiv_rn(__fsub_rn(mxc, mn_c), 3.0f);
+  __nv_bfloat16 sb = __float2bfloat16_rn(third);
+  scale_bits = __bfloat16_as_ushort(sb);
+  scale = __bfloat162float(sb);
+  zero_bits = __bfloat16_as_ushort(__float2bfloat16_rn(mn_c));  // exact: mn is a bf16 value
+}
+
+template <int G>
+__global__ void __launch_bounds__(256)
+lq_compress_kernel(CacheView cv, LayerList layers, EvictList ev, int64_t tile0) {
+  __shared__ __align__(16) uint16_t sK[G][kD];
+  __shared__ __align__(16) uint16_t sV[G][kD];
+  constexpr int NS = G / 16;
+  const int tau = blockIdx.x;
+  const int64_t pair = blockIdx.y;
+  const int layer = layers.layer[blockIdx.z];
+  const int tid = threadIdx.x;
+  uint8_t* fpbase = cv.fp + layer * cv.fp_layer_stride + pair * cv.fp_head_stride;
+  uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
+                  (tile0 + tau) * quant_tile_bytes(G);
+
+  // 1. gather the removed rows
+  for (int idx = tid; idx < G * 32; idx += 256) {
+    const int c = idx & 15, which = (idx >> 4) & 1, e = idx >> 5;
+    const int slot = ev.slot[tau * G + e];
+    const uint4 val = *reinterpret_cast<const uint4*>(fpbase + fp_chunk_off(slot, c) +
+                                                      (which ? kFpTileVOffset : 0));
+    *reinterpret_cast<uint4*>(which ? &sV[e][c * 8] : &sK[e][c * 8]) = val;
+  }
+  __syncthreads();
+
+  // 2. back-fill the holes from the newest window
+  for (int idx = tid; idx < G * 32; idx += 256) {
+    const int c = idx & 15, which = (idx >> 4) & 1, e = idx >> 5;
+    const int dst = ev.slot[tau * G + e];
+    const int src = 2 * cv.W + tau * G + e;
+    const int vo = which ? kFpTileVOffset : 0;
+    const uint4 val = *reinterpret_cast<const uint4*>(fpbase + fp_chunk_off(src, c) + vo);
+    *reinterpret_cast<uint4*>(fpbase + fp_chunk_off(dst, c) + vo) = val;
+  }
+
+  // 3. quantise
+  if (tid < kD) {
+    const int d = tid;
+    float mn = bf16_bits_to_float(sK[0][d]), mx = mn;
+#pragma unroll 4
+    for (int e = 1; e < G; ++e) {
+      const float x = bf16_bits_to_float(sK[e][d]);
+      mn = fminf(mn, x);
+      mx = fmaxf(mx, x);
+    }
+    uint16_t sb, zb;
+    float mnc, scale;
+    group_params(mn, mx, sb, zb, mnc, scale);
+    reinterpret_cast<uint16_t*>(tile + qt_kscale_off())[kparam_index(d)] = sb;
+    reinterpret_cast<uint16_t*>(tile + qt_kzero_off())[kparam_index(d)] = zb;
+#pragma unroll 4
+    for (int e = 0; e < G; ++e)
+      sK[e][d] = static_cast<uint16_t>(quant_code(bf16_bits_to_float(sK[e][d]), mnc, scale));
+  } else {
+    const int warp = (tid >> 5) - 4, lane = tid & 31;
+    constexpr int LPG = G / 4;  // lanes per value group
+    for (int e = warp; e < G; e += 4) {
+      const uint2 raw = *reinterpret_cast<const uint2*>(&sV[e][4 * lane]);
+      float x[4] = {bf16_bits_to_float(raw.x & 0xFFFFu), bf16_bits_to_float(raw.x >> 16),
+                    bf16_bits_to_float(raw.y & 0xFFFFu), bf16_bits_to_float(raw.y >> 16)};
+      float mn = fminf(fminf(x[0], x[1]), fminf(x[2], x[3]));
+      float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+#pragma unroll
+      for (int o = 1; o < LPG; o <<= 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, o));
+        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+      }
+      uint16_t sb, zb;
+      float mnc, scale;
+      group_params(mn, mx, sb, zb, mnc, scale);
+      if ((lane % LPG) == 0) {
+        const int g = lane / LPG;
+        reinterpret_cast<uint16_t*>(tile + qt_vscale_off(G))[vscale_index(e, g, G)] = sb;
+        reinterpret_cast<uint16_t*>(tile + qt_vzero_off(G))[vzero_index(e, g, G)] = zb;
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        sV[e][4 * lane + i] = static_cast<uint16_t>(quant_code(x[i], mnc, scale));
+    }
+  }
+  __syncthreads();
+
+  // 4. pack into fragment order
+  uint32_t* kw = reinterpret_cast<uint32_t*>(tile + qt_kcodes_off());
+  uint32_t* vw = reinterpret_cast<uint32_t*>(tile + qt_vcodes_off(G));
+  for (int idx = tid; idx < 2 * NS * 128; idx += 256) {
+    const int which = idx / (NS * 128);
+    const int wd = idx % (NS * 128);
+    const int u = wd >> 7, lane = (wd >> 2) & 31, sub = wd & 3;
+    const int hi = lane >> 2, j = lane & 3;
+    uint32_t word = 0;
+    if (which == 0) {
+      const int nt = sub >> 1, w = sub & 1;
+      const int t = 16 * u + 8 * nt + hi;
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+          word |= static_cast<uint32_t>(sK[t][16 * ks + 8 * w + 2 * j + h]) << (16 * h + 2 * ks);
+      kw[wd] = word;
+    } else {
+      const int dh = sub & 1, th = sub >> 1;
+#pragma unroll
+      for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+          word |= static_cast<uint32_t>(sV[16 * u + 8 * th + 2 * j + h][16 * mt + 8 * dh + hi])
+                  << (16 * h + 2 * mt);
+      vw[wd] = word;
+    }
+  }
+}
+
+cudaError_t launch_compress(const CacheView& cv, const LayerList& layers, const EvictList& ev,
+                            int64_t tile0, cudaStream_t st) {
+  dim3 grid(cv.W / cv.G, cv.B * cv.Hkv, layers.n);
+  if (cv.G == 32)
+    lq_compress_kernel<32><<<grid, 256, 0, st>>>(cv, layers, ev, tile0);
+  else if (cv.G == 64)
+    lq_compress_kernel<64><<<grid, 256, 0, st>>>(cv, layers, ev, tile0);
+  else
+    return cudaErrorInvalidValue;
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// Canonical export (introspection; not on the hot path).
+// ---------------------------------------------------------------------------------------
+__global__ void lq_export_codes_kernel(CacheView cv, int layer, int64_t n_quant, uint8_t* k_codes,
+                                       uint8_t* v_codes) {
+  // one thread per output byte: (pair, token, byte j) -> channels 4j..4j+3
+  const int64_t per_pair = n_quant * (kD / 4);
+  const int64_t total = static_cast<int64_t>(cv.B) * cv.Hkv * per_pair;
+  for (int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; idx < total;
+       idx += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int64_t pair = idx / per_pair;
+    const int64_t rem = idx % per_pair;
+    const int64_t tq = rem / (kD / 4);
+    const int jb = static_cast<int>(rem % (kD / 4));
+    const uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
+                          (tq / cv.G) * quant_tile_bytes(cv.G);
+    const uint32_t* kw = reinterpret_cast<const uint32_t*>(tile + qt_kcodes_off());
+    const uint32_t* vw = reinterpret_cast<const uint32_t*>(tile + qt_vcodes_off(cv.G));
+    const int t = static_cast<int>(tq % cv.G);
+    uint32_t kb = 0, vb = 0;
+    for (int i = 0; i < 4; ++i) {
+      int word, bit;
+      kcode_pos(t, 4 * jb + i, word, bit);
+      kb |= ((kw[word] >> bit) & 3u) << (2 * i);
+      vcode_pos(t, 4 * jb + i, word, bit);
+      vb |= ((vw[word] >> bit) & 3u) << (2 * i);
+    }
+    if (k_codes) k_codes[idx] = static_cast<uint8_t>(kb);
+    if (v_codes) v_codes[idx] = static_cast<uint8_t>(vb);
+  }
+}
+
+__global__ void lq_export_params_kernel(CacheView cv, int layer, int64_t n_quant, uint16_t* k_scale,
+                                        uint16_t* k_zero, uint16_t* v_scale, uint16_t* v_zero) {
+  const int G = cv.G, NG = kD / G;
+  const int64_t pairs = static_cast<int64_t>(cv.B) * cv.Hkv;
+  const int64_t nk = pairs * (n_quant / G) * kD;  // K entries
+  const int64_t nv = pairs * n_quant * NG;        // V entries
+  for (int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; idx < nk + nv;
+       idx += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    if (idx < nk) {
+      const int d = static_cast<int>(idx % kD);
+      const int64_t grp = (idx / kD) % (n_quant / G);
+      const int64_t pair = idx / kD / (n_quant / G);
+      const uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
+                            grp * quant_tile_bytes(G);
+      if (k_scale) k_scale[idx] = reinterpret_cast<const uint16_t*>(tile + qt_kscale_off())[kparam_index(d)];
+      if (k_zero) k_zero[idx] = reinterpret_cast<const uint16_t*>(tile + qt_kzero_off())[kparam_index(d)];
+    } else {
+      const int64_t i2 = idx - nk;
+      const int g = static_cast<int>(i2 % NG);
+      const int64_t tq = (i2 / NG) % n_quant;
+      const int64_t pair = i2 / NG / n_quant;
+      const uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
+                            (tq / G) * quant_tile_bytes(G);
+      const int t = static_cast<int>(tq % G);
+      if (v_scale) v_scale[i2] = reinterpret_cast<const uint16_t*>(tile + qt_vscale_off(G))[vscale_index(t, g, G)];
+      if (v_zero) v_zero[i2] = reinterpret_cast<const uint16_t*>(tile + qt_vzero_off(G))[vzero_index(t, g, G)];
+    }
+  }
+}
+
+__global__ void lq_export_fp_kernel(CacheView cv, int layer, int n_fp, const int* __restrict__ slot_of_rank,
+                                    uint4* fp_k, uint4* fp_v) {
+  const int64_t total = static_cast<int64_t>(cv.B) * cv.Hkv * n_fp * 16;
+  for (int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; idx < total;
+       idx += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int c = static_cast<int>(idx & 15);
+    const int rank = static_cast<int>((idx >> 4) % n_fp);
+    const int64_t pair = (idx >> 4) / n_fp;
+    const uint8_t* base = cv.fp + layer * cv.fp_layer_stride + pair * cv.fp_head_stride;
+    const int64_t off = fp_chunk_off(slot_of_rank[rank], c);
+    if (fp_k) fp_k[idx] = *reinterpret_cast<const uint4*>(base + off);
+    if (fp_v) fp_v[idx] = *reinterpret_cast<const uint4*>(base + off + kFpTileVOffset);
+  }
+}
+
+cudaError_t launch_export(const CacheView& cv, int layer, int n_fp, int64_t n_quant,
+                          const int* slot_of_rank_dev, uint8_t* k_codes, uint8_t* v_codes,
+                          uint16_t* k_scale, uint16_t* k_zero, uint16_t* v_scale, uint16_t* v_zero,
+                          uint16_t* fp_k, uint16_t* fp_v, cudaStream_t st) {
+  if (n_quant > 0 && (k_codes || v_codes))
+    lq_export_codes_kernel<<<1184, 256, 0, st>>>(cv, layer, n_quant, k_codes, v_codes);
+  if (n_quant > 0 && (k_scale || k_zero || v_scale || v_zero))
+    lq_export_params_kernel<<<1184, 256, 0, st>>>(cv, layer, n_quant, k_scale, k_zero, v_scale, v_zero);
+  if (n_fp > 0 && (fp_k || fp_v))
+    lq_export_fp_kernel<<<1184, 256, 0, st>>>(cv, layer, n_fp, slot_of_rank_dev,
+                                              reinterpret_cast<uint4*>(fp_k), reinterpret_cast<uint4*>(fp_v));
+  return cudaGetLastError();
+}
+
+}  // namespace lq

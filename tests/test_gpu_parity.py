@@ -1,0 +1,163 @@
+"""GPU parity: the CUDA library (through the C-ABI) against the CPU oracle on the same seeded inputs.
+Packed codes, scale/zero bits, full-precision rows and index sets must match bit for bit; attention
+outputs within max|delta| <= 2e-3*max|ref| + 1e-3."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_common import assert_images_equal, attn_tolerance, run_case
+from paper_2503_19950_b200 import (LQ_KERNEL_AUTO, LQ_KERNEL_MMA, LQ_KERNEL_SCALAR, LogQuantCache, LogQuantError,
+                                   binding, build, synth)
+
+pytestmark = pytest.mark.gpu
+
+KERNELS = [LQ_KERNEL_SCALAR]
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+
+
+def test_generator_is_bit_identical_on_cpu_and_gpu():
+    for shape, ax in [((2, 3, 50, 128), 2), ((4, 8, 128), None)]:
+        a = synth.tensor_f32(5, 17, shape, "cpu", ax, 11, 100)
+        b = synth.tensor_f32(5, 17, shape, "cuda", ax, 11, 100)
+        assert torch.equal(a, b.cpu())
+    k0, v0 = synth.keys_values(3, 2, 2, 40, 128, "cpu", 5, 64, synth.outlier_channels(3, 2, 128, 3))
+    k1, v1 = synth.keys_values(3, 2, 2, 40, 128, "cuda", 5, 64, synth.outlier_channels(3, 2, 128, 3))
+    assert torch.equal(k0, k1.cpu()) and torch.equal(v0, v1.cpu())
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_config1_tiny_decode(kernel):
+    # 1 layer, batch 1, 8 q heads / 2 KV heads, W=128, G=32: prefill 1024 (5 overflow events), 16 decode
+    # steps, the first of which triggers the sixth event.  Full parity at every step.
+    worst = run_case(B=1, Hq=8, Hkv=2, W=128, G=32, n_prefill=1024, n_steps=16, seed=1, kernel=kernel, n_outliers=4)
+    assert worst <= 1.0
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("B,Hq,Hkv,W,G,n_prefill,n_steps", [
+    (2, 8, 2, 32, 32, 0, 3),        # a cache of 1..3 tokens, nothing quantised
+    (1, 4, 4, 32, 32, 95, 4),       # crosses the first overflow (MHA, r = 1)
+    (2, 14, 2, 64, 64, 64 * 9 + 7, 3),   # GQA-7, G = 64, ragged fp tail
+    (1, 16, 2, 64, 32, 64 * 6 + 33, 2),  # r = 8
+    (3, 6, 2, 256, 64, 256 * 5 + 100, 2),  # W = 256, r = 3
+    (1, 2, 1, 512, 64, 512 * 4 + 1, 2),  # largest window
+])
+def test_shapes_and_edge_cases(kernel, B, Hq, Hkv, W, G, n_prefill, n_steps):
+    worst = run_case(B, Hq, Hkv, W, G, n_prefill, n_steps, seed=7, kernel=kernel)
+    assert worst <= 1.0
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_chunked_prefill_and_manual_compress_give_the_same_image(kernel):
+    # a prompt appended in ragged chunks, with the caller driving lq_compress, equals n single appends
+    worst = run_case(2, 8, 2, 64, 32, 64 * 7 + 19, 2, seed=9, kernel=kernel, prefill_chunk=37, auto_compress=False)
+    assert worst <= 1.0
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_spiky_attention_and_custom_scale(kernel):
+    # large queries make the softmax nearly one-hot: exercises the running-max rescale path
+    worst = run_case(1, 8, 2, 64, 32, 64 * 8 + 5, 3, seed=11, kernel=kernel, sm_scale=0.25, q_gain=3.0)
+    assert worst <= 1.0
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("n_splits", [1, 2, 7, 64])
+def test_any_split_count_gives_the_same_answer(kernel, n_splits):
+    worst = run_case(1, 8, 2, 64, 32, 64 * 12 + 3, 1, seed=13, kernel=kernel, n_splits=n_splits, check_image_every=0)
+    assert worst <= 1.0
+
+
+def test_bf16_output():
+    worst = run_case(2, 8, 2, 64, 32, 64 * 5 + 3, 2, seed=15, kernel=LQ_KERNEL_AUTO, out_dtype=torch.bfloat16,
+                     check_image_every=0)
+    assert worst <= 1.0
+
+
+def test_constant_and_degenerate_groups():
+    # constant keys/values (scale = 0), signed zeros and a wide-range group, bit-exact against the oracle
+    B, Hq, Hkv, W, G, D = 1, 4, 1, 32, 32, 128
+    N = 3 * W + 1
+    k, v = synth.keys_values(21, B, Hkv, N, D, "cuda")
+    k[:, :, :, 0] = 1.5          # constant channel -> scale 0
+    k[:, :, 1::2, 1] = -0.0      # signed zeros as the group minimum
+    k[:, :, 0::2, 1] = 0.0
+    k[:, :, :, 2] = k[:, :, :, 2] * 1000
+    v[:, :, 3, :] = -2.25        # constant token -> all value groups have scale 0
+    v[:, :, 5, :32] = 0.0
+    cache = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=N + 4)
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G)
+    cache.append(0, k, v)
+    oc.append(synth.bf16_bits(k), synth.bf16_bits(v))
+    assert oc.n_events == 1
+    assert_images_equal(cache.export(0), oc.export())
+    q = synth.queries(21, B, Hq, D, 0, "cuda")
+    out = torch.empty(B, Hq, D, device="cuda")
+    cache.decode_attn(0, q, out)
+    ref = oc.attention(synth.bf16_bits(q), 1 / np.sqrt(D))
+    assert np.abs(out.cpu().numpy() - ref).max() <= attn_tolerance(ref)
+
+
+def test_multi_layer_compress_all_and_independence():
+    B, Hq, Hkv, W, G, D, L = 2, 8, 2, 32, 32, 128, 3
+    cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=8 * W, auto_compress=False)
+    ocs = [oracle.OracleCache(B, Hq, Hkv, D, W, G) for _ in range(L)]
+    lens = [3 * W, 3 * W, 40]
+    for l in range(L):
+        k, v = synth.keys_values(30, B, Hkv, lens[l], D, "cuda", layer=l)
+        cache.append(l, k, v)
+        ocs[l].append(synth.bf16_bits(k), synth.bf16_bits(v))
+    cache.compress(-1)  # layers 0 and 1 overflow in one launch; layer 2 is skipped
+    for l in range(L):
+        k, v = synth.keys_values(31, B, Hkv, 1, D, "cuda", layer=l)
+        cache.append(l, k, v)
+        ocs[l].append(synth.bf16_bits(k), synth.bf16_bits(v))
+        assert_images_equal(cache.export(l), ocs[l].export())
+        q = synth.queries(30, B, Hq, D, 0, "cuda", layer=l)
+        out = torch.empty(B, Hq, D, device="cuda")
+        cache.decode_attn(l, q, out)
+        ref = ocs[l].attention(synth.bf16_bits(q), 1 / np.sqrt(D))
+        assert np.abs(out.cpu().numpy() - ref).max() <= attn_tolerance(ref)
+    assert [cache.info(l).n_events for l in range(L)] == [1, 1, 0]
+
+
+def test_decode_step_with_host_buffers():
+    B, Hq, Hkv, W, G, D = 2, 8, 2, 32, 32, 128
+    N = 3 * W  # the first host step has to run the overflow itself, even with auto_compress = 0
+    cache = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=N + 8, auto_compress=False)
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G)
+    k, v = synth.keys_values(40, B, Hkv, N, D, "cuda", token_total=N + 4)
+    cache.append(0, k, v)
+    oc.append(synth.bf16_bits(k), synth.bf16_bits(v))
+    for step in range(3):
+        k1, v1 = synth.keys_values(40, B, Hkv, 1, D, "cpu", token_start=N + step, token_total=N + 4)
+        q = synth.queries(40, B, Hq, D, step, "cpu")
+        k1, v1, q = k1.pin_memory(), v1.pin_memory(), q.pin_memory()
+        out = torch.empty(B, Hq, D, dtype=torch.float32).pin_memory()
+        cache.decode_step_host(0, k1, v1, q, out)
+        oc.append(synth.bf16_bits(k1), synth.bf16_bits(v1))
+        ref = oc.attention(synth.bf16_bits(q), 1 / np.sqrt(D))
+        assert np.abs(out.numpy() - ref).max() <= attn_tolerance(ref)
+    assert_images_equal(cache.export(0), oc.export())
+
+
+def test_argument_errors_on_device():
+    cache = LogQuantCache(1, 1, 4, 2, 32, 32, max_tokens=64)
+    q = torch.zeros(1, 4, 128, dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(1, 4, 128, device="cuda")
+    with pytest.raises(LogQuantError) as e:
+        cache.decode_attn(0, q, out)  # empty cache
+    assert e.value.status == binding.LQ_ERR_INVALID_ARG
+    with pytest.raises(LogQuantError) as e:
+        cache.decode_attn(3, q, out)
+    assert e.value.status == binding.LQ_ERR_INVALID_ARG
+    k = torch.zeros(1, 2, 65, 128, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(LogQuantError) as e:
+        cache.append(0, k, k)
+    assert e.value.status == binding.LQ_ERR_CAPACITY
+    assert cache.info(0).n_seen == 0

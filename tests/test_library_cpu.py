@@ -1,0 +1,129 @@
+"""CPU-only checks of the CUDA library: it loads, exports what include/lq.h declares, validates
+arguments, and its host-side mirror of Algorithm 1 agrees with the oracle (bookkeeping-only mode)."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from helpers import alg1_python
+from paper_2503_19950_b200 import LQ_DEVICE_NONE, LogQuantCache, LogQuantError, binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "lq.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = sorted(set(re.findall(r"\b(lq_[a-z_]+)\s*\(", header)))
+    assert "lq_decode_attn" in declared and "lq_compress" in declared and len(declared) >= 9
+    lib = binding.load_library()
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert sorted(binding.SYMBOLS) == declared
+
+
+def test_status_strings():
+    lib = binding.load_library()
+    assert lib.lq_status_str(0) == b"ok"
+    assert len({lib.lq_status_str(i) for i in range(8)}) == 8
+
+
+def _dry(W=4, G=4, **kw):
+    args = dict(n_layers=1, batch=1, n_q_heads=4, n_kv_heads=2, window=W, group=G, max_tokens=4096,
+                device=LQ_DEVICE_NONE)
+    args.update(kw)
+    return LogQuantCache(**args)
+
+
+@pytest.mark.parametrize("bad", [dict(group=16), dict(group=48, window=96), dict(window=100), dict(head_dim=64),
+                                 dict(bits=4), dict(n_q_heads=18, n_kv_heads=2), dict(window=1024)])
+def test_unsupported_configurations(bad):
+    with pytest.raises(LogQuantError) as e:
+        _dry(W=bad.pop("window", 128), G=bad.pop("group", 32), **bad)
+    assert e.value.status == binding.LQ_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("bad", [dict(n_q_heads=5, n_kv_heads=2), dict(batch=0), dict(max_tokens=0), dict(n_layers=0)])
+def test_invalid_configurations(bad):
+    with pytest.raises(LogQuantError) as e:
+        _dry(W=128, G=32, **bad)
+    assert e.value.status == binding.LQ_ERR_INVALID_ARG
+
+
+def test_no_gpu_means_no_compute():
+    # without a CUDA device there is no fallback: creation on device 0 fails here, and the
+    # bookkeeping-only mode refuses the compute calls
+    import torch
+    if not torch.cuda.is_available():
+        with pytest.raises(LogQuantError):
+            LogQuantCache(1, 1, 4, 2, 128, 32, 1024, device=0)
+    c = _dry(W=128, G=32)
+    c.append(0, None, None, n_tokens=10)
+    with pytest.raises(LogQuantError) as e:
+        c._check(c._lib.lq_decode_attn(c._h, 0, None, 0.0, None, 0, None))
+    assert e.value.status == binding.LQ_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("W,G", [(32, 32), (64, 32), (128, 64), (256, 64)])
+def test_host_mirror_of_algorithm1_matches_oracle(W, G):
+    c = _dry(W=W, G=G, max_tokens=40 * W)
+    n = 0
+    rng = np.random.default_rng(W)
+    while n < 30 * W:
+        step = int(rng.integers(1, 2 * W))
+        c.append(0, None, None, n_tokens=step)
+        n += step
+        kept, quant, ev = oracle.filter_ids(W, n)
+        img = c.export(0, ids_only=True)
+        inf = c.info(0)
+        assert (inf.n_seen, inf.n_fp, inf.n_quant, inf.n_events) == (n, len(kept), len(quant), ev)
+        assert img["kept_ids"].tolist() == kept.tolist()
+        assert img["quant_ids"].tolist() == quant.tolist()
+    A, Q = alg1_python(W, n)
+    assert img["kept_ids"].tolist() == A and img["quant_ids"].tolist() == Q
+
+
+def test_manual_compress_state_rules():
+    W, G = 32, 32
+    c = _dry(W=W, G=G, auto_compress=False, n_layers=3)
+    with pytest.raises(LogQuantError) as e:
+        c.compress(0)
+    assert e.value.status == binding.LQ_ERR_NOT_FULL
+    c.append(0, None, None, n_tokens=3 * W)
+    with pytest.raises(LogQuantError) as e:
+        c.append(0, None, None, n_tokens=1)
+    assert e.value.status == binding.LQ_ERR_WINDOW_FULL
+    assert c.info(0).n_seen == 3 * W  # the failed call changed nothing
+    ids = c.next_evicted_ids(0)
+    assert ids.tolist() == list(range(1, 2 * W, 2))
+    c.append(1, None, None, n_tokens=5)
+    c.compress(-1)  # layer 0 is full, layers 1 and 2 are skipped
+    assert (c.info(0).n_fp, c.info(0).n_quant, c.info(0).n_events) == (2 * W, W, 1)
+    assert (c.info(1).n_fp, c.info(1).n_events, c.info(2).n_seen) == (5, 0, 0)
+    c.append(0, None, None, n_tokens=W)
+    ids2 = c.next_evicted_ids(0)
+    A, _ = alg1_python(W, 4 * W)  # state right before the second event
+    assert ids2.tolist() == A[1:2 * W:2]
+    with pytest.raises(LogQuantError) as e:
+        c.append(0, None, None, n_tokens=10 ** 6)
+    assert e.value.status == binding.LQ_ERR_CAPACITY
+
+
+def test_info_byte_accounting():
+    c = _dry(W=128, G=32, batch=8, n_q_heads=32, n_kv_heads=8, max_tokens=9000)
+    c.append(0, None, None, n_tokens=8193)
+    inf = c.info(0)
+    assert (inf.n_quant, inf.n_fp) == (7936, 257)
+    assert inf.bytes_quant_per_token == 96
+    assert inf.bytes_decode_step == 64 * (7936 * 96 + 257 * 512)  # 57.18 MB
+    c2 = _dry(W=256, G=64, batch=4, n_q_heads=28, n_kv_heads=4, max_tokens=33000)
+    c2.append(0, None, None, n_tokens=32769)
+    inf = c2.info(0)
+    assert (inf.n_quant, inf.n_fp, inf.bytes_quant_per_token) == (32256, 513, 80)

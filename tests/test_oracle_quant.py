@@ -149,3 +149,16 @@ def test_export_sizes_match_byte_formulas():
     per_tok = sum(img[n].nbytes for n in ("k_codes", "v_codes", "k_scale", "k_zero", "v_scale", "v_zero"))
     assert per_tok == B * Hkv * oc.n_quant * 96  # 96 B per quantised token per KV head at G = 32
     assert img["fp_k"].nbytes + img["fp_v"].nbytes == B * Hkv * oc.n_fp * 512
+
+
+def test_signed_zero_is_canonical():
+    # min (or max) equal to zero is stored as +0 whatever the sign bit of the inputs
+    neg0, pos0, one = 0x8000, 0x0000, 0x3F80
+    for grp in ([neg0, pos0, one, one], [pos0, neg0, one, one], [neg0, neg0, one, one]):
+        s, z, c = oracle.quantize_group(np.array(grp, np.uint16))
+        assert z == 0x0000 and c.tolist() == [0, 0, 3, 3]
+    s, z, c = oracle.quantize_group(np.array([neg0, pos0, neg0, neg0], np.uint16))
+    assert (s, z) == (0, 0) and not c.any()
+    minus1 = 0xBF80
+    s, z, c = oracle.quantize_group(np.array([minus1, neg0, minus1, pos0], np.uint16))
+    assert z == minus1 and c.tolist() == [0, 3, 0, 3]
