@@ -1,0 +1,364 @@
+#!/usr/bin/env python
+"""Benchmark of the LogQuant decode hot path on B200.
+
+One "step" = one decode step of a Llama-3-8B-shaped stack: for each of the L layer caches,
+append the new token's K/V (running the window-overflow step when the bf16 window is full) and run
+decode attention over the whole mixed cache.  Metric: KV tokens/s = B * (n_quant + n_fp) * L / t_step
+summed over all ranks (independent replicas, no collective on the data path).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+Prints ONE JSON line.  `--impl reference` times the CPU oracle (oracle/, as it stands) on the host
+cores on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2503_19950_b200 import synth  # noqa: E402
+
+WORKLOADS = {
+    # BASELINE config 2: Llama-3-8B layer shape, batch 8, context 8192, W=128, G=32, 32 stacked layers
+    "llama3-8b-8k": dict(L=32, B=8, Hq=32, Hkv=8, W=128, G=32, ctx=8192, n_outliers=3, seed=2),
+    # config 4: long-context GQA-7
+    "gqa7-32k": dict(L=28, B=4, Hq=28, Hkv=4, W=256, G=64, ctx=32768, n_outliers=0, seed=4, planted=True),
+    # config 3: batch sweep at context 4096
+    "llama3-8b-4k-b16": dict(L=32, B=16, Hq=32, Hkv=8, W=128, G=32, ctx=4096, n_outliers=3, seed=3),
+    "llama3-8b-4k-b32": dict(L=16, B=32, Hq=32, Hkv=8, W=128, G=32, ctx=4096, n_outliers=3, seed=3),
+    "llama3-8b-4k-b64": dict(L=8, B=64, Hq=32, Hkv=8, W=128, G=32, ctx=4096, n_outliers=3, seed=3),
+    # config 5: 128k MHA (layers reduced to what is needed to exceed L2 several times)
+    "mha-128k": dict(L=8, B=1, Hq=32, Hkv=32, W=256, G=32, ctx=131072, n_outliers=3, seed=5),
+    # config 1 (parity-sized; latency-bound)
+    "tiny": dict(L=1, B=1, Hq=8, Hkv=2, W=128, G=32, ctx=1024, n_outliers=4, seed=1),
+}
+D = 128
+Q_ROTATE = 16  # distinct query/new-token sets cycled through the steps
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU during the timed region (NVML)."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4)}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def make_step_inputs(wl, device, n_sets):
+    """Per layer: n_sets rotating (k_new, v_new, q) triples, resident on `device`."""
+    L, B, Hq, Hkv = wl["L"], wl["B"], wl["Hq"], wl["Hkv"]
+    ks, vs, qs = [], [], []
+    for l in range(L):
+        k, v = synth.keys_values(wl["seed"] + 100, B, Hkv, n_sets, D, device, layer=l,
+                                 outliers=wl.get("_outliers"))
+        ks.append([k[:, :, i:i + 1].contiguous() for i in range(n_sets)])
+        vs.append([v[:, :, i:i + 1].contiguous() for i in range(n_sets)])
+        qs.append([synth.queries(wl["seed"], B, Hq, D, i, device, layer=l) for i in range(n_sets)])
+    return ks, vs, qs
+
+
+def prefill(cache, wl, device, layers=None, chunk=1024, sink=None):
+    """Append ctx tokens to every layer, generated chunk by chunk on `device`.
+    sink(layer, k, v) additionally receives each chunk (used to feed the CPU oracle)."""
+    L, B, Hkv, ctx = wl["L"], wl["B"], wl["Hkv"], wl["ctx"]
+    u = synth.unit_vectors(wl["seed"], Hkv, D) if wl.get("planted") else None
+    for l in (range(L) if layers is None else layers):
+        for t0 in range(0, ctx, chunk):
+            n = min(chunk, ctx - t0)
+            k, v = synth.keys_values(wl["seed"], B, Hkv, n, D, device, token_start=t0, token_total=ctx,
+                                     outliers=wl.get("_outliers"), layer=l)
+            if u is not None:
+                k = synth.plant_spikes(k, u, 16.0, t0, ctx)
+            if cache is not None:
+                cache.append(l, k, v)
+            if sink is not None:
+                sink(l, k, v)
+
+
+def run_ours(args, wl, rank, world, device):
+    from paper_2503_19950_b200 import LogQuantCache, build
+    build.build()
+    L, B, Hq, Hkv, W, G, ctx = (wl[k] for k in ("L", "B", "Hq", "Hkv", "W", "G", "ctx"))
+    steps, warmup = args.steps, args.warmup
+    total_steps = 2 * (steps + warmup) + steps + warmup + 8  # device-timed, profiled and host-buffer passes
+    cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=ctx + total_steps + 8, device=device.index or 0)
+    prefill(cache, wl, device)
+    ks, vs, qs = make_step_inputs(wl, device, Q_ROTATE)
+    outs = [torch.empty(B, Hq, D, device=device) for _ in range(L)]
+    torch.cuda.synchronize()
+
+    def one_step(i):
+        s = i % Q_ROTATE
+        for l in range(L):
+            cache.append(l, ks[l][s], vs[l][s])
+            cache.decode_attn(l, qs[l][s], outs[l])
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    def timed(n, fn, start_idx):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        kv_tokens = 0
+        barrier()
+        ev0.record()
+        for i in range(n):
+            fn(start_idx + i)
+            inf = cache.info_fast()
+            kv_tokens += B * (inf[0] + inf[1]) * L
+        ev1.record()
+        barrier()
+        return ev0.elapsed_time(ev1), kv_tokens
+
+    step_idx = 0
+    for i in range(warmup):
+        one_step(step_idx)
+        step_idx += 1
+    launches0 = cache.info(0).n_kernel_launches
+    with ClockSampler(device.index or 0) as clk:
+        ms, kv_tokens = timed(steps, one_step, step_idx)
+    step_idx += steps
+    launches = cache.info(0).n_kernel_launches - launches0
+    bytes_step_last = sum(cache.info(l).bytes_decode_step for l in range(L))
+
+    # ---- kernel-only timing of the split-K attention kernel (roofline) ----
+    cache.profile_enable(True)
+    byte_sum = 0
+    for i in range(min(steps, 8192 // L)):
+        s = (step_idx + i) % Q_ROTATE
+        for l in range(L):
+            cache.append(l, ks[l][s], vs[l][s])
+            byte_sum += cache.info(l).bytes_decode_step
+            cache.decode_attn(l, qs[l][s], outs[l])
+    k_ms, k_n = cache.profile_read()
+    cache.profile_enable(False)
+    step_idx += min(steps, 8192 // L)
+
+    # ---- end to end through the C-ABI with host buffers (pinned), copies inside the timed region ----
+    hk = [[ks[l][s].cpu().pin_memory() for s in range(Q_ROTATE)] for l in range(L)]
+    hv = [[vs[l][s].cpu().pin_memory() for s in range(Q_ROTATE)] for l in range(L)]
+    hq = [[qs[l][s].cpu().pin_memory() for s in range(Q_ROTATE)] for l in range(L)]
+    hout = [torch.empty(B, Hq, D, dtype=torch.float32).pin_memory() for _ in range(L)]
+
+    def host_step(i):
+        s = i % Q_ROTATE
+        for l in range(L):
+            cache.decode_step_host(l, hk[l][s], hv[l][s], hq[l][s], hout[l], sync=False)
+        torch.cuda.current_stream().synchronize()  # the step's result is on the host
+
+    e2e_steps = max(3, min(steps, 32))
+    for i in range(3):
+        host_step(step_idx)
+        step_idx += 1
+    t0 = time.perf_counter()
+    barrier()
+    t0 = time.perf_counter()
+    kv_e2e = 0
+    for i in range(e2e_steps):
+        host_step(step_idx + i)
+        inf = cache.info_fast()
+        kv_e2e += B * (inf[0] + inf[1]) * L
+    barrier()
+    e2e_s = time.perf_counter() - t0
+    status = cache.kernel_status()
+    assert status == 0, f"kernel status word {status}"
+    assert all(torch.isfinite(o).all() for o in outs)
+
+    times = torch.tensor([ms, e2e_s * 1e3], dtype=torch.float64, device=device)
+    if world > 1:
+        torch.distributed.all_reduce(times, op=torch.distributed.ReduceOp.MAX)
+    ms_max, e2e_ms_max = times.tolist()
+    peak, peak_kind = peaks()
+    bytes_per_launch = byte_sum / max(k_n, 1)
+    q_out_part = 0  # q, out and partials are not counted in the algorithmic bytes
+    achieved = bytes_per_launch / (k_ms / max(k_n, 1) * 1e-3) / 1e9 if k_n else None
+    inf = cache.info(0)
+    line = {
+        "metric": "decode_attn_kv_tokens_per_s", "value": kv_tokens * world / (ms_max * 1e-3),
+        "unit": "KV tokens/s", "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms_max / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "layers": L, "batch": B, "q_heads": Hq, "kv_heads": Hkv,
+                   "head_dim": D, "context": ctx, "window": W, "group": G, "bits": 2,
+                   "n_quant": int(inf.n_quant), "n_fp": int(inf.n_fp), "n_splits": int(inf.n_splits),
+                   "step": "per layer: lq_append (+lq_compress on overflow) + lq_decode_attn",
+                   "l2": "inputs larger than L2: %.2f GB of cache touched per step" % (bytes_step_last / 1e9),
+                   "replicas": "independent per GPU, no collective on the data path"},
+        "per_layer_us": ms_max / steps / L * 1e3,
+        "algorithmic_gbs_whole_step": bytes_step_last / (ms_max / steps * 1e-3) / 1e9,
+        "gpu_launches": int(launches),
+        "clocks": clk.summary(),
+        "e2e": {"value": kv_e2e * world / (e2e_ms_max * 1e-3), "unit": "KV tokens/s",
+                "h2d_bytes_per_step": L * (2 * B * Hkv * D * 2 + B * Hq * D * 2),
+                "d2h_bytes_per_step": L * B * Hq * D * 4, "steps": e2e_steps,
+                "api": "lq_decode_step_host (pinned host buffers, one stream sync per step)"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak if achieved else None, "traffic": None, "peak_kind": peak_kind,
+                     "kernel": "lq_decode_mma_kernel", "bytes_per_launch": bytes_per_launch,
+                     "us_per_launch": k_ms / max(k_n, 1) * 1e3, "launches_timed": int(k_n),
+                     "frac_of_8tbs_nominal": achieved / 8000.0 if achieved else None},
+    }
+    traffic_file = os.path.join(ROOT, "profiles", "traffic_%s.json" % args.workload)
+    if os.path.exists(traffic_file):
+        with open(traffic_file) as f:
+            line["roofline"]["traffic"] = json.load(f).get("dram_bytes_per_launch")
+    return line, cache
+
+
+def oracle_layer_step(wl, device, n_threads, min_seconds, max_reps):
+    """Times the CPU oracle on one layer of the workload: append one token + attention."""
+    import oracle
+    B, Hq, Hkv, W, G, ctx = (wl[k] for k in ("B", "Hq", "Hkv", "W", "G", "ctx"))
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G)
+    wl1 = dict(wl, L=1)
+    prefill(None, wl1, device, sink=lambda l, k, v: oc.append(synth.bf16_bits(k), synth.bf16_bits(v)))
+    k, v = synth.keys_values(wl["seed"] + 100, B, Hkv, Q_ROTATE, D, device, layer=0, outliers=wl.get("_outliers"))
+    kb, vb = synth.bf16_bits(k), synth.bf16_bits(v)
+    reps, t_total, kv = 0, 0.0, 0
+    times = []
+    while (t_total < min_seconds and reps < max_reps) or reps < 1:
+        s = reps % Q_ROTATE
+        q = synth.bf16_bits(synth.queries(wl["seed"], B, Hq, D, s, device, layer=0))
+        t0 = time.perf_counter()
+        oc.append(np.ascontiguousarray(kb[:, :, s:s + 1]), np.ascontiguousarray(vb[:, :, s:s + 1]))
+        oc.attention(q, 1.0 / np.sqrt(D), n_threads=n_threads)
+        dt = time.perf_counter() - t0
+        times.append(dt)
+        t_total += dt
+        kv += B * (oc.n_quant + oc.n_fp)
+        reps += 1
+    return kv / t_total, reps, t_total, times
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=128)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama3-8b-8k", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="override the number of stacked layer caches (profiling runs)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    wl = dict(WORKLOADS[args.workload])
+    if args.layers > 0:
+        wl["L"] = args.layers
+    wl["_outliers"] = synth.outlier_channels(wl["seed"], wl["Hkv"], D, wl["n_outliers"]) if wl["n_outliers"] else None
+    cores = os.cpu_count() or 1
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        import oracle
+        oracle.build()
+        device = torch.device("cuda", local) if torch.cuda.is_available() else torch.device("cpu")
+        for _ in range(max(args.warmup, 0)):
+            pass  # the oracle has no warm state; its first timed step is as good as any
+        tput, reps, t_total, times = oracle_layer_step(wl, device, cores, min_seconds=0.0, max_reps=max(args.steps, 1))
+        sample = "one of %d layers of %s per step: append 1 token + attention, float64" % (wl["L"], args.workload)
+        line = {"impl": "reference", "metric": "decode_attn_kv_tokens_per_s", "value": tput, "unit": "KV tokens/s",
+                "n_gpus": args.gpus, "steps": reps, "warmup": args.warmup, "ms_per_step": t_total / reps * 1e3,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                "config": {"workload": args.workload, "batch": wl["B"], "q_heads": wl["Hq"], "kv_heads": wl["Hkv"],
+                           "context": wl["ctx"], "window": wl["W"], "group": wl["G"]},
+                "cpu_baseline": {"value": tput, "unit": "KV tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+                "e2e": {"value": tput, "unit": "KV tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(line))
+        return 0
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the LogQuant kernels")
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    if world > 1:
+        torch.distributed.init_process_group("nccl", device_id=device)
+    line, cache = run_ours(args, wl, rank, world, device)
+    if rank == 0:
+        if not args.no_cpu_baseline:
+            import oracle
+            oracle.build()
+            tput, reps, t_total, _ = oracle_layer_step(wl, device, cores, min_seconds=10.0, max_reps=64)
+            line["cpu_baseline"] = {"value": tput, "unit": "KV tokens/s", "cores": cores, "kind": "oracle",
+                                    "sample": "%d decode steps of one of the %d layers (append 1 token + float64 "
+                                              "attention over all %d sequences), %.1f s" % (reps, wl["L"], wl["B"], t_total)}
+        print(json.dumps(line))
+    cache.close()
+    if world > 1:
+        torch.distributed.barrier()
+        torch.distributed.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

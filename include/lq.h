@@ -85,6 +85,7 @@ typedef struct {
   int64_t bytes_quant_per_token; /* per KV head: codes + amortised scale/zero (96 at G=32, 80 at G=64) */
   int32_t n_splits;            /* split-K partitions the next lq_decode_attn would use           */
   int32_t reserved;
+  int64_t n_kernel_launches;   /* kernels this cache has launched so far (all layers)            */
 } lq_info_t;
 
 /*
@@ -146,13 +147,27 @@ lq_status_t lq_decode_attn(lq_cache_t* cache, int32_t layer, const void* q, floa
 /* One decode step of one layer with HOST buffers: copies k_host, v_host ([B,Hkv,1,D] bf16) and
  * q_host ([B,Hq,D] bf16) to the device, appends (running the overflow step first when the window
  * is full, whatever auto_compress says), runs decode attention and copies the fp32 result to
- * out_host ([B,Hq,D]).  Synchronises `stream` before returning.  Pinned host memory is
- * recommended. */
+ * out_host ([B,Hq,D]).  sync != 0: synchronises `stream` before returning.  sync == 0: everything
+ * is only enqueued (the host buffers must be pinned and must stay untouched, and out_host is
+ * valid, once the caller has synchronised the stream); each layer has its own staging buffers,
+ * so steps of different layers may be enqueued back to back. */
 lq_status_t lq_decode_step_host(lq_cache_t* cache, int32_t layer, const void* k_host,
                                 const void* v_host, const void* q_host, float sm_scale,
-                                float* out_host, void* stream);
+                                float* out_host, int32_t sync, void* stream);
 
-/* Introspection (not on the hot path). */
+/* Kernel timing for benchmarks.  While enabled, every lq_decode_attn brackets its split-K
+ * attention kernel with a pair of CUDA events on the call's stream (at most 8192 pairs are kept;
+ * later launches are not timed).  lq_profile_read synchronises the device and returns the summed
+ * duration in milliseconds and the number of timed launches since profiling was enabled. */
+lq_status_t lq_profile_enable(lq_cache_t* cache, int32_t on);
+lq_status_t lq_profile_read(lq_cache_t* cache, double* total_ms, int64_t* n_launches);
+
+/* Device status word of the cache: 0 = healthy; bit 0 = a bounded wait inside a kernel gave up
+ * (its output is then invalid).  Kernels never trap or spin for ever; they record the failure
+ * here.  Synchronises the device. */
+lq_status_t lq_kernel_status(lq_cache_t* cache, int32_t* status_word);
+
+/* Introspection (host-side bookkeeping only; never synchronises). */
 lq_status_t lq_cache_info(const lq_cache_t* cache, int32_t layer, lq_info_t* info);
 
 /* Copy the canonical image of one layer into the caller's HOST buffers.  Synchronises the device. */

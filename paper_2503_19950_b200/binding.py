@@ -26,7 +26,8 @@ class lq_config_t(C.Structure):
 class lq_info_t(C.Structure):
     _fields_ = [("n_seen", C.c_int64), ("n_fp", C.c_int64), ("n_quant", C.c_int64), ("n_events", C.c_int64),
                 ("bytes_device", C.c_int64), ("bytes_decode_step", C.c_int64),
-                ("bytes_quant_per_token", C.c_int64), ("n_splits", C.c_int32), ("reserved", C.c_int32)]
+                ("bytes_quant_per_token", C.c_int64), ("n_splits", C.c_int32), ("reserved", C.c_int32),
+                ("n_kernel_launches", C.c_int64)]
 
 
 class lq_image_t(C.Structure):
@@ -35,8 +36,8 @@ class lq_image_t(C.Structure):
 
 
 SYMBOLS = ["lq_cache_create", "lq_destroy", "lq_append", "lq_compress", "lq_decode_attn",
-           "lq_decode_step_host", "lq_cache_info", "lq_export", "lq_next_evicted_ids", "lq_status_str",
-           "lq_last_error"]
+           "lq_decode_step_host", "lq_profile_enable", "lq_profile_read", "lq_kernel_status", "lq_cache_info", "lq_export",
+           "lq_next_evicted_ids", "lq_status_str", "lq_last_error"]
 
 _lib = None
 
@@ -61,7 +62,10 @@ def load_library():
         L.lq_append.argtypes = [vp, i32, vp, vp, i32, vp]
         L.lq_compress.argtypes = [vp, i32, vp]
         L.lq_decode_attn.argtypes = [vp, i32, vp, C.c_float, vp, i32, vp]
-        L.lq_decode_step_host.argtypes = [vp, i32, vp, vp, vp, C.c_float, vp, vp]
+        L.lq_decode_step_host.argtypes = [vp, i32, vp, vp, vp, C.c_float, vp, i32, vp]
+        L.lq_kernel_status.argtypes = [vp, C.POINTER(C.c_int32)]
+        L.lq_profile_enable.argtypes = [vp, i32]
+        L.lq_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         L.lq_cache_info.argtypes = [vp, i32, C.POINTER(lq_info_t)]
         L.lq_export.argtypes = [vp, i32, C.POINTER(lq_image_t)]
         L.lq_next_evicted_ids.argtypes = [vp, i32, vp]
@@ -144,11 +148,29 @@ class LogQuantCache:
         self._check(self._lib.lq_decode_attn(self._h, layer, _ptr(q), sm_scale, _ptr(out), out_dtype,
                                              _stream(stream)))
 
-    def decode_step_host(self, layer, k_host, v_host, q_host, out_host, sm_scale=0.0, stream=None):
+    def decode_step_host(self, layer, k_host, v_host, q_host, out_host, sm_scale=0.0, sync=True, stream=None):
         self._check(self._lib.lq_decode_step_host(self._h, layer, _ptr(k_host), _ptr(v_host), _ptr(q_host),
-                                                  sm_scale, _ptr(out_host), _stream(stream)))
+                                                  sm_scale, _ptr(out_host), int(sync), _stream(stream)))
+
+    def profile_enable(self, on=True):
+        self._check(self._lib.lq_profile_enable(self._h, int(on)))
+
+    def profile_read(self):
+        ms, n = C.c_double(0), C.c_int64(0)
+        self._check(self._lib.lq_profile_read(self._h, C.byref(ms), C.byref(n)))
+        return ms.value, n.value
 
     # -- introspection --------------------------------------------------------------------
+    def kernel_status(self) -> int:
+        w = C.c_int32(0)
+        self._check(self._lib.lq_kernel_status(self._h, C.byref(w)))
+        return w.value
+
+    def info_fast(self, layer=0):
+        """(n_quant, n_fp) of one layer."""
+        inf = self.info(layer)
+        return inf.n_quant, inf.n_fp
+
     def info(self, layer=0) -> lq_info_t:
         info = lq_info_t()
         self._check(self._lib.lq_cache_info(self._h, layer, C.byref(info)))

@@ -42,11 +42,16 @@ struct lq_cache {
   float* part_o = nullptr;
   float* part_ml = nullptr;
   int* status = nullptr;
-  // staging for the host-buffer entry point
-  void* stage_k = nullptr;
-  void* stage_v = nullptr;
-  void* stage_q = nullptr;
-  float* stage_out = nullptr;
+  // staging for the host-buffer entry point, one slice per layer
+  uint8_t* stage_k = nullptr;
+  uint8_t* stage_v = nullptr;
+  uint8_t* stage_q = nullptr;
+  uint8_t* stage_out = nullptr;
+  int64_t n_launches = 0;
+  // optional timing of the split-K attention kernel
+  bool profiling = false;
+  std::vector<cudaEvent_t> ev_pool;  // 2 events per timed launch
+  size_t ev_used = 0;
   std::string last_error;
 };
 
@@ -80,6 +85,7 @@ void free_all(lq_cache* c) {
     cudaFree(c->stage_v);
     cudaFree(c->stage_q);
     cudaFree(c->stage_out);
+    for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   }
 }
 
@@ -140,6 +146,7 @@ lq_status_t run_events(lq_cache* c, const std::vector<int>& full_layers, cudaStr
     if (!c->dry) {
       cudaError_t e = launch_compress(c->cv, ll, ev, Li.n_quant / c->cfg.group, st);
       if (e != cudaSuccess) return cuda_fail(c, e, "lq_compress_kernel");
+      c->n_launches++;
     }
     for (int k : members) {
       done[k] = 1;
@@ -159,7 +166,7 @@ int choose_splits(const lq_cache* c, const LayerState& L) {
   return static_cast<int>(s);
 }
 
-bool use_mma(const lq_cache* c) { return c->cfg.kernel == LQ_KERNEL_MMA; }  // TEMP until the MMA kernel lands
+bool use_mma(const lq_cache* c) { return c->cfg.kernel != LQ_KERNEL_SCALAR; }
 
 }  // namespace
 
@@ -224,10 +231,12 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
               dev_alloc(c, reinterpret_cast<void**>(&c->part_o), pairs * c->max_splits * r * kD * 4) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->part_ml), pairs * c->max_splits * r * 2 * 4) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->status), 256) &&
-              dev_alloc(c, &c->stage_k, pairs * kD * 2) && dev_alloc(c, &c->stage_v, pairs * kD * 2) &&
-              dev_alloc(c, &c->stage_q, static_cast<int64_t>(cfg->batch) * cfg->n_q_heads * kD * 2) &&
+              dev_alloc(c, reinterpret_cast<void**>(&c->stage_k), cfg->n_layers * pairs * kD * 2) &&
+              dev_alloc(c, reinterpret_cast<void**>(&c->stage_v), cfg->n_layers * pairs * kD * 2) &&
+              dev_alloc(c, reinterpret_cast<void**>(&c->stage_q),
+                        static_cast<int64_t>(cfg->n_layers) * cfg->batch * cfg->n_q_heads * kD * 2) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_out),
-                        static_cast<int64_t>(cfg->batch) * cfg->n_q_heads * kD * 4);
+                        static_cast<int64_t>(cfg->n_layers) * cfg->batch * cfg->n_q_heads * kD * 4);
     if (ok) ok = cudaMemset(c->status, 0, 256) == cudaSuccess;
     // the fp store must never hold non-finite garbage in unused slots of a partly filled tile
     if (ok) ok = cudaMemset(cv.fp, 0, static_cast<size_t>(cv.fp_layer_stride) * cfg->n_layers) == cudaSuccess;
@@ -270,6 +279,7 @@ lq_status_t lq_append(lq_cache_t* c, int32_t layer, const void* k, const void* v
     if (!c->dry) {
       cudaError_t e = launch_append(c->cv, layer, k, v, n, done, take, L.n_fp, st);
       if (e != cudaSuccess) return cuda_fail(c, e, "lq_append_kernel");
+      c->n_launches++;
     }
     for (int t = 0; t < take; ++t) {
       L.age_slot.push_back(L.n_fp + t);
@@ -319,6 +329,8 @@ lq_status_t lq_decode_attn(lq_cache_t* c, int32_t layer, const void* q, float sm
   a.out_bf16 = out_dtype;
   a.status = c->status;
   cudaError_t e;
+  const bool timed = c->profiling && c->ev_used + 2 <= c->ev_pool.size();
+  if (timed) cudaEventRecord(c->ev_pool[c->ev_used], st);
   if (use_mma(c)) {
     a.S = c->cfg.n_splits > 0 ? std::min(c->cfg.n_splits, c->max_splits)
                               : std::min(c->max_splits, decode_mma_max_splits(c->cv, L.n_fp, L.n_quant, c->sm_count));
@@ -329,13 +341,18 @@ lq_status_t lq_decode_attn(lq_cache_t* c, int32_t layer, const void* q, float sm
     e = launch_decode_scalar(a, st);
     if (e != cudaSuccess) return cuda_fail(c, e, "lq_decode_scalar_kernel");
   }
+  if (timed) {
+    cudaEventRecord(c->ev_pool[c->ev_used + 1], st);
+    c->ev_used += 2;
+  }
   e = launch_merge(a, st);
   if (e != cudaSuccess) return cuda_fail(c, e, "lq_merge_kernel");
+  c->n_launches += 2;
   return LQ_OK;
 }
 
 lq_status_t lq_decode_step_host(lq_cache_t* c, int32_t layer, const void* k_host, const void* v_host,
-                                const void* q_host, float sm_scale, float* out_host, void* stream) {
+                                const void* q_host, float sm_scale, float* out_host, int32_t sync, void* stream) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers) return LQ_ERR_INVALID_ARG;
   if (c->dry) return LQ_ERR_UNSUPPORTED;
   if (!k_host || !v_host || !q_host || !out_host) return LQ_ERR_INVALID_ARG;
@@ -344,22 +361,65 @@ lq_status_t lq_decode_step_host(lq_cache_t* c, int32_t layer, const void* k_host
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t kvb = static_cast<size_t>(c->cfg.batch) * c->cfg.n_kv_heads * kD * 2;
   const size_t qb = static_cast<size_t>(c->cfg.batch) * c->cfg.n_q_heads * kD * 2;
+  uint8_t* sk = c->stage_k + layer * kvb;
+  uint8_t* sv = c->stage_v + layer * kvb;
+  uint8_t* sq = c->stage_q + layer * qb;
+  uint8_t* so = c->stage_out + layer * qb * 2;
   cudaError_t e;
-  if ((e = cudaMemcpyAsync(c->stage_k, k_host, kvb, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
-      (e = cudaMemcpyAsync(c->stage_v, v_host, kvb, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
-      (e = cudaMemcpyAsync(c->stage_q, q_host, qb, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+  if ((e = cudaMemcpyAsync(sk, k_host, kvb, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(sv, v_host, kvb, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(sq, q_host, qb, cudaMemcpyHostToDevice, st)) != cudaSuccess)
     return cuda_fail(c, e, "host-to-device copy");
   if (L.n_fp == 3 * c->cfg.window) {
     lq_status_t s = run_events(c, std::vector<int>{layer}, st);
     if (s != LQ_OK) return s;
   }
-  lq_status_t s = lq_append(c, layer, c->stage_k, c->stage_v, 1, stream);
+  lq_status_t s = lq_append(c, layer, sk, sv, 1, stream);
   if (s != LQ_OK) return s;
-  s = lq_decode_attn(c, layer, c->stage_q, sm_scale, c->stage_out, 0, stream);
+  s = lq_decode_attn(c, layer, sq, sm_scale, so, 0, stream);
   if (s != LQ_OK) return s;
-  if ((e = cudaMemcpyAsync(out_host, c->stage_out, qb * 2, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+  if ((e = cudaMemcpyAsync(out_host, so, qb * 2, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
     return cuda_fail(c, e, "device-to-host copy");
-  if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(c, e, "cudaStreamSynchronize");
+  if (sync && (e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(c, e, "cudaStreamSynchronize");
+  return LQ_OK;
+}
+
+lq_status_t lq_profile_enable(lq_cache_t* c, int32_t on) {
+  if (!c) return LQ_ERR_INVALID_ARG;
+  if (c->dry) return LQ_ERR_UNSUPPORTED;
+  if (on && c->ev_pool.empty()) {
+    c->ev_pool.resize(2 * 8192);
+    for (auto& ev : c->ev_pool)
+      if (cudaEventCreate(&ev) != cudaSuccess) return cuda_fail(c, cudaGetLastError(), "cudaEventCreate");
+  }
+  c->profiling = on != 0;
+  c->ev_used = 0;
+  return LQ_OK;
+}
+
+lq_status_t lq_profile_read(lq_cache_t* c, double* total_ms, int64_t* n_launches) {
+  if (!c || !total_ms || !n_launches) return LQ_ERR_INVALID_ARG;
+  if (c->dry) return LQ_ERR_UNSUPPORTED;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(c, e, "cudaDeviceSynchronize");
+  double sum = 0.0;
+  for (size_t i = 0; i + 1 < c->ev_used; i += 2) {
+    float ms = 0.f;
+    if ((e = cudaEventElapsedTime(&ms, c->ev_pool[i], c->ev_pool[i + 1])) != cudaSuccess)
+      return cuda_fail(c, e, "cudaEventElapsedTime");
+    sum += ms;
+  }
+  *total_ms = sum;
+  *n_launches = static_cast<int64_t>(c->ev_used / 2);
+  return LQ_OK;
+}
+
+lq_status_t lq_kernel_status(lq_cache_t* c, int32_t* word) {
+  if (!c || !word) return LQ_ERR_INVALID_ARG;
+  *word = 0;
+  if (c->dry) return LQ_OK;
+  cudaError_t e = cudaMemcpy(word, c->status, sizeof(int32_t), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(c, e, "status read");
   return LQ_OK;
 }
 
@@ -372,6 +432,7 @@ lq_status_t lq_cache_info(const lq_cache_t* c, int32_t layer, lq_info_t* info) {
   info->n_quant = L.n_quant;
   info->n_events = L.n_events;
   info->bytes_device = c->bytes_device;
+  info->n_kernel_launches = c->n_launches;
   info->bytes_quant_per_token = quant_tile_bytes(c->cfg.group) / c->cfg.group;
   info->bytes_decode_step = static_cast<int64_t>(c->cfg.batch) * c->cfg.n_kv_heads *
                             (L.n_quant * info->bytes_quant_per_token + static_cast<int64_t>(L.n_fp) * 4 * kD);

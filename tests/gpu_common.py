@@ -74,6 +74,7 @@ def run_case(B, Hq, Hkv, W, G, n_prefill, n_steps, seed, kernel, n_outliers=3, c
         err = float(np.abs(got - ref).max())
         assert err <= tol, f"step {step}: max|delta| {err:.3e} > tol {tol:.3e}"
         worst = max(worst, err / tol)
+    assert cache.kernel_status() == 0
     cache.close()
     oc.close()
     return worst

@@ -12,7 +12,7 @@ from paper_2503_19950_b200 import (LQ_KERNEL_AUTO, LQ_KERNEL_MMA, LQ_KERNEL_SCAL
 
 pytestmark = pytest.mark.gpu
 
-KERNELS = [LQ_KERNEL_SCALAR]
+KERNELS = [LQ_KERNEL_SCALAR, LQ_KERNEL_MMA]
 
 
 @pytest.fixture(scope="module", autouse=True)
