@@ -71,7 +71,7 @@ typedef struct {
   int32_t auto_compress; /* 1: lq_append runs the overflow step itself when the window is full   */
   int32_t device;        /* CUDA device ordinal, or LQ_DEVICE_NONE for bookkeeping only          */
   int32_t kernel;        /* LQ_KERNEL_*                                                          */
-  int32_t n_splits;      /* split-K partitions per (batch row, KV head); 0 = chosen by the library */
+  int32_t n_splits;      /* split-K CTAs per (batch row, KV head); 0 = chosen by the library     */
 } lq_config_t;
 
 typedef struct {
@@ -83,8 +83,9 @@ typedef struct {
   int64_t bytes_decode_step;   /* algorithmic bytes one lq_decode_attn on this layer has to read:
                                   B*Hkv*(n_quant*bytes_quant_per_token + n_fp*4*D); q/out excluded */
   int64_t bytes_quant_per_token; /* per KV head: codes + amortised scale/zero (96 at G=32, 80 at G=64) */
-  int32_t n_splits;            /* split-K partitions the next lq_decode_attn would use           */
-  int32_t reserved;
+  int32_t n_splits;            /* split-K partial records per (batch row, KV head) the next
+                                  lq_decode_attn would use                                        */
+  int32_t n_ctas;              /* CTAs of its attention kernel (tensor-core kernel; else 0)      */
   int64_t n_kernel_launches;   /* kernels this cache has launched so far (all layers)            */
 } lq_info_t;
 

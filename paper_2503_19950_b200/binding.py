@@ -7,7 +7,7 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "liblogquant.so")
+_LIB_PATH = os.path.join(_HERE, "liblogquant%s.so" % os.environ.get("LQ_LIB_SUFFIX", ""))
 
 LQ_DEVICE_NONE = -1
 LQ_KERNEL_AUTO, LQ_KERNEL_SCALAR, LQ_KERNEL_MMA = 0, 1, 2
@@ -26,7 +26,7 @@ class lq_config_t(C.Structure):
 class lq_info_t(C.Structure):
     _fields_ = [("n_seen", C.c_int64), ("n_fp", C.c_int64), ("n_quant", C.c_int64), ("n_events", C.c_int64),
                 ("bytes_device", C.c_int64), ("bytes_decode_step", C.c_int64),
-                ("bytes_quant_per_token", C.c_int64), ("n_splits", C.c_int32), ("reserved", C.c_int32),
+                ("bytes_quant_per_token", C.c_int64), ("n_splits", C.c_int32), ("n_ctas", C.c_int32),
                 ("n_kernel_launches", C.c_int64)]
 
 

@@ -42,6 +42,7 @@ struct lq_cache {
   float* part_o = nullptr;
   float* part_ml = nullptr;
   int* status = nullptr;
+  int* tickets = nullptr;  // per (b, kv) arrival counters of the fused split-K merge
   // staging for the host-buffer entry point, one slice per layer
   uint8_t* stage_k = nullptr;
   uint8_t* stage_v = nullptr;
@@ -81,6 +82,7 @@ void free_all(lq_cache* c) {
     cudaFree(c->part_o);
     cudaFree(c->part_ml);
     cudaFree(c->status);
+    cudaFree(c->tickets);
     cudaFree(c->stage_k);
     cudaFree(c->stage_v);
     cudaFree(c->stage_q);
@@ -222,15 +224,17 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
     if (e != cudaSuccess) { delete c; cudaGetLastError(); return LQ_ERR_CUDA; }
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, cfg->device) == cudaSuccess) c->sm_count = prop.multiProcessorCount;
+    // split-K partial records reserved per (b, kv)
     c->max_splits = cfg->n_splits > 0
                         ? cfg->n_splits
-                        : static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(512, (8LL * c->sm_count + pairs - 1) / pairs)));
+                        : static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(256, (8LL * c->sm_count + pairs - 1) / pairs)));
     const int r = ratio(c);
     bool ok = dev_alloc(c, reinterpret_cast<void**>(&cv.quant), cv.quant_layer_stride * cfg->n_layers) &&
               dev_alloc(c, reinterpret_cast<void**>(&cv.fp), cv.fp_layer_stride * cfg->n_layers) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->part_o), pairs * c->max_splits * r * kD * 4) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->part_ml), pairs * c->max_splits * r * 2 * 4) &&
-              dev_alloc(c, reinterpret_cast<void**>(&c->status), 256) &&
+              dev_alloc(c, reinterpret_cast<void**>(&c->status), 256 + (1 << 20)) &&
+              dev_alloc(c, reinterpret_cast<void**>(&c->tickets), pairs * 8) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_k), cfg->n_layers * pairs * kD * 2) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_v), cfg->n_layers * pairs * kD * 2) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_q),
@@ -238,6 +242,7 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_out),
                         static_cast<int64_t>(cfg->n_layers) * cfg->batch * cfg->n_q_heads * kD * 4);
     if (ok) ok = cudaMemset(c->status, 0, 256) == cudaSuccess;
+    if (ok) ok = cudaMemset(c->tickets, 0, pairs * 8) == cudaSuccess;
     // the fp store must never hold non-finite garbage in unused slots of a partly filled tile
     if (ok) ok = cudaMemset(cv.fp, 0, static_cast<size_t>(cv.fp_layer_stride) * cfg->n_layers) == cudaSuccess;
     if (!ok) {
@@ -311,7 +316,7 @@ lq_status_t lq_decode_attn(lq_cache_t* c, int32_t layer, const void* q, float sm
                            int32_t out_dtype, void* stream) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers || (out_dtype != 0 && out_dtype != 1)) return LQ_ERR_INVALID_ARG;
   if (c->dry) return LQ_ERR_UNSUPPORTED;
-  if (!q || !out) return LQ_ERR_INVALID_ARG;
+  if (!q || !out || (reinterpret_cast<uintptr_t>(q) & 15)) return LQ_ERR_INVALID_ARG;
   LayerState& L = c->layers[layer];
   if (L.n_fp + L.n_quant == 0) return LQ_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -328,12 +333,15 @@ lq_status_t lq_decode_attn(lq_cache_t* c, int32_t layer, const void* q, float sm
   a.out = out;
   a.out_bf16 = out_dtype;
   a.status = c->status;
+  a.tickets = nullptr;
   cudaError_t e;
   const bool timed = c->profiling && c->ev_used + 2 <= c->ev_pool.size();
   if (timed) cudaEventRecord(c->ev_pool[c->ev_used], st);
+  a.tiles_fp = a.tiles_quant = 0;
+  a.zero = 0;
   if (use_mma(c)) {
-    a.S = c->cfg.n_splits > 0 ? std::min(c->cfg.n_splits, c->max_splits)
-                              : std::min(c->max_splits, decode_mma_max_splits(c->cv, L.n_fp, L.n_quant, c->sm_count));
+    plan_decode_mma(a, c->sm_count, c->max_splits, c->cfg.n_splits);
+    a.tickets = c->tickets;  // the CTA that completes a (b, kv) pair merges it: no second launch
     e = launch_decode_mma(a, st);
     if (e != cudaSuccess) return cuda_fail(c, e, "lq_decode_mma_kernel");
   } else {
@@ -345,9 +353,12 @@ lq_status_t lq_decode_attn(lq_cache_t* c, int32_t layer, const void* q, float sm
     cudaEventRecord(c->ev_pool[c->ev_used + 1], st);
     c->ev_used += 2;
   }
-  e = launch_merge(a, st);
-  if (e != cudaSuccess) return cuda_fail(c, e, "lq_merge_kernel");
-  c->n_launches += 2;
+  if (a.tickets == nullptr) {
+    e = launch_merge(a, st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "lq_merge_kernel");
+    c->n_launches++;
+  }
+  c->n_launches++;
   return LQ_OK;
 }
 
@@ -414,6 +425,13 @@ lq_status_t lq_profile_read(lq_cache_t* c, double* total_ms, int64_t* n_launches
   return LQ_OK;
 }
 
+#ifdef LQ_EXP_TRACE
+lq_status_t lq_debug_trace(lq_cache_t* c, void* host, int bytes) {
+  cudaDeviceSynchronize();
+  return cudaMemcpy(host, c->status + 64, bytes, cudaMemcpyDeviceToHost) == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
+}
+#endif
+
 lq_status_t lq_kernel_status(lq_cache_t* c, int32_t* word) {
   if (!c || !word) return LQ_ERR_INVALID_ARG;
   *word = 0;
@@ -438,10 +456,15 @@ lq_status_t lq_cache_info(const lq_cache_t* c, int32_t layer, lq_info_t* info) {
                             (L.n_quant * info->bytes_quant_per_token + static_cast<int64_t>(L.n_fp) * 4 * kD);
   if (c->dry || L.n_fp + L.n_quant == 0)
     info->n_splits = 0;
-  else if (use_mma(c))
-    info->n_splits = c->cfg.n_splits > 0 ? std::min(c->cfg.n_splits, c->max_splits)
-                                         : std::min(c->max_splits, decode_mma_max_splits(c->cv, L.n_fp, L.n_quant, c->sm_count));
-  else
+  else if (use_mma(c)) {
+    DecodeArgs a;
+    a.cv = c->cv;
+    a.n_fp = L.n_fp;
+    a.n_quant = L.n_quant;
+    plan_decode_mma(a, c->sm_count, c->max_splits, c->cfg.n_splits);
+    info->n_splits = a.S;
+    info->n_ctas = a.S * c->cfg.batch * c->cfg.n_kv_heads;
+  } else
     info->n_splits = choose_splits(c, L);
   return LQ_OK;
 }

@@ -1,10 +1,13 @@
 // Tensor-core decode attention over the mixed cache (LQ_KERNEL_MMA): split-K first pass.
 //
-// One CTA = one (b, kv head, split); 4 warps, each with a private ring of shared-memory stages
-// filled by 1-D bulk copies (cp.async.bulk + mbarrier, no multicast).  A warp walks its own
-// contiguous range of "units" -- fp tiles (16 bf16 tokens, 8 KB) first, then quant units (one or
-// two key groups) -- and keeps a private online-softmax state (m, l, o) that the CTA merges at
-// the end into one split-K partial (Eq. 3 makes any visiting order legal).
+// Work partition: the tiles of all (b, kv head) pairs are laid on one cost line and cut into
+// equal ranges, one per CTA (a multiple of the SM count), so every SM gets the same instruction
+// load whatever the batch size; a CTA that straddles a pair boundary simply emits one split-K
+// partial per pair it touches.  Inside a CTA each of the 4 warps owns a private ring of
+// shared-memory stages filled by 1-D bulk copies (cp.async.bulk + mbarrier, no multicast) and a
+// private online-softmax state (m, l, o); the CTA merges the warp states into the partial (Eq. 3
+// makes any visiting order legal).  Units: fp tiles (16 bf16 tokens, 8 KB) first, then quant
+// tiles (one key group of G tokens each).
 //
 // Contractions (mma.sync.m16n8k16, fp32 accumulate), r = query heads per KV head (<= 8):
 //   q.k   tokens on M (16), query heads on N, channels on K.  Heads are handled in column blocks
@@ -15,11 +18,14 @@
 //         and one packed fma (both have 8-bit significands), so q.k^ is exact up to fp32
 //         accumulation.  The key zero contributes q.z per group, computed by 8 MMAs per group.
 //         bf16 keys: ldmatrix fragments of the swizzled rows, bf16 x bf16 exact.
-//   p.v   channels on M (16), heads on N (8), tokens on K.  2-bit values: fp16 subnormal codes
-//         c*2^(p-24) times p*s_v rounded to fp16; the value zero goes through one extra MMA per
-//         16 tokens.  bf16 values: ldmatrix.trans fragments times p split into bf16 hi + lo.
+//   p.v   channels on M (16), tokens on K.
+//         r <= 4: columns are again (hi, lo) per head, everything in bf16: value codes as bf16
+//         subnormals, p*s_v split into hi + lo with packed bf16 multiply/fma, value zero through
+//         one extra MMA per 16 tokens; bf16 values through ldmatrix.trans.
+//         r  > 4: heads on the 8 columns; value codes as fp16 subnormals times p*s_v rounded to
+//         fp16; bf16 values times p split into bf16 hi + lo (two MMAs).
 //   The softmax probabilities come out of q.k with (token, head) = (lane/4, lane%4) and are
-//   moved to the (head, token pair) arrangement p.v needs with 4 warp shuffles per 16 tokens.
+//   moved to the (column, token pair) arrangement p.v needs with 4 warp shuffles per 16 tokens.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -30,8 +36,9 @@ namespace lq {
 namespace {
 
 constexpr int kWarps = 4;
-constexpr int kStageBytes = 8192;
+constexpr int kStageBytes = 5120;  // one quant tile (3 KB at G=32, 5 KB at G=64) or half an fp tile (4 KB)
 constexpr int kStages = 2;
+constexpr int kCtasPerSm = 4;
 constexpr uint32_t kFull = 0xFFFFFFFFu;
 constexpr int kSpinLimit = 1 << 22;
 
@@ -96,6 +103,12 @@ __device__ __forceinline__ uint32_t bf16x2_fma(uint32_t a, uint32_t b, uint32_t 
   asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
   return d;
 }
+__device__ __forceinline__ float pow2i(int k) { return __int_as_float((k + 127) << 23); }  // 2^k, -126 <= k <= 127
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 // pack two floats: `lo` into bits [15:0], `hi` into bits [31:16]
 __device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
   uint32_t d;
@@ -120,52 +133,81 @@ __device__ __forceinline__ uint2 lds64(uint32_t addr) {
   return v;
 }
 
-// one code position of a packed word as two bf16 (key) / fp16 (value) subnormals
-template <int KS>
-__device__ __forceinline__ uint32_t kext(uint32_t w, uint32_t w8) {
-  return KS < 4 ? (w & (0x00030003u << (2 * KS))) : (w8 & (0x00030003u << (2 * (KS - 4))));
+// one code position of a packed word as two bf16 subnormals (positions 0,2,4,6 of each byte)
+template <int I>
+__device__ __forceinline__ uint32_t ext_bf16(uint32_t w, uint32_t w8) {
+#ifdef LQ_EXP_NOEXT
+  return I < 4 ? w : w8;
+#else
+  return I < 4 ? (w & (0x00030003u << (2 * I))) : (w8 & (0x00030003u << (2 * (I - 4))));
+#endif
 }
-template <int MT>
-__device__ __forceinline__ uint32_t vext(uint32_t w, uint32_t w10) {
-  return MT < 5 ? (w & (0x00030003u << (2 * MT))) : (w10 & (0x00030003u << (2 * (MT - 5))));
+// same with an index that becomes a constant once the caller's loop is unrolled
+__device__ __forceinline__ uint32_t ext_bf16_i(int i, uint32_t w, uint32_t w8) {
+#ifdef LQ_EXP_NOEXT
+  return i < 4 ? w : w8;
+#else
+  return i < 4 ? (w & (0x00030003u << (2 * i))) : (w8 & (0x00030003u << (2 * (i - 4))));
+#endif
+}
+// ... or as two fp16 subnormals (positions 0..8 direct, 10..14 after a shift by 10)
+template <int I>
+__device__ __forceinline__ uint32_t ext_f16(uint32_t w, uint32_t w10) {
+  return I < 5 ? (w & (0x00030003u << (2 * I))) : (w10 & (0x00030003u << (2 * (I - 5))));
 }
 
+// NCB = number of column blocks of 4 heads.  NCB == 1: p.v columns are (hi, lo) per head and the
+// probabilities carry a factor 2^64 (kPExp) so that products with bf16 subnormal codes stay normal.
 template <int NCB>
 struct WarpState {
-  float out[8][4];  // o^T: [channel tile][c-fragment]; columns = query heads
-  float zacc[4];    // sum_t p_t * vzero_t per (value group, head)
+  float out[8][4];  // o^T: [channel tile][c-fragment]
+  float zacc[4];    // sum_t p_t * vzero_t per (value group, column)
   float m[NCB];     // running max (log2 units) of head 4cb + lane%4
-  float l[NCB];     // this lane's share of the running denominator
-  bool quant_mode;  // out rows carry the code-position factor 2^(p(mt)-24)
+  float l[NCB];     // this lane's share of the running denominator (times 2^kPExp)
+  bool quant_mode;  // out rows carry the code-position factor
+};
+template <int NCB>
+struct Mode {
+  static constexpr float kPExp = NCB == 1 ? 64.f : 0.f;
 };
 
-// factor carried by the out rows of channel tile mt while in quant mode
-__device__ __forceinline__ float vpos_scale(int mt) { return exp2f(static_cast<float>(2 * (mt < 5 ? mt : mt - 5) - 24)); }
-
-// ---- online softmax on the 16 scores a lane quad column holds, then p in p.v arrangement ----
-// s[cb][th]: score (log2 units) of token 8*th + lane/4 for head 4cb + lane%4.
-// Returns pT[th][i]: probability of token 8*th + 2*(lane%4) + i for head lane/4.
+// factor the out rows of channel tile mt carry in quant mode, relative to fp mode
 template <int NCB>
-__device__ __forceinline__ void softmax_step(WarpState<NCB>& st, float (&s)[NCB][2], float (&pT)[2][2], int lane) {
-  const int n = lane >> 2, j = lane & 3;
+__device__ __forceinline__ int vpos_log2(int mt) {
+  return NCB == 1 ? 2 * (mt & 3) - 133 : 2 * (mt < 5 ? mt : mt - 5) - 24;
+}
+
+// ---- online softmax over the NSUB*16 scores of one tile ---------------------------------------
+// s[u][cb][th]: score (log2 units) of token 16u + 8th + lane/4 for head 4cb + lane%4; replaced by
+// the probabilities 2^(s - m + kPExp).
+template <int NCB, int NSUB>
+__device__ __forceinline__ void tile_softmax(WarpState<NCB>& st, float (&s)[NSUB][NCB][2], int lane, int opaque_zero) {
+  const int j = lane & 3;
   float corr[NCB];
   bool changed = false;
 #pragma unroll
   for (int cb = 0; cb < NCB; ++cb) {
-    float mx = fmaxf(s[cb][0], s[cb][1]);
+    float mx = fmaxf(s[0][cb][0], s[0][cb][1]);
+#pragma unroll
+    for (int u = 1; u < NSUB; ++u) mx = fmaxf(mx, fmaxf(s[u][cb][0], s[u][cb][1]));
     mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 4));
     mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 8));
     mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 16));
-    const float mn = fmaxf(st.m[cb], mx);
-    changed |= mn > st.m[cb];
-    corr[cb] = exp2f(st.m[cb] - mn);  // m = -inf initially -> 0
+    // the reference m only has to stay within 2^8 of the running maximum (p <= 256 is harmless),
+    // so it moves -- and the accumulators are rescaled -- only when a score exceeds it by more than 8
+    const bool up = mx > st.m[cb] + 8.f;  // m = -inf initially -> true
+    const float mn = up ? mx : st.m[cb];
+    changed |= up;
+    corr[cb] = ex2(st.m[cb] - mn);  // m = -inf -> 0; unchanged -> 1
     st.m[cb] = mn;
   }
-  if (__any_sync(kFull, changed)) {
+  // Written as a loop with an opaque exit so that it stays a real (rarely taken) branch instead
+  // of 36 multiplies and selects on every tile.
+  int again = __any_sync(kFull, changed);
+  while (again) {
     float ca, cbv;
     if (NCB == 1) {
-      ca = __shfl_sync(kFull, corr[0], (2 * j) & 3);
-      cbv = __shfl_sync(kFull, corr[0], (2 * j + 1) & 3);
+      ca = cbv = corr[0];  // all four accumulators of a lane belong to head lane%4
     } else {
       const float a0 = __shfl_sync(kFull, corr[0], (2 * j) & 3), a1 = __shfl_sync(kFull, corr[NCB - 1], (2 * j) & 3);
       const float b0 = __shfl_sync(kFull, corr[0], (2 * j + 1) & 3), b1 = __shfl_sync(kFull, corr[NCB - 1], (2 * j + 1) & 3);
@@ -179,32 +221,61 @@ __device__ __forceinline__ void softmax_step(WarpState<NCB>& st, float (&s)[NCB]
     st.zacc[0] *= ca; st.zacc[1] *= cbv; st.zacc[2] *= ca; st.zacc[3] *= cbv;
 #pragma unroll
     for (int cb = 0; cb < NCB; ++cb) st.l[cb] *= corr[cb];
+    again = opaque_zero;  // always 0, but only known at run time
   }
-  float p[NCB][2];
 #pragma unroll
   for (int cb = 0; cb < NCB; ++cb) {
-    p[cb][0] = exp2f(s[cb][0] - st.m[cb]);
-    p[cb][1] = exp2f(s[cb][1] - st.m[cb]);
-    st.l[cb] += p[cb][0] + p[cb][1];
+    const float off = Mode<NCB>::kPExp - st.m[cb];
+    float lsum = 0.f;
+#pragma unroll
+    for (int u = 0; u < NSUB; ++u) {
+      s[u][cb][0] = ex2(s[u][cb][0] + off);
+      s[u][cb][1] = ex2(s[u][cb][1] + off);
+      lsum += s[u][cb][0] + s[u][cb][1];
+    }
+    st.l[cb] += lsum;
   }
+}
+
+// probabilities of one 16-token sub-tile moved to the B-operand arrangement of p.v:
+// pT[th][i] = p(token 8th + 2*(lane%4) + i) for the head of column lane/4
+template <int NCB>
+__device__ __forceinline__ void transpose_p(const float (&p)[NCB][2], float (&pT)[2][2], int lane) {
+  const int n = lane >> 2, j = lane & 3;
 #pragma unroll
   for (int th = 0; th < 2; ++th)
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
-      const int src = 4 * (2 * j + i) + (n & 3);
-      float v = __shfl_sync(kFull, p[0][th], src);
-      if (NCB == 2) {
-        const float v1 = __shfl_sync(kFull, p[NCB - 1][th], src);
-        v = (n >> 2) ? v1 : v;
+      if (NCB == 1) {
+        pT[th][i] = __shfl_sync(kFull, p[0][th], 4 * (2 * j + i) + (n >> 1));  // column n -> head n/2
+      } else {
+        const int src = 4 * (2 * j + i) + (n & 3);  // column n -> head n
+        const float v0 = __shfl_sync(kFull, p[0][th], src), v1 = __shfl_sync(kFull, p[NCB - 1][th], src);
+        pT[th][i] = (n >> 2) ? v1 : v0;
       }
-      pT[th][i] = v;
     }
 }
 
-// ---- one fp tile: 16 bf16 tokens (rows swizzled in 16-byte chunks by row & 7) -------------
+// NCB == 1: split the probabilities into bf16 hi (even columns) / lo (odd columns).
+// H = hi in every lane; P = hi in even, lo in odd columns; Pz = 0 in even, lo in odd columns.
+__device__ __forceinline__ void split_p_bf16(const float (&pT)[2][2], uint32_t oddmask, uint32_t (&H)[2],
+                                             uint32_t (&P)[2], uint32_t (&Pz)[2]) {
+#pragma unroll
+  for (int th = 0; th < 2; ++th) {
+    H[th] = pack_bf16x2(pT[th][0], pT[th][1]);
+    const float f0 = __uint_as_float((H[th] << 16) & oddmask);
+    const float f1 = __uint_as_float(H[th] & oddmask & 0xFFFF0000u);
+    P[th] = pack_bf16x2(pT[th][0] - f0, pT[th][1] - f1);
+    Pz[th] = P[th] & oddmask;
+  }
+}
+
+// ---- one fp tile: 16 bf16 tokens (rows swizzled in 16-byte chunks by row & 7), loaded as two
+// units: the K rows (scores, softmax; leaves the p.v B operands in b0/b1), then the V rows -------
 template <int NCB>
-__device__ __forceinline__ void process_fp_tile(WarpState<NCB>& st, const uint32_t (&qs)[NCB][8][2], uint32_t tile,
-                                                int n_valid, const float (&kc)[4], int lane) {
+__device__ __forceinline__ void process_fp_keys(WarpState<NCB>& st, const uint32_t (&qs)[NCB][8][2], uint32_t krows,
+                                                int n_valid, const float (&kc)[4], int lane, uint32_t oddmask,
+                                                int opaque_zero, uint32_t (&b0)[2], uint32_t (&b1)[2]) {
   const int n = lane >> 2;
   float acc[NCB][4][4];
 #pragma unroll
@@ -216,7 +287,7 @@ __device__ __forceinline__ void process_fp_tile(WarpState<NCB>& st, const uint32
   {
     const int mi = lane >> 3, rr = lane & 7;
     const int token = rr + 8 * (mi & 1);
-    const uint32_t rowaddr = tile + token * 256;
+    const uint32_t rowaddr = krows + token * 256;
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
       const int chunk = 2 * ks + (mi >> 1);
@@ -226,7 +297,7 @@ __device__ __forceinline__ void process_fp_tile(WarpState<NCB>& st, const uint32
       for (int cb = 0; cb < NCB; ++cb) mma_bf16(acc[cb][ks & 3], a0, a1, a2, a3, qs[cb][ks][0], qs[cb][ks][1]);
     }
   }
-  float s[NCB][2];
+  float s[1][NCB][2];
 #pragma unroll
   for (int cb = 0; cb < NCB; ++cb) {
     float s0 = acc[cb][0][0] * kc[0], s1 = acc[cb][0][2] * kc[0];
@@ -235,156 +306,210 @@ __device__ __forceinline__ void process_fp_tile(WarpState<NCB>& st, const uint32
       s0 = fmaf(acc[cb][c][0], kc[c], s0);
       s1 = fmaf(acc[cb][c][2], kc[c], s1);
     }
-    s[cb][0] = n < n_valid ? s0 : -INFINITY;
-    s[cb][1] = n + 8 < n_valid ? s1 : -INFINITY;
+    s[0][cb][0] = n < n_valid ? s0 : -INFINITY;
+    s[0][cb][1] = n + 8 < n_valid ? s1 : -INFINITY;
   }
+  tile_softmax<NCB, 1>(st, s, lane, opaque_zero);
   float pT[2][2];
-  softmax_step<NCB>(st, s, pT, lane);
-  // p split into bf16 hi + lo
-  uint32_t bhi[2], blo[2];
+  transpose_p<NCB>(s[0], pT, lane);
+  // NCB == 1: only b0 (hi/lo by column); NCB == 2: b0 = hi, b1 = lo
+  if (NCB == 1) {
+    uint32_t H[2], Pz[2];
+    split_p_bf16(pT, oddmask, H, b0, Pz);
+    b1[0] = b1[1] = 0;
+  } else {
 #pragma unroll
-  for (int th = 0; th < 2; ++th) {
-    bhi[th] = pack_bf16x2(pT[th][0], pT[th][1]);
-    blo[th] = pack_bf16x2(pT[th][0] - bf16lo_f32(bhi[th]), pT[th][1] - bf16hi_f32(bhi[th]));
-  }
-  {
-    const int mi = lane >> 3, rr = lane & 7;
-    const int token = rr + 8 * (mi >> 1);
-    const uint32_t rowaddr = tile + kFpTileVOffset + token * 256;
-#pragma unroll
-    for (int mt = 0; mt < 8; ++mt) {
-      const int chunk = 2 * mt + (mi & 1);
-      uint32_t a0, a1, a2, a3;
-      ldmatrix_x4_trans(rowaddr + ((chunk ^ (token & 7)) << 4), a0, a1, a2, a3);
-      mma_bf16(st.out[mt], a0, a1, a2, a3, bhi[0], bhi[1]);
-      mma_bf16(st.out[mt], a0, a1, a2, a3, blo[0], blo[1]);
+    for (int th = 0; th < 2; ++th) {
+      b0[th] = pack_bf16x2(pT[th][0], pT[th][1]);
+      b1[th] = pack_bf16x2(pT[th][0] - bf16lo_f32(b0[th]), pT[th][1] - bf16hi_f32(b0[th]));
     }
+  }
+}
+
+template <int NCB>
+__device__ __forceinline__ void process_fp_values(WarpState<NCB>& st, uint32_t vrows, int lane,
+                                                  const uint32_t (&b0)[2], const uint32_t (&b1)[2]) {
+  const int mi = lane >> 3, rr = lane & 7;
+  const int token = rr + 8 * (mi >> 1);
+  const uint32_t rowaddr = vrows + token * 256;
+#pragma unroll
+  for (int mt = 0; mt < 8; ++mt) {
+    const int chunk = 2 * mt + (mi & 1);
+    uint32_t a0, a1, a2, a3;
+    ldmatrix_x4_trans(rowaddr + ((chunk ^ (token & 7)) << 4), a0, a1, a2, a3);
+    mma_bf16(st.out[mt], a0, a1, a2, a3, b0[0], b0[1]);
+    if (NCB != 1) mma_bf16(st.out[mt], a0, a1, a2, a3, b1[0], b1[1]);
   }
 }
 
 // ---- one quant tile: one key group of G tokens ---------------------------------------------
 template <int G, int NCB>
 __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uint32_t (&qs)[NCB][8][2], uint32_t tile,
-                                                   const float (&kc)[4], float kq, int lane) {
+                                                   const float (&kc)[4], float kq, int lane, uint32_t oddmask,
+                                                   int opaque_zero) {
   constexpr int NS = G / 16, NG = kD / G, VS = vsz_subtile_bytes(G);
   const int n = lane >> 2, j = lane & 3;
-  // q*s split into hi (even columns) / lo (odd columns), and the bias q.z of the group
-  uint32_t bq[NCB][8][2];
-  float bias[NCB];
+  // ---- q.k on all G tokens.  Per pair of k-steps: the key scale of the lane's channels is folded
+  // into the query (even columns RN(q*s), odd columns the exact residual), the group's q.zero
+  // bias advances by one MMA per k-step (A = zero rows via ldmatrix with equal row addresses),
+  // and every sub-tile's score accumulator advances by one MMA per k-step.
+  float s[NS][NCB][2];
+#ifdef LQ_EXP_NOQK
+#pragma unroll
+  for (int u = 0; u < NS; ++u)
+#pragma unroll
+    for (int cb = 0; cb < NCB; ++cb) s[u][cb][0] = s[u][cb][1] = static_cast<float>(lane + u) * kq;
+  if (false)
+#endif
   {
+    uint32_t kw[NS][4], kws[NS][4];
+#pragma unroll
+    for (int u = 0; u < NS; ++u) {
+      const uint4 w = lds128(tile + qt_kcodes_off() + u * 512 + 16 * lane);
+      // words: (nt0,w0) (nt0,w1) (nt1,w0) (nt1,w1);  a0=(nt0,w0) a1=(nt1,w0) a2=(nt0,w1) a3=(nt1,w1)
+      kw[u][0] = w.x; kw[u][1] = w.z; kw[u][2] = w.y; kw[u][3] = w.w;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) kws[u][e] = kw[u][e] >> 8;
+    }
+    float acc[NS][NCB][4];
     float accb[NCB][4][4];
 #pragma unroll
-    for (int cb = 0; cb < NCB; ++cb)
+    for (int cb = 0; cb < NCB; ++cb) {
 #pragma unroll
-      for (int c = 0; c < 4; ++c)
+      for (int u = 0; u < NS; ++u) acc[u][cb][0] = acc[u][cb][1] = acc[u][cb][2] = acc[u][cb][3] = 0.f;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) accb[cb][c][e] = 0.f;
-    const bool odd = n & 1;
+      for (int c = 0; c < 4; ++c) accb[cb][c][0] = accb[cb][c][1] = accb[cb][c][2] = accb[cb][c][3] = 0.f;
+    }
+    const uint32_t zaddr = tile + qt_kzero_off() + ((lane >> 4) << 4);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const uint4 sw = lds128(tile + qt_kscale_off() + 16 * (4 * i + j));
-      const uint4 zw = lds128(tile + qt_kzero_off() + 16 * (4 * i + j));
       const uint32_t s4[4] = {sw.x, sw.y, sw.z, sw.w};
-      const uint32_t z4[4] = {zw.x, zw.y, zw.z, zw.w};
 #pragma unroll
       for (int kk = 0; kk < 2; ++kk) {
         const int ks = 2 * i + kk;
+        uint32_t z0, z1, z2, z3;
+        ldmatrix_x4(zaddr + 32 * ks, z0, z1, z2, z3);
+        uint32_t bq[NCB][2];
 #pragma unroll
         for (int cb = 0; cb < NCB; ++cb) {
 #pragma unroll
           for (int w = 0; w < 2; ++w) {
             const uint32_t hi = bf16x2_mul(qs[cb][ks][w], s4[2 * kk + w]);
-            const uint32_t lo = bf16x2_fma(qs[cb][ks][w], s4[2 * kk + w], hi ^ 0x80008000u);
-            bq[cb][ks][w] = odd ? lo : hi;
+            bq[cb][w] = bf16x2_fma(qs[cb][ks][w], s4[2 * kk + w], bf16x2_mul(hi, oddmask & 0xBF80BF80u));
           }
-          mma_bf16(accb[cb][ks & 3], z4[2 * kk], z4[2 * kk], z4[2 * kk + 1], z4[2 * kk + 1], qs[cb][ks][0],
-                   qs[cb][ks][1]);
+          mma_bf16(accb[cb][ks & 3], z0, z1, z2, z3, qs[cb][ks][0], qs[cb][ks][1]);
+        }
+#pragma unroll
+        for (int u = 0; u < NS; ++u) {
+          const uint32_t a0 = ext_bf16_i(ks, kw[u][0], kws[u][0]), a1 = ext_bf16_i(ks, kw[u][1], kws[u][1]),
+                         a2 = ext_bf16_i(ks, kw[u][2], kws[u][2]), a3 = ext_bf16_i(ks, kw[u][3], kws[u][3]);
+#pragma unroll
+          for (int cb = 0; cb < NCB; ++cb) mma_bf16(acc[u][cb], a0, a1, a2, a3, bq[cb][0], bq[cb][1]);
         }
       }
     }
 #pragma unroll
     for (int cb = 0; cb < NCB; ++cb) {
-      float b = accb[cb][0][0] * kc[0];
+      float bias = accb[cb][0][0] * kc[0];
 #pragma unroll
-      for (int c = 1; c < 4; ++c) b = fmaf(accb[cb][c][0], kc[c], b);
-      bias[cb] = b;
+      for (int c = 1; c < 4; ++c) bias = fmaf(accb[cb][c][0], kc[c], bias);
+#pragma unroll
+      for (int u = 0; u < NS; ++u) {
+        s[u][cb][0] = fmaf(acc[u][cb][0] + acc[u][cb][1], kq, bias);
+        s[u][cb][1] = fmaf(acc[u][cb][2] + acc[u][cb][3], kq, bias);
+      }
     }
   }
+#ifndef LQ_EXP_NOSOFTMAX
+  tile_softmax<NCB, NS>(st, s, lane, opaque_zero);
+#endif
+#ifdef LQ_EXP_NOPV
+  st.l[0] += s[0][0][0] + s[NS - 1][0][1];
+  return;
+#endif
 
-#pragma unroll 1
+#pragma unroll
   for (int u = 0; u < NS; ++u) {
-    // ---- q.k on 16 tokens ----
-    float s[NCB][2];
-    {
-      const uint4 kw = lds128(tile + qt_kcodes_off() + u * 512 + 16 * lane);
-      // words: (nt0,w0) (nt0,w1) (nt1,w0) (nt1,w1);  a0=(nt0,w0) a1=(nt1,w0) a2=(nt0,w1) a3=(nt1,w1)
-      const uint32_t w0 = kw.x, w1 = kw.z, w2 = kw.y, w3 = kw.w;
-      const uint32_t w0s = w0 >> 8, w1s = w1 >> 8, w2s = w2 >> 8, w3s = w3 >> 8;
-      float acc[NCB][4];
-#pragma unroll
-      for (int cb = 0; cb < NCB; ++cb) acc[cb][0] = acc[cb][1] = acc[cb][2] = acc[cb][3] = 0.f;
-#define LQ_QK_STEP(KS)                                                                           \
-  {                                                                                              \
-    const uint32_t a0 = kext<KS>(w0, w0s), a1 = kext<KS>(w1, w1s), a2 = kext<KS>(w2, w2s),       \
-                   a3 = kext<KS>(w3, w3s);                                                       \
-    _Pragma("unroll") for (int cb = 0; cb < NCB; ++cb)                                           \
-        mma_bf16(acc[cb], a0, a1, a2, a3, bq[cb][KS][0], bq[cb][KS][1]);                         \
-  }
-      LQ_QK_STEP(0) LQ_QK_STEP(1) LQ_QK_STEP(2) LQ_QK_STEP(3)
-      LQ_QK_STEP(4) LQ_QK_STEP(5) LQ_QK_STEP(6) LQ_QK_STEP(7)
-#undef LQ_QK_STEP
-#pragma unroll
-      for (int cb = 0; cb < NCB; ++cb) {
-        s[cb][0] = fmaf(acc[cb][0] + acc[cb][1], kq, bias[cb]);
-        s[cb][1] = fmaf(acc[cb][2] + acc[cb][3], kq, bias[cb]);
-      }
-    }
     float pT[2][2];
-    softmax_step<NCB>(st, s, pT, lane);
-
-    // ---- value zero: one MMA, A = zero (fp16) with value groups on rows ----
-    {
-      uint32_t z0 = 0, z1 = 0;
-      if (n < NG) {
-        const uint2 zw = lds64(tile + qt_vzero_off(G) + u * VS + 8 * (4 * n + j));
-        z0 = pack_f16x2(bf16lo_f32(zw.x), bf16hi_f32(zw.x));
-        z1 = pack_f16x2(bf16lo_f32(zw.y), bf16hi_f32(zw.y));
+    transpose_p<NCB>(s[u], pT, lane);
+    const uint4 vw = lds128(tile + qt_vcodes_off(G) + u * 512 + 16 * lane);
+    if (NCB == 1) {
+      uint32_t H[2], P[2], Pz[2];
+      split_p_bf16(pT, oddmask, H, P, Pz);
+      // value zero: A = zero (bf16 pairs straight from the tile), value groups on rows
+      {
+        uint2 zw = make_uint2(0u, 0u);
+        if (n < NG) zw = lds64(tile + qt_vzero_off(G) + u * VS + 8 * (4 * n + j));
+        mma_bf16(st.zacc, zw.x, 0u, zw.y, 0u, P[0], P[1]);
       }
-      mma_f16(st.zacc, z0, 0u, z1, 0u, pack_f16x2(pT[0][0], pT[0][1]), pack_f16x2(pT[1][0], pT[1][1]));
-    }
-    // ---- p * value scale per value group, fp16 ----
-    uint32_t bp[NG][2];
-    if (NG == 4) {
+      // p * value scale per value group: even columns RN(hi*s), odd columns lo*s + residual
+      uint32_t bp[NG][2];
+      uint32_t sv[NG][2];
+      if (NG == 4) {
+        const uint4 s0 = lds128(tile + qt_vscale_off(G) + u * VS + 16 * j);
+        const uint4 s1 = lds128(tile + qt_vscale_off(G) + u * VS + 16 * (4 + j));
+        sv[0][0] = s0.x; sv[0][1] = s0.y; sv[1][0] = s0.z; sv[1][1] = s0.w;
+        sv[2 % NG][0] = s1.x; sv[2 % NG][1] = s1.y; sv[3 % NG][0] = s1.z; sv[3 % NG][1] = s1.w;
+      } else {
+        const uint4 s0 = lds128(tile + qt_vscale_off(G) + u * VS + 16 * j);
+        sv[0][0] = s0.x; sv[0][1] = s0.y; sv[1 % NG][0] = s0.z; sv[1 % NG][1] = s0.w;
+      }
 #pragma unroll
-      for (int i = 0; i < 2; ++i) {
-        const uint4 sv = lds128(tile + qt_vscale_off(G) + u * VS + 16 * (4 * i + j));
-        const uint32_t w4[4] = {sv.x, sv.y, sv.z, sv.w};
+      for (int g = 0; g < NG; ++g)
+#pragma unroll
+        for (int th = 0; th < 2; ++th) {
+          const uint32_t hh = bf16x2_mul(H[th], sv[g][th]);
+          const uint32_t r1 = bf16x2_fma(H[th], sv[g][th], bf16x2_mul(hh, oddmask & 0xBF80BF80u));
+          bp[g][th] = bf16x2_fma(Pz[th], sv[g][th], r1);
+        }
+      const uint32_t v0s = vw.x >> 8, v1s = vw.y >> 8, v2s = vw.z >> 8, v3s = vw.w >> 8;
+#define LQ_PV_STEP(MT)                                                                                        \
+  mma_bf16(st.out[MT], ext_bf16<MT>(vw.x, v0s), ext_bf16<MT>(vw.y, v1s), ext_bf16<MT>(vw.z, v2s),             \
+           ext_bf16<MT>(vw.w, v3s), bp[((MT) * 16) / G][0], bp[((MT) * 16) / G][1]);
+      LQ_PV_STEP(0) LQ_PV_STEP(1) LQ_PV_STEP(2) LQ_PV_STEP(3)
+      LQ_PV_STEP(4) LQ_PV_STEP(5) LQ_PV_STEP(6) LQ_PV_STEP(7)
+#undef LQ_PV_STEP
+    } else {
+      // value zero: A = zero converted to fp16, value groups on rows
+      {
+        uint32_t z0 = 0, z1 = 0;
+        if (n < NG) {
+          const uint2 zw = lds64(tile + qt_vzero_off(G) + u * VS + 8 * (4 * n + j));
+          z0 = pack_f16x2(bf16lo_f32(zw.x), bf16hi_f32(zw.x));
+          z1 = pack_f16x2(bf16lo_f32(zw.y), bf16hi_f32(zw.y));
+        }
+        mma_f16(st.zacc, z0, 0u, z1, 0u, pack_f16x2(pT[0][0], pT[0][1]), pack_f16x2(pT[1][0], pT[1][1]));
+      }
+      uint32_t bp[NG][2];
+      if (NG == 4) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const uint4 svw = lds128(tile + qt_vscale_off(G) + u * VS + 16 * (4 * i + j));
+          const uint32_t w4[4] = {svw.x, svw.y, svw.z, svw.w};
+#pragma unroll
+          for (int gg = 0; gg < 2; ++gg)
+#pragma unroll
+            for (int th = 0; th < 2; ++th) {
+              const uint32_t w = w4[2 * gg + th];
+              bp[(2 * i + gg) % NG][th] = pack_f16x2(pT[th][0] * bf16lo_f32(w), pT[th][1] * bf16hi_f32(w));
+            }
+        }
+      } else {
+        const uint4 svw = lds128(tile + qt_vscale_off(G) + u * VS + 16 * j);
+        const uint32_t w4[4] = {svw.x, svw.y, svw.z, svw.w};
 #pragma unroll
         for (int gg = 0; gg < 2; ++gg)
 #pragma unroll
           for (int th = 0; th < 2; ++th) {
             const uint32_t w = w4[2 * gg + th];
-            bp[(2 * i + gg) % NG][th] = pack_f16x2(pT[th][0] * bf16lo_f32(w), pT[th][1] * bf16hi_f32(w));
+            bp[gg % NG][th] = pack_f16x2(pT[th][0] * bf16lo_f32(w), pT[th][1] * bf16hi_f32(w));
           }
       }
-    } else {
-      const uint4 sv = lds128(tile + qt_vscale_off(G) + u * VS + 16 * j);
-      const uint32_t w4[4] = {sv.x, sv.y, sv.z, sv.w};
-#pragma unroll
-      for (int gg = 0; gg < 2; ++gg)
-#pragma unroll
-        for (int th = 0; th < 2; ++th) {
-          const uint32_t w = w4[2 * gg + th];
-          bp[gg % NG][th] = pack_f16x2(pT[th][0] * bf16lo_f32(w), pT[th][1] * bf16hi_f32(w));
-        }
-    }
-    // ---- p.v on 16 tokens ----
-    {
-      const uint4 vw = lds128(tile + qt_vcodes_off(G) + u * 512 + 16 * lane);
       const uint32_t v0s = vw.x >> 10, v1s = vw.y >> 10, v2s = vw.z >> 10, v3s = vw.w >> 10;
-#define LQ_PV_STEP(MT)                                                                              \
-  mma_f16(st.out[MT], vext<MT>(vw.x, v0s), vext<MT>(vw.y, v1s), vext<MT>(vw.z, v2s), vext<MT>(vw.w, v3s), \
-          bp[((MT) * 16) / G][0], bp[((MT) * 16) / G][1]);
+#define LQ_PV_STEP(MT)                                                                                        \
+  mma_f16(st.out[MT], ext_f16<MT>(vw.x, v0s), ext_f16<MT>(vw.y, v1s), ext_f16<MT>(vw.z, v2s),                 \
+          ext_f16<MT>(vw.w, v3s), bp[((MT) * 16) / G][0], bp[((MT) * 16) / G][1]);
       LQ_PV_STEP(0) LQ_PV_STEP(1) LQ_PV_STEP(2) LQ_PV_STEP(3)
       LQ_PV_STEP(4) LQ_PV_STEP(5) LQ_PV_STEP(6) LQ_PV_STEP(7)
 #undef LQ_PV_STEP
@@ -392,98 +517,161 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
   }
 }
 
-struct MmaSplitPlan {
-  int units_fp;      // fp tiles per (b, kv)
-  int units_quant;   // quant units per (b, kv)
-  int tiles_quant;   // quant tiles per (b, kv)
-  int tiles_per_unit;
-};
+// shared memory: [per-warp stages][query rows of the pair][mbarriers][flags]
+constexpr int kSmemStages = kWarps * kStages * kStageBytes;
+constexpr int kSmemQ = kMaxRatio * kD * 2;
+constexpr int kSmemBars = (kWarps * kStages + 1) * 8;
+constexpr int kSmemBytes = kSmemStages + kSmemQ + kSmemBars + 16;
+constexpr int kMergeMax = 2048;  // S * r records the fused second pass can stage
 
+// Work items of one (b, kv) pair, in queue order: fp tiles [0, tiles_fp), then quant tiles.  The S
+// CTAs of the pair (4 warps each) pull items one at a time from a global counter, so every warp of
+// every SM stays busy until the pair is finished whatever the speed of its SM; any assignment is
+// legal because every warp keeps its own online-softmax state.  A warp always has its next claim
+// in flight (the atomic's latency hides behind the tile being processed) and two loads in flight.
 template <int G, int NCB>
-__global__ void __launch_bounds__(kWarps * 32, 3) lq_decode_mma_kernel(DecodeArgs a, MmaSplitPlan plan) {
+__global__ void __launch_bounds__(kWarps * 32, kCtasPerSm) lq_decode_mma_kernel(DecodeArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   const CacheView& cv = a.cv;
   const int r = cv.Hq / cv.Hkv;
-  const int S = a.S;
-  const int64_t pair = blockIdx.x / S;
-  const int split = blockIdx.x % S;
-  const int b = static_cast<int>(pair / cv.Hkv), kv = static_cast<int>(pair % cv.Hkv);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n = lane >> 2, j = lane & 3;
+  const uint32_t oddmask = (n & 1) ? 0xFFFFFFFFu : 0u;
   constexpr int TILE = quant_tile_bytes(G);
+  static_assert(TILE <= kStageBytes && kFpTileVOffset <= kStageBytes, "stage too small");
 
-  uint8_t* my_stages = smem + warp * (kStages * kStageBytes);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kWarps * kStages * kStageBytes) + warp * kStages;
-  const uint32_t stage0 = smem_u32(my_stages);
-  const uint32_t bar0 = smem_u32(bars);
+  const int pair = blockIdx.x / a.S, slot = blockIdx.x % a.S;
+  const int b = pair / cv.Hkv, kv = pair % cv.Hkv;
+  const int n_items = a.tiles_fp + a.tiles_quant;
+  int* queue = a.tickets + 2 * pair;
 
+  const uint32_t stage0 = smem_u32(smem + warp * (kStages * kStageBytes));
+  const uint32_t qsm = smem_u32(smem + kSmemStages);
+  const uint32_t bar0 = smem_u32(smem + kSmemStages + kSmemQ) + warp * kStages * 8;
+  const uint32_t qbar = smem_u32(smem + kSmemStages + kSmemQ) + kWarps * kStages * 8;
+  int* is_last = reinterpret_cast<int*>(smem + kSmemStages + kSmemQ + kSmemBars);
+
+  // Programmatic dependent launch: let the next kernel of the stream start launching, and do
+  // not touch anything an earlier kernel may still be writing before it has finished.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+
+  // claims: the first kStages items of every warp are fixed (item = warp index + i * #warps), the
+  // rest come from the pair's counter; lane 0 keeps the next dynamic claim in `pref`, an atomicAdd
+  // issued one step ahead so that its latency hides behind the tile being processed
+  const int n_warps = a.S * kWarps, gw = slot * kWarps + warp;
+  int pref = 0;
   if (lane == 0) {
+    pref = atomicAdd(queue, 1) + kStages * n_warps;
 #pragma unroll
     for (int s = 0; s < kStages; ++s) mbar_init(bar0 + 8 * s, 1);
+    if (warp == 0) mbar_init(qbar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  __syncwarp();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    // the r query rows of this pair are contiguous: one bulk copy
+    mbar_expect_tx(qbar, r * kD * 2);
+    bulk_load(qsm, static_cast<const uint8_t*>(a.q) + (static_cast<int64_t>(b) * cv.Hq + kv * r) * kD * 2, r * kD * 2,
+              qbar);
+  }
 
-  // this warp's unit range
-  const int U = plan.units_fp + plan.units_quant;
-  const int NW = S * kWarps, wi = split * kWarps + warp;
-  const int begin = static_cast<int>(static_cast<int64_t>(U) * wi / NW);
-  const int end = static_cast<int>(static_cast<int64_t>(U) * (wi + 1) / NW);
-  const int n_my = end - begin;
+#ifdef LQ_EXP_TRACE
+  unsigned long long tr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  unsigned long long gt0;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt0));
+  tr[0] = clock64();
+#define TR(i) tr[i] = clock64()
+#define TRACC(i, t) tr[i] += clock64() - (t)
+#else
+#define TR(i)
+#define TRACC(i, t)
+#endif
+  float kc[4];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) kc[c] = a.scale_log2 * pow2i(2 * c - 64);
+  const float kq = a.scale_log2 * pow2i(69);
 
   const uint8_t* fpbase = cv.fp + a.layer * cv.fp_layer_stride + pair * cv.fp_head_stride;
   const uint8_t* qbase = cv.quant + a.layer * cv.quant_layer_stride + pair * cv.quant_head_stride;
 
-  auto unit_src = [&](int unit, uint32_t& bytes) -> const uint8_t* {
-    if (unit < plan.units_fp) {
-      bytes = kFpTileBytes;
-      return fpbase + static_cast<int64_t>(unit) * kFpTileBytes;
+  // load pipeline.  A stage holds: the K rows of fp tile i (desc = i), its V rows (desc = -1-i)
+  // or quant tile t (desc = tiles_fp + t).  pending_v >= 0: the V rows of that fp tile come next.
+  int issued = 0, pending_v = -1, n_claims = 0;
+  bool drained = false;
+  int desc0 = 0, desc1 = 0;
+  auto issue_next = [&]() {
+    const uint8_t* src;
+    uint32_t bytes;
+    int desc;
+    if (pending_v >= 0) {
+      desc = -1 - pending_v;
+      bytes = kFpTileVOffset;
+      src = fpbase + static_cast<int64_t>(pending_v) * kFpTileBytes + kFpTileVOffset;
+      pending_v = -1;
+    } else {
+      if (drained) return;
+      int item;
+      if (n_claims < kStages) {
+        item = gw + n_claims * n_warps;
+      } else {
+        item = __shfl_sync(kFull, pref, 0);
+        if (item < n_items && lane == 0) pref = atomicAdd(queue, 1) + kStages * n_warps;
+      }
+      ++n_claims;
+      if (item >= n_items) { drained = true; return; }
+      desc = item;
+      if (item < a.tiles_fp) {
+        bytes = kFpTileVOffset;
+        src = fpbase + static_cast<int64_t>(item) * kFpTileBytes;
+        pending_v = item;
+      } else {
+        bytes = TILE;
+        src = qbase + static_cast<int64_t>(item - a.tiles_fp) * TILE;
+      }
     }
-    const int uq = unit - plan.units_fp;
-    const int t0 = uq * plan.tiles_per_unit;
-    const int nt = min(plan.tiles_per_unit, plan.tiles_quant - t0);
-    bytes = nt * TILE;
-    return qbase + static_cast<int64_t>(t0) * TILE;
-  };
-  auto issue = [&](int k) {
+    const uint32_t s = issued % kStages;
+    if (s == 0) desc0 = desc; else desc1 = desc;
     if (lane == 0) {
-      uint32_t bytes;
-      const uint8_t* src = unit_src(begin + k, bytes);
-      const int s = k % kStages;
       mbar_expect_tx(bar0 + 8 * s, bytes);
       bulk_load(stage0 + s * kStageBytes, src, bytes, bar0 + 8 * s);
     }
+    ++issued;
   };
+  bool failed = false;
+#ifndef LQ_EXP_NOLOAD
 #pragma unroll
-  for (int k = 0; k < kStages; ++k)
-    if (k < n_my) issue(k);
+  for (int s = 0; s < kStages; ++s) issue_next();
+#endif
+  TR(7);
 
   // query fragments: B operand, column n -> head 4cb + n/2 (even column = hi, odd = lo of q*s);
   // k-step ks carries the factor 2^(64 - 2*(ks&3)) that cancels the code-position factor
   uint32_t qs[NCB][8][2];
   {
-    const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(a.q);
+    int spins = 0;
+    while (!mbar_try_wait(qbar, 0)) {
+      if (++spins > kSpinLimit) { failed = true; break; }
+    }
+    failed = __any_sync(kFull, failed);
 #pragma unroll
     for (int cb = 0; cb < NCB; ++cb) {
       const int head = 4 * cb + (n >> 1);
       const bool valid = head < r;
-      const __nv_bfloat16* qrow = q + (static_cast<int64_t>(b) * cv.Hq + kv * r + (valid ? head : 0)) * kD;
+      const uint32_t qrow = qsm + (valid ? head : 0) * (kD * 2);
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks)
 #pragma unroll
         for (int w = 0; w < 2; ++w) {
-          const uint32_t raw = *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8 * w + 2 * j);
-          const float f = exp2f(static_cast<float>(64 - 2 * (ks & 3)));
+          uint32_t raw;
+          asm volatile("ld.shared.u32 %0, [%1];" : "=r"(raw) : "r"(qrow + 2 * (16 * ks + 8 * w + 2 * j)));
+          const float f = pow2i(64 - 2 * (ks & 3));
           qs[cb][ks][w] = valid ? pack_bf16x2(bf16lo_f32(raw) * f, bf16hi_f32(raw) * f) : 0u;
         }
     }
   }
-  float kc[4];
-#pragma unroll
-  for (int c = 0; c < 4; ++c) kc[c] = a.scale_log2 * exp2f(static_cast<float>(2 * c - 64));
-  const float kq = a.scale_log2 * exp2f(69.f);
-
+  TR(1);
   WarpState<NCB> st;
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) st.out[mt][0] = st.out[mt][1] = st.out[mt][2] = st.out[mt][3] = 0.f;
@@ -492,82 +680,107 @@ __global__ void __launch_bounds__(kWarps * 32, 3) lq_decode_mma_kernel(DecodeArg
   for (int cb = 0; cb < NCB; ++cb) { st.m[cb] = -INFINITY; st.l[cb] = 0.f; }
   st.quant_mode = false;
 
-  bool failed = false;
+  uint32_t fb0[2] = {0u, 0u}, fb1[2] = {0u, 0u};  // p.v B operands of the fp tile whose V rows are still to come
 #pragma unroll 1
-  for (int k = 0; k < n_my; ++k) {
-    const int s = k % kStages;
-    const uint32_t parity = (k / kStages) & 1;
-    int spins = 0;
-    while (!mbar_try_wait(bar0 + 8 * s, parity)) {
-      if (++spins > kSpinLimit) { failed = true; break; }
+  for (int done = 0; done < issued && !failed; ++done) {
+    const uint32_t s = done % kStages;
+    const uint32_t parity = (done / kStages) & 1;
+    {
+      int spins = 0;
+      bool bad = false;
+#ifdef LQ_EXP_TRACE
+      const unsigned long long tw = clock64();
+#endif
+      while (!mbar_try_wait(bar0 + 8 * s, parity)) {
+        if (++spins > kSpinLimit) { bad = true; break; }
+      }
+      TRACC(6, tw);
+      if (__any_sync(kFull, bad)) { failed = true; break; }
     }
-    if (__any_sync(kFull, failed)) break;
-    const int unit = begin + k;
     const uint32_t sbase = stage0 + s * kStageBytes;
-    if (unit < plan.units_fp) {
-      const int nv = min(16, a.n_fp - unit * 16);
-      process_fp_tile<NCB>(st, qs, sbase, nv, kc, lane);
-    } else {
-      if (!st.quant_mode) {
+    const int desc = s == 0 ? desc0 : desc1;
+    if (desc >= a.tiles_fp) {
+      // items come in queue order, so a warp sees all its fp tiles before its first quant tile: from
+      // here on the out rows carry the code-position factor (two steps keep the constants normal).
+      // An opaque one-trip loop keeps this a branch instead of 64 multiplies and selects per tile.
+      int sw = st.quant_mode ? 0 : 1;
+      while (sw) {
 #pragma unroll
         for (int mt = 0; mt < 8; ++mt) {
-          const float f = vpos_scale(mt);
-          st.out[mt][0] *= f; st.out[mt][1] *= f; st.out[mt][2] *= f; st.out[mt][3] *= f;
+          const float f = pow2i(vpos_log2<NCB>(mt) + 70);
+          st.out[mt][0] = st.out[mt][0] * 0x1p-70f * f; st.out[mt][1] = st.out[mt][1] * 0x1p-70f * f;
+          st.out[mt][2] = st.out[mt][2] * 0x1p-70f * f; st.out[mt][3] = st.out[mt][3] * 0x1p-70f * f;
         }
         st.quant_mode = true;
+        sw = a.zero;
       }
-      const int uq = unit - plan.units_fp;
-      const int nt = min(plan.tiles_per_unit, plan.tiles_quant - uq * plan.tiles_per_unit);
-#pragma unroll 1
-      for (int t = 0; t < nt; ++t) process_quant_tile<G, NCB>(st, qs, sbase + t * TILE, kc, kq, lane);
+#ifndef LQ_EXP_LOADONLY
+      process_quant_tile<G, NCB>(st, qs, sbase, kc, kq, lane, oddmask, a.zero);
+#endif
+    } else if (desc >= 0) {
+      const int nv = min(16, a.n_fp - desc * 16);
+      process_fp_keys<NCB>(st, qs, sbase, nv, kc, lane, oddmask, a.zero, fb0, fb1);
+    } else {
+      process_fp_values<NCB>(st, sbase, lane, fb0, fb1);
     }
     __syncwarp();
-    if (k + kStages < n_my) issue(k + kStages);
+    issue_next();
   }
+  TR(3);
+  if (lane == 0 && pref < 0) atomicOr(a.status, 2);  // never true; makes sure the last claim has returned
   if (failed) {
-    // a bulk copy never completed: flag it, give the copies in flight a bounded chance to land
-    // before this CTA's shared memory is released, and contribute nothing
+    // a bulk copy never completed: flag it and contribute nothing (checked again at the end)
     if (lane == 0) atomicOr(a.status, 1);
-    for (int s = 0; s < kStages; ++s) {
-      int spins = 0;
-      while (!mbar_try_wait(bar0 + 8 * s, 0) && !mbar_try_wait(bar0 + 8 * s, 1) && ++spins < 1024) {}
-    }
 #pragma unroll
     for (int cb = 0; cb < NCB; ++cb) { st.m[cb] = -INFINITY; st.l[cb] = 0.f; }
   }
 
   // ---- fold zero term, undo position factors, reduce l over the token lanes ----
-  constexpr int NG = kD / G;
+  constexpr float kPInv = NCB == 1 ? 0x1p-64f : 1.0f;
+  float o0[8], o1[8];  // NCB == 1: rows (n, n+8) of head j; NCB == 2: unused
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) {
     const int g = (mt * 16) / G;
-    const float z0 = __shfl_sync(kFull, st.zacc[0], 4 * g + j), z1 = __shfl_sync(kFull, st.zacc[1], 4 * g + j);
-    const float f = st.quant_mode ? 1.0f / vpos_scale(mt) : 1.0f;
-    st.out[mt][0] = fmaf(st.out[mt][0], f, z0);
-    st.out[mt][1] = fmaf(st.out[mt][1], f, z1);
-    st.out[mt][2] = fmaf(st.out[mt][2], f, z0);
-    st.out[mt][3] = fmaf(st.out[mt][3], f, z1);
+    // quant mode: out = true * 2^(kPExp + vpos); fp mode: out = true * 2^kPExp
+    const float f = st.quant_mode ? pow2i(-vpos_log2<NCB>(mt) - 70) * (NCB == 1 ? 0x1p6f : 0x1p70f) : kPInv;
+    if (NCB == 1) {
+      const float z = __shfl_sync(kFull, st.zacc[0] + st.zacc[1], 4 * g + j) * kPInv;
+      o0[mt] = fmaf(st.out[mt][0] + st.out[mt][1], f, z);
+      o1[mt] = fmaf(st.out[mt][2] + st.out[mt][3], f, z);
+    } else {
+      const float z0 = __shfl_sync(kFull, st.zacc[0], 4 * g + j), z1 = __shfl_sync(kFull, st.zacc[1], 4 * g + j);
+      st.out[mt][0] = fmaf(st.out[mt][0], f, z0);
+      st.out[mt][1] = fmaf(st.out[mt][1], f, z1);
+      st.out[mt][2] = fmaf(st.out[mt][2], f, z0);
+      st.out[mt][3] = fmaf(st.out[mt][3], f, z1);
+    }
   }
-  (void)NG;
 #pragma unroll
   for (int cb = 0; cb < NCB; ++cb) {
     st.l[cb] += __shfl_xor_sync(kFull, st.l[cb], 4);
     st.l[cb] += __shfl_xor_sync(kFull, st.l[cb], 8);
     st.l[cb] += __shfl_xor_sync(kFull, st.l[cb], 16);
+    st.l[cb] *= kPInv;
   }
 
-  // ---- CTA merge of the 4 warp states through shared memory (stages are idle now) ----
+  // ---- CTA merge of the 4 warp states through shared memory (the stages are idle now) ----
   __syncthreads();
-  float* wout = reinterpret_cast<float*>(smem);                 // [warp][d][8]
-  float* wm = wout + kWarps * kD * 8;                           // [warp][8]
-  float* wl = wm + kWarps * 8;                                  // [warp][8]
+  float* wout = reinterpret_cast<float*>(smem);  // [warp][d][8]
+  float* wm = wout + kWarps * kD * 8;            // [warp][8]
+  float* wl = wm + kWarps * 8;                   // [warp][8]
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) {
-    float* o = wout + (warp * kD + 16 * mt + n) * 8 + 2 * j;
-    o[0] = st.out[mt][0];
-    o[1] = st.out[mt][1];
-    o[64] = st.out[mt][2];  // row + 8
-    o[65] = st.out[mt][3];
+    if (NCB == 1) {
+      float* o = wout + (warp * kD + 16 * mt + n) * 8 + j;
+      o[0] = o0[mt];
+      o[64] = o1[mt];  // row + 8
+    } else {
+      float* o = wout + (warp * kD + 16 * mt + n) * 8 + 2 * j;
+      o[0] = st.out[mt][0];
+      o[1] = st.out[mt][1];
+      o[64] = st.out[mt][2];
+      o[65] = st.out[mt][3];
+    }
   }
   if (n == 0) {
 #pragma unroll
@@ -578,63 +791,156 @@ __global__ void __launch_bounds__(kWarps * 32, 3) lq_decode_mma_kernel(DecodeArg
   }
   __syncthreads();
   const int d = threadIdx.x;
-  const int64_t rec = (pair * S + split) * r;
-  for (int h = 0; h < r; ++h) {
-    float M = -INFINITY;
+  const int64_t rec0 = static_cast<int64_t>(pair) * a.S * r;
+  {
+    const int64_t rec = rec0 + static_cast<int64_t>(slot) * r;
+    for (int h = 0; h < r; ++h) {
+      float M = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w)
-      if (wl[w * 8 + h] > 0.f) M = fmaxf(M, wm[w * 8 + h]);
-    float o = 0.f, L = 0.f;
+      for (int w = 0; w < kWarps; ++w)
+        if (wl[w * 8 + h] > 0.f) M = fmaxf(M, wm[w * 8 + h]);
+      float o = 0.f, L = 0.f;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w)
-      if (wl[w * 8 + h] > 0.f) {
-        const float f = exp2f(wm[w * 8 + h] - M);
-        o = fmaf(wout[(w * kD + d) * 8 + h], f, o);
-        L = fmaf(wl[w * 8 + h], f, L);
+      for (int w = 0; w < kWarps; ++w)
+        if (wl[w * 8 + h] > 0.f) {
+          const float f = exp2f(wm[w * 8 + h] - M);
+          o = fmaf(wout[(w * kD + d) * 8 + h], f, o);
+          L = fmaf(wl[w * 8 + h], f, L);
+        }
+      a.part_o[(rec + h) * kD + d] = o;
+      if (d == 0) {
+        a.part_ml[(rec + h) * 2 + 0] = M;
+        a.part_ml[(rec + h) * 2 + 1] = L;
       }
-    a.part_o[(rec + h) * kD + d] = o;
-    if (d == 0) {
-      a.part_ml[(rec + h) * 2 + 0] = M;
-      a.part_ml[(rec + h) * 2 + 1] = L;
+    }
+  }
+  TR(2);
+  // ---- second pass, fused: the CTA that completes a pair (last ticket) merges its S partials.
+  // Nobody waits for anybody: a CTA either finds that it is last, or leaves.
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int last = atomicAdd(queue + 1, 1) == a.S - 1;
+    if (last) { queue[0] = 0; queue[1] = 0; }  // every claim of every CTA has returned: ready for the next launch
+    *is_last = last;
+  }
+  __syncthreads();
+  if (*is_last) {
+    __threadfence();
+    // weights first (S*r small records, staged in the idle stage memory) ...
+    float* sm_m = reinterpret_cast<float*>(smem);
+    float* sm_l = sm_m + kMergeMax;
+    float* sm_w = sm_l + kMergeMax;
+    float* red = sm_w + kMergeMax;  // [warp][r][128] partial sums
+    const int nrec = a.S * r;
+    for (int t = threadIdx.x; t < nrec; t += kWarps * 32) {
+      sm_m[t] = __ldcg(a.part_ml + (rec0 + t) * 2);
+      sm_l[t] = __ldcg(a.part_ml + (rec0 + t) * 2 + 1);
+    }
+    __syncthreads();
+    if (threadIdx.x < r) {
+      const int h = threadIdx.x;
+      float M = -INFINITY, L = 0.f;
+      for (int s = 0; s < a.S; ++s)
+        if (sm_l[s * r + h] > 0.f) M = fmaxf(M, sm_m[s * r + h]);
+      for (int s = 0; s < a.S; ++s)
+        if (sm_l[s * r + h] > 0.f) L = fmaf(sm_l[s * r + h], exp2f(sm_m[s * r + h] - M), L);
+      const float inv = 1.0f / L;
+      for (int s = 0; s < a.S; ++s)
+        sm_w[s * r + h] = sm_l[s * r + h] > 0.f ? exp2f(sm_m[s * r + h] - M) * inv : 0.f;
+    }
+    __syncthreads();
+    // ... then warp w sums the records s = w, w+4, ... with 16-byte loads (lane = 4 channels), all
+    // independent, and the four warp sums meet in shared memory
+    for (int h = 0; h < r; ++h) {
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int s = warp; s < a.S; s += kWarps) {
+        const float4 v = __ldcg(reinterpret_cast<const float4*>(a.part_o + (rec0 + s * r + h) * kD) + lane);
+        const float w = sm_w[s * r + h];
+        acc.x = fmaf(v.x, w, acc.x); acc.y = fmaf(v.y, w, acc.y);
+        acc.z = fmaf(v.z, w, acc.z); acc.w = fmaf(v.w, w, acc.w);
+      }
+      reinterpret_cast<float4*>(red + (warp * r + h) * kD)[lane] = acc;
+    }
+    __syncthreads();
+    for (int h = 0; h < r; ++h) {
+      float o = 0.f;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) o += red[(w * r + h) * kD + d];
+      const int64_t oi = (static_cast<int64_t>(b) * cv.Hq + kv * r + h) * kD + d;
+      if (a.out_bf16)
+        static_cast<__nv_bfloat16*>(a.out)[oi] = __float2bfloat16_rn(o);
+      else
+        static_cast<float*>(a.out)[oi] = o;
+    }
+  }
+  TR(4);
+#ifdef LQ_EXP_TRACE
+  if (lane == 0) {
+    unsigned long long gt1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt1));
+    unsigned long long* dst = reinterpret_cast<unsigned long long*>(a.status + 64) + (static_cast<size_t>(blockIdx.x) * kWarps + warp) * 10;
+    for (int i = 0; i < 8; ++i) dst[i] = tr[i];
+    dst[8] = gt0; dst[9] = gt1;
+  }
+#endif
+  if (failed) {
+    // give copies still in flight a bounded chance to land before the shared memory is released
+    for (int s = 0; s < kStages; ++s) {
+      int spins = 0;
+      while (!mbar_try_wait(bar0 + 8 * s, 0) && !mbar_try_wait(bar0 + 8 * s, 1) && ++spins < 1024) {}
     }
   }
 }
 
-MmaSplitPlan make_plan(const CacheView& cv, int n_fp, int64_t n_quant) {
-  MmaSplitPlan p;
-  p.units_fp = (n_fp + kFpTileSlots - 1) / kFpTileSlots;
-  p.tiles_quant = static_cast<int>(n_quant / cv.G);
-  p.tiles_per_unit = kStageBytes / quant_tile_bytes(cv.G);
-  p.units_quant = (p.tiles_quant + p.tiles_per_unit - 1) / p.tiles_per_unit;
-  return p;
-}
-
-constexpr int kSmemBytes = kWarps * kStages * kStageBytes + kWarps * kStages * 8;
-
 }  // namespace
 
-int decode_mma_max_splits(const CacheView& cv, int n_fp, int64_t n_quant, int sm_count) {
-  const MmaSplitPlan p = make_plan(cv, n_fp, n_quant);
-  const int pairs = cv.B * cv.Hkv;
-  const int U = p.units_fp + p.units_quant;
-  int S = (3 * sm_count) / pairs;
-  S = S < (U + kWarps - 1) / kWarps ? S : (U + kWarps - 1) / kWarps;
-  return S < 1 ? 1 : S;
+void plan_decode_mma(DecodeArgs& a, int sm_count, int max_records, int s_override) {
+  const int pairs = a.cv.B * a.cv.Hkv;
+  const int r = a.cv.Hq / a.cv.Hkv;
+  a.tiles_fp = (a.n_fp + kFpTileSlots - 1) / kFpTileSlots;
+  a.tiles_quant = static_cast<int>(a.n_quant / a.cv.G);
+  const int items = a.tiles_fp + a.tiles_quant;
+  // about one resident wave of CTAs in total; work is pulled from per-pair queues, so a few CTAs
+  // more or less than a wave cost nothing
+  int S = s_override > 0 ? s_override : (kCtasPerSm * sm_count + pairs / 2) / pairs;
+  S = std::min(S, (items + kWarps - 1) / kWarps);  // at least one item per warp
+  S = std::min(S, max_records);
+  S = std::min(S, kMergeMax / r);
+  a.S = std::max(S, 1);
 }
 
 cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
-  const MmaSplitPlan plan = make_plan(a.cv, a.n_fp, a.n_quant);
   const int r = a.cv.Hq / a.cv.Hkv;
-  const int blocks = a.cv.B * a.cv.Hkv * a.S;
-  void (*kern)(DecodeArgs, MmaSplitPlan) = nullptr;
+  void (*kern)(DecodeArgs) = nullptr;
   if (a.cv.G == 32) kern = r <= 4 ? lq_decode_mma_kernel<32, 1> : lq_decode_mma_kernel<32, 2>;
   else if (a.cv.G == 64) kern = r <= 4 ? lq_decode_mma_kernel<64, 1> : lq_decode_mma_kernel<64, 2>;
   else return cudaErrorInvalidValue;
-  static_assert(kSmemBytes >= static_cast<int>((kWarps * kD * 8 + 2 * kWarps * 8) * sizeof(float)), "merge scratch");
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  static_assert(kSmemStages >= static_cast<int>((kWarps * kD * 8 + 2 * kWarps * 8) * sizeof(float)) &&
+                    kSmemStages >= (3 * kMergeMax + kWarps * kMaxRatio * kD) * 4,
+                "merge scratch");
+  // opt in to the dynamic shared memory size once per (device, kernel variant)
+  static bool configured[64][4] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  kern<<<blocks, kWarps * 32, kSmemBytes, st>>>(a, plan);
-  return cudaGetLastError();
+  const int variant = (a.cv.G == 64 ? 2 : 0) + (r <= 4 ? 0 : 1);
+  if (dev < 0 || dev >= 64 || !configured[dev][variant]) {
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) configured[dev][variant] = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(a.cv.B * a.cv.Hkv * a.S);
+  cfg.blockDim = dim3(kWarps * 32);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, a);
 }
 
 }  // namespace lq

@@ -29,7 +29,7 @@ __device__ __forceinline__ float load_k(const TokenRef& r, int64_t t, int d) {
   kcode_pos(static_cast<int>(tq % r.G), d, word, bit);
   const uint32_t code = (reinterpret_cast<const uint32_t*>(tile + qt_kcodes_off())[word] >> bit) & 3u;
   const float s = bf16f(reinterpret_cast<const uint16_t*>(tile + qt_kscale_off())[kparam_index(d)]);
-  const float z = bf16f(reinterpret_cast<const uint16_t*>(tile + qt_kzero_off())[kparam_index(d)]);
+  const float z = bf16f(reinterpret_cast<const uint16_t*>(tile + qt_kzero_off())[d]);
   return fmaf(static_cast<float>(code), s, z);
 }
 
@@ -166,13 +166,14 @@ __global__ void __launch_bounds__(128) lq_merge_kernel(DecodeArgs a) {
   const int64_t pair = static_cast<int64_t>(b) * cv.Hkv + h / r;
   const int j = h % r;
   const int d = threadIdx.x;
+  const int count = a.S;
   float M = -INFINITY;
-  for (int s = 0; s < a.S; ++s) {
+  for (int s = 0; s < count; ++s) {
     const int64_t rec = (pair * a.S + s) * r + j;
     if (a.part_ml[rec * 2 + 1] > 0.f) M = fmaxf(M, a.part_ml[rec * 2]);
   }
   float L = 0.f, o = 0.f;
-  for (int s = 0; s < a.S; ++s) {
+  for (int s = 0; s < count; ++s) {
     const int64_t rec = (pair * a.S + s) * r + j;
     const float ls = a.part_ml[rec * 2 + 1];
     if (ls > 0.f) {

@@ -53,7 +53,9 @@ struct DecodeArgs {
   int layer;
   int n_fp;
   int64_t n_quant;
-  int S;  // partitions per (b, kv)
+  int S;  // split-K partitions (= CTAs of the attention kernel) per (b, kv); record (pair, s) at pair*S + s
+  int tiles_fp, tiles_quant;  // fp tiles (16 slots) and quant tiles (G tokens) per (b, kv)
+  int zero;                   // always 0; an opaque loop bound for the kernels
   float scale_log2;  // sm_scale * log2(e)
   const void* q;     // [B, Hq, D] bf16
   float* part_o;
@@ -61,11 +63,14 @@ struct DecodeArgs {
   void* out;
   int out_bf16;
   int* status;  // device word; kernels OR error bits into it (bounded waits that gave up)
+  int* tickets; // per (b, kv): [0] work-queue head, [1] arrival counter of the fused second pass; both 0 at rest
+                // (null: static split and a separate merge launch)
 };
 
 cudaError_t launch_decode_scalar(const DecodeArgs& a, cudaStream_t st);
+// Fills S and the tile counts of `a` for the tensor-core kernel (S <= max_records; s_override > 0 forces S).
+void plan_decode_mma(DecodeArgs& a, int sm_count, int max_records, int s_override);
 cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st);
-int decode_mma_max_splits(const CacheView& cv, int n_fp, int64_t n_quant, int sm_count);
 cudaError_t launch_merge(const DecodeArgs& a, cudaStream_t st);
 
 }  // namespace lq

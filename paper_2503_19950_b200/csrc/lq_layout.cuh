@@ -14,7 +14,7 @@
 // 2-bit store, per (layer, b, kv head): a sequence of "quant tiles"; one tile = one key group =
 //   G consecutive removed tokens = G/16 sub-tiles of 16 tokens.  Byte offsets inside a tile:
 //     0                      K scale, 128 bf16 in fragment order      (256 B)
-//     256                    K zero,  128 bf16 in fragment order      (256 B)
+//     256                    K zero,  128 bf16 in channel order       (256 B)
 //     512                    K codes, G/16 sub-tiles x 512 B
 //     512 + 32 G             V codes, G/16 sub-tiles x 512 B
 //     512 + 64 G             V scale, G/16 sub-tiles x (4096/G) B
@@ -26,7 +26,10 @@
 //     [16h + 2ks + 1 : 16h + 2ks]  = code of token 16u + 8nt + n, channel 16ks + 8w + 2j + h.
 //     (word (nt, w) masked at code position ks is the B-fragment register w of the k-step ks
 //      for the 8 tokens of n-tile nt: two codes, one per 16-bit half.)
-//   K scale / zero: channel 16ks + 8w + 2j + h at bf16 index 8*(4*(ks/2) + j) + 2*(2*(ks%2) + w) + h.
+//   K scale: channel 16ks + 8w + 2j + h at bf16 index 8*(4*(ks/2) + j) + 2*(2*(ks%2) + w) + h
+//     (four 16-byte loads give a lane the scale of every channel it multiplies).  K zero stays in
+//     channel order: an ldmatrix with all eight row addresses equal turns 32 bytes of it into the A
+//     fragment (every row the same) of the per-group q.zero product.
 //   V codes of sub-tile u: word 4*lane + dh + 2*th (lane = 4*r + j), bits [16h + 2mt + 1 : 16h + 2mt]
 //     = code of token 16u + 8th + 2j + h, channel 16mt + 8dh + r
 //     (word (th, dh) masked at position mt is the A-fragment register dh + 2*th of m-tile mt).
@@ -68,7 +71,7 @@ __host__ __device__ inline int64_t fp_chunk_off(int slot, int c) {
   return static_cast<int64_t>(slot >> 4) * kFpTileBytes + s * 256 + ((c ^ (s & 7)) << 4);
 }
 
-// bf16 index of channel d inside the K scale / K zero block
+// bf16 index of channel d inside the K scale block (the K zero block is in channel order)
 __host__ __device__ inline int kparam_index(int d) {
   int ks = d >> 4, w = (d >> 3) & 1, j = (d >> 1) & 3, h = d & 1;
   return 8 * (4 * (ks >> 1) + j) + 2 * (2 * (ks & 1) + w) + h;

@@ -13,6 +13,10 @@ namespace lq {
 __global__ void __launch_bounds__(256)
 lq_append_kernel(CacheView cv, int layer, const uint4* __restrict__ k, const uint4* __restrict__ v,
                  int n_src, int src0, int n, int slot0) {
+  // programmatic dependent launch: overlap this kernel's launch with the tail of the previous
+  // kernel of the stream, but write nothing before that kernel has finished
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   const int64_t total = static_cast<int64_t>(cv.B) * cv.Hkv * n * 32;
   if (idx >= total) return;
@@ -31,9 +35,17 @@ cudaError_t launch_append(const CacheView& cv, int layer, const void* k, const v
                           int src0, int n, int slot0, cudaStream_t st) {
   const int64_t total = static_cast<int64_t>(cv.B) * cv.Hkv * n * 32;
   const int blocks = static_cast<int>((total + 255) / 256);
-  lq_append_kernel<<<blocks, 256, 0, st>>>(cv, layer, static_cast<const uint4*>(k),
-                                           static_cast<const uint4*>(v), n_src, src0, n, slot0);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(blocks);
+  cfg.blockDim = dim3(256);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, lq_append_kernel, cv, layer, static_cast<const uint4*>(k),
+                            static_cast<const uint4*>(v), n_src, src0, n, slot0);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -123,7 +135,7 @@ lq_compress_kernel(CacheView cv, LayerList layers, EvictList ev, int64_t tile0) 
     float mnc, scale;
     group_params(mn, mx, sb, zb, mnc, scale);
     reinterpret_cast<uint16_t*>(tile + qt_kscale_off())[kparam_index(d)] = sb;
-    reinterpret_cast<uint16_t*>(tile + qt_kzero_off())[kparam_index(d)] = zb;
+    reinterpret_cast<uint16_t*>(tile + qt_kzero_off())[d] = zb;
 #pragma unroll 4
     for (int e = 0; e < G; ++e)
       sK[e][d] = static_cast<uint16_t>(quant_code(bf16_bits_to_float(sK[e][d]), mnc, scale));
@@ -246,7 +258,7 @@ __global__ void lq_export_params_kernel(CacheView cv, int layer, int64_t n_quant
       const uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
                             grp * quant_tile_bytes(G);
       if (k_scale) k_scale[idx] = reinterpret_cast<const uint16_t*>(tile + qt_kscale_off())[kparam_index(d)];
-      if (k_zero) k_zero[idx] = reinterpret_cast<const uint16_t*>(tile + qt_kzero_off())[kparam_index(d)];
+      if (k_zero) k_zero[idx] = reinterpret_cast<const uint16_t*>(tile + qt_kzero_off())[d];
     } else {
       const int64_t i2 = idx - nk;
       const int g = static_cast<int>(i2 % NG);
