@@ -228,7 +228,7 @@ def run_ours(args, wl, rank, world, device):
     e2e_s = time.perf_counter() - t0
     status = cache.kernel_status()
     assert status == 0, f"kernel status word {status}"
-    assert os.environ.get("LQ_LIB_SUFFIX") or all(torch.isfinite(o).all() for o in outs)
+    assert all(torch.isfinite(o).all() for o in outs)
 
     times = torch.tensor([ms, e2e_s * 1e3], dtype=torch.float64, device=device)
     if world > 1:

@@ -233,7 +233,7 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
               dev_alloc(c, reinterpret_cast<void**>(&cv.fp), cv.fp_layer_stride * cfg->n_layers) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->part_o), pairs * c->max_splits * r * kD * 4) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->part_ml), pairs * c->max_splits * r * 2 * 4) &&
-              dev_alloc(c, reinterpret_cast<void**>(&c->status), 256 + (1 << 20)) &&
+              dev_alloc(c, reinterpret_cast<void**>(&c->status), 256) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->tickets), pairs * 8) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_k), cfg->n_layers * pairs * kD * 2) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_v), cfg->n_layers * pairs * kD * 2) &&
@@ -425,12 +425,6 @@ lq_status_t lq_profile_read(lq_cache_t* c, double* total_ms, int64_t* n_launches
   return LQ_OK;
 }
 
-#ifdef LQ_EXP_TRACE
-lq_status_t lq_debug_trace(lq_cache_t* c, void* host, int bytes) {
-  cudaDeviceSynchronize();
-  return cudaMemcpy(host, c->status + 64, bytes, cudaMemcpyDeviceToHost) == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
-}
-#endif
 
 lq_status_t lq_kernel_status(lq_cache_t* c, int32_t* word) {
   if (!c || !word) return LQ_ERR_INVALID_ARG;

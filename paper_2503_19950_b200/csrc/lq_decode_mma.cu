@@ -36,9 +36,15 @@ namespace lq {
 namespace {
 
 constexpr int kWarps = 4;
-constexpr int kStageBytes = 5120;  // one quant tile (3 KB at G=32, 5 KB at G=64) or half an fp tile (4 KB)
-constexpr int kStages = 2;
-constexpr int kCtasPerSm = 4;
+constexpr int kStageBytes = 6144;  // two G=32 tiles, one G=64 tile, or half an fp tile (K rows / V rows)
+#ifndef LQ_STAGES
+#define LQ_STAGES 2
+#endif
+#ifndef LQ_CTAS_PER_SM
+#define LQ_CTAS_PER_SM 4
+#endif
+constexpr int kStages = LQ_STAGES;
+constexpr int kCtasPerSm = LQ_CTAS_PER_SM;
 constexpr uint32_t kFull = 0xFFFFFFFFu;
 constexpr int kSpinLimit = 1 << 22;
 
@@ -136,19 +142,11 @@ __device__ __forceinline__ uint2 lds64(uint32_t addr) {
 // one code position of a packed word as two bf16 subnormals (positions 0,2,4,6 of each byte)
 template <int I>
 __device__ __forceinline__ uint32_t ext_bf16(uint32_t w, uint32_t w8) {
-#ifdef LQ_EXP_NOEXT
-  return I < 4 ? w : w8;
-#else
   return I < 4 ? (w & (0x00030003u << (2 * I))) : (w8 & (0x00030003u << (2 * (I - 4))));
-#endif
 }
 // same with an index that becomes a constant once the caller's loop is unrolled
 __device__ __forceinline__ uint32_t ext_bf16_i(int i, uint32_t w, uint32_t w8) {
-#ifdef LQ_EXP_NOEXT
-  return i < 4 ? w : w8;
-#else
   return i < 4 ? (w & (0x00030003u << (2 * i))) : (w8 & (0x00030003u << (2 * (i - 4))));
-#endif
 }
 // ... or as two fp16 subnormals (positions 0..8 direct, 10..14 after a shift by 10)
 template <int I>
@@ -354,13 +352,6 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
   // bias advances by one MMA per k-step (A = zero rows via ldmatrix with equal row addresses),
   // and every sub-tile's score accumulator advances by one MMA per k-step.
   float s[NS][NCB][2];
-#ifdef LQ_EXP_NOQK
-#pragma unroll
-  for (int u = 0; u < NS; ++u)
-#pragma unroll
-    for (int cb = 0; cb < NCB; ++cb) s[u][cb][0] = s[u][cb][1] = static_cast<float>(lane + u) * kq;
-  if (false)
-#endif
   {
     uint32_t kw[NS][4], kws[NS][4];
 #pragma unroll
@@ -421,13 +412,7 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
       }
     }
   }
-#ifndef LQ_EXP_NOSOFTMAX
   tile_softmax<NCB, NS>(st, s, lane, opaque_zero);
-#endif
-#ifdef LQ_EXP_NOPV
-  st.l[0] += s[0][0][0] + s[NS - 1][0][1];
-  return;
-#endif
 
 #pragma unroll
   for (int u = 0; u < NS; ++u) {
@@ -542,7 +527,8 @@ __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm) lq_decode_mma_kernel(
 
   const int pair = blockIdx.x / a.S, slot = blockIdx.x % a.S;
   const int b = pair / cv.Hkv, kv = pair % cv.Hkv;
-  const int n_items = a.tiles_fp + a.tiles_quant;
+  constexpr int TPS = kStageBytes / quant_tile_bytes(G);  // quant tiles per claim (and per stage)
+  const int n_items = a.tiles_fp + (a.tiles_quant + TPS - 1) / TPS;
   int* queue = a.tickets + 2 * pair;
 
   const uint32_t stage0 = smem_u32(smem + warp * (kStages * kStageBytes));
@@ -577,17 +563,6 @@ __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm) lq_decode_mma_kernel(
               qbar);
   }
 
-#ifdef LQ_EXP_TRACE
-  unsigned long long tr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  unsigned long long gt0;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt0));
-  tr[0] = clock64();
-#define TR(i) tr[i] = clock64()
-#define TRACC(i, t) tr[i] += clock64() - (t)
-#else
-#define TR(i)
-#define TRACC(i, t)
-#endif
   float kc[4];
 #pragma unroll
   for (int c = 0; c < 4; ++c) kc[c] = a.scale_log2 * pow2i(2 * c - 64);
@@ -600,7 +575,7 @@ __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm) lq_decode_mma_kernel(
   // or quant tile t (desc = tiles_fp + t).  pending_v >= 0: the V rows of that fp tile come next.
   int issued = 0, pending_v = -1, n_claims = 0;
   bool drained = false;
-  int desc0 = 0, desc1 = 0;
+  int desc0 = 0, desc1 = 0, desc2 = 0;
   auto issue_next = [&]() {
     const uint8_t* src;
     uint32_t bytes;
@@ -627,12 +602,13 @@ __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm) lq_decode_mma_kernel(
         src = fpbase + static_cast<int64_t>(item) * kFpTileBytes;
         pending_v = item;
       } else {
-        bytes = TILE;
-        src = qbase + static_cast<int64_t>(item - a.tiles_fp) * TILE;
+        const int t0 = (item - a.tiles_fp) * TPS;
+        bytes = min(TPS, a.tiles_quant - t0) * TILE;
+        src = qbase + static_cast<int64_t>(t0) * TILE;
       }
     }
     const uint32_t s = issued % kStages;
-    if (s == 0) desc0 = desc; else desc1 = desc;
+    if (s == 0) desc0 = desc; else if (s == 1) desc1 = desc; else desc2 = desc;
     if (lane == 0) {
       mbar_expect_tx(bar0 + 8 * s, bytes);
       bulk_load(stage0 + s * kStageBytes, src, bytes, bar0 + 8 * s);
@@ -640,11 +616,8 @@ __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm) lq_decode_mma_kernel(
     ++issued;
   };
   bool failed = false;
-#ifndef LQ_EXP_NOLOAD
 #pragma unroll
   for (int s = 0; s < kStages; ++s) issue_next();
-#endif
-  TR(7);
 
   // query fragments: B operand, column n -> head 4cb + n/2 (even column = hi, odd = lo of q*s);
   // k-step ks carries the factor 2^(64 - 2*(ks&3)) that cancels the code-position factor
@@ -671,7 +644,6 @@ __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm) lq_decode_mma_kernel(
         }
     }
   }
-  TR(1);
   WarpState<NCB> st;
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) st.out[mt][0] = st.out[mt][1] = st.out[mt][2] = st.out[mt][3] = 0.f;
@@ -688,17 +660,13 @@ __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm) lq_decode_mma_kernel(
     {
       int spins = 0;
       bool bad = false;
-#ifdef LQ_EXP_TRACE
-      const unsigned long long tw = clock64();
-#endif
       while (!mbar_try_wait(bar0 + 8 * s, parity)) {
         if (++spins > kSpinLimit) { bad = true; break; }
       }
-      TRACC(6, tw);
       if (__any_sync(kFull, bad)) { failed = true; break; }
     }
     const uint32_t sbase = stage0 + s * kStageBytes;
-    const int desc = s == 0 ? desc0 : desc1;
+    const int desc = s == 0 ? desc0 : (s == 1 ? desc1 : desc2);
     if (desc >= a.tiles_fp) {
       // items come in queue order, so a warp sees all its fp tiles before its first quant tile: from
       // here on the out rows carry the code-position factor (two steps keep the constants normal).
@@ -714,9 +682,9 @@ __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm) lq_decode_mma_kernel(
         st.quant_mode = true;
         sw = a.zero;
       }
-#ifndef LQ_EXP_LOADONLY
-      process_quant_tile<G, NCB>(st, qs, sbase, kc, kq, lane, oddmask, a.zero);
-#endif
+      const int nt = min(TPS, a.tiles_quant - (desc - a.tiles_fp) * TPS);
+#pragma unroll 1
+      for (int t = 0; t < nt; ++t) process_quant_tile<G, NCB>(st, qs, sbase + t * TILE, kc, kq, lane, oddmask, a.zero);
     } else if (desc >= 0) {
       const int nv = min(16, a.n_fp - desc * 16);
       process_fp_keys<NCB>(st, qs, sbase, nv, kc, lane, oddmask, a.zero, fb0, fb1);
@@ -726,7 +694,6 @@ __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm) lq_decode_mma_kernel(
     __syncwarp();
     issue_next();
   }
-  TR(3);
   if (lane == 0 && pref < 0) atomicOr(a.status, 2);  // never true; makes sure the last claim has returned
   if (failed) {
     // a bulk copy never completed: flag it and contribute nothing (checked again at the end)
@@ -814,7 +781,6 @@ __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm) lq_decode_mma_kernel(
       }
     }
   }
-  TR(2);
   // ---- second pass, fused: the CTA that completes a pair (last ticket) merges its S partials.
   // Nobody waits for anybody: a CTA either finds that it is last, or leaves.
   __threadfence();
@@ -874,16 +840,6 @@ __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm) lq_decode_mma_kernel(
         static_cast<float*>(a.out)[oi] = o;
     }
   }
-  TR(4);
-#ifdef LQ_EXP_TRACE
-  if (lane == 0) {
-    unsigned long long gt1;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt1));
-    unsigned long long* dst = reinterpret_cast<unsigned long long*>(a.status + 64) + (static_cast<size_t>(blockIdx.x) * kWarps + warp) * 10;
-    for (int i = 0; i < 8; ++i) dst[i] = tr[i];
-    dst[8] = gt0; dst[9] = gt1;
-  }
-#endif
   if (failed) {
     // give copies still in flight a bounded chance to land before the shared memory is released
     for (int s = 0; s < kStages; ++s) {
@@ -900,7 +856,7 @@ void plan_decode_mma(DecodeArgs& a, int sm_count, int max_records, int s_overrid
   const int r = a.cv.Hq / a.cv.Hkv;
   a.tiles_fp = (a.n_fp + kFpTileSlots - 1) / kFpTileSlots;
   a.tiles_quant = static_cast<int>(a.n_quant / a.cv.G);
-  const int items = a.tiles_fp + a.tiles_quant;
+  const int items = a.tiles_fp + a.tiles_quant / (kStageBytes / quant_tile_bytes(a.cv.G));
   // about one resident wave of CTAs in total; work is pulled from per-pair queues, so a few CTAs
   // more or less than a wave cost nothing
   int S = s_override > 0 ? s_override : (kCtasPerSm * sm_count + pairs / 2) / pairs;

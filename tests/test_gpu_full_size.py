@@ -1,0 +1,77 @@
+"""GPU parity at the full sizes of the benchmark configurations (one layer cache each), in the launch
+configuration bench.py times (default kernel, library-chosen split count): bit-exact canonical image
+and attention within tolerance against the float64 oracle for every (batch row, head)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_common import assert_images_equal, attn_tolerance
+from paper_2503_19950_b200 import LogQuantCache, build, synth
+
+pytestmark = pytest.mark.gpu
+D = 128
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+
+
+def _run(B, Hq, Hkv, W, G, ctx, seed, n_steps, n_outliers=3, planted=False, image_stride=1):
+    dev = "cuda"
+    total = ctx + n_steps
+    outl = synth.outlier_channels(seed, Hkv, D, n_outliers) if n_outliers else None
+    u = synth.unit_vectors(seed, Hkv, D) if planted else None
+    cache = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=total + 8)
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G)
+    chunk = 2048
+    for t0 in list(range(0, ctx, chunk)) + [ctx + i for i in range(n_steps)]:
+        n = min(chunk, ctx - t0) if t0 < ctx else 1
+        k, v = synth.keys_values(seed, B, Hkv, n, D, dev, token_start=t0, token_total=total, outliers=outl)
+        if u is not None:
+            k = synth.plant_spikes(k, u, 16.0, t0, ctx)
+        cache.append(0, k, v)
+        oc.append(synth.bf16_bits(k), synth.bf16_bits(v))
+        if t0 < ctx:
+            continue
+        step = t0 - ctx
+        inf = cache.info(0)
+        assert (inf.n_fp, inf.n_quant, inf.n_events) == (oc.n_fp, oc.n_quant, oc.n_events)
+        if step % image_stride == 0:
+            assert_images_equal(cache.export(0), oc.export())
+        q = synth.queries(seed, B, Hq, D, step, dev)
+        if u is not None:
+            q = (q.float() + 4.0 * u.to(dev).repeat_interleave(Hq // Hkv, dim=0)[None]).to(torch.bfloat16)
+        out = torch.full((B, Hq, D), float("nan"), device=dev)
+        cache.decode_attn(0, q, out)
+        torch.cuda.synchronize()
+        ref = oc.attention(synth.bf16_bits(q), 1 / np.sqrt(D), n_threads=16)
+        got = out.cpu().numpy().astype(np.float64)
+        err, tol = float(np.abs(got - ref).max()), attn_tolerance(ref)
+        assert np.isfinite(got).all() and err <= tol, f"step {step}: max|delta| {err:.3e} > {tol:.3e}"
+    assert cache.kernel_status() == 0
+    return cache.info(0)
+
+
+def test_config2_llama3_8b_layer_8k():
+    # 32 q / 8 kv heads, batch 8, context 8192, W=128, G=32: 61 overflow events in the prefill, the 62nd
+    # on the first decode step
+    inf = _run(B=8, Hq=32, Hkv=8, W=128, G=32, ctx=8192, seed=2, n_steps=2)
+    assert (inf.n_quant, inf.n_fp) == (7936, 258)
+
+
+def test_config3_batch16_4k():
+    inf = _run(B=16, Hq=32, Hkv=8, W=128, G=32, ctx=4096, seed=3, n_steps=1)
+    assert (inf.n_quant, inf.n_fp) == (3840, 257)
+
+
+def test_config4_gqa7_32k_planted_spikes():
+    # 28 q / 4 kv heads, W=256, G=64, keys with planted high-logit tokens at log-spaced distances
+    inf = _run(B=4, Hq=28, Hkv=4, W=256, G=64, ctx=32768, seed=4, n_steps=1, n_outliers=0, planted=True)
+    assert (inf.n_quant, inf.n_fp) == (32256, 513)
+
+
+def test_config5_mha_128k_one_layer():
+    inf = _run(B=1, Hq=32, Hkv=32, W=256, G=32, ctx=131072, seed=5, n_steps=1)
+    assert (inf.n_quant, inf.n_fp) == (130560, 513)
