@@ -108,6 +108,19 @@ class ClockSampler:
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def reduce_max_over_ranks(values, world, device):
+    """MAX over ranks of a list of per-rank timings (the job is as slow as its slowest replica)."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return t.tolist()
+
+
+def aggregate_throughput(units_per_rank, world, ms_max):
+    """Whole-job throughput of `world` independent replicas that each processed units_per_rank."""
+    return units_per_rank * world / (ms_max * 1e-3)
+
+
 def make_step_inputs(wl, device, n_sets):
     """Per layer: n_sets rotating (k_new, v_new, q) triples, resident on `device`."""
     L, B, Hq, Hkv = wl["L"], wl["B"], wl["Hq"], wl["Hkv"]
@@ -230,17 +243,14 @@ def run_ours(args, wl, rank, world, device):
     assert status == 0, f"kernel status word {status}"
     assert all(torch.isfinite(o).all() for o in outs)
 
-    times = torch.tensor([ms, e2e_s * 1e3], dtype=torch.float64, device=device)
-    if world > 1:
-        torch.distributed.all_reduce(times, op=torch.distributed.ReduceOp.MAX)
-    ms_max, e2e_ms_max = times.tolist()
+    ms_max, e2e_ms_max = reduce_max_over_ranks([ms, e2e_s * 1e3], world, device)
     peak, peak_kind = peaks()
     bytes_per_launch = byte_sum / max(k_n, 1)
     q_out_part = 0  # q, out and partials are not counted in the algorithmic bytes
     achieved = bytes_per_launch / (k_ms / max(k_n, 1) * 1e-3) / 1e9 if k_n else None
     inf = cache.info(0)
     line = {
-        "metric": "decode_attn_kv_tokens_per_s", "value": kv_tokens * world / (ms_max * 1e-3),
+        "metric": "decode_attn_kv_tokens_per_s", "value": aggregate_throughput(kv_tokens, world, ms_max),
         "unit": "KV tokens/s", "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": ms_max / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
@@ -254,7 +264,7 @@ def run_ours(args, wl, rank, world, device):
         "algorithmic_gbs_whole_step": bytes_step_last / (ms_max / steps * 1e-3) / 1e9,
         "gpu_launches": int(launches),
         "clocks": clk.summary(),
-        "e2e": {"value": kv_e2e * world / (e2e_ms_max * 1e-3), "unit": "KV tokens/s",
+        "e2e": {"value": aggregate_throughput(kv_e2e, world, e2e_ms_max), "unit": "KV tokens/s",
                 "h2d_bytes_per_step": L * (2 * B * Hkv * D * 2 + B * Hq * D * 2),
                 "d2h_bytes_per_step": L * B * Hq * D * 4, "steps": e2e_steps,
                 "api": "lq_decode_step_host (pinned host buffers, one stream sync per step)"},
@@ -264,15 +274,20 @@ def run_ours(args, wl, rank, world, device):
                      "us_per_launch": k_ms / max(k_n, 1) * 1e3, "launches_timed": int(k_n),
                      "frac_of_8tbs_nominal": achieved / 8000.0 if achieved else None},
     }
-    traffic_file = os.path.join(ROOT, "profiles", "traffic_%s.json" % args.workload)
+    # DRAM bytes per launch of the dominant kernel, from the committed ncu summary of this workload
+    traffic_file = os.path.join(ROOT, "profiles", "decode_attention_%s.md" % args.workload)
     if os.path.exists(traffic_file):
+        import re
         with open(traffic_file) as f:
-            line["roofline"]["traffic"] = json.load(f).get("dram_bytes_per_launch")
+            m = re.search(r"dram_bytes_per_launch:\s*([0-9.eE+]+)", f.read())
+        if m:
+            line["roofline"]["traffic"] = float(m.group(1))
     return line, cache
 
 
-def oracle_layer_step(wl, device, n_threads, min_seconds, max_reps):
-    """Times the CPU oracle on one layer of the workload: append one token + attention."""
+def oracle_layer_step(wl, device, n_threads, min_seconds, max_reps, warmup=0):
+    """Times the CPU oracle on one layer of the workload: append one token + attention.
+    Runs until min_seconds of timed work or max_reps steps, whichever comes first (at least one)."""
     import oracle
     B, Hq, Hkv, W, G, ctx = (wl[k] for k in ("B", "Hq", "Hkv", "W", "G", "ctx"))
     oc = oracle.OracleCache(B, Hq, Hkv, D, W, G)
@@ -282,6 +297,11 @@ def oracle_layer_step(wl, device, n_threads, min_seconds, max_reps):
     kb, vb = synth.bf16_bits(k), synth.bf16_bits(v)
     reps, t_total, kv = 0, 0.0, 0
     times = []
+    for i in range(warmup):
+        q = synth.bf16_bits(synth.queries(wl["seed"], B, Hq, D, i % Q_ROTATE, device, layer=0))
+        oc.append(np.ascontiguousarray(kb[:, :, i % Q_ROTATE:i % Q_ROTATE + 1]),
+                  np.ascontiguousarray(vb[:, :, i % Q_ROTATE:i % Q_ROTATE + 1]))
+        oc.attention(q, 1.0 / np.sqrt(D), n_threads=n_threads)
     while (t_total < min_seconds and reps < max_reps) or reps < 1:
         s = reps % Q_ROTATE
         q = synth.bf16_bits(synth.queries(wl["seed"], B, Hq, D, s, device, layer=0))
@@ -323,9 +343,8 @@ def main():
         import oracle
         oracle.build()
         device = torch.device("cuda", local) if torch.cuda.is_available() else torch.device("cpu")
-        for _ in range(max(args.warmup, 0)):
-            pass  # the oracle has no warm state; its first timed step is as good as any
-        tput, reps, t_total, times = oracle_layer_step(wl, device, cores, min_seconds=0.0, max_reps=max(args.steps, 1))
+        tput, reps, t_total, times = oracle_layer_step(wl, device, cores, min_seconds=1e9, max_reps=max(args.steps, 1),
+                                                       warmup=max(args.warmup, 0))
         sample = "one of %d layers of %s per step: append 1 token + attention, float64" % (wl["L"], args.workload)
         line = {"impl": "reference", "metric": "decode_attn_kv_tokens_per_s", "value": tput, "unit": "KV tokens/s",
                 "n_gpus": args.gpus, "steps": reps, "warmup": args.warmup, "ms_per_step": t_total / reps * 1e3,
@@ -348,7 +367,7 @@ def main():
         if not args.no_cpu_baseline:
             import oracle
             oracle.build()
-            tput, reps, t_total, _ = oracle_layer_step(wl, device, cores, min_seconds=10.0, max_reps=64)
+            tput, reps, t_total, _ = oracle_layer_step(wl, device, cores, min_seconds=10.0, max_reps=512)
             line["cpu_baseline"] = {"value": tput, "unit": "KV tokens/s", "cores": cores, "kind": "oracle",
                                     "sample": "%d decode steps of one of the %d layers (append 1 token + float64 "
                                               "attention over all %d sequences), %.1f s" % (reps, wl["L"], wl["B"], t_total)}
