@@ -47,7 +47,7 @@ typedef enum {
   LQ_ERR_OOM = 3,         /* device allocation failed                                           */
   LQ_ERR_WINDOW_FULL = 4, /* lq_append would exceed 3W full-precision tokens (auto_compress=0)  */
   LQ_ERR_NOT_FULL = 5,    /* lq_compress on a layer that holds fewer than 3W full-precision tokens */
-  LQ_ERR_CAPACITY = 6,    /* max_tokens would be exceeded                                       */
+  LQ_ERR_CAPACITY = 6,    /* max_tokens would be exceeded, or a size beyond a fixed scratch     */
   LQ_ERR_CUDA = 7         /* a CUDA runtime call or a kernel launch failed                      */
 } lq_status_t;
 
@@ -178,6 +178,49 @@ lq_status_t lq_export(const lq_cache_t* cache, int32_t layer, lq_image_t* image_
  * lq_compress on `layer` would remove, in removal order (W entries; LQ_ERR_NOT_FULL if the
  * layer holds fewer than 3W full-precision tokens). */
 lq_status_t lq_next_evicted_ids(const lq_cache_t* cache, int32_t layer, int32_t* ids_host);
+
+/*
+ * Device-resident canonical image of one layer: the same arrays and layouts as lq_image_t, but the
+ * pointers are DEVICE pointers into memory the caller owns (ids are not needed for attention).
+ */
+typedef struct {
+  int32_t batch, n_q_heads, n_kv_heads, head_dim, group;
+  int32_t n_fp;      /* rows of fp_k / fp_v per (batch row, KV head)                              */
+  int64_t n_quant;   /* quantised tokens per (batch row, KV head); a multiple of group            */
+  const uint16_t* fp_k;    /* [B][Hkv][n_fp][D] bf16 bits                                          */
+  const uint16_t* fp_v;
+  const uint8_t* k_codes;  /* [B][Hkv][n_quant][D/4]                                               */
+  const uint8_t* v_codes;
+  const uint16_t* k_scale; /* [B][Hkv][n_quant/G][D]                                               */
+  const uint16_t* k_zero;
+  const uint16_t* v_scale; /* [B][Hkv][n_quant][D/G]                                               */
+  const uint16_t* v_zero;
+} lq_device_image_t;
+
+/*
+ * Decode attention that allocates nothing (the paper has no counterpart: this entry point exists for
+ * callers, not for the method).  For processes that may not call cudaMalloc -- a server that handed
+ * its whole memory budget to a fixed arena at start-up, code running under another component's
+ * allocator policy, or code called while a stream is being captured -- lq_cache_create is out of
+ * reach, because it allocates the stores and the split-K workspace.  Here the caller keeps the cache
+ * itself, as a canonical image in its own device memory, and passes q ([B,Hq,D] bf16, device) and
+ * out ([B,Hq,D] fp32, device); the only scratch, the split-K partials, lives in a fixed 4.06 MiB
+ * array inside the library image (held by every GPU that loads the library until the process exits).
+ * The result equals lq_decode_attn on the same cache content (plain fp32 kernel, same tolerance).
+ *
+ * Limits and rules:
+ *   - batch * n_q_heads <= 8192 (LQ_ERR_CAPACITY otherwise: the scratch holds 8192 partial records);
+ *     head_dim 128, group 32 or 64, n_q_heads / n_kv_heads <= 8 (LQ_ERR_UNSUPPORTED otherwise).
+ *   - No cudaMalloc, cudaFree or other allocating call is made, ever.  The first call on each device
+ *     looks up the scratch's device address (cudaGetSymbolAddress) with that device current; make
+ *     that first call before any stream capture begins.
+ *   - All calls on a device share the one scratch array.  Nothing in it needs clearing (every record a
+ *     call reads, it has written first), but two calls whose kernels overlap on the GPU -- different
+ *     streams, or the same image from two threads -- race on it: serialise them.
+ *   - Enqueues two kernels on `stream` and returns without synchronising.
+ */
+lq_status_t lq_decode_attn_image_static(const lq_device_image_t* image, const void* q, float sm_scale,
+                                        float* out, void* stream);
 
 const char* lq_status_str(lq_status_t status);
 

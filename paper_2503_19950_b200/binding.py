@@ -35,9 +35,15 @@ class lq_image_t(C.Structure):
                                           "v_scale", "v_zero", "fp_k", "fp_v")]
 
 
+class lq_device_image_t(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
+                ("group", C.c_int32), ("n_fp", C.c_int32), ("n_quant", C.c_int64)] + \
+               [(n, C.c_void_p) for n in ("fp_k", "fp_v", "k_codes", "v_codes", "k_scale", "k_zero", "v_scale", "v_zero")]
+
+
 SYMBOLS = ["lq_cache_create", "lq_destroy", "lq_append", "lq_compress", "lq_decode_attn",
            "lq_decode_step_host", "lq_profile_enable", "lq_profile_read", "lq_kernel_status", "lq_cache_info", "lq_export",
-           "lq_next_evicted_ids", "lq_status_str", "lq_last_error"]
+           "lq_next_evicted_ids", "lq_decode_attn_image_static", "lq_status_str", "lq_last_error"]
 
 _lib = None
 
@@ -69,6 +75,7 @@ def load_library():
         L.lq_cache_info.argtypes = [vp, i32, C.POINTER(lq_info_t)]
         L.lq_export.argtypes = [vp, i32, C.POINTER(lq_image_t)]
         L.lq_next_evicted_ids.argtypes = [vp, i32, vp]
+        L.lq_decode_attn_image_static.argtypes = [C.POINTER(lq_device_image_t), vp, C.c_float, vp, vp]
         L.lq_status_str.argtypes = [i32]
         L.lq_status_str.restype = C.c_char_p
         L.lq_last_error.argtypes = [vp]
@@ -101,6 +108,17 @@ def _stream(stream):
         import torch
         return torch.cuda.current_stream().cuda_stream if torch.cuda.is_available() else None
     return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def decode_attn_image_static(image: dict, n_q_heads: int, group: int, q, out, sm_scale=0.0, stream=None) -> int:
+    """lq_decode_attn_image_static on a canonical image whose arrays are torch tensors on the device
+    (keys as in LogQuantCache.export, without the ids).  Allocates nothing; returns the status code."""
+    B, Hkv, n_fp, D = image["fp_k"].shape
+    n_quant = image["k_codes"].shape[2]
+    st = lq_device_image_t(B, n_q_heads, Hkv, D, group, n_fp, n_quant,
+                           *[(_ptr(image[k]) if image[k].numel() else None)
+                             for k in ("fp_k", "fp_v", "k_codes", "v_codes", "k_scale", "k_zero", "v_scale", "v_zero")])
+    return load_library().lq_decode_attn_image_static(C.byref(st), _ptr(q), sm_scale, _ptr(out), _stream(stream))
 
 
 class LogQuantCache:

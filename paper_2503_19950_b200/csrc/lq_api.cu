@@ -182,7 +182,7 @@ const char* lq_status_str(lq_status_t s) {
     case LQ_ERR_OOM: return "out of device memory";
     case LQ_ERR_WINDOW_FULL: return "full-precision window is full";
     case LQ_ERR_NOT_FULL: return "full-precision window is not full";
-    case LQ_ERR_CAPACITY: return "max_tokens exceeded";
+    case LQ_ERR_CAPACITY: return "capacity exceeded (max_tokens of the cache, or the fixed scratch of the static entry point)";
     case LQ_ERR_CUDA: return "CUDA error";
   }
   return "unknown status";
