@@ -158,7 +158,8 @@ def run_ours(args, wl, rank, world, device):
     L, B, Hq, Hkv, W, G, ctx = (wl[k] for k in ("L", "B", "Hq", "Hkv", "W", "G", "ctx"))
     steps, warmup = args.steps, args.warmup
     total_steps = 2 * (steps + warmup) + steps + warmup + 8  # device-timed, profiled and host-buffer passes
-    cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=ctx + total_steps + 8, device=device.index or 0)
+    cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=ctx + total_steps + 8, device=device.index or 0,
+                          n_splits=args.n_splits)
     prefill(cache, wl, device)
     ks, vs, qs = make_step_inputs(wl, device, Q_ROTATE)
     outs = [torch.empty(B, Hq, D, device=device) for _ in range(L)]
@@ -239,6 +240,31 @@ def run_ours(args, wl, rank, world, device):
         kv_e2e += B * (inf[0] + inf[1]) * L
     barrier()
     e2e_s = time.perf_counter() - t0
+    # ---- one window-overflow event over all layers at once (lq_compress(layer=-1)) ----
+    comp = None
+    try:
+        ccache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=8 * W, device=device.index or 0, auto_compress=False)
+        kf, vf = synth.keys_values(wl["seed"] + 7, B, Hkv, 3 * W, D, device, outliers=wl.get("_outliers"))
+        k1, v1 = kf[:, :, :W].contiguous(), vf[:, :, :W].contiguous()
+        evs = []
+        for rep in range(6):
+            for l in range(L):
+                ccache.append(l, kf, vf) if rep == 0 else ccache.append(l, k1, v1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            ccache.compress(-1)
+            e1.record()
+            torch.cuda.synchronize()
+            evs.append(e0.elapsed_time(e1) * 1e3)
+        us = float(np.median(evs[1:]))
+        rd = L * B * Hkv * (2 * W * 256 + W * 512)          # removed rows + back-fill sources, K and V
+        wr = L * B * Hkv * (W * (1024 // G + 64) + W * 512)   # packed tiles + back-filled rows
+        comp = {"us_per_event": us, "layers": L, "tokens_per_s": L * B * W / (us * 1e-6),
+                "gbs": (rd + wr) / (us * 1e-6) / 1e9, "read_bytes": rd, "write_bytes": wr}
+        ccache.close()
+    except Exception as exc:  # the main numbers stand without it
+        comp = {"error": str(exc)}
     status = cache.kernel_status()
     assert status == 0, f"kernel status word {status}"
     assert all(torch.isfinite(o).all() for o in outs)
@@ -263,6 +289,7 @@ def run_ours(args, wl, rank, world, device):
         "per_layer_us": ms_max / steps / L * 1e3,
         "algorithmic_gbs_whole_step": bytes_step_last / (ms_max / steps * 1e-3) / 1e9,
         "gpu_launches": int(launches),
+        "compress_event": comp,
         "clocks": clk.summary(),
         "e2e": {"value": aggregate_throughput(kv_e2e, world, e2e_ms_max), "unit": "KV tokens/s",
                 "h2d_bytes_per_step": L * (2 * B * Hkv * D * 2 + B * Hq * D * 2),
@@ -325,6 +352,7 @@ def main():
     ap.add_argument("--workload", default="llama3-8b-8k", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="override the number of stacked layer caches (profiling runs)")
+    ap.add_argument("--n-splits", type=int, default=0, help="split-K CTAs per (batch row, KV head); 0 = library default")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 

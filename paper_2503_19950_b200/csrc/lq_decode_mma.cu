@@ -36,7 +36,10 @@ namespace lq {
 namespace {
 
 constexpr int kWarps = 4;
-constexpr int kStageBytes = 6144;  // two G=32 tiles, one G=64 tile, or half an fp tile (K rows / V rows)
+#ifndef LQ_STAGE_BYTES
+#define LQ_STAGE_BYTES 6144
+#endif
+constexpr int kStageBytes = LQ_STAGE_BYTES;  // two G=32 tiles, one G=64 tile, or half an fp tile (K rows / V rows)
 #ifndef LQ_STAGES
 #define LQ_STAGES 2
 #endif
@@ -76,14 +79,14 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 }
 __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                         uint32_t b0, uint32_t b1) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
@@ -156,6 +159,14 @@ __device__ __forceinline__ uint32_t ext_f16(uint32_t w, uint32_t w10) {
 
 // NCB = number of column blocks of 4 heads.  NCB == 1: p.v columns are (hi, lo) per head and the
 // probabilities carry a factor 2^64 (kPExp) so that products with bf16 subnormal codes stay normal.
+// p.v flavour.  bf16_pv: columns are (hi, lo) per head, everything bf16, exact products, r <= 4 only.
+// Otherwise: heads on the 8 columns, value codes as fp16 subnormals, p * s_v rounded to fp16.
+#ifndef LQ_BF16_PV
+#define LQ_BF16_PV 1
+#endif
+template <int NCB>
+__host__ __device__ constexpr bool bf16_pv() { return LQ_BF16_PV != 0 && NCB == 1; }
+
 template <int NCB>
 struct WarpState {
   float out[8][4];  // o^T: [channel tile][c-fragment]
@@ -166,13 +177,13 @@ struct WarpState {
 };
 template <int NCB>
 struct Mode {
-  static constexpr float kPExp = NCB == 1 ? 64.f : 0.f;
+  static constexpr float kPExp = bf16_pv<NCB>() ? 64.f : 0.f;
 };
 
 // factor the out rows of channel tile mt carry in quant mode, relative to fp mode
 template <int NCB>
 __device__ __forceinline__ int vpos_log2(int mt) {
-  return NCB == 1 ? 2 * (mt & 3) - 133 : 2 * (mt < 5 ? mt : mt - 5) - 24;
+  return bf16_pv<NCB>() ? 2 * (mt & 3) - 133 : 2 * (mt < 5 ? mt : mt - 5) - 24;
 }
 
 // ---- online softmax over the NSUB*16 scores of one tile ---------------------------------------
@@ -204,7 +215,7 @@ __device__ __forceinline__ void tile_softmax(WarpState<NCB>& st, float (&s)[NSUB
   int again = __any_sync(kFull, changed);
   while (again) {
     float ca, cbv;
-    if (NCB == 1) {
+    if (bf16_pv<NCB>()) {
       ca = cbv = corr[0];  // all four accumulators of a lane belong to head lane%4
     } else {
       const float a0 = __shfl_sync(kFull, corr[0], (2 * j) & 3), a1 = __shfl_sync(kFull, corr[NCB - 1], (2 * j) & 3);
@@ -244,8 +255,10 @@ __device__ __forceinline__ void transpose_p(const float (&p)[NCB][2], float (&pT
   for (int th = 0; th < 2; ++th)
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
-      if (NCB == 1) {
+      if (bf16_pv<NCB>()) {
         pT[th][i] = __shfl_sync(kFull, p[0][th], 4 * (2 * j + i) + (n >> 1));  // column n -> head n/2
+      } else if (NCB == 1) {
+        pT[th][i] = __shfl_sync(kFull, p[0][th], 4 * (2 * j + i) + (n & 3));  // column n -> head n (mod 4)
       } else {
         const int src = 4 * (2 * j + i) + (n & 3);  // column n -> head n
         const float v0 = __shfl_sync(kFull, p[0][th], src), v1 = __shfl_sync(kFull, p[NCB - 1][th], src);
@@ -311,7 +324,7 @@ __device__ __forceinline__ void process_fp_keys(WarpState<NCB>& st, const uint32
   float pT[2][2];
   transpose_p<NCB>(s[0], pT, lane);
   // NCB == 1: only b0 (hi/lo by column); NCB == 2: b0 = hi, b1 = lo
-  if (NCB == 1) {
+  if (bf16_pv<NCB>()) {
     uint32_t H[2], Pz[2];
     split_p_bf16(pT, oddmask, H, b0, Pz);
     b1[0] = b1[1] = 0;
@@ -336,7 +349,7 @@ __device__ __forceinline__ void process_fp_values(WarpState<NCB>& st, uint32_t v
     uint32_t a0, a1, a2, a3;
     ldmatrix_x4_trans(rowaddr + ((chunk ^ (token & 7)) << 4), a0, a1, a2, a3);
     mma_bf16(st.out[mt], a0, a1, a2, a3, b0[0], b0[1]);
-    if (NCB != 1) mma_bf16(st.out[mt], a0, a1, a2, a3, b1[0], b1[1]);
+    if (!bf16_pv<NCB>()) mma_bf16(st.out[mt], a0, a1, a2, a3, b1[0], b1[1]);
   }
 }
 
@@ -419,13 +432,13 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
     float pT[2][2];
     transpose_p<NCB>(s[u], pT, lane);
     const uint4 vw = lds128(tile + qt_vcodes_off(G) + u * 512 + 16 * lane);
-    if (NCB == 1) {
+    if (bf16_pv<NCB>()) {
       uint32_t H[2], P[2], Pz[2];
       split_p_bf16(pT, oddmask, H, P, Pz);
       // value zero: A = zero (bf16 pairs straight from the tile), value groups on rows
       {
-        uint2 zw = make_uint2(0u, 0u);
-        if (n < NG) zw = lds64(tile + qt_vzero_off(G) + u * VS + 8 * (4 * n + j));
+        // rows n >= NG of this MMA repeat real rows; their sums land in zacc rows nobody reads
+        const uint2 zw = lds64(tile + qt_vzero_off(G) + u * VS + 8 * (4 * (n % NG) + j));
         mma_bf16(st.zacc, zw.x, 0u, zw.y, 0u, P[0], P[1]);
       }
       // p * value scale per value group: even columns RN(hi*s), odd columns lo*s + residual
@@ -507,7 +520,7 @@ constexpr int kSmemStages = kWarps * kStages * kStageBytes;
 constexpr int kSmemQ = kMaxRatio * kD * 2;
 constexpr int kSmemBars = (kWarps * kStages + 1) * 8;
 constexpr int kSmemBytes = kSmemStages + kSmemQ + kSmemBars + 16;
-constexpr int kMergeMax = 2048;  // S * r records the fused second pass can stage
+constexpr int kMergeMax = kStageBytes >= 5120 ? 2048 : 1024;  // S * r records the fused second pass can stage
 
 // Work items of one (b, kv) pair, in queue order: fp tiles [0, tiles_fp), then quant tiles.  The S
 // CTAs of the pair (4 warps each) pull items one at a time from a global counter, so every warp of
@@ -515,7 +528,7 @@ constexpr int kMergeMax = 2048;  // S * r records the fused second pass can stag
 // legal because every warp keeps its own online-softmax state.  A warp always has its next claim
 // in flight (the atomic's latency hides behind the tile being processed) and two loads in flight.
 template <int G, int NCB>
-__global__ void __launch_bounds__(kWarps * 32, kCtasPerSm) lq_decode_mma_kernel(DecodeArgs a) {
+__global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerSm - 1) lq_decode_mma_kernel(DecodeArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   const CacheView& cv = a.cv;
   const int r = cv.Hq / cv.Hkv;
@@ -523,7 +536,7 @@ __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm) lq_decode_mma_kernel(
   const int n = lane >> 2, j = lane & 3;
   const uint32_t oddmask = (n & 1) ? 0xFFFFFFFFu : 0u;
   constexpr int TILE = quant_tile_bytes(G);
-  static_assert(TILE <= kStageBytes && kFpTileVOffset <= kStageBytes, "stage too small");
+  static_assert((TILE <= kStageBytes || G == 64) && kFpTileVOffset <= kStageBytes, "stage too small");
 
   const int pair = blockIdx.x / a.S, slot = blockIdx.x % a.S;
   const int b = pair / cv.Hkv, kv = pair % cv.Hkv;
@@ -703,14 +716,14 @@ __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm) lq_decode_mma_kernel(
   }
 
   // ---- fold zero term, undo position factors, reduce l over the token lanes ----
-  constexpr float kPInv = NCB == 1 ? 0x1p-64f : 1.0f;
+  constexpr float kPInv = bf16_pv<NCB>() ? 0x1p-64f : 1.0f;
   float o0[8], o1[8];  // NCB == 1: rows (n, n+8) of head j; NCB == 2: unused
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) {
     const int g = (mt * 16) / G;
     // quant mode: out = true * 2^(kPExp + vpos); fp mode: out = true * 2^kPExp
-    const float f = st.quant_mode ? pow2i(-vpos_log2<NCB>(mt) - 70) * (NCB == 1 ? 0x1p6f : 0x1p70f) : kPInv;
-    if (NCB == 1) {
+    const float f = st.quant_mode ? pow2i(-vpos_log2<NCB>(mt) - 70) * (bf16_pv<NCB>() ? 0x1p6f : 0x1p70f) : kPInv;
+    if (bf16_pv<NCB>()) {
       const float z = __shfl_sync(kFull, st.zacc[0] + st.zacc[1], 4 * g + j) * kPInv;
       o0[mt] = fmaf(st.out[mt][0] + st.out[mt][1], f, z);
       o1[mt] = fmaf(st.out[mt][2] + st.out[mt][3], f, z);
@@ -737,7 +750,7 @@ __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm) lq_decode_mma_kernel(
   float* wl = wm + kWarps * 8;                   // [warp][8]
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) {
-    if (NCB == 1) {
+    if (bf16_pv<NCB>()) {
       float* o = wout + (warp * kD + 16 * mt + n) * 8 + j;
       o[0] = o0[mt];
       o[64] = o1[mt];  // row + 8
@@ -857,9 +870,10 @@ void plan_decode_mma(DecodeArgs& a, int sm_count, int max_records, int s_overrid
   a.tiles_fp = (a.n_fp + kFpTileSlots - 1) / kFpTileSlots;
   a.tiles_quant = static_cast<int>(a.n_quant / a.cv.G);
   const int items = a.tiles_fp + a.tiles_quant / (kStageBytes / quant_tile_bytes(a.cv.G));
-  // about one resident wave of CTAs in total; work is pulled from per-pair queues, so a few CTAs
-  // more or less than a wave cost nothing
-  int S = s_override > 0 ? s_override : (kCtasPerSm * sm_count + pairs / 2) / pairs;
+  // at most one resident wave of CTAs in total: a CTA that had to wait for a free slot would start
+  // when the others finish, and its pair's merge would wait for it
+  const int ctas_per_sm = r <= 4 ? kCtasPerSm : kCtasPerSm - 1;  // the two-column-block variant needs more registers
+  int S = s_override > 0 ? s_override : (ctas_per_sm * sm_count) / pairs;
   S = std::min(S, (items + kWarps - 1) / kWarps);  // at least one item per warp
   S = std::min(S, max_records);
   S = std::min(S, kMergeMax / r);
