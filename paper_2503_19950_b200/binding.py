@@ -7,7 +7,7 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "liblogquant%s.so" % os.environ.get("LQ_LIB_SUFFIX", ""))
+_LIB_PATH = os.path.join(_HERE, "liblogquant.so")
 
 LQ_DEVICE_NONE = -1
 LQ_KERNEL_AUTO, LQ_KERNEL_SCALAR, LQ_KERNEL_MMA = 0, 1, 2

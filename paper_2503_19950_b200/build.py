@@ -7,7 +7,7 @@ import sys
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
-LIB = os.path.join(_HERE, "liblogquant%s.so" % os.environ.get("LQ_LIB_SUFFIX", ""))
+LIB = os.path.join(_HERE, "liblogquant.so")
 SOURCES = ["lq_api.cu", "lq_store_kernels.cu", "lq_decode_scalar.cu", "lq_decode_mma.cu", "lq_decode_static.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-shared", "--expt-relaxed-constexpr"]
@@ -24,7 +24,7 @@ def _stale() -> bool:
 def build(force: bool = False, verbose: bool = False) -> str:
     if force or _stale():
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-        cmd = [nvcc] + NVCC_FLAGS + os.environ.get("LQ_EXTRA_NVCC_FLAGS", "").split() + (["-Xptxas", "-v"] if verbose else []) + \
+        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
               [os.path.join(CSRC, s) for s in SOURCES] + ["-o", LIB + ".tmp"]
         res = subprocess.run(cmd, capture_output=True, text=True)
         if verbose or res.returncode:

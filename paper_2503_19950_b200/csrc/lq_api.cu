@@ -224,17 +224,17 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
     if (e != cudaSuccess) { delete c; cudaGetLastError(); return LQ_ERR_CUDA; }
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, cfg->device) == cudaSuccess) c->sm_count = prop.multiProcessorCount;
-    // split-K partial records reserved per (b, kv)
-    c->max_splits = cfg->n_splits > 0
+    // split-K partial records reserved per (b, kv) (one more than the CTAs per pair: some pairs get an extra CTA)
+    c->max_splits = 1 + (cfg->n_splits > 0
                         ? cfg->n_splits
-                        : static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(256, (8LL * c->sm_count + pairs - 1) / pairs)));
+                        : static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(256, (8LL * c->sm_count + pairs - 1) / pairs))));
     const int r = ratio(c);
     bool ok = dev_alloc(c, reinterpret_cast<void**>(&cv.quant), cv.quant_layer_stride * cfg->n_layers) &&
               dev_alloc(c, reinterpret_cast<void**>(&cv.fp), cv.fp_layer_stride * cfg->n_layers) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->part_o), pairs * c->max_splits * r * kD * 4) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->part_ml), pairs * c->max_splits * r * 2 * 4) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->status), 256) &&
-              dev_alloc(c, reinterpret_cast<void**>(&c->tickets), pairs * 8) &&
+              dev_alloc(c, reinterpret_cast<void**>(&c->tickets), pairs * 128) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_k), cfg->n_layers * pairs * kD * 2) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_v), cfg->n_layers * pairs * kD * 2) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_q),
@@ -242,7 +242,7 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_out),
                         static_cast<int64_t>(cfg->n_layers) * cfg->batch * cfg->n_q_heads * kD * 4);
     if (ok) ok = cudaMemset(c->status, 0, 256) == cudaSuccess;
-    if (ok) ok = cudaMemset(c->tickets, 0, pairs * 8) == cudaSuccess;
+    if (ok) ok = cudaMemset(c->tickets, 0, pairs * 128) == cudaSuccess;
     // the fp store must never hold non-finite garbage in unused slots of a partly filled tile
     if (ok) ok = cudaMemset(cv.fp, 0, static_cast<size_t>(cv.fp_layer_stride) * cfg->n_layers) == cudaSuccess;
     if (!ok) {
@@ -339,6 +339,7 @@ lq_status_t lq_decode_attn(lq_cache_t* c, int32_t layer, const void* q, float sm
   if (timed) cudaEventRecord(c->ev_pool[c->ev_used], st);
   a.tiles_fp = a.tiles_quant = 0;
   a.zero = 0;
+  a.n_extra = 0;
   if (use_mma(c)) {
     plan_decode_mma(a, c->sm_count, c->max_splits, c->cfg.n_splits);
     a.tickets = c->tickets;  // the CTA that completes a (b, kv) pair merges it: no second launch
@@ -426,6 +427,7 @@ lq_status_t lq_profile_read(lq_cache_t* c, double* total_ms, int64_t* n_launches
 }
 
 
+
 lq_status_t lq_kernel_status(lq_cache_t* c, int32_t* word) {
   if (!c || !word) return LQ_ERR_INVALID_ARG;
   *word = 0;
@@ -456,8 +458,8 @@ lq_status_t lq_cache_info(const lq_cache_t* c, int32_t layer, lq_info_t* info) {
     a.n_fp = L.n_fp;
     a.n_quant = L.n_quant;
     plan_decode_mma(a, c->sm_count, c->max_splits, c->cfg.n_splits);
-    info->n_splits = a.S;
-    info->n_ctas = a.S * c->cfg.batch * c->cfg.n_kv_heads;
+    info->n_splits = a.S - 1;
+    info->n_ctas = (a.S - 1) * c->cfg.batch * c->cfg.n_kv_heads + a.n_extra;
   } else
     info->n_splits = choose_splits(c, L);
   return LQ_OK;

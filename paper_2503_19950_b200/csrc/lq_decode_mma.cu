@@ -36,17 +36,16 @@ namespace lq {
 namespace {
 
 constexpr int kWarps = 4;
-#ifndef LQ_STAGE_BYTES
-#define LQ_STAGE_BYTES 6144
-#endif
-constexpr int kStageBytes = LQ_STAGE_BYTES;  // two G=32 tiles, one G=64 tile, or half an fp tile (K rows / V rows)
-#ifndef LQ_STAGES
-#define LQ_STAGES 2
-#endif
+// every warp owns 12 KB of stages: 2 x 6 KB, each holding two G = 32 tiles (3 KB), one G = 64 tile
+// (5 KB) or half an fp tile (K rows or V rows, 4 KB).  Claims of two tiles measured faster than
+// single tiles (1.55 vs 1.9 us per tile and warp): the per-claim bookkeeping is not free.
+constexpr int kWarpStageBytes = 12288;
+__host__ __device__ constexpr int stage_bytes(int) { return 6144; }
+__host__ __device__ constexpr int n_stages(int G) { return kWarpStageBytes / stage_bytes(G); }
+constexpr int kMaxStages = 3;
 #ifndef LQ_CTAS_PER_SM
 #define LQ_CTAS_PER_SM 4
 #endif
-constexpr int kStages = LQ_STAGES;
 constexpr int kCtasPerSm = LQ_CTAS_PER_SM;
 constexpr uint32_t kFull = 0xFFFFFFFFu;
 constexpr int kSpinLimit = 1 << 22;
@@ -516,11 +515,11 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
 }
 
 // shared memory: [per-warp stages][query rows of the pair][mbarriers][flags]
-constexpr int kSmemStages = kWarps * kStages * kStageBytes;
+constexpr int kSmemStages = kWarps * kWarpStageBytes;
 constexpr int kSmemQ = kMaxRatio * kD * 2;
-constexpr int kSmemBars = (kWarps * kStages + 1) * 8;
+constexpr int kSmemBars = (kWarps * kMaxStages + 1) * 8;
 constexpr int kSmemBytes = kSmemStages + kSmemQ + kSmemBars + 16;
-constexpr int kMergeMax = kStageBytes >= 5120 ? 2048 : 1024;  // S * r records the fused second pass can stage
+constexpr int kMergeMax = 2048;  // S * r records the fused second pass can stage
 
 // Work items of one (b, kv) pair, in queue order: fp tiles [0, tiles_fp), then quant tiles.  The S
 // CTAs of the pair (4 warps each) pull items one at a time from a global counter, so every warp of
@@ -536,29 +535,34 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   const int n = lane >> 2, j = lane & 3;
   const uint32_t oddmask = (n & 1) ? 0xFFFFFFFFu : 0u;
   constexpr int TILE = quant_tile_bytes(G);
-  static_assert((TILE <= kStageBytes || G == 64) && kFpTileVOffset <= kStageBytes, "stage too small");
+  constexpr int kStages = n_stages(G), kStageBytes = stage_bytes(G);
+  static_assert(TILE <= kStageBytes && kFpTileVOffset <= kStageBytes && kStages <= kMaxStages, "stage geometry");
 
-  const int pair = blockIdx.x / a.S, slot = blockIdx.x % a.S;
+  // pairs [0, n_extra) have S CTAs each, the others S - 1 (a.S is also the record stride)
+  int pair, slot, n_ctas_pair;
+  {
+    const int c = blockIdx.x, big = a.n_extra * a.S;
+    if (c < big) { pair = c / a.S; slot = c % a.S; n_ctas_pair = a.S; }
+    else { pair = a.n_extra + (c - big) / (a.S - 1); slot = (c - big) % (a.S - 1); n_ctas_pair = a.S - 1; }
+  }
   const int b = pair / cv.Hkv, kv = pair % cv.Hkv;
-  constexpr int TPS = kStageBytes / quant_tile_bytes(G);  // quant tiles per claim (and per stage)
+  constexpr int TPS = kStageBytes / TILE;  // quant tiles per claim (and per stage)
   const int n_items = a.tiles_fp + (a.tiles_quant + TPS - 1) / TPS;
-  int* queue = a.tickets + 2 * pair;
+  int* queue = a.tickets + 32 * pair;  // one 128-byte line per pair: [0] work-queue head, [1] arrival ticket
 
-  const uint32_t stage0 = smem_u32(smem + warp * (kStages * kStageBytes));
+  const uint32_t stage0 = smem_u32(smem + warp * kWarpStageBytes);
   const uint32_t qsm = smem_u32(smem + kSmemStages);
-  const uint32_t bar0 = smem_u32(smem + kSmemStages + kSmemQ) + warp * kStages * 8;
-  const uint32_t qbar = smem_u32(smem + kSmemStages + kSmemQ) + kWarps * kStages * 8;
+  const uint32_t bar0 = smem_u32(smem + kSmemStages + kSmemQ) + warp * kMaxStages * 8;
+  const uint32_t qbar = smem_u32(smem + kSmemStages + kSmemQ) + kWarps * kMaxStages * 8;
   int* is_last = reinterpret_cast<int*>(smem + kSmemStages + kSmemQ + kSmemBars);
 
-  // Programmatic dependent launch: let the next kernel of the stream start launching, and do
-  // not touch anything an earlier kernel may still be writing before it has finished.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // Programmatic dependent launch: do not touch anything an earlier kernel may still be writing
+  // before it has finished (the matching launch_dependents comes after the main loop).
   asm volatile("griddepcontrol.wait;" ::: "memory");
-
   // claims: the first kStages items of every warp are fixed (item = warp index + i * #warps), the
   // rest come from the pair's counter; lane 0 keeps the next dynamic claim in `pref`, an atomicAdd
   // issued one step ahead so that its latency hides behind the tile being processed
-  const int n_warps = a.S * kWarps, gw = slot * kWarps + warp;
+  const int n_warps = n_ctas_pair * kWarps, gw = slot * kWarps + warp;
   int pref = 0;
   if (lane == 0) {
     pref = atomicAdd(queue, 1) + kStages * n_warps;
@@ -707,6 +711,9 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     __syncwarp();
     issue_next();
   }
+  // the main loop is over: from here on the next kernel of the stream may start launching into
+  // the slots that free up (earlier, its waiting CTAs would only take issue slots from this loop)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (lane == 0 && pref < 0) atomicOr(a.status, 2);  // never true; makes sure the last claim has returned
   if (failed) {
     // a bulk copy never completed: flag it and contribute nothing (checked again at the end)
@@ -787,19 +794,32 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
           o = fmaf(wout[(w * kD + d) * 8 + h], f, o);
           L = fmaf(wl[w * 8 + h], f, L);
         }
-      a.part_o[(rec + h) * kD + d] = o;
-      if (d == 0) {
-        a.part_ml[(rec + h) * 2 + 0] = M;
-        a.part_ml[(rec + h) * 2 + 1] = L;
+      if (n_ctas_pair == 1) {
+        // the only CTA of its pair: this is the final result
+        const int64_t oi = (static_cast<int64_t>(b) * cv.Hq + kv * r + h) * kD + d;
+        const float res = o / L;
+        if (a.out_bf16)
+          static_cast<__nv_bfloat16*>(a.out)[oi] = __float2bfloat16_rn(res);
+        else
+          static_cast<float*>(a.out)[oi] = res;
+      } else {
+        a.part_o[(rec + h) * kD + d] = o;
+        if (d == 0) {
+          a.part_ml[(rec + h) * 2 + 0] = M;
+          a.part_ml[(rec + h) * 2 + 1] = L;
+        }
       }
     }
   }
+  if (n_ctas_pair == 1) {
+    if (threadIdx.x == 0) queue[0] = 0;  // all claims of this CTA have returned (checked above)
+  } else {
   // ---- second pass, fused: the CTA that completes a pair (last ticket) merges its S partials.
   // Nobody waits for anybody: a CTA either finds that it is last, or leaves.
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) {
-    const int last = atomicAdd(queue + 1, 1) == a.S - 1;
+    const int last = atomicAdd(queue + 1, 1) == n_ctas_pair - 1;
     if (last) { queue[0] = 0; queue[1] = 0; }  // every claim of every CTA has returned: ready for the next launch
     *is_last = last;
   }
@@ -811,7 +831,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     float* sm_l = sm_m + kMergeMax;
     float* sm_w = sm_l + kMergeMax;
     float* red = sm_w + kMergeMax;  // [warp][r][128] partial sums
-    const int nrec = a.S * r;
+    const int nrec = n_ctas_pair * r;
     for (int t = threadIdx.x; t < nrec; t += kWarps * 32) {
       sm_m[t] = __ldcg(a.part_ml + (rec0 + t) * 2);
       sm_l[t] = __ldcg(a.part_ml + (rec0 + t) * 2 + 1);
@@ -820,12 +840,12 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     if (threadIdx.x < r) {
       const int h = threadIdx.x;
       float M = -INFINITY, L = 0.f;
-      for (int s = 0; s < a.S; ++s)
+      for (int s = 0; s < n_ctas_pair; ++s)
         if (sm_l[s * r + h] > 0.f) M = fmaxf(M, sm_m[s * r + h]);
-      for (int s = 0; s < a.S; ++s)
+      for (int s = 0; s < n_ctas_pair; ++s)
         if (sm_l[s * r + h] > 0.f) L = fmaf(sm_l[s * r + h], exp2f(sm_m[s * r + h] - M), L);
       const float inv = 1.0f / L;
-      for (int s = 0; s < a.S; ++s)
+      for (int s = 0; s < n_ctas_pair; ++s)
         sm_w[s * r + h] = sm_l[s * r + h] > 0.f ? exp2f(sm_m[s * r + h] - M) * inv : 0.f;
     }
     __syncthreads();
@@ -833,7 +853,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     // independent, and the four warp sums meet in shared memory
     for (int h = 0; h < r; ++h) {
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int s = warp; s < a.S; s += kWarps) {
+      for (int s = warp; s < n_ctas_pair; s += kWarps) {
         const float4 v = __ldcg(reinterpret_cast<const float4*>(a.part_o + (rec0 + s * r + h) * kD) + lane);
         const float w = sm_w[s * r + h];
         acc.x = fmaf(v.x, w, acc.x); acc.y = fmaf(v.y, w, acc.y);
@@ -853,9 +873,10 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
         static_cast<float*>(a.out)[oi] = o;
     }
   }
+  }  // ticket path
   if (failed) {
     // give copies still in flight a bounded chance to land before the shared memory is released
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < n_stages(G); ++s) {
       int spins = 0;
       while (!mbar_try_wait(bar0 + 8 * s, 0) && !mbar_try_wait(bar0 + 8 * s, 1) && ++spins < 1024) {}
     }
@@ -869,15 +890,25 @@ void plan_decode_mma(DecodeArgs& a, int sm_count, int max_records, int s_overrid
   const int r = a.cv.Hq / a.cv.Hkv;
   a.tiles_fp = (a.n_fp + kFpTileSlots - 1) / kFpTileSlots;
   a.tiles_quant = static_cast<int>(a.n_quant / a.cv.G);
-  const int items = a.tiles_fp + a.tiles_quant / (kStageBytes / quant_tile_bytes(a.cv.G));
+  const int items = a.tiles_fp + a.tiles_quant / (stage_bytes(a.cv.G) / quant_tile_bytes(a.cv.G));
   // at most one resident wave of CTAs in total: a CTA that had to wait for a free slot would start
   // when the others finish, and its pair's merge would wait for it
   const int ctas_per_sm = r <= 4 ? kCtasPerSm : kCtasPerSm - 1;  // the two-column-block variant needs more registers
   int S = s_override > 0 ? s_override : (ctas_per_sm * sm_count) / pairs;
   S = std::min(S, (items + kWarps - 1) / kWarps);  // at least one item per warp
-  S = std::min(S, max_records);
-  S = std::min(S, kMergeMax / r);
-  a.S = std::max(S, 1);
+  S = std::min(S, max_records - 1);
+  S = std::min(S, kMergeMax / r - 1);
+  S = std::max(S, 1);
+  // S CTAs for every pair, one more for the first n_extra pairs, so that the grid fills the wave
+  // exactly: every SM then carries the same number of CTAs (an SM with 4 CTAs runs each of them a
+  // third slower than an SM with 3, and the pair queues cannot move work between pairs)
+  int extra = 0;
+  if (s_override <= 0 && S + 1 <= max_records && (S + 1) * kWarps <= items) {
+    extra = ctas_per_sm * sm_count - S * pairs;
+    extra = std::max(0, std::min(extra, pairs));
+  }
+  a.n_extra = extra;
+  a.S = S + 1;  // record stride; pairs >= n_extra use S of them
 }
 
 cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
@@ -901,7 +932,7 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
     if (dev >= 0 && dev < 64) configured[dev][variant] = true;
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(a.cv.B * a.cv.Hkv * a.S);
+  cfg.gridDim = dim3(a.cv.B * a.cv.Hkv * (a.S - 1) + a.n_extra);
   cfg.blockDim = dim3(kWarps * 32);
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = st;

@@ -53,7 +53,10 @@ struct DecodeArgs {
   int layer;
   int n_fp;
   int64_t n_quant;
-  int S;  // split-K partitions (= CTAs of the attention kernel) per (b, kv); record (pair, s) at pair*S + s
+  int S;  // records reserved per (b, kv): record (pair, s) at pair*S + s.  Scalar kernel: every pair has S
+          // partitions.  Tensor-core kernel: pair p has S - 1 + (p < n_extra) CTAs, so that the grid is an
+          // exact multiple of the SM count (equal load on every SM)
+  int n_extra;
   int tiles_fp, tiles_quant;  // fp tiles (16 slots) and quant tiles (G tokens) per (b, kv)
   int zero;                   // always 0; an opaque loop bound for the kernels
   float scale_log2;  // sm_scale * log2(e)
@@ -63,7 +66,8 @@ struct DecodeArgs {
   void* out;
   int out_bf16;
   int* status;  // device word; kernels OR error bits into it (bounded waits that gave up)
-  int* tickets; // per (b, kv): [0] work-queue head, [1] arrival counter of the fused second pass; both 0 at rest
+  int* tickets; // one 128-byte line per (b, kv): [0] work-queue head, [1] arrival counter of the fused second
+                // pass; both 0 at rest
                 // (null: static split and a separate merge launch)
 };
 
