@@ -751,22 +751,26 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   }
 
   // ---- CTA merge of the 4 warp states through shared memory (the stages are idle now) ----
+  // wout[warp][head][d] with rows padded to 132 floats: conflict-free reads along d
+  constexpr int kRow = kD + 4;
   __syncthreads();
-  float* wout = reinterpret_cast<float*>(smem);  // [warp][d][8]
-  float* wm = wout + kWarps * kD * 8;            // [warp][8]
-  float* wl = wm + kWarps * 8;                   // [warp][8]
+  float* wout = reinterpret_cast<float*>(smem);      // [warp][8][kRow]
+  float* wm = wout + kWarps * 8 * kRow;              // [warp][8]
+  float* wl = wm + kWarps * 8;                       // [warp][8]
+  float* wf = wl + kWarps * 8;                       // [warp][8] factor of each warp state in the CTA state
+  float* cml = wf + kWarps * 8;                      // [8][2] (m, l) of the CTA state
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) {
     if (bf16_pv<NCB>()) {
-      float* o = wout + (warp * kD + 16 * mt + n) * 8 + j;
+      float* o = wout + (warp * 8 + j) * kRow + 16 * mt + n;
       o[0] = o0[mt];
-      o[64] = o1[mt];  // row + 8
+      o[8] = o1[mt];  // channel + 8
     } else {
-      float* o = wout + (warp * kD + 16 * mt + n) * 8 + 2 * j;
+      float* o = wout + (warp * 8 + 2 * j) * kRow + 16 * mt + n;
       o[0] = st.out[mt][0];
-      o[1] = st.out[mt][1];
-      o[64] = st.out[mt][2];
-      o[65] = st.out[mt][3];
+      o[kRow] = st.out[mt][1];
+      o[8] = st.out[mt][2];
+      o[kRow + 8] = st.out[mt][3];
     }
   }
   if (n == 0) {
@@ -777,27 +781,34 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     }
   }
   __syncthreads();
+  if (threadIdx.x < r) {
+    const int h = threadIdx.x;
+    float M = -INFINITY, L = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w)
+      if (wl[w * 8 + h] > 0.f) M = fmaxf(M, wm[w * 8 + h]);
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+      const float f = wl[w * 8 + h] > 0.f ? ex2(wm[w * 8 + h] - M) : 0.f;
+      wf[w * 8 + h] = f;
+      L = fmaf(wl[w * 8 + h], f, L);
+    }
+    cml[2 * h] = M;
+    cml[2 * h + 1] = L;
+  }
+  __syncthreads();
   const int d = threadIdx.x;
   const int64_t rec0 = static_cast<int64_t>(pair) * a.S * r;
   {
     const int64_t rec = rec0 + static_cast<int64_t>(slot) * r;
     for (int h = 0; h < r; ++h) {
-      float M = -INFINITY;
+      float o = 0.f;
 #pragma unroll
-      for (int w = 0; w < kWarps; ++w)
-        if (wl[w * 8 + h] > 0.f) M = fmaxf(M, wm[w * 8 + h]);
-      float o = 0.f, L = 0.f;
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w)
-        if (wl[w * 8 + h] > 0.f) {
-          const float f = exp2f(wm[w * 8 + h] - M);
-          o = fmaf(wout[(w * kD + d) * 8 + h], f, o);
-          L = fmaf(wl[w * 8 + h], f, L);
-        }
+      for (int w = 0; w < kWarps; ++w) o = fmaf(wout[(w * 8 + h) * kRow + d], wf[w * 8 + h], o);
       if (n_ctas_pair == 1) {
         // the only CTA of its pair: this is the final result
         const int64_t oi = (static_cast<int64_t>(b) * cv.Hq + kv * r + h) * kD + d;
-        const float res = o / L;
+        const float res = o / cml[2 * h + 1];
         if (a.out_bf16)
           static_cast<__nv_bfloat16*>(a.out)[oi] = __float2bfloat16_rn(res);
         else
@@ -805,8 +816,8 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
       } else {
         a.part_o[(rec + h) * kD + d] = o;
         if (d == 0) {
-          a.part_ml[(rec + h) * 2 + 0] = M;
-          a.part_ml[(rec + h) * 2 + 1] = L;
+          a.part_ml[(rec + h) * 2 + 0] = cml[2 * h];
+          a.part_ml[(rec + h) * 2 + 1] = cml[2 * h + 1];
         }
       }
     }
@@ -814,65 +825,65 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   if (n_ctas_pair == 1) {
     if (threadIdx.x == 0) queue[0] = 0;  // all claims of this CTA have returned (checked above)
   } else {
-  // ---- second pass, fused: the CTA that completes a pair (last ticket) merges its S partials.
-  // Nobody waits for anybody: a CTA either finds that it is last, or leaves.
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const int last = atomicAdd(queue + 1, 1) == n_ctas_pair - 1;
-    if (last) { queue[0] = 0; queue[1] = 0; }  // every claim of every CTA has returned: ready for the next launch
-    *is_last = last;
-  }
-  __syncthreads();
-  if (*is_last) {
-    __threadfence();
-    // weights first (S*r small records, staged in the idle stage memory) ...
-    float* sm_m = reinterpret_cast<float*>(smem);
-    float* sm_l = sm_m + kMergeMax;
-    float* sm_w = sm_l + kMergeMax;
-    float* red = sm_w + kMergeMax;  // [warp][r][128] partial sums
-    const int nrec = n_ctas_pair * r;
-    for (int t = threadIdx.x; t < nrec; t += kWarps * 32) {
-      sm_m[t] = __ldcg(a.part_ml + (rec0 + t) * 2);
-      sm_l[t] = __ldcg(a.part_ml + (rec0 + t) * 2 + 1);
+    // ---- second pass, fused: the CTA that completes a pair (last ticket) merges its partials.
+    // Nobody waits for anybody: a CTA either finds that it is last, or leaves.
+    __syncthreads();  // every partial store of this CTA has been issued
+    if (threadIdx.x == 0) {
+      __threadfence();  // release, cumulative over the stores the barrier ordered before this thread
+      const int last = atomicAdd(queue + 1, 1) == n_ctas_pair - 1;
+      if (last) { queue[0] = 0; queue[1] = 0; }  // every claim of every CTA has returned: ready for the next launch
+      *is_last = last;
     }
     __syncthreads();
-    if (threadIdx.x < r) {
-      const int h = threadIdx.x;
-      float M = -INFINITY, L = 0.f;
-      for (int s = 0; s < n_ctas_pair; ++s)
-        if (sm_l[s * r + h] > 0.f) M = fmaxf(M, sm_m[s * r + h]);
-      for (int s = 0; s < n_ctas_pair; ++s)
-        if (sm_l[s * r + h] > 0.f) L = fmaf(sm_l[s * r + h], exp2f(sm_m[s * r + h] - M), L);
-      const float inv = 1.0f / L;
-      for (int s = 0; s < n_ctas_pair; ++s)
-        sm_w[s * r + h] = sm_l[s * r + h] > 0.f ? exp2f(sm_m[s * r + h] - M) * inv : 0.f;
-    }
-    __syncthreads();
-    // ... then warp w sums the records s = w, w+4, ... with 16-byte loads (lane = 4 channels), all
-    // independent, and the four warp sums meet in shared memory
-    for (int h = 0; h < r; ++h) {
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int s = warp; s < n_ctas_pair; s += kWarps) {
-        const float4 v = __ldcg(reinterpret_cast<const float4*>(a.part_o + (rec0 + s * r + h) * kD) + lane);
-        const float w = sm_w[s * r + h];
-        acc.x = fmaf(v.x, w, acc.x); acc.y = fmaf(v.y, w, acc.y);
-        acc.z = fmaf(v.z, w, acc.z); acc.w = fmaf(v.w, w, acc.w);
+    if (*is_last) {
+      __threadfence();
+      // weights first (S*r small records, staged in the idle stage memory) ...
+      float* sm_m = reinterpret_cast<float*>(smem);
+      float* sm_l = sm_m + kMergeMax;
+      float* sm_w = sm_l + kMergeMax;
+      float* red = sm_w + kMergeMax;  // [warp][r][128] partial sums
+      const int nrec = n_ctas_pair * r;
+      for (int t = threadIdx.x; t < nrec; t += kWarps * 32) {
+        sm_m[t] = __ldcg(a.part_ml + (rec0 + t) * 2);
+        sm_l[t] = __ldcg(a.part_ml + (rec0 + t) * 2 + 1);
       }
-      reinterpret_cast<float4*>(red + (warp * r + h) * kD)[lane] = acc;
-    }
-    __syncthreads();
-    for (int h = 0; h < r; ++h) {
-      float o = 0.f;
+      __syncthreads();
+      if (threadIdx.x < r) {
+        const int h = threadIdx.x;
+        float M = -INFINITY, L = 0.f;
+        for (int s = 0; s < n_ctas_pair; ++s)
+          if (sm_l[s * r + h] > 0.f) M = fmaxf(M, sm_m[s * r + h]);
+        for (int s = 0; s < n_ctas_pair; ++s)
+          if (sm_l[s * r + h] > 0.f) L = fmaf(sm_l[s * r + h], exp2f(sm_m[s * r + h] - M), L);
+        const float inv = 1.0f / L;
+        for (int s = 0; s < n_ctas_pair; ++s)
+          sm_w[s * r + h] = sm_l[s * r + h] > 0.f ? exp2f(sm_m[s * r + h] - M) * inv : 0.f;
+      }
+      __syncthreads();
+      // ... then warp w sums the records s = w, w+4, ... with 16-byte loads (lane = 4 channels), all
+      // independent, and the four warp sums meet in shared memory
+      for (int h = 0; h < r; ++h) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s = warp; s < n_ctas_pair; s += kWarps) {
+          const float4 v = __ldcg(reinterpret_cast<const float4*>(a.part_o + (rec0 + s * r + h) * kD) + lane);
+          const float w = sm_w[s * r + h];
+          acc.x = fmaf(v.x, w, acc.x); acc.y = fmaf(v.y, w, acc.y);
+          acc.z = fmaf(v.z, w, acc.z); acc.w = fmaf(v.w, w, acc.w);
+        }
+        reinterpret_cast<float4*>(red + (warp * r + h) * kD)[lane] = acc;
+      }
+      __syncthreads();
+      for (int h = 0; h < r; ++h) {
+        float o = 0.f;
 #pragma unroll
-      for (int w = 0; w < kWarps; ++w) o += red[(w * r + h) * kD + d];
-      const int64_t oi = (static_cast<int64_t>(b) * cv.Hq + kv * r + h) * kD + d;
-      if (a.out_bf16)
-        static_cast<__nv_bfloat16*>(a.out)[oi] = __float2bfloat16_rn(o);
-      else
-        static_cast<float*>(a.out)[oi] = o;
+        for (int w = 0; w < kWarps; ++w) o += red[(w * r + h) * kD + d];
+        const int64_t oi = (static_cast<int64_t>(b) * cv.Hq + kv * r + h) * kD + d;
+        if (a.out_bf16)
+          static_cast<__nv_bfloat16*>(a.out)[oi] = __float2bfloat16_rn(o);
+        else
+          static_cast<float*>(a.out)[oi] = o;
+      }
     }
-  }
   }  // ticket path
   if (failed) {
     // give copies still in flight a bounded chance to land before the shared memory is released
@@ -917,7 +928,7 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
   if (a.cv.G == 32) kern = r <= 4 ? lq_decode_mma_kernel<32, 1> : lq_decode_mma_kernel<32, 2>;
   else if (a.cv.G == 64) kern = r <= 4 ? lq_decode_mma_kernel<64, 1> : lq_decode_mma_kernel<64, 2>;
   else return cudaErrorInvalidValue;
-  static_assert(kSmemStages >= static_cast<int>((kWarps * kD * 8 + 2 * kWarps * 8) * sizeof(float)) &&
+  static_assert(kSmemStages >= static_cast<int>((kWarps * 8 * (kD + 4) + 3 * kWarps * 8 + 16) * sizeof(float)) &&
                     kSmemStages >= (3 * kMergeMax + kWarps * kMaxRatio * kD) * 4,
                 "merge scratch");
   // opt in to the dynamic shared memory size once per (device, kernel variant)
