@@ -111,6 +111,11 @@ __device__ __forceinline__ uint32_t bf16x2_fma(uint32_t a, uint32_t b, uint32_t 
   asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
   return d;
 }
+__device__ __forceinline__ uint32_t bf16x2_neg(uint32_t a) {
+  uint32_t d;
+  asm("neg.bf16x2 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
 __device__ __forceinline__ float pow2i(int k) { return __int_as_float((k + 127) << 23); }  // 2^k, -126 <= k <= 127
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -267,16 +272,13 @@ __device__ __forceinline__ void transpose_p(const float (&p)[NCB][2], float (&pT
 }
 
 // NCB == 1: split the probabilities into bf16 hi (even columns) / lo (odd columns).
-// H = hi in every lane; P = hi in even, lo in odd columns; Pz = 0 in even, lo in odd columns.
-__device__ __forceinline__ void split_p_bf16(const float (&pT)[2][2], uint32_t oddmask, uint32_t (&H)[2],
-                                             uint32_t (&P)[2], uint32_t (&Pz)[2]) {
+// H = hi in every lane; P = hi in even, lo in odd columns.
+__device__ __forceinline__ void split_p_bf16(const float (&pT)[2][2], bool odd, uint32_t (&H)[2], uint32_t (&P)[2]) {
 #pragma unroll
   for (int th = 0; th < 2; ++th) {
     H[th] = pack_bf16x2(pT[th][0], pT[th][1]);
-    const float f0 = __uint_as_float((H[th] << 16) & oddmask);
-    const float f1 = __uint_as_float(H[th] & oddmask & 0xFFFF0000u);
-    P[th] = pack_bf16x2(pT[th][0] - f0, pT[th][1] - f1);
-    Pz[th] = P[th] & oddmask;
+    P[th] = H[th];
+    if (odd) P[th] = pack_bf16x2(pT[th][0] - bf16lo_f32(H[th]), pT[th][1] - bf16hi_f32(H[th]));
   }
 }
 
@@ -324,8 +326,8 @@ __device__ __forceinline__ void process_fp_keys(WarpState<NCB>& st, const uint32
   transpose_p<NCB>(s[0], pT, lane);
   // NCB == 1: only b0 (hi/lo by column); NCB == 2: b0 = hi, b1 = lo
   if (bf16_pv<NCB>()) {
-    uint32_t H[2], Pz[2];
-    split_p_bf16(pT, oddmask, H, b0, Pz);
+    uint32_t H[2];
+    split_p_bf16(pT, oddmask != 0u, H, b0);
     b1[0] = b1[1] = 0;
   } else {
 #pragma unroll
@@ -398,8 +400,9 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
         for (int cb = 0; cb < NCB; ++cb) {
 #pragma unroll
           for (int w = 0; w < 2; ++w) {
-            const uint32_t hi = bf16x2_mul(qs[cb][ks][w], s4[2 * kk + w]);
-            bq[cb][w] = bf16x2_fma(qs[cb][ks][w], s4[2 * kk + w], bf16x2_mul(hi, oddmask & 0xBF80BF80u));
+            // even columns RN(q*s); odd columns the exact residual q*s - RN(q*s)
+            bq[cb][w] = bf16x2_mul(qs[cb][ks][w], s4[2 * kk + w]);
+            if (oddmask) bq[cb][w] = bf16x2_fma(qs[cb][ks][w], s4[2 * kk + w], bf16x2_neg(bq[cb][w]));
           }
           mma_bf16(accb[cb][ks & 3], z0, z1, z2, z3, qs[cb][ks][0], qs[cb][ks][1]);
         }
@@ -432,8 +435,8 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
     transpose_p<NCB>(s[u], pT, lane);
     const uint4 vw = lds128(tile + qt_vcodes_off(G) + u * 512 + 16 * lane);
     if (bf16_pv<NCB>()) {
-      uint32_t H[2], P[2], Pz[2];
-      split_p_bf16(pT, oddmask, H, P, Pz);
+      uint32_t H[2], P[2];
+      split_p_bf16(pT, oddmask != 0u, H, P);
       // value zero: A = zero (bf16 pairs straight from the tile), value groups on rows
       {
         // rows n >= NG of this MMA repeat real rows; their sums land in zacc rows nobody reads
@@ -456,9 +459,11 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
       for (int g = 0; g < NG; ++g)
 #pragma unroll
         for (int th = 0; th < 2; ++th) {
-          const uint32_t hh = bf16x2_mul(H[th], sv[g][th]);
-          const uint32_t r1 = bf16x2_fma(H[th], sv[g][th], bf16x2_mul(hh, oddmask & 0xBF80BF80u));
-          bp[g][th] = bf16x2_fma(Pz[th], sv[g][th], r1);
+          bp[g][th] = bf16x2_mul(H[th], sv[g][th]);
+          if (oddmask) {
+            const uint32_t r1 = bf16x2_fma(H[th], sv[g][th], bf16x2_neg(bp[g][th]));
+            bp[g][th] = bf16x2_fma(P[th], sv[g][th], r1);
+          }
         }
       const uint32_t v0s = vw.x >> 8, v1s = vw.y >> 8, v2s = vw.z >> 8, v3s = vw.w >> 8;
 #define LQ_PV_STEP(MT)                                                                                        \
@@ -537,16 +542,19 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   constexpr int TILE = quant_tile_bytes(G);
   constexpr int kStages = n_stages(G), kStageBytes = stage_bytes(G);
   static_assert(TILE <= kStageBytes && kFpTileVOffset <= kStageBytes && kStages <= kMaxStages, "stage geometry");
-
-  // pairs [0, n_extra) have S CTAs each, the others S - 1 (a.S is also the record stride)
+  // CTA c works for pair c % P in slot c / P: pairs [0, n_extra) have S CTAs, the others S - 1 (a.S
+  // is also the record stride).  Interleaving gives every pair CTAs from every launch rank of the
+  // SMs, so no pair consists only of CTAs whose first loads queue behind everybody else's.
   int pair, slot, n_ctas_pair;
   {
-    const int c = blockIdx.x, big = a.n_extra * a.S;
-    if (c < big) { pair = c / a.S; slot = c % a.S; n_ctas_pair = a.S; }
-    else { pair = a.n_extra + (c - big) / (a.S - 1); slot = (c - big) % (a.S - 1); n_ctas_pair = a.S - 1; }
+    const int P = cv.B * cv.Hkv;
+    pair = blockIdx.x % P;
+    slot = blockIdx.x / P;
+    n_ctas_pair = pair < a.n_extra ? a.S : a.S - 1;
   }
   const int b = pair / cv.Hkv, kv = pair % cv.Hkv;
   constexpr int TPS = kStageBytes / TILE;  // quant tiles per claim (and per stage)
+  const int n_warps = n_ctas_pair * kWarps, gw = slot * kWarps + warp;
   const int n_items = a.tiles_fp + (a.tiles_quant + TPS - 1) / TPS;
   int* queue = a.tickets + 32 * pair;  // one 128-byte line per pair: [0] work-queue head, [1] arrival ticket
 
@@ -562,7 +570,6 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   // claims: the first kStages items of every warp are fixed (item = warp index + i * #warps), the
   // rest come from the pair's counter; lane 0 keeps the next dynamic claim in `pref`, an atomicAdd
   // issued one step ahead so that its latency hides behind the tile being processed
-  const int n_warps = n_ctas_pair * kWarps, gw = slot * kWarps + warp;
   int pref = 0;
   if (lane == 0) {
     pref = atomicAdd(queue, 1) + kStages * n_warps;
@@ -837,51 +844,87 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     __syncthreads();
     if (*is_last) {
       __threadfence();
-      // weights first (S*r small records, staged in the idle stage memory) ...
+      // The (m, l) records go to shared memory while the first batch of partial rows is already in
+      // flight; every record's weight is then computed by its own thread, and each warp sums whole
+      // rows (lane = 4 channels, 16-byte loads, kBatch independent loads at a time) of the heads it
+      // owns.  r >= 3: warp w owns heads w, w + 4; r < 3: the records of a head are split over 4 / r
+      // warps and the sums meet in shared memory.
+      constexpr int kBatch = 8;
       float* sm_m = reinterpret_cast<float*>(smem);
       float* sm_l = sm_m + kMergeMax;
       float* sm_w = sm_l + kMergeMax;
-      float* red = sm_w + kMergeMax;  // [warp][r][128] partial sums
+      float* red = sm_w + kMergeMax;  // [unit][128] partial sums (r < 3 only)
       const int nrec = n_ctas_pair * r;
-      for (int t = threadIdx.x; t < nrec; t += kWarps * 32) {
-        sm_m[t] = __ldcg(a.part_ml + (rec0 + t) * 2);
-        sm_l[t] = __ldcg(a.part_ml + (rec0 + t) * 2 + 1);
-      }
-      __syncthreads();
-      if (threadIdx.x < r) {
-        const int h = threadIdx.x;
-        float M = -INFINITY, L = 0.f;
-        for (int s = 0; s < n_ctas_pair; ++s)
-          if (sm_l[s * r + h] > 0.f) M = fmaxf(M, sm_m[s * r + h]);
-        for (int s = 0; s < n_ctas_pair; ++s)
-          if (sm_l[s * r + h] > 0.f) L = fmaf(sm_l[s * r + h], exp2f(sm_m[s * r + h] - M), L);
-        const float inv = 1.0f / L;
-        for (int s = 0; s < n_ctas_pair; ++s)
-          sm_w[s * r + h] = sm_l[s * r + h] > 0.f ? exp2f(sm_m[s * r + h] - M) * inv : 0.f;
-      }
-      __syncthreads();
-      // ... then warp w sums the records s = w, w+4, ... with 16-byte loads (lane = 4 channels), all
-      // independent, and the four warp sums meet in shared memory
-      for (int h = 0; h < r; ++h) {
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s = warp; s < n_ctas_pair; s += kWarps) {
-          const float4 v = __ldcg(reinterpret_cast<const float4*>(a.part_o + (rec0 + s * r + h) * kD) + lane);
-          const float w = sm_w[s * r + h];
-          acc.x = fmaf(v.x, w, acc.x); acc.y = fmaf(v.y, w, acc.y);
-          acc.z = fmaf(v.z, w, acc.z); acc.w = fmaf(v.w, w, acc.w);
-        }
-        reinterpret_cast<float4*>(red + (warp * r + h) * kD)[lane] = acc;
-      }
-      __syncthreads();
-      for (int h = 0; h < r; ++h) {
-        float o = 0.f;
+      const int np = r >= 3 ? 1 : 4 / r, n_units = r * np;
+      float4 v[kBatch];
+      if (warp < n_units) {
+        const int h = warp % r, p = warp / r;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) o += red[(w * r + h) * kD + d];
-        const int64_t oi = (static_cast<int64_t>(b) * cv.Hq + kv * r + h) * kD + d;
-        if (a.out_bf16)
-          static_cast<__nv_bfloat16*>(a.out)[oi] = __float2bfloat16_rn(o);
-        else
-          static_cast<float*>(a.out)[oi] = o;
+        for (int k = 0; k < kBatch; ++k) {
+          const int sr = p + k * np;
+          if (sr < n_ctas_pair) v[k] = __ldcg(reinterpret_cast<const float4*>(a.part_o + (rec0 + sr * r + h) * kD) + lane);
+        }
+      }
+      for (int t = threadIdx.x; t < nrec; t += kWarps * 32) {
+        const float2 ml = __ldcg(reinterpret_cast<const float2*>(a.part_ml) + rec0 + t);
+        sm_m[t] = ml.x;
+        sm_l[t] = ml.y;
+      }
+      __syncthreads();
+      for (int t = threadIdx.x; t < nrec; t += kWarps * 32) {
+        const int h = t % r;
+        float M = -INFINITY, L = 0.f;
+        for (int sr = 0; sr < n_ctas_pair; ++sr)
+          if (sm_l[sr * r + h] > 0.f) M = fmaxf(M, sm_m[sr * r + h]);
+        for (int sr = 0; sr < n_ctas_pair; ++sr)
+          if (sm_l[sr * r + h] > 0.f) L = fmaf(sm_l[sr * r + h], ex2(sm_m[sr * r + h] - M), L);
+        sm_w[t] = sm_l[t] > 0.f ? ex2(sm_m[t] - M) / L : 0.f;
+      }
+      __syncthreads();
+      for (int u = warp; u < n_units; u += kWarps) {
+        const int h = u % r, p = u / r;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s0 = p; s0 < n_ctas_pair; s0 += kBatch * np) {
+          if (u != warp || s0 != p) {
+#pragma unroll
+            for (int k = 0; k < kBatch; ++k) {
+              const int sr = s0 + k * np;
+              if (sr < n_ctas_pair)
+                v[k] = __ldcg(reinterpret_cast<const float4*>(a.part_o + (rec0 + sr * r + h) * kD) + lane);
+            }
+          }
+#pragma unroll
+          for (int k = 0; k < kBatch; ++k) {
+            const int sr = s0 + k * np;
+            if (sr < n_ctas_pair) {
+              const float w = sm_w[sr * r + h];
+              acc.x = fmaf(v[k].x, w, acc.x); acc.y = fmaf(v[k].y, w, acc.y);
+              acc.z = fmaf(v[k].z, w, acc.z); acc.w = fmaf(v[k].w, w, acc.w);
+            }
+          }
+        }
+        if (np == 1) {
+          const int64_t oi = (static_cast<int64_t>(b) * cv.Hq + kv * r + h) * kD + 4 * lane;
+          if (a.out_bf16)
+            *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(a.out) + oi) =
+                make_uint2(pack_bf16x2(acc.x, acc.y), pack_bf16x2(acc.z, acc.w));
+          else
+            *reinterpret_cast<float4*>(static_cast<float*>(a.out) + oi) = acc;
+        } else {
+          reinterpret_cast<float4*>(red + u * kD)[lane] = acc;
+        }
+      }
+      if (np > 1) {
+        __syncthreads();
+        for (int h = 0; h < r; ++h) {
+          float o = 0.f;
+          for (int p = 0; p < np; ++p) o += red[(h + r * p) * kD + d];
+          const int64_t oi = (static_cast<int64_t>(b) * cv.Hq + kv * r + h) * kD + d;
+          if (a.out_bf16)
+            static_cast<__nv_bfloat16*>(a.out)[oi] = __float2bfloat16_rn(o);
+          else
+            static_cast<float*>(a.out)[oi] = o;
+        }
       }
     }
   }  // ticket path
