@@ -83,6 +83,14 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// same with a zero accumulator input (no registers to clear)
+__device__ __forceinline__ void mma_bf16_z(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                           uint32_t b0, uint32_t b1) {
+  asm(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
+}
 __device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                         uint32_t b0, uint32_t b1) {
   asm(
@@ -290,12 +298,6 @@ __device__ __forceinline__ void process_fp_keys(WarpState<NCB>& st, const uint32
                                                 int opaque_zero, uint32_t (&b0)[2], uint32_t (&b1)[2]) {
   const int n = lane >> 2;
   float acc[NCB][4][4];
-#pragma unroll
-  for (int cb = 0; cb < NCB; ++cb)
-#pragma unroll
-    for (int c = 0; c < 4; ++c)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) acc[cb][c][e] = 0.f;
   {
     const int mi = lane >> 3, rr = lane & 7;
     const int token = rr + 8 * (mi & 1);
@@ -306,7 +308,10 @@ __device__ __forceinline__ void process_fp_keys(WarpState<NCB>& st, const uint32
       uint32_t a0, a1, a2, a3;
       ldmatrix_x4(rowaddr + ((chunk ^ (token & 7)) << 4), a0, a1, a2, a3);
 #pragma unroll
-      for (int cb = 0; cb < NCB; ++cb) mma_bf16(acc[cb][ks & 3], a0, a1, a2, a3, qs[cb][ks][0], qs[cb][ks][1]);
+      for (int cb = 0; cb < NCB; ++cb) {
+        if (ks < 4) mma_bf16_z(acc[cb][ks & 3], a0, a1, a2, a3, qs[cb][ks][0], qs[cb][ks][1]);
+        else mma_bf16(acc[cb][ks & 3], a0, a1, a2, a3, qs[cb][ks][0], qs[cb][ks][1]);
+      }
     }
   }
   float s[1][NCB][2];
@@ -354,17 +359,48 @@ __device__ __forceinline__ void process_fp_values(WarpState<NCB>& st, uint32_t v
   }
 }
 
+// ---- q.zero of the key groups of one claim: bias[t][cb] for head 4cb + lane%4 of tile t (log2 units).
+// One MMA per k-step serves two tiles: the A fragment's rows 0-7 repeat the zero row of tile 0 and
+// rows 8-15 that of tile 1 (ldmatrix with equal row addresses inside each 8x8 matrix); the four
+// accumulators collect the k-steps of equal code-position factor, which kc[] undoes.
+// zaddr: this lane's row address, k-step 0.
+template <int NCB>
+__device__ __forceinline__ void quant_bias(const uint32_t (&qs)[NCB][8][2], uint32_t zaddr, const float (&kc)[4],
+                                           float (&bias)[2][NCB]) {
+  float accb[NCB][4][4];
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks) {
+    uint32_t z0, z1, z2, z3;
+    ldmatrix_x4(zaddr + 32 * ks, z0, z1, z2, z3);
+#pragma unroll
+    for (int cb = 0; cb < NCB; ++cb) {
+      if (ks < 4) mma_bf16_z(accb[cb][ks & 3], z0, z1, z2, z3, qs[cb][ks][0], qs[cb][ks][1]);
+      else mma_bf16(accb[cb][ks & 3], z0, z1, z2, z3, qs[cb][ks][0], qs[cb][ks][1]);
+    }
+  }
+#pragma unroll
+  for (int cb = 0; cb < NCB; ++cb) {
+    float b0 = accb[cb][0][0] * kc[0], b1 = accb[cb][0][2] * kc[0];
+#pragma unroll
+    for (int c = 1; c < 4; ++c) {
+      b0 = fmaf(accb[cb][c][0], kc[c], b0);
+      b1 = fmaf(accb[cb][c][2], kc[c], b1);
+    }
+    bias[0][cb] = b0;
+    bias[1][cb] = b1;
+  }
+}
+
 // ---- one quant tile: one key group of G tokens ---------------------------------------------
 template <int G, int NCB>
 __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uint32_t (&qs)[NCB][8][2], uint32_t tile,
-                                                   const float (&kc)[4], float kq, int lane, uint32_t oddmask,
+                                                   const float (&bias)[NCB], float kq, int lane, uint32_t oddmask,
                                                    int opaque_zero) {
   constexpr int NS = G / 16, NG = kD / G, VS = vsz_subtile_bytes(G);
   const int n = lane >> 2, j = lane & 3;
   // ---- q.k on all G tokens.  Per pair of k-steps: the key scale of the lane's channels is folded
-  // into the query (even columns RN(q*s), odd columns the exact residual), the group's q.zero
-  // bias advances by one MMA per k-step (A = zero rows via ldmatrix with equal row addresses),
-  // and every sub-tile's score accumulator advances by one MMA per k-step.
+  // into the query (even columns RN(q*s), odd columns the exact residual) and every sub-tile's
+  // score accumulator advances by one MMA per k-step; the group's q.zero comes in as `bias`.
   float s[NS][NCB][2];
   {
     uint32_t kw[NS][4], kws[NS][4];
@@ -377,15 +413,6 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
       for (int e = 0; e < 4; ++e) kws[u][e] = kw[u][e] >> 8;
     }
     float acc[NS][NCB][4];
-    float accb[NCB][4][4];
-#pragma unroll
-    for (int cb = 0; cb < NCB; ++cb) {
-#pragma unroll
-      for (int u = 0; u < NS; ++u) acc[u][cb][0] = acc[u][cb][1] = acc[u][cb][2] = acc[u][cb][3] = 0.f;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) accb[cb][c][0] = accb[cb][c][1] = accb[cb][c][2] = accb[cb][c][3] = 0.f;
-    }
-    const uint32_t zaddr = tile + qt_kzero_off() + ((lane >> 4) << 4);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const uint4 sw = lds128(tile + qt_kscale_off() + 16 * (4 * i + j));
@@ -393,8 +420,6 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
 #pragma unroll
       for (int kk = 0; kk < 2; ++kk) {
         const int ks = 2 * i + kk;
-        uint32_t z0, z1, z2, z3;
-        ldmatrix_x4(zaddr + 32 * ks, z0, z1, z2, z3);
         uint32_t bq[NCB][2];
 #pragma unroll
         for (int cb = 0; cb < NCB; ++cb) {
@@ -404,26 +429,25 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
             bq[cb][w] = bf16x2_mul(qs[cb][ks][w], s4[2 * kk + w]);
             if (oddmask) bq[cb][w] = bf16x2_fma(qs[cb][ks][w], s4[2 * kk + w], bf16x2_neg(bq[cb][w]));
           }
-          mma_bf16(accb[cb][ks & 3], z0, z1, z2, z3, qs[cb][ks][0], qs[cb][ks][1]);
         }
 #pragma unroll
         for (int u = 0; u < NS; ++u) {
           const uint32_t a0 = ext_bf16_i(ks, kw[u][0], kws[u][0]), a1 = ext_bf16_i(ks, kw[u][1], kws[u][1]),
                          a2 = ext_bf16_i(ks, kw[u][2], kws[u][2]), a3 = ext_bf16_i(ks, kw[u][3], kws[u][3]);
 #pragma unroll
-          for (int cb = 0; cb < NCB; ++cb) mma_bf16(acc[u][cb], a0, a1, a2, a3, bq[cb][0], bq[cb][1]);
+          for (int cb = 0; cb < NCB; ++cb) {
+            if (ks == 0) mma_bf16_z(acc[u][cb], a0, a1, a2, a3, bq[cb][0], bq[cb][1]);
+            else mma_bf16(acc[u][cb], a0, a1, a2, a3, bq[cb][0], bq[cb][1]);
+          }
         }
       }
     }
 #pragma unroll
     for (int cb = 0; cb < NCB; ++cb) {
-      float bias = accb[cb][0][0] * kc[0];
-#pragma unroll
-      for (int c = 1; c < 4; ++c) bias = fmaf(accb[cb][c][0], kc[c], bias);
 #pragma unroll
       for (int u = 0; u < NS; ++u) {
-        s[u][cb][0] = fmaf(acc[u][cb][0] + acc[u][cb][1], kq, bias);
-        s[u][cb][1] = fmaf(acc[u][cb][2] + acc[u][cb][3], kq, bias);
+        s[u][cb][0] = fmaf(acc[u][cb][0] + acc[u][cb][1], kq, bias[cb]);
+        s[u][cb][1] = fmaf(acc[u][cb][2] + acc[u][cb][3], kq, bias[cb]);
       }
     }
   }
@@ -707,8 +731,16 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
         sw = a.zero;
       }
       const int nt = min(TPS, a.tiles_quant - (desc - a.tiles_fp) * TPS);
+      float bias2[2][NCB];
+      quant_bias<NCB>(qs, sbase + qt_kzero_off() + ((lane >> 4) << 4) + (((lane >> 3) & 1) && nt > 1 ? TILE : 0), kc,
+                      bias2);
 #pragma unroll 1
-      for (int t = 0; t < nt; ++t) process_quant_tile<G, NCB>(st, qs, sbase + t * TILE, kc, kq, lane, oddmask, a.zero);
+      for (int t = 0; t < nt; ++t) {
+        float bias[NCB];
+#pragma unroll
+        for (int cb = 0; cb < NCB; ++cb) bias[cb] = t ? bias2[1][cb] : bias2[0][cb];
+        process_quant_tile<G, NCB>(st, qs, sbase + t * TILE, bias, kq, lane, oddmask, a.zero);
+      }
     } else if (desc >= 0) {
       const int nv = min(16, a.n_fp - desc * 16);
       process_fp_keys<NCB>(st, qs, sbase, nv, kc, lane, oddmask, a.zero, fb0, fb1);
