@@ -1,13 +1,13 @@
 // Tensor-core decode attention over the mixed cache (LQ_KERNEL_MMA): split-K first pass.
 //
-// Work partition: the tiles of all (b, kv head) pairs are laid on one cost line and cut into
-// equal ranges, one per CTA (a multiple of the SM count), so every SM gets the same instruction
-// load whatever the batch size; a CTA that straddles a pair boundary simply emits one split-K
-// partial per pair it touches.  Inside a CTA each of the 4 warps owns a private ring of
-// shared-memory stages filled by 1-D bulk copies (cp.async.bulk + mbarrier, no multicast) and a
-// private online-softmax state (m, l, o); the CTA merges the warp states into the partial (Eq. 3
-// makes any visiting order legal).  Units: fp tiles (16 bf16 tokens, 8 KB) first, then quant
-// tiles (one key group of G tokens each).
+// Work partition: every (b, kv) pair gets S or S + 1 CTAs so that the grid is exactly one resident
+// wave (4 CTAs per SM, 3 for more than 4 query heads per KV head); inside a pair the items -- fp
+// tiles (16 bf16 tokens, 8 KB) first, then quant tiles (one key group of G tokens each) -- are
+// divided statically among the pair's warps by cost.  Each of the 4 warps of a CTA owns a private
+// ring of shared-memory stages filled by 1-D bulk copies (cp.async.bulk + mbarrier, no multicast)
+// and a private online-softmax state (m, l, o); the CTA merges the warp states into one split-K
+// partial (Eq. 3 makes any visiting order legal), and the CTA that completes a pair merges the
+// pair's partials and writes the output.
 //
 // Contractions (mma.sync.m16n8k16, fp32 accumulate), r = query heads per KV head (<= 8):
 //   q.k   tokens on M (16), query heads on N, channels on K.  Heads are handled in column blocks
@@ -49,6 +49,10 @@ constexpr int kMaxStages = 3;
 constexpr int kCtasPerSm = LQ_CTAS_PER_SM;
 constexpr uint32_t kFull = 0xFFFFFFFFu;
 constexpr int kSpinLimit = 1 << 22;
+#ifndef LQ_FP_COST8
+#define LQ_FP_COST8 8
+#endif
+constexpr int kFpCost8 = LQ_FP_COST8;  // cost of one fp tile (16 bf16 tokens) in eighths of a quant tile
 
 // ---- PTX wrappers ----------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -550,11 +554,10 @@ constexpr int kSmemBars = (kWarps * kMaxStages + 1) * 8;
 constexpr int kSmemBytes = kSmemStages + kSmemQ + kSmemBars + 16;
 constexpr int kMergeMax = 2048;  // S * r records the fused second pass can stage
 
-// Work items of one (b, kv) pair, in queue order: fp tiles [0, tiles_fp), then quant tiles.  The S
-// CTAs of the pair (4 warps each) pull items one at a time from a global counter, so every warp of
-// every SM stays busy until the pair is finished whatever the speed of its SM; any assignment is
-// legal because every warp keeps its own online-softmax state.  A warp always has its next claim
-// in flight (the atomic's latency hides behind the tile being processed) and two loads in flight.
+// Work items of one (b, kv) pair, in order: fp tiles [0, tiles_fp), then quant tiles.  The CTAs of
+// the pair (4 warps each) share them by a static, cost-weighted partition (see below); any
+// assignment is legal because every warp keeps its own online-softmax state.  A warp keeps up to
+// two loads in flight.
 template <int G, int NCB>
 __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerSm - 1) lq_decode_mma_kernel(DecodeArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
@@ -579,8 +582,22 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   const int b = pair / cv.Hkv, kv = pair % cv.Hkv;
   constexpr int TPS = kStageBytes / TILE;  // quant tiles per claim (and per stage)
   const int n_warps = n_ctas_pair * kWarps, gw = slot * kWarps + warp;
-  const int n_items = a.tiles_fp + (a.tiles_quant + TPS - 1) / TPS;
-  int* queue = a.tickets + 32 * pair;  // one 128-byte line per pair: [0] work-queue head, [1] arrival ticket
+  // Static partition: the pair's items -- fp tiles (cost kFpCost8 / 8 each), then quant tiles (cost
+  // 1) -- lie on a cost line that is cut into n_warps equal ranges; warp gw takes the items between
+  // cut gw and cut gw + 1 (boundaries rounded to the nearest item).  Every SM carries the same number
+  // of identical warps, so equal work gives (nearly) equal finishing times without any work queue;
+  // weighting the ranges by the launch order of the CTAs on an SM measured slower.
+  int it, it_end;
+  {
+    const int F8 = a.tiles_fp * kFpCost8, C8 = F8 + a.tiles_quant * 8;
+    auto cut = [&](int k) {
+      const int pos8 = static_cast<int>(static_cast<int64_t>(k) * C8 / n_warps);
+      return pos8 < F8 ? (pos8 + kFpCost8 / 2) / kFpCost8 : a.tiles_fp + (pos8 - F8 + 4) / 8;
+    };
+    it = cut(gw);
+    it_end = cut(gw + 1);
+  }
+  int* queue = a.tickets + 32 * pair;  // one 128-byte line per pair: [1] is the arrival ticket
 
   const uint32_t stage0 = smem_u32(smem + warp * kWarpStageBytes);
   const uint32_t qsm = smem_u32(smem + kSmemStages);
@@ -591,12 +608,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   // Programmatic dependent launch: do not touch anything an earlier kernel may still be writing
   // before it has finished (the matching launch_dependents comes after the main loop).
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  // claims: the first kStages items of every warp are fixed (item = warp index + i * #warps), the
-  // rest come from the pair's counter; lane 0 keeps the next dynamic claim in `pref`, an atomicAdd
-  // issued one step ahead so that its latency hides behind the tile being processed
-  int pref = 0;
   if (lane == 0) {
-    pref = atomicAdd(queue, 1) + kStages * n_warps;
 #pragma unroll
     for (int s = 0; s < kStages; ++s) mbar_init(bar0 + 8 * s, 1);
     if (warp == 0) mbar_init(qbar, 1);
@@ -621,10 +633,9 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
 
   // load pipeline.  A stage holds: the K rows of fp tile i (desc = i), its V rows (desc = -1-i)
   // or quant tile t (desc = tiles_fp + t).  pending_v >= 0: the V rows of that fp tile come next.
-  int issued = 0, pending_v = -1, n_claims = 0;
-  bool drained = false;
+  int issued = 0, pending_v = -1;
   int desc0 = 0, desc1 = 0, desc2 = 0;
-  auto issue_next = [&]() {
+  auto issue_next = [&](int cap) {
     const uint8_t* src;
     uint32_t bytes;
     int desc;
@@ -634,25 +645,19 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
       src = fpbase + static_cast<int64_t>(pending_v) * kFpTileBytes + kFpTileVOffset;
       pending_v = -1;
     } else {
-      if (drained) return;
-      int item;
-      if (n_claims < kStages) {
-        item = gw + n_claims * n_warps;
-      } else {
-        item = __shfl_sync(kFull, pref, 0);
-        if (item < n_items && lane == 0) pref = atomicAdd(queue, 1) + kStages * n_warps;
-      }
-      ++n_claims;
-      if (item >= n_items) { drained = true; return; }
-      desc = item;
-      if (item < a.tiles_fp) {
+      if (it >= it_end) return;
+      desc = it;
+      if (it < a.tiles_fp) {
         bytes = kFpTileVOffset;
-        src = fpbase + static_cast<int64_t>(item) * kFpTileBytes;
-        pending_v = item;
+        src = fpbase + static_cast<int64_t>(it) * kFpTileBytes;
+        pending_v = it;
+        ++it;
       } else {
-        const int t0 = (item - a.tiles_fp) * TPS;
-        bytes = min(TPS, a.tiles_quant - t0) * TILE;
-        src = qbase + static_cast<int64_t>(t0) * TILE;
+        const int nt = min(min(TPS, cap), it_end - it);
+        desc = it | (nt << 24);
+        bytes = nt * TILE;
+        src = qbase + static_cast<int64_t>(it - a.tiles_fp) * TILE;
+        it += nt;
       }
     }
     const uint32_t s = issued % kStages;
@@ -664,8 +669,9 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     ++issued;
   };
   bool failed = false;
-#pragma unroll
-  for (int s = 0; s < kStages; ++s) issue_next();
+  // Only one small load per warp before the query fragments are built: all warps start at the same
+  // time, and the first bytes every warp needs should not queue behind everybody's second load.
+  issue_next(1);
 
   // query fragments: B operand, column n -> head 4cb + n/2 (even column = hi, odd = lo of q*s);
   // k-step ks carries the factor 2^(64 - 2*(ks&3)) that cancels the code-position factor
@@ -692,6 +698,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
         }
     }
   }
+  for (int s = 1; s < kStages; ++s) issue_next(TPS);
   WarpState<NCB> st;
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) st.out[mt][0] = st.out[mt][1] = st.out[mt][2] = st.out[mt][3] = 0.f;
@@ -716,7 +723,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     const uint32_t sbase = stage0 + s * kStageBytes;
     const int desc = s == 0 ? desc0 : (s == 1 ? desc1 : desc2);
     if (desc >= a.tiles_fp) {
-      // items come in queue order, so a warp sees all its fp tiles before its first quant tile: from
+      // items come in order, so a warp sees all its fp tiles before its first quant tile: from
       // here on the out rows carry the code-position factor (two steps keep the constants normal).
       // An opaque one-trip loop keeps this a branch instead of 64 multiplies and selects per tile.
       int sw = st.quant_mode ? 0 : 1;
@@ -730,7 +737,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
         st.quant_mode = true;
         sw = a.zero;
       }
-      const int nt = min(TPS, a.tiles_quant - (desc - a.tiles_fp) * TPS);
+      const int nt = desc >> 24;
       float bias2[2][NCB];
       quant_bias<NCB>(qs, sbase + qt_kzero_off() + ((lane >> 4) << 4) + (((lane >> 3) & 1) && nt > 1 ? TILE : 0), kc,
                       bias2);
@@ -748,12 +755,11 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
       process_fp_values<NCB>(st, sbase, lane, fb0, fb1);
     }
     __syncwarp();
-    issue_next();
+    issue_next(TPS);
   }
   // the main loop is over: from here on the next kernel of the stream may start launching into
   // the slots that free up (earlier, its waiting CTAs would only take issue slots from this loop)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (lane == 0 && pref < 0) atomicOr(a.status, 2);  // never true; makes sure the last claim has returned
   if (failed) {
     // a bulk copy never completed: flag it and contribute nothing (checked again at the end)
     if (lane == 0) atomicOr(a.status, 1);
@@ -862,7 +868,6 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     }
   }
   if (n_ctas_pair == 1) {
-    if (threadIdx.x == 0) queue[0] = 0;  // all claims of this CTA have returned (checked above)
   } else {
     // ---- second pass, fused: the CTA that completes a pair (last ticket) merges its partials.
     // Nobody waits for anybody: a CTA either finds that it is last, or leaves.
@@ -870,7 +875,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     if (threadIdx.x == 0) {
       __threadfence();  // release, cumulative over the stores the barrier ordered before this thread
       const int last = atomicAdd(queue + 1, 1) == n_ctas_pair - 1;
-      if (last) { queue[0] = 0; queue[1] = 0; }  // every claim of every CTA has returned: ready for the next launch
+      if (last) queue[1] = 0;  // ready for the next launch
       *is_last = last;
     }
     __syncthreads();
@@ -987,7 +992,7 @@ void plan_decode_mma(DecodeArgs& a, int sm_count, int max_records, int s_overrid
   S = std::max(S, 1);
   // S CTAs for every pair, one more for the first n_extra pairs, so that the grid fills the wave
   // exactly: every SM then carries the same number of CTAs (an SM with 4 CTAs runs each of them a
-  // third slower than an SM with 3, and the pair queues cannot move work between pairs)
+  // third slower than an SM with 3, and work does not move between pairs)
   int extra = 0;
   if (s_override <= 0 && S + 1 <= max_records && (S + 1) * kWarps <= items) {
     extra = ctas_per_sm * sm_count - S * pairs;

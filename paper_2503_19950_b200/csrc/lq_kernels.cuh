@@ -66,8 +66,8 @@ struct DecodeArgs {
   void* out;
   int out_bf16;
   int* status;  // device word; kernels OR error bits into it (bounded waits that gave up)
-  int* tickets; // one 128-byte line per (b, kv): [0] work-queue head, [1] arrival counter of the fused second
-                // pass; both 0 at rest
+  int* tickets; // one 128-byte line per (b, kv): word [1] is the arrival counter of the fused second
+                // pass, 0 at rest
                 // (null: static split and a separate merge launch)
 };
 
