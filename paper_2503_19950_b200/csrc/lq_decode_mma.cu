@@ -881,87 +881,91 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     __syncthreads();
     if (*is_last) {
       __threadfence();
-      // The (m, l) records go to shared memory while the first batch of partial rows is already in
-      // flight; every record's weight is then computed by its own thread, and each warp sums whole
-      // rows (lane = 4 channels, 16-byte loads, kBatch independent loads at a time) of the heads it
-      // owns.  r >= 3: warp w owns heads w, w + 4; r < 3: the records of a head are split over 4 / r
-      // warps and the sums meet in shared memory.
-      constexpr int kBatch = 8;
-      float* sm_m = reinterpret_cast<float*>(smem);
-      float* sm_l = sm_m + kMergeMax;
-      float* sm_w = sm_l + kMergeMax;
-      float* red = sm_w + kMergeMax;  // [unit][128] partial sums (r < 3 only)
-      const int nrec = n_ctas_pair * r;
-      const int np = r >= 3 ? 1 : 4 / r, n_units = r * np;
-      float4 v[kBatch];
-      if (warp < n_units) {
-        const int h = warp % r, p = warp / r;
+      // Warp w sums the records of the CTAs s = w, w + 4, ... for every head (lane = 4 channels,
+      // 16-byte loads, kSB * RMAX independent loads in flight; the first batch is issued before the
+      // weights are known), and the four warp sums meet in shared memory.  The weight of a record
+      // is computed by the lane that loaded its (m, l): warp w normalises heads w, w + 4.
+      constexpr int RMAX = NCB == 1 ? 4 : 8;  // query heads per KV head this variant serves
+      constexpr int kSB = NCB == 1 ? 3 : 2;   // CTA records per batch
+      float* sm_w = reinterpret_cast<float*>(smem);  // [S * r] weights
+      float* red = sm_w + kMergeMax;                 // [warp][r][128] partial sums
+      const int nS = n_ctas_pair;
+      auto row = [&](int sr, int h) {
+        return __ldcg(reinterpret_cast<const float4*>(a.part_o + (rec0 + sr * r + h) * kD) + lane);
+      };
+      float4 v[kSB][RMAX];
 #pragma unroll
-        for (int k = 0; k < kBatch; ++k) {
-          const int sr = p + k * np;
-          if (sr < n_ctas_pair) v[k] = __ldcg(reinterpret_cast<const float4*>(a.part_o + (rec0 + sr * r + h) * kD) + lane);
+      for (int i = 0; i < kSB; ++i)
+#pragma unroll
+        for (int h = 0; h < RMAX; ++h)
+          if (h < r && warp + 4 * i < nS) v[i][h] = row(warp + 4 * i, h);
+      for (int h = warp; h < r; h += kWarps) {
+        const float2* mlp = reinterpret_cast<const float2*>(a.part_ml) + rec0 + h;
+        const float2 ml0 = lane < nS ? __ldcg(mlp + lane * r) : make_float2(-INFINITY, 0.f);
+        auto ml_at = [&](int k0) {  // (m, l) of record k0 + lane; the first 32 stay in registers
+          if (k0 == 0) return ml0;
+          return k0 + lane < nS ? __ldcg(mlp + (k0 + lane) * r) : make_float2(-INFINITY, 0.f);
+        };
+        float M = -INFINITY;
+        for (int k0 = 0; k0 < nS; k0 += 32) {
+          const float2 ml = ml_at(k0);
+          if (ml.y > 0.f) M = fmaxf(M, ml.x);
         }
-      }
-      for (int t = threadIdx.x; t < nrec; t += kWarps * 32) {
-        const float2 ml = __ldcg(reinterpret_cast<const float2*>(a.part_ml) + rec0 + t);
-        sm_m[t] = ml.x;
-        sm_l[t] = ml.y;
+#pragma unroll
+        for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(kFull, M, o));
+        float L = 0.f;
+        for (int k0 = 0; k0 < nS; k0 += 32) {
+          const float2 ml = ml_at(k0);
+          if (ml.y > 0.f) L = fmaf(ml.y, ex2(ml.x - M), L);
+        }
+#pragma unroll
+        for (int o = 16; o; o >>= 1) L += __shfl_xor_sync(kFull, L, o);
+        const float inv = 1.0f / L;
+        for (int k0 = 0; k0 < nS; k0 += 32) {
+          const float2 ml = ml_at(k0);
+          if (k0 + lane < nS) sm_w[(k0 + lane) * r + h] = ml.y > 0.f ? ex2(ml.x - M) * inv : 0.f;
+        }
       }
       __syncthreads();
-      for (int t = threadIdx.x; t < nrec; t += kWarps * 32) {
-        const int h = t % r;
-        float M = -INFINITY, L = 0.f;
-        for (int sr = 0; sr < n_ctas_pair; ++sr)
-          if (sm_l[sr * r + h] > 0.f) M = fmaxf(M, sm_m[sr * r + h]);
-        for (int sr = 0; sr < n_ctas_pair; ++sr)
-          if (sm_l[sr * r + h] > 0.f) L = fmaf(sm_l[sr * r + h], ex2(sm_m[sr * r + h] - M), L);
-        sm_w[t] = sm_l[t] > 0.f ? ex2(sm_m[t] - M) / L : 0.f;
+      float4 acc[RMAX];
+#pragma unroll
+      for (int h = 0; h < RMAX; ++h) acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int s0 = warp; s0 < nS; s0 += 4 * kSB) {
+        if (s0 != warp) {
+#pragma unroll
+          for (int i = 0; i < kSB; ++i)
+#pragma unroll
+            for (int h = 0; h < RMAX; ++h)
+              if (h < r && s0 + 4 * i < nS) v[i][h] = row(s0 + 4 * i, h);
+        }
+#pragma unroll
+        for (int i = 0; i < kSB; ++i)
+#pragma unroll
+          for (int h = 0; h < RMAX; ++h)
+            if (h < r && s0 + 4 * i < nS) {
+              const float w = sm_w[(s0 + 4 * i) * r + h];
+              acc[h].x = fmaf(v[i][h].x, w, acc[h].x); acc[h].y = fmaf(v[i][h].y, w, acc[h].y);
+              acc[h].z = fmaf(v[i][h].z, w, acc[h].z); acc[h].w = fmaf(v[i][h].w, w, acc[h].w);
+            }
       }
+#pragma unroll
+      for (int h = 0; h < RMAX; ++h)
+        if (h < r) reinterpret_cast<float4*>(red + (warp * r + h) * kD)[lane] = acc[h];
       __syncthreads();
-      for (int u = warp; u < n_units; u += kWarps) {
-        const int h = u % r, p = u / r;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s0 = p; s0 < n_ctas_pair; s0 += kBatch * np) {
-          if (u != warp || s0 != p) {
+      for (int idx = threadIdx.x; idx < r * 32; idx += kWarps * 32) {
+        const int h = idx >> 5, c = idx & 31;
+        float4 o = reinterpret_cast<const float4*>(red + h * kD)[c];
 #pragma unroll
-            for (int k = 0; k < kBatch; ++k) {
-              const int sr = s0 + k * np;
-              if (sr < n_ctas_pair)
-                v[k] = __ldcg(reinterpret_cast<const float4*>(a.part_o + (rec0 + sr * r + h) * kD) + lane);
-            }
-          }
-#pragma unroll
-          for (int k = 0; k < kBatch; ++k) {
-            const int sr = s0 + k * np;
-            if (sr < n_ctas_pair) {
-              const float w = sm_w[sr * r + h];
-              acc.x = fmaf(v[k].x, w, acc.x); acc.y = fmaf(v[k].y, w, acc.y);
-              acc.z = fmaf(v[k].z, w, acc.z); acc.w = fmaf(v[k].w, w, acc.w);
-            }
-          }
+        for (int w = 1; w < kWarps; ++w) {
+          const float4 t = reinterpret_cast<const float4*>(red + (w * r + h) * kD)[c];
+          o.x += t.x; o.y += t.y; o.z += t.z; o.w += t.w;
         }
-        if (np == 1) {
-          const int64_t oi = (static_cast<int64_t>(b) * cv.Hq + kv * r + h) * kD + 4 * lane;
-          if (a.out_bf16)
-            *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(a.out) + oi) =
-                make_uint2(pack_bf16x2(acc.x, acc.y), pack_bf16x2(acc.z, acc.w));
-          else
-            *reinterpret_cast<float4*>(static_cast<float*>(a.out) + oi) = acc;
-        } else {
-          reinterpret_cast<float4*>(red + u * kD)[lane] = acc;
-        }
-      }
-      if (np > 1) {
-        __syncthreads();
-        for (int h = 0; h < r; ++h) {
-          float o = 0.f;
-          for (int p = 0; p < np; ++p) o += red[(h + r * p) * kD + d];
-          const int64_t oi = (static_cast<int64_t>(b) * cv.Hq + kv * r + h) * kD + d;
-          if (a.out_bf16)
-            static_cast<__nv_bfloat16*>(a.out)[oi] = __float2bfloat16_rn(o);
-          else
-            static_cast<float*>(a.out)[oi] = o;
-        }
+        const int64_t oi = (static_cast<int64_t>(b) * cv.Hq + kv * r + h) * kD + 4 * c;
+        if (a.out_bf16)
+          *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(a.out) + oi) =
+              make_uint2(pack_bf16x2(o.x, o.y), pack_bf16x2(o.z, o.w));
+        else
+          *reinterpret_cast<float4*>(static_cast<float*>(a.out) + oi) = o;
       }
     }
   }  // ticket path
@@ -1009,7 +1013,7 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
   else if (a.cv.G == 64) kern = r <= 4 ? lq_decode_mma_kernel<64, 1> : lq_decode_mma_kernel<64, 2>;
   else return cudaErrorInvalidValue;
   static_assert(kSmemStages >= static_cast<int>((kWarps * 8 * (kD + 4) + 3 * kWarps * 8 + 16) * sizeof(float)) &&
-                    kSmemStages >= (3 * kMergeMax + kWarps * kMaxRatio * kD) * 4,
+                    kSmemStages >= (kMergeMax + kWarps * kMaxRatio * kD) * 4,
                 "merge scratch");
   // opt in to the dynamic shared memory size once per (device, kernel variant)
   static bool configured[64][4] = {};
