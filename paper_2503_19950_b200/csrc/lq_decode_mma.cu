@@ -222,7 +222,7 @@ __device__ __forceinline__ void tile_softmax(WarpState<NCB>& st, float (&s)[NSUB
     // so it moves -- and the accumulators are rescaled -- only when a score exceeds it by more than 8
     const bool up = mx > st.m[cb] + 8.f;  // m = -inf initially -> true
     const float mn = up ? mx : st.m[cb];
-    changed |= up;
+    changed |= up && st.m[cb] > -INFINITY;  // nothing to rescale before the first tile
     corr[cb] = ex2(st.m[cb] - mn);  // m = -inf -> 0; unchanged -> 1
     st.m[cb] = mn;
   }
@@ -283,14 +283,15 @@ __device__ __forceinline__ void transpose_p(const float (&p)[NCB][2], float (&pT
     }
 }
 
-// NCB == 1: split the probabilities into bf16 hi (even columns) / lo (odd columns).
-// H = hi in every lane; P = hi in even, lo in odd columns.
+// NCB == 1: split the probabilities into bf16 hi (even columns) / lo (odd columns).  The odd
+// columns carry the lo parts NEGATED all the way to the accumulators (the epilogue subtracts them):
+// the residuals then need no separate negation.  H = hi in every lane; P = hi in even, -lo in odd columns.
 __device__ __forceinline__ void split_p_bf16(const float (&pT)[2][2], bool odd, uint32_t (&H)[2], uint32_t (&P)[2]) {
 #pragma unroll
   for (int th = 0; th < 2; ++th) {
     H[th] = pack_bf16x2(pT[th][0], pT[th][1]);
     P[th] = H[th];
-    if (odd) P[th] = pack_bf16x2(pT[th][0] - bf16lo_f32(H[th]), pT[th][1] - bf16hi_f32(H[th]));
+    if (odd) P[th] = pack_bf16x2(bf16lo_f32(H[th]) - pT[th][0], bf16hi_f32(H[th]) - pT[th][1]);
   }
 }
 
@@ -471,7 +472,8 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
         const uint2 zw = lds64(tile + qt_vzero_off(G) + u * VS + 8 * (4 * (n % NG) + j));
         mma_bf16(st.zacc, zw.x, 0u, zw.y, 0u, P[0], P[1]);
       }
-      // p * value scale per value group: even columns RN(hi*s), odd columns lo*s + residual
+      // p * value scale per value group: even columns RN(hi*s), odd columns -(lo*s + residual)
+      const uint32_t Hn[2] = {H[0] ^ 0x80008000u, H[1] ^ 0x80008000u};
       uint32_t bp[NG][2];
       uint32_t sv[NG][2];
       if (NG == 4) {
@@ -489,8 +491,8 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
         for (int th = 0; th < 2; ++th) {
           bp[g][th] = bf16x2_mul(H[th], sv[g][th]);
           if (oddmask) {
-            const uint32_t r1 = bf16x2_fma(H[th], sv[g][th], bf16x2_neg(bp[g][th]));
-            bp[g][th] = bf16x2_fma(P[th], sv[g][th], r1);
+            const uint32_t r1n = bf16x2_fma(Hn[th], sv[g][th], bp[g][th]);  // RN(hi*s) - hi*s, exact
+            bp[g][th] = bf16x2_fma(P[th], sv[g][th], r1n);
           }
         }
       const uint32_t v0s = vw.x >> 8, v1s = vw.y >> 8, v2s = vw.z >> 8, v3s = vw.w >> 8;
@@ -693,8 +695,9 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
         for (int w = 0; w < 2; ++w) {
           uint32_t raw;
           asm volatile("ld.shared.u32 %0, [%1];" : "=r"(raw) : "r"(qrow + 2 * (16 * ks + 8 * w + 2 * j)));
-          const float f = pow2i(64 - 2 * (ks & 3));
-          qs[cb][ks][w] = valid ? pack_bf16x2(bf16lo_f32(raw) * f, bf16hi_f32(raw) * f) : 0u;
+          // 2^(64 - 2*(ks&3)) as a bf16 pair: the product is exact (a power of two, no overflow)
+          const uint32_t f2 = (static_cast<uint32_t>(127 + 64 - 2 * (ks & 3)) << 7) * 0x00010001u;
+          qs[cb][ks][w] = valid ? bf16x2_mul(raw, f2) : 0u;
         }
     }
   }
@@ -776,9 +779,9 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     // quant mode: out = true * 2^(kPExp + vpos); fp mode: out = true * 2^kPExp
     const float f = st.quant_mode ? pow2i(-vpos_log2<NCB>(mt) - 70) * (bf16_pv<NCB>() ? 0x1p6f : 0x1p70f) : kPInv;
     if (bf16_pv<NCB>()) {
-      const float z = __shfl_sync(kFull, st.zacc[0] + st.zacc[1], 4 * g + j) * kPInv;
-      o0[mt] = fmaf(st.out[mt][0] + st.out[mt][1], f, z);
-      o1[mt] = fmaf(st.out[mt][2] + st.out[mt][3], f, z);
+      const float z = __shfl_sync(kFull, st.zacc[0] - st.zacc[1], 4 * g + j) * kPInv;
+      o0[mt] = fmaf(st.out[mt][0] - st.out[mt][1], f, z);
+      o1[mt] = fmaf(st.out[mt][2] - st.out[mt][3], f, z);
     } else {
       const float z0 = __shfl_sync(kFull, st.zacc[0], 4 * g + j), z1 = __shfl_sync(kFull, st.zacc[1], 4 * g + j);
       st.out[mt][0] = fmaf(st.out[mt][0], f, z0);
