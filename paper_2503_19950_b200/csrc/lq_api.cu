@@ -42,6 +42,7 @@ struct lq_cache {
   float* part_o = nullptr;
   float* part_ml = nullptr;
   int* status = nullptr;
+  int* ingest_idx = nullptr;  // index list of the one-launch prompt ingestion (max_tokens ints)
   int* tickets = nullptr;  // per (b, kv) arrival counters of the fused split-K merge
   // staging for the host-buffer entry point, one slice per layer
   uint8_t* stage_k = nullptr;
@@ -83,6 +84,7 @@ void free_all(lq_cache* c) {
     cudaFree(c->part_ml);
     cudaFree(c->status);
     cudaFree(c->tickets);
+    cudaFree(c->ingest_idx);
     cudaFree(c->stage_k);
     cudaFree(c->stage_v);
     cudaFree(c->stage_q);
@@ -235,6 +237,7 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
               dev_alloc(c, reinterpret_cast<void**>(&c->part_ml), pairs * c->max_splits * r * 2 * 4) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->status), 256) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->tickets), pairs * 128) &&
+              dev_alloc(c, reinterpret_cast<void**>(&c->ingest_idx), (cfg->max_tokens + 3 * cfg->window) * 4) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_k), cfg->n_layers * pairs * kD * 2) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_v), cfg->n_layers * pairs * kD * 2) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_q),
@@ -265,6 +268,46 @@ lq_status_t lq_destroy(lq_cache_t* c) {
   return LQ_OK;
 }
 
+namespace {
+
+// A prompt appended to an empty layer: the host plays Algorithm 1 token by token on its mirror of
+// the filter (which never looks at the data), collects the removed token ids of every overflow
+// step and the final slot map, and one kernel writes both stores.
+lq_status_t ingest_prompt(lq_cache* c, int layer, const void* k, const void* v, int n, cudaStream_t st) {
+  LayerState& L = c->layers[layer];
+  const int W = c->cfg.window, G = c->cfg.group;
+  std::vector<int32_t> idx;
+  idx.reserve(static_cast<size_t>(n) + 3 * W);
+  std::vector<int32_t> ids(W);
+  int done = 0;
+  while (done < n) {
+    if (L.n_fp == 3 * W) {
+      next_evicted(c, L, nullptr, ids.data());
+      idx.insert(idx.end(), ids.begin(), ids.end());
+      apply_event(c, L);
+    }
+    const int take = std::min(n - done, 3 * W - L.n_fp);
+    for (int t = 0; t < take; ++t) {
+      L.age_slot.push_back(L.n_fp + t);
+      L.slot_token[L.n_fp + t] = static_cast<int32_t>(L.n_seen + t);
+    }
+    L.n_fp += take;
+    L.n_seen += take;
+    done += take;
+  }
+  const int n_tiles = static_cast<int>(idx.size()) / G;
+  for (int s = 0; s < L.n_fp; ++s) idx.push_back(L.slot_token[s]);
+  // pageable source: the runtime stages it before the call returns, so `idx` may die here
+  cudaError_t e = cudaMemcpyAsync(c->ingest_idx, idx.data(), idx.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return cuda_fail(c, e, "prompt index upload");
+  e = launch_ingest(c->cv, layer, k, v, n, c->ingest_idx, n_tiles, L.n_fp, 0, st);
+  if (e != cudaSuccess) return cuda_fail(c, e, "lq_ingest_kernel");
+  c->n_launches++;
+  return LQ_OK;
+}
+
+}  // namespace
+
 lq_status_t lq_append(lq_cache_t* c, int32_t layer, const void* k, const void* v, int32_t n, void* stream) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers || n < 0) return LQ_ERR_INVALID_ARG;
   if (!c->dry && (!k || !v)) return LQ_ERR_INVALID_ARG;
@@ -274,6 +317,7 @@ lq_status_t lq_append(lq_cache_t* c, int32_t layer, const void* k, const void* v
   if (L.n_seen + n > c->cfg.max_tokens) return LQ_ERR_CAPACITY;
   if (!c->cfg.auto_compress && L.n_fp + n > 3 * W) return LQ_ERR_WINDOW_FULL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!c->dry && c->cfg.auto_compress && L.n_seen == 0 && n > 3 * W) return ingest_prompt(c, layer, k, v, n, st);
   int done = 0;
   while (done < n) {
     if (L.n_fp == 3 * W) {

@@ -87,40 +87,11 @@ __device__ __forceinline__ void group_params(float mn, float mx, uint16_t& scale
   zero_bits = __bfloat16_as_ushort(__float2bfloat16_rn(mn_c));  // exact: mn is a bf16 value
 }
 
+// Steps 3 and 4 of the overflow step for one key group whose G rows sit in shared memory
+// (sK, sV: [G][128] bf16 bits; overwritten by the codes).  256 threads.
 template <int G>
-__global__ void __launch_bounds__(256)
-lq_compress_kernel(CacheView cv, LayerList layers, EvictList ev, int64_t tile0) {
-  __shared__ __align__(16) uint16_t sK[G][kD];
-  __shared__ __align__(16) uint16_t sV[G][kD];
+__device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kD], uint16_t (&sV)[G][kD], uint8_t* tile, int tid) {
   constexpr int NS = G / 16;
-  const int tau = blockIdx.x;
-  const int64_t pair = blockIdx.y;
-  const int layer = layers.layer[blockIdx.z];
-  const int tid = threadIdx.x;
-  uint8_t* fpbase = cv.fp + layer * cv.fp_layer_stride + pair * cv.fp_head_stride;
-  uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
-                  (tile0 + tau) * quant_tile_bytes(G);
-
-  // 1. gather the removed rows
-  for (int idx = tid; idx < G * 32; idx += 256) {
-    const int c = idx & 15, which = (idx >> 4) & 1, e = idx >> 5;
-    const int slot = ev.slot[tau * G + e];
-    const uint4 val = *reinterpret_cast<const uint4*>(fpbase + fp_chunk_off(slot, c) +
-                                                      (which ? kFpTileVOffset : 0));
-    *reinterpret_cast<uint4*>(which ? &sV[e][c * 8] : &sK[e][c * 8]) = val;
-  }
-  __syncthreads();
-
-  // 2. back-fill the holes from the newest window
-  for (int idx = tid; idx < G * 32; idx += 256) {
-    const int c = idx & 15, which = (idx >> 4) & 1, e = idx >> 5;
-    const int dst = ev.slot[tau * G + e];
-    const int src = 2 * cv.W + tau * G + e;
-    const int vo = which ? kFpTileVOffset : 0;
-    const uint4 val = *reinterpret_cast<const uint4*>(fpbase + fp_chunk_off(src, c) + vo);
-    *reinterpret_cast<uint4*>(fpbase + fp_chunk_off(dst, c) + vo) = val;
-  }
-
   // 3. quantise
   if (tid < kD) {
     const int d = tid;
@@ -199,6 +170,42 @@ lq_compress_kernel(CacheView cv, LayerList layers, EvictList ev, int64_t tile0) 
   }
 }
 
+template <int G>
+__global__ void __launch_bounds__(256)
+lq_compress_kernel(CacheView cv, LayerList layers, EvictList ev, int64_t tile0) {
+  __shared__ __align__(16) uint16_t sK[G][kD];
+  __shared__ __align__(16) uint16_t sV[G][kD];
+  const int tau = blockIdx.x;
+  const int64_t pair = blockIdx.y;
+  const int layer = layers.layer[blockIdx.z];
+  const int tid = threadIdx.x;
+  uint8_t* fpbase = cv.fp + layer * cv.fp_layer_stride + pair * cv.fp_head_stride;
+  uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
+                  (tile0 + tau) * quant_tile_bytes(G);
+
+  // 1. gather the removed rows
+  for (int idx = tid; idx < G * 32; idx += 256) {
+    const int c = idx & 15, which = (idx >> 4) & 1, e = idx >> 5;
+    const int slot = ev.slot[tau * G + e];
+    const uint4 val = *reinterpret_cast<const uint4*>(fpbase + fp_chunk_off(slot, c) +
+                                                      (which ? kFpTileVOffset : 0));
+    *reinterpret_cast<uint4*>(which ? &sV[e][c * 8] : &sK[e][c * 8]) = val;
+  }
+  __syncthreads();
+
+  // 2. back-fill the holes from the newest window
+  for (int idx = tid; idx < G * 32; idx += 256) {
+    const int c = idx & 15, which = (idx >> 4) & 1, e = idx >> 5;
+    const int dst = ev.slot[tau * G + e];
+    const int src = 2 * cv.W + tau * G + e;
+    const int vo = which ? kFpTileVOffset : 0;
+    const uint4 val = *reinterpret_cast<const uint4*>(fpbase + fp_chunk_off(src, c) + vo);
+    *reinterpret_cast<uint4*>(fpbase + fp_chunk_off(dst, c) + vo) = val;
+  }
+
+  quantise_pack_tile<G>(sK, sV, tile, tid);
+}
+
 cudaError_t launch_compress(const CacheView& cv, const LayerList& layers, const EvictList& ev,
                             int64_t tile0, cudaStream_t st) {
   dim3 grid(cv.W / cv.G, cv.B * cv.Hkv, layers.n);
@@ -206,6 +213,60 @@ cudaError_t launch_compress(const CacheView& cv, const LayerList& layers, const 
     lq_compress_kernel<32><<<grid, 256, 0, st>>>(cv, layers, ev, tile0);
   else if (cv.G == 64)
     lq_compress_kernel<64><<<grid, 256, 0, st>>>(cv, layers, ev, tile0);
+  else
+    return cudaErrorInvalidValue;
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// Prompt ingestion in one launch.  Appending an n-token prompt to an empty layer one token at a
+// time (Algorithm 1) ends in a state the host knows in advance, because the filter never looks at
+// the data: the removed tokens of every overflow step, in store order, and the token that ends up
+// in every fp slot.  idx = [n_tiles * G removed prompt positions][n_fp final slot -> prompt
+// position].  CTAs [0, n_tiles) each quantise one key group straight from the prompt tensors, the
+// remaining CTAs write the surviving rows to their final slots; the result is bit-identical to
+// the token-by-token path.
+// ---------------------------------------------------------------------------------------
+template <int G>
+__global__ void __launch_bounds__(256)
+lq_ingest_kernel(CacheView cv, int layer, const uint4* __restrict__ k, const uint4* __restrict__ v, int n_src,
+                 const int* __restrict__ idx, int n_tiles, int n_fp, int64_t tile0) {
+  __shared__ __align__(16) uint16_t sK[G][kD];
+  __shared__ __align__(16) uint16_t sV[G][kD];
+  const int64_t pair = blockIdx.y;
+  const int tid = threadIdx.x;
+  if (static_cast<int>(blockIdx.x) < n_tiles) {
+    const int tau = blockIdx.x;
+    uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
+                    (tile0 + tau) * quant_tile_bytes(G);
+    for (int i = tid; i < G * 32; i += 256) {
+      const int c = i & 15, which = (i >> 4) & 1, e = i >> 5;
+      const int64_t t = idx[tau * G + e];
+      const uint4 val = (which ? v : k)[(pair * n_src + t) * 16 + c];
+      *reinterpret_cast<uint4*>(which ? &sV[e][c * 8] : &sK[e][c * 8]) = val;
+    }
+    __syncthreads();
+    quantise_pack_tile<G>(sK, sV, tile, tid);
+  } else {
+    const int i = (static_cast<int>(blockIdx.x) - n_tiles) * 256 + tid;
+    if (i >= n_fp * 32) return;
+    const int c = i & 15, which = (i >> 4) & 1, slot = i >> 5;
+    const int64_t t = idx[n_tiles * G + slot];
+    uint8_t* base = cv.fp + layer * cv.fp_layer_stride + pair * cv.fp_head_stride;
+    *reinterpret_cast<uint4*>(base + fp_chunk_off(slot, c) + (which ? kFpTileVOffset : 0)) =
+        (which ? v : k)[(pair * n_src + t) * 16 + c];
+  }
+}
+
+cudaError_t launch_ingest(const CacheView& cv, int layer, const void* k, const void* v, int n_src, const int* idx_dev,
+                          int n_tiles, int n_fp, int64_t tile0, cudaStream_t st) {
+  dim3 grid(n_tiles + (n_fp * 32 + 255) / 256, cv.B * cv.Hkv);
+  const uint4* k4 = static_cast<const uint4*>(k);
+  const uint4* v4 = static_cast<const uint4*>(v);
+  if (cv.G == 32)
+    lq_ingest_kernel<32><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, n_fp, tile0);
+  else if (cv.G == 64)
+    lq_ingest_kernel<64><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, n_fp, tile0);
   else
     return cudaErrorInvalidValue;
   return cudaGetLastError();

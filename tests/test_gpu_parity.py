@@ -126,6 +126,44 @@ def test_multi_layer_compress_all_and_independence():
     assert [cache.info(l).n_events for l in range(L)] == [1, 1, 0]
 
 
+@pytest.mark.parametrize("W,G,n", [(32, 32, 3 * 32 + 1), (64, 32, 777), (128, 64, 2048 + 55)])
+def test_prompt_ingestion_in_one_launch_equals_token_by_token(W, G, n):
+    """A prompt appended to an empty layer goes through one kernel; the same tokens appended after a
+    first single token go through the append / overflow kernels.  Both must leave the same image, the
+    same physical stores (identical attention bits) and the oracle's image."""
+    B, Hq, Hkv, D = 2, 8, 2, 128
+    k, v = synth.keys_values(77, B, Hkv, n, D, "cuda", outliers=synth.outlier_channels(77, Hkv, D, 3))
+    one = LogQuantCache(2, B, Hq, Hkv, W, G, max_tokens=n + 2 * W + 8)
+    seq = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=n + 2 * W + 8)
+    before = one.info(1).n_kernel_launches
+    one.append(1, k, v)
+    assert one.info(1).n_kernel_launches == before + 1
+    seq.append(0, k[:, :, :1].contiguous(), v[:, :, :1].contiguous())
+    for t0 in range(1, n, 97):
+        seq.append(0, k[:, :, t0:t0 + 97].contiguous(), v[:, :, t0:t0 + 97].contiguous())
+    assert seq.info(0).n_kernel_launches > 2
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G)
+    oc.append(synth.bf16_bits(k), synth.bf16_bits(v))
+    a, b = one.export(1), seq.export(0)
+    assert_images_equal(a, b)
+    assert_images_equal(a, oc.export())
+    i1, i2 = one.info(1), seq.info(0)
+    assert (i1.n_seen, i1.n_fp, i1.n_quant, i1.n_events) == (i2.n_seen, i2.n_fp, i2.n_quant, i2.n_events)
+    q = synth.queries(77, B, Hq, D, 0, "cuda")
+    o1, o2 = torch.empty(B, Hq, D, device="cuda"), torch.empty(B, Hq, D, device="cuda")
+    one.decode_attn(1, q, o1)
+    seq.decode_attn(0, q, o2)
+    torch.cuda.synchronize()
+    assert torch.equal(o1, o2)
+    # the next overflow step removes the same tokens in both
+    k2, v2 = synth.keys_values(78, B, Hkv, 2 * W, D, "cuda")
+    one.append(1, k2, v2)
+    seq.append(0, k2, v2)
+    assert_images_equal(one.export(1), seq.export(0))
+    assert one.kernel_status() == 0 and seq.kernel_status() == 0
+    one.close(); seq.close(); oc.close()
+
+
 def test_decode_step_with_host_buffers():
     B, Hq, Hkv, W, G, D = 2, 8, 2, 32, 32, 128
     N = 3 * W  # the first host step has to run the overflow itself, even with auto_compress = 0
