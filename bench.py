@@ -134,10 +134,13 @@ def make_step_inputs(wl, device, n_sets):
     return ks, vs, qs
 
 
-def prefill(cache, wl, device, layers=None, chunk=1024, sink=None):
-    """Append ctx tokens to every layer, generated chunk by chunk on `device`.
+def prefill(cache, wl, device, layers=None, chunk=None, sink=None):
+    """Append ctx tokens to every layer, generated on `device`: the whole prompt in one call (one
+    ingestion launch per layer) when K and V of a layer fit in 4 GB, else 1024 tokens at a time.
     sink(layer, k, v) additionally receives each chunk (used to feed the CPU oracle)."""
     L, B, Hkv, ctx = wl["L"], wl["B"], wl["Hkv"], wl["ctx"]
+    if chunk is None:
+        chunk = ctx if 2 * B * Hkv * ctx * D * 2 <= 4e9 else 1024
     u = synth.unit_vectors(wl["seed"], Hkv, D) if wl.get("planted") else None
     for l in (range(L) if layers is None else layers):
         for t0 in range(0, ctx, chunk):
