@@ -41,6 +41,11 @@ def lib():
         L.lqo_filter.restype = i64
         L.lqo_filter.argtypes = [i32, i64, p, p, p, p]
         L.lqo_quantize_group.argtypes = [p, i32, p, p, p]
+        L.lqo_quantize_group_bits.argtypes = [p, i32, i32, p, p, p]
+        L.lqo_pack4.argtypes = [p, i64, p]
+        L.lqo_unpack4.argtypes = [p, i64, p]
+        L.lqo_create_bits.restype = p
+        L.lqo_create_bits.argtypes = [i32] * 7
         L.lqo_dequant.restype = f64
         L.lqo_dequant.argtypes = [C.c_uint16, C.c_uint16, C.c_uint8]
         L.lqo_pack2.argtypes = [p, i64, p]
@@ -85,12 +90,15 @@ def filter_ids(W: int, N: int):
     return kept[: nk.value].copy(), quant[: nq.value].copy(), int(ev)
 
 
-def quantize_group(x_bf16: np.ndarray):
+def quantize_group(x_bf16: np.ndarray, bits: int = 2):
     """One quantisation group (uint16 bf16 bits) -> (scale bits, zero bits, codes)."""
     x = _c(x_bf16, np.uint16)
     s, z = np.zeros(1, np.uint16), np.zeros(1, np.uint16)
     codes = np.zeros(x.size, np.uint8)
-    lib().lqo_quantize_group(_ptr(x), x.size, _ptr(s), _ptr(z), _ptr(codes))
+    if bits == 2:
+        lib().lqo_quantize_group(_ptr(x), x.size, _ptr(s), _ptr(z), _ptr(codes))
+    else:
+        lib().lqo_quantize_group_bits(_ptr(x), x.size, bits, _ptr(s), _ptr(z), _ptr(codes))
     return int(s[0]), int(z[0]), codes
 
 
@@ -109,6 +117,20 @@ def unpack2(bytes_: np.ndarray) -> np.ndarray:
     b = _c(bytes_, np.uint8)
     out = np.zeros(b.size * 4, np.uint8)
     lib().lqo_unpack2(_ptr(b), out.size, _ptr(out))
+    return out
+
+
+def pack4(codes: np.ndarray) -> np.ndarray:
+    c = _c(codes, np.uint8)
+    out = np.zeros(c.size // 2, np.uint8)
+    lib().lqo_pack4(_ptr(c), c.size, _ptr(out))
+    return out
+
+
+def unpack4(bytes_: np.ndarray) -> np.ndarray:
+    b = _c(bytes_, np.uint8)
+    out = np.zeros(b.size * 2, np.uint8)
+    lib().lqo_unpack4(_ptr(b), out.size, _ptr(out))
     return out
 
 
@@ -154,9 +176,9 @@ def hardware_threads() -> int:
 class OracleCache:
     """One layer's mixed cache for B sequences: Algorithm 1 + quantiser + attention."""
 
-    def __init__(self, B, Hq, Hkv, D, W, G):
-        self.B, self.Hq, self.Hkv, self.D, self.W, self.G = B, Hq, Hkv, D, W, G
-        self._h = lib().lqo_create(B, Hq, Hkv, D, W, G)
+    def __init__(self, B, Hq, Hkv, D, W, G, bits=2):
+        self.B, self.Hq, self.Hkv, self.D, self.W, self.G, self.bits = B, Hq, Hkv, D, W, G, bits
+        self._h = lib().lqo_create_bits(B, Hq, Hkv, D, W, G, bits)
         if not self._h:
             raise ValueError("unsupported oracle configuration")
 
@@ -196,7 +218,8 @@ class OracleCache:
         nf, nq = self.n_fp, self.n_quant
         img = dict(
             kept_ids=np.zeros(nf, np.int32), quant_ids=np.zeros(nq, np.int32),
-            k_codes=np.zeros((B, H, nq, D // 4), np.uint8), v_codes=np.zeros((B, H, nq, D // 4), np.uint8),
+            k_codes=np.zeros((B, H, nq, D * self.bits // 8), np.uint8),
+            v_codes=np.zeros((B, H, nq, D * self.bits // 8), np.uint8),
             k_scale=np.zeros((B, H, nq // G, D), np.uint16), k_zero=np.zeros((B, H, nq // G, D), np.uint16),
             v_scale=np.zeros((B, H, nq, D // G), np.uint16), v_zero=np.zeros((B, H, nq, D // G), np.uint16),
             fp_k=np.zeros((B, H, nf, D), np.uint16), fp_v=np.zeros((B, H, nf, D), np.uint16))

@@ -17,7 +17,11 @@
 //                         x^    = zero + code * scale
 //                     keys: one group = G consecutive evicted tokens of one channel;
 //                     values: one group = G consecutive channels of one token.
-//   * packer        : 4 codes per byte, channel 4j+i in bits [2i+1:2i] of byte j.
+//                     The paper's second precision (the 4-bit rows of its accuracy tables,
+//                     Sec. 3.2) is the same quantiser with 16 levels: scale = bf16_rne((max -
+//                     min) / 15), codes 0..15.
+//   * packer        : 2-bit: 4 codes per byte, channel 4j+i in bits [2i+1:2i] of byte j;
+//                     4-bit: 2 codes per byte, channel 2j+i in bits [4i+3:4i] of byte j.
 //   * attention     : Eq. 2 with the 1/sqrt(d) scale of the appendix (passed in as
 //                     sm_scale), float64, one pass with max subtraction, over the union
 //                     of the full-precision list and the dequantised store.  Eq. 3
@@ -60,8 +64,9 @@ uint16_t f32_to_bf16_rne(float f) {
 // ---- quantiser: one group of n values, read with a stride --------------------------
 // All arithmetic is IEEE binary32 with one rounding per operation (the file is built
 // with -ffp-contract=off so no multiply-add is ever contracted).
+// top = highest code: 3 for 2 bits, 15 for 4 bits.
 void quantize_group(const uint16_t* x, int n, int64_t stride, uint16_t* scale_out,
-                    uint16_t* zero_out, uint8_t* codes, int64_t code_stride) {
+                    uint16_t* zero_out, uint8_t* codes, int64_t code_stride, int top = 3) {
   float mn = bf16_to_f32(x[0]);
   float mx = mn;
   for (int i = 1; i < n; ++i) {
@@ -72,7 +77,7 @@ void quantize_group(const uint16_t* x, int n, int64_t stride, uint16_t* scale_ou
   mn = mn + 0.0f;  // a zero-valued min or max is taken as +0 (the sign of zero is not information)
   mx = mx + 0.0f;
   volatile float range = mx - mn;
-  volatile float third = range / 3.0f;
+  volatile float third = range / static_cast<float>(top);  // one step of the code grid
   uint16_t sb = f32_to_bf16_rne(third);
   float scale = bf16_to_f32(sb);
   *scale_out = sb;
@@ -84,7 +89,7 @@ void quantize_group(const uint16_t* x, int n, int64_t stride, uint16_t* scale_ou
       volatile float q = d / scale;
       float r = std::nearbyintf(q);  // default rounding mode: ties to even
       if (r < 0.0f) r = 0.0f;
-      if (r > 3.0f) r = 3.0f;
+      if (r > static_cast<float>(top)) r = static_cast<float>(top);
       c = static_cast<uint8_t>(r);
     }
     codes[i * code_stride] = c;
@@ -106,6 +111,7 @@ struct Head {  // one (batch row, kv head)
 
 struct Cache {
   int B, Hq, Hkv, D, W, G;
+  int bits = 2;
   int64_t n_seen = 0, n_events = 0;
   std::vector<int64_t> A;  // ids of the tokens kept at original precision, age order
   std::vector<int64_t> Q;  // ids of the quantised tokens, store order
@@ -138,14 +144,15 @@ void overflow_event(Cache& c) {
       for (int d = 0; d < D; ++d) {
         size_t grp = (nq0 / G + blk) * D + d;
         quantize_group(&ek[static_cast<size_t>(blk) * G * D + d], G, D, &h.k_scale[grp],
-                       &h.k_zero[grp], &h.k_codes[(nq0 + static_cast<size_t>(blk) * G) * D + d], D);
+                       &h.k_zero[grp], &h.k_codes[(nq0 + static_cast<size_t>(blk) * G) * D + d], D,
+                       (1 << c.bits) - 1);
       }
     // values: group = G consecutive channels of one token
     for (int e = 0; e < W; ++e)
       for (int g = 0; g < D / G; ++g) {
         size_t grp = (nq0 + e) * (D / G) + g;
         quantize_group(&ev[static_cast<size_t>(e) * D + g * G], G, 1, &h.v_scale[grp],
-                       &h.v_zero[grp], &h.v_codes[(nq0 + e) * D + g * G], 1);
+                       &h.v_zero[grp], &h.v_codes[(nq0 + e) * D + g * G], 1, (1 << c.bits) - 1);
       }
     // shrink the full-precision rows to the kept positions
     std::vector<uint16_t> nk(keep_pos.size() * D), nv(keep_pos.size() * D);
@@ -240,6 +247,11 @@ void lqo_quantize_group(const uint16_t* x, int n, uint16_t* scale, uint16_t* zer
   quantize_group(x, n, 1, scale, zero, codes, 1);
 }
 
+// the same with 2 or 4 bits per code
+void lqo_quantize_group_bits(const uint16_t* x, int n, int bits, uint16_t* scale, uint16_t* zero, uint8_t* codes) {
+  quantize_group(x, n, 1, scale, zero, codes, 1, (1 << bits) - 1);
+}
+
 double lqo_dequant(uint16_t scale, uint16_t zero, uint8_t code) { return dequant(scale, zero, code); }
 
 // 4 codes per byte: code of element 4j+i in bits [2i+1:2i] of byte j.  n % 4 == 0.
@@ -254,6 +266,19 @@ void lqo_pack2(const uint8_t* codes, int64_t n, uint8_t* bytes) {
 void lqo_unpack2(const uint8_t* bytes, int64_t n, uint8_t* codes) {
   for (int64_t j = 0; j < n / 4; ++j)
     for (int i = 0; i < 4; ++i) codes[4 * j + i] = (bytes[j] >> (2 * i)) & 3u;
+}
+
+// 2 codes per byte: code of element 2j+i in bits [4i+3:4i] of byte j.  n % 2 == 0.
+void lqo_pack4(const uint8_t* codes, int64_t n, uint8_t* bytes) {
+  for (int64_t j = 0; j < n / 2; ++j)
+    bytes[j] = static_cast<uint8_t>((codes[2 * j] & 15u) | ((codes[2 * j + 1] & 15u) << 4));
+}
+
+void lqo_unpack4(const uint8_t* bytes, int64_t n, uint8_t* codes) {
+  for (int64_t j = 0; j < n / 2; ++j) {
+    codes[2 * j] = bytes[j] & 15u;
+    codes[2 * j + 1] = bytes[j] >> 4;
+  }
 }
 
 uint16_t lqo_f32_to_bf16(float f) { return f32_to_bf16_rne(f); }
@@ -311,6 +336,14 @@ void* lqo_create(int B, int Hq, int Hkv, int D, int W, int G) {
   return c;
 }
 
+// the same cache with 2 or 4 bits per code
+void* lqo_create_bits(int B, int Hq, int Hkv, int D, int W, int G, int bits) {
+  if (bits != 2 && bits != 4) return nullptr;
+  Cache* c = static_cast<Cache*>(lqo_create(B, Hq, Hkv, D, W, G));
+  if (c) c->bits = bits;
+  return c;
+}
+
 void lqo_destroy(void* p) { delete static_cast<Cache*>(p); }
 
 // k, v: [B][Hkv][n][D] bf16 bit patterns.  A prompt of n tokens is n single appends.
@@ -335,7 +368,7 @@ int64_t lqo_n_quant(void* p) { return static_cast<int64_t>(static_cast<Cache*>(p
 int64_t lqo_n_events(void* p) { return static_cast<Cache*>(p)->n_events; }
 
 // Canonical image.  kept_ids ascending (list A is in age order, hence ascending);
-// quant_ids in store order; codes packed 4 per byte; scale/zero as bf16 bit patterns;
+// quant_ids in store order; codes packed 4 per byte (2 per byte at 4 bits); scale/zero as bf16 bit patterns;
 // fp rows in kept_ids order.  Any pointer may be null to skip that array.
 void lqo_export(void* p, int32_t* kept_ids, int32_t* quant_ids, uint8_t* k_codes, uint8_t* v_codes,
                 uint16_t* k_scale, uint16_t* k_zero, uint16_t* v_scale, uint16_t* v_zero,
@@ -346,8 +379,13 @@ void lqo_export(void* p, int32_t* kept_ids, int32_t* quant_ids, uint8_t* k_codes
   if (quant_ids) for (size_t i = 0; i < nq; ++i) quant_ids[i] = static_cast<int32_t>(c.Q[i]);
   for (size_t hh = 0; hh < c.heads.size(); ++hh) {
     const Head& h = c.heads[hh];
-    if (k_codes) lqo_pack2(h.k_codes.data(), nq * D, k_codes + hh * nq * D / 4);
-    if (v_codes) lqo_pack2(h.v_codes.data(), nq * D, v_codes + hh * nq * D / 4);
+    if (c.bits == 2) {
+      if (k_codes) lqo_pack2(h.k_codes.data(), nq * D, k_codes + hh * nq * D / 4);
+      if (v_codes) lqo_pack2(h.v_codes.data(), nq * D, v_codes + hh * nq * D / 4);
+    } else {
+      if (k_codes) lqo_pack4(h.k_codes.data(), nq * D, k_codes + hh * nq * D / 2);
+      if (v_codes) lqo_pack4(h.v_codes.data(), nq * D, v_codes + hh * nq * D / 2);
+    }
     if (k_scale) std::copy(h.k_scale.begin(), h.k_scale.end(), k_scale + hh * (nq / G) * D);
     if (k_zero) std::copy(h.k_zero.begin(), h.k_zero.end(), k_zero + hh * (nq / G) * D);
     if (v_scale) std::copy(h.v_scale.begin(), h.v_scale.end(), v_scale + hh * nq * (D / G));

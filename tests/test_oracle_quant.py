@@ -1,4 +1,4 @@
-"""Pins for the oracle's 2-bit quantiser and packer."""
+"""Pins for the oracle's 2-bit and 4-bit quantisers and packers."""
 import os
 
 import numpy as np
@@ -162,3 +162,116 @@ def test_signed_zero_is_canonical():
     minus1 = 0xBF80
     s, z, c = oracle.quantize_group(np.array([minus1, neg0, minus1, pos0], np.uint16))
     assert z == minus1 and c.tolist() == [0, 3, 0, 3]
+
+
+# ---- 4-bit variant (the paper's second precision) ------------------------------------------
+GOLD4 = os.path.join(os.path.dirname(__file__), "golden", "quant4_worked_example.txt")
+
+
+def _gold4():
+    out = []
+    for line in open(GOLD4):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        vals, sz, codes, bts = [s.split() for s in line.split("|")]
+        out.append(([float(v) for v in vals], float(sz[0]), float(sz[1]), [int(c) for c in codes],
+                    [int(b, 16) for b in bts]))
+    return out
+
+
+@pytest.mark.parametrize("vals,scale,zero,codes,packed", _gold4())
+def test_worked_examples_4bit(vals, scale, zero, codes, packed):
+    x = f32_to_bf16_bits(np.array(vals, np.float32))
+    assert np.array_equal(bf16_bits_to_f64(x), np.array(vals))  # the fixture is bf16-exact
+    s, z, c = oracle.quantize_group(x, bits=4)
+    assert oracle.bf16_to_f32(s) == scale and oracle.bf16_to_f32(z) == zero
+    assert c.tolist() == codes
+    assert oracle.pack4(c).tolist() == packed
+
+
+def test_pack4_unpack4_all_bytes():
+    allb = np.arange(256, dtype=np.uint8)
+    codes = oracle.unpack4(allb)
+    assert codes.max() == 15 and codes.size == 512
+    assert np.array_equal(oracle.pack4(codes), allb)
+    assert np.array_equal(codes[0::2], allb & 15) and np.array_equal(codes[1::2], allb >> 4)
+
+
+@pytest.mark.parametrize("n", [32, 64])
+@pytest.mark.parametrize("spread", [1.0, 10.0, 1e-3, 300.0])
+def test_round_trip_bound_and_order_4bit(n, spread):
+    rng = np.random.default_rng(4321 + n)
+    for trial in range(200):
+        x = f32_to_bf16_bits((rng.standard_normal(n) * spread + rng.standard_normal() * spread).astype(np.float32))
+        s, z, c = oracle.quantize_group(x, bits=4)
+        xv = bf16_bits_to_f64(x)
+        sv, zv = oracle.bf16_to_f32(s), oracle.bf16_to_f32(z)
+        assert zv == xv.min()
+        assert abs(sv - (xv.max() - xv.min()) / 15) <= 2.0 ** -8 * sv
+        xh = zv + c.astype(np.float64) * sv
+        # half a step, plus what the bf16 rounding of the step can move the top of the grid (15 steps)
+        assert np.all(np.abs(xv - xh) <= sv / 2 * (1 + 1e-6) + 15 * sv * 2.0 ** -8)
+        assert c[np.argmin(xv)] == 0 and c[np.argmax(xv)] == 15
+        order = np.argsort(xv, kind="stable")
+        assert np.all(np.diff(c[order].astype(int)) >= 0)
+        # the finer grid is never worse than the 2-bit one by more than its own half step
+        s2, z2, c2 = oracle.quantize_group(x)
+        e2 = np.abs(xv - (oracle.bf16_to_f32(z2) + c2.astype(np.float64) * oracle.bf16_to_f32(s2))).max()
+        assert np.abs(xv - xh).max() <= e2 + sv
+
+
+def test_lattice_groups_round_trip_exactly_4bit():
+    # x = zero + k * step with a power-of-two step: scale is exact and every value is a grid point
+    rng = np.random.default_rng(7)
+    for step in (0.5, 2.0 ** -6, 4.0):
+        for trial in range(50):
+            k = rng.integers(0, 16, 32)
+            k[0], k[1] = 0, 15
+            zero = float(rng.integers(-8, 8)) * step
+            vals = (zero + k * step).astype(np.float32)
+            x = f32_to_bf16_bits(vals)
+            if not np.array_equal(bf16_bits_to_f64(x), vals.astype(np.float64)):
+                continue
+            s, z, c = oracle.quantize_group(x, bits=4)
+            assert oracle.bf16_to_f32(s) == step and oracle.bf16_to_f32(z) == zero
+            assert np.array_equal(c, k.astype(np.uint8))
+
+
+def test_cache_4bit_grouping_and_image_sizes():
+    B, Hq, Hkv, D, W, G = 1, 2, 1, 128, 32, 32
+    rng = np.random.default_rng(9)
+    n = 3 * W + 1
+    k = f32_to_bf16_bits(rng.standard_normal((B, Hkv, n, D)).astype(np.float32))
+    v = f32_to_bf16_bits(rng.standard_normal((B, Hkv, n, D)).astype(np.float32))
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G, bits=4)
+    oc.append(k, v)
+    img = oc.export()
+    assert img["k_codes"].shape == (B, Hkv, W, D // 2) and img["v_codes"].shape == (B, Hkv, W, D // 2)
+    ev = img["quant_ids"]
+    assert ev.tolist() == list(range(1, 2 * W, 2))
+    # keys: one group = G removed tokens of one channel; values: G channels of one token
+    kc = oracle.unpack4(img["k_codes"].reshape(-1)).reshape(W, D)
+    vc = oracle.unpack4(img["v_codes"].reshape(-1)).reshape(W, D)
+    for d in (0, 17, 127):
+        s, z, c = oracle.quantize_group(k[0, 0, ev[:G], d], bits=4)
+        assert (s, z) == (img["k_scale"][0, 0, 0, d], img["k_zero"][0, 0, 0, d])
+        assert np.array_equal(c, kc[:G, d])
+    for e in (0, 5, W - 1):
+        for g in range(D // G):
+            s, z, c = oracle.quantize_group(v[0, 0, ev[e], g * G:(g + 1) * G], bits=4)
+            assert (s, z) == (img["v_scale"][0, 0, e, g], img["v_zero"][0, 0, e, g])
+            assert np.array_equal(c, vc[e, g * G:(g + 1) * G])
+    # attention over the dequantised rows agrees with the dense definition on those rows
+    q = f32_to_bf16_bits(rng.standard_normal((B, Hq, D)).astype(np.float32))
+    out = oc.attention(q, 1 / np.sqrt(D))
+    K, V = oc.dense_rows(0, 0)
+    ref = oracle.attention_dense(bf16_bits_to_f64(q[0, 1]), K, V, 1 / np.sqrt(D))
+    assert np.allclose(out[0, 1], ref, rtol=0, atol=1e-12)
+    # 4-bit rows are closer to the originals than 2-bit rows
+    oc2 = oracle.OracleCache(B, Hq, Hkv, D, W, G)
+    oc2.append(k, v)
+    K2, _ = oc2.dense_rows(0, 0)
+    orig = bf16_bits_to_f64(k[0, 0, ev])
+    nf = oc.n_fp
+    assert np.abs(K[nf:] - orig).max() < np.abs(K2[nf:] - orig).max() / 3
