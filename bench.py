@@ -32,6 +32,8 @@ from paper_2503_19950_b200 import synth  # noqa: E402
 WORKLOADS = {
     # BASELINE config 2: Llama-3-8B layer shape, batch 8, context 8192, W=128, G=32, 32 stacked layers
     "llama3-8b-8k": dict(L=32, B=8, Hq=32, Hkv=8, W=128, G=32, ctx=8192, n_outliers=3, seed=2),
+    # config 2 with the paper's second precision (4-bit codes, 160 B per token)
+    "llama3-8b-8k-int4": dict(L=32, B=8, Hq=32, Hkv=8, W=128, G=32, ctx=8192, n_outliers=3, seed=2, bits=4),
     # config 4: long-context GQA-7
     "gqa7-32k": dict(L=28, B=4, Hq=28, Hkv=4, W=256, G=64, ctx=32768, n_outliers=0, seed=4, planted=True),
     # config 3: batch sweep at context 4096
@@ -161,7 +163,8 @@ def run_ours(args, wl, rank, world, device):
     L, B, Hq, Hkv, W, G, ctx = (wl[k] for k in ("L", "B", "Hq", "Hkv", "W", "G", "ctx"))
     steps, warmup = args.steps, args.warmup
     total_steps = 2 * (steps + warmup) + steps + warmup + 8  # device-timed, profiled and host-buffer passes
-    cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=ctx + total_steps + 8, device=device.index or 0,
+    bits = wl.get("bits", 2)
+    cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=ctx + total_steps + 8, device=device.index or 0, bits=bits,
                           n_splits=args.n_splits)
     prefill(cache, wl, device)
     ks, vs, qs = make_step_inputs(wl, device, Q_ROTATE)
@@ -263,7 +266,8 @@ def run_ours(args, wl, rank, world, device):
     # ---- one window-overflow event over all layers at once (lq_compress(layer=-1)) ----
     comp = None
     try:
-        ccache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=8 * W, device=device.index or 0, auto_compress=False)
+        ccache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=8 * W, device=device.index or 0, auto_compress=False,
+                               bits=bits)
         kf, vf = synth.keys_values(wl["seed"] + 7, B, Hkv, 3 * W, D, device, outliers=wl.get("_outliers"))
         k1, v1 = kf[:, :, :W].contiguous(), vf[:, :, :W].contiguous()
         evs = []
@@ -279,7 +283,7 @@ def run_ours(args, wl, rank, world, device):
             evs.append(e0.elapsed_time(e1) * 1e3)
         us = float(np.median(evs[1:]))
         rd = L * B * Hkv * (2 * W * 256 + W * 512)          # removed rows + back-fill sources, K and V
-        wr = L * B * Hkv * (W * (1024 // G + 64) + W * 512)   # packed tiles + back-filled rows
+        wr = L * B * Hkv * (W * (1024 // G + 32 * bits) + W * 512)   # packed tiles + back-filled rows
         comp = {"us_per_event": us, "layers": L, "tokens_per_s": L * B * W / (us * 1e-6),
                 "gbs": (rd + wr) / (us * 1e-6) / 1e9, "read_bytes": rd, "write_bytes": wr}
         ccache.close()
@@ -301,7 +305,7 @@ def run_ours(args, wl, rank, world, device):
         "ms_per_step": ms_max / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": args.workload, "layers": L, "batch": B, "q_heads": Hq, "kv_heads": Hkv,
-                   "head_dim": D, "context": ctx, "window": W, "group": G, "bits": 2,
+                   "head_dim": D, "context": ctx, "window": W, "group": G, "bits": bits,
                    "n_quant": int(inf.n_quant), "n_fp": int(inf.n_fp), "n_splits": int(inf.n_splits), "n_ctas": int(inf.n_ctas),
                    "step": "per layer: lq_append (+lq_compress on overflow) + lq_decode_attn",
                    "l2": "inputs larger than L2: %.2f GB of cache touched per step" % (bytes_step_last / 1e9),
@@ -341,7 +345,7 @@ def oracle_layer_step(wl, device, n_threads, min_seconds, max_reps, warmup=0):
     Runs until min_seconds of timed work or max_reps steps, whichever comes first (at least one)."""
     import oracle
     B, Hq, Hkv, W, G, ctx = (wl[k] for k in ("B", "Hq", "Hkv", "W", "G", "ctx"))
-    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G)
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G, bits=wl.get("bits", 2))
     wl1 = dict(wl, L=1)
     prefill(None, wl1, device, sink=lambda l, k, v: oc.append(synth.bf16_bits(k), synth.bf16_bits(v)))
     k, v = synth.keys_values(wl["seed"] + 100, B, Hkv, Q_ROTATE, D, device, layer=0, outliers=wl.get("_outliers"))

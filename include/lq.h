@@ -66,7 +66,7 @@ typedef struct {
   int32_t head_dim;      /* D; only 128 is implemented                                           */
   int32_t window;        /* W of Algorithm 1; W % G == 0, W <= 512                               */
   int32_t group;         /* G: quantisation group size, 32 or 64                                 */
-  int32_t bits;          /* 2                                                                    */
+  int32_t bits;          /* 2, or 4 (the paper's second precision; needs group == 32)             */
   int64_t max_tokens;    /* capacity per sequence (tokens ever appended)                         */
   int32_t auto_compress; /* 1: lq_append runs the overflow step itself when the window is full   */
   int32_t device;        /* CUDA device ordinal, or LQ_DEVICE_NONE for bookkeeping only          */
@@ -96,6 +96,7 @@ typedef struct {
  *   kept_ids  [n_fp]    int32, ascending: ids (append order, from 0) of the full-precision tokens
  *   quant_ids [n_quant] int32, in store order: event order, then age order inside an event
  *   k_codes, v_codes [B][Hkv][n_quant][D/4] uint8: channel 4j+i of a token in bits [2i+1:2i] of byte j
+ *                    (bits = 4: [..][D/2], channel 2j+i in bits [4i+3:4i] of byte j)
  *   k_scale, k_zero  [B][Hkv][n_quant/G][D] uint16 (bf16 bit patterns)
  *   v_scale, v_zero  [B][Hkv][n_quant][D/G] uint16
  *   fp_k, fp_v       [B][Hkv][n_fp][D] uint16, rows in kept_ids order

@@ -206,7 +206,8 @@ class LogQuantCache:
         img = dict(kept_ids=np.zeros(nf, np.int32), quant_ids=np.zeros(nq, np.int32))
         if not ids_only:
             img.update(
-                k_codes=np.zeros((B, H, nq, D // 4), np.uint8), v_codes=np.zeros((B, H, nq, D // 4), np.uint8),
+                k_codes=np.zeros((B, H, nq, D * self.cfg.bits // 8), np.uint8),
+                v_codes=np.zeros((B, H, nq, D * self.cfg.bits // 8), np.uint8),
                 k_scale=np.zeros((B, H, nq // G, D), np.uint16), k_zero=np.zeros((B, H, nq // G, D), np.uint16),
                 v_scale=np.zeros((B, H, nq, D // G), np.uint16), v_zero=np.zeros((B, H, nq, D // G), np.uint16),
                 fp_k=np.zeros((B, H, nf, D), np.uint16), fp_v=np.zeros((B, H, nf, D), np.uint16))

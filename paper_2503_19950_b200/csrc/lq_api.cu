@@ -198,8 +198,9 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
       cfg->window < 1 || cfg->group < 1 || cfg->max_tokens < 1 || cfg->n_splits < 0)
     return LQ_ERR_INVALID_ARG;
   if (cfg->n_q_heads % cfg->n_kv_heads) return LQ_ERR_INVALID_ARG;
-  if (cfg->head_dim != kD || cfg->bits != 2) return LQ_ERR_UNSUPPORTED;
+  if (cfg->head_dim != kD || (cfg->bits != 2 && cfg->bits != 4)) return LQ_ERR_UNSUPPORTED;
   if (cfg->group != 32 && cfg->group != 64) return LQ_ERR_UNSUPPORTED;
+  if (cfg->bits == 4 && cfg->group != 32) return LQ_ERR_UNSUPPORTED;  // a 4-bit tile of G = 64 exceeds a stage
   if (cfg->window % cfg->group || cfg->window > kMaxW) return LQ_ERR_UNSUPPORTED;
   if (cfg->n_q_heads / cfg->n_kv_heads > kMaxRatio || cfg->n_layers > 128) return LQ_ERR_UNSUPPORTED;
   if (cfg->kernel < LQ_KERNEL_AUTO || cfg->kernel > LQ_KERNEL_MMA) return LQ_ERR_INVALID_ARG;
@@ -213,8 +214,9 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
   CacheView& cv = c->cv;
   std::memset(&cv, 0, sizeof cv);
   cv.B = cfg->batch; cv.Hq = cfg->n_q_heads; cv.Hkv = cfg->n_kv_heads; cv.G = G; cv.W = W;
+  cv.planes = cfg->bits / 2;
   cv.quant_tiles_cap = (cfg->max_tokens + G - 1) / G;
-  cv.quant_head_stride = cv.quant_tiles_cap * quant_tile_bytes(G);
+  cv.quant_head_stride = cv.quant_tiles_cap * quant_tile_bytes(G, cv.planes);
   cv.quant_layer_stride = cv.quant_head_stride * pairs;
   cv.fp_head_stride = static_cast<int64_t>(3 * W / kFpTileSlots) * kFpTileBytes;
   cv.fp_layer_stride = cv.fp_head_stride * pairs;
@@ -491,7 +493,7 @@ lq_status_t lq_cache_info(const lq_cache_t* c, int32_t layer, lq_info_t* info) {
   info->n_events = L.n_events;
   info->bytes_device = c->bytes_device;
   info->n_kernel_launches = c->n_launches;
-  info->bytes_quant_per_token = quant_tile_bytes(c->cfg.group) / c->cfg.group;
+  info->bytes_quant_per_token = quant_tile_bytes(c->cfg.group, c->cfg.bits / 2) / c->cfg.group;
   info->bytes_decode_step = static_cast<int64_t>(c->cfg.batch) * c->cfg.n_kv_heads *
                             (L.n_quant * info->bytes_quant_per_token + static_cast<int64_t>(L.n_fp) * 4 * kD);
   if (c->dry || L.n_fp + L.n_quant == 0)
@@ -535,7 +537,7 @@ lq_status_t lq_export(const lq_cache_t* cc, int32_t layer, lq_image_t* img) {
   const int64_t pairs = static_cast<int64_t>(c->cfg.batch) * c->cfg.n_kv_heads;
   const int G = c->cfg.group;
   const int64_t nq = L.n_quant, nf = L.n_fp;
-  const int64_t sz_codes = pairs * nq * (kD / 4);
+  const int64_t sz_codes = pairs * nq * (kD * c->cfg.bits / 8);
   const int64_t sz_kp = pairs * (nq / G) * kD * 2;
   const int64_t sz_vp = pairs * nq * (kD / G) * 2;
   const int64_t sz_fp = pairs * nf * kD * 2;

@@ -123,6 +123,11 @@ __device__ __forceinline__ uint32_t bf16x2_fma(uint32_t a, uint32_t b, uint32_t 
   asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
   return d;
 }
+__device__ __forceinline__ uint32_t f16x2_mul(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
 __device__ __forceinline__ uint32_t bf16x2_neg(uint32_t a) {
   uint32_t d;
   asm("neg.bf16x2 %0, %1;" : "=r"(d) : "r"(a));
@@ -397,7 +402,10 @@ __device__ __forceinline__ void quant_bias(const uint32_t (&qs)[NCB][8][2], uint
 }
 
 // ---- one quant tile: one key group of G tokens ---------------------------------------------
-template <int G, int NCB>
+// PL = 2-bit planes per code.  A 4-bit code is 4 * (high plane) + (low plane): the high plane goes
+// through the same contractions first, its score accumulators are multiplied by 4 before the low
+// plane is added, and in p.v it meets p * s_v * 4 (all exact).
+template <int G, int NCB, int PL>
 __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uint32_t (&qs)[NCB][8][2], uint32_t tile,
                                                    const float (&bias)[NCB], float kq, int lane, uint32_t oddmask,
                                                    int opaque_zero) {
@@ -408,41 +416,52 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
   // score accumulator advances by one MMA per k-step; the group's q.zero comes in as `bias`.
   float s[NS][NCB][2];
   {
-    uint32_t kw[NS][4], kws[NS][4];
-#pragma unroll
-    for (int u = 0; u < NS; ++u) {
-      const uint4 w = lds128(tile + qt_kcodes_off() + u * 512 + 16 * lane);
-      // words: (nt0,w0) (nt0,w1) (nt1,w0) (nt1,w1);  a0=(nt0,w0) a1=(nt1,w0) a2=(nt0,w1) a3=(nt1,w1)
-      kw[u][0] = w.x; kw[u][1] = w.z; kw[u][2] = w.y; kw[u][3] = w.w;
-#pragma unroll
-      for (int e = 0; e < 4; ++e) kws[u][e] = kw[u][e] >> 8;
-    }
     float acc[NS][NCB][4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const uint4 sw = lds128(tile + qt_kscale_off() + 16 * (4 * i + j));
-      const uint32_t s4[4] = {sw.x, sw.y, sw.z, sw.w};
+    for (int pl = PL - 1; pl >= 0; --pl) {
+      uint32_t kw[NS][4], kws[NS][4];
 #pragma unroll
-      for (int kk = 0; kk < 2; ++kk) {
-        const int ks = 2 * i + kk;
-        uint32_t bq[NCB][2];
+      for (int u = 0; u < NS; ++u) {
+        const uint4 w = lds128(tile + qt_kcodes_off() + pl * qt_plane_bytes(G) + u * 512 + 16 * lane);
+        // words: (nt0,w0) (nt0,w1) (nt1,w0) (nt1,w1);  a0=(nt0,w0) a1=(nt1,w0) a2=(nt0,w1) a3=(nt1,w1)
+        kw[u][0] = w.x; kw[u][1] = w.z; kw[u][2] = w.y; kw[u][3] = w.w;
 #pragma unroll
-        for (int cb = 0; cb < NCB; ++cb) {
+        for (int e = 0; e < 4; ++e) kws[u][e] = kw[u][e] >> 8;
+      }
+      if (pl != PL - 1) {
 #pragma unroll
-          for (int w = 0; w < 2; ++w) {
-            // even columns RN(q*s); odd columns the exact residual q*s - RN(q*s)
-            bq[cb][w] = bf16x2_mul(qs[cb][ks][w], s4[2 * kk + w]);
-            if (oddmask) bq[cb][w] = bf16x2_fma(qs[cb][ks][w], s4[2 * kk + w], bf16x2_neg(bq[cb][w]));
-          }
-        }
+        for (int u = 0; u < NS; ++u)
 #pragma unroll
-        for (int u = 0; u < NS; ++u) {
-          const uint32_t a0 = ext_bf16_i(ks, kw[u][0], kws[u][0]), a1 = ext_bf16_i(ks, kw[u][1], kws[u][1]),
-                         a2 = ext_bf16_i(ks, kw[u][2], kws[u][2]), a3 = ext_bf16_i(ks, kw[u][3], kws[u][3]);
+          for (int cb = 0; cb < NCB; ++cb)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[u][cb][e] *= 4.0f;
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint4 sw = lds128(tile + qt_kscale_off() + 16 * (4 * i + j));
+        const uint32_t s4[4] = {sw.x, sw.y, sw.z, sw.w};
+#pragma unroll
+        for (int kk = 0; kk < 2; ++kk) {
+          const int ks = 2 * i + kk;
+          uint32_t bq[NCB][2];
 #pragma unroll
           for (int cb = 0; cb < NCB; ++cb) {
-            if (ks == 0) mma_bf16_z(acc[u][cb], a0, a1, a2, a3, bq[cb][0], bq[cb][1]);
-            else mma_bf16(acc[u][cb], a0, a1, a2, a3, bq[cb][0], bq[cb][1]);
+#pragma unroll
+            for (int w = 0; w < 2; ++w) {
+              // even columns RN(q*s); odd columns the exact residual q*s - RN(q*s)
+              bq[cb][w] = bf16x2_mul(qs[cb][ks][w], s4[2 * kk + w]);
+              if (oddmask) bq[cb][w] = bf16x2_fma(qs[cb][ks][w], s4[2 * kk + w], bf16x2_neg(bq[cb][w]));
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < NS; ++u) {
+            const uint32_t a0 = ext_bf16_i(ks, kw[u][0], kws[u][0]), a1 = ext_bf16_i(ks, kw[u][1], kws[u][1]),
+                           a2 = ext_bf16_i(ks, kw[u][2], kws[u][2]), a3 = ext_bf16_i(ks, kw[u][3], kws[u][3]);
+#pragma unroll
+            for (int cb = 0; cb < NCB; ++cb) {
+              if (ks == 0 && pl == PL - 1) mma_bf16_z(acc[u][cb], a0, a1, a2, a3, bq[cb][0], bq[cb][1]);
+              else mma_bf16(acc[u][cb], a0, a1, a2, a3, bq[cb][0], bq[cb][1]);
+            }
           }
         }
       }
@@ -462,14 +481,13 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
   for (int u = 0; u < NS; ++u) {
     float pT[2][2];
     transpose_p<NCB>(s[u], pT, lane);
-    const uint4 vw = lds128(tile + qt_vcodes_off(G) + u * 512 + 16 * lane);
     if (bf16_pv<NCB>()) {
       uint32_t H[2], P[2];
       split_p_bf16(pT, oddmask != 0u, H, P);
       // value zero: A = zero (bf16 pairs straight from the tile), value groups on rows
       {
         // rows n >= NG of this MMA repeat real rows; their sums land in zacc rows nobody reads
-        const uint2 zw = lds64(tile + qt_vzero_off(G) + u * VS + 8 * (4 * (n % NG) + j));
+        const uint2 zw = lds64(tile + qt_vzero_off(G, PL) + u * VS + 8 * (4 * (n % NG) + j));
         mma_bf16(st.zacc, zw.x, 0u, zw.y, 0u, P[0], P[1]);
       }
       // p * value scale per value group: even columns RN(hi*s), odd columns -(lo*s + residual)
@@ -477,12 +495,12 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
       uint32_t bp[NG][2];
       uint32_t sv[NG][2];
       if (NG == 4) {
-        const uint4 s0 = lds128(tile + qt_vscale_off(G) + u * VS + 16 * j);
-        const uint4 s1 = lds128(tile + qt_vscale_off(G) + u * VS + 16 * (4 + j));
+        const uint4 s0 = lds128(tile + qt_vscale_off(G, PL) + u * VS + 16 * j);
+        const uint4 s1 = lds128(tile + qt_vscale_off(G, PL) + u * VS + 16 * (4 + j));
         sv[0][0] = s0.x; sv[0][1] = s0.y; sv[1][0] = s0.z; sv[1][1] = s0.w;
         sv[2 % NG][0] = s1.x; sv[2 % NG][1] = s1.y; sv[3 % NG][0] = s1.z; sv[3 % NG][1] = s1.w;
       } else {
-        const uint4 s0 = lds128(tile + qt_vscale_off(G) + u * VS + 16 * j);
+        const uint4 s0 = lds128(tile + qt_vscale_off(G, PL) + u * VS + 16 * j);
         sv[0][0] = s0.x; sv[0][1] = s0.y; sv[1 % NG][0] = s0.z; sv[1 % NG][1] = s0.w;
       }
 #pragma unroll
@@ -495,19 +513,28 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
             bp[g][th] = bf16x2_fma(P[th], sv[g][th], r1n);
           }
         }
-      const uint32_t v0s = vw.x >> 8, v1s = vw.y >> 8, v2s = vw.z >> 8, v3s = vw.w >> 8;
+#pragma unroll
+      for (int pl = PL - 1; pl >= 0; --pl) {
+        const uint4 vw = lds128(tile + qt_vcodes_off(G, PL) + pl * qt_plane_bytes(G) + u * 512 + 16 * lane);
+        uint32_t bx[NG][2];  // the high plane meets 4 * p * s_v
+#pragma unroll
+        for (int g = 0; g < NG; ++g)
+#pragma unroll
+          for (int th = 0; th < 2; ++th) bx[g][th] = pl ? bf16x2_mul(bp[g][th], 0x40804080u) : bp[g][th];
+        const uint32_t v0s = vw.x >> 8, v1s = vw.y >> 8, v2s = vw.z >> 8, v3s = vw.w >> 8;
 #define LQ_PV_STEP(MT)                                                                                        \
   mma_bf16(st.out[MT], ext_bf16<MT>(vw.x, v0s), ext_bf16<MT>(vw.y, v1s), ext_bf16<MT>(vw.z, v2s),             \
-           ext_bf16<MT>(vw.w, v3s), bp[((MT) * 16) / G][0], bp[((MT) * 16) / G][1]);
-      LQ_PV_STEP(0) LQ_PV_STEP(1) LQ_PV_STEP(2) LQ_PV_STEP(3)
-      LQ_PV_STEP(4) LQ_PV_STEP(5) LQ_PV_STEP(6) LQ_PV_STEP(7)
+           ext_bf16<MT>(vw.w, v3s), bx[((MT) * 16) / G][0], bx[((MT) * 16) / G][1]);
+        LQ_PV_STEP(0) LQ_PV_STEP(1) LQ_PV_STEP(2) LQ_PV_STEP(3)
+        LQ_PV_STEP(4) LQ_PV_STEP(5) LQ_PV_STEP(6) LQ_PV_STEP(7)
 #undef LQ_PV_STEP
+      }
     } else {
       // value zero: A = zero converted to fp16, value groups on rows
       {
         uint32_t z0 = 0, z1 = 0;
         if (n < NG) {
-          const uint2 zw = lds64(tile + qt_vzero_off(G) + u * VS + 8 * (4 * n + j));
+          const uint2 zw = lds64(tile + qt_vzero_off(G, PL) + u * VS + 8 * (4 * n + j));
           z0 = pack_f16x2(bf16lo_f32(zw.x), bf16hi_f32(zw.x));
           z1 = pack_f16x2(bf16lo_f32(zw.y), bf16hi_f32(zw.y));
         }
@@ -517,7 +544,7 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
       if (NG == 4) {
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
-          const uint4 svw = lds128(tile + qt_vscale_off(G) + u * VS + 16 * (4 * i + j));
+          const uint4 svw = lds128(tile + qt_vscale_off(G, PL) + u * VS + 16 * (4 * i + j));
           const uint32_t w4[4] = {svw.x, svw.y, svw.z, svw.w};
 #pragma unroll
           for (int gg = 0; gg < 2; ++gg)
@@ -528,7 +555,7 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
             }
         }
       } else {
-        const uint4 svw = lds128(tile + qt_vscale_off(G) + u * VS + 16 * j);
+        const uint4 svw = lds128(tile + qt_vscale_off(G, PL) + u * VS + 16 * j);
         const uint32_t w4[4] = {svw.x, svw.y, svw.z, svw.w};
 #pragma unroll
         for (int gg = 0; gg < 2; ++gg)
@@ -538,13 +565,22 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
             bp[gg % NG][th] = pack_f16x2(pT[th][0] * bf16lo_f32(w), pT[th][1] * bf16hi_f32(w));
           }
       }
-      const uint32_t v0s = vw.x >> 10, v1s = vw.y >> 10, v2s = vw.z >> 10, v3s = vw.w >> 10;
+#pragma unroll
+      for (int pl = PL - 1; pl >= 0; --pl) {
+        const uint4 vw = lds128(tile + qt_vcodes_off(G, PL) + pl * qt_plane_bytes(G) + u * 512 + 16 * lane);
+        uint32_t bx[NG][2];  // the high plane meets 4 * p * s_v
+#pragma unroll
+        for (int g = 0; g < NG; ++g)
+#pragma unroll
+          for (int th = 0; th < 2; ++th) bx[g][th] = pl ? f16x2_mul(bp[g][th], 0x44004400u) : bp[g][th];
+        const uint32_t v0s = vw.x >> 10, v1s = vw.y >> 10, v2s = vw.z >> 10, v3s = vw.w >> 10;
 #define LQ_PV_STEP(MT)                                                                                        \
   mma_f16(st.out[MT], ext_f16<MT>(vw.x, v0s), ext_f16<MT>(vw.y, v1s), ext_f16<MT>(vw.z, v2s),                 \
-          ext_f16<MT>(vw.w, v3s), bp[((MT) * 16) / G][0], bp[((MT) * 16) / G][1]);
-      LQ_PV_STEP(0) LQ_PV_STEP(1) LQ_PV_STEP(2) LQ_PV_STEP(3)
-      LQ_PV_STEP(4) LQ_PV_STEP(5) LQ_PV_STEP(6) LQ_PV_STEP(7)
+          ext_f16<MT>(vw.w, v3s), bx[((MT) * 16) / G][0], bx[((MT) * 16) / G][1]);
+        LQ_PV_STEP(0) LQ_PV_STEP(1) LQ_PV_STEP(2) LQ_PV_STEP(3)
+        LQ_PV_STEP(4) LQ_PV_STEP(5) LQ_PV_STEP(6) LQ_PV_STEP(7)
 #undef LQ_PV_STEP
+      }
     }
   }
 }
@@ -560,7 +596,7 @@ constexpr int kMergeMax = 2048;  // S * r records the fused second pass can stag
 // the pair (4 warps each) share them by a static, cost-weighted partition (see below); any
 // assignment is legal because every warp keeps its own online-softmax state.  A warp keeps up to
 // two loads in flight.
-template <int G, int NCB>
+template <int G, int NCB, int PL>
 __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerSm - 1) lq_decode_mma_kernel(DecodeArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   const CacheView& cv = a.cv;
@@ -568,7 +604,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n = lane >> 2, j = lane & 3;
   const uint32_t oddmask = (n & 1) ? 0xFFFFFFFFu : 0u;
-  constexpr int TILE = quant_tile_bytes(G);
+  constexpr int TILE = quant_tile_bytes(G, PL);
   constexpr int kStages = n_stages(G), kStageBytes = stage_bytes(G);
   static_assert(TILE <= kStageBytes && kFpTileVOffset <= kStageBytes && kStages <= kMaxStages, "stage geometry");
   // CTA c works for pair c % P in slot c / P: pairs [0, n_extra) have S CTAs, the others S - 1 (a.S
@@ -749,7 +785,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
         float bias[NCB];
 #pragma unroll
         for (int cb = 0; cb < NCB; ++cb) bias[cb] = t ? bias2[1][cb] : bias2[0][cb];
-        process_quant_tile<G, NCB>(st, qs, sbase + t * TILE, bias, kq, lane, oddmask, a.zero);
+        process_quant_tile<G, NCB, PL>(st, qs, sbase + t * TILE, bias, kq, lane, oddmask, a.zero);
       }
     } else if (desc >= 0) {
       const int nv = min(16, a.n_fp - desc * 16);
@@ -988,7 +1024,7 @@ void plan_decode_mma(DecodeArgs& a, int sm_count, int max_records, int s_overrid
   const int r = a.cv.Hq / a.cv.Hkv;
   a.tiles_fp = (a.n_fp + kFpTileSlots - 1) / kFpTileSlots;
   a.tiles_quant = static_cast<int>(a.n_quant / a.cv.G);
-  const int items = a.tiles_fp + a.tiles_quant / (stage_bytes(a.cv.G) / quant_tile_bytes(a.cv.G));
+  const int items = a.tiles_fp + a.tiles_quant / (stage_bytes(a.cv.G) / quant_tile_bytes(a.cv.G, a.cv.planes));
   // at most one resident wave of CTAs in total: a CTA that had to wait for a free slot would start
   // when the others finish, and its pair's merge would wait for it
   const int ctas_per_sm = r <= 4 ? kCtasPerSm : kCtasPerSm - 1;  // the two-column-block variant needs more registers
@@ -1012,18 +1048,19 @@ void plan_decode_mma(DecodeArgs& a, int sm_count, int max_records, int s_overrid
 cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
   const int r = a.cv.Hq / a.cv.Hkv;
   void (*kern)(DecodeArgs) = nullptr;
-  if (a.cv.G == 32) kern = r <= 4 ? lq_decode_mma_kernel<32, 1> : lq_decode_mma_kernel<32, 2>;
-  else if (a.cv.G == 64) kern = r <= 4 ? lq_decode_mma_kernel<64, 1> : lq_decode_mma_kernel<64, 2>;
+  if (a.cv.G == 32 && a.cv.planes == 1) kern = r <= 4 ? lq_decode_mma_kernel<32, 1, 1> : lq_decode_mma_kernel<32, 2, 1>;
+  else if (a.cv.G == 32 && a.cv.planes == 2) kern = r <= 4 ? lq_decode_mma_kernel<32, 1, 2> : lq_decode_mma_kernel<32, 2, 2>;
+  else if (a.cv.G == 64 && a.cv.planes == 1) kern = r <= 4 ? lq_decode_mma_kernel<64, 1, 1> : lq_decode_mma_kernel<64, 2, 1>;
   else return cudaErrorInvalidValue;
   static_assert(kSmemStages >= static_cast<int>((kWarps * 8 * (kD + 4) + 3 * kWarps * 8 + 16) * sizeof(float)) &&
                     kSmemStages >= (kMergeMax + kWarps * kMaxRatio * kD) * 4,
                 "merge scratch");
   // opt in to the dynamic shared memory size once per (device, kernel variant)
-  static bool configured[64][4] = {};
+  static bool configured[64][8] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  const int variant = (a.cv.G == 64 ? 2 : 0) + (r <= 4 ? 0 : 1);
+  const int variant = (a.cv.planes == 2 ? 4 : 0) + (a.cv.G == 64 ? 2 : 0) + (r <= 4 ? 0 : 1);
   if (dev < 0 || dev >= 64 || !configured[dev][variant]) {
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;

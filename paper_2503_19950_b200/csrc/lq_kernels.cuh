@@ -10,6 +10,7 @@ namespace lq {
 // Geometry and base pointers shared by every kernel.
 struct CacheView {
   int B, Hq, Hkv, G, W;
+  int planes;                 // 2-bit code planes per code: 1 (2-bit cache) or 2 (4-bit cache)
   int64_t quant_tiles_cap;    // capacity in tiles per (layer, b, kv)
   int64_t quant_head_stride;  // bytes between (b, kv) heads of the 2-bit store
   int64_t quant_layer_stride;

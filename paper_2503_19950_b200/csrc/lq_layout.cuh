@@ -20,6 +20,9 @@
 //     512 + 64 G             V scale, G/16 sub-tiles x (4096/G) B
 //     512 + 64 G + 256       V zero,  G/16 sub-tiles x (4096/G) B
 //     tile bytes = 1024 + 64 G   (3072 at G = 32, 5120 at G = 64; 96 / 80 B per token)
+//   4-bit codes (G = 32 only): every code is split into two 2-bit planes; the K codes area holds
+//   plane 0 then plane 1 (32 G bytes each), likewise the V codes area, and the offsets after the
+//   codes move accordingly: tile bytes = 1024 + 128 G = 5120 (160 B per token).
 //
 //   Fragment coordinates use lane = 4*(lane/4) + j of a warp, as in mma.sync.m16n8k16:
 //   K codes of sub-tile u: 32-bit word 4*lane + 2*nt + w  (lane = 4*n + j), bits
@@ -49,13 +52,16 @@ constexpr int kFpTileVOffset = kFpTileSlots * kD * 2;
 constexpr int kMaxW = 512;
 constexpr int kMaxRatio = 8;  // query heads per KV head
 
-__host__ __device__ constexpr int quant_tile_bytes(int G) { return 1024 + 64 * G; }
+// P = code planes: 1 for 2-bit codes; 2 for 4-bit codes, stored as two 2-bit planes (plane 0 = the low
+// two bits, plane 1 = the high two bits of every code), each plane in the 2-bit fragment order
+__host__ __device__ constexpr int quant_tile_bytes(int G, int P = 1) { return 1024 + 64 * G * P; }
+__host__ __device__ constexpr int qt_plane_bytes(int G) { return 32 * G; }  // K or V codes of one plane
 __host__ __device__ constexpr int qt_kscale_off() { return 0; }
 __host__ __device__ constexpr int qt_kzero_off() { return 256; }
 __host__ __device__ constexpr int qt_kcodes_off() { return 512; }
-__host__ __device__ constexpr int qt_vcodes_off(int G) { return 512 + 32 * G; }
-__host__ __device__ constexpr int qt_vscale_off(int G) { return 512 + 64 * G; }
-__host__ __device__ constexpr int qt_vzero_off(int G) { return 512 + 64 * G + 256; }
+__host__ __device__ constexpr int qt_vcodes_off(int G, int P = 1) { return 512 + 32 * G * P; }
+__host__ __device__ constexpr int qt_vscale_off(int G, int P = 1) { return 512 + 64 * G * P; }
+__host__ __device__ constexpr int qt_vzero_off(int G, int P = 1) { return 512 + 64 * G * P + 256; }
 __host__ __device__ constexpr int vsz_subtile_bytes(int G) { return 4096 / G; }
 
 // ---- element addressing (used by the overflow, export and scalar kernels) -------------

@@ -62,25 +62,27 @@ cudaError_t launch_append(const CacheView& cv, int layer, const void* k, const v
 //
 // Quantiser arithmetic (IEEE binary32, one rounding per operation, ties to even):
 //   zero = min, scale = bf16(fdiv(fsub(max, min), 3)), code = clamp(rint(fdiv(fsub(x, min), scale)), 0, 3),
-//   all codes 0 when scale == 0.  A zero-valued min or max is taken as +0.
+//   all codes 0 when scale == 0.  A zero-valued min or max is taken as +0.  The 4-bit cache uses 15
+//   in place of 3 and stores every code as two 2-bit planes (low bits, high bits).
 // ---------------------------------------------------------------------------------------
 __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) {
   return __uint_as_float(static_cast<uint32_t>(b) << 16);
 }
 
-__device__ __forceinline__ uint32_t quant_code(float x, float mn, float scale) {
+// top = highest code: 3 (2 bits) or 15 (4 bits)
+__device__ __forceinline__ uint32_t quant_code(float x, float mn, float scale, float top) {
   if (scale == 0.0f) return 0u;
   float q = __fdiv_rn(__fsub_rn(x, mn), scale);
   float r = rintf(q);
-  r = fminf(fmaxf(r, 0.0f), 3.0f);
+  r = fminf(fmaxf(r, 0.0f), top);
   return static_cast<uint32_t>(r);
 }
 
-__device__ __forceinline__ void group_params(float mn, float mx, uint16_t& scale_bits,
+__device__ __forceinline__ void group_params(float mn, float mx, float top, uint16_t& scale_bits,
                                              uint16_t& zero_bits, float& mn_c, float& scale) {
   mn_c = __fadd_rn(mn, 0.0f);  // -0 -> +0
   float mxc = __fadd_rn(mx, 0.0f);
-  float third = __fdiv_rn(__fsub_rn(mxc, mn_c), 3.0f);
+  float third = __fdiv_rn(__fsub_rn(mxc, mn_c), top);  // one step of the code grid
   __nv_bfloat16 sb = __float2bfloat16_rn(third);
   scale_bits = __bfloat16_as_ushort(sb);
   scale = __bfloat162float(sb);
@@ -89,9 +91,10 @@ __device__ __forceinline__ void group_params(float mn, float mx, uint16_t& scale
 
 // Steps 3 and 4 of the overflow step for one key group whose G rows sit in shared memory
 // (sK, sV: [G][128] bf16 bits; overwritten by the codes).  256 threads.
-template <int G>
+template <int G, int P>
 __device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kD], uint16_t (&sV)[G][kD], uint8_t* tile, int tid) {
   constexpr int NS = G / 16;
+  constexpr float kTop = P == 1 ? 3.0f : 15.0f;
   // 3. quantise
   if (tid < kD) {
     const int d = tid;
@@ -104,12 +107,12 @@ __device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kD], uint16
     }
     uint16_t sb, zb;
     float mnc, scale;
-    group_params(mn, mx, sb, zb, mnc, scale);
+    group_params(mn, mx, kTop, sb, zb, mnc, scale);
     reinterpret_cast<uint16_t*>(tile + qt_kscale_off())[kparam_index(d)] = sb;
     reinterpret_cast<uint16_t*>(tile + qt_kzero_off())[d] = zb;
 #pragma unroll 4
     for (int e = 0; e < G; ++e)
-      sK[e][d] = static_cast<uint16_t>(quant_code(bf16_bits_to_float(sK[e][d]), mnc, scale));
+      sK[e][d] = static_cast<uint16_t>(quant_code(bf16_bits_to_float(sK[e][d]), mnc, scale, kTop));
   } else {
     const int warp = (tid >> 5) - 4, lane = tid & 31;
     constexpr int LPG = G / 4;  // lanes per value group
@@ -126,25 +129,26 @@ __device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kD], uint16
       }
       uint16_t sb, zb;
       float mnc, scale;
-      group_params(mn, mx, sb, zb, mnc, scale);
+      group_params(mn, mx, kTop, sb, zb, mnc, scale);
       if ((lane % LPG) == 0) {
         const int g = lane / LPG;
-        reinterpret_cast<uint16_t*>(tile + qt_vscale_off(G))[vscale_index(e, g, G)] = sb;
-        reinterpret_cast<uint16_t*>(tile + qt_vzero_off(G))[vzero_index(e, g, G)] = zb;
+        reinterpret_cast<uint16_t*>(tile + qt_vscale_off(G, P))[vscale_index(e, g, G)] = sb;
+        reinterpret_cast<uint16_t*>(tile + qt_vzero_off(G, P))[vzero_index(e, g, G)] = zb;
       }
 #pragma unroll
       for (int i = 0; i < 4; ++i)
-        sV[e][4 * lane + i] = static_cast<uint16_t>(quant_code(x[i], mnc, scale));
+        sV[e][4 * lane + i] = static_cast<uint16_t>(quant_code(x[i], mnc, scale, kTop));
     }
   }
   __syncthreads();
 
-  // 4. pack into fragment order
-  uint32_t* kw = reinterpret_cast<uint32_t*>(tile + qt_kcodes_off());
-  uint32_t* vw = reinterpret_cast<uint32_t*>(tile + qt_vcodes_off(G));
-  for (int idx = tid; idx < 2 * NS * 128; idx += 256) {
-    const int which = idx / (NS * 128);
+  // 4. pack into fragment order, one 2-bit plane after the other
+  for (int idx = tid; idx < 2 * P * NS * 128; idx += 256) {
+    const int which = idx / (P * NS * 128);
+    const int pl = (idx / (NS * 128)) % P;
     const int wd = idx % (NS * 128);
+    uint32_t* kw = reinterpret_cast<uint32_t*>(tile + qt_kcodes_off() + pl * qt_plane_bytes(G));
+    uint32_t* vw = reinterpret_cast<uint32_t*>(tile + qt_vcodes_off(G, P) + pl * qt_plane_bytes(G));
     const int u = wd >> 7, lane = (wd >> 2) & 31, sub = wd & 3;
     const int hi = lane >> 2, j = lane & 3;
     uint32_t word = 0;
@@ -155,7 +159,7 @@ __device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kD], uint16
       for (int ks = 0; ks < 8; ++ks)
 #pragma unroll
         for (int h = 0; h < 2; ++h)
-          word |= static_cast<uint32_t>(sK[t][16 * ks + 8 * w + 2 * j + h]) << (16 * h + 2 * ks);
+          word |= static_cast<uint32_t>((sK[t][16 * ks + 8 * w + 2 * j + h] >> (2 * pl)) & 3u) << (16 * h + 2 * ks);
       kw[wd] = word;
     } else {
       const int dh = sub & 1, th = sub >> 1;
@@ -163,14 +167,14 @@ __device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kD], uint16
       for (int mt = 0; mt < 8; ++mt)
 #pragma unroll
         for (int h = 0; h < 2; ++h)
-          word |= static_cast<uint32_t>(sV[16 * u + 8 * th + 2 * j + h][16 * mt + 8 * dh + hi])
+          word |= static_cast<uint32_t>((sV[16 * u + 8 * th + 2 * j + h][16 * mt + 8 * dh + hi] >> (2 * pl)) & 3u)
                   << (16 * h + 2 * mt);
       vw[wd] = word;
     }
   }
 }
 
-template <int G>
+template <int G, int P>
 __global__ void __launch_bounds__(256)
 lq_compress_kernel(CacheView cv, LayerList layers, EvictList ev, int64_t tile0) {
   __shared__ __align__(16) uint16_t sK[G][kD];
@@ -181,7 +185,7 @@ lq_compress_kernel(CacheView cv, LayerList layers, EvictList ev, int64_t tile0) 
   const int tid = threadIdx.x;
   uint8_t* fpbase = cv.fp + layer * cv.fp_layer_stride + pair * cv.fp_head_stride;
   uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
-                  (tile0 + tau) * quant_tile_bytes(G);
+                  (tile0 + tau) * quant_tile_bytes(G, P);
 
   // 1. gather the removed rows
   for (int idx = tid; idx < G * 32; idx += 256) {
@@ -203,16 +207,18 @@ lq_compress_kernel(CacheView cv, LayerList layers, EvictList ev, int64_t tile0) 
     *reinterpret_cast<uint4*>(fpbase + fp_chunk_off(dst, c) + vo) = val;
   }
 
-  quantise_pack_tile<G>(sK, sV, tile, tid);
+  quantise_pack_tile<G, P>(sK, sV, tile, tid);
 }
 
 cudaError_t launch_compress(const CacheView& cv, const LayerList& layers, const EvictList& ev,
                             int64_t tile0, cudaStream_t st) {
   dim3 grid(cv.W / cv.G, cv.B * cv.Hkv, layers.n);
-  if (cv.G == 32)
-    lq_compress_kernel<32><<<grid, 256, 0, st>>>(cv, layers, ev, tile0);
-  else if (cv.G == 64)
-    lq_compress_kernel<64><<<grid, 256, 0, st>>>(cv, layers, ev, tile0);
+  if (cv.G == 32 && cv.planes == 1)
+    lq_compress_kernel<32, 1><<<grid, 256, 0, st>>>(cv, layers, ev, tile0);
+  else if (cv.G == 32 && cv.planes == 2)
+    lq_compress_kernel<32, 2><<<grid, 256, 0, st>>>(cv, layers, ev, tile0);
+  else if (cv.G == 64 && cv.planes == 1)
+    lq_compress_kernel<64, 1><<<grid, 256, 0, st>>>(cv, layers, ev, tile0);
   else
     return cudaErrorInvalidValue;
   return cudaGetLastError();
@@ -227,7 +233,7 @@ cudaError_t launch_compress(const CacheView& cv, const LayerList& layers, const 
 // remaining CTAs write the surviving rows to their final slots; the result is bit-identical to
 // the token-by-token path.
 // ---------------------------------------------------------------------------------------
-template <int G>
+template <int G, int P>
 __global__ void __launch_bounds__(256)
 lq_ingest_kernel(CacheView cv, int layer, const uint4* __restrict__ k, const uint4* __restrict__ v, int n_src,
                  const int* __restrict__ idx, int n_tiles, int n_fp, int64_t tile0) {
@@ -238,7 +244,7 @@ lq_ingest_kernel(CacheView cv, int layer, const uint4* __restrict__ k, const uin
   if (static_cast<int>(blockIdx.x) < n_tiles) {
     const int tau = blockIdx.x;
     uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
-                    (tile0 + tau) * quant_tile_bytes(G);
+                    (tile0 + tau) * quant_tile_bytes(G, P);
     for (int i = tid; i < G * 32; i += 256) {
       const int c = i & 15, which = (i >> 4) & 1, e = i >> 5;
       const int64_t t = idx[tau * G + e];
@@ -246,7 +252,7 @@ lq_ingest_kernel(CacheView cv, int layer, const uint4* __restrict__ k, const uin
       *reinterpret_cast<uint4*>(which ? &sV[e][c * 8] : &sK[e][c * 8]) = val;
     }
     __syncthreads();
-    quantise_pack_tile<G>(sK, sV, tile, tid);
+    quantise_pack_tile<G, P>(sK, sV, tile, tid);
   } else {
     const int i = (static_cast<int>(blockIdx.x) - n_tiles) * 256 + tid;
     if (i >= n_fp * 32) return;
@@ -263,10 +269,12 @@ cudaError_t launch_ingest(const CacheView& cv, int layer, const void* k, const v
   dim3 grid(n_tiles + (n_fp * 32 + 255) / 256, cv.B * cv.Hkv);
   const uint4* k4 = static_cast<const uint4*>(k);
   const uint4* v4 = static_cast<const uint4*>(v);
-  if (cv.G == 32)
-    lq_ingest_kernel<32><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, n_fp, tile0);
-  else if (cv.G == 64)
-    lq_ingest_kernel<64><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, n_fp, tile0);
+  if (cv.G == 32 && cv.planes == 1)
+    lq_ingest_kernel<32, 1><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, n_fp, tile0);
+  else if (cv.G == 32 && cv.planes == 2)
+    lq_ingest_kernel<32, 2><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, n_fp, tile0);
+  else if (cv.G == 64 && cv.planes == 1)
+    lq_ingest_kernel<64, 1><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, n_fp, tile0);
   else
     return cudaErrorInvalidValue;
   return cudaGetLastError();
@@ -277,27 +285,33 @@ cudaError_t launch_ingest(const CacheView& cv, int layer, const void* k, const v
 // ---------------------------------------------------------------------------------------
 __global__ void lq_export_codes_kernel(CacheView cv, int layer, int64_t n_quant, uint8_t* k_codes,
                                        uint8_t* v_codes) {
-  // one thread per output byte: (pair, token, byte j) -> channels 4j..4j+3
-  const int64_t per_pair = n_quant * (kD / 4);
+  // one thread per output byte: (pair, token, byte j) -> channels 4j..4j+3 (2-bit) or 2j, 2j+1 (4-bit)
+  const int P = cv.planes, cpb = 4 / P;  // codes per byte
+  const int64_t per_pair = n_quant * (kD / cpb);
   const int64_t total = static_cast<int64_t>(cv.B) * cv.Hkv * per_pair;
   for (int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; idx < total;
        idx += static_cast<int64_t>(gridDim.x) * blockDim.x) {
     const int64_t pair = idx / per_pair;
     const int64_t rem = idx % per_pair;
-    const int64_t tq = rem / (kD / 4);
-    const int jb = static_cast<int>(rem % (kD / 4));
+    const int64_t tq = rem / (kD / cpb);
+    const int jb = static_cast<int>(rem % (kD / cpb));
     const uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
-                          (tq / cv.G) * quant_tile_bytes(cv.G);
-    const uint32_t* kw = reinterpret_cast<const uint32_t*>(tile + qt_kcodes_off());
-    const uint32_t* vw = reinterpret_cast<const uint32_t*>(tile + qt_vcodes_off(cv.G));
+                          (tq / cv.G) * quant_tile_bytes(cv.G, P);
     const int t = static_cast<int>(tq % cv.G);
     uint32_t kb = 0, vb = 0;
-    for (int i = 0; i < 4; ++i) {
-      int word, bit;
-      kcode_pos(t, 4 * jb + i, word, bit);
-      kb |= ((kw[word] >> bit) & 3u) << (2 * i);
-      vcode_pos(t, 4 * jb + i, word, bit);
-      vb |= ((vw[word] >> bit) & 3u) << (2 * i);
+    for (int i = 0; i < cpb; ++i) {
+      uint32_t kcode = 0, vcode = 0;
+      for (int pl = 0; pl < P; ++pl) {
+        const uint32_t* kw = reinterpret_cast<const uint32_t*>(tile + qt_kcodes_off() + pl * qt_plane_bytes(cv.G));
+        const uint32_t* vw = reinterpret_cast<const uint32_t*>(tile + qt_vcodes_off(cv.G, P) + pl * qt_plane_bytes(cv.G));
+        int word, bit;
+        kcode_pos(t, cpb * jb + i, word, bit);
+        kcode |= ((kw[word] >> bit) & 3u) << (2 * pl);
+        vcode_pos(t, cpb * jb + i, word, bit);
+        vcode |= ((vw[word] >> bit) & 3u) << (2 * pl);
+      }
+      kb |= kcode << (2 * P * i);
+      vb |= vcode << (2 * P * i);
     }
     if (k_codes) k_codes[idx] = static_cast<uint8_t>(kb);
     if (v_codes) v_codes[idx] = static_cast<uint8_t>(vb);
@@ -317,7 +331,7 @@ __global__ void lq_export_params_kernel(CacheView cv, int layer, int64_t n_quant
       const int64_t grp = (idx / kD) % (n_quant / G);
       const int64_t pair = idx / kD / (n_quant / G);
       const uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
-                            grp * quant_tile_bytes(G);
+                            grp * quant_tile_bytes(G, cv.planes);
       if (k_scale) k_scale[idx] = reinterpret_cast<const uint16_t*>(tile + qt_kscale_off())[kparam_index(d)];
       if (k_zero) k_zero[idx] = reinterpret_cast<const uint16_t*>(tile + qt_kzero_off())[d];
     } else {
@@ -326,10 +340,10 @@ __global__ void lq_export_params_kernel(CacheView cv, int layer, int64_t n_quant
       const int64_t tq = (i2 / NG) % n_quant;
       const int64_t pair = i2 / NG / n_quant;
       const uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
-                            (tq / G) * quant_tile_bytes(G);
+                            (tq / G) * quant_tile_bytes(G, cv.planes);
       const int t = static_cast<int>(tq % G);
-      if (v_scale) v_scale[i2] = reinterpret_cast<const uint16_t*>(tile + qt_vscale_off(G))[vscale_index(t, g, G)];
-      if (v_zero) v_zero[i2] = reinterpret_cast<const uint16_t*>(tile + qt_vzero_off(G))[vzero_index(t, g, G)];
+      if (v_scale) v_scale[i2] = reinterpret_cast<const uint16_t*>(tile + qt_vscale_off(G, cv.planes))[vscale_index(t, g, G)];
+      if (v_zero) v_zero[i2] = reinterpret_cast<const uint16_t*>(tile + qt_vzero_off(G, cv.planes))[vzero_index(t, g, G)];
     }
   }
 }

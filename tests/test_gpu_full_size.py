@@ -18,13 +18,13 @@ def _built():
     build.build()
 
 
-def _run(B, Hq, Hkv, W, G, ctx, seed, n_steps, n_outliers=3, planted=False, image_stride=1):
+def _run(B, Hq, Hkv, W, G, ctx, seed, n_steps, n_outliers=3, planted=False, image_stride=1, bits=2):
     dev = "cuda"
     total = ctx + n_steps
     outl = synth.outlier_channels(seed, Hkv, D, n_outliers) if n_outliers else None
     u = synth.unit_vectors(seed, Hkv, D) if planted else None
-    cache = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=total + 8)
-    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G)
+    cache = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=total + 8, bits=bits)
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G, bits=bits)
     chunk = 2048
     for t0 in list(range(0, ctx, chunk)) + [ctx + i for i in range(n_steps)]:
         n = min(chunk, ctx - t0) if t0 < ctx else 1
@@ -75,3 +75,9 @@ def test_config4_gqa7_32k_planted_spikes():
 def test_config5_mha_128k_one_layer():
     inf = _run(B=1, Hq=32, Hkv=32, W=256, G=32, ctx=131072, seed=5, n_steps=1)
     assert (inf.n_quant, inf.n_fp) == (130560, 513)
+
+
+def test_config2_with_four_bit_codes():
+    # the llama3-8b-8k-int4 workload of bench.py: config 2 at the paper's second precision
+    inf = _run(B=8, Hq=32, Hkv=8, W=128, G=32, ctx=8192, seed=2, n_steps=2, bits=4)
+    assert inf.bytes_quant_per_token == 160

@@ -53,6 +53,43 @@ def test_shapes_and_edge_cases(kernel, B, Hq, Hkv, W, G, n_prefill, n_steps):
 
 
 @pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("B,Hq,Hkv,W,n_prefill,n_steps,chunk", [
+    (1, 8, 2, 128, 1024, 4, None),          # the tiny configuration at 4 bits, prompt ingested in one launch
+    (2, 4, 4, 32, 95, 4, 40),               # r = 1, crosses the first overflow step by step
+    (2, 14, 2, 64, 64 * 7 + 9, 3, None),    # GQA-7: two column blocks, fp16 p.v
+    (1, 16, 2, 32, 32 * 11 + 5, 2, 100),    # r = 8
+])
+def test_four_bit_cache(kernel, B, Hq, Hkv, W, n_prefill, n_steps, chunk):
+    """bits = 4 (16 levels, two codes per byte in the image; two 2-bit planes on the device): same bar."""
+    worst = run_case(B, Hq, Hkv, W, 32, n_prefill, n_steps, seed=13, kernel=kernel, bits=4, prefill_chunk=chunk)
+    assert worst <= 1.0
+
+
+def test_four_bit_is_closer_to_exact_attention_than_two_bit():
+    B, Hq, Hkv, W, G, D, n = 2, 8, 2, 64, 32, 128, 64 * 12
+    k, v = synth.keys_values(17, B, Hkv, n, D, "cuda", outliers=synth.outlier_channels(17, Hkv, D, 3))
+    q = synth.queries(17, B, Hq, D, 0, "cuda")
+    kf, vf = k.float().repeat_interleave(Hq // Hkv, 1), v.float().repeat_interleave(Hq // Hkv, 1)
+    p = torch.softmax(torch.einsum("bhd,bhtd->bht", q.float(), kf) / D ** 0.5, -1)
+    exact = torch.einsum("bht,bhtd->bhd", p, vf)
+    err = {}
+    for bits in (2, 4):
+        c = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=n + 8, bits=bits)
+        c.append(0, k, v)
+        out = torch.empty(B, Hq, D, device="cuda")
+        c.decode_attn(0, q, out)
+        err[bits] = float((out - exact).abs().max())
+        assert c.info(0).bytes_quant_per_token == (96 if bits == 2 else 160)
+        c.close()
+    assert err[4] < err[2] / 2
+
+
+def test_four_bit_needs_group_32():
+    with pytest.raises(LogQuantError):
+        LogQuantCache(1, 1, 8, 2, 64, 64, max_tokens=512, bits=4)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
 def test_chunked_prefill_and_manual_compress_give_the_same_image(kernel):
     # a prompt appended in ragged chunks, with the caller driving lq_compress, equals n single appends
     worst = run_case(2, 8, 2, 64, 32, 64 * 7 + 19, 2, seed=9, kernel=kernel, prefill_chunk=37, auto_compress=False)

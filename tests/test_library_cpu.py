@@ -43,7 +43,8 @@ def _dry(W=4, G=4, **kw):
 
 
 @pytest.mark.parametrize("bad", [dict(group=16), dict(group=48, window=96), dict(window=100), dict(head_dim=64),
-                                 dict(bits=4), dict(n_q_heads=18, n_kv_heads=2), dict(window=1024)])
+                                 dict(bits=3), dict(bits=8), dict(bits=4, group=64, window=128),
+                                 dict(n_q_heads=18, n_kv_heads=2), dict(window=1024)])
 def test_unsupported_configurations(bad):
     with pytest.raises(LogQuantError) as e:
         _dry(W=bad.pop("window", 128), G=bad.pop("group", 32), **bad)
@@ -127,3 +128,8 @@ def test_info_byte_accounting():
     c2.append(0, None, None, n_tokens=32769)
     inf = c2.info(0)
     assert (inf.n_quant, inf.n_fp, inf.bytes_quant_per_token) == (32256, 513, 80)
+    c4 = _dry(W=128, G=32, batch=8, n_q_heads=32, n_kv_heads=8, max_tokens=9000, bits=4)
+    c4.append(0, None, None, n_tokens=8193)
+    inf = c4.info(0)
+    assert (inf.n_quant, inf.n_fp, inf.bytes_quant_per_token) == (7936, 257, 160)
+    assert inf.bytes_decode_step == 64 * (7936 * 160 + 257 * 512)
