@@ -58,6 +58,14 @@ typedef enum {
 #define LQ_KERNEL_SCALAR 1 /* plain fp32 FMA kernel (slow; kept as an independent cross-check)   */
 #define LQ_KERNEL_MMA 2    /* mma.sync tensor-core kernel with bulk-copy staging                 */
 
+/* Which tokens an overflow step removes from the 3W full-precision tokens (in age order A[0..3W)):
+ *   LQ_FILTER_LOG     Algorithm 1: A[1], A[3], ..., A[2W-1]; kept tokens thin out with distance.
+ *   LQ_FILTER_RECENT  comparator, not the paper's method: the W oldest, A[0..W), so that only a recent
+ *                     window stays at full precision (the retention rule of the sliding-window
+ *                     quantisers the paper compares with, Sec. 2.2-2.3), same memory as LQ_FILTER_LOG. */
+#define LQ_FILTER_LOG 0
+#define LQ_FILTER_RECENT 1
+
 typedef struct {
   int32_t n_layers;      /* independent stacked layer caches, >= 1                               */
   int32_t batch;         /* B: sequences; all share one length                                   */
@@ -72,6 +80,7 @@ typedef struct {
   int32_t device;        /* CUDA device ordinal, or LQ_DEVICE_NONE for bookkeeping only          */
   int32_t kernel;        /* LQ_KERNEL_*                                                          */
   int32_t n_splits;      /* split-K CTAs per (batch row, KV head); 0 = chosen by the library     */
+  int32_t filter;        /* LQ_FILTER_*: which W tokens leave the full-precision store on overflow */
 } lq_config_t;
 
 typedef struct {

@@ -46,6 +46,8 @@ def lib():
         L.lqo_unpack4.argtypes = [p, i64, p]
         L.lqo_create_bits.restype = p
         L.lqo_create_bits.argtypes = [i32] * 7
+        L.lqo_create_policy.restype = p
+        L.lqo_create_policy.argtypes = [i32] * 8
         L.lqo_dequant.restype = f64
         L.lqo_dequant.argtypes = [C.c_uint16, C.c_uint16, C.c_uint8]
         L.lqo_pack2.argtypes = [p, i64, p]
@@ -176,9 +178,9 @@ def hardware_threads() -> int:
 class OracleCache:
     """One layer's mixed cache for B sequences: Algorithm 1 + quantiser + attention."""
 
-    def __init__(self, B, Hq, Hkv, D, W, G, bits=2):
+    def __init__(self, B, Hq, Hkv, D, W, G, bits=2, recent_only=False):
         self.B, self.Hq, self.Hkv, self.D, self.W, self.G, self.bits = B, Hq, Hkv, D, W, G, bits
-        self._h = lib().lqo_create_bits(B, Hq, Hkv, D, W, G, bits)
+        self._h = lib().lqo_create_policy(B, Hq, Hkv, D, W, G, bits, int(recent_only))
         if not self._h:
             raise ValueError("unsupported oracle configuration")
 

@@ -112,6 +112,7 @@ struct Head {  // one (batch row, kv head)
 struct Cache {
   int B, Hq, Hkv, D, W, G;
   int bits = 2;
+  int recent_only = 0;  // comparator: the W oldest tokens leave instead of Algorithm 1's odd positions
   int64_t n_seen = 0, n_events = 0;
   std::vector<int64_t> A;  // ids of the tokens kept at original precision, age order
   std::vector<int64_t> Q;  // ids of the quantised tokens, store order
@@ -123,8 +124,14 @@ struct Cache {
 void overflow_event(Cache& c) {
   const int W = c.W, D = c.D, G = c.G;
   std::vector<int64_t> evict_pos, keep_pos;
-  for (int i = 0; i < 2 * W; ++i) (i % 2 ? evict_pos : keep_pos).push_back(i);
-  for (int i = 2 * W; i < 3 * W; ++i) keep_pos.push_back(i);
+  if (c.recent_only) {
+    // Comparator (not the paper's method): only a recent window stays at full precision, as in the
+    // sliding-window quantisers the paper compares with (Sec. 2.2-2.3): A becomes A[W:3W].
+    for (int i = 0; i < 3 * W; ++i) (i < W ? evict_pos : keep_pos).push_back(i);
+  } else {
+    for (int i = 0; i < 2 * W; ++i) (i % 2 ? evict_pos : keep_pos).push_back(i);
+    for (int i = 2 * W; i < 3 * W; ++i) keep_pos.push_back(i);
+  }
   for (auto& h : c.heads) {
     // gather the W leaving rows, in eviction order
     std::vector<uint16_t> ek(static_cast<size_t>(W) * D), ev(static_cast<size_t>(W) * D);
@@ -341,6 +348,13 @@ void* lqo_create_bits(int B, int Hq, int Hkv, int D, int W, int G, int bits) {
   if (bits != 2 && bits != 4) return nullptr;
   Cache* c = static_cast<Cache*>(lqo_create(B, Hq, Hkv, D, W, G));
   if (c) c->bits = bits;
+  return c;
+}
+
+// ... and with the recent-window comparator in place of Algorithm 1's filter
+void* lqo_create_policy(int B, int Hq, int Hkv, int D, int W, int G, int bits, int recent_only) {
+  Cache* c = static_cast<Cache*>(lqo_create_bits(B, Hq, Hkv, D, W, G, bits));
+  if (c) c->recent_only = recent_only ? 1 : 0;
   return c;
 }
 

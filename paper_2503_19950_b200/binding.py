@@ -11,6 +11,7 @@ _LIB_PATH = os.path.join(_HERE, "liblogquant.so")
 
 LQ_DEVICE_NONE = -1
 LQ_KERNEL_AUTO, LQ_KERNEL_SCALAR, LQ_KERNEL_MMA = 0, 1, 2
+LQ_FILTER_LOG, LQ_FILTER_RECENT = 0, 1
 LQ_OK, LQ_ERR_INVALID_ARG, LQ_ERR_UNSUPPORTED, LQ_ERR_OOM, LQ_ERR_WINDOW_FULL, LQ_ERR_NOT_FULL, \
     LQ_ERR_CAPACITY, LQ_ERR_CUDA = range(8)
 
@@ -20,7 +21,7 @@ class lq_config_t(C.Structure):
                 ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("window", C.c_int32),
                 ("group", C.c_int32), ("bits", C.c_int32), ("max_tokens", C.c_int64),
                 ("auto_compress", C.c_int32), ("device", C.c_int32), ("kernel", C.c_int32),
-                ("n_splits", C.c_int32)]
+                ("n_splits", C.c_int32), ("filter", C.c_int32)]
 
 
 class lq_info_t(C.Structure):
@@ -125,10 +126,10 @@ class LogQuantCache:
     """Owner of one lq_cache_t.  Methods mirror the C entry points one to one."""
 
     def __init__(self, n_layers, batch, n_q_heads, n_kv_heads, window, group, max_tokens, head_dim=128, bits=2,
-                 auto_compress=True, device=0, kernel=LQ_KERNEL_AUTO, n_splits=0):
+                 auto_compress=True, device=0, kernel=LQ_KERNEL_AUTO, n_splits=0, filter=0):
         self._lib = load_library()
         self.cfg = lq_config_t(n_layers, batch, n_q_heads, n_kv_heads, head_dim, window, group, bits, max_tokens,
-                               int(auto_compress), device, kernel, n_splits)
+                               int(auto_compress), device, kernel, n_splits, filter)
         self._h = C.c_void_p()
         self._check(self._lib.lq_cache_create(C.byref(self.cfg), C.byref(self._h)), create=True)
 

@@ -95,11 +95,15 @@ void free_all(lq_cache* c) {
 
 int ratio(const lq_cache* c) { return c->cfg.n_q_heads / c->cfg.n_kv_heads; }
 
-// slots and ids of the tokens the next overflow removes: A[1], A[3], ..., A[2W-1] in age order
+// age position of the e-th token the next overflow removes: A[1], A[3], ..., A[2W-1] (Algorithm 1),
+// or A[0], ..., A[W-1] for the recent-window comparator
+int evict_pos(const lq_cache* c, int e) { return c->cfg.filter == LQ_FILTER_RECENT ? e : 2 * e + 1; }
+
+// slots and ids of the tokens the next overflow removes, in age order
 void next_evicted(const lq_cache* c, const LayerState& L, EvictList* ev, int32_t* ids) {
   const int W = c->cfg.window;
   for (int e = 0; e < W; ++e) {
-    const int slot = L.age_slot[2 * e + 1];
+    const int slot = L.age_slot[evict_pos(c, e)];
     if (ev) ev->slot[e] = static_cast<uint16_t>(slot);
     if (ids) ids[e] = L.slot_token[slot];
   }
@@ -110,9 +114,12 @@ void apply_event(const lq_cache* c, LayerState& L) {
   const int W = c->cfg.window;
   std::vector<int32_t> na;
   na.reserve(3 * W);
-  for (int i = 0; i < 2 * W; i += 2) na.push_back(L.age_slot[i]);
+  if (c->cfg.filter == LQ_FILTER_RECENT)
+    for (int i = W; i < 2 * W; ++i) na.push_back(L.age_slot[i]);
+  else
+    for (int i = 0; i < 2 * W; i += 2) na.push_back(L.age_slot[i]);
   for (int e = 0; e < W; ++e) {
-    const int hole = L.age_slot[2 * e + 1];
+    const int hole = L.age_slot[evict_pos(c, e)];
     L.quant_ids.push_back(L.slot_token[hole]);
     // the row of slot 2W+e (age position 2W+e) is moved into the hole
     L.slot_token[hole] = L.slot_token[2 * W + e];
@@ -204,6 +211,7 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
   if (cfg->window % cfg->group || cfg->window > kMaxW) return LQ_ERR_UNSUPPORTED;
   if (cfg->n_q_heads / cfg->n_kv_heads > kMaxRatio || cfg->n_layers > 128) return LQ_ERR_UNSUPPORTED;
   if (cfg->kernel < LQ_KERNEL_AUTO || cfg->kernel > LQ_KERNEL_MMA) return LQ_ERR_INVALID_ARG;
+  if (cfg->filter != LQ_FILTER_LOG && cfg->filter != LQ_FILTER_RECENT) return LQ_ERR_INVALID_ARG;
 
   lq_cache* c = new (std::nothrow) lq_cache;
   if (!c) return LQ_ERR_OOM;

@@ -925,7 +925,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
       // weights are known), and the four warp sums meet in shared memory.  The weight of a record
       // is computed by the lane that loaded its (m, l): warp w normalises heads w, w + 4.
       constexpr int RMAX = NCB == 1 ? 4 : 8;  // query heads per KV head this variant serves
-      constexpr int kSB = NCB == 1 ? 3 : 2;   // CTA records per batch
+      constexpr int kSB = 3;                  // CTA records per batch
       float* sm_w = reinterpret_cast<float*>(smem);  // [S * r] weights
       float* red = sm_w + kMergeMax;                 // [warp][r][128] partial sums
       const int nS = n_ctas_pair;

@@ -25,15 +25,15 @@ def assert_images_equal(got: dict, want: dict):
 
 def run_case(B, Hq, Hkv, W, G, n_prefill, n_steps, seed, kernel, n_outliers=3, check_image_every=1,
              sm_scale=0.0, n_splits=0, prefill_chunk=None, auto_compress=True, out_dtype=torch.float32,
-             q_gain=1.0, bits=2):
+             q_gain=1.0, bits=2, recent_only=False):
     """Prefill n_prefill tokens, then n_steps x (append 1 token, attention).  Returns max error ratio."""
     D = 128
     dev = "cuda"
     total = n_prefill + n_steps
     outl = synth.outlier_channels(seed, Hkv, D, n_outliers) if n_outliers else None
     cache = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=total + 8, auto_compress=auto_compress, kernel=kernel,
-                          n_splits=n_splits, bits=bits)
-    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G, bits=bits)
+                          n_splits=n_splits, bits=bits, filter=1 if recent_only else 0)
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G, bits=bits, recent_only=recent_only)
 
     def feed(start, n):
         k, v = synth.keys_values(seed, B, Hkv, n, D, dev, token_start=start, token_total=total, outliers=outl)

@@ -84,6 +84,15 @@ def test_four_bit_is_closer_to_exact_attention_than_two_bit():
     assert err[4] < err[2] / 2
 
 
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("bits,chunk", [(2, None), (4, 50)])
+def test_recent_window_comparator(kernel, bits, chunk):
+    """LQ_FILTER_RECENT: same kernels, other removal list (prompt ingestion and step-by-step overflow)."""
+    worst = run_case(2, 8, 2, 64, 32, 64 * 8 + 21, 3, seed=19, kernel=kernel, bits=bits, prefill_chunk=chunk,
+                     recent_only=True)
+    assert worst <= 1.0
+
+
 def test_four_bit_needs_group_32():
     with pytest.raises(LogQuantError):
         LogQuantCache(1, 1, 8, 2, 64, 64, max_tokens=512, bits=4)

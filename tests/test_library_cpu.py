@@ -91,6 +91,33 @@ def test_host_mirror_of_algorithm1_matches_oracle(W, G):
     assert img["kept_ids"].tolist() == A and img["quant_ids"].tolist() == Q
 
 
+@pytest.mark.parametrize("W,G", [(32, 32), (128, 64)])
+def test_recent_window_comparator_keeps_exactly_the_newest_tokens(W, G):
+    """LQ_FILTER_RECENT (comparator): the W oldest of the 3W full-precision tokens leave on overflow, so the
+    kept set is always the newest n_fp tokens and the store order is the token order (closed form), in the
+    host mirror and in the oracle alike."""
+    c = _dry(W=W, G=G, max_tokens=20 * W, filter=binding.LQ_FILTER_RECENT)
+    oc = oracle.OracleCache(1, 4, 2, 128, W, G, recent_only=True)
+    n = 0
+    rng = np.random.default_rng(W + 1)
+    while n < 12 * W:
+        step = int(rng.integers(1, 2 * W))
+        c.append(0, None, None, n_tokens=step)
+        oc.append(np.zeros((1, 2, step, 128), np.uint16), np.zeros((1, 2, step, 128), np.uint16))
+        n += step
+        inf = c.info(0)
+        n_ev = 0 if n <= 3 * W else (n - 3 * W + W - 1) // W
+        assert (inf.n_seen, inf.n_events, inf.n_quant, inf.n_fp) == (n, n_ev, n_ev * W, n - n_ev * W)
+        img = c.export(0, ids_only=True)
+        assert img["kept_ids"].tolist() == list(range(n_ev * W, n))
+        assert img["quant_ids"].tolist() == list(range(n_ev * W))
+        oimg = oc.export()
+        assert oimg["kept_ids"].tolist() == img["kept_ids"].tolist()
+        assert oimg["quant_ids"].tolist() == img["quant_ids"].tolist()
+    with pytest.raises(LogQuantError):
+        _dry(W=W, G=G, filter=7)
+
+
 def test_manual_compress_state_rules():
     W, G = 32, 32
     c = _dry(W=W, G=G, auto_compress=False, n_layers=3)
