@@ -165,7 +165,11 @@ lq_status_t lq_decode_attn(lq_cache_t* cache, int32_t layer, const void* q, floa
  * out_host ([B,Hq,D]).  sync != 0: synchronises `stream` before returning.  sync == 0: everything
  * is only enqueued (the host buffers must be pinned and must stay untouched, and out_host is
  * valid, once the caller has synchronised the stream); each layer has its own staging buffers,
- * so steps of different layers may be enqueued back to back. */
+ * so steps of different layers may be enqueued back to back.  When k_host, v_host and out_host are
+ * page-locked, device-addressable (cudaHostAlloc / cudaHostRegister, as reported by
+ * cudaPointerGetAttributes) and 16-byte aligned -- all four buffers --, the kernels read the inputs
+ * from and write the result to host memory directly (the append launch also stages the query in
+ * device memory); otherwise every buffer is copied through device staging memory. */
 lq_status_t lq_decode_step_host(lq_cache_t* cache, int32_t layer, const void* k_host,
                                 const void* v_host, const void* q_host, float sm_scale,
                                 float* out_host, int32_t sync, void* stream);

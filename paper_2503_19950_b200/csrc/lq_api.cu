@@ -318,7 +318,19 @@ lq_status_t ingest_prompt(lq_cache* c, int layer, const void* k, const void* v, 
 
 }  // namespace
 
+namespace {
+lq_status_t append_impl(lq_cache_t* c, int32_t layer, const void* k, const void* v, int32_t n, void* stream,
+                        const void* extra_src, void* extra_dst, int extra_bytes);
+}
+
 lq_status_t lq_append(lq_cache_t* c, int32_t layer, const void* k, const void* v, int32_t n, void* stream) {
+  return append_impl(c, layer, k, v, n, stream, nullptr, nullptr, 0);
+}
+
+namespace {
+// lq_append; the last launch also copies extra_bytes from extra_src to extra_dst (device-addressable)
+lq_status_t append_impl(lq_cache_t* c, int32_t layer, const void* k, const void* v, int32_t n, void* stream,
+                        const void* extra_src, void* extra_dst, int extra_bytes) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers || n < 0) return LQ_ERR_INVALID_ARG;
   if (!c->dry && (!k || !v)) return LQ_ERR_INVALID_ARG;
   if (!c->dry && ((reinterpret_cast<uintptr_t>(k) | reinterpret_cast<uintptr_t>(v)) & 15)) return LQ_ERR_INVALID_ARG;
@@ -327,7 +339,8 @@ lq_status_t lq_append(lq_cache_t* c, int32_t layer, const void* k, const void* v
   if (L.n_seen + n > c->cfg.max_tokens) return LQ_ERR_CAPACITY;
   if (!c->cfg.auto_compress && L.n_fp + n > 3 * W) return LQ_ERR_WINDOW_FULL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (!c->dry && c->cfg.auto_compress && L.n_seen == 0 && n > 3 * W) return ingest_prompt(c, layer, k, v, n, st);
+  if (!c->dry && c->cfg.auto_compress && L.n_seen == 0 && n > 3 * W && extra_bytes == 0)
+    return ingest_prompt(c, layer, k, v, n, st);
   int done = 0;
   while (done < n) {
     if (L.n_fp == 3 * W) {
@@ -336,7 +349,9 @@ lq_status_t lq_append(lq_cache_t* c, int32_t layer, const void* k, const void* v
     }
     const int take = std::min(n - done, 3 * W - L.n_fp);
     if (!c->dry) {
-      cudaError_t e = launch_append(c->cv, layer, k, v, n, done, take, L.n_fp, st);
+      const bool last = done + take == n;
+      cudaError_t e = launch_append(c->cv, layer, k, v, n, done, take, L.n_fp, st, last ? extra_src : nullptr,
+                                    last ? extra_dst : nullptr, last ? extra_bytes : 0);
       if (e != cudaSuccess) return cuda_fail(c, e, "lq_append_kernel");
       c->n_launches++;
     }
@@ -350,6 +365,7 @@ lq_status_t lq_append(lq_cache_t* c, int32_t layer, const void* k, const void* v
   }
   return LQ_OK;
 }
+}  // namespace
 
 lq_status_t lq_compress(lq_cache_t* c, int32_t layer, void* stream) {
   if (!c || layer < -1 || layer >= c->cfg.n_layers) return LQ_ERR_INVALID_ARG;
@@ -432,19 +448,40 @@ lq_status_t lq_decode_step_host(lq_cache_t* c, int32_t layer, const void* k_host
   uint8_t* sq = c->stage_q + layer * qb;
   uint8_t* so = c->stage_out + layer * qb * 2;
   cudaError_t e;
-  if ((e = cudaMemcpyAsync(sk, k_host, kvb, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
-      (e = cudaMemcpyAsync(sv, v_host, kvb, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
-      (e = cudaMemcpyAsync(sq, q_host, qb, cudaMemcpyHostToDevice, st)) != cudaSuccess)
-    return cuda_fail(c, e, "host-to-device copy");
+  // Page-locked host buffers that the device can address are used in place: the append kernel reads
+  // the new k and v rows straight from host memory and the attention kernel writes its result
+  // straight into out_host; the query, which every CTA of a pair reads, is moved to device memory
+  // by the append launch.  No separate copy is left.  Anything else goes through the staging
+  // buffers with one copy each.
+  auto mapped = [](const void* p) -> void* {
+    cudaPointerAttributes at;
+    if ((reinterpret_cast<uintptr_t>(p) & 15) != 0) return nullptr;
+    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+  };
+  void* dk = mapped(k_host);
+  void* dv = mapped(v_host);
+  void* dq = mapped(q_host);
+  void* dout = mapped(out_host);
+  const bool direct = dk && dv && dq && dout;
+  if (!direct) {
+    if ((e = cudaMemcpyAsync(sk, k_host, kvb, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(sv, v_host, kvb, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+      return cuda_fail(c, e, "host-to-device copy");
+    if ((e = cudaMemcpyAsync(sq, q_host, qb, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+      return cuda_fail(c, e, "host-to-device copy");
+  }
   if (L.n_fp == 3 * c->cfg.window) {
     lq_status_t s = run_events(c, std::vector<int>{layer}, st);
     if (s != LQ_OK) return s;
   }
-  lq_status_t s = lq_append(c, layer, sk, sv, 1, stream);
+  // in place: the append launch also moves the query into device memory (every CTA of a pair reads it)
+  lq_status_t s = direct ? append_impl(c, layer, dk, dv, 1, stream, dq, sq, static_cast<int>(qb))
+                         : lq_append(c, layer, sk, sv, 1, stream);
   if (s != LQ_OK) return s;
-  s = lq_decode_attn(c, layer, sq, sm_scale, so, 0, stream);
+  s = lq_decode_attn(c, layer, sq, sm_scale, direct ? dout : so, 0, stream);
   if (s != LQ_OK) return s;
-  if ((e = cudaMemcpyAsync(out_host, so, qb * 2, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+  if (!direct && (e = cudaMemcpyAsync(out_host, so, qb * 2, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
     return cuda_fail(c, e, "device-to-host copy");
   if (sync && (e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(c, e, "cudaStreamSynchronize");
   return LQ_OK;

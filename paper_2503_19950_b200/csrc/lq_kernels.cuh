@@ -31,8 +31,10 @@ struct LayerList {
 
 // K1: write n_tokens new rows into fp slots [slot0, slot0 + n_tokens) of one layer.
 // k, v: [B, Hkv, n_src_tokens, D] bf16; tokens [src0, src0 + n_tokens) of them are written.
+// extra_bytes (a multiple of 16) are copied from extra_src to extra_dst by the same launch.
 cudaError_t launch_append(const CacheView& cv, int layer, const void* k, const void* v,
-                          int n_src_tokens, int src0, int n_tokens, int slot0, cudaStream_t st);
+                          int n_src_tokens, int src0, int n_tokens, int slot0, cudaStream_t st,
+                          const void* extra_src = nullptr, void* extra_dst = nullptr, int extra_bytes = 0);
 
 // K2: overflow step for the listed layers (all of them in the same state): quantise + pack the W
 // rows of `ev` into quant tiles [tile0, tile0 + W/G), then move rows 2W+e into slot ev.slot[e].

@@ -8,18 +8,24 @@ namespace lq {
 
 // ---------------------------------------------------------------------------------------
 // K1  append: Algorithm 1, branch length(A) < 3W -- the new rows go to the next free slots.
-// One thread per 16-byte chunk of a K or V row.
+// One thread per 16-byte chunk of a K or V row.  The threads after those copy `extra_chunks`
+// 16-byte chunks from extra_src to extra_dst (the host-buffer step stages its query this way, in
+// the same launch).
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 lq_append_kernel(CacheView cv, int layer, const uint4* __restrict__ k, const uint4* __restrict__ v,
-                 int n_src, int src0, int n, int slot0) {
+                 int n_src, int src0, int n, int slot0, const uint4* __restrict__ extra_src, uint4* extra_dst,
+                 int extra_chunks) {
   // programmatic dependent launch: overlap this kernel's launch with the tail of the previous
   // kernel of the stream, but write nothing before that kernel has finished
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   const int64_t total = static_cast<int64_t>(cv.B) * cv.Hkv * n * 32;
-  if (idx >= total) return;
+  if (idx >= total) {
+    if (idx - total < extra_chunks) extra_dst[idx - total] = extra_src[idx - total];
+    return;
+  }
   const int c = static_cast<int>(idx & 15);
   const int which = static_cast<int>((idx >> 4) & 1);
   const int64_t row = idx >> 5;
@@ -32,8 +38,9 @@ lq_append_kernel(CacheView cv, int layer, const uint4* __restrict__ k, const uin
 }
 
 cudaError_t launch_append(const CacheView& cv, int layer, const void* k, const void* v, int n_src,
-                          int src0, int n, int slot0, cudaStream_t st) {
-  const int64_t total = static_cast<int64_t>(cv.B) * cv.Hkv * n * 32;
+                          int src0, int n, int slot0, cudaStream_t st, const void* extra_src, void* extra_dst,
+                          int extra_bytes) {
+  const int64_t total = static_cast<int64_t>(cv.B) * cv.Hkv * n * 32 + extra_bytes / 16;
   const int blocks = static_cast<int>((total + 255) / 256);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(blocks);
@@ -45,7 +52,8 @@ cudaError_t launch_append(const CacheView& cv, int layer, const void* k, const v
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, lq_append_kernel, cv, layer, static_cast<const uint4*>(k),
-                            static_cast<const uint4*>(v), n_src, src0, n, slot0);
+                            static_cast<const uint4*>(v), n_src, src0, n, slot0,
+                            static_cast<const uint4*>(extra_src), static_cast<uint4*>(extra_dst), extra_bytes / 16);
 }
 
 // ---------------------------------------------------------------------------------------

@@ -210,7 +210,9 @@ def test_prompt_ingestion_in_one_launch_equals_token_by_token(W, G, n):
     one.close(); seq.close(); oc.close()
 
 
-def test_decode_step_with_host_buffers():
+@pytest.mark.parametrize("pinned", [True, False])
+def test_decode_step_with_host_buffers(pinned):
+    """Page-locked buffers are read and written by the kernels in place; pageable ones are copied."""
     B, Hq, Hkv, W, G, D = 2, 8, 2, 32, 32, 128
     N = 3 * W  # the first host step has to run the overflow itself, even with auto_compress = 0
     cache = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=N + 8, auto_compress=False)
@@ -221,8 +223,9 @@ def test_decode_step_with_host_buffers():
     for step in range(3):
         k1, v1 = synth.keys_values(40, B, Hkv, 1, D, "cpu", token_start=N + step, token_total=N + 4)
         q = synth.queries(40, B, Hq, D, step, "cpu")
-        k1, v1, q = k1.pin_memory(), v1.pin_memory(), q.pin_memory()
-        out = torch.empty(B, Hq, D, dtype=torch.float32).pin_memory()
+        out = torch.full((B, Hq, D), float("nan"), dtype=torch.float32)
+        if pinned:
+            k1, v1, q, out = k1.pin_memory(), v1.pin_memory(), q.pin_memory(), out.pin_memory()
         cache.decode_step_host(0, k1, v1, q, out)
         oc.append(synth.bf16_bits(k1), synth.bf16_bits(v1))
         ref = oc.attention(synth.bf16_bits(q), 1 / np.sqrt(D))
