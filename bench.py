@@ -313,6 +313,8 @@ def run_ours(args, wl, rank, world, device):
         "per_layer_us": ms_max / steps / L * 1e3,
         "algorithmic_gbs_whole_step": bytes_step_last / (ms_max / steps * 1e-3) / 1e9,
         "gpu_launches": int(launches),
+        # bf16 cache bytes / mixed cache bytes actually read per step (scale and zero counted)
+        "compression_ratio": (B * Hkv * (int(inf.n_quant) + int(inf.n_fp)) * 4 * D) / max(int(inf.bytes_decode_step), 1),
         "compress_event": comp,
         "clocks": clk.summary(),
         "e2e": {"value": aggregate_throughput(kv_e2e, world, e2e_ms_max), "unit": "KV tokens/s",
