@@ -174,8 +174,7 @@ def run_ours(args, wl, rank, world, device):
     def one_step(i):
         s = i % Q_ROTATE
         for l in range(L):
-            cache.append(l, ks[l][s], vs[l][s])
-            cache.decode_attn(l, qs[l][s], outs[l])
+            cache.append_decode_attn(l, ks[l][s], vs[l][s], qs[l][s], outs[l])
 
     def barrier():
         torch.cuda.synchronize()
@@ -307,7 +306,8 @@ def run_ours(args, wl, rank, world, device):
         "config": {"workload": args.workload, "layers": L, "batch": B, "q_heads": Hq, "kv_heads": Hkv,
                    "head_dim": D, "context": ctx, "window": W, "group": G, "bits": bits,
                    "n_quant": int(inf.n_quant), "n_fp": int(inf.n_fp), "n_splits": int(inf.n_splits), "n_ctas": int(inf.n_ctas),
-                   "step": "per layer: lq_append (+lq_compress on overflow) + lq_decode_attn",
+                   "step": "per layer: lq_append_decode_attn (append and attention in one launch; the overflow step and "
+                           "a separate append when the window is full)",
                    "l2": "inputs larger than L2: %.2f GB of cache touched per step" % (bytes_step_last / 1e9),
                    "replicas": "independent per GPU, no collective on the data path"},
         "per_layer_us": ms_max / steps / L * 1e3,

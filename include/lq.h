@@ -159,6 +159,17 @@ lq_status_t lq_compress(lq_cache_t* cache, int32_t layer, void* stream);
 lq_status_t lq_decode_attn(lq_cache_t* cache, int32_t layer, const void* q, float sm_scale,
                            void* out, int32_t out_dtype, void* stream);
 
+/* lq_append of ONE token followed by lq_decode_attn, in one launch: the attention kernel takes the
+ * new row from k, v ([B, Hkv, 1, D] bf16, device) where it belongs in its pass over the cache and
+ * writes it to the full-precision store on the way (Algorithm 1's append and Eq. 2 of the same
+ * step; the result is the one of the two separate calls).  When the window is full (the overflow
+ * step has to run in between; auto_compress = 0 then gives LQ_ERR_WINDOW_FULL), the plain kernel
+ * is selected, or the cache is so large that the saved launch no longer pays, the call simply
+ * makes the two calls.  Errors leave the cache unchanged. */
+lq_status_t lq_append_decode_attn(lq_cache_t* cache, int32_t layer, const void* k, const void* v,
+                                  const void* q, float sm_scale, void* out, int32_t out_dtype,
+                                  void* stream);
+
 /* One decode step of one layer with HOST buffers: copies k_host, v_host ([B,Hkv,1,D] bf16) and
  * q_host ([B,Hq,D] bf16) to the device, appends (running the overflow step first when the window
  * is full, whatever auto_compress says), runs decode attention and copies the fp32 result to

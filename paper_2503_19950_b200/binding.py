@@ -42,7 +42,7 @@ class lq_device_image_t(C.Structure):
                [(n, C.c_void_p) for n in ("fp_k", "fp_v", "k_codes", "v_codes", "k_scale", "k_zero", "v_scale", "v_zero")]
 
 
-SYMBOLS = ["lq_cache_create", "lq_destroy", "lq_append", "lq_compress", "lq_decode_attn",
+SYMBOLS = ["lq_cache_create", "lq_destroy", "lq_append", "lq_compress", "lq_decode_attn", "lq_append_decode_attn",
            "lq_decode_step_host", "lq_profile_enable", "lq_profile_read", "lq_kernel_status", "lq_cache_info", "lq_export",
            "lq_next_evicted_ids", "lq_decode_attn_image_static", "lq_status_str", "lq_last_error"]
 
@@ -69,6 +69,7 @@ def load_library():
         L.lq_append.argtypes = [vp, i32, vp, vp, i32, vp]
         L.lq_compress.argtypes = [vp, i32, vp]
         L.lq_decode_attn.argtypes = [vp, i32, vp, C.c_float, vp, i32, vp]
+        L.lq_append_decode_attn.argtypes = [vp, i32, vp, vp, vp, C.c_float, vp, i32, vp]
         L.lq_decode_step_host.argtypes = [vp, i32, vp, vp, vp, C.c_float, vp, i32, vp]
         L.lq_kernel_status.argtypes = [vp, C.POINTER(C.c_int32)]
         L.lq_profile_enable.argtypes = [vp, i32]
@@ -160,6 +161,14 @@ class LogQuantCache:
 
     def compress(self, layer=-1, stream=None):
         self._check(self._lib.lq_compress(self._h, layer, None if self.cfg.device < 0 else _stream(stream)))
+
+    def append_decode_attn(self, layer, k, v, q, out, sm_scale=0.0, stream=None):
+        """Append one token and run decode attention in one launch (k, v: [B, Hkv, 1, D] bf16)."""
+        import torch
+        assert k.shape[2] == 1 and v.shape == k.shape
+        out_dtype = 1 if out.dtype == torch.bfloat16 else 0
+        self._check(self._lib.lq_append_decode_attn(self._h, layer, _ptr(k), _ptr(v), _ptr(q), sm_scale, _ptr(out),
+                                                    out_dtype, _stream(stream)))
 
     def decode_attn(self, layer, q, out, sm_scale=0.0, stream=None):
         import torch

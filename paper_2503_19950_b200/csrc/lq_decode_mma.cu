@@ -401,6 +401,17 @@ __device__ __forceinline__ void quant_bias(const uint32_t (&qs)[NCB][8][2], uint
   }
 }
 
+// ---- fused append: one new row (256 B, lane = 8 B) replaces row `row` of a landed K or V half tile
+// in shared memory and goes to the same place of the fp store ---------------------------------
+__device__ __forceinline__ void patch_new_row(uint32_t half_tile_smem, uint8_t* half_tile_global, const void* rows,
+                                              int pair, int row, int lane) {
+  const uint2 x = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint8_t*>(rows) + pair * (kD * 2)) + lane);
+  const int off = row * 256 + (((lane >> 1) ^ (row & 7)) << 4) + (lane & 1) * 8;
+  asm volatile("st.shared.v2.u32 [%0], {%1,%2};" ::"r"(half_tile_smem + off), "r"(x.x), "r"(x.y) : "memory");
+  *reinterpret_cast<uint2*>(half_tile_global + off) = x;
+  __syncwarp();
+}
+
 // ---- one quant tile: one key group of G tokens ---------------------------------------------
 // PL = 2-bit planes per code.  A 4-bit code is 4 * (high plane) + (low plane): the high plane goes
 // through the same contractions first, its score accumulators are multiplied by 4 before the low
@@ -596,7 +607,9 @@ constexpr int kMergeMax = 2048;  // S * r records the fused second pass can stag
 // the pair (4 warps each) share them by a static, cost-weighted partition (see below); any
 // assignment is legal because every warp keeps its own online-softmax state.  A warp keeps up to
 // two loads in flight.
-template <int G, int NCB, int PL>
+// FUSED: the launch also appends one token (DecodeArgs::new_k); a separate instantiation so that
+// the plain kernel's main loop is not touched.
+template <int G, int NCB, int PL, bool FUSED>
 __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerSm - 1) lq_decode_mma_kernel(DecodeArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   const CacheView& cv = a.cv;
@@ -788,9 +801,15 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
         process_quant_tile<G, NCB, PL>(st, qs, sbase + t * TILE, bias, kq, lane, oddmask, a.zero);
       }
     } else if (desc >= 0) {
+      if (FUSED && desc == (a.new_slot >> 4))
+        patch_new_row(sbase, const_cast<uint8_t*>(fpbase) + static_cast<int64_t>(desc) * kFpTileBytes, a.new_k, pair,
+                      a.new_slot & 15, lane);
       const int nv = min(16, a.n_fp - desc * 16);
       process_fp_keys<NCB>(st, qs, sbase, nv, kc, lane, oddmask, a.zero, fb0, fb1);
     } else {
+      if (FUSED && -1 - desc == (a.new_slot >> 4))
+        patch_new_row(sbase, const_cast<uint8_t*>(fpbase) + static_cast<int64_t>(-1 - desc) * kFpTileBytes + kFpTileVOffset,
+                      a.new_v, pair, a.new_slot & 15, lane);
       process_fp_values<NCB>(st, sbase, lane, fb0, fb1);
     }
     __syncwarp();
@@ -1048,19 +1067,24 @@ void plan_decode_mma(DecodeArgs& a, int sm_count, int max_records, int s_overrid
 cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
   const int r = a.cv.Hq / a.cv.Hkv;
   void (*kern)(DecodeArgs) = nullptr;
-  if (a.cv.G == 32 && a.cv.planes == 1) kern = r <= 4 ? lq_decode_mma_kernel<32, 1, 1> : lq_decode_mma_kernel<32, 2, 1>;
-  else if (a.cv.G == 32 && a.cv.planes == 2) kern = r <= 4 ? lq_decode_mma_kernel<32, 1, 2> : lq_decode_mma_kernel<32, 2, 2>;
-  else if (a.cv.G == 64 && a.cv.planes == 1) kern = r <= 4 ? lq_decode_mma_kernel<64, 1, 1> : lq_decode_mma_kernel<64, 2, 1>;
+  const bool fused = a.new_k != nullptr;
+#define LQ_PICK(G_, P_)                                                                                   \
+  kern = r <= 4 ? (fused ? lq_decode_mma_kernel<G_, 1, P_, true> : lq_decode_mma_kernel<G_, 1, P_, false>) \
+                : (fused ? lq_decode_mma_kernel<G_, 2, P_, true> : lq_decode_mma_kernel<G_, 2, P_, false>)
+  if (a.cv.G == 32 && a.cv.planes == 1) LQ_PICK(32, 1);
+  else if (a.cv.G == 32 && a.cv.planes == 2) LQ_PICK(32, 2);
+  else if (a.cv.G == 64 && a.cv.planes == 1) LQ_PICK(64, 1);
   else return cudaErrorInvalidValue;
+#undef LQ_PICK
   static_assert(kSmemStages >= static_cast<int>((kWarps * 8 * (kD + 4) + 3 * kWarps * 8 + 16) * sizeof(float)) &&
                     kSmemStages >= (kMergeMax + kWarps * kMaxRatio * kD) * 4,
                 "merge scratch");
   // opt in to the dynamic shared memory size once per (device, kernel variant)
-  static bool configured[64][8] = {};
+  static bool configured[64][16] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  const int variant = (a.cv.planes == 2 ? 4 : 0) + (a.cv.G == 64 ? 2 : 0) + (r <= 4 ? 0 : 1);
+  const int variant = (fused ? 8 : 0) + (a.cv.planes == 2 ? 4 : 0) + (a.cv.G == 64 ? 2 : 0) + (r <= 4 ? 0 : 1);
   if (dev < 0 || dev >= 64 || !configured[dev][variant]) {
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;

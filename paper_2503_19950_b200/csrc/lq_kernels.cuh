@@ -73,6 +73,12 @@ struct DecodeArgs {
   float* part_ml;
   void* out;
   int out_bf16;
+  // tensor-core kernel, fused append: when new_k is not null, row new_slot of the fp store (counted in n_fp) is
+  // not in memory yet; the warp that visits its tile takes the row from new_k / new_v ([B, Hkv, 1, 128] bf16) and
+  // writes it to the store
+  const void* new_k;
+  const void* new_v;
+  int new_slot;
   int* status;  // device word; kernels OR error bits into it (bounded waits that gave up)
   int* tickets; // one 128-byte line per (b, kv): word [1] is the arrival counter of the fused second
                 // pass, 0 at rest

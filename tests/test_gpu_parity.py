@@ -210,6 +210,45 @@ def test_prompt_ingestion_in_one_launch_equals_token_by_token(W, G, n):
     one.close(); seq.close(); oc.close()
 
 
+@pytest.mark.parametrize("B,Hq,Hkv,W,G,bits,n0", [
+    (2, 8, 2, 32, 32, 2, 3 * 32 - 5),     # crosses an overflow step (falls back to the two calls there)
+    (1, 14, 2, 64, 64, 2, 64 * 5 + 15),   # GQA-7; the new row opens a new 16-slot tile on the way
+    (2, 8, 8, 32, 32, 4, 32 * 7 + 1),     # r = 1, 4-bit codes
+])
+def test_append_and_attention_in_one_launch(B, Hq, Hkv, W, G, bits, n0):
+    """lq_append_decode_attn: same image, same attention bits as lq_append + lq_decode_attn, one launch."""
+    D, n_steps = 128, 20
+    k, v = synth.keys_values(23, B, Hkv, n0 + n_steps, D, "cuda")
+    fused = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=n0 + n_steps + 8, bits=bits)
+    plain = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=n0 + n_steps + 8, bits=bits)
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G, bits=bits)
+    for c in (fused, plain):
+        c.append(0, k[:, :, :n0].contiguous(), v[:, :, :n0].contiguous())
+    oc.append(synth.bf16_bits(k[:, :, :n0]), synth.bf16_bits(v[:, :, :n0]))
+    single = 0
+    for t in range(n_steps):
+        k1, v1 = k[:, :, n0 + t:n0 + t + 1].contiguous(), v[:, :, n0 + t:n0 + t + 1].contiguous()
+        q = synth.queries(23, B, Hq, D, t, "cuda")
+        o1 = torch.full((B, Hq, D), float("nan"), device="cuda")
+        o2 = torch.full((B, Hq, D), float("nan"), device="cuda")
+        before = fused.info(0).n_kernel_launches
+        fused.append_decode_attn(0, k1, v1, q, o1)
+        single += fused.info(0).n_kernel_launches == before + 1
+        plain.append(0, k1, v1)
+        plain.decode_attn(0, q, o2)
+        torch.cuda.synchronize()
+        assert torch.equal(o1, o2), f"step {t}"
+        oc.append(synth.bf16_bits(k1), synth.bf16_bits(v1))
+        ref = oc.attention(synth.bf16_bits(q), 1 / np.sqrt(D))
+        assert np.abs(o1.cpu().numpy() - ref).max() <= attn_tolerance(ref)
+        if t % 6 == 0 or t == n_steps - 1:
+            assert_images_equal(fused.export(0), oc.export())
+    assert single >= n_steps - 1  # every step but the one that had to run the overflow step in between
+    # (caches above 192 MB per launch take the two calls as well; the full-size tests cover those sizes)
+    assert fused.kernel_status() == 0
+    fused.close(); plain.close(); oc.close()
+
+
 @pytest.mark.parametrize("pinned", [True, False])
 def test_decode_step_with_host_buffers(pinned):
     """Page-locked buffers are read and written by the kernels in place; pageable ones are copied."""
