@@ -43,16 +43,12 @@ constexpr int kWarpStageBytes = 12288;
 __host__ __device__ constexpr int stage_bytes(int) { return 6144; }
 __host__ __device__ constexpr int n_stages(int G) { return kWarpStageBytes / stage_bytes(G); }
 constexpr int kMaxStages = 3;
-#ifndef LQ_CTAS_PER_SM
-#define LQ_CTAS_PER_SM 4
-#endif
-constexpr int kCtasPerSm = LQ_CTAS_PER_SM;
+constexpr int kCtasPerSm = 4;  // at 128 registers and 51 KB of shared memory; 3 and 5 both measured slower
 constexpr uint32_t kFull = 0xFFFFFFFFu;
 constexpr int kSpinLimit = 1 << 22;
-#ifndef LQ_FP_COST8
-#define LQ_FP_COST8 8
-#endif
-constexpr int kFpCost8 = LQ_FP_COST8;  // cost of one fp tile (16 bf16 tokens) in eighths of a quant tile
+// cost of one fp tile (16 bf16 tokens, two loads) in eighths of a quant tile: 4 to 12 measured alike,
+// 2 and 16 slower
+constexpr int kFpCost8 = 8;
 
 // ---- PTX wrappers ----------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -182,11 +178,8 @@ __device__ __forceinline__ uint32_t ext_f16(uint32_t w, uint32_t w10) {
 // probabilities carry a factor 2^64 (kPExp) so that products with bf16 subnormal codes stay normal.
 // p.v flavour.  bf16_pv: columns are (hi, lo) per head, everything bf16, exact products, r <= 4 only.
 // Otherwise: heads on the 8 columns, value codes as fp16 subnormals, p * s_v rounded to fp16.
-#ifndef LQ_BF16_PV
-#define LQ_BF16_PV 1
-#endif
 template <int NCB>
-__host__ __device__ constexpr bool bf16_pv() { return LQ_BF16_PV != 0 && NCB == 1; }
+__host__ __device__ constexpr bool bf16_pv() { return NCB == 1; }
 
 template <int NCB>
 struct WarpState {

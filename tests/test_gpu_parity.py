@@ -98,6 +98,30 @@ def test_four_bit_needs_group_32():
         LogQuantCache(1, 1, 8, 2, 64, 64, max_tokens=512, bits=4)
 
 
+def _random_cases(n, seed):
+    rng = np.random.default_rng(seed)
+    cases = []
+    while len(cases) < n:
+        G = int(rng.choice([32, 64]))
+        W = int(rng.choice([w for w in (32, 64, 96, 128, 192, 256) if w % G == 0]))
+        Hkv = int(rng.choice([1, 2, 4]))
+        r = int(rng.choice([1, 2, 3, 4, 5, 7, 8]))
+        bits = 4 if (G == 32 and rng.random() < 0.3) else 2
+        B = int(rng.integers(1, 4))
+        n_prefill = int(rng.integers(1, 9 * W))
+        chunk = None if rng.random() < 0.5 else int(rng.integers(1, 3 * W))
+        cases.append((B, Hkv * r, Hkv, W, G, bits, n_prefill, chunk, bool(rng.random() < 0.2)))
+    return cases
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,W,G,bits,n_prefill,chunk,recent", _random_cases(12, 2024))
+def test_seeded_random_configurations(B, Hq, Hkv, W, G, bits, n_prefill, chunk, recent):
+    """A seeded draw over head ratios, windows, groups, code widths, prompt lengths, chunkings and filters."""
+    worst = run_case(B, Hq, Hkv, W, G, n_prefill, 2, seed=100 + n_prefill, kernel=LQ_KERNEL_MMA, bits=bits,
+                     prefill_chunk=chunk, recent_only=recent, check_image_every=1)
+    assert worst <= 1.0
+
+
 @pytest.mark.parametrize("kernel", KERNELS)
 def test_chunked_prefill_and_manual_compress_give_the_same_image(kernel):
     # a prompt appended in ragged chunks, with the caller driving lq_compress, equals n single appends
