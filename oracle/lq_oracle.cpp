@@ -17,6 +17,12 @@
 //                         x^    = zero + code * scale
 //                     keys: one group = G consecutive evicted tokens of one channel;
 //                     values: one group = G consecutive channels of one token.
+//                     When W is not a multiple of G (the paper's own settings, Sec. 3.1: G = 64
+//                     with a reserved length of 128 or 256 tokens, i.e. W = 42 or 85) an overflow
+//                     step does not yield whole key groups.  The paper does not say what happens
+//                     then; the reading taken here: tokens the filter removes wait, still at
+//                     original precision, in removal order, and every time G of them are waiting
+//                     the oldest G form one key group and are quantised.
 //                     The paper's second precision (the 4-bit rows of its accuracy tables,
 //                     Sec. 3.2) is the same quantiser with 16 levels: scale = bf16_rne((max -
 //                     min) / 15), codes 0..15.
@@ -104,6 +110,7 @@ double dequant(uint16_t scale, uint16_t zero, uint8_t code) {
 // ---- the cache ---------------------------------------------------------------------
 struct Head {  // one (batch row, kv head)
   std::vector<uint16_t> fp_k, fp_v;      // [len(A)][D], rows in the order of list A
+  std::vector<uint16_t> pend_k, pend_v;  // [len(P)][D], rows in the order of list P
   std::vector<uint8_t> k_codes, v_codes;  // [nq][D], one code per byte (unpacked)
   std::vector<uint16_t> k_scale, k_zero;  // [nq/G][D]
   std::vector<uint16_t> v_scale, v_zero;  // [nq][D/G]
@@ -115,6 +122,7 @@ struct Cache {
   int recent_only = 0;  // comparator: the W oldest tokens leave instead of Algorithm 1's odd positions
   int64_t n_seen = 0, n_events = 0;
   std::vector<int64_t> A;  // ids of the tokens kept at original precision, age order
+  std::vector<int64_t> P;  // ids of the tokens the filter removed that still wait for a full key group
   std::vector<int64_t> Q;  // ids of the quantised tokens, store order
   std::vector<Head> heads;  // [B*Hkv]
 };
@@ -133,34 +141,11 @@ void overflow_event(Cache& c) {
     for (int i = 2 * W; i < 3 * W; ++i) keep_pos.push_back(i);
   }
   for (auto& h : c.heads) {
-    // gather the W leaving rows, in eviction order
-    std::vector<uint16_t> ek(static_cast<size_t>(W) * D), ev(static_cast<size_t>(W) * D);
+    // the W leaving rows join the waiting rows, in removal order
     for (int e = 0; e < W; ++e) {
-      std::memcpy(&ek[static_cast<size_t>(e) * D], &h.fp_k[evict_pos[e] * D], D * 2);
-      std::memcpy(&ev[static_cast<size_t>(e) * D], &h.fp_v[evict_pos[e] * D], D * 2);
+      h.pend_k.insert(h.pend_k.end(), &h.fp_k[evict_pos[e] * D], &h.fp_k[evict_pos[e] * D] + D);
+      h.pend_v.insert(h.pend_v.end(), &h.fp_v[evict_pos[e] * D], &h.fp_v[evict_pos[e] * D] + D);
     }
-    const size_t nq0 = h.k_codes.size() / D;
-    h.k_codes.resize((nq0 + W) * D);
-    h.v_codes.resize((nq0 + W) * D);
-    h.k_scale.resize((nq0 + W) / G * D);
-    h.k_zero.resize((nq0 + W) / G * D);
-    h.v_scale.resize((nq0 + W) * (D / G));
-    h.v_zero.resize((nq0 + W) * (D / G));
-    // keys: group = G consecutive evicted tokens of one channel
-    for (int blk = 0; blk < W / G; ++blk)
-      for (int d = 0; d < D; ++d) {
-        size_t grp = (nq0 / G + blk) * D + d;
-        quantize_group(&ek[static_cast<size_t>(blk) * G * D + d], G, D, &h.k_scale[grp],
-                       &h.k_zero[grp], &h.k_codes[(nq0 + static_cast<size_t>(blk) * G) * D + d], D,
-                       (1 << c.bits) - 1);
-      }
-    // values: group = G consecutive channels of one token
-    for (int e = 0; e < W; ++e)
-      for (int g = 0; g < D / G; ++g) {
-        size_t grp = (nq0 + e) * (D / G) + g;
-        quantize_group(&ev[static_cast<size_t>(e) * D + g * G], G, 1, &h.v_scale[grp],
-                       &h.v_zero[grp], &h.v_codes[(nq0 + e) * D + g * G], 1, (1 << c.bits) - 1);
-      }
     // shrink the full-precision rows to the kept positions
     std::vector<uint16_t> nk(keep_pos.size() * D), nv(keep_pos.size() * D);
     for (size_t i = 0; i < keep_pos.size(); ++i) {
@@ -171,10 +156,39 @@ void overflow_event(Cache& c) {
     h.fp_v.swap(nv);
   }
   std::vector<int64_t> nA;
-  for (auto p : evict_pos) c.Q.push_back(c.A[p]);
+  for (auto p : evict_pos) c.P.push_back(c.A[p]);
   for (auto p : keep_pos) nA.push_back(c.A[p]);
   c.A.swap(nA);
   c.n_events++;
+  // every G waiting tokens form one key group (W a multiple of G: exactly W / G groups, nothing waits)
+  while (static_cast<int>(c.P.size()) >= G) {
+    for (auto& h : c.heads) {
+      const size_t nq0 = h.k_codes.size() / D;
+      h.k_codes.resize((nq0 + G) * D);
+      h.v_codes.resize((nq0 + G) * D);
+      h.k_scale.resize((nq0 + G) / G * D);
+      h.k_zero.resize((nq0 + G) / G * D);
+      h.v_scale.resize((nq0 + G) * (D / G));
+      h.v_zero.resize((nq0 + G) * (D / G));
+      // keys: group = the G oldest waiting tokens of one channel
+      for (int d = 0; d < D; ++d) {
+        size_t grp = (nq0 / G) * D + d;
+        quantize_group(&h.pend_k[d], G, D, &h.k_scale[grp], &h.k_zero[grp], &h.k_codes[nq0 * D + d], D,
+                       (1 << c.bits) - 1);
+      }
+      // values: group = G consecutive channels of one token
+      for (int e = 0; e < G; ++e)
+        for (int g = 0; g < D / G; ++g) {
+          size_t grp = (nq0 + e) * (D / G) + g;
+          quantize_group(&h.pend_v[static_cast<size_t>(e) * D + g * G], G, 1, &h.v_scale[grp], &h.v_zero[grp],
+                         &h.v_codes[(nq0 + e) * D + g * G], 1, (1 << c.bits) - 1);
+        }
+      h.pend_k.erase(h.pend_k.begin(), h.pend_k.begin() + static_cast<size_t>(G) * D);
+      h.pend_v.erase(h.pend_v.begin(), h.pend_v.begin() + static_cast<size_t>(G) * D);
+    }
+    c.Q.insert(c.Q.end(), c.P.begin(), c.P.begin() + G);
+    c.P.erase(c.P.begin(), c.P.begin() + G);
+  }
 }
 
 // Dense softmax attention of one query over n tokens, float64 (Eq. 2 with sm_scale).
@@ -200,16 +214,20 @@ void attention_dense(const double* q, const double* K, const double* V, int64_t 
   }
 }
 
-// All tokens of one head as float64 rows: first the full-precision list (order of A),
-// then the quantised store (order of Q), dequantised.
+// All tokens of one head as float64 rows: first the full-precision list (order of A), the
+// waiting rows (order of P), then the quantised store (order of Q), dequantised.
 void dense_rows(const Cache& c, const Head& h, std::vector<double>& K, std::vector<double>& V) {
   const int D = c.D, G = c.G;
-  const size_t nf = c.A.size(), nq = c.Q.size();
+  const size_t na = c.A.size(), nf = c.A.size() + c.P.size(), nq = c.Q.size();
   K.resize((nf + nq) * D);
   V.resize((nf + nq) * D);
-  for (size_t i = 0; i < nf * D; ++i) {
+  for (size_t i = 0; i < na * D; ++i) {
     K[i] = bf16_to_f32(h.fp_k[i]);
     V[i] = bf16_to_f32(h.fp_v[i]);
+  }
+  for (size_t i = 0; i < c.P.size() * D; ++i) {
+    K[na * D + i] = bf16_to_f32(h.pend_k[i]);
+    V[na * D + i] = bf16_to_f32(h.pend_v[i]);
   }
   for (size_t t = 0; t < nq; ++t)
     for (int d = 0; d < D; ++d) {
@@ -336,7 +354,7 @@ void lqo_attention_merge(const double* m, const double* l, const double* o, int 
 
 // ---- the cache object ------------------------------------------------------------------
 void* lqo_create(int B, int Hq, int Hkv, int D, int W, int G) {
-  if (B < 1 || Hkv < 1 || Hq % Hkv || D < 1 || W < 1 || G < 1 || W % G || D % G || D % 4) return nullptr;
+  if (B < 1 || Hkv < 1 || Hq % Hkv || D < 1 || W < 1 || G < 1 || D % G || D % 4) return nullptr;
   Cache* c = new Cache;
   c->B = B; c->Hq = Hq; c->Hkv = Hkv; c->D = D; c->W = W; c->G = G;
   c->heads.resize(static_cast<size_t>(B) * Hkv);
@@ -377,7 +395,10 @@ void lqo_append(void* p, const uint16_t* k, const uint16_t* v, int n) {
 }
 
 int64_t lqo_n_seen(void* p) { return static_cast<Cache*>(p)->n_seen; }
-int64_t lqo_n_fp(void* p) { return static_cast<int64_t>(static_cast<Cache*>(p)->A.size()); }
+// tokens at original precision: the filter's list plus those waiting for a full key group
+int64_t lqo_n_fp(void* p) {
+  return static_cast<int64_t>(static_cast<Cache*>(p)->A.size() + static_cast<Cache*>(p)->P.size());
+}
 int64_t lqo_n_quant(void* p) { return static_cast<int64_t>(static_cast<Cache*>(p)->Q.size()); }
 int64_t lqo_n_events(void* p) { return static_cast<Cache*>(p)->n_events; }
 
@@ -388,8 +409,15 @@ void lqo_export(void* p, int32_t* kept_ids, int32_t* quant_ids, uint8_t* k_codes
                 uint16_t* k_scale, uint16_t* k_zero, uint16_t* v_scale, uint16_t* v_zero,
                 uint16_t* fp_k, uint16_t* fp_v) {
   Cache& c = *static_cast<Cache*>(p);
-  const size_t nf = c.A.size(), nq = c.Q.size(), D = c.D, G = c.G;
-  if (kept_ids) for (size_t i = 0; i < nf; ++i) kept_ids[i] = static_cast<int32_t>(c.A[i]);
+  const size_t nq = c.Q.size(), D = c.D, G = c.G;
+  // tokens at original precision in ascending id order: (id, list, position in that list)
+  struct Row { int64_t id; int from_p; size_t pos; };
+  std::vector<Row> rows;
+  for (size_t i = 0; i < c.A.size(); ++i) rows.push_back({c.A[i], 0, i});
+  for (size_t i = 0; i < c.P.size(); ++i) rows.push_back({c.P[i], 1, i});
+  std::sort(rows.begin(), rows.end(), [](const Row& x, const Row& y) { return x.id < y.id; });
+  const size_t nf = rows.size();
+  if (kept_ids) for (size_t i = 0; i < nf; ++i) kept_ids[i] = static_cast<int32_t>(rows[i].id);
   if (quant_ids) for (size_t i = 0; i < nq; ++i) quant_ids[i] = static_cast<int32_t>(c.Q[i]);
   for (size_t hh = 0; hh < c.heads.size(); ++hh) {
     const Head& h = c.heads[hh];
@@ -404,8 +432,12 @@ void lqo_export(void* p, int32_t* kept_ids, int32_t* quant_ids, uint8_t* k_codes
     if (k_zero) std::copy(h.k_zero.begin(), h.k_zero.end(), k_zero + hh * (nq / G) * D);
     if (v_scale) std::copy(h.v_scale.begin(), h.v_scale.end(), v_scale + hh * nq * (D / G));
     if (v_zero) std::copy(h.v_zero.begin(), h.v_zero.end(), v_zero + hh * nq * (D / G));
-    if (fp_k) std::copy(h.fp_k.begin(), h.fp_k.end(), fp_k + hh * nf * D);
-    if (fp_v) std::copy(h.fp_v.begin(), h.fp_v.end(), fp_v + hh * nf * D);
+    for (size_t i = 0; i < nf; ++i) {
+      const uint16_t* sk = (rows[i].from_p ? h.pend_k.data() : h.fp_k.data()) + rows[i].pos * D;
+      const uint16_t* sv = (rows[i].from_p ? h.pend_v.data() : h.fp_v.data()) + rows[i].pos * D;
+      if (fp_k) std::copy(sk, sk + D, fp_k + (hh * nf + i) * D);
+      if (fp_v) std::copy(sv, sv + D, fp_v + (hh * nf + i) * D);
+    }
   }
 }
 

@@ -275,3 +275,55 @@ def test_cache_4bit_grouping_and_image_sizes():
     orig = bf16_bits_to_f64(k[0, 0, ev])
     nf = oc.n_fp
     assert np.abs(K[nf:] - orig).max() < np.abs(K2[nf:] - orig).max() / 3
+
+
+# ---- W not a multiple of G: key groups span overflow steps -------------------------------------
+@pytest.mark.parametrize("W,G", [(42, 64), (85, 64), (48, 32), (21, 32)])
+def test_key_groups_across_overflow_steps(W, G):
+    """The paper's own settings (G = 64, W = 42 or 85) give no whole key groups per overflow step.  Reading:
+    removed tokens wait at original precision, in removal order, until G of them form a key group.  Pins: the
+    id sets follow from the (separately pinned) filter in closed form, a group that spans two steps has the
+    codes of the stand-alone quantiser on the original rows, and attention is the dense definition."""
+    B, Hq, Hkv, D = 1, 2, 1, 128
+    rng = np.random.default_rng(W * 100 + G)
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G)
+    n_total = 0
+    ks, vs = [], []
+    for step in (3 * W, 1, W, 2 * W + 7, 5, 3 * W):
+        k = f32_to_bf16_bits(rng.standard_normal((B, Hkv, step, D)).astype(np.float32))
+        v = f32_to_bf16_bits(rng.standard_normal((B, Hkv, step, D)).astype(np.float32))
+        oc.append(k, v)
+        ks.append(k); vs.append(v)
+        n_total += step
+        kept, removed, n_ev = oracle.filter_ids(W, n_total)
+        nq = len(removed) // G * G
+        img = oc.export()
+        assert oc.n_events == n_ev and oc.n_quant == nq and oc.n_fp == n_total - nq
+        assert img["quant_ids"].tolist() == removed[:nq].tolist()
+        assert img["kept_ids"].tolist() == sorted(kept.tolist() + removed[nq:].tolist())
+    K_all = np.concatenate(ks, axis=2)[0, 0]
+    V_all = np.concatenate(vs, axis=2)[0, 0]
+    # full-precision rows are the original rows of their ids
+    assert np.array_equal(img["fp_k"][0, 0], K_all[img["kept_ids"]])
+    assert np.array_equal(img["fp_v"][0, 0], V_all[img["kept_ids"]])
+    # every key group (several span two overflow steps) against the stand-alone quantiser
+    kc = oracle.unpack2(img["k_codes"].reshape(-1)).reshape(nq, D)
+    vc = oracle.unpack2(img["v_codes"].reshape(-1)).reshape(nq, D)
+    qids = img["quant_ids"]
+    for grp in range(nq // G):
+        ids = qids[grp * G:(grp + 1) * G]
+        for d in (0, 63, 127):
+            s, z, c = oracle.quantize_group(K_all[ids, d])
+            assert (s, z) == (img["k_scale"][0, 0, grp, d], img["k_zero"][0, 0, grp, d])
+            assert np.array_equal(c, kc[grp * G:(grp + 1) * G, d])
+    for e in (0, nq // 2, nq - 1):
+        for g in range(D // G):
+            s, z, c = oracle.quantize_group(V_all[qids[e], g * G:(g + 1) * G])
+            assert (s, z) == (img["v_scale"][0, 0, e, g], img["v_zero"][0, 0, e, g])
+            assert np.array_equal(c, vc[e, g * G:(g + 1) * G])
+    q = f32_to_bf16_bits(rng.standard_normal((B, Hq, D)).astype(np.float32))
+    out = oc.attention(q, 1 / np.sqrt(D))
+    K, V = oc.dense_rows(0, 0)
+    assert K.shape[0] == n_total
+    ref = oracle.attention_dense(bf16_bits_to_f64(q[0, 0]), K, V, 1 / np.sqrt(D))
+    assert np.allclose(out[0, 0], ref, rtol=0, atol=1e-12)
