@@ -72,7 +72,8 @@ typedef struct {
   int32_t n_q_heads;     /* Hq; Hq % Hkv == 0 and Hq / Hkv <= 8                                  */
   int32_t n_kv_heads;    /* Hkv                                                                  */
   int32_t head_dim;      /* D; only 128 is implemented                                           */
-  int32_t window;        /* W of Algorithm 1; W % G == 0, W <= 512                               */
+  int32_t window;        /* W of Algorithm 1, <= 512.  W % G != 0 (the paper's W = 42 or 85 with G = 64): removed
+                            tokens wait at full precision, in removal order, until G of them form a key group */
   int32_t group;         /* G: quantisation group size, 32 or 64                                 */
   int32_t bits;          /* 2, or 4 (the paper's second precision; needs group == 32)             */
   int64_t max_tokens;    /* capacity per sequence (tokens ever appended)                         */
@@ -85,8 +86,9 @@ typedef struct {
 
 typedef struct {
   int64_t n_seen;   /* tokens appended so far                                                    */
-  int64_t n_fp;     /* tokens in the full-precision store (2W < n_fp <= 3W after the first event) */
-  int64_t n_quant;  /* tokens in the 2-bit store (a multiple of W)                               */
+  int64_t n_fp;     /* tokens in the full-precision store (2W < n_fp <= 3W after the first event; up to
+                       3W + G - 1 when W % G != 0: those waiting for a full key group count)       */
+  int64_t n_quant;  /* tokens in the quantised store (a multiple of G)                           */
   int64_t n_events; /* window overflows processed                                                */
   int64_t bytes_device;        /* device bytes owned by the whole cache (all layers + workspace) */
   int64_t bytes_decode_step;   /* algorithmic bytes one lq_decode_attn on this layer has to read:

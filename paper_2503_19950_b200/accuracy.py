@@ -47,7 +47,10 @@ def planted_case(seed, B, Hq, Hkv, n, kappa, a, device):
 
 def run(ctx=8192, lengths=16, B=2, kappa=16.0, a=4.0, seed=4, device="cuda"):
     shapes = [dict(name="Hq32/Hkv8 W128 G32", Hq=32, Hkv=8, W=128, G=32, bits=(2, 4)),
-              dict(name="Hq28/Hkv4 W256 G64", Hq=28, Hkv=4, W=256, G=64, bits=(2,))]
+              dict(name="Hq28/Hkv4 W256 G64", Hq=28, Hkv=4, W=256, G=64, bits=(2,)),
+              # the paper's own settings (Sec. 3.1): group 64, reserved length 128 and 256 tokens, i.e. W = 42, 85
+              dict(name="Hq32/Hkv8 W42 G64", Hq=32, Hkv=8, W=42, G=64, bits=(2,)),
+              dict(name="Hq32/Hkv8 W85 G64", Hq=32, Hkv=8, W=85, G=64, bits=(2,))]
     rows = []
     for sh in shapes:
         for bits in sh["bits"]:

@@ -24,8 +24,11 @@ namespace {
 struct LayerState {
   int64_t n_seen = 0, n_events = 0, n_quant = 0;
   int n_fp = 0;
-  std::vector<int32_t> age_slot;    // age order (oldest first) -> physical fp slot; size n_fp
-  std::vector<int32_t> slot_token;  // physical fp slot -> token id; size 3W
+  // n_fp = rows of the fp store in use (always the dense prefix [0, n_fp)) = age_slot.size() + pend_slot.size()
+  std::vector<int32_t> age_slot;    // the filter's list A, age order (oldest first) -> physical fp slot
+  std::vector<int32_t> pend_slot;   // removed by the filter, waiting for a full key group (only when W % G != 0),
+                                    // removal order -> physical fp slot
+  std::vector<int32_t> slot_token;  // physical fp slot -> token id; size 3W + G
   std::vector<int32_t> quant_ids;   // token ids in 2-bit store order
 };
 
@@ -104,7 +107,10 @@ void next_evicted(const lq_cache* c, const LayerState& L, EvictList* ev, int32_t
   const int W = c->cfg.window;
   for (int e = 0; e < W; ++e) {
     const int slot = L.age_slot[evict_pos(c, e)];
-    if (ev) ev->slot[e] = static_cast<uint16_t>(slot);
+    if (ev) {
+      ev->slot[e] = static_cast<uint16_t>(slot);
+      ev->src[e] = static_cast<uint16_t>(2 * W + e);  // the row of age position 2W + e moves into the hole
+    }
     if (ids) ids[e] = L.slot_token[slot];
   }
 }
@@ -131,7 +137,92 @@ void apply_event(const lq_cache* c, LayerState& L) {
   L.n_events++;
 }
 
+int kept(const LayerState& L) { return static_cast<int>(L.age_slot.size()); }
+bool residual_mode(const lq_cache* c) { return c->cfg.window % c->cfg.group != 0; }
+
+// W not a multiple of G, step 1 of an overflow: the W removed tokens join the waiting list; no row moves.
+void apply_event_residual(const lq_cache* c, LayerState& L) {
+  const int W = c->cfg.window;
+  std::vector<char> gone(3 * W, 0);
+  for (int e = 0; e < W; ++e) {
+    gone[evict_pos(c, e)] = 1;
+    L.pend_slot.push_back(L.age_slot[evict_pos(c, e)]);
+  }
+  std::vector<int32_t> na;
+  na.reserve(3 * W);
+  for (int i = 0; i < 3 * W; ++i)
+    if (!gone[i]) na.push_back(L.age_slot[i]);
+  L.age_slot.swap(na);
+  L.n_events++;
+}
+
+// W not a multiple of G, step 2: the G oldest waiting tokens form a key group.  Fills the launch
+// description (rows to quantise, and which top rows of the dense prefix move into the holes below
+// the new end of the prefix) and updates the host maps.  ids: the G token ids, in store order.
+void plan_group_residual(const lq_cache* c, LayerState& L, EvictList* ev, int32_t* ids) {
+  const int G = c->cfg.group;
+  const int live = L.n_fp, new_live = live - G;
+  std::vector<char> is_hole(live, 0);
+  for (int e = 0; e < G; ++e) is_hole[L.pend_slot[e]] = 1;
+  std::vector<int> sources;  // rows above the new end that survive
+  for (int s = new_live; s < live; ++s)
+    if (!is_hole[s]) sources.push_back(s);
+  size_t next = 0;
+  std::vector<std::pair<int, int>> moves;  // (src, dst)
+  for (int e = 0; e < G; ++e) {
+    const int hole = L.pend_slot[e];
+    if (ids) ids[e] = L.slot_token[hole];
+    L.quant_ids.push_back(L.slot_token[hole]);
+    ev->slot[e] = static_cast<uint16_t>(hole);
+    if (hole < new_live) {
+      ev->src[e] = static_cast<uint16_t>(sources[next]);
+      moves.emplace_back(sources[next], hole);
+      ++next;
+    } else {
+      ev->src[e] = kNoMove;
+    }
+  }
+  L.pend_slot.erase(L.pend_slot.begin(), L.pend_slot.begin() + G);
+  for (auto& mv : moves) {
+    L.slot_token[mv.second] = L.slot_token[mv.first];
+    for (auto& s : L.age_slot)
+      if (s == mv.first) s = mv.second;
+    for (auto& s : L.pend_slot)
+      if (s == mv.first) s = mv.second;
+  }
+  L.n_fp = new_live;
+  L.n_quant += G;
+}
+
+// one overflow of one layer when W is not a multiple of G (host state and launches)
+lq_status_t run_event_residual(lq_cache* c, int layer, cudaStream_t st) {
+  LayerState& L = c->layers[layer];
+  apply_event_residual(c, L);
+  while (static_cast<int>(L.pend_slot.size()) >= c->cfg.group) {
+    EvictList ev;
+    std::memset(&ev, 0, sizeof ev);
+    const int64_t tile0 = L.n_quant / c->cfg.group;
+    plan_group_residual(c, L, &ev, nullptr);
+    if (!c->dry) {
+      LayerList ll;
+      ll.n = 1;
+      ll.layer[0] = static_cast<uint8_t>(layer);
+      cudaError_t e = launch_compress(c->cv, ll, ev, tile0, 1, st);
+      if (e != cudaSuccess) return cuda_fail(c, e, "lq_compress_kernel");
+      c->n_launches++;
+    }
+  }
+  return LQ_OK;
+}
+
 lq_status_t run_events(lq_cache* c, const std::vector<int>& full_layers, cudaStream_t st) {
+  if (residual_mode(c)) {
+    for (int layer : full_layers) {
+      lq_status_t s = run_event_residual(c, layer, st);
+      if (s != LQ_OK) return s;
+    }
+    return LQ_OK;
+  }
   // group layers whose removal lists coincide into one launch
   std::vector<char> done(full_layers.size(), 0);
   for (size_t i = 0; i < full_layers.size(); ++i) {
@@ -155,7 +246,7 @@ lq_status_t run_events(lq_cache* c, const std::vector<int>& full_layers, cudaStr
       members.push_back(static_cast<int>(k));
     }
     if (!c->dry) {
-      cudaError_t e = launch_compress(c->cv, ll, ev, Li.n_quant / c->cfg.group, st);
+      cudaError_t e = launch_compress(c->cv, ll, ev, Li.n_quant / c->cfg.group, c->cfg.window / c->cfg.group, st);
       if (e != cudaSuccess) return cuda_fail(c, e, "lq_compress_kernel");
       c->n_launches++;
     }
@@ -208,7 +299,7 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
   if (cfg->head_dim != kD || (cfg->bits != 2 && cfg->bits != 4)) return LQ_ERR_UNSUPPORTED;
   if (cfg->group != 32 && cfg->group != 64) return LQ_ERR_UNSUPPORTED;
   if (cfg->bits == 4 && cfg->group != 32) return LQ_ERR_UNSUPPORTED;  // a 4-bit tile of G = 64 exceeds a stage
-  if (cfg->window % cfg->group || cfg->window > kMaxW) return LQ_ERR_UNSUPPORTED;
+  if (cfg->window > kMaxW) return LQ_ERR_UNSUPPORTED;
   if (cfg->n_q_heads / cfg->n_kv_heads > kMaxRatio || cfg->n_layers > 128) return LQ_ERR_UNSUPPORTED;
   if (cfg->kernel < LQ_KERNEL_AUTO || cfg->kernel > LQ_KERNEL_MMA) return LQ_ERR_INVALID_ARG;
   if (cfg->filter != LQ_FILTER_LOG && cfg->filter != LQ_FILTER_RECENT) return LQ_ERR_INVALID_ARG;
@@ -226,10 +317,12 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
   cv.quant_tiles_cap = (cfg->max_tokens + G - 1) / G;
   cv.quant_head_stride = cv.quant_tiles_cap * quant_tile_bytes(G, cv.planes);
   cv.quant_layer_stride = cv.quant_head_stride * pairs;
-  cv.fp_head_stride = static_cast<int64_t>(3 * W / kFpTileSlots) * kFpTileBytes;
+  // W % G != 0: up to G - 1 removed tokens wait in the fp store for a full key group
+  const int fp_slots = 3 * W + (W % G ? G : 0);
+  cv.fp_head_stride = static_cast<int64_t>((fp_slots + kFpTileSlots - 1) / kFpTileSlots) * kFpTileBytes;
   cv.fp_layer_stride = cv.fp_head_stride * pairs;
   c->layers.resize(cfg->n_layers);
-  for (auto& L : c->layers) L.slot_token.assign(3 * W, -1);
+  for (auto& L : c->layers) L.slot_token.assign(3 * W + G, -1);
 
   if (!c->dry) {
     cudaError_t e = cudaSetDevice(cfg->device);
@@ -247,7 +340,7 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
               dev_alloc(c, reinterpret_cast<void**>(&c->part_ml), pairs * c->max_splits * r * 2 * 4) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->status), 256) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->tickets), pairs * 128) &&
-              dev_alloc(c, reinterpret_cast<void**>(&c->ingest_idx), (cfg->max_tokens + 3 * cfg->window) * 4) &&
+              dev_alloc(c, reinterpret_cast<void**>(&c->ingest_idx), (cfg->max_tokens + 3 * cfg->window + cfg->group) * 4) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_k), cfg->n_layers * pairs * kD * 2) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_v), cfg->n_layers * pairs * kD * 2) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_q),
@@ -288,15 +381,24 @@ lq_status_t ingest_prompt(lq_cache* c, int layer, const void* k, const void* v, 
   const int W = c->cfg.window, G = c->cfg.group;
   std::vector<int32_t> idx;
   idx.reserve(static_cast<size_t>(n) + 3 * W);
-  std::vector<int32_t> ids(W);
+  std::vector<int32_t> ids(std::max(W, G));
   int done = 0;
   while (done < n) {
-    if (L.n_fp == 3 * W) {
-      next_evicted(c, L, nullptr, ids.data());
-      idx.insert(idx.end(), ids.begin(), ids.end());
-      apply_event(c, L);
+    if (kept(L) == 3 * W) {
+      if (residual_mode(c)) {
+        apply_event_residual(c, L);
+        while (static_cast<int>(L.pend_slot.size()) >= G) {
+          EvictList unused;
+          plan_group_residual(c, L, &unused, ids.data());
+          idx.insert(idx.end(), ids.begin(), ids.begin() + G);
+        }
+      } else {
+        next_evicted(c, L, nullptr, ids.data());
+        idx.insert(idx.end(), ids.begin(), ids.end());
+        apply_event(c, L);
+      }
     }
-    const int take = std::min(n - done, 3 * W - L.n_fp);
+    const int take = std::min(n - done, 3 * W - kept(L));
     for (int t = 0; t < take; ++t) {
       L.age_slot.push_back(L.n_fp + t);
       L.slot_token[L.n_fp + t] = static_cast<int32_t>(L.n_seen + t);
@@ -337,17 +439,17 @@ lq_status_t append_impl(lq_cache_t* c, int32_t layer, const void* k, const void*
   LayerState& L = c->layers[layer];
   const int W = c->cfg.window;
   if (L.n_seen + n > c->cfg.max_tokens) return LQ_ERR_CAPACITY;
-  if (!c->cfg.auto_compress && L.n_fp + n > 3 * W) return LQ_ERR_WINDOW_FULL;
+  if (!c->cfg.auto_compress && kept(L) + n > 3 * W) return LQ_ERR_WINDOW_FULL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (!c->dry && c->cfg.auto_compress && L.n_seen == 0 && n > 3 * W && extra_bytes == 0)
     return ingest_prompt(c, layer, k, v, n, st);
   int done = 0;
   while (done < n) {
-    if (L.n_fp == 3 * W) {
+    if (kept(L) == 3 * W) {
       lq_status_t s = run_events(c, std::vector<int>{layer}, st);
       if (s != LQ_OK) return s;
     }
-    const int take = std::min(n - done, 3 * W - L.n_fp);
+    const int take = std::min(n - done, 3 * W - kept(L));
     if (!c->dry) {
       const bool last = done + take == n;
       cudaError_t e = launch_append(c->cv, layer, k, v, n, done, take, L.n_fp, st, last ? extra_src : nullptr,
@@ -372,11 +474,11 @@ lq_status_t lq_compress(lq_cache_t* c, int32_t layer, void* stream) {
   const int W = c->cfg.window;
   std::vector<int> full;
   if (layer >= 0) {
-    if (c->layers[layer].n_fp != 3 * W) return LQ_ERR_NOT_FULL;
+    if (kept(c->layers[layer]) != 3 * W) return LQ_ERR_NOT_FULL;
     full.push_back(layer);
   } else {
     for (int i = 0; i < c->cfg.n_layers; ++i)
-      if (c->layers[i].n_fp == 3 * W) full.push_back(i);
+      if (kept(c->layers[i]) == 3 * W) full.push_back(i);
   }
   if (full.empty()) return LQ_OK;
   return run_events(c, full, static_cast<cudaStream_t>(stream));
@@ -407,7 +509,7 @@ lq_status_t lq_append_decode_attn(lq_cache_t* c, int32_t layer, const void* k, c
   const int64_t step_bytes = static_cast<int64_t>(c->cfg.batch) * c->cfg.n_kv_heads *
                              (L.n_quant * (quant_tile_bytes(c->cfg.group, c->cfg.bits / 2) / c->cfg.group) +
                               static_cast<int64_t>(L.n_fp) * 4 * kD);
-  if (L.n_fp == 3 * W || !use_mma(c) || step_bytes > (192LL << 20)) {
+  if (kept(L) == 3 * W || !use_mma(c) || step_bytes > (192LL << 20)) {
     // the window is full (the overflow step has to run between the two), the plain kernel is
     // selected, or the launch is long: the two separate calls
     lq_status_t s = lq_append(c, layer, k, v, 1, stream);
@@ -524,7 +626,7 @@ lq_status_t lq_decode_step_host(lq_cache_t* c, int32_t layer, const void* k_host
     if ((e = cudaMemcpyAsync(sq, q_host, qb, cudaMemcpyHostToDevice, st)) != cudaSuccess)
       return cuda_fail(c, e, "host-to-device copy");
   }
-  if (L.n_fp == 3 * c->cfg.window) {
+  if (kept(L) == 3 * c->cfg.window) {
     lq_status_t s = run_events(c, std::vector<int>{layer}, st);
     if (s != LQ_OK) return s;
   }
@@ -612,7 +714,7 @@ lq_status_t lq_cache_info(const lq_cache_t* c, int32_t layer, lq_info_t* info) {
 lq_status_t lq_next_evicted_ids(const lq_cache_t* c, int32_t layer, int32_t* ids) {
   if (!c || !ids || layer < 0 || layer >= c->cfg.n_layers) return LQ_ERR_INVALID_ARG;
   const LayerState& L = c->layers[layer];
-  if (L.n_fp != 3 * c->cfg.window) return LQ_ERR_NOT_FULL;
+  if (kept(L) != 3 * c->cfg.window) return LQ_ERR_NOT_FULL;
   next_evicted(c, L, nullptr, ids);
   return LQ_OK;
 }
@@ -622,10 +724,12 @@ lq_status_t lq_export(const lq_cache_t* cc, int32_t layer, lq_image_t* img) {
   if (!c || !img || layer < 0 || layer >= c->cfg.n_layers) return LQ_ERR_INVALID_ARG;
   const LayerState& L = c->layers[layer];
   // kept ids ascending, with the slot each lives in
-  std::vector<std::pair<int32_t, int32_t>> kept;  // (token id, slot)
-  for (int i = 0; i < L.n_fp; ++i) kept.emplace_back(L.slot_token[L.age_slot[i]], L.age_slot[i]);
-  std::sort(kept.begin(), kept.end());
-  if (img->kept_ids) for (int i = 0; i < L.n_fp; ++i) img->kept_ids[i] = kept[i].first;
+  // (tokens still waiting for a full key group are at full precision too)
+  std::vector<std::pair<int32_t, int32_t>> rows;  // (token id, slot)
+  for (int slot : L.age_slot) rows.emplace_back(L.slot_token[slot], slot);
+  for (int slot : L.pend_slot) rows.emplace_back(L.slot_token[slot], slot);
+  std::sort(rows.begin(), rows.end());
+  if (img->kept_ids) for (int i = 0; i < L.n_fp; ++i) img->kept_ids[i] = rows[i].first;
   if (img->quant_ids) std::copy(L.quant_ids.begin(), L.quant_ids.end(), img->quant_ids);
   const bool want_dev = img->k_codes || img->v_codes || img->k_scale || img->k_zero || img->v_scale ||
                         img->v_zero || img->fp_k || img->fp_v;
@@ -652,7 +756,7 @@ lq_status_t lq_export(const lq_cache_t* cc, int32_t layer, lq_image_t* img) {
     if (b.host && b.bytes > 0 && cudaMalloc(&b.dev, static_cast<size_t>(b.bytes)) != cudaSuccess) status = LQ_ERR_OOM;
   if (status == LQ_OK && nf > 0) {
     std::vector<int> slots(nf);
-    for (int i = 0; i < nf; ++i) slots[i] = kept[i].second;
+    for (int i = 0; i < nf; ++i) slots[i] = rows[i].second;
     if (cudaMalloc(&slots_dev, nf * sizeof(int)) != cudaSuccess) status = LQ_ERR_OOM;
     else cudaMemcpy(slots_dev, slots.data(), nf * sizeof(int), cudaMemcpyHostToDevice);
   }

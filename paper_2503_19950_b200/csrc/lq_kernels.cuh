@@ -21,8 +21,10 @@ struct CacheView {
 };
 
 struct EvictList {
-  uint16_t slot[kMaxW];  // physical fp slots of the W removed tokens, in removal order
+  uint16_t slot[kMaxW];  // physical fp slots of the tokens to quantise, in removal order
+  uint16_t src[kMaxW];   // slot whose row moves into slot[e] afterwards (kNoMove: nothing moves there)
 };
+constexpr uint16_t kNoMove = 0xFFFF;
 
 struct LayerList {
   int n;
@@ -39,7 +41,7 @@ cudaError_t launch_append(const CacheView& cv, int layer, const void* k, const v
 // K2: overflow step for the listed layers (all of them in the same state): quantise + pack the W
 // rows of `ev` into quant tiles [tile0, tile0 + W/G), then move rows 2W+e into slot ev.slot[e].
 cudaError_t launch_compress(const CacheView& cv, const LayerList& layers, const EvictList& ev,
-                            int64_t tile0, cudaStream_t st);
+                            int64_t tile0, int n_groups, cudaStream_t st);
 
 // Prompt ingestion into an empty layer in one launch: idx_dev = [n_tiles*G removed prompt positions in store
 // order][n_fp: final fp slot -> prompt position]; k, v = [B, Hkv, n_src, 128] bf16.

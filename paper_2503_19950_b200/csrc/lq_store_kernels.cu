@@ -61,9 +61,9 @@ cudaError_t launch_append(const CacheView& cv, int layer, const void* k, const v
 //
 // One CTA per (key group tau of the event, (b, kv) head, layer).  It
 //   1. gathers the G removed rows of its group (K and V) into shared memory,
-//   2. back-fills the G holes with the rows of slots 2W + tau*G + e (the newest window), so the
-//      valid slots stay the dense prefix [0, 2W) -- legal because the order of the cache is free
-//      (Eq. 3) -- and only this CTA ever touches these 2G slots,
+//   2. back-fills the G holes with rows the host names (the top rows of the dense prefix: slots
+//      2W + tau*G + e when W is a multiple of G), so the valid slots stay a dense prefix -- legal
+//      because the order of the cache is free (Eq. 3) -- and only this CTA ever touches these 2G slots,
 //   3. quantises: keys per channel down the G tokens (one thread per channel), values per token
 //      across G channels (one warp per token, group min/max by __shfl_xor_sync),
 //   4. packs the codes into the fragment order of the tile and stores the tile.
@@ -205,11 +205,12 @@ lq_compress_kernel(CacheView cv, LayerList layers, EvictList ev, int64_t tile0) 
   }
   __syncthreads();
 
-  // 2. back-fill the holes from the newest window
+  // 2. back-fill the holes (from the newest window; the host names the source rows)
   for (int idx = tid; idx < G * 32; idx += 256) {
     const int c = idx & 15, which = (idx >> 4) & 1, e = idx >> 5;
     const int dst = ev.slot[tau * G + e];
-    const int src = 2 * cv.W + tau * G + e;
+    const int src = ev.src[tau * G + e];
+    if (src == kNoMove) continue;
     const int vo = which ? kFpTileVOffset : 0;
     const uint4 val = *reinterpret_cast<const uint4*>(fpbase + fp_chunk_off(src, c) + vo);
     *reinterpret_cast<uint4*>(fpbase + fp_chunk_off(dst, c) + vo) = val;
@@ -219,8 +220,8 @@ lq_compress_kernel(CacheView cv, LayerList layers, EvictList ev, int64_t tile0) 
 }
 
 cudaError_t launch_compress(const CacheView& cv, const LayerList& layers, const EvictList& ev,
-                            int64_t tile0, cudaStream_t st) {
-  dim3 grid(cv.W / cv.G, cv.B * cv.Hkv, layers.n);
+                            int64_t tile0, int n_groups, cudaStream_t st) {
+  dim3 grid(n_groups, cv.B * cv.Hkv, layers.n);
   if (cv.G == 32 && cv.planes == 1)
     lq_compress_kernel<32, 1><<<grid, 256, 0, st>>>(cv, layers, ev, tile0);
   else if (cv.G == 32 && cv.planes == 2)

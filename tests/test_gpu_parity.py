@@ -98,12 +98,26 @@ def test_four_bit_needs_group_32():
         LogQuantCache(1, 1, 8, 2, 64, 64, max_tokens=512, bits=4)
 
 
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("B,Hq,Hkv,W,G,bits,n_prefill,n_steps,chunk", [
+    (2, 8, 2, 42, 64, 2, 42 * 9 + 5, 4, None),    # the paper's W = 42 (reserved length 128), G = 64; one-launch prompt
+    (1, 14, 2, 85, 64, 2, 85 * 7 + 30, 3, 97),    # W = 85 (reserved length 256), GQA-7, step-by-step overflow
+    (2, 4, 4, 100, 32, 2, 100 * 5 + 1, 3, 1),     # G = 32, r = 1, one token at a time
+    (1, 8, 2, 50, 32, 4, 50 * 8 + 17, 50, 60),    # 4-bit codes; the decode steps cross an overflow
+])
+def test_window_not_a_multiple_of_the_group(kernel, B, Hq, Hkv, W, G, bits, n_prefill, n_steps, chunk):
+    """W % G != 0: removed tokens wait at full precision until G of them form a key group."""
+    worst = run_case(B, Hq, Hkv, W, G, n_prefill, n_steps, seed=29, kernel=kernel, bits=bits, prefill_chunk=chunk,
+                     check_image_every=7 if n_steps > 10 else 1)
+    assert worst <= 1.0
+
+
 def _random_cases(n, seed):
     rng = np.random.default_rng(seed)
     cases = []
     while len(cases) < n:
         G = int(rng.choice([32, 64]))
-        W = int(rng.choice([w for w in (32, 64, 96, 128, 192, 256) if w % G == 0]))
+        W = int(rng.choice([32, 42, 64, 85, 96, 100, 128, 192, 256]))
         Hkv = int(rng.choice([1, 2, 4]))
         r = int(rng.choice([1, 2, 3, 4, 5, 7, 8]))
         bits = 4 if (G == 32 and rng.random() < 0.3) else 2
@@ -238,6 +252,7 @@ def test_prompt_ingestion_in_one_launch_equals_token_by_token(W, G, n):
     (2, 8, 2, 32, 32, 2, 3 * 32 - 5),     # crosses an overflow step (falls back to the two calls there)
     (1, 14, 2, 64, 64, 2, 64 * 5 + 15),   # GQA-7; the new row opens a new 16-slot tile on the way
     (2, 8, 8, 32, 32, 4, 32 * 7 + 1),     # r = 1, 4-bit codes
+    (2, 8, 2, 42, 64, 2, 42 * 5 + 11),    # W not a multiple of G: waiting tokens in the fp store
 ])
 def test_append_and_attention_in_one_launch(B, Hq, Hkv, W, G, bits, n0):
     """lq_append_decode_attn: same image, same attention bits as lq_append + lq_decode_attn, one launch."""

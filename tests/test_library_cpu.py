@@ -42,7 +42,7 @@ def _dry(W=4, G=4, **kw):
     return LogQuantCache(**args)
 
 
-@pytest.mark.parametrize("bad", [dict(group=16), dict(group=48, window=96), dict(window=100), dict(head_dim=64),
+@pytest.mark.parametrize("bad", [dict(group=16), dict(group=48, window=96), dict(head_dim=64),
                                  dict(bits=3), dict(bits=8), dict(bits=4, group=64, window=128),
                                  dict(n_q_heads=18, n_kv_heads=2), dict(window=1024)])
 def test_unsupported_configurations(bad):
@@ -116,6 +116,28 @@ def test_recent_window_comparator_keeps_exactly_the_newest_tokens(W, G):
         assert oimg["quant_ids"].tolist() == img["quant_ids"].tolist()
     with pytest.raises(LogQuantError):
         _dry(W=W, G=G, filter=7)
+
+
+@pytest.mark.parametrize("W,G", [(42, 64), (85, 64), (100, 32), (21, 32)])
+def test_host_mirror_with_key_groups_across_overflow_steps(W, G):
+    """W not a multiple of G: removed tokens wait at full precision until G of them form a key group.  The
+    host mirror must agree with the oracle (which is pinned against the filter's closed form) on every count
+    and on both id lists, whatever the chunking of the appends."""
+    c = _dry(W=W, G=G, max_tokens=40 * W + 64)
+    oc = oracle.OracleCache(1, 4, 2, 128, W, G)
+    rng = np.random.default_rng(W)
+    n = 0
+    while n < 30 * W:
+        step = int(rng.integers(1, 2 * W))
+        c.append(0, None, None, n_tokens=step)
+        oc.append(np.zeros((1, 2, step, 128), np.uint16), np.zeros((1, 2, step, 128), np.uint16))
+        n += step
+        inf = c.info(0)
+        assert (inf.n_seen, inf.n_fp, inf.n_quant, inf.n_events) == (n, oc.n_fp, oc.n_quant, oc.n_events)
+        assert inf.n_quant % G == 0 and inf.n_fp <= 3 * W + G - 1
+        img, oimg = c.export(0, ids_only=True), oc.export()
+        assert img["kept_ids"].tolist() == oimg["kept_ids"].tolist()
+        assert img["quant_ids"].tolist() == oimg["quant_ids"].tolist()
 
 
 def test_manual_compress_state_rules():
