@@ -4,7 +4,8 @@ import numpy as np
 import torch
 
 import oracle
-from paper_2503_19950_b200 import LogQuantCache, synth
+from paper_2503_19950_b200 import LogQuantCache, LogQuantError, synth
+from paper_2503_19950_b200.binding import LQ_ERR_WINDOW_FULL
 
 IMAGE_KEYS = ["kept_ids", "quant_ids", "k_codes", "v_codes", "k_scale", "k_zero", "v_scale", "v_zero", "fp_k", "fp_v"]
 
@@ -40,10 +41,14 @@ def run_case(B, Hq, Hkv, W, G, n_prefill, n_steps, seed, kernel, n_outliers=3, c
         if auto_compress:
             cache.append(0, k, v)
         else:
-            for t in range(n):  # caller-driven overflow handling
-                if cache.info(0).n_fp == 3 * W:
+            for t in range(n):  # caller-driven overflow handling: append, and on "window full" compress and retry
+                kt, vt = k[:, :, t:t + 1].contiguous(), v[:, :, t:t + 1].contiguous()
+                try:
+                    cache.append(0, kt, vt)
+                except LogQuantError as err:
+                    assert err.status == LQ_ERR_WINDOW_FULL
                     cache.compress(0)
-                cache.append(0, k[:, :, t:t + 1].contiguous(), v[:, :, t:t + 1].contiguous())
+                    cache.append(0, kt, vt)
         oc.append(synth.bf16_bits(k), synth.bf16_bits(v))
 
     done = 0

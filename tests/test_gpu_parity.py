@@ -112,6 +112,45 @@ def test_window_not_a_multiple_of_the_group(kernel, B, Hq, Hkv, W, G, bits, n_pr
     assert worst <= 1.0
 
 
+def test_window_not_a_multiple_of_the_group_manual_overflow_and_layers():
+    """W % G != 0 with caller-driven overflow steps (auto_compress = 0), several layers in one lq_compress(-1)
+    call, and the host-buffer step."""
+    B, Hq, Hkv, W, G, D, L = 2, 8, 2, 42, 64, 128, 3
+    assert run_case(B, Hq, Hkv, W, G, 42 * 6 + 3, 3, seed=31, kernel=LQ_KERNEL_MMA, auto_compress=False) <= 1.0
+    cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=12 * W, auto_compress=False)
+    ocs = [oracle.OracleCache(B, Hq, Hkv, D, W, G) for _ in range(L)]
+    for rnd in range(4):  # layers 0 and 1 enter every round with a full window; layer 2 stays short
+        for l, n in enumerate((3 * W, 3 * W, 30) if rnd == 0 else (0, 0, 0)):
+            if n:
+                k, v = synth.keys_values(50 + rnd, B, Hkv, n, D, "cuda", layer=l)
+                cache.append(l, k, v)
+                ocs[l].append(synth.bf16_bits(k), synth.bf16_bits(v))
+        cache.compress(-1)
+        for l in range(L):  # the oracle runs the overflow step when the next token arrives: feed one
+            k, v = synth.keys_values(60 + rnd, B, Hkv, 1, D, "cpu", layer=l)
+            q = synth.queries(60 + rnd, B, Hq, D, 0, "cpu", layer=l)
+            out = torch.empty(B, Hq, D, dtype=torch.float32)
+            k, v, q, out = k.pin_memory(), v.pin_memory(), q.pin_memory(), out.pin_memory()
+            if l < 2:
+                cache.decode_step_host(l, k, v, q, out)
+            else:
+                cache.append(l, k.cuda(), v.cuda())
+                o = torch.empty(B, Hq, D, device="cuda")
+                cache.decode_attn(l, q.cuda(), o)
+                out = o.cpu()
+            ocs[l].append(synth.bf16_bits(k), synth.bf16_bits(v))
+            assert_images_equal(cache.export(l), ocs[l].export())
+            ref = ocs[l].attention(synth.bf16_bits(q), 1 / np.sqrt(D))
+            assert np.abs(out.numpy() - ref).max() <= attn_tolerance(ref)
+        for l in range(2):  # bring layers 0 and 1 back to W - 1 below full for the next round
+            k, v = synth.keys_values(70 + rnd, B, Hkv, W - 1, D, "cuda", layer=l)
+            cache.append(l, k, v)
+            ocs[l].append(synth.bf16_bits(k), synth.bf16_bits(v))
+    assert [cache.info(l).n_events for l in range(L)] == [4, 4, 0]
+    assert cache.kernel_status() == 0
+    cache.close()
+
+
 def _random_cases(n, seed):
     rng = np.random.default_rng(seed)
     cases = []
