@@ -151,6 +151,17 @@ def test_window_not_a_multiple_of_the_group_manual_overflow_and_layers():
     cache.close()
 
 
+@pytest.mark.parametrize("B,Hq,Hkv,W,G,n_prefill", [
+    (64, 32, 8, 32, 32, 32 * 6 + 17),   # 512 pairs: one CTA for most pairs, two for the rest
+    (75, 8, 8, 32, 32, 32 * 12 + 31),   # 600 pairs: more pairs than one wave of CTAs, r = 1
+    (40, 56, 8, 64, 64, 64 * 7 + 3),    # 320 pairs, GQA-7
+])
+def test_more_pairs_than_ctas_per_wave(B, Hq, Hkv, W, G, n_prefill):
+    """Many (b, kv) pairs: the grid degenerates to one or two CTAs per pair, or to several waves."""
+    worst = run_case(B, Hq, Hkv, W, G, n_prefill, 2, seed=37, kernel=LQ_KERNEL_MMA)
+    assert worst <= 1.0
+
+
 def _random_cases(n, seed):
     rng = np.random.default_rng(seed)
     cases = []
