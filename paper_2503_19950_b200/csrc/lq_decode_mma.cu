@@ -37,8 +37,8 @@ namespace {
 
 constexpr int kWarps = 4;
 // every warp owns 12 KB of stages: 2 x 6 KB, each holding two G = 32 tiles (3 KB), one G = 64 tile
-// (5 KB) or half an fp tile (K rows or V rows, 4 KB).  Claims of two tiles measured faster than
-// single tiles (1.55 vs 1.9 us per tile and warp): the per-claim bookkeeping is not free.
+// (5 KB) or half an fp tile (K rows or V rows, 4 KB).  Loads of two tiles measured faster than
+// single tiles (1.55 vs 1.9 us per tile and warp): the per-load bookkeeping is not free.
 constexpr int kWarpStageBytes = 12288;
 __host__ __device__ constexpr int stage_bytes(int) { return 6144; }
 __host__ __device__ constexpr int n_stages(int G) { return kWarpStageBytes / stage_bytes(G); }
@@ -362,7 +362,7 @@ __device__ __forceinline__ void process_fp_values(WarpState<NCB>& st, uint32_t v
   }
 }
 
-// ---- q.zero of the key groups of one claim: bias[t][cb] for head 4cb + lane%4 of tile t (log2 units).
+// ---- q.zero of the key groups of one stage: bias[t][cb] for head 4cb + lane%4 of tile t (log2 units).
 // One MMA per k-step serves two tiles: the A fragment's rows 0-7 repeat the zero row of tile 0 and
 // rows 8-15 that of tile 1 (ldmatrix with equal row addresses inside each 8x8 matrix); the four
 // accumulators collect the k-steps of equal code-position factor, which kc[] undoes.
@@ -624,7 +624,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     n_ctas_pair = pair < a.n_extra ? a.S : a.S - 1;
   }
   const int b = pair / cv.Hkv, kv = pair % cv.Hkv;
-  constexpr int TPS = kStageBytes / TILE;  // quant tiles per claim (and per stage)
+  constexpr int TPS = kStageBytes / TILE;  // quant tiles per load (and per stage)
   const int n_warps = n_ctas_pair * kWarps, gw = slot * kWarps + warp;
   // Static partition: the pair's items -- fp tiles (cost kFpCost8 / 8 each), then quant tiles (cost
   // 1) -- lie on a cost line that is cut into n_warps equal ranges; warp gw takes the items between
@@ -641,7 +641,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     it = cut(gw);
     it_end = cut(gw + 1);
   }
-  int* queue = a.tickets + 32 * pair;  // one 128-byte line per pair: [1] is the arrival ticket
+  int* ticket = a.tickets + 32 * pair + 1;  // one 128-byte line per pair; word 1 is the arrival ticket
 
   const uint32_t stage0 = smem_u32(smem + warp * kWarpStageBytes);
   const uint32_t qsm = smem_u32(smem + kSmemStages);
@@ -925,8 +925,8 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     __syncthreads();  // every partial store of this CTA has been issued
     if (threadIdx.x == 0) {
       __threadfence();  // release, cumulative over the stores the barrier ordered before this thread
-      const int last = atomicAdd(queue + 1, 1) == n_ctas_pair - 1;
-      if (last) queue[1] = 0;  // ready for the next launch
+      const int last = atomicAdd(ticket, 1) == n_ctas_pair - 1;
+      if (last) *ticket = 0;  // ready for the next launch
       *is_last = last;
     }
     __syncthreads();
