@@ -376,3 +376,22 @@ def test_argument_errors_on_device():
         cache.append(0, k, k)
     assert e.value.status == binding.LQ_ERR_CAPACITY
     assert cache.info(0).n_seen == 0
+    # the one-launch step: capacity and window errors leave the cache as it was
+    k1 = torch.zeros(1, 2, 1, 128, dtype=torch.bfloat16, device="cuda")
+    cache.append(0, k[:, :, :64].contiguous(), k[:, :, :64].contiguous())
+    with pytest.raises(LogQuantError) as e:
+        cache.append_decode_attn(0, k1, k1, q, out)
+    assert e.value.status == binding.LQ_ERR_CAPACITY and cache.info(0).n_seen == 64
+    with pytest.raises(LogQuantError) as e:
+        cache.append_decode_attn(1, k1, k1, q, out)
+    assert e.value.status == binding.LQ_ERR_INVALID_ARG
+    manual = LogQuantCache(1, 1, 4, 2, 32, 32, max_tokens=256, auto_compress=False)
+    manual.append(0, k[:, :, :64].contiguous(), k[:, :, :64].contiguous())
+    manual.append(0, k[:, :, :32].contiguous(), k[:, :, :32].contiguous())
+    with pytest.raises(LogQuantError) as e:
+        manual.append_decode_attn(0, k1, k1, q, out)  # window full and the caller drives the overflow step
+    assert e.value.status == binding.LQ_ERR_WINDOW_FULL and manual.info(0).n_seen == 96
+    manual.compress(0)
+    manual.append_decode_attn(0, k1, k1, q, out)
+    assert manual.info(0).n_seen == 97 and torch.isfinite(out).all()
+    manual.close()
