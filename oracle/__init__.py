@@ -69,6 +69,7 @@ def lib():
         L.lqo_export.argtypes = [p] * 11
         L.lqo_dense_rows.argtypes = [p, i32, i32, p, p]
         L.lqo_attention.argtypes = [p, p, f64, p, i32]
+        L.lqo_attention_subset.argtypes = [p, p, f64, p, i32, p]
         L.lqo_hardware_threads.restype = C.c_uint
     return _lib
 
@@ -241,4 +242,15 @@ class OracleCache:
         assert q.shape == (self.B, self.Hq, self.D)
         out = np.zeros((self.B, self.Hq, self.D), np.float64)
         lib().lqo_attention(self._h, _ptr(q), float(sm_scale), _ptr(out), n_threads)
+        return out
+
+    def attention_subset(self, q_bf16: np.ndarray, sm_scale: float, fp_only: bool = False, pad=None) -> np.ndarray:
+        """Attention over the tokens at original precision only (fp_only) and/or without the first pad[b]
+        positions of sequence b (left padding of a ragged batch)."""
+        q = _c(q_bf16, np.uint16)
+        assert q.shape == (self.B, self.Hq, self.D)
+        padv = None if pad is None else _c(pad, np.int32)
+        assert padv is None or padv.shape == (self.B,)
+        out = np.zeros((self.B, self.Hq, self.D), np.float64)
+        lib().lqo_attention_subset(self._h, _ptr(q), float(sm_scale), _ptr(out), int(fp_only), _ptr(padv))
         return out

@@ -33,6 +33,12 @@
 //                     of the full-precision list and the dequantised store.  Eq. 3
 //                     (position-agnostic attention) is what allows the union to be
 //                     visited in any order.
+//   * attention over a subset: the same sum over fewer tokens.  (i) Full-precision tokens only:
+//                     what the eviction variants of Sec. 2.3 compute (tokens the filter removes are
+//                     dropped, not quantised).  (ii) Left padding: the first pad[b] positions of
+//                     sequence b are padding of a ragged batch; they pass through filter and
+//                     quantiser like any token (both are position-based) and attention leaves
+//                     them out.
 //
 // Parity status: filter, quantiser, packer and attention are pinned by tests that do
 // not go through this file's own formulas (hand simulation of Algorithm 1, closed
@@ -477,6 +483,39 @@ void lqo_attention(void* p, const uint16_t* q, double sm_scale, double* out, int
     std::vector<std::thread> th;
     for (int i = 0; i < n_threads; ++i) th.emplace_back(work, i, n_threads);
     for (auto& t : th) t.join();
+  }
+}
+
+// Decode attention over a subset of the cache.  fp_only != 0: the tokens at original precision only.
+// pad (may be null): [B], tokens of sequence b with id < pad[b] are left out.  A query whose subset is
+// empty gets zeros.
+void lqo_attention_subset(void* p, const uint16_t* q, double sm_scale, double* out, int fp_only, const int32_t* pad) {
+  Cache& c = *static_cast<Cache*>(p);
+  const int r = c.Hq / c.Hkv, D = c.D;
+  std::vector<int64_t> ids;  // token id of every row dense_rows returns, in its order
+  ids.insert(ids.end(), c.A.begin(), c.A.end());
+  ids.insert(ids.end(), c.P.begin(), c.P.end());
+  const size_t nf = ids.size();
+  ids.insert(ids.end(), c.Q.begin(), c.Q.end());
+  std::vector<double> K, V, Ks, Vs, qd(D);
+  for (int pair = 0; pair < c.B * c.Hkv; ++pair) {
+    const int b = pair / c.Hkv, kv = pair % c.Hkv;
+    dense_rows(c, c.heads[pair], K, V);
+    Ks.clear();
+    Vs.clear();
+    for (size_t i = 0; i < ids.size(); ++i) {
+      if (fp_only && i >= nf) continue;
+      if (pad && ids[i] < pad[b]) continue;
+      Ks.insert(Ks.end(), K.begin() + i * D, K.begin() + (i + 1) * D);
+      Vs.insert(Vs.end(), V.begin() + i * D, V.begin() + (i + 1) * D);
+    }
+    const int64_t n = static_cast<int64_t>(Ks.size()) / D;
+    for (int j = 0; j < r; ++j) {
+      const size_t qo = (static_cast<size_t>(b) * c.Hq + kv * r + j) * D;
+      for (int d = 0; d < D; ++d) qd[d] = bf16_to_f32(q[qo + d]);
+      if (n == 0) std::fill(out + qo, out + qo + D, 0.0);
+      else attention_dense(qd.data(), Ks.data(), Vs.data(), n, D, sm_scale, out + qo);
+    }
   }
 }
 

@@ -137,3 +137,67 @@ def test_quantisation_error_of_attention_is_small_but_nonzero():
                                        bf16_bits_to_f64(v[0, 0]), 1 / np.sqrt(D)) for h in range(Hq)])
     err = np.abs(out[0] - exact).max()
     assert 1e-6 < err < 0.2
+
+
+def _subset_case(W=32, G=32, N=7 * 32 + 5, B=3, Hq=4, Hkv=2, seed=11):
+    rng = np.random.default_rng(seed)
+    k, v = _rand_bf16(rng, (B, Hkv, N, 128)), _rand_bf16(rng, (B, Hkv, N, 128))
+    q = _rand_bf16(rng, (B, Hq, 128))
+    oc = oracle.OracleCache(B, Hq, Hkv, 128, W, G)
+    oc.append(k, v)
+    return oc, q, k, v
+
+
+def test_subset_attention_full_precision_only_is_attention_over_the_kept_tokens():
+    # the eviction variants of Sec. 2.3: tokens the filter removes are dropped.  Expected value from torch
+    # on the ORIGINAL bf16 rows of the ids Algorithm 1 keeps (hand simulation in helpers.alg1_python).
+    from helpers import alg1_python
+    oc, q, k, v = _subset_case()
+    B, Hq, Hkv, N = 3, 4, 2, k.shape[2]
+    kept, _ = alg1_python(32, N)
+    out = oc.attention_subset(q, 0.09, fp_only=True)
+    for b in range(B):
+        for h in range(Hq):
+            ref = _torch_attention(bf16_bits_to_f64(q[b, h]), bf16_bits_to_f64(k[b, h // 2][kept]),
+                                   bf16_bits_to_f64(v[b, h // 2][kept]), 0.09)
+            np.testing.assert_allclose(out[b, h], ref, rtol=0, atol=1e-13)
+    # nothing selected away: the plain attention
+    assert np.array_equal(oc.attention_subset(q, 0.09), oc.attention(q, 0.09))
+    assert np.array_equal(oc.attention_subset(q, 0.09, pad=np.zeros(B, np.int32)), oc.attention(q, 0.09))
+
+
+def test_subset_attention_left_padding_drops_exactly_the_padded_ids():
+    oc, q, k, v = _subset_case()
+    B, Hq, Hkv, G = 3, 4, 2, 32
+    img = oc.export()
+    nq = oc.n_quant
+    pad = np.array([0, 37, 150], np.int32)  # none; inside the first removed groups; beyond several groups
+    out = oc.attention_subset(q, 0.11, pad=pad)
+    kc = oracle.unpack2(img["k_codes"]).reshape(B, Hkv, nq, 128).astype(np.float64)
+    vc = oracle.unpack2(img["v_codes"]).reshape(B, Hkv, nq, 128).astype(np.float64)
+    Kq = bf16_bits_to_f64(img["k_zero"]).repeat(G, axis=2) + kc * bf16_bits_to_f64(img["k_scale"]).repeat(G, axis=2)
+    Vq = bf16_bits_to_f64(img["v_zero"]).repeat(G, axis=3) + vc * bf16_bits_to_f64(img["v_scale"]).repeat(G, axis=3)
+    ids = np.concatenate([img["kept_ids"], img["quant_ids"]])
+    for b in range(B):
+        sel = ids >= pad[b]
+        assert sel.sum() == k.shape[2] - pad[b]
+        for h in range(Hq):
+            K = np.concatenate([bf16_bits_to_f64(img["fp_k"][b, h // 2]), Kq[b, h // 2]])[sel]
+            V = np.concatenate([bf16_bits_to_f64(img["fp_v"][b, h // 2]), Vq[b, h // 2]])[sel]
+            ref = _torch_attention(bf16_bits_to_f64(q[b, h]), K, V, 0.11)
+            np.testing.assert_allclose(out[b, h], ref, rtol=0, atol=1e-13)
+    # padded VALUES never reach the output: rewriting the value rows of sequence 2's padding inside whole
+    # removed groups (a value group lies inside one token) changes nothing for that sequence
+    k2, v2 = k.copy(), v.copy()
+    v2[2, :, :150] = _rand_bf16(np.random.default_rng(5), (Hkv, 150, 128), 3.0)
+    oc2 = oracle.OracleCache(B, Hq, Hkv, 128, 32, G)
+    oc2.append(k2, v2)
+    out2 = oc2.attention_subset(q, 0.11, pad=pad)
+    np.testing.assert_allclose(out2[2], out[2], rtol=0, atol=1e-13)
+    # both selections together
+    both = oc.attention_subset(q, 0.11, fp_only=True, pad=pad)
+    for b in range(B):
+        keep = img["kept_ids"][img["kept_ids"] >= pad[b]]
+        ref = _torch_attention(bf16_bits_to_f64(q[b, 0]), bf16_bits_to_f64(k[b, 0][keep]),
+                               bf16_bits_to_f64(v[b, 0][keep]), 0.11)
+        np.testing.assert_allclose(both[b, 0], ref, rtol=0, atol=1e-13)
