@@ -161,13 +161,31 @@ lq_status_t lq_compress(lq_cache_t* cache, int32_t layer, void* stream);
 lq_status_t lq_decode_attn(lq_cache_t* cache, int32_t layer, const void* q, float sm_scale,
                            void* out, int32_t out_dtype, void* stream);
 
+/* The same over the full-precision store only: the result of the eviction variants the paper compares
+ * with in Sec. 2.3 (tokens the filter removes are dropped instead of quantised).  A comparator for accuracy
+ * measurements; the quantised store is still maintained, this call just leaves it out. */
+lq_status_t lq_decode_attn_fp_only(lq_cache_t* cache, int32_t layer, const void* q, float sm_scale,
+                                   void* out, int32_t out_dtype, void* stream);
+
+/* Left padding of a ragged batch.  pad: HOST array of `batch` int32 >= 0, copied by the call; the first pad[b]
+ * token positions of sequence b are padding in every layer.  Padding tokens are appended, filtered and
+ * quantised like any token (Algorithm 1 and the quantiser only look at positions), but every decode
+ * attention call leaves them out: sequence b attends to its tokens pad[b], pad[b] + 1, ...  Leading key
+ * groups of the quantised store that hold nothing but padding of a sequence are not even read for it.
+ * May be called at any time and takes effect from the next decode call; NULL clears all padding.  A decode
+ * call gives LQ_ERR_INVALID_ARG while some sequence has pad[b] >= the tokens appended to that layer.
+ * The masks (about max_tokens / 8 bytes per sequence and layer) are allocated by the first call
+ * (LQ_ERR_OOM if that fails) and re-derived on the host and uploaded on the decode call's stream after every
+ * overflow step or prompt ingestion of a layer.  lq_decode_attn_image_static knows no padding. */
+lq_status_t lq_set_padding(lq_cache_t* cache, const int32_t* pad);
+
 /* lq_append of ONE token followed by lq_decode_attn, in one launch: the attention kernel takes the
  * new row from k, v ([B, Hkv, 1, D] bf16, device) where it belongs in its pass over the cache and
  * writes it to the full-precision store on the way (Algorithm 1's append and Eq. 2 of the same
  * step; the result is the one of the two separate calls).  When the window is full (the overflow
  * step has to run in between; auto_compress = 0 then gives LQ_ERR_WINDOW_FULL), the plain kernel
- * is selected, or the cache is so large that the saved launch no longer pays, the call simply
- * makes the two calls.  Errors leave the cache unchanged. */
+ * is selected, the batch is padded, or the cache is so large that the saved launch no longer pays, the
+ * call simply makes the two calls.  Errors leave the cache unchanged. */
 lq_status_t lq_append_decode_attn(lq_cache_t* cache, int32_t layer, const void* k, const void* v,
                                   const void* q, float sm_scale, void* out, int32_t out_dtype,
                                   void* stream);

@@ -8,7 +8,8 @@ compressed cache is from the output over the original bf16 cache, for
   * a recent-window filter with the same number of full-precision tokens (LQ_FILTER_RECENT, the retention
     rule of the sliding-window quantisers the paper compares with, Sec. 2.2-2.3),
 
-each with 2-bit and (at G = 32) 4-bit codes.  Keys carry planted high-logit tokens at log-spaced
+each with 2-bit and (at G = 32) 4-bit codes, and for the eviction variant of both filters (the removed tokens are
+dropped instead of quantised, Sec. 2.3: `lq_decode_attn_fp_only`).  Keys carry planted high-logit tokens at log-spaced
 distances behind the query position (the shape of the attention pattern in the paper's Fig. 1); the
 prompt length is varied so that the planted tokens fall on and off the filter's kept grid.
 
@@ -54,7 +55,10 @@ def run(ctx=8192, lengths=16, B=2, kappa=16.0, a=4.0, seed=4, device="cuda"):
     rows = []
     for sh in shapes:
         for bits in sh["bits"]:
-            for filt, fname in ((LQ_FILTER_LOG, "log (Algorithm 1)"), (LQ_FILTER_RECENT, "recent window")):
+            variants = [(LQ_FILTER_LOG, "log (Algorithm 1)", False), (LQ_FILTER_RECENT, "recent window", False)]
+            if bits == 2:
+                variants += [(LQ_FILTER_LOG, "log, eviction", True), (LQ_FILTER_RECENT, "recent window, eviction", True)]
+            for filt, fname, evict in variants:
                 num = den = worst = 0.0
                 for i in range(lengths):
                     n = ctx + 37 * i  # off the window grid on purpose
@@ -64,16 +68,20 @@ def run(ctx=8192, lengths=16, B=2, kappa=16.0, a=4.0, seed=4, device="cuda"):
                                           filter=filt)
                     cache.append(0, k, v)
                     out = torch.empty(B, sh["Hq"], D, device=device)
-                    cache.decode_attn(0, q, out)
+                    if evict:
+                        cache.decode_attn_fp_only(0, q, out)
+                    else:
+                        cache.decode_attn(0, q, out)
                     torch.cuda.synchronize()
                     inf = cache.info(0)
                     err = (out.double() - ref).abs()
                     num += float(err.sum())
                     den += float(ref.abs().sum())
                     worst = max(worst, float(err.max() / ref.abs().max()))
-                    ratio = (n * 4 * D) / (inf.n_quant * inf.bytes_quant_per_token + inf.n_fp * 4 * D)
+                    kept_bytes = inf.n_fp * 4 * D + (0 if evict else inf.n_quant * inf.bytes_quant_per_token)
+                    ratio = (n * 4 * D) / kept_bytes
                     cache.close()
-                rows.append(dict(shape=sh["name"], bits=bits, filter=fname, rel_l1=num / den, worst_rel_max=worst,
+                rows.append(dict(shape=sh["name"], bits=0 if evict else bits, filter=fname, rel_l1=num / den, worst_rel_max=worst,
                                  compression=ratio))
     return rows
 

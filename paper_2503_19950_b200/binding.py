@@ -43,6 +43,7 @@ class lq_device_image_t(C.Structure):
 
 
 SYMBOLS = ["lq_cache_create", "lq_destroy", "lq_append", "lq_compress", "lq_decode_attn", "lq_append_decode_attn",
+           "lq_decode_attn_fp_only", "lq_set_padding",
            "lq_decode_step_host", "lq_profile_enable", "lq_profile_read", "lq_kernel_status", "lq_cache_info", "lq_export",
            "lq_next_evicted_ids", "lq_decode_attn_image_static", "lq_status_str", "lq_last_error"]
 
@@ -70,6 +71,8 @@ def load_library():
         L.lq_compress.argtypes = [vp, i32, vp]
         L.lq_decode_attn.argtypes = [vp, i32, vp, C.c_float, vp, i32, vp]
         L.lq_append_decode_attn.argtypes = [vp, i32, vp, vp, vp, C.c_float, vp, i32, vp]
+        L.lq_decode_attn_fp_only.argtypes = [vp, i32, vp, C.c_float, vp, i32, vp]
+        L.lq_set_padding.argtypes = [vp, vp]
         L.lq_decode_step_host.argtypes = [vp, i32, vp, vp, vp, C.c_float, vp, i32, vp]
         L.lq_kernel_status.argtypes = [vp, C.POINTER(C.c_int32)]
         L.lq_profile_enable.argtypes = [vp, i32]
@@ -175,6 +178,23 @@ class LogQuantCache:
         out_dtype = 1 if out.dtype == torch.bfloat16 else 0
         self._check(self._lib.lq_decode_attn(self._h, layer, _ptr(q), sm_scale, _ptr(out), out_dtype,
                                              _stream(stream)))
+
+    def decode_attn_fp_only(self, layer, q, out, sm_scale=0.0, stream=None):
+        import torch
+        out_dtype = 1 if out.dtype == torch.bfloat16 else 0
+        self._check(self._lib.lq_decode_attn_fp_only(self._h, layer, _ptr(q), sm_scale, _ptr(out), out_dtype,
+                                                     _stream(stream)))
+
+    def set_padding(self, pad):
+        """pad: `batch` leading padding positions per sequence (any int sequence), or None to clear."""
+        if pad is None:
+            self._check(self._lib.lq_set_padding(self._h, None))
+            return
+        pad = [int(x) for x in pad]
+        if len(pad) != self.cfg.batch:
+            raise ValueError("one padding length per sequence of the batch")
+        arr = (C.c_int32 * self.cfg.batch)(*pad)
+        self._check(self._lib.lq_set_padding(self._h, C.cast(arr, C.c_void_p)))
 
     def decode_step_host(self, layer, k_host, v_host, q_host, out_host, sm_scale=0.0, sync=True, stream=None):
         self._check(self._lib.lq_decode_step_host(self._h, layer, _ptr(k_host), _ptr(v_host), _ptr(q_host),

@@ -53,6 +53,16 @@ struct lq_cache {
   uint8_t* stage_q = nullptr;
   uint8_t* stage_out = nullptr;
   int64_t n_launches = 0;
+  // left padding of a ragged batch (lq_set_padding): pad[b] leading positions of sequence b that attention
+  // leaves out.  Device copy per layer: [B][4] row info, [B][fp_words] slot mask, [B][q_words] store mask,
+  // rebuilt (mask_dirty) when the layer's stores changed.
+  std::vector<int32_t> pad;
+  bool has_pad = false;
+  std::vector<char> mask_dirty;
+  uint32_t* masks = nullptr;
+  int fp_words = 0, q_words = 0;
+  int64_t mask_layer_words = 0;
+  std::vector<uint32_t> mask_host;
   // optional timing of the split-K attention kernel
   bool profiling = false;
   std::vector<cudaEvent_t> ev_pool;  // 2 events per timed launch
@@ -92,6 +102,7 @@ void free_all(lq_cache* c) {
     cudaFree(c->stage_v);
     cudaFree(c->stage_q);
     cudaFree(c->stage_out);
+    cudaFree(c->masks);
     for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   }
 }
@@ -216,6 +227,8 @@ lq_status_t run_event_residual(lq_cache* c, int layer, cudaStream_t st) {
 }
 
 lq_status_t run_events(lq_cache* c, const std::vector<int>& full_layers, cudaStream_t st) {
+  if (!c->mask_dirty.empty())
+    for (int layer : full_layers) c->mask_dirty[layer] = 1;
   if (residual_mode(c)) {
     for (int layer : full_layers) {
       lq_status_t s = run_event_residual(c, layer, st);
@@ -255,6 +268,52 @@ lq_status_t run_events(lq_cache* c, const std::vector<int>& full_layers, cudaStr
       apply_event(c, c->layers[full_layers[k]]);
     }
   }
+  return LQ_OK;
+}
+
+// Padding masks of one layer from the host mirror of its stores (which token id sits in which fp slot and at
+// which place of the quantised store) and upload.  Rows appended later lie beyond the rebuilt prefix of the fp
+// store, carry ids above every pad (checked by the caller) and need no bit.
+lq_status_t upload_masks(lq_cache* c, int layer, cudaStream_t st) {
+  const LayerState& L = c->layers[layer];
+  const int B = c->cfg.batch, G = c->cfg.group;
+  c->mask_host.assign(static_cast<size_t>(c->mask_layer_words), 0u);
+  int32_t* rowinfo = reinterpret_cast<int32_t*>(c->mask_host.data());
+  uint32_t* fpm = c->mask_host.data() + 4 * B;
+  uint32_t* qm = fpm + static_cast<size_t>(c->fp_words) * B;
+  const int64_t tiles = L.n_quant / G;
+  for (int b = 0; b < B; ++b) {
+    const int pad = c->pad[b];
+    bool any_fp = false;
+    for (int s = 0; s < L.n_fp; ++s)
+      if (L.slot_token[s] < pad) {
+        fpm[static_cast<size_t>(b) * c->fp_words + s / 32] |= 1u << (s % 32);
+        any_fp = true;
+      }
+    int64_t skip = 0, last = 0;  // leading tiles that are padding entirely; one past the last tile with padding
+    bool leading = true;
+    for (int64_t t = 0; t < tiles; ++t) {
+      int n_masked = 0;
+      for (int i = 0; i < G; ++i) {
+        const int64_t qi = t * G + i;
+        if (L.quant_ids[qi] < pad) {
+          qm[static_cast<size_t>(b) * c->q_words + qi / 32] |= 1u << (qi % 32);
+          ++n_masked;
+        }
+      }
+      if (leading && n_masked == G) skip = t + 1;
+      else leading = false;
+      if (n_masked) last = t + 1;
+    }
+    rowinfo[4 * b + 0] = static_cast<int32_t>(skip);
+    rowinfo[4 * b + 1] = static_cast<int32_t>(last);
+    rowinfo[4 * b + 2] = any_fp ? 1 : 0;
+  }
+  // pageable source: staged by the runtime before the call returns
+  cudaError_t e = cudaMemcpyAsync(c->masks + layer * c->mask_layer_words, c->mask_host.data(),
+                                  c->mask_host.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return cuda_fail(c, e, "padding mask upload");
+  c->mask_dirty[layer] = 0;
   return LQ_OK;
 }
 
@@ -378,6 +437,7 @@ namespace {
 // step and the final slot map, and one kernel writes both stores.
 lq_status_t ingest_prompt(lq_cache* c, int layer, const void* k, const void* v, int n, cudaStream_t st) {
   LayerState& L = c->layers[layer];
+  if (!c->mask_dirty.empty()) c->mask_dirty[layer] = 1;
   const int W = c->cfg.window, G = c->cfg.group;
   std::vector<int32_t> idx;
   idx.reserve(static_cast<size_t>(n) + 3 * W);
@@ -486,12 +546,40 @@ lq_status_t lq_compress(lq_cache_t* c, int32_t layer, void* stream) {
 
 namespace {
 lq_status_t decode_impl(lq_cache_t* c, int32_t layer, const void* q, float sm_scale, void* out, int32_t out_dtype,
-                        void* stream, const void* new_k, const void* new_v, int new_slot);
+                        void* stream, const void* new_k, const void* new_v, int new_slot, bool fp_only = false);
 }
 
 lq_status_t lq_decode_attn(lq_cache_t* c, int32_t layer, const void* q, float sm_scale, void* out,
                            int32_t out_dtype, void* stream) {
   return decode_impl(c, layer, q, sm_scale, out, out_dtype, stream, nullptr, nullptr, 0);
+}
+
+lq_status_t lq_decode_attn_fp_only(lq_cache_t* c, int32_t layer, const void* q, float sm_scale, void* out,
+                                   int32_t out_dtype, void* stream) {
+  return decode_impl(c, layer, q, sm_scale, out, out_dtype, stream, nullptr, nullptr, 0, true);
+}
+
+lq_status_t lq_set_padding(lq_cache_t* c, const int32_t* pad_host) {
+  if (!c) return LQ_ERR_INVALID_ARG;
+  if (!pad_host) {
+    c->has_pad = false;
+    return LQ_OK;
+  }
+  const int B = c->cfg.batch;
+  for (int b = 0; b < B; ++b)
+    if (pad_host[b] < 0) return LQ_ERR_INVALID_ARG;
+  if (!c->dry && !c->masks) {
+    const int slots = 3 * c->cfg.window + c->cfg.group;
+    c->fp_words = (slots + 31) / 32;
+    c->q_words = static_cast<int>((c->cfg.max_tokens + 31) / 32);
+    c->mask_layer_words = static_cast<int64_t>(B) * (4 + c->fp_words + c->q_words);
+    if (!dev_alloc(c, reinterpret_cast<void**>(&c->masks), c->mask_layer_words * c->cfg.n_layers * 4)) return LQ_ERR_OOM;
+  }
+  c->pad.assign(pad_host, pad_host + B);
+  c->has_pad = false;
+  for (int b = 0; b < B; ++b) c->has_pad |= pad_host[b] > 0;
+  c->mask_dirty.assign(c->cfg.n_layers, 1);
+  return LQ_OK;
 }
 
 lq_status_t lq_append_decode_attn(lq_cache_t* c, int32_t layer, const void* k, const void* v, const void* q,
@@ -509,9 +597,9 @@ lq_status_t lq_append_decode_attn(lq_cache_t* c, int32_t layer, const void* k, c
   const int64_t step_bytes = static_cast<int64_t>(c->cfg.batch) * c->cfg.n_kv_heads *
                              (L.n_quant * (quant_tile_bytes(c->cfg.group, c->cfg.bits / 2) / c->cfg.group) +
                               static_cast<int64_t>(L.n_fp) * 4 * kD);
-  if (kept(L) == 3 * W || !use_mma(c) || step_bytes > (192LL << 20)) {
+  if (kept(L) == 3 * W || !use_mma(c) || step_bytes > (192LL << 20) || c->has_pad) {
     // the window is full (the overflow step has to run between the two), the plain kernel is
-    // selected, or the launch is long: the two separate calls
+    // selected, the launch is long, or the batch is padded: the two separate calls
     lq_status_t s = lq_append(c, layer, k, v, 1, stream);
     if (s != LQ_OK) return s;
     return lq_decode_attn(c, layer, q, sm_scale, out, out_dtype, stream);
@@ -534,7 +622,7 @@ lq_status_t lq_append_decode_attn(lq_cache_t* c, int32_t layer, const void* k, c
 
 namespace {
 lq_status_t decode_impl(lq_cache_t* c, int32_t layer, const void* q, float sm_scale, void* out, int32_t out_dtype,
-                        void* stream, const void* new_k, const void* new_v, int new_slot) {
+                        void* stream, const void* new_k, const void* new_v, int new_slot, bool fp_only) {
   if (!c || layer < 0 || layer >= c->cfg.n_layers || (out_dtype != 0 && out_dtype != 1)) return LQ_ERR_INVALID_ARG;
   if (c->dry) return LQ_ERR_UNSUPPORTED;
   if (!q || !out || (reinterpret_cast<uintptr_t>(q) & 15)) return LQ_ERR_INVALID_ARG;
@@ -545,7 +633,25 @@ lq_status_t decode_impl(lq_cache_t* c, int32_t layer, const void* q, float sm_sc
   a.cv = c->cv;
   a.layer = layer;
   a.n_fp = L.n_fp;
-  a.n_quant = L.n_quant;
+  a.n_quant = fp_only ? 0 : L.n_quant;
+  a.rowinfo = nullptr;
+  a.qmask = a.fpmask = nullptr;
+  a.qmask_words = a.fpmask_words = 0;
+  if (c->has_pad) {
+    // every sequence keeps at least its newest token
+    for (int b = 0; b < c->cfg.batch; ++b)
+      if (c->pad[b] >= L.n_seen) return LQ_ERR_INVALID_ARG;
+    if (c->mask_dirty[layer]) {
+      lq_status_t ms = upload_masks(c, layer, st);
+      if (ms != LQ_OK) return ms;
+    }
+    const uint32_t* base = c->masks + layer * c->mask_layer_words;
+    a.rowinfo = reinterpret_cast<const int32_t*>(base);
+    a.fpmask = base + 4 * c->cfg.batch;
+    a.qmask = a.fpmask + static_cast<int64_t>(c->fp_words) * c->cfg.batch;
+    a.fpmask_words = c->fp_words;
+    a.qmask_words = c->q_words;
+  }
   if (!(sm_scale > 0.f)) sm_scale = 1.0f / std::sqrt(static_cast<float>(kD));
   a.scale_log2 = sm_scale * 1.4426950408889634f;
   a.q = q;

@@ -295,10 +295,12 @@ __device__ __forceinline__ void split_p_bf16(const float (&pT)[2][2], bool odd, 
 
 // ---- one fp tile: 16 bf16 tokens (rows swizzled in 16-byte chunks by row & 7), loaded as two
 // units: the K rows (scores, softmax; leaves the p.v B operands in b0/b1), then the V rows -------
+// pad16: bit i set = slot i of the tile is padding (left out); at least one valid slot is not
 template <int NCB>
 __device__ __forceinline__ void process_fp_keys(WarpState<NCB>& st, const uint32_t (&qs)[NCB][8][2], uint32_t krows,
                                                 int n_valid, const float (&kc)[4], int lane, uint32_t oddmask,
-                                                int opaque_zero, uint32_t (&b0)[2], uint32_t (&b1)[2]) {
+                                                int opaque_zero, uint32_t (&b0)[2], uint32_t (&b1)[2],
+                                                uint32_t pad16 = 0u) {
   const int n = lane >> 2;
   float acc[NCB][4][4];
   {
@@ -326,8 +328,8 @@ __device__ __forceinline__ void process_fp_keys(WarpState<NCB>& st, const uint32
       s0 = fmaf(acc[cb][c][0], kc[c], s0);
       s1 = fmaf(acc[cb][c][2], kc[c], s1);
     }
-    s[0][cb][0] = n < n_valid ? s0 : -INFINITY;
-    s[0][cb][1] = n + 8 < n_valid ? s1 : -INFINITY;
+    s[0][cb][0] = n < n_valid && !((pad16 >> n) & 1u) ? s0 : -INFINITY;
+    s[0][cb][1] = n + 8 < n_valid && !((pad16 >> (n + 8)) & 1u) ? s1 : -INFINITY;
   }
   tile_softmax<NCB, 1>(st, s, lane, opaque_zero);
   float pT[2][2];
@@ -409,10 +411,11 @@ __device__ __forceinline__ void patch_new_row(uint32_t half_tile_smem, uint8_t* 
 // PL = 2-bit planes per code.  A 4-bit code is 4 * (high plane) + (low plane): the high plane goes
 // through the same contractions first, its score accumulators are multiplied by 4 before the low
 // plane is added, and in p.v it meets p * s_v * 4 (all exact).
+// pad0/pad1: bit i set = token i (pad0) or 32 + i (pad1) of the tile is padding (left out); not all of them are
 template <int G, int NCB, int PL>
 __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uint32_t (&qs)[NCB][8][2], uint32_t tile,
                                                    const float (&bias)[NCB], float kq, int lane, uint32_t oddmask,
-                                                   int opaque_zero) {
+                                                   int opaque_zero, uint32_t pad0 = 0u, uint32_t pad1 = 0u) {
   constexpr int NS = G / 16, NG = kD / G, VS = vsz_subtile_bytes(G);
   const int n = lane >> 2, j = lane & 3;
   // ---- q.k on all G tokens.  Per pair of k-steps: the key scale of the lane's channels is folded
@@ -476,6 +479,17 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
       for (int u = 0; u < NS; ++u) {
         s[u][cb][0] = fmaf(acc[u][cb][0] + acc[u][cb][1], kq, bias[cb]);
         s[u][cb][1] = fmaf(acc[u][cb][2] + acc[u][cb][3], kq, bias[cb]);
+      }
+    }
+    if (pad0 | pad1) {  // always false in the instantiation without padding (constant arguments)
+#pragma unroll
+      for (int u = 0; u < NS; ++u) {
+        const uint32_t w = (u < 2 ? pad0 : pad1) >> (16 * (u & 1) + n);
+#pragma unroll
+        for (int cb = 0; cb < NCB; ++cb) {
+          if (w & 1u) s[u][cb][0] = -INFINITY;
+          if (w & 0x100u) s[u][cb][1] = -INFINITY;
+        }
       }
     }
   }
@@ -602,7 +616,9 @@ constexpr int kMergeMax = 2048;  // S * r records the fused second pass can stag
 // two loads in flight.
 // FUSED: the launch also appends one token (DecodeArgs::new_k); a separate instantiation so that
 // the plain kernel's main loop is not touched.
-template <int G, int NCB, int PL, bool FUSED>
+// PADDED: the batch is left-padded (DecodeArgs::rowinfo): per sequence, leading quant tiles that are
+// padding entirely are not visited, and tiles and slots with padding among their tokens get -inf scores.
+template <int G, int NCB, int PL, bool FUSED, bool PADDED>
 __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerSm - 1) lq_decode_mma_kernel(DecodeArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   const CacheView& cv = a.cv;
@@ -631,9 +647,15 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   // cut gw and cut gw + 1 (boundaries rounded to the nearest item).  Every SM carries the same number
   // of identical warps, so equal work gives (nearly) equal finishing times without any work queue;
   // weighting the ranges by the launch order of the CTAs on an SM measured slower.
+  // quant item i of this pair is tile qskip + i of the store
+  const int qskip = PADDED ? min(a.rowinfo[4 * b + 0], a.tiles_quant) : 0;
+  const int qpad_end = PADDED ? a.rowinfo[4 * b + 1] : 0;
+  const bool fp_padded = PADDED && a.rowinfo[4 * b + 2] != 0;
+  const uint32_t* qmask = PADDED ? a.qmask + static_cast<int64_t>(b) * a.qmask_words : nullptr;
+  const uint32_t* fpmask = PADDED ? a.fpmask + static_cast<int64_t>(b) * a.fpmask_words : nullptr;
   int it, it_end;
   {
-    const int F8 = a.tiles_fp * kFpCost8, C8 = F8 + a.tiles_quant * 8;
+    const int F8 = a.tiles_fp * kFpCost8, C8 = F8 + (a.tiles_quant - qskip) * 8;
     auto cut = [&](int k) {
       const int pos8 = static_cast<int>(static_cast<int64_t>(k) * C8 / n_warps);
       return pos8 < F8 ? (pos8 + kFpCost8 / 2) / kFpCost8 : a.tiles_fp + (pos8 - F8 + 4) / 8;
@@ -700,7 +722,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
         const int nt = min(min(TPS, cap), it_end - it);
         desc = it | (nt << 24);
         bytes = nt * TILE;
-        src = qbase + static_cast<int64_t>(it - a.tiles_fp) * TILE;
+        src = qbase + static_cast<int64_t>(it - a.tiles_fp + qskip) * TILE;
         it += nt;
       }
     }
@@ -791,14 +813,31 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
         float bias[NCB];
 #pragma unroll
         for (int cb = 0; cb < NCB; ++cb) bias[cb] = t ? bias2[1][cb] : bias2[0][cb];
-        process_quant_tile<G, NCB, PL>(st, qs, sbase + t * TILE, bias, kq, lane, oddmask, a.zero);
+        if (PADDED) {
+          const int tile = (desc & 0xFFFFFF) - a.tiles_fp + qskip + t;
+          uint32_t pad0 = 0u, pad1 = 0u;
+          if (tile < qpad_end) {
+            pad0 = __ldg(qmask + tile * (G / 32));
+            if (G == 64) pad1 = __ldg(qmask + tile * (G / 32) + 1);
+          }
+          if (pad0 == kFull && (G == 32 || pad1 == kFull)) continue;  // nothing but padding
+          process_quant_tile<G, NCB, PL>(st, qs, sbase + t * TILE, bias, kq, lane, oddmask, a.zero, pad0, pad1);
+        } else {
+          process_quant_tile<G, NCB, PL>(st, qs, sbase + t * TILE, bias, kq, lane, oddmask, a.zero);
+        }
       }
     } else if (desc >= 0) {
       if (FUSED && desc == (a.new_slot >> 4))
         patch_new_row(sbase, const_cast<uint8_t*>(fpbase) + static_cast<int64_t>(desc) * kFpTileBytes, a.new_k, pair,
                       a.new_slot & 15, lane);
       const int nv = min(16, a.n_fp - desc * 16);
-      process_fp_keys<NCB>(st, qs, sbase, nv, kc, lane, oddmask, a.zero, fb0, fb1);
+      uint32_t pad16 = 0u;
+      if (fp_padded) pad16 = (__ldg(fpmask + (desc >> 1)) >> (16 * (desc & 1))) & ((1u << nv) - 1u);
+      if (PADDED && pad16 == (1u << nv) - 1u) {
+        fb0[0] = fb0[1] = fb1[0] = fb1[1] = 0u;  // nothing but padding: its V rows meet p = 0
+      } else {
+        process_fp_keys<NCB>(st, qs, sbase, nv, kc, lane, oddmask, a.zero, fb0, fb1, pad16);
+      }
     } else {
       if (FUSED && -1 - desc == (a.new_slot >> 4))
         patch_new_row(sbase, const_cast<uint8_t*>(fpbase) + static_cast<int64_t>(-1 - desc) * kFpTileBytes + kFpTileVOffset,
@@ -1061,9 +1100,15 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
   const int r = a.cv.Hq / a.cv.Hkv;
   void (*kern)(DecodeArgs) = nullptr;
   const bool fused = a.new_k != nullptr;
-#define LQ_PICK(G_, P_)                                                                                   \
-  kern = r <= 4 ? (fused ? lq_decode_mma_kernel<G_, 1, P_, true> : lq_decode_mma_kernel<G_, 1, P_, false>) \
-                : (fused ? lq_decode_mma_kernel<G_, 2, P_, true> : lq_decode_mma_kernel<G_, 2, P_, false>)
+  const bool padded = a.rowinfo != nullptr;
+  if (fused && padded) return cudaErrorInvalidValue;  // the caller appends separately for a padded batch
+#define LQ_PICK(G_, P_)                                                                                       \
+  kern = r <= 4 ? (fused    ? lq_decode_mma_kernel<G_, 1, P_, true, false>                                    \
+                   : padded ? lq_decode_mma_kernel<G_, 1, P_, false, true>                                    \
+                            : lq_decode_mma_kernel<G_, 1, P_, false, false>)                                  \
+                : (fused    ? lq_decode_mma_kernel<G_, 2, P_, true, false>                                    \
+                   : padded ? lq_decode_mma_kernel<G_, 2, P_, false, true>                                    \
+                            : lq_decode_mma_kernel<G_, 2, P_, false, false>)
   if (a.cv.G == 32 && a.cv.planes == 1) LQ_PICK(32, 1);
   else if (a.cv.G == 32 && a.cv.planes == 2) LQ_PICK(32, 2);
   else if (a.cv.G == 64 && a.cv.planes == 1) LQ_PICK(64, 1);
@@ -1073,11 +1118,11 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
                     kSmemStages >= (kMergeMax + kWarps * kMaxRatio * kD) * 4,
                 "merge scratch");
   // opt in to the dynamic shared memory size once per (device, kernel variant)
-  static bool configured[64][16] = {};
+  static bool configured[64][32] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  const int variant = (fused ? 8 : 0) + (a.cv.planes == 2 ? 4 : 0) + (a.cv.G == 64 ? 2 : 0) + (r <= 4 ? 0 : 1);
+  const int variant = (padded ? 16 : 0) + (fused ? 8 : 0) + (a.cv.planes == 2 ? 4 : 0) + (a.cv.G == 64 ? 2 : 0) + (r <= 4 ? 0 : 1);
   if (dev < 0 || dev >= 64 || !configured[dev][variant]) {
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;

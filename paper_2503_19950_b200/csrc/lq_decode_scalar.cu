@@ -91,9 +91,18 @@ __global__ void __launch_bounds__(128) lq_decode_scalar_kernel(DecodeArgs a) {
 #pragma unroll
   for (int j = 0; j < kMaxRatio; ++j) { m[j] = -INFINITY; l[j] = 0.f; acc[j] = 0.f; }
 
+  // left padding: bit set = attention leaves the token out
+  const uint32_t* fpmask = a.fpmask ? a.fpmask + static_cast<int64_t>(b) * a.fpmask_words : nullptr;
+  const uint32_t* qmask = a.qmask ? a.qmask + static_cast<int64_t>(b) * a.qmask_words : nullptr;
+  auto is_padding = [&](int64_t t) {
+    if (t < a.n_fp) return fpmask != nullptr && ((fpmask[t >> 5] >> (t & 31)) & 1u) != 0u;
+    const int64_t tq = t - a.n_fp;
+    return qmask != nullptr && ((qmask[tq >> 5] >> (tq & 31)) & 1u) != 0u;
+  };
+
   for (int64_t t0 = begin; t0 < end; t0 += 128) {
     const int64_t t = t0 + tid;
-    const bool valid = t < end;
+    const bool valid = t < end && !is_padding(t);
     float sc[kMaxRatio];
 #pragma unroll
     for (int j = 0; j < kMaxRatio; ++j) sc[j] = 0.f;

@@ -81,6 +81,15 @@ struct DecodeArgs {
   const void* new_k;
   const void* new_v;
   int new_slot;
+  // left padding (null when the cache has none): per sequence b, tokens attention leaves out.
+  //   rowinfo[4*b + 0] = leading quant tiles that are padding entirely (not even loaded),
+  //   rowinfo[4*b + 1] = first quant tile from which on no token is padding (tiles in between consult qmask),
+  //   rowinfo[4*b + 2] = 1 if some slot of the fp store is padding (fpmask is consulted);
+  //   qmask[b*qmask_words + i/32] bit i%32: token i of the quantised store, fpmask likewise per fp slot.
+  const int32_t* rowinfo;
+  const uint32_t* qmask;
+  const uint32_t* fpmask;
+  int qmask_words, fpmask_words;
   int* status;  // device word; kernels OR error bits into it (bounded waits that gave up)
   int* tickets; // one 128-byte line per (b, kv): word [1] is the arrival counter of the fused second
                 // pass, 0 at rest

@@ -26,8 +26,10 @@ def assert_images_equal(got: dict, want: dict):
 
 def run_case(B, Hq, Hkv, W, G, n_prefill, n_steps, seed, kernel, n_outliers=3, check_image_every=1,
              sm_scale=0.0, n_splits=0, prefill_chunk=None, auto_compress=True, out_dtype=torch.float32,
-             q_gain=1.0, bits=2, recent_only=False):
-    """Prefill n_prefill tokens, then n_steps x (append 1 token, attention).  Returns max error ratio."""
+             q_gain=1.0, bits=2, recent_only=False, pad=None, fp_only=False):
+    """Prefill n_prefill tokens, then n_steps x (append 1 token, attention).  Returns max error ratio.
+    pad: leading padding positions per sequence (set before the first token); fp_only: attention over the
+    full-precision store only."""
     D = 128
     dev = "cuda"
     total = n_prefill + n_steps
@@ -35,6 +37,8 @@ def run_case(B, Hq, Hkv, W, G, n_prefill, n_steps, seed, kernel, n_outliers=3, c
     cache = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=total + 8, auto_compress=auto_compress, kernel=kernel,
                           n_splits=n_splits, bits=bits, filter=1 if recent_only else 0)
     oc = oracle.OracleCache(B, Hq, Hkv, D, W, G, bits=bits, recent_only=recent_only)
+    if pad is not None:
+        cache.set_padding(pad)
 
     def feed(start, n):
         k, v = synth.keys_values(seed, B, Hkv, n, D, dev, token_start=start, token_total=total, outliers=outl)
@@ -68,9 +72,15 @@ def run_case(B, Hq, Hkv, W, G, n_prefill, n_steps, seed, kernel, n_outliers=3, c
             assert_images_equal(cache.export(0), oc.export())
         q = (synth.queries(seed, B, Hq, D, step, dev).float() * q_gain).to(torch.bfloat16)
         out = torch.full((B, Hq, D), float("nan"), dtype=out_dtype, device=dev)
-        cache.decode_attn(0, q, out, sm_scale=sm_scale)
+        if fp_only:
+            cache.decode_attn_fp_only(0, q, out, sm_scale=sm_scale)
+        else:
+            cache.decode_attn(0, q, out, sm_scale=sm_scale)
         torch.cuda.synchronize()
-        ref = oc.attention(synth.bf16_bits(q), scale, n_threads=8)
+        if fp_only or pad is not None:
+            ref = oc.attention_subset(synth.bf16_bits(q), scale, fp_only=fp_only, pad=pad)
+        else:
+            ref = oc.attention(synth.bf16_bits(q), scale, n_threads=8)
         got = out.float().cpu().numpy().astype(np.float64)
         assert np.isfinite(got).all()
         tol = attn_tolerance(ref)

@@ -395,3 +395,75 @@ def test_argument_errors_on_device():
     manual.append_decode_attn(0, k1, k1, q, out)
     assert manual.info(0).n_seen == 97 and torch.isfinite(out).all()
     manual.close()
+
+
+# ---- left padding of a ragged batch, and attention over the full-precision store only ----------------
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("B,Hq,Hkv,W,G,bits,n_prefill,n_steps,chunk,pad", [
+    (3, 8, 2, 32, 32, 2, 500, 40, None, [0, 37, 300]),      # none / inside the first groups / whole leading groups
+    (2, 14, 2, 64, 64, 2, 64 * 9 + 3, 70, 200, [129, 5]),   # GQA-7 (two column blocks), G = 64: two mask words
+    (2, 8, 8, 32, 32, 4, 32 * 8 + 17, 20, None, [64, 201]), # r = 1, 4-bit codes
+    (2, 8, 2, 42, 64, 2, 42 * 9 + 5, 50, None, [11, 260]),  # W not a multiple of G: waiting tokens may be padding
+    (1, 4, 1, 32, 32, 2, 40, 70, None, [39]),               # padding still in the window; crosses the first overflow
+])
+def test_left_padded_batch(kernel, B, Hq, Hkv, W, G, bits, n_prefill, n_steps, chunk, pad):
+    """Sequence b attends to tokens pad[b].. only; the stores are those of the unpadded run (same image)."""
+    worst = run_case(B, Hq, Hkv, W, G, n_prefill, n_steps, 31, kernel, bits=bits, prefill_chunk=chunk, pad=pad,
+                     check_image_every=9)
+    assert worst <= 1.0
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("B,Hq,Hkv,W,G,n_prefill,pad", [
+    (2, 8, 2, 32, 32, 700, None), (2, 14, 2, 64, 64, 1000, None), (2, 8, 2, 32, 32, 700, [90, 0])])
+def test_attention_over_the_full_precision_store_only(kernel, B, Hq, Hkv, W, G, n_prefill, pad):
+    worst = run_case(B, Hq, Hkv, W, G, n_prefill, 12, 32, kernel, fp_only=True, pad=pad, check_image_every=0)
+    assert worst <= 1.0
+
+
+def test_padding_can_change_and_bad_padding_is_refused():
+    B, Hq, Hkv, W, G, D, N = 2, 8, 2, 32, 32, 128, 400
+    cache = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=N + 16)
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G)
+    k, v = synth.keys_values(33, B, Hkv, N, D, "cuda")
+    cache.append(0, k, v)
+    oc.append(synth.bf16_bits(k), synth.bf16_bits(v))
+    q = synth.queries(33, B, Hq, D, 0, "cuda")
+    out = torch.empty(B, Hq, D, device="cuda")
+
+    def check(pad):
+        cache.decode_attn(0, q, out)
+        torch.cuda.synchronize()
+        ref = oc.attention_subset(synth.bf16_bits(q), 1 / np.sqrt(D), pad=pad)
+        assert np.abs(out.cpu().numpy() - ref).max() <= attn_tolerance(ref)
+        return out.clone()
+
+    plain = check(None)
+    cache.set_padding([100, 0])
+    padded = check([100, 0])
+    assert not torch.equal(padded[0], plain[0]) and torch.equal(padded[1], plain[1])
+    cache.set_padding([0, 399])  # sequence 1 keeps its newest token only: the output is that token's value row
+    one = check([0, 399])
+    assert torch.allclose(one[1, 0], v[1, 0, 399].float(), atol=1e-5)
+    cache.set_padding(None)
+    assert torch.equal(check(None), plain)
+    # the one-launch step takes the two-call path on a padded batch and still agrees with the oracle
+    cache.set_padding([7, 150])
+    k1, v1 = synth.keys_values(34, B, Hkv, 1, D, "cuda")
+    cache.append_decode_attn(0, k1, v1, q, out)
+    torch.cuda.synchronize()
+    oc.append(synth.bf16_bits(k1), synth.bf16_bits(v1))
+    ref = oc.attention_subset(synth.bf16_bits(q), 1 / np.sqrt(D), pad=[7, 150])
+    assert np.abs(out.cpu().numpy() - ref).max() <= attn_tolerance(ref)
+    # refused: negative, or a sequence with nothing left
+    with pytest.raises(LogQuantError) as e:
+        cache.set_padding([-1, 0])
+    assert e.value.status == binding.LQ_ERR_INVALID_ARG
+    cache.set_padding([N + 1, 0])
+    with pytest.raises(LogQuantError) as e:
+        cache.decode_attn(0, q, out)
+    assert e.value.status == binding.LQ_ERR_INVALID_ARG
+    cache.set_padding([N, 0])  # N + 1 tokens appended: the newest one is left
+    check([N, 0])
+    assert cache.kernel_status() == 0
+    cache.close(); oc.close()

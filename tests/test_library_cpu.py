@@ -72,6 +72,20 @@ def test_no_gpu_means_no_compute():
     assert e.value.status == binding.LQ_ERR_UNSUPPORTED
 
 
+def test_padding_arguments_without_a_device():
+    c = _dry(W=128, G=32, batch=3)
+    c.set_padding([0, 5, 9])
+    c.set_padding(None)
+    with pytest.raises(LogQuantError) as e:
+        c.set_padding([0, -2, 1])
+    assert e.value.status == binding.LQ_ERR_INVALID_ARG
+    with pytest.raises(ValueError):
+        c.set_padding([1, 2])
+    with pytest.raises(LogQuantError) as e:  # still no compute without a device
+        c._check(c._lib.lq_decode_attn_fp_only(c._h, 0, None, 0.0, None, 0, None))
+    assert e.value.status == binding.LQ_ERR_UNSUPPORTED
+
+
 @pytest.mark.parametrize("W,G", [(32, 32), (64, 32), (128, 64), (256, 64)])
 def test_host_mirror_of_algorithm1_matches_oracle(W, G):
     c = _dry(W=W, G=G, max_tokens=40 * W)
