@@ -176,6 +176,8 @@ __device__ __forceinline__ uint32_t ext_f16(uint32_t w, uint32_t w10) {
 
 // NCB = number of column blocks of 4 heads.  NCB == 1: p.v columns are (hi, lo) per head and the
 // probabilities carry a factor 2^64 (kPExp) so that products with bf16 subnormal codes stay normal.
+// NCB == 2: the probabilities (at most 2^8 because the reference maximum moves lazily) carry 2^-8, so
+// that p * s_v fits fp16 for every value scale fp16 itself can hold.
 // p.v flavour.  bf16_pv: columns are (hi, lo) per head, everything bf16, exact products, r <= 4 only.
 // Otherwise: heads on the 8 columns, value codes as fp16 subnormals, p * s_v rounded to fp16.
 template <int NCB>
@@ -191,7 +193,7 @@ struct WarpState {
 };
 template <int NCB>
 struct Mode {
-  static constexpr float kPExp = bf16_pv<NCB>() ? 64.f : 0.f;
+  static constexpr float kPExp = bf16_pv<NCB>() ? 64.f : -8.f;
 };
 
 // factor the out rows of channel tile mt carry in quant mode, relative to fp mode
@@ -858,19 +860,20 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   }
 
   // ---- fold zero term, undo position factors, reduce l over the token lanes ----
-  constexpr float kPInv = bf16_pv<NCB>() ? 0x1p-64f : 1.0f;
+  constexpr float kPInv = bf16_pv<NCB>() ? 0x1p-64f : 0x1p8f;
   float o0[8], o1[8];  // NCB == 1: rows (n, n+8) of head j; NCB == 2: unused
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) {
     const int g = (mt * 16) / G;
     // quant mode: out = true * 2^(kPExp + vpos); fp mode: out = true * 2^kPExp
-    const float f = st.quant_mode ? pow2i(-vpos_log2<NCB>(mt) - 70) * (bf16_pv<NCB>() ? 0x1p6f : 0x1p70f) : kPInv;
+    const float f = st.quant_mode ? pow2i(-vpos_log2<NCB>(mt) - 70) * (bf16_pv<NCB>() ? 0x1p6f : 0x1p78f) : kPInv;
     if (bf16_pv<NCB>()) {
       const float z = __shfl_sync(kFull, st.zacc[0] - st.zacc[1], 4 * g + j) * kPInv;
       o0[mt] = fmaf(st.out[mt][0] - st.out[mt][1], f, z);
       o1[mt] = fmaf(st.out[mt][2] - st.out[mt][3], f, z);
     } else {
-      const float z0 = __shfl_sync(kFull, st.zacc[0], 4 * g + j), z1 = __shfl_sync(kFull, st.zacc[1], 4 * g + j);
+      const float z0 = __shfl_sync(kFull, st.zacc[0], 4 * g + j) * kPInv;
+      const float z1 = __shfl_sync(kFull, st.zacc[1], 4 * g + j) * kPInv;
       st.out[mt][0] = fmaf(st.out[mt][0], f, z0);
       st.out[mt][1] = fmaf(st.out[mt][1], f, z1);
       st.out[mt][2] = fmaf(st.out[mt][2], f, z0);

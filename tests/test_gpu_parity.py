@@ -467,3 +467,29 @@ def test_padding_can_change_and_bad_padding_is_refused():
     check([N, 0])
     assert cache.kernel_status() == 0
     cache.close(); oc.close()
+
+
+@pytest.mark.parametrize("Hq,Hkv,G,W", [(8, 2, 32, 32), (14, 2, 64, 64), (12, 2, 32, 32)])
+def test_large_value_magnitudes(Hq, Hkv, G, W):
+    """Values of magnitude ~2000 (value scales of several hundred, far above what p * s_v would bear in fp16
+    without the 2^-8 on the probabilities of the path for more than 4 query heads per KV head)."""
+    B, D, N = 2, 128, W * 9 + 7
+    k, v = synth.keys_values(51, B, Hkv, N, D, "cuda")
+    v = (v.float() * 600.0).to(torch.bfloat16)
+    cache = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=N + 8)
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G)
+    cache.append(0, k, v)
+    oc.append(synth.bf16_bits(k), synth.bf16_bits(v))
+    assert_images_equal(cache.export(0), oc.export())
+    assert float(torch.from_numpy(oc.export()["v_scale"].astype(np.int32)).max()) > 0  # quantised tokens exist
+    for step in range(3):
+        q = synth.queries(51, B, Hq, D, step, "cuda")
+        out = torch.full((B, Hq, D), float("nan"), device="cuda")
+        cache.decode_attn(0, q, out)
+        torch.cuda.synchronize()
+        ref = oc.attention(synth.bf16_bits(q), 1 / np.sqrt(D))
+        got = out.cpu().numpy().astype(np.float64)
+        assert np.isfinite(got).all()
+        assert np.abs(got - ref).max() <= attn_tolerance(ref)
+    assert cache.kernel_status() == 0
+    cache.close(); oc.close()
