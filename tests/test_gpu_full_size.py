@@ -18,13 +18,15 @@ def _built():
     build.build()
 
 
-def _run(B, Hq, Hkv, W, G, ctx, seed, n_steps, n_outliers=3, planted=False, image_stride=1, bits=2):
+def _run(B, Hq, Hkv, W, G, ctx, seed, n_steps, n_outliers=3, planted=False, image_stride=1, bits=2, pad=None):
     dev = "cuda"
     total = ctx + n_steps
     outl = synth.outlier_channels(seed, Hkv, D, n_outliers) if n_outliers else None
     u = synth.unit_vectors(seed, Hkv, D) if planted else None
     cache = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=total + 8, bits=bits)
     oc = oracle.OracleCache(B, Hq, Hkv, D, W, G, bits=bits)
+    if pad is not None:
+        cache.set_padding(pad)
     chunk = 2048
     for t0 in list(range(0, ctx, chunk)) + [ctx + i for i in range(n_steps)]:
         n = min(chunk, ctx - t0) if t0 < ctx else 1
@@ -46,7 +48,10 @@ def _run(B, Hq, Hkv, W, G, ctx, seed, n_steps, n_outliers=3, planted=False, imag
         out = torch.full((B, Hq, D), float("nan"), device=dev)
         cache.decode_attn(0, q, out)
         torch.cuda.synchronize()
-        ref = oc.attention(synth.bf16_bits(q), 1 / np.sqrt(D), n_threads=16)
+        if pad is not None:
+            ref = oc.attention_subset(synth.bf16_bits(q), 1 / np.sqrt(D), pad=pad)
+        else:
+            ref = oc.attention(synth.bf16_bits(q), 1 / np.sqrt(D), n_threads=16)
         got = out.cpu().numpy().astype(np.float64)
         err, tol = float(np.abs(got - ref).max()), attn_tolerance(ref)
         assert np.isfinite(got).all() and err <= tol, f"step {step}: max|delta| {err:.3e} > {tol:.3e}"
@@ -81,3 +86,17 @@ def test_config2_with_four_bit_codes():
     # the llama3-8b-8k-int4 workload of bench.py: config 2 at the paper's second precision
     inf = _run(B=8, Hq=32, Hkv=8, W=128, G=32, ctx=8192, seed=2, n_steps=2, bits=4)
     assert inf.bytes_quant_per_token == 160
+
+
+def test_config2_left_padded_batch():
+    # config 2 as a ragged batch: prompts of 8192, 8191, 8000, 7169, 4096, 2049, 300 and 2 real tokens,
+    # left-padded to 8192 positions
+    pad = [0, 1, 192, 1023, 4096, 6143, 7892, 8190]
+    inf = _run(B=8, Hq=32, Hkv=8, W=128, G=32, ctx=8192, seed=6, n_steps=2, pad=pad)
+    assert (inf.n_quant, inf.n_fp) == (7936, 258)
+
+
+def test_config4_left_padded_batch():
+    inf = _run(B=4, Hq=28, Hkv=4, W=256, G=64, ctx=32768, seed=7, n_steps=1, n_outliers=0, planted=True,
+               pad=[0, 31, 16385, 32700])
+    assert (inf.n_quant, inf.n_fp) == (32256, 513)
