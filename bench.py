@@ -32,6 +32,12 @@ from paper_2503_19950_b200 import synth  # noqa: E402
 WORKLOADS = {
     # BASELINE config 2: Llama-3-8B layer shape, batch 8, context 8192, W=128, G=32, 32 stacked layers
     "llama3-8b-8k": dict(L=32, B=8, Hq=32, Hkv=8, W=128, G=32, ctx=8192, n_outliers=3, seed=2),
+    # config 2 in the paper's own setting (Sec. 3.1): group 64, reserved length 128 tokens, i.e. W = 42 (not a
+    # multiple of G: removed tokens wait at full precision until 64 of them form a key group)
+    "llama3-8b-8k-w42": dict(L=32, B=8, Hq=32, Hkv=8, W=42, G=64, ctx=8192, n_outliers=3, seed=2),
+    # config 2 as a ragged batch: prompts of 8192, 7168, ..., 1024 tokens, left-padded to 8192 positions
+    "llama3-8b-8k-ragged": dict(L=32, B=8, Hq=32, Hkv=8, W=128, G=32, ctx=8192, n_outliers=3, seed=2,
+                                pad=[0, 1024, 2048, 3072, 4096, 5120, 6144, 7168]),
     # config 2 with the paper's second precision (4-bit codes, 160 B per token)
     "llama3-8b-8k-int4": dict(L=32, B=8, Hq=32, Hkv=8, W=128, G=32, ctx=8192, n_outliers=3, seed=2, bits=4),
     # config 4: long-context GQA-7
@@ -166,6 +172,10 @@ def run_ours(args, wl, rank, world, device):
     bits = wl.get("bits", 2)
     cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=ctx + total_steps + 8, device=device.index or 0, bits=bits,
                           n_splits=args.n_splits)
+    pad = wl.get("pad")
+    n_pad = sum(pad) if pad else 0
+    if pad:
+        cache.set_padding(pad)
     prefill(cache, wl, device)
     ks, vs, qs = make_step_inputs(wl, device, Q_ROTATE)
     outs = [torch.empty(B, Hq, D, device=device) for _ in range(L)]
@@ -190,7 +200,7 @@ def run_ours(args, wl, rank, world, device):
         for i in range(n):
             fn(start_idx + i)
             inf = cache.info_fast()
-            kv_tokens += B * (inf[0] + inf[1]) * L
+            kv_tokens += (B * (inf[0] + inf[1]) - n_pad) * L
         ev1.record()
         barrier()
         return ev0.elapsed_time(ev1), kv_tokens
@@ -224,6 +234,13 @@ def run_ours(args, wl, rank, world, device):
     b2b_us = round_us[len(round_us) // 2] / L
     b2b_best_us = round_us[0] / L
     bytes_b2b = sum(cache.info(l).bytes_decode_step for l in range(L)) / L
+    if pad:
+        # algorithmic bytes of a padded batch: the stored bytes of the tokens that are not padding
+        img, inf0 = cache.export(0), cache.info(0)
+        real_q = sum(int((img["quant_ids"] >= pb).sum()) for pb in pad)
+        real_f = sum(int((img["kept_ids"] >= pb).sum()) for pb in pad)
+        bytes_b2b = Hkv * (real_q * inf0.bytes_quant_per_token + real_f * 4 * D)
+        del img
     cache.profile_enable(True)
     byte_sum = 0
     for i in range(min(steps, 8192 // L)):
@@ -259,7 +276,7 @@ def run_ours(args, wl, rank, world, device):
     for i in range(e2e_steps):
         host_step(step_idx + i)
         inf = cache.info_fast()
-        kv_e2e += B * (inf[0] + inf[1]) * L
+        kv_e2e += (B * (inf[0] + inf[1]) - n_pad) * L
     barrier()
     e2e_s = time.perf_counter() - t0
     # ---- one window-overflow event over all layers at once (lq_compress(layer=-1)) ----
@@ -305,7 +322,7 @@ def run_ours(args, wl, rank, world, device):
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": args.workload, "layers": L, "batch": B, "q_heads": Hq, "kv_heads": Hkv,
                    "head_dim": D, "context": ctx, "window": W, "group": G, "bits": bits,
-                   "n_quant": int(inf.n_quant), "n_fp": int(inf.n_fp), "n_splits": int(inf.n_splits), "n_ctas": int(inf.n_ctas),
+                   "padding": pad, "n_quant": int(inf.n_quant), "n_fp": int(inf.n_fp), "n_splits": int(inf.n_splits), "n_ctas": int(inf.n_ctas),
                    "step": "per layer: lq_append_decode_attn (append and attention in one launch; the overflow step and "
                            "a separate append when the window is full)",
                    "l2": "inputs larger than L2: %.2f GB of cache touched per step" % (bytes_step_last / 1e9),
@@ -364,11 +381,14 @@ def oracle_layer_step(wl, device, n_threads, min_seconds, max_reps, warmup=0):
         q = synth.bf16_bits(synth.queries(wl["seed"], B, Hq, D, s, device, layer=0))
         t0 = time.perf_counter()
         oc.append(np.ascontiguousarray(kb[:, :, s:s + 1]), np.ascontiguousarray(vb[:, :, s:s + 1]))
-        oc.attention(q, 1.0 / np.sqrt(D), n_threads=n_threads)
+        if wl.get("pad"):
+            oc.attention_subset(q, 1.0 / np.sqrt(D), pad=wl["pad"])  # (single-threaded in the oracle)
+        else:
+            oc.attention(q, 1.0 / np.sqrt(D), n_threads=n_threads)
         dt = time.perf_counter() - t0
         times.append(dt)
         t_total += dt
-        kv += B * (oc.n_quant + oc.n_fp)
+        kv += B * (oc.n_quant + oc.n_fp) - sum(wl.get("pad") or [])
         reps += 1
     return kv / t_total, reps, t_total, times
 

@@ -60,9 +60,10 @@ struct lq_cache {
   bool has_pad = false;
   std::vector<char> mask_dirty;
   uint32_t* masks = nullptr;
-  int fp_words = 0, q_words = 0;
+  int fp_words = 0, q_words = 0, map_words = 0;
   int64_t mask_layer_words = 0;
   std::vector<uint32_t> mask_host;
+  std::vector<int> pad_grid, pad_stride;  // per layer: CTAs and record stride of the padded tensor-core launch
   // optional timing of the split-K attention kernel
   bool profiling = false;
   std::vector<cudaEvent_t> ev_pool;  // 2 events per timed launch
@@ -205,37 +206,53 @@ void plan_group_residual(const lq_cache* c, LayerState& L, EvictList* ev, int32_
   L.n_quant += G;
 }
 
-// one overflow of one layer when W is not a multiple of G (host state and launches)
-lq_status_t run_event_residual(lq_cache* c, int layer, cudaStream_t st) {
-  LayerState& L = c->layers[layer];
-  apply_event_residual(c, L);
-  while (static_cast<int>(L.pend_slot.size()) >= c->cfg.group) {
+// overflow of the given layers when W is not a multiple of G (host state and launches): the removed tokens
+// join the waiting lists; then, while some layer has G tokens waiting, its G oldest form a key group.  Layers
+// whose group comes from the same rows and goes to the same place (layers in lockstep) share one launch.
+lq_status_t run_events_residual(lq_cache* c, const std::vector<int>& full_layers, cudaStream_t st) {
+  for (int layer : full_layers) apply_event_residual(c, c->layers[layer]);
+  struct Plan {
     EvictList ev;
-    std::memset(&ev, 0, sizeof ev);
-    const int64_t tile0 = L.n_quant / c->cfg.group;
-    plan_group_residual(c, L, &ev, nullptr);
-    if (!c->dry) {
+    int64_t tile0;
+    int layer;
+  };
+  for (;;) {
+    std::vector<Plan> plans;
+    for (int layer : full_layers) {
+      LayerState& L = c->layers[layer];
+      if (static_cast<int>(L.pend_slot.size()) < c->cfg.group) continue;
+      plans.emplace_back();
+      Plan& p = plans.back();
+      std::memset(&p.ev, 0, sizeof p.ev);
+      p.tile0 = L.n_quant / c->cfg.group;
+      p.layer = layer;
+      plan_group_residual(c, L, &p.ev, nullptr);
+    }
+    if (plans.empty()) return LQ_OK;
+    std::vector<char> done(plans.size(), 0);
+    for (size_t i = 0; i < plans.size(); ++i) {
+      if (done[i]) continue;
       LayerList ll;
-      ll.n = 1;
-      ll.layer[0] = static_cast<uint8_t>(layer);
-      cudaError_t e = launch_compress(c->cv, ll, ev, tile0, 1, st);
-      if (e != cudaSuccess) return cuda_fail(c, e, "lq_compress_kernel");
-      c->n_launches++;
+      ll.n = 0;
+      for (size_t k = i; k < plans.size() && ll.n < 128; ++k) {
+        if (done[k] || plans[k].tile0 != plans[i].tile0 || std::memcmp(&plans[k].ev, &plans[i].ev, sizeof(EvictList)) != 0)
+          continue;
+        ll.layer[ll.n++] = static_cast<uint8_t>(plans[k].layer);
+        done[k] = 1;
+      }
+      if (!c->dry) {
+        cudaError_t e = launch_compress(c->cv, ll, plans[i].ev, plans[i].tile0, 1, st);
+        if (e != cudaSuccess) return cuda_fail(c, e, "lq_compress_kernel");
+        c->n_launches++;
+      }
     }
   }
-  return LQ_OK;
 }
 
 lq_status_t run_events(lq_cache* c, const std::vector<int>& full_layers, cudaStream_t st) {
   if (!c->mask_dirty.empty())
     for (int layer : full_layers) c->mask_dirty[layer] = 1;
-  if (residual_mode(c)) {
-    for (int layer : full_layers) {
-      lq_status_t s = run_event_residual(c, layer, st);
-      if (s != LQ_OK) return s;
-    }
-    return LQ_OK;
-  }
+  if (residual_mode(c)) return run_events_residual(c, full_layers, st);
   // group layers whose removal lists coincide into one launch
   std::vector<char> done(full_layers.size(), 0);
   for (size_t i = 0; i < full_layers.size(); ++i) {
@@ -270,6 +287,8 @@ lq_status_t run_events(lq_cache* c, const std::vector<int>& full_layers, cudaStr
   }
   return LQ_OK;
 }
+
+bool use_mma(const lq_cache* c) { return c->cfg.kernel != LQ_KERNEL_SCALAR; }
 
 // Padding masks of one layer from the host mirror of its stores (which token id sits in which fp slot and at
 // which place of the quantised store) and upload.  Rows appended later lie beyond the rebuilt prefix of the fp
@@ -309,6 +328,17 @@ lq_status_t upload_masks(lq_cache* c, int layer, cudaStream_t st) {
     rowinfo[4 * b + 1] = static_cast<int32_t>(last);
     rowinfo[4 * b + 2] = any_fp ? 1 : 0;
   }
+  if (use_mma(c)) {
+    // the CTAs of the tensor-core launch, shared out by the work each sequence has left
+    int32_t* pair_ctas = reinterpret_cast<int32_t*>(qm + static_cast<size_t>(c->q_words) * B);
+    int32_t* cta_map = pair_ctas + B * c->cfg.n_kv_heads;
+    DecodeArgs a;
+    a.cv = c->cv;
+    a.n_fp = L.n_fp;
+    a.n_quant = L.n_quant;
+    c->pad_grid[layer] = plan_decode_mma_padded(a, c->sm_count, c->max_splits, rowinfo, cta_map, pair_ctas,
+                                                &c->pad_stride[layer]);
+  }
   // pageable source: staged by the runtime before the call returns
   cudaError_t e = cudaMemcpyAsync(c->masks + layer * c->mask_layer_words, c->mask_host.data(),
                                   c->mask_host.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, st);
@@ -327,7 +357,6 @@ int choose_splits(const lq_cache* c, const LayerState& L) {
   return static_cast<int>(s);
 }
 
-bool use_mma(const lq_cache* c) { return c->cfg.kernel != LQ_KERNEL_SCALAR; }
 
 }  // namespace
 
@@ -568,17 +597,21 @@ lq_status_t lq_set_padding(lq_cache_t* c, const int32_t* pad_host) {
   const int B = c->cfg.batch;
   for (int b = 0; b < B; ++b)
     if (pad_host[b] < 0) return LQ_ERR_INVALID_ARG;
+  if (B * c->cfg.n_kv_heads > 0xFFFF) return LQ_ERR_UNSUPPORTED;  // the CTA map packs the pair into 16 bits
   if (!c->dry && !c->masks) {
     const int slots = 3 * c->cfg.window + c->cfg.group;
     c->fp_words = (slots + 31) / 32;
     c->q_words = static_cast<int>((c->cfg.max_tokens + 31) / 32);
-    c->mask_layer_words = static_cast<int64_t>(B) * (4 + c->fp_words + c->q_words);
+    c->map_words = std::max(max_ctas_decode_mma(c->sm_count), B * c->cfg.n_kv_heads);  // at least one CTA per pair
+    c->mask_layer_words = static_cast<int64_t>(B) * (4 + c->fp_words + c->q_words) + B * c->cfg.n_kv_heads + c->map_words;
     if (!dev_alloc(c, reinterpret_cast<void**>(&c->masks), c->mask_layer_words * c->cfg.n_layers * 4)) return LQ_ERR_OOM;
   }
   c->pad.assign(pad_host, pad_host + B);
   c->has_pad = false;
   for (int b = 0; b < B; ++b) c->has_pad |= pad_host[b] > 0;
   c->mask_dirty.assign(c->cfg.n_layers, 1);
+  c->pad_grid.assign(c->cfg.n_layers, 0);
+  c->pad_stride.assign(c->cfg.n_layers, 1);
   return LQ_OK;
 }
 
@@ -637,6 +670,8 @@ lq_status_t decode_impl(lq_cache_t* c, int32_t layer, const void* q, float sm_sc
   a.rowinfo = nullptr;
   a.qmask = a.fpmask = nullptr;
   a.qmask_words = a.fpmask_words = 0;
+  a.cta_map = a.pair_ctas = nullptr;
+  a.n_ctas = 0;
   if (c->has_pad) {
     // every sequence keeps at least its newest token
     for (int b = 0; b < c->cfg.batch; ++b)
@@ -651,6 +686,8 @@ lq_status_t decode_impl(lq_cache_t* c, int32_t layer, const void* q, float sm_sc
     a.qmask = a.fpmask + static_cast<int64_t>(c->fp_words) * c->cfg.batch;
     a.fpmask_words = c->fp_words;
     a.qmask_words = c->q_words;
+    a.pair_ctas = reinterpret_cast<const int32_t*>(a.qmask + static_cast<int64_t>(c->q_words) * c->cfg.batch);
+    a.cta_map = a.pair_ctas + c->cfg.batch * c->cfg.n_kv_heads;
   }
   if (!(sm_scale > 0.f)) sm_scale = 1.0f / std::sqrt(static_cast<float>(kD));
   a.scale_log2 = sm_scale * 1.4426950408889634f;
@@ -672,6 +709,11 @@ lq_status_t decode_impl(lq_cache_t* c, int32_t layer, const void* q, float sm_sc
   a.n_extra = 0;
   if (use_mma(c)) {
     plan_decode_mma(a, c->sm_count, c->max_splits, c->cfg.n_splits);
+    if (a.rowinfo) {
+      a.S = c->pad_stride[layer];
+      a.n_ctas = c->pad_grid[layer];
+      a.n_extra = 0;
+    }
     a.tickets = c->tickets;  // the CTA that completes a (b, kv) pair merges it: no second launch
     e = launch_decode_mma(a, st);
     if (e != cudaSuccess) return cuda_fail(c, e, "lq_decode_mma_kernel");

@@ -29,6 +29,10 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <algorithm>
+#include <utility>
+#include <vector>
+
 #include "lq_kernels.cuh"
 
 namespace lq {
@@ -635,7 +639,13 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   // is also the record stride).  Interleaving gives every pair CTAs from every launch rank of the
   // SMs, so no pair consists only of CTAs whose first loads queue behind everybody else's.
   int pair, slot, n_ctas_pair;
-  {
+  if (PADDED) {
+    // sequences of a padded batch have different amounts of work: the host shared the CTAs out accordingly
+    const int e = a.cta_map[blockIdx.x];
+    pair = e & 0xFFFF;
+    slot = e >> 16;
+    n_ctas_pair = a.pair_ctas[pair];
+  } else {
     const int P = cv.B * cv.Hkv;
     pair = blockIdx.x % P;
     slot = blockIdx.x / P;
@@ -673,9 +683,6 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   const uint32_t qbar = smem_u32(smem + kSmemStages + kSmemQ) + kWarps * kMaxStages * 8;
   int* is_last = reinterpret_cast<int*>(smem + kSmemStages + kSmemQ + kSmemBars);
 
-  // Programmatic dependent launch: do not touch anything an earlier kernel may still be writing
-  // before it has finished (the matching launch_dependents comes after the main loop).
-  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (lane == 0) {
 #pragma unroll
     for (int s = 0; s < kStages; ++s) mbar_init(bar0 + 8 * s, 1);
@@ -684,6 +691,10 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
+  // Programmatic dependent launch: everything above touches only this CTA's shared memory and the
+  // launch arguments; nothing an earlier kernel may still be writing is read before it has finished
+  // (the matching launch_dependents comes after the main loop).
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (threadIdx.x == 0) {
     // the r query rows of this pair are contiguous: one bulk copy
     mbar_expect_tx(qbar, r * kD * 2);
@@ -1099,6 +1110,68 @@ void plan_decode_mma(DecodeArgs& a, int sm_count, int max_records, int s_overrid
   a.S = S + 1;  // record stride; pairs >= n_extra use S of them
 }
 
+int max_ctas_decode_mma(int sm_count) { return kCtasPerSm * sm_count; }
+
+int plan_decode_mma_padded(const DecodeArgs& a, int sm_count, int max_records, const int32_t* rowinfo_host,
+                           int32_t* cta_map, int32_t* pair_ctas, int* stride) {
+  const int pairs = a.cv.B * a.cv.Hkv;
+  const int r = a.cv.Hq / a.cv.Hkv;
+  const int tiles_fp = (a.n_fp + kFpTileSlots - 1) / kFpTileSlots;
+  const int tiles_quant = static_cast<int>(a.n_quant / a.cv.G);
+  const int tps = stage_bytes(a.cv.G) / quant_tile_bytes(a.cv.G, a.cv.planes);
+  const int wave = (r <= 4 ? kCtasPerSm : kCtasPerSm - 1) * sm_count;
+  const int cap_records = std::max(1, std::min(max_records, kMergeMax / r));
+  std::vector<int64_t> work(pairs);
+  std::vector<int> cap(pairs);
+  int64_t total = 0;
+  for (int p = 0; p < pairs; ++p) {
+    const int tq = std::max(0, tiles_quant - rowinfo_host[4 * (p / a.cv.Hkv) + 0]);
+    work[p] = static_cast<int64_t>(tiles_fp) * kFpCost8 + 8LL * tq;  // the kernel's cost line
+    const int items = tiles_fp + tq / tps;
+    cap[p] = std::max(1, std::min(cap_records, items / kWarps));  // at least one item per warp
+    total += work[p];
+  }
+  // largest-remainder shares of one wave, clipped to the caps
+  int given = 0;
+  std::vector<std::pair<int64_t, int>> rest(pairs);
+  for (int p = 0; p < pairs; ++p) {
+    const int64_t share = total > 0 ? work[p] * wave / total : 0;
+    pair_ctas[p] = static_cast<int32_t>(std::max<int64_t>(1, std::min<int64_t>(share, cap[p])));
+    rest[p] = {total > 0 ? work[p] * wave % total : 0, p};
+    given += pair_ctas[p];
+  }
+  std::sort(rest.begin(), rest.end(), [](const std::pair<int64_t, int>& x, const std::pair<int64_t, int>& y) {
+    return x.first != y.first ? x.first > y.first : x.second < y.second;
+  });
+  for (bool progress = true; given < wave && progress;) {
+    progress = false;
+    for (int i = 0; i < pairs && given < wave; ++i) {
+      const int p = rest[i].second;
+      if (pair_ctas[p] < cap[p]) {
+        ++pair_ctas[p];
+        ++given;
+        progress = true;
+      }
+    }
+  }
+  while (given > wave) {  // the minimum of one CTA per pair overshot the wave: take from the largest
+    int big = 0;
+    for (int p = 1; p < pairs; ++p)
+      if (pair_ctas[p] > pair_ctas[big]) big = p;
+    if (pair_ctas[big] <= 1) break;
+    --pair_ctas[big];
+    --given;
+  }
+  // slot-major order: every pair gets CTAs of every launch rank of the SMs
+  int n = 0, most = 1;
+  for (int p = 0; p < pairs; ++p) most = std::max(most, static_cast<int>(pair_ctas[p]));
+  for (int slot = 0; slot < most; ++slot)
+    for (int p = 0; p < pairs; ++p)
+      if (slot < pair_ctas[p]) cta_map[n++] = p | (slot << 16);
+  *stride = most;
+  return n;
+}
+
 cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
   const int r = a.cv.Hq / a.cv.Hkv;
   void (*kern)(DecodeArgs) = nullptr;
@@ -1132,7 +1205,7 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
     if (dev >= 0 && dev < 64) configured[dev][variant] = true;
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(a.cv.B * a.cv.Hkv * (a.S - 1) + a.n_extra);
+  cfg.gridDim = dim3(padded ? a.n_ctas : a.cv.B * a.cv.Hkv * (a.S - 1) + a.n_extra);
   cfg.blockDim = dim3(kWarps * 32);
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = st;

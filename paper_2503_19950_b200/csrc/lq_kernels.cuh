@@ -86,10 +86,15 @@ struct DecodeArgs {
   //   rowinfo[4*b + 1] = first quant tile from which on no token is padding (tiles in between consult qmask),
   //   rowinfo[4*b + 2] = 1 if some slot of the fp store is padding (fpmask is consulted);
   //   qmask[b*qmask_words + i/32] bit i%32: token i of the quantised store, fpmask likewise per fp slot.
+  //   Tensor-core kernel: the CTAs of a padded launch are shared out by the work each sequence has left:
+  //   cta_map[c] = pair | slot << 16 for CTA c (n_ctas of them), pair_ctas[pair] = CTAs of that pair (<= S).
   const int32_t* rowinfo;
   const uint32_t* qmask;
   const uint32_t* fpmask;
   int qmask_words, fpmask_words;
+  const int32_t* cta_map;
+  const int32_t* pair_ctas;
+  int n_ctas;
   int* status;  // device word; kernels OR error bits into it (bounded waits that gave up)
   int* tickets; // one 128-byte line per (b, kv): word [1] is the arrival counter of the fused second
                 // pass, 0 at rest
@@ -99,6 +104,13 @@ struct DecodeArgs {
 cudaError_t launch_decode_scalar(const DecodeArgs& a, cudaStream_t st);
 // Fills S and the tile counts of `a` for the tensor-core kernel (S <= max_records; s_override > 0 forces S).
 void plan_decode_mma(DecodeArgs& a, int sm_count, int max_records, int s_override);
+// Padded batch: shares one resident wave of CTAs out over the (b, kv) pairs in proportion to the tiles each
+// sequence still has to visit (rowinfo as in DecodeArgs, on the host).  Fills cta_map (room for
+// max_ctas_decode_mma(sm_count) entries) and pair_ctas (B * Hkv entries); returns the grid size and sets
+// *stride to the record stride (the largest CTA count of a pair, <= max_records).
+int max_ctas_decode_mma(int sm_count);
+int plan_decode_mma_padded(const DecodeArgs& a, int sm_count, int max_records, const int32_t* rowinfo_host,
+                           int32_t* cta_map, int32_t* pair_ctas, int* stride);
 cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st);
 cudaError_t launch_merge(const DecodeArgs& a, cudaStream_t st);
 

@@ -405,6 +405,8 @@ def test_argument_errors_on_device():
     (2, 8, 8, 32, 32, 4, 32 * 8 + 17, 20, None, [64, 201]), # r = 1, 4-bit codes
     (2, 8, 2, 42, 64, 2, 42 * 9 + 5, 50, None, [11, 260]),  # W not a multiple of G: waiting tokens may be padding
     (1, 4, 1, 32, 32, 2, 40, 70, None, [39]),               # padding still in the window; crosses the first overflow
+    (80, 8, 8, 32, 32, 2, 150, 3, None, [(7 * i) % 120 for i in range(80)]),  # more (b, kv) pairs than one wave of CTAs
+    (2, 8, 1, 32, 32, 2, 3000, 3, None, [0, 2900]),         # very unequal work: the CTAs go where the tokens are
 ])
 def test_left_padded_batch(kernel, B, Hq, Hkv, W, G, bits, n_prefill, n_steps, chunk, pad):
     """Sequence b attends to tokens pad[b].. only; the stores are those of the unpadded run (same image)."""
@@ -441,7 +443,8 @@ def test_padding_can_change_and_bad_padding_is_refused():
     plain = check(None)
     cache.set_padding([100, 0])
     padded = check([100, 0])
-    assert not torch.equal(padded[0], plain[0]) and torch.equal(padded[1], plain[1])
+    # (sequence 1 is untouched up to summation order: the padded launch shares its CTAs out differently)
+    assert not torch.allclose(padded[0], plain[0], atol=1e-3) and torch.allclose(padded[1], plain[1], atol=1e-3)
     cache.set_padding([0, 399])  # sequence 1 keeps its newest token only: the output is that token's value row
     one = check([0, 399])
     assert torch.allclose(one[1, 0], v[1, 0, 399].float(), atol=1e-5)
