@@ -630,9 +630,9 @@ lq_status_t lq_append_decode_attn(lq_cache_t* c, int32_t layer, const void* k, c
   const int64_t step_bytes = static_cast<int64_t>(c->cfg.batch) * c->cfg.n_kv_heads *
                              (L.n_quant * (quant_tile_bytes(c->cfg.group, c->cfg.bits / 2) / c->cfg.group) +
                               static_cast<int64_t>(L.n_fp) * 4 * kD);
-  if (kept(L) == 3 * W || !use_mma(c) || step_bytes > (192LL << 20) || c->has_pad) {
+  if (kept(L) == 3 * W || !use_mma(c) || step_bytes > (192LL << 20)) {
     // the window is full (the overflow step has to run between the two), the plain kernel is
-    // selected, the launch is long, or the batch is padded: the two separate calls
+    // selected, or the launch is long: the two separate calls
     lq_status_t s = lq_append(c, layer, k, v, 1, stream);
     if (s != LQ_OK) return s;
     return lq_decode_attn(c, layer, q, sm_scale, out, out_dtype, stream);

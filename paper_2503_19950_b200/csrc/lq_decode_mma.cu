@@ -1177,19 +1177,16 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
   void (*kern)(DecodeArgs) = nullptr;
   const bool fused = a.new_k != nullptr;
   const bool padded = a.rowinfo != nullptr;
-  if (fused && padded) return cudaErrorInvalidValue;  // the caller appends separately for a padded batch
-#define LQ_PICK(G_, P_)                                                                                       \
-  kern = r <= 4 ? (fused    ? lq_decode_mma_kernel<G_, 1, P_, true, false>                                    \
-                   : padded ? lq_decode_mma_kernel<G_, 1, P_, false, true>                                    \
-                            : lq_decode_mma_kernel<G_, 1, P_, false, false>)                                  \
-                : (fused    ? lq_decode_mma_kernel<G_, 2, P_, true, false>                                    \
-                   : padded ? lq_decode_mma_kernel<G_, 2, P_, false, true>                                    \
-                            : lq_decode_mma_kernel<G_, 2, P_, false, false>)
+#define LQ_PICK2(G_, N_, P_)                                                                      \
+  (fused ? (padded ? lq_decode_mma_kernel<G_, N_, P_, true, true> : lq_decode_mma_kernel<G_, N_, P_, true, false>) \
+         : (padded ? lq_decode_mma_kernel<G_, N_, P_, false, true> : lq_decode_mma_kernel<G_, N_, P_, false, false>))
+#define LQ_PICK(G_, P_) kern = r <= 4 ? LQ_PICK2(G_, 1, P_) : LQ_PICK2(G_, 2, P_)
   if (a.cv.G == 32 && a.cv.planes == 1) LQ_PICK(32, 1);
   else if (a.cv.G == 32 && a.cv.planes == 2) LQ_PICK(32, 2);
   else if (a.cv.G == 64 && a.cv.planes == 1) LQ_PICK(64, 1);
   else return cudaErrorInvalidValue;
 #undef LQ_PICK
+#undef LQ_PICK2
   static_assert(kSmemStages >= static_cast<int>((kWarps * 8 * (kD + 4) + 3 * kWarps * 8 + 16) * sizeof(float)) &&
                     kSmemStages >= (kMergeMax + kWarps * kMaxRatio * kD) * 4,
                 "merge scratch");

@@ -298,13 +298,15 @@ def test_prompt_ingestion_in_one_launch_equals_token_by_token(W, G, n):
     one.close(); seq.close(); oc.close()
 
 
-@pytest.mark.parametrize("B,Hq,Hkv,W,G,bits,n0", [
-    (2, 8, 2, 32, 32, 2, 3 * 32 - 5),     # crosses an overflow step (falls back to the two calls there)
-    (1, 14, 2, 64, 64, 2, 64 * 5 + 15),   # GQA-7; the new row opens a new 16-slot tile on the way
-    (2, 8, 8, 32, 32, 4, 32 * 7 + 1),     # r = 1, 4-bit codes
-    (2, 8, 2, 42, 64, 2, 42 * 5 + 11),    # W not a multiple of G: waiting tokens in the fp store
+@pytest.mark.parametrize("B,Hq,Hkv,W,G,bits,n0,pad", [
+    (2, 8, 2, 32, 32, 2, 3 * 32 - 5, None),     # crosses an overflow step (falls back to the two calls there)
+    (1, 14, 2, 64, 64, 2, 64 * 5 + 15, None),   # GQA-7; the new row opens a new 16-slot tile on the way
+    (2, 8, 8, 32, 32, 4, 32 * 7 + 1, None),     # r = 1, 4-bit codes
+    (2, 8, 2, 42, 64, 2, 42 * 5 + 11, None),    # W not a multiple of G: waiting tokens in the fp store
+    (3, 8, 2, 32, 32, 2, 32 * 6 + 20, [150, 0, 33]),   # left-padded batch
+    (2, 14, 2, 64, 64, 2, 64 * 4 + 60, [7, 200]),      # left-padded, GQA-7, crosses an overflow step
 ])
-def test_append_and_attention_in_one_launch(B, Hq, Hkv, W, G, bits, n0):
+def test_append_and_attention_in_one_launch(B, Hq, Hkv, W, G, bits, n0, pad):
     """lq_append_decode_attn: same image, same attention bits as lq_append + lq_decode_attn, one launch."""
     D, n_steps = 128, 20
     k, v = synth.keys_values(23, B, Hkv, n0 + n_steps, D, "cuda")
@@ -313,6 +315,8 @@ def test_append_and_attention_in_one_launch(B, Hq, Hkv, W, G, bits, n0):
     oc = oracle.OracleCache(B, Hq, Hkv, D, W, G, bits=bits)
     for c in (fused, plain):
         c.append(0, k[:, :, :n0].contiguous(), v[:, :, :n0].contiguous())
+        if pad is not None:
+            c.set_padding(pad)
     oc.append(synth.bf16_bits(k[:, :, :n0]), synth.bf16_bits(v[:, :, :n0]))
     single = 0
     for t in range(n_steps):
@@ -328,7 +332,7 @@ def test_append_and_attention_in_one_launch(B, Hq, Hkv, W, G, bits, n0):
         torch.cuda.synchronize()
         assert torch.equal(o1, o2), f"step {t}"
         oc.append(synth.bf16_bits(k1), synth.bf16_bits(v1))
-        ref = oc.attention(synth.bf16_bits(q), 1 / np.sqrt(D))
+        ref = oc.attention_subset(synth.bf16_bits(q), 1 / np.sqrt(D), pad=pad)
         assert np.abs(o1.cpu().numpy() - ref).max() <= attn_tolerance(ref)
         if t % 6 == 0 or t == n_steps - 1:
             assert_images_equal(fused.export(0), oc.export())
