@@ -71,6 +71,13 @@ def test_config3_batch16_4k():
     assert (inf.n_quant, inf.n_fp) == (3840, 257)
 
 
+@pytest.mark.parametrize("B", [32, 64])
+def test_config3_larger_batches_4k(B):
+    # 256 and 512 (b, kv) pairs: one to three CTAs per pair, and at batch 64 a step of two launches
+    inf = _run(B=B, Hq=32, Hkv=8, W=128, G=32, ctx=4096, seed=3, n_steps=1, image_stride=1)
+    assert (inf.n_quant, inf.n_fp) == (3840, 257)
+
+
 def test_config4_gqa7_32k_planted_spikes():
     # 28 q / 4 kv heads, W=256, G=64, keys with planted high-logit tokens at log-spaced distances
     inf = _run(B=4, Hq=28, Hkv=4, W=256, G=64, ctx=32768, seed=4, n_steps=1, n_outliers=0, planted=True)
