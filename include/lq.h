@@ -102,7 +102,7 @@ typedef struct {
 
 /*
  * Canonical image of one layer (host buffers supplied by the caller; a null member is skipped).
- * Sizes use n_fp, n_quant from lq_cache_info.  This is the format parity is judged on; the
+ * Sizes use n_fp, n_quant from lq_cache_info.  This is the format parity is checked on; the
  * device-side layout is private.
  *   kept_ids  [n_fp]    int32, ascending: ids (append order, from 0) of the full-precision tokens
  *   quant_ids [n_quant] int32, in store order: event order, then age order inside an event
