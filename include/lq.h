@@ -178,7 +178,9 @@ lq_status_t lq_decode_attn_fp_only(lq_cache_t* cache, int32_t layer, const void*
  * call gives LQ_ERR_INVALID_ARG while some sequence has pad[b] >= the tokens appended to that layer.
  * The masks (about max_tokens / 8 bytes per sequence and layer) are allocated by the first call
  * (LQ_ERR_OOM if that fails) and re-derived on the host and uploaded on the decode call's stream after every
- * overflow step or prompt ingestion of a layer.  lq_decode_attn_image_static knows no padding. */
+ * overflow step or prompt ingestion of a layer.  The tensor-core kernel shares its CTAs out over the
+ * sequences in proportion to the tokens each has left (config n_splits then only caps the share of one
+ * (batch row, KV head)).  lq_decode_attn_image_static knows no padding. */
 lq_status_t lq_set_padding(lq_cache_t* cache, const int32_t* pad);
 
 /* lq_append of ONE token followed by lq_decode_attn, in one launch: the attention kernel takes the
