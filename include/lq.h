@@ -157,7 +157,9 @@ lq_status_t lq_compress(lq_cache_t* cache, int32_t layer, void* stream);
 /* One-token decode attention over the whole mixed cache of one layer (Eq. 2; order of the two
  * stores and of the split-K partitions is free by Eq. 3).  q: device bf16 [B, Hq, D];
  * sm_scale <= 0 selects 1/sqrt(D); out: device [B, Hq, D], out_dtype 0 = fp32, 1 = bf16.
- * Accumulation is fp32.  An empty cache gives LQ_ERR_INVALID_ARG.  Range: any finite bf16 keys, queries
+ * Accumulation is fp32.  The result is reproducible bit for bit from call to call, except when more than
+ * 12 CTAs share one (batch row, KV head) -- long contexts with few such pairs --, where the partial results
+ * are summed in arrival order.  An empty cache gives LQ_ERR_INVALID_ARG.  Range: any finite bf16 keys, queries
  * and values with up to 4 query heads per KV head; with 5 to 8 the quantised values pass through fp16
  * operands, so value zero-points and scales must lie within fp16 range (|v| < 65504). */
 lq_status_t lq_decode_attn(lq_cache_t* cache, int32_t layer, const void* q, float sm_scale,

@@ -47,6 +47,7 @@ struct lq_cache {
   int* status = nullptr;
   int* ingest_idx = nullptr;  // index list of the one-launch prompt ingestion (max_tokens ints)
   int* tickets = nullptr;  // per (b, kv) arrival counters of the fused split-K merge
+  float* acc = nullptr;    // per (b, kv) sums of the partials added on arrival (DecodeArgs::acc)
   // staging for the host-buffer entry point, one slice per layer
   uint8_t* stage_k = nullptr;
   uint8_t* stage_v = nullptr;
@@ -98,6 +99,7 @@ void free_all(lq_cache* c) {
     cudaFree(c->part_ml);
     cudaFree(c->status);
     cudaFree(c->tickets);
+    cudaFree(c->acc);
     cudaFree(c->ingest_idx);
     cudaFree(c->stage_k);
     cudaFree(c->stage_v);
@@ -428,6 +430,7 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
               dev_alloc(c, reinterpret_cast<void**>(&c->part_ml), pairs * c->max_splits * r * 2 * 4) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->status), 256) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->tickets), pairs * 128) &&
+              dev_alloc(c, reinterpret_cast<void**>(&c->acc), static_cast<int64_t>(pairs) * kAccStride * 4) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->ingest_idx), (cfg->max_tokens + 3 * cfg->window + cfg->group) * 4) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_k), cfg->n_layers * pairs * kD * 2) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_v), cfg->n_layers * pairs * kD * 2) &&
@@ -437,6 +440,7 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
                         static_cast<int64_t>(cfg->n_layers) * cfg->batch * cfg->n_q_heads * kD * 4);
     if (ok) ok = cudaMemset(c->status, 0, 256) == cudaSuccess;
     if (ok) ok = cudaMemset(c->tickets, 0, pairs * 128) == cudaSuccess;
+    if (ok) ok = cudaMemset(c->acc, 0, static_cast<size_t>(pairs) * kAccStride * 4) == cudaSuccess;
     // the fp store must never hold non-finite garbage in unused slots of a partly filled tile
     if (ok) ok = cudaMemset(cv.fp, 0, static_cast<size_t>(cv.fp_layer_stride) * cfg->n_layers) == cudaSuccess;
     if (!ok) {
@@ -701,6 +705,7 @@ lq_status_t decode_impl(lq_cache_t* c, int32_t layer, const void* q, float sm_sc
   a.new_v = new_v;
   a.new_slot = new_slot;
   a.tickets = nullptr;
+  a.acc = nullptr;
   cudaError_t e;
   const bool timed = c->profiling && c->ev_used + 2 <= c->ev_pool.size();
   if (timed) cudaEventRecord(c->ev_pool[c->ev_used], st);
@@ -715,6 +720,7 @@ lq_status_t decode_impl(lq_cache_t* c, int32_t layer, const void* q, float sm_sc
       a.n_extra = 0;
     }
     a.tickets = c->tickets;  // the CTA that completes a (b, kv) pair merges it: no second launch
+    a.acc = c->acc;
     e = launch_decode_mma(a, st);
     if (e != cudaSuccess) return cuda_fail(c, e, "lq_decode_mma_kernel");
   } else {

@@ -615,6 +615,7 @@ constexpr int kSmemQ = kMaxRatio * kD * 2;
 constexpr int kSmemBars = (kWarps * kMaxStages + 1) * 8;
 constexpr int kSmemBytes = kSmemStages + kSmemQ + kSmemBars + 16;
 constexpr int kMergeMax = 2048;  // S * r records the fused second pass can stage
+constexpr int kMergeOneBatch = 12;  // CTA records the fused second pass loads in one batch (kSB per warp)
 
 // Work items of one (b, kv) pair, in order: fp tiles [0, tiles_fp), then quant tiles.  The CTAs of
 // the pair (4 warps each) share them by a static, cost-weighted partition (see below); any
@@ -755,12 +756,31 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   // query fragments: B operand, column n -> head 4cb + n/2 (even column = hi, odd = lo of q*s);
   // k-step ks carries the factor 2^(64 - 2*(ks&3)) that cancels the code-position factor
   uint32_t qs[NCB][8][2];
+  // Pairs with more CTAs than the last one could fetch the records of in one batch of loads (kMergeOneBatch):
+  // every CTA also adds its partial to one sum per pair (DecodeArgs::acc), scaled to a reference score that
+  // all of them compute alike: q . k of the token in fp slot 0 (any real score of the pair will do).  Thread
+  // h of warp 0 keeps the reference of head h.  (Sums in arrival order: such pairs are not reproducible bit
+  // for bit from run to run; the others are.)
+  const bool use_acc = a.acc != nullptr && n_ctas_pair > kMergeOneBatch;
+  float ref = 0.f;
+  uint2 k0row = make_uint2(0u, 0u);
+  if (use_acc && warp == 0) k0row = __ldcg(reinterpret_cast<const uint2*>(fpbase) + lane);  // row 0: lane = 4 channels
   {
     int spins = 0;
     while (!mbar_try_wait(qbar, 0)) {
       if (++spins > kSpinLimit) { failed = true; break; }
     }
     failed = __any_sync(kFull, failed);
+    if (use_acc && warp == 0) {
+      const float k0 = bf16lo_f32(k0row.x), k1 = bf16hi_f32(k0row.x), k2 = bf16lo_f32(k0row.y), k3 = bf16hi_f32(k0row.y);
+      for (int h = 0; h < r; ++h) {
+        const uint2 qq = lds64(qsm + h * (kD * 2) + lane * 8);
+        float dot = k0 * bf16lo_f32(qq.x) + k1 * bf16hi_f32(qq.x) + k2 * bf16lo_f32(qq.y) + k3 * bf16hi_f32(qq.y);
+#pragma unroll
+        for (int o = 16; o; o >>= 1) dot += __shfl_xor_sync(kFull, dot, o);
+        if (lane == h) ref = dot * a.scale_log2;
+      }
+    }
 #pragma unroll
     for (int cb = 0; cb < NCB; ++cb) {
       const int head = 4 * cb + (n >> 1);
@@ -908,6 +928,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   float* wl = wm + kWarps * 8;                       // [warp][8]
   float* wf = wl + kWarps * 8;                       // [warp][8] factor of each warp state in the CTA state
   float* cml = wf + kWarps * 8;                      // [8][2] (m, l) of the CTA state
+  float* wsc = cml + 16;                             // [8] scale of the CTA state in the pair's sum
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) {
     if (bf16_pv<NCB>()) {
@@ -944,6 +965,16 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     }
     cml[2 * h] = M;
     cml[2 * h + 1] = L;
+    // scale of this CTA's partial in the pair's sum; far above the reference the sum could overflow and far
+    // below it the scale would underflow: the pair is then flagged and merged from the records instead
+    float sc = 0.f;
+    if (use_acc && L > 0.f) {
+      const float dd = M - ref;
+      if (!(dd <= 64.f && dd >= -100.f)) atomicOr(ticket + 1, 1);
+      else sc = ex2(dd);
+      if (sc > 0.f) atomicAdd(a.acc + static_cast<int64_t>(pair) * kAccStride + kMaxRatio * kD + h, L * sc);
+    }
+    wsc[h] = sc;
   }
   __syncthreads();
   const int d = threadIdx.x;
@@ -964,6 +995,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
           static_cast<float*>(a.out)[oi] = res;
       } else {
         a.part_o[(rec + h) * kD + d] = o;
+        if (use_acc && wsc[h] > 0.f) atomicAdd(a.acc + static_cast<int64_t>(pair) * kAccStride + h * kD + d, o * wsc[h]);
         if (d == 0) {
           a.part_ml[(rec + h) * 2 + 0] = cml[2 * h];
           a.part_ml[(rec + h) * 2 + 1] = cml[2 * h + 1];
@@ -985,12 +1017,44 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     __syncthreads();
     if (*is_last) {
       __threadfence();
+      // Fast path: the partials have already been summed on arrival (DecodeArgs::acc); one round trip
+      // fetches the sums.  It is taken unless a CTA flagged the pair (partial too far above the
+      // reference score) or a denominator is not a positive finite number (everything far below it).
+      float* accp = a.acc + static_cast<int64_t>(pair) * kAccStride;
+      constexpr int RALL = NCB == 1 ? 4 : 8;  // query heads per KV head this variant serves
+      bool fast = use_acc;
+      float so[RALL], sl[RALL];
+      if (use_acc) {
+        // all loads in flight at once: the flag, the denominators, this thread's channel of every head
+        const int flagged = *reinterpret_cast<volatile int*>(ticket + 1);
+#pragma unroll
+        for (int h = 0; h < RALL; ++h) {
+          sl[h] = h < r ? __ldcg(accp + kMaxRatio * kD + h) : 1.f;
+          so[h] = h < r ? __ldcg(accp + h * kD + d) : 0.f;
+        }
+        fast = flagged == 0;
+#pragma unroll
+        for (int h = 0; h < RALL; ++h) fast = fast && sl[h] > 0.f && sl[h] < INFINITY;
+      }
+      if (fast) {
+#pragma unroll
+        for (int h = 0; h < RALL; ++h) {
+          if (h < r) {
+            const float res = so[h] / sl[h];
+            const int64_t oi = (static_cast<int64_t>(b) * cv.Hq + kv * r + h) * kD + d;
+            if (a.out_bf16)
+              static_cast<__nv_bfloat16*>(a.out)[oi] = __float2bfloat16_rn(res);
+            else
+              static_cast<float*>(a.out)[oi] = res;
+          }
+        }
+      } else {
       // Warp w sums the records of the CTAs s = w, w + 4, ... for every head (lane = 4 channels,
       // 16-byte loads, kSB * RMAX independent loads in flight; the first batch is issued before the
       // weights are known), and the four warp sums meet in shared memory.  The weight of a record
       // is computed by the lane that loaded its (m, l): warp w normalises heads w, w + 4.
       constexpr int RMAX = NCB == 1 ? 4 : 8;  // query heads per KV head this variant serves
-      constexpr int kSB = 3;                  // CTA records per batch
+      constexpr int kSB = kMergeOneBatch / kWarps;  // CTA records per batch and warp
       float* sm_w = reinterpret_cast<float*>(smem);  // [S * r] weights
       float* red = sm_w + kMergeMax;                 // [warp][r][128] partial sums
       const int nS = n_ctas_pair;
@@ -1070,6 +1134,14 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
               make_uint2(pack_bf16x2(o.x, o.y), pack_bf16x2(o.z, o.w));
         else
           *reinterpret_cast<float4*>(static_cast<float*>(a.out) + oi) = o;
+      }
+      }  // merge from the records
+      if (use_acc) {
+        // leave the sums, the flag (and, above, the ticket) at rest for the next launch
+        __syncthreads();
+        for (int h = 0; h < r; ++h) accp[h * kD + d] = 0.f;
+        if (d < r) accp[kMaxRatio * kD + d] = 0.f;
+        if (d == 0) ticket[1] = 0;
       }
     }
   }  // ticket path
@@ -1187,7 +1259,7 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
   else return cudaErrorInvalidValue;
 #undef LQ_PICK
 #undef LQ_PICK2
-  static_assert(kSmemStages >= static_cast<int>((kWarps * 8 * (kD + 4) + 3 * kWarps * 8 + 16) * sizeof(float)) &&
+  static_assert(kSmemStages >= static_cast<int>((kWarps * 8 * (kD + 4) + 3 * kWarps * 8 + 16 + 8) * sizeof(float)) &&
                     kSmemStages >= (kMergeMax + kWarps * kMaxRatio * kD) * 4,
                 "merge scratch");
   // opt in to the dynamic shared memory size once per (device, kernel variant)

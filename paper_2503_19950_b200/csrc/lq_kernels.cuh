@@ -97,9 +97,16 @@ struct DecodeArgs {
   int n_ctas;
   int* status;  // device word; kernels OR error bits into it (bounded waits that gave up)
   int* tickets; // one 128-byte line per (b, kv): word [1] is the arrival counter of the fused second
-                // pass, 0 at rest
+                // pass, word [2] the "sum out of range" flag of the accumulators below; both 0 at rest
                 // (null: static split and a separate merge launch)
+  // Tensor-core kernel, pairs with more than one CTA: besides its record every CTA adds its partial, scaled to
+  // a reference score all CTAs of the pair compute alike, to acc with global atomics, so that the CTA that
+  // completes the pair only has to read one sum: acc[pair * kAccStride + h * 128 + d] and, for the
+  // denominators, acc[pair * kAccStride + kMaxRatio * 128 + h]; all zero at rest.  null: records only.
+  float* acc;
 };
+
+constexpr int kAccStride = kMaxRatio * 128 + 32;  // floats per (b, kv) pair in DecodeArgs::acc
 
 cudaError_t launch_decode_scalar(const DecodeArgs& a, cudaStream_t st);
 // Fills S and the tile counts of `a` for the tensor-core kernel (S <= max_records; s_override > 0 forces S).
