@@ -326,6 +326,9 @@ def run_ours(args, wl, rank, world, device):
                    "step": "per layer: lq_append_decode_attn (append and attention in one launch; the overflow step and "
                            "a separate append when the window is full)",
                    "l2": "inputs larger than L2: %.2f GB of cache touched per step" % (bytes_step_last / 1e9),
+                   "merge": ("partials summed on arrival with global atomics (more than 12 CTAs per (b, kv) pair; not "
+                             "bit-reproducible), records as fallback" if int(inf.n_splits) >= 12 else
+                             "ordered merge of the CTA records by the last CTA of a pair (bit-reproducible)"),
                    "replicas": "independent per GPU, no collective on the data path"},
         "per_layer_us": ms_max / steps / L * 1e3,
         "algorithmic_gbs_whole_step": bytes_step_last / (ms_max / steps * 1e-3) / 1e9,
