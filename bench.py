@@ -406,6 +406,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="override the number of stacked layer caches (profiling runs)")
     ap.add_argument("--n-splits", type=int, default=0, help="split-K CTAs per (batch row, KV head); 0 = library default")
+    ap.add_argument("--shorten-prefill", type=int, default=0,
+                    help="prefill this many tokens fewer than the workload's context (e.g. W/2: the overflow step then "
+                         "falls in the middle of the timed steps instead of on the first decode step)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -415,6 +418,8 @@ def main():
     wl = dict(WORKLOADS[args.workload])
     if args.layers > 0:
         wl["L"] = args.layers
+    if args.shorten_prefill > 0:
+        wl["ctx"] = max(1, wl["ctx"] - args.shorten_prefill)
     wl["_outliers"] = synth.outlier_channels(wl["seed"], wl["Hkv"], D, wl["n_outliers"]) if wl["n_outliers"] else None
     cores = os.cpu_count() or 1
 
