@@ -305,6 +305,12 @@ def run_ours(args, wl, rank, world, device):
         ccache.close()
     except Exception as exc:  # the main numbers stand without it
         comp = {"error": str(exc)}
+    planted_bf16 = None
+    if wl.get("planted"):
+        # context only: which of the planted high-logit tokens (distances 2^i behind the end of the prompt) are
+        # still at full precision in the log-spaced selection at the end of the run
+        kept = set(int(t) for t in cache.export(0)["kept_ids"])
+        planted_bf16 = [1 << i for i in range(32) if (1 << i) <= ctx and (ctx - (1 << i)) in kept]
     status = cache.kernel_status()
     assert status == 0, f"kernel status word {status}"
     assert all(torch.isfinite(o).all() for o in outs)
@@ -322,7 +328,7 @@ def run_ours(args, wl, rank, world, device):
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": args.workload, "layers": L, "batch": B, "q_heads": Hq, "kv_heads": Hkv,
                    "head_dim": D, "context": ctx, "window": W, "group": G, "bits": bits,
-                   "padding": pad, "n_quant": int(inf.n_quant), "n_fp": int(inf.n_fp), "n_splits": int(inf.n_splits), "n_ctas": int(inf.n_ctas),
+                   "padding": pad, "planted_distances_still_bf16": planted_bf16, "n_quant": int(inf.n_quant), "n_fp": int(inf.n_fp), "n_splits": int(inf.n_splits), "n_ctas": int(inf.n_ctas),
                    "step": "per layer: lq_append_decode_attn (append and attention in one launch; the overflow step and "
                            "a separate append when the window is full)",
                    "l2": "inputs larger than L2: %.2f GB of cache touched per step" % (bytes_step_last / 1e9),
