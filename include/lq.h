@@ -82,6 +82,13 @@ typedef struct {
   int32_t kernel;        /* LQ_KERNEL_*                                                          */
   int32_t n_splits;      /* split-K CTAs per (batch row, KV head); 0 = chosen by the library     */
   int32_t filter;        /* LQ_FILTER_*: which W tokens leave the full-precision store on overflow */
+  /* Optional device allocator (all three NULL / 0: cudaMalloc and cudaFree).  dev_alloc returns device memory of
+     at least `bytes` bytes, 256-byte aligned, on `device`, or NULL on failure (the call that needed it then gives
+     LQ_ERR_OOM); every block is handed back to dev_free by lq_destroy (or at once when creation fails).  Both
+     are called on the host, from the thread that calls into the library, with alloc_ctx passed through. */
+  void* (*dev_alloc)(size_t bytes, void* alloc_ctx);
+  void (*dev_free)(void* ptr, void* alloc_ctx);
+  void* alloc_ctx;
 } lq_config_t;
 
 typedef struct {

@@ -16,12 +16,17 @@ LQ_OK, LQ_ERR_INVALID_ARG, LQ_ERR_UNSUPPORTED, LQ_ERR_OOM, LQ_ERR_WINDOW_FULL, L
     LQ_ERR_CAPACITY, LQ_ERR_CUDA = range(8)
 
 
+ALLOC_FN = C.CFUNCTYPE(C.c_void_p, C.c_size_t, C.c_void_p)
+FREE_FN = C.CFUNCTYPE(None, C.c_void_p, C.c_void_p)
+
+
 class lq_config_t(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("batch", C.c_int32), ("n_q_heads", C.c_int32),
                 ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("window", C.c_int32),
                 ("group", C.c_int32), ("bits", C.c_int32), ("max_tokens", C.c_int64),
                 ("auto_compress", C.c_int32), ("device", C.c_int32), ("kernel", C.c_int32),
-                ("n_splits", C.c_int32), ("filter", C.c_int32)]
+                ("n_splits", C.c_int32), ("filter", C.c_int32),
+                ("dev_alloc", ALLOC_FN), ("dev_free", FREE_FN), ("alloc_ctx", C.c_void_p)]
 
 
 class lq_info_t(C.Structure):
@@ -130,10 +135,35 @@ class LogQuantCache:
     """Owner of one lq_cache_t.  Methods mirror the C entry points one to one."""
 
     def __init__(self, n_layers, batch, n_q_heads, n_kv_heads, window, group, max_tokens, head_dim=128, bits=2,
-                 auto_compress=True, device=0, kernel=LQ_KERNEL_AUTO, n_splits=0, filter=0):
+                 auto_compress=True, device=0, kernel=LQ_KERNEL_AUTO, n_splits=0, filter=0, allocator=None):
+        """allocator: None (cudaMalloc / cudaFree), "torch" (every device block of the cache is a uint8 tensor from
+        torch's caching allocator, kept alive until the cache is closed), or a pair of callables
+        (alloc(bytes) -> device address or 0, free(address))."""
         self._lib = load_library()
+        self._blocks = {}
+        alloc_cb, free_cb = ALLOC_FN(0), FREE_FN(0)
+        if allocator == "torch":
+            import torch
+
+            def _alloc(nbytes, _ctx):
+                try:
+                    t = torch.empty(max(int(nbytes), 1), dtype=torch.uint8, device=torch.device("cuda", device))
+                except RuntimeError:
+                    return 0
+                self._blocks[t.data_ptr()] = t
+                return t.data_ptr()
+
+            def _free(ptr, _ctx):
+                self._blocks.pop(ptr, None)
+
+            alloc_cb, free_cb = ALLOC_FN(_alloc), FREE_FN(_free)
+        elif allocator is not None:
+            user_alloc, user_free = allocator
+            alloc_cb = ALLOC_FN(lambda nbytes, _ctx: int(user_alloc(int(nbytes))) or 0)
+            free_cb = FREE_FN(lambda ptr, _ctx: user_free(ptr))
+        self._callbacks = (alloc_cb, free_cb)  # keep the trampolines alive as long as the cache
         self.cfg = lq_config_t(n_layers, batch, n_q_heads, n_kv_heads, head_dim, window, group, bits, max_tokens,
-                               int(auto_compress), device, kernel, n_splits, filter)
+                               int(auto_compress), device, kernel, n_splits, filter, alloc_cb, free_cb, None)
         self._h = C.c_void_p()
         self._check(self._lib.lq_cache_create(C.byref(self.cfg), C.byref(self._h)), create=True)
 

@@ -82,7 +82,10 @@ lq_status_t cuda_fail(lq_cache* c, cudaError_t e, const char* what) {
 }
 
 bool dev_alloc(lq_cache* c, void** p, int64_t bytes) {
-  if (cudaMalloc(p, static_cast<size_t>(bytes)) != cudaSuccess) {
+  if (c->cfg.dev_alloc) {  // the caller's allocator
+    *p = c->cfg.dev_alloc(static_cast<size_t>(bytes), c->cfg.alloc_ctx);
+    if (*p == nullptr) return false;
+  } else if (cudaMalloc(p, static_cast<size_t>(bytes)) != cudaSuccess) {
     cudaGetLastError();
     *p = nullptr;
     return false;
@@ -91,21 +94,29 @@ bool dev_alloc(lq_cache* c, void** p, int64_t bytes) {
   return true;
 }
 
+void dev_release(lq_cache* c, void* p) {
+  if (p == nullptr) return;
+  if (c->cfg.dev_free) c->cfg.dev_free(p, c->cfg.alloc_ctx);
+  else cudaFree(p);
+}
+
 void free_all(lq_cache* c) {
   if (!c->dry) {
-    cudaFree(c->cv.quant);
-    cudaFree(c->cv.fp);
-    cudaFree(c->part_o);
-    cudaFree(c->part_ml);
-    cudaFree(c->status);
-    cudaFree(c->tickets);
-    cudaFree(c->acc);
-    cudaFree(c->ingest_idx);
-    cudaFree(c->stage_k);
-    cudaFree(c->stage_v);
-    cudaFree(c->stage_q);
-    cudaFree(c->stage_out);
-    cudaFree(c->masks);
+    // the caller's allocator does not wait for work in flight the way cudaFree does
+    if (c->cfg.dev_free) cudaDeviceSynchronize();
+    dev_release(c, c->cv.quant);
+    dev_release(c, c->cv.fp);
+    dev_release(c, c->part_o);
+    dev_release(c, c->part_ml);
+    dev_release(c, c->status);
+    dev_release(c, c->tickets);
+    dev_release(c, c->acc);
+    dev_release(c, c->ingest_idx);
+    dev_release(c, c->stage_k);
+    dev_release(c, c->stage_v);
+    dev_release(c, c->stage_q);
+    dev_release(c, c->stage_out);
+    dev_release(c, c->masks);
     for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   }
 }
@@ -386,6 +397,7 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
       cfg->window < 1 || cfg->group < 1 || cfg->max_tokens < 1 || cfg->n_splits < 0)
     return LQ_ERR_INVALID_ARG;
   if (cfg->n_q_heads % cfg->n_kv_heads) return LQ_ERR_INVALID_ARG;
+  if ((cfg->dev_alloc == nullptr) != (cfg->dev_free == nullptr)) return LQ_ERR_INVALID_ARG;
   if (cfg->head_dim != kD || (cfg->bits != 2 && cfg->bits != 4)) return LQ_ERR_UNSUPPORTED;
   if (cfg->group != 32 && cfg->group != 64) return LQ_ERR_UNSUPPORTED;
   if (cfg->bits == 4 && cfg->group != 32) return LQ_ERR_UNSUPPORTED;  // a 4-bit tile of G = 64 exceeds a stage

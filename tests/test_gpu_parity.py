@@ -531,3 +531,42 @@ def test_partials_summed_on_arrival_and_the_record_fallback(k0_gain, pad0):
         assert np.abs(got - ref).max() <= attn_tolerance(ref), (step, k0_gain, pad0)
     assert cache.kernel_status() == 0
     cache.close(); oc.close()
+
+
+def test_caller_supplied_device_allocator():
+    """Every device block of a cache can come from the caller (here torch's caching allocator); a failing
+    allocator gives LQ_ERR_OOM and hands back what it had handed out."""
+    B, Hq, Hkv, W, G, D, N = 2, 8, 2, 32, 32, 128, 300
+    cache = LogQuantCache(2, B, Hq, Hkv, W, G, max_tokens=N + 8, allocator="torch")
+    blocks = cache._blocks  # address -> tensor, filled and emptied by the hooks
+    assert sum(t.numel() for t in blocks.values()) >= cache.info(0).bytes_device > 0
+    n_blocks = len(blocks)
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G)
+    k, v = synth.keys_values(71, B, Hkv, N, D, "cuda")
+    cache.append(1, k, v)
+    oc.append(synth.bf16_bits(k), synth.bf16_bits(v))
+    assert_images_equal(cache.export(1), oc.export())
+    q = synth.queries(71, B, Hq, D, 0, "cuda")
+    out = torch.empty(B, Hq, D, device="cuda")
+    cache.set_padding([10, 0])  # the masks are allocated through the same hook
+    assert len(blocks) == n_blocks + 1
+    cache.decode_attn(1, q, out)
+    torch.cuda.synchronize()
+    ref = oc.attention_subset(synth.bf16_bits(q), 1 / np.sqrt(D), pad=[10, 0])
+    assert np.abs(out.cpu().numpy() - ref).max() <= attn_tolerance(ref)
+    cache.close()
+    assert not blocks  # every block went back through dev_free
+
+    live, calls = {}, [0]
+
+    def alloc(nbytes):
+        calls[0] += 1
+        if calls[0] > 3:
+            return 0  # out of memory on the fourth block
+        t = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        live[t.data_ptr()] = t
+        return t.data_ptr()
+
+    with pytest.raises(LogQuantError) as e:
+        LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=N, allocator=(alloc, lambda ptr: live.pop(ptr)))
+    assert e.value.status == binding.LQ_ERR_OOM and not live

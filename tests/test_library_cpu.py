@@ -72,6 +72,14 @@ def test_no_gpu_means_no_compute():
     assert e.value.status == binding.LQ_ERR_UNSUPPORTED
 
 
+def test_allocator_hooks_come_in_pairs():
+    cfg = binding.lq_config_t(1, 1, 4, 2, 128, 128, 32, 2, 1024, 1, LQ_DEVICE_NONE, 0, 0, 0,
+                              binding.ALLOC_FN(lambda n, ctx: 0), binding.FREE_FN(0), None)
+    import ctypes
+    h = ctypes.c_void_p()
+    assert binding.load_library().lq_cache_create(ctypes.byref(cfg), ctypes.byref(h)) == binding.LQ_ERR_INVALID_ARG
+
+
 def test_padding_arguments_without_a_device():
     c = _dry(W=128, G=32, batch=3)
     c.set_padding([0, 5, 9])
