@@ -570,3 +570,22 @@ def test_caller_supplied_device_allocator():
     with pytest.raises(LogQuantError) as e:
         LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=N, allocator=(alloc, lambda ptr: live.pop(ptr)))
     assert e.value.status == binding.LQ_ERR_OOM and not live
+
+
+def _random_padded_cases(n, seed):
+    rng = np.random.default_rng(seed)
+    cases = []
+    for B, Hq, Hkv, W, G, bits, n_prefill, chunk, recent in _random_cases(n, seed):
+        B = max(B, 2)
+        pad = [int(rng.integers(0, n_prefill + 1)) if rng.random() < 0.75 else 0 for _ in range(B)]
+        kernel = LQ_KERNEL_MMA if rng.random() < 0.75 else LQ_KERNEL_SCALAR
+        cases.append((B, Hq, Hkv, W, G, bits, n_prefill, chunk, recent, pad, kernel, bool(rng.random() < 0.7)))
+    return cases
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,W,G,bits,n_prefill,chunk,recent,pad,kernel,auto", _random_padded_cases(10, 4242))
+def test_seeded_random_padded_configurations(B, Hq, Hkv, W, G, bits, n_prefill, chunk, recent, pad, kernel, auto):
+    """A seeded draw like the one above with left padding, both kernels and caller-driven overflow steps."""
+    worst = run_case(B, Hq, Hkv, W, G, n_prefill, 3, seed=200 + n_prefill, kernel=kernel, bits=bits, prefill_chunk=chunk,
+                     recent_only=recent, pad=pad, auto_compress=auto, check_image_every=1)
+    assert worst <= 1.0
