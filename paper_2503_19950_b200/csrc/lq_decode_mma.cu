@@ -1048,6 +1048,42 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
               static_cast<float*>(a.out)[oi] = res;
           }
         }
+      } else if (NCB == 1 && n_ctas_pair <= kMergeOneBatch) {
+        // Up to 4 heads and few records: warp w merges head w on its own -- every record of the head in one
+        // batch of loads, the weights spread over the lanes and handed round by shuffles -- and writes the
+        // result; no shared memory, no barrier.  (Records are summed in slot order: bit-reproducible.)
+        if (warp < r) {
+          const int h = warp, nS = n_ctas_pair;
+          float4 v[kMergeOneBatch];
+#pragma unroll
+          for (int sr = 0; sr < kMergeOneBatch; ++sr)
+            if (sr < nS) v[sr] = __ldcg(reinterpret_cast<const float4*>(a.part_o + (rec0 + sr * r + h) * kD) + lane);
+          const float2 ml = lane < nS ? __ldcg(reinterpret_cast<const float2*>(a.part_ml) + rec0 + lane * r + h)
+                                      : make_float2(-INFINITY, 0.f);
+          float M = ml.y > 0.f ? ml.x : -INFINITY;
+#pragma unroll
+          for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(kFull, M, o));
+          const float e = ml.y > 0.f ? ex2(ml.x - M) : 0.f;
+          float L = ml.y * e;
+#pragma unroll
+          for (int o = 16; o; o >>= 1) L += __shfl_xor_sync(kFull, L, o);
+          const float wgt = e / L;
+          float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+          for (int sr = 0; sr < kMergeOneBatch; ++sr) {
+            const float w = __shfl_sync(kFull, wgt, sr);
+            if (sr < nS) {
+              o.x = fmaf(v[sr].x, w, o.x); o.y = fmaf(v[sr].y, w, o.y);
+              o.z = fmaf(v[sr].z, w, o.z); o.w = fmaf(v[sr].w, w, o.w);
+            }
+          }
+          const int64_t oi = (static_cast<int64_t>(b) * cv.Hq + kv * r + h) * kD + 4 * lane;
+          if (a.out_bf16)
+            *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(a.out) + oi) =
+                make_uint2(pack_bf16x2(o.x, o.y), pack_bf16x2(o.z, o.w));
+          else
+            *reinterpret_cast<float4*>(static_cast<float*>(a.out) + oi) = o;
+        }
       } else {
       // Warp w sums the records of the CTAs s = w, w + 4, ... for every head (lane = 4 channels,
       // 16-byte loads, kSB * RMAX independent loads in flight; the first batch is issued before the
