@@ -30,7 +30,7 @@ if ROOT not in sys.path:
 from paper_2503_19950_b200 import synth  # noqa: E402
 
 WORKLOADS = {
-    # BASELINE config 2: Llama-3-8B layer shape, batch 8, context 8192, W=128, G=32, 32 stacked layers
+    # the configuration the metric is quoted on: Llama-3-8B layer shape, batch 8, context 8192, W=128, G=32, 32 stacked layers
     "llama3-8b-8k": dict(L=32, B=8, Hq=32, Hkv=8, W=128, G=32, ctx=8192, n_outliers=3, seed=2),
     # config 2 in the paper's own setting (Sec. 3.1): group 64, reserved length 128 tokens, i.e. W = 42 (not a
     # multiple of G: removed tokens wait at full precision until 64 of them form a key group)
@@ -341,6 +341,10 @@ def run_ours(args, wl, rank, world, device):
         "gpu_launches": int(launches),
         # bf16 cache bytes / mixed cache bytes actually read per step (scale and zero counted)
         "compression_ratio": (B * Hkv * (int(inf.n_quant) + int(inf.n_fp)) * 4 * D) / max(int(inf.bytes_decode_step), 1),
+        # the paper's own formula (Eq. 4-5), which counts the 2-bit codes only: 16 L / (2 (L - R) + 16 R) with L tokens
+        # in the cache and R of them at full precision (for bits = 4: 4 in place of 2)
+        "compression_ratio_paper_formula": 16.0 * (int(inf.n_quant) + int(inf.n_fp)) /
+                                           (bits * int(inf.n_quant) + 16.0 * int(inf.n_fp)),
         "compress_event": comp,
         "clocks": clk.summary(),
         "e2e": {"value": aggregate_throughput(kv_e2e, world, e2e_ms_max), "unit": "KV tokens/s",
@@ -365,7 +369,102 @@ def run_ours(args, wl, rank, world, device):
             m = re.search(r"dram_bytes_per_launch:\s*([0-9.eE+]+)", f.read())
         if m:
             line["roofline"]["traffic"] = float(m.group(1))
+    line["_replay"] = {"ks0": ks[0], "vs0": vs[0], "qs0": qs[0], "n_decode_tokens": int(cache.info(0).n_seen) - ctx}
     return line, cache
+
+
+def roofline_only(name, device, layers, rounds=24, n_splits=0):
+    """Back-to-back timing of the attention kernel on another workload (a few layer caches, a few seconds):
+    the same measurement as the `roofline` object of the main line."""
+    from paper_2503_19950_b200 import LogQuantCache
+    wl = dict(WORKLOADS[name], L=layers)
+    wl["_outliers"] = synth.outlier_channels(wl["seed"], wl["Hkv"], D, wl["n_outliers"]) if wl["n_outliers"] else None
+    L, B, Hq, Hkv, W, G, ctx = (wl[k] for k in ("L", "B", "Hq", "Hkv", "W", "G", "ctx"))
+    cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=ctx + 64, device=device.index or 0, bits=wl.get("bits", 2),
+                          n_splits=n_splits)
+    prefill(cache, wl, device)
+    ks, vs, qs = make_step_inputs(wl, device, 4)
+    outs = [torch.empty(B, Hq, D, device=device) for _ in range(L)]
+    for l in range(L):  # first decode step: the overflow step runs here, the timed launches see the state after it
+        cache.append_decode_attn(l, ks[l][0], vs[l][0], qs[l][0], outs[l])
+    evs = []
+    for rep in range(rounds + 3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for l in range(L):
+            cache.decode_attn(l, qs[l][rep % 4], outs[l])
+        e1.record()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    us = sorted(e0.elapsed_time(e1) * 1e3 for e0, e1 in evs[3:])
+    b2b_us = us[len(us) // 2] / L
+    inf = cache.info(0)
+    nbytes = int(inf.bytes_decode_step)
+    peak, peak_kind = peaks()
+    ok = cache.kernel_status() == 0 and all(bool(torch.isfinite(o).all()) for o in outs)
+    cache.close()
+    return {"workload": name, "layers": L, "bound": "hbm", "achieved": nbytes / (b2b_us * 1e-6) / 1e9, "peak": peak,
+            "unit": "GB/s", "frac": nbytes / (b2b_us * 1e-6) / 1e9 / peak, "peak_kind": peak_kind,
+            "bytes_per_launch": nbytes, "us_per_launch": b2b_us, "us_per_launch_best": us[0] / L,
+            "kv_tokens_per_s": B * (int(inf.n_quant) + int(inf.n_fp)) / (b2b_us * 1e-6),
+            "n_quant": int(inf.n_quant), "n_fp": int(inf.n_fp), "n_ctas": int(inf.n_ctas), "finite_and_status_ok": ok,
+            "frac_of_8tbs_nominal": nbytes / (b2b_us * 1e-6) / 1e9 / 8000.0,
+            "timing": "median over %d rounds of %d back-to-back launches, one per layer cache" % (len(us), L)}
+
+
+def parity_against_oracle(cache, wl, device, replay):
+    """Checker leg (uses oracle/): replays every token layer 0 of the timed cache has received into the CPU oracle,
+    takes one more decode step through the call the bench times (lq_append_decode_attn) and compares the canonical
+    image and the attention output of that step with the oracle's."""
+    import oracle
+    B, Hq, Hkv, W, G = (wl[k] for k in ("B", "Hq", "Hkv", "W", "G"))
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G, bits=wl.get("bits", 2))
+    prefill(None, dict(wl, L=1), device, sink=lambda l, k, v: oc.append(synth.bf16_bits(k), synth.bf16_bits(v)))
+    n = replay["n_decode_tokens"]
+    for j in range(n + 1):  # decode token j of a layer was set j % Q_ROTATE; the last one is appended below
+        s = j % Q_ROTATE
+        oc.append(synth.bf16_bits(replay["ks0"][s]), synth.bf16_bits(replay["vs0"][s]))
+    s = n % Q_ROTATE
+    out = torch.full((B, Hq, D), float("nan"), device=device)
+    cache.append_decode_attn(0, replay["ks0"][s], replay["vs0"][s], replay["qs0"][s], out)
+    torch.cuda.synchronize()
+    inf = cache.info(0)
+    state_ok = (inf.n_seen, inf.n_fp, inf.n_quant, inf.n_events) == (oc.n_seen, oc.n_fp, oc.n_quant, oc.n_events)
+    got, want = cache.export(0), oc.export()
+    image_ok = state_ok and all(np.array_equal(got[key], want[key]) for key in want)
+    pad = wl.get("pad")
+    if pad:
+        ref = oc.attention_subset(synth.bf16_bits(replay["qs0"][s]), 1.0 / np.sqrt(D), pad=pad)
+    else:
+        ref = oc.attention(synth.bf16_bits(replay["qs0"][s]), 1.0 / np.sqrt(D), n_threads=os.cpu_count() or 1)
+    o = out.cpu().numpy().astype(np.float64)
+    err = float(np.abs(o - ref).max()) if np.isfinite(o).all() else float("inf")
+    tol = 2e-3 * float(np.abs(ref).max()) + 1e-3
+    return {"max_err": err, "tol": tol, "image_bit_exact": bool(image_ok), "ok": bool(image_ok and err <= tol),
+            "checked": "layer 0 after %d decode tokens, one step through lq_append_decode_attn: canonical image and "
+                       "[B, Hq, D] output against the float64 oracle" % (n + 1)}
+
+
+def oracle_compress_event(wl, device, reps=5):
+    """Times the CPU oracle on one window-overflow step of one layer (the append that finds 3W tokens)."""
+    import oracle
+    B, Hq, Hkv, W, G = (wl[k] for k in ("B", "Hq", "Hkv", "W", "G"))
+    kf, vf = synth.keys_values(wl["seed"] + 7, B, Hkv, 3 * W + 1, D, device, outliers=wl.get("_outliers"))
+    kb, vb = synth.bf16_bits(kf), synth.bf16_bits(vf)
+    ts = []
+    for rep in range(reps):
+        oc = oracle.OracleCache(B, Hq, Hkv, D, W, G, bits=wl.get("bits", 2))
+        oc.append(np.ascontiguousarray(kb[:, :, :3 * W]), np.ascontiguousarray(vb[:, :, :3 * W]))
+        k1, v1 = np.ascontiguousarray(kb[:, :, 3 * W:]), np.ascontiguousarray(vb[:, :, 3 * W:])
+        t0 = time.perf_counter()
+        oc.append(k1, v1)
+        ts.append(time.perf_counter() - t0)
+        assert oc.n_events == 1
+        oc.close()
+    us = float(np.median(ts)) * 1e6
+    return {"us_per_event_one_layer": us, "tokens_per_s": B * W / (us * 1e-6), "threads": 1,
+            "what": "oracle append of the token that finds 3W full-precision tokens: filter, quantise and pack W tokens "
+                    "of all %d sequences, one layer" % B}
 
 
 def oracle_layer_step(wl, device, n_threads, min_seconds, max_reps, warmup=0):
@@ -402,12 +501,42 @@ def oracle_layer_step(wl, device, n_threads, min_seconds, max_reps, warmup=0):
     return kv / t_total, reps, t_total, times
 
 
+def spawn_replicas(n, argv, need_gpus=True, timeout=None):
+    """Re-runs this script as n ranks under torch.distributed.run (rendezvous on 127.0.0.1).  Fails loudly when
+    the machine has fewer than n GPUs."""
+    import socket
+    import subprocess
+    if need_gpus and torch.cuda.device_count() < n:
+        sys.stderr.write("bench.py: --gpus %d asked for, %d CUDA device(s) visible\n" % (n, torch.cuda.device_count()))
+        return 2
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.run(cmd, timeout=timeout).returncode
+
+
+def replica_selftest(args, rank, world):
+    """CPU-only check of the replica plumbing (no kernel, no oracle): every rank 'processes' a fixed number of
+    units in a rank-dependent time; rank 0 prints the line the real run would print from these."""
+    torch.distributed.init_process_group("gloo")
+    units, ms = 1000, 10.0 + 5.0 * rank
+    ms_max = reduce_max_over_ranks([ms], world, torch.device("cpu"))[0]
+    if rank == 0:
+        print(json.dumps({"impl": "replica-selftest", "n_gpus": world, "value": aggregate_throughput(units, world, ms_max),
+                          "ms_per_step": ms_max, "scaling": "weak"}))
+    torch.distributed.barrier()
+    torch.distributed.destroy_process_group()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=128)
     ap.add_argument("--warmup", type=int, default=8)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference", "replica-selftest"])
     ap.add_argument("--workload", default="llama3-8b-8k", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="override the number of stacked layer caches (profiling runs)")
@@ -415,8 +544,19 @@ def main():
     ap.add_argument("--shorten-prefill", type=int, default=0,
                     help="prefill this many tokens fewer than the workload's context (e.g. W/2: the overflow step then "
                          "falls in the middle of the timed steps instead of on the first decode step)")
+    ap.add_argument("--also", default=None,
+                    help="comma-separated workloads whose attention kernel is timed back to back as well and reported "
+                         "under roofline_<workload> (default: gqa7-32k and llama3-8b-4k-b64 beside the default workload)")
+    ap.add_argument("--also-layers", type=int, default=4, help="layer caches of the --also workloads")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.also is None:
+        args.also = "gqa7-32k,llama3-8b-4k-b64" if args.workload == "llama3-8b-8k" and args.layers == 0 else ""
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # replicas only: --gpus N without a launcher starts N ranks of this script (one per GPU), which time N
+        # independent replicas; no collective touches the data path
+        return spawn_replicas(args.gpus, sys.argv[1:], need_gpus=args.impl == "ours")
 
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
@@ -429,6 +569,8 @@ def main():
     wl["_outliers"] = synth.outlier_channels(wl["seed"], wl["Hkv"], D, wl["n_outliers"]) if wl["n_outliers"] else None
     cores = os.cpu_count() or 1
 
+    if args.impl == "replica-selftest":
+        return replica_selftest(args, rank, world)
     if args.impl == "reference":
         if rank != 0:
             return 0
@@ -455,10 +597,21 @@ def main():
     if world > 1:
         torch.distributed.init_process_group("nccl", device_id=device)
     line, cache = run_ours(args, wl, rank, world, device)
+    replay = line.pop("_replay")
+    parity_failed = False
     if rank == 0:
+        for name in [n for n in args.also.split(",") if n]:
+            try:
+                line["roofline_" + name.replace("-", "_")] = roofline_only(name, device, args.also_layers)
+            except Exception as exc:  # the main line stands without it
+                line["roofline_" + name.replace("-", "_")] = {"error": str(exc)}
         if not args.no_cpu_baseline:
             import oracle
             oracle.build()
+            line["parity"] = parity_against_oracle(cache, wl, device, replay)
+            parity_failed = not line["parity"]["ok"]
+            if isinstance(line.get("compress_event"), dict) and "error" not in line["compress_event"]:
+                line["compress_event"]["cpu_oracle"] = oracle_compress_event(wl, device)
             tput, reps, t_total, _ = oracle_layer_step(wl, device, cores, min_seconds=10.0, max_reps=512)
             tput1, reps1, t1, _ = oracle_layer_step(wl, device, 1, min_seconds=3.0, max_reps=64)
             line["cpu_baseline"] = {"value": tput, "unit": "KV tokens/s", "cores": cores, "kind": "oracle",
@@ -474,6 +627,9 @@ def main():
     if world > 1:
         torch.distributed.barrier()
         torch.distributed.destroy_process_group()
+    if parity_failed:
+        sys.stderr.write("bench.py: the timed path disagrees with the oracle: %s\n" % json.dumps(line["parity"]))
+        return 1
     return 0
 
 

@@ -247,11 +247,12 @@ lq_status_t lq_next_evicted_ids(const lq_cache_t* cache, int32_t layer, int32_t*
  */
 typedef struct {
   int32_t batch, n_q_heads, n_kv_heads, head_dim, group;
+  int32_t bits;      /* code width of k_codes / v_codes: 2 or 4 (anything else: LQ_ERR_INVALID_ARG)  */
   int32_t n_fp;      /* rows of fp_k / fp_v per (batch row, KV head)                              */
   int64_t n_quant;   /* quantised tokens per (batch row, KV head); a multiple of group            */
   const uint16_t* fp_k;    /* [B][Hkv][n_fp][D] bf16 bits                                          */
   const uint16_t* fp_v;
-  const uint8_t* k_codes;  /* [B][Hkv][n_quant][D/4]                                               */
+  const uint8_t* k_codes;  /* [B][Hkv][n_quant][D/4] (bits = 2) or [..][D/2] (bits = 4)                */
   const uint8_t* v_codes;
   const uint16_t* k_scale; /* [B][Hkv][n_quant/G][D]                                               */
   const uint16_t* k_zero;
@@ -272,7 +273,8 @@ typedef struct {
  *
  * Limits and rules:
  *   - batch * n_q_heads <= 8192 (LQ_ERR_CAPACITY otherwise: the scratch holds 8192 partial records);
- *     head_dim 128, group 32 or 64, n_q_heads / n_kv_heads <= 8 (LQ_ERR_UNSUPPORTED otherwise).
+ *     head_dim 128, group 32 or 64, n_q_heads / n_kv_heads <= 8 (LQ_ERR_UNSUPPORTED otherwise); bits 2 or 4,
+ *     which must be the width the codes of the image were packed with (LQ_ERR_INVALID_ARG for other values).
  *   - No cudaMalloc, cudaFree or other allocating call is made, ever.  The first call on each device
  *     looks up the scratch's device address (cudaGetSymbolAddress) with that device current; make
  *     that first call before any stream capture begins.

@@ -43,7 +43,7 @@ class lq_image_t(C.Structure):
 
 class lq_device_image_t(C.Structure):
     _fields_ = [("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
-                ("group", C.c_int32), ("n_fp", C.c_int32), ("n_quant", C.c_int64)] + \
+                ("group", C.c_int32), ("bits", C.c_int32), ("n_fp", C.c_int32), ("n_quant", C.c_int64)] + \
                [(n, C.c_void_p) for n in ("fp_k", "fp_v", "k_codes", "v_codes", "k_scale", "k_zero", "v_scale", "v_zero")]
 
 
@@ -120,12 +120,13 @@ def _stream(stream):
     return stream if isinstance(stream, int) else stream.cuda_stream
 
 
-def decode_attn_image_static(image: dict, n_q_heads: int, group: int, q, out, sm_scale=0.0, stream=None) -> int:
+def decode_attn_image_static(image: dict, n_q_heads: int, group: int, q, out, sm_scale=0.0, stream=None,
+                             bits: int = 2) -> int:
     """lq_decode_attn_image_static on a canonical image whose arrays are torch tensors on the device
     (keys as in LogQuantCache.export, without the ids).  Allocates nothing; returns the status code."""
     B, Hkv, n_fp, D = image["fp_k"].shape
     n_quant = image["k_codes"].shape[2]
-    st = lq_device_image_t(B, n_q_heads, Hkv, D, group, n_fp, n_quant,
+    st = lq_device_image_t(B, n_q_heads, Hkv, D, group, bits, n_fp, n_quant,
                            *[(_ptr(image[k]) if image[k].numel() else None)
                              for k in ("fp_k", "fp_v", "k_codes", "v_codes", "k_scale", "k_zero", "v_scale", "v_zero")])
     return load_library().lq_decode_attn_image_static(C.byref(st), _ptr(q), sm_scale, _ptr(out), _stream(stream))

@@ -28,6 +28,7 @@ static __device__ __align__(256) float g_static_partials[kStaticMaxRecords * kRe
 
 struct ImageArgs {
   int B, Hq, Hkv, G, n_fp, S;
+  int bits;  // 2 or 4: width of a code in k_codes / v_codes
   long long n_quant;
   const uint16_t *fp_k, *fp_v, *k_scale, *k_zero, *v_scale, *v_zero;
   const uint8_t *k_codes, *v_codes;
@@ -39,10 +40,17 @@ struct ImageArgs {
 
 __device__ __forceinline__ float bf16f(uint16_t b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }
 
+// code of channel d of token row `row` in the canonical packing: 8 / bits codes per byte, channel (8/bits)*j + i of
+// a token in bits [bits*i + bits - 1 : bits*i] of byte j
+__device__ __forceinline__ uint32_t image_code(const uint8_t* codes, int bits, long long row, int d) {
+  const int per_byte = 8 / bits;
+  return (codes[row * (kD / per_byte) + d / per_byte] >> (bits * (d % per_byte))) & ((1u << bits) - 1u);
+}
+
 __device__ __forceinline__ float image_k(const ImageArgs& a, long long pair, long long t, int d) {
   if (t < a.n_fp) return bf16f(a.fp_k[(pair * a.n_fp + t) * kD + d]);
   const long long tq = t - a.n_fp;
-  const uint32_t code = (a.k_codes[(pair * a.n_quant + tq) * (kD / 4) + d / 4] >> (2 * (d & 3))) & 3u;
+  const uint32_t code = image_code(a.k_codes, a.bits, pair * a.n_quant + tq, d);
   const long long grp = (pair * (a.n_quant / a.G) + tq / a.G) * kD + d;
   return fmaf(static_cast<float>(code), bf16f(a.k_scale[grp]), bf16f(a.k_zero[grp]));
 }
@@ -50,7 +58,7 @@ __device__ __forceinline__ float image_k(const ImageArgs& a, long long pair, lon
 __device__ __forceinline__ float image_v(const ImageArgs& a, long long pair, long long t, int d) {
   if (t < a.n_fp) return bf16f(a.fp_v[(pair * a.n_fp + t) * kD + d]);
   const long long tq = t - a.n_fp;
-  const uint32_t code = (a.v_codes[(pair * a.n_quant + tq) * (kD / 4) + d / 4] >> (2 * (d & 3))) & 3u;
+  const uint32_t code = image_code(a.v_codes, a.bits, pair * a.n_quant + tq, d);
   const long long grp = (pair * a.n_quant + tq) * (kD / a.G) + d / a.G;
   return fmaf(static_cast<float>(code), bf16f(a.v_scale[grp]), bf16f(a.v_zero[grp]));
 }
@@ -164,6 +172,7 @@ extern "C" lq_status_t lq_decode_attn_image_static(const lq_device_image_t* img,
   if (img->batch < 1 || img->n_q_heads < 1 || img->n_kv_heads < 1 || img->n_q_heads % img->n_kv_heads ||
       img->n_fp < 0 || img->n_quant < 0 || img->n_fp + img->n_quant < 1)
     return LQ_ERR_INVALID_ARG;
+  if (img->bits != 2 && img->bits != 4) return LQ_ERR_INVALID_ARG;
   if (img->head_dim != kD || (img->group != 32 && img->group != 64) || img->n_q_heads / img->n_kv_heads > kMaxR ||
       img->n_quant % img->group)
     return LQ_ERR_UNSUPPORTED;
@@ -193,7 +202,7 @@ extern "C" lq_status_t lq_decode_attn_image_static(const lq_device_image_t* img,
   }
 
   ImageArgs a;
-  a.B = img->batch; a.Hq = img->n_q_heads; a.Hkv = img->n_kv_heads; a.G = img->group;
+  a.B = img->batch; a.Hq = img->n_q_heads; a.Hkv = img->n_kv_heads; a.G = img->group; a.bits = img->bits;
   a.n_fp = img->n_fp; a.n_quant = img->n_quant; a.S = static_cast<int>(S);
   a.fp_k = img->fp_k; a.fp_v = img->fp_v; a.k_codes = img->k_codes; a.v_codes = img->v_codes;
   a.k_scale = img->k_scale; a.k_zero = img->k_zero; a.v_scale = img->v_scale; a.v_zero = img->v_zero;

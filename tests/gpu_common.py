@@ -64,8 +64,7 @@ def run_case(B, Hq, Hkv, W, G, n_prefill, n_steps, seed, kernel, n_outliers=3, c
     worst = 0.0
     scale = sm_scale if sm_scale > 0 else 1.0 / np.sqrt(D)
     for step in range(n_steps):
-        if step or n_prefill == 0 or True:
-            feed(n_prefill + step, 1)
+        feed(n_prefill + step, 1)
         inf = cache.info(0)
         assert (inf.n_seen, inf.n_fp, inf.n_quant, inf.n_events) == (oc.n_seen, oc.n_fp, oc.n_quant, oc.n_events)
         if check_image_every and step % check_image_every == 0:

@@ -1,6 +1,9 @@
-"""GPU parity at the full sizes of the benchmark configurations (one layer cache each), in the launch
-configuration bench.py times (default kernel, library-chosen split count): bit-exact canonical image
-and attention within tolerance against the float64 oracle for every (batch row, head)."""
+"""GPU parity at the full sizes of the benchmark configurations (one layer cache each), default kernel and
+library-chosen split count: bit-exact canonical image and attention within tolerance against the float64
+oracle for every (batch row, head).  The first group of tests drives decode through lq_append + lq_decode_attn;
+the `timed entry point` tests drive it through the calls bench.py times -- lq_append_decode_attn (append and
+attention in one launch) and lq_decode_step_host (host buffers, pinned and pageable) -- over 128 and more
+decode steps with one window overflow in the middle of the run."""
 import numpy as np
 import pytest
 import torch
@@ -107,3 +110,80 @@ def test_config4_left_padded_batch():
     inf = _run(B=4, Hq=28, Hkv=4, W=256, G=64, ctx=32768, seed=7, n_steps=1, n_outliers=0, planted=True,
                pad=[0, 31, 16385, 32700])
     assert (inf.n_quant, inf.n_fp) == (32256, 513)
+
+
+# ---- the entry points bench.py times, at full size -------------------------------------------------
+def _run_timed_entry(entry, B, Hq, Hkv, W, G, ctx, seed, check_steps, n_outliers=3, planted=False):
+    """Prefill ctx tokens, then max(check_steps) decode steps through `entry`: "fused" = lq_append_decode_attn,
+    "host_pinned" / "host_pageable" = lq_decode_step_host.  Steps are counted from 1; on the steps named in
+    check_steps the image and the attention output are compared with the oracle, on the others only the
+    bookkeeping (so that an overflow step in between is crossed by both sides)."""
+    dev = "cuda"
+    n_steps = max(check_steps)
+    total = ctx + n_steps
+    outl = synth.outlier_channels(seed, Hkv, D, n_outliers) if n_outliers else None
+    u = synth.unit_vectors(seed, Hkv, D) if planted else None
+    cache = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=total + 8)
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G)
+    chunk = 2048
+    for t0 in range(0, ctx, chunk):
+        n = min(chunk, ctx - t0)
+        k, v = synth.keys_values(seed, B, Hkv, n, D, dev, token_start=t0, token_total=total, outliers=outl)
+        if u is not None:
+            k = synth.plant_spikes(k, u, 16.0, t0, ctx)
+        cache.append(0, k, v)
+        oc.append(synth.bf16_bits(k), synth.bf16_bits(v))
+    events0 = oc.n_events
+    host = entry.startswith("host")
+    pin = (lambda t: t.cpu().pin_memory()) if entry == "host_pinned" else (lambda t: t.cpu())
+    out = torch.full((B, Hq, D), float("nan"), device=dev)
+    out_host = torch.full((B, Hq, D), float("nan"))
+    if entry == "host_pinned":
+        out_host = out_host.pin_memory()
+    for step in range(1, n_steps + 1):
+        k, v = synth.keys_values(seed, B, Hkv, 1, D, dev, token_start=ctx + step - 1, token_total=total, outliers=outl)
+        q = synth.queries(seed, B, Hq, D, step, dev)
+        if u is not None:
+            q = (q.float() + 4.0 * u.to(dev).repeat_interleave(Hq // Hkv, dim=0)[None]).to(torch.bfloat16)
+        if host:
+            cache.decode_step_host(0, pin(k), pin(v), pin(q), out_host, sync=True)
+            got = out_host.numpy().astype(np.float64)
+        else:
+            cache.append_decode_attn(0, k, v, q, out)
+        oc.append(synth.bf16_bits(k), synth.bf16_bits(v))
+        inf = cache.info(0)
+        assert (inf.n_seen, inf.n_fp, inf.n_quant, inf.n_events) == (oc.n_seen, oc.n_fp, oc.n_quant, oc.n_events)
+        if step not in check_steps:
+            continue
+        if not host:
+            torch.cuda.synchronize()
+            got = out.cpu().numpy().astype(np.float64)
+        assert_images_equal(cache.export(0), oc.export())
+        ref = oc.attention(synth.bf16_bits(q), 1 / np.sqrt(D), n_threads=16)
+        err, tol = float(np.abs(got - ref).max()), attn_tolerance(ref)
+        assert np.isfinite(got).all() and err <= tol, f"{entry} step {step}: max|delta| {err:.3e} > {tol:.3e}"
+    assert cache.kernel_status() == 0
+    return oc.n_events - events0
+
+
+@pytest.mark.parametrize("entry", ["fused", "host_pinned", "host_pageable"])
+def test_config2_timed_entry_points_over_128_steps(entry):
+    # the prompt is W/2 tokens short of 8192, so the overflow step falls on decode step 65: steps 1, 2 and 64
+    # come before it, 65 is the step that runs it, 128 well after it
+    events = _run_timed_entry(entry, B=8, Hq=32, Hkv=8, W=128, G=32, ctx=8192 - 64, seed=2,
+                              check_steps=[1, 2, 64, 65, 128])
+    assert events == 1
+
+
+def test_config2_fused_entry_point_overflow_on_the_first_step():
+    # full 8192-token prompt: the bf16 window is exactly full, the first decode step runs the overflow step
+    events = _run_timed_entry("fused", B=8, Hq=32, Hkv=8, W=128, G=32, ctx=8192, seed=2, check_steps=[1, 2, 64, 128])
+    assert events == 1
+
+
+@pytest.mark.parametrize("entry", ["fused", "host_pinned"])
+def test_config4_timed_entry_points_across_an_overflow(entry):
+    # W = 256: with the prompt W/2 short the overflow step falls on decode step 129
+    events = _run_timed_entry(entry, B=4, Hq=28, Hkv=4, W=256, G=64, ctx=32768 - 128, seed=4,
+                              check_steps=[1, 2, 64, 128, 129, 130], n_outliers=0, planted=True)
+    assert events == 1

@@ -39,3 +39,29 @@ def test_two_ranks_report_units_of_all_ranks_over_the_slowest_time():
             ms_max, value = out[rank]
             assert ms_max == [15.0, 100.0]
             assert abs(value - 2 * 1000 / 15e-3) < 1e-6
+
+
+def test_gpus_flag_without_a_launcher_starts_that_many_replica_ranks():
+    """`bench.py --gpus 2` with no WORLD_SIZE in the environment re-runs itself as two ranks; the CPU-only
+    self-test arm takes them through the same max-over-ranks reduction as the real run (gloo, no GPU)."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR",
+                                                            "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "replica-selftest"],
+                         capture_output=True, text=True, env=env, timeout=300)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [json.loads(l) for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1  # rank 0 alone prints
+    assert lines[0]["n_gpus"] == 2 and lines[0]["ms_per_step"] == 15.0
+    assert abs(lines[0]["value"] - 2 * 1000 / 15e-3) < 1e-6
+
+
+def test_gpus_flag_fails_loudly_without_that_many_devices():
+    import subprocess
+    if torch.cuda.device_count() >= 2:
+        return
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "1"],
+                         capture_output=True, text=True, env=env, timeout=300)
+    assert res.returncode != 0 and "CUDA device" in res.stderr
