@@ -57,6 +57,8 @@ typedef enum {
 #define LQ_KERNEL_AUTO 0   /* the tensor-core kernel                                             */
 #define LQ_KERNEL_SCALAR 1 /* plain fp32 FMA kernel (slow; kept as an independent cross-check)   */
 #define LQ_KERNEL_MMA 2    /* mma.sync tensor-core kernel with bulk-copy staging                 */
+#define LQ_KERNEL_UMMA 3   /* tcgen05 kernel: codes unpacked into tensor memory, accumulators in tensor memory
+                              (bits = 2 only; the cache then uses the device layout made for it)  */
 
 /* Which tokens an overflow step removes from the 3W full-precision tokens (in age order A[0..3W)):
  *   LQ_FILTER_LOG     Algorithm 1: A[1], A[3], ..., A[2W-1]; kept tokens thin out with distance.

@@ -10,7 +10,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "liblogquant.so")
 
 LQ_DEVICE_NONE = -1
-LQ_KERNEL_AUTO, LQ_KERNEL_SCALAR, LQ_KERNEL_MMA = 0, 1, 2
+LQ_KERNEL_AUTO, LQ_KERNEL_SCALAR, LQ_KERNEL_MMA, LQ_KERNEL_UMMA = 0, 1, 2, 3
 LQ_FILTER_LOG, LQ_FILTER_RECENT = 0, 1
 LQ_OK, LQ_ERR_INVALID_ARG, LQ_ERR_UNSUPPORTED, LQ_ERR_OOM, LQ_ERR_WINDOW_FULL, LQ_ERR_NOT_FULL, \
     LQ_ERR_CAPACITY, LQ_ERR_CUDA = range(8)

@@ -301,7 +301,7 @@ lq_status_t run_events(lq_cache* c, const std::vector<int>& full_layers, cudaStr
   return LQ_OK;
 }
 
-bool use_mma(const lq_cache* c) { return c->cfg.kernel != LQ_KERNEL_SCALAR; }
+bool use_mma(const lq_cache* c) { return c->cfg.kernel == LQ_KERNEL_AUTO || c->cfg.kernel == LQ_KERNEL_MMA; }
 
 // Padding masks of one layer from the host mirror of its stores (which token id sits in which fp slot and at
 // which place of the quantised store) and upload.  Rows appended later lie beyond the rebuilt prefix of the fp
@@ -403,7 +403,8 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
   if (cfg->bits == 4 && cfg->group != 32) return LQ_ERR_UNSUPPORTED;  // a 4-bit tile of G = 64 exceeds a stage
   if (cfg->window > kMaxW) return LQ_ERR_UNSUPPORTED;
   if (cfg->n_q_heads / cfg->n_kv_heads > kMaxRatio || cfg->n_layers > 128) return LQ_ERR_UNSUPPORTED;
-  if (cfg->kernel < LQ_KERNEL_AUTO || cfg->kernel > LQ_KERNEL_MMA) return LQ_ERR_INVALID_ARG;
+  if (cfg->kernel < LQ_KERNEL_AUTO || cfg->kernel > LQ_KERNEL_UMMA) return LQ_ERR_INVALID_ARG;
+  if (cfg->kernel == LQ_KERNEL_UMMA && cfg->bits != 2) return LQ_ERR_UNSUPPORTED;
   if (cfg->filter != LQ_FILTER_LOG && cfg->filter != LQ_FILTER_RECENT) return LQ_ERR_INVALID_ARG;
 
   lq_cache* c = new (std::nothrow) lq_cache;
@@ -416,12 +417,13 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
   std::memset(&cv, 0, sizeof cv);
   cv.B = cfg->batch; cv.Hq = cfg->n_q_heads; cv.Hkv = cfg->n_kv_heads; cv.G = G; cv.W = W;
   cv.planes = cfg->bits / 2;
+  cv.layout = cfg->kernel == LQ_KERNEL_UMMA ? kLayoutRow : kLayoutFragment;
   cv.quant_tiles_cap = (cfg->max_tokens + G - 1) / G;
   cv.quant_head_stride = cv.quant_tiles_cap * quant_tile_bytes(G, cv.planes);
   cv.quant_layer_stride = cv.quant_head_stride * pairs;
   // W % G != 0: up to G - 1 removed tokens wait in the fp store for a full key group
   const int fp_slots = 3 * W + (W % G ? G : 0);
-  cv.fp_head_stride = static_cast<int64_t>((fp_slots + kFpTileSlots - 1) / kFpTileSlots) * kFpTileBytes;
+  cv.fp_head_stride = fp_store_bytes(cv.layout, fp_slots);
   cv.fp_layer_stride = cv.fp_head_stride * pairs;
   c->layers.resize(cfg->n_layers);
   for (auto& L : c->layers) L.slot_token.assign(3 * W + G, -1);

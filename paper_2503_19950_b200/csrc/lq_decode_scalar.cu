@@ -20,38 +20,39 @@ struct TokenRef {  // where token t of the unified index space [fp tokens | quan
   int n_fp;
   int G;
   int P;  // 2-bit planes per code
+  int layout;
 };
 
 __device__ __forceinline__ float load_k(const TokenRef& r, int64_t t, int d) {
-  if (t < r.n_fp) return bf16f(*reinterpret_cast<const uint16_t*>(r.fp + fp_elem_off(static_cast<int>(t), d)));
+  if (t < r.n_fp) return bf16f(*reinterpret_cast<const uint16_t*>(r.fp + fp_elem_off(r.layout, static_cast<int>(t), d)));
   const int64_t tq = t - r.n_fp;
   const uint8_t* tile = r.quant + (tq / r.G) * quant_tile_bytes(r.G, r.P);
-  int word, bit;
-  kcode_pos(static_cast<int>(tq % r.G), d, word, bit);
   uint32_t code = 0;
-  for (int pl = 0; pl < r.P; ++pl)
-    code |= ((reinterpret_cast<const uint32_t*>(tile + qt_kcodes_off() + pl * qt_plane_bytes(r.G))[word] >> bit) & 3u)
-            << (2 * pl);
-  const float s = bf16f(reinterpret_cast<const uint16_t*>(tile + qt_kscale_off())[kparam_index(d)]);
-  const float z = bf16f(reinterpret_cast<const uint16_t*>(tile + qt_kzero_off())[d]);
+  for (int pl = 0; pl < r.P; ++pl) {
+    int off, bit;
+    kcode_pos(r.layout, r.G, r.P, pl, static_cast<int>(tq % r.G), d, off, bit);
+    code |= ((*reinterpret_cast<const uint32_t*>(tile + off) >> bit) & 3u) << (2 * pl);
+  }
+  const float s = bf16f(*reinterpret_cast<const uint16_t*>(tile + kscale_off(r.layout, r.G, d)));
+  const float z = bf16f(*reinterpret_cast<const uint16_t*>(tile + kzero_off(r.layout, r.G, d)));
   return fmaf(static_cast<float>(code), s, z);
 }
 
 __device__ __forceinline__ float load_v(const TokenRef& r, int64_t t, int d) {
   if (t < r.n_fp)
-    return bf16f(*reinterpret_cast<const uint16_t*>(r.fp + kFpTileVOffset + fp_elem_off(static_cast<int>(t), d)));
+    return bf16f(*reinterpret_cast<const uint16_t*>(r.fp + fp_v_delta(r.layout) + fp_elem_off(r.layout, static_cast<int>(t), d)));
   const int64_t tq = t - r.n_fp;
   const uint8_t* tile = r.quant + (tq / r.G) * quant_tile_bytes(r.G, r.P);
   const int tt = static_cast<int>(tq % r.G);
-  int word, bit;
-  vcode_pos(tt, d, word, bit);
   uint32_t code = 0;
-  for (int pl = 0; pl < r.P; ++pl)
-    code |= ((reinterpret_cast<const uint32_t*>(tile + qt_vcodes_off(r.G, r.P) + pl * qt_plane_bytes(r.G))[word] >> bit) & 3u)
-            << (2 * pl);
+  for (int pl = 0; pl < r.P; ++pl) {
+    int off, bit;
+    vcode_pos(r.layout, r.G, r.P, pl, tt, d, off, bit);
+    code |= ((*reinterpret_cast<const uint32_t*>(tile + off) >> bit) & 3u) << (2 * pl);
+  }
   const int g = d / r.G;
-  const float s = bf16f(reinterpret_cast<const uint16_t*>(tile + qt_vscale_off(r.G, r.P))[vscale_index(tt, g, r.G)]);
-  const float z = bf16f(reinterpret_cast<const uint16_t*>(tile + qt_vzero_off(r.G, r.P))[vzero_index(tt, g, r.G)]);
+  const float s = bf16f(*reinterpret_cast<const uint16_t*>(tile + vscale_off(r.layout, r.G, r.P, tt, g)));
+  const float z = bf16f(*reinterpret_cast<const uint16_t*>(tile + vzero_off(r.layout, r.G, r.P, tt, g)));
   return fmaf(static_cast<float>(code), s, z);
 }
 
@@ -81,6 +82,7 @@ __global__ void __launch_bounds__(128) lq_decode_scalar_kernel(DecodeArgs a) {
   ref.n_fp = a.n_fp;
   ref.G = cv.G;
   ref.P = cv.planes;
+  ref.layout = cv.layout;
 
   const int64_t T = a.n_fp + a.n_quant;
   const int64_t chunk = (T + S - 1) / S;

@@ -11,6 +11,7 @@ namespace lq {
 struct CacheView {
   int B, Hq, Hkv, G, W;
   int planes;                 // 2-bit code planes per code: 1 (2-bit cache) or 2 (4-bit cache)
+  int layout;                 // kLayoutFragment (mma.sync kernel) or kLayoutRow (tcgen05 kernel), see lq_layout.cuh
   int64_t quant_tiles_cap;    // capacity in tiles per (layer, b, kv)
   int64_t quant_head_stride;  // bytes between (b, kv) heads of the 2-bit store
   int64_t quant_layer_stride;

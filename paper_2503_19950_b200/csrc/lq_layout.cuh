@@ -107,4 +107,94 @@ __host__ __device__ inline int vzero_index(int t, int g, int G) {
   return u * (vsz_subtile_bytes(G) / 2) + 2 * word + h;
 }
 
+
+// =======================================================================================
+// Layout 1 (kLayoutRow): the layout of the tcgen05 decode kernel (LQ_KERNEL_UMMA).  Same bytes per
+// token as layout 0, but every packed word holds 16 codes of ONE row of a tensor-core A operand, so
+// that the thread that owns the row (a token for q.k, a channel for p.v) unpacks it on its own and
+// writes it to tensor memory.
+//
+// Full-precision store, per (layer, b, kv head): "fp units" of 32 slots, 16 KB each:
+//   [K rows 8 KB][V rows 8 KB]; inside either half the 16-byte chunk c (8 channels) of slot s sits at
+//   (s/8)*2048 + c*128 + (s%8)*16: groups of 8 slots, chunk-major inside a group.  Read by the tensor
+//   core straight from shared memory in the canonical no-swizzle form, as a K-major A operand for q.k
+//   (rows = tokens: 8-row groups 2048 B apart, 16-byte k-chunks 128 B apart) and as an MN-major A
+//   operand for p.v (rows = channels: 8-channel chunks 128 B apart, 8-token groups 2048 B apart).
+//
+// 2-bit store: one tile per key group of G tokens, 1024 + 64 G bytes as in layout 0 (planes == 1 only):
+//     0            K codes: [half (2)][token (G)][4 words]; word j of half hf holds channels
+//                  16*(4hf+j) .. +15 of the token
+//     32 G         V codes: [channel (128)][G/16 words]; word j holds tokens 16j .. 16j+15 of the channel
+//     64 G         K scale, 128 bf16 in channel order;  64 G + 256: K zero likewise
+//     64 G + 512   V scale and zero per token: [token (G)][scale of group 0..NG-1, zero of group 0..NG-1]
+//   Inside a code word element e (0..15) of the row sits at bit 16*(e&1) + 8*(e>>3) + 2*((e>>1)&3):
+//   masking the word (or the word shifted right by 8) with 0x00030003 << 2i yields elements 2i', 2i'+1
+//   as a pair of bf16 subnormals, i.e. one 32-bit column of the A operand of k-step (word), times 2^(2i).
+// =======================================================================================
+constexpr int kLayoutFragment = 0;
+constexpr int kLayoutRow = 1;
+constexpr int kFpUnitSlots = 32;
+constexpr int kFpUnitBytes = 2 * kFpUnitSlots * kD * 2;
+constexpr int kFpUnitVOffset = kFpUnitSlots * kD * 2;
+
+__host__ __device__ constexpr int row_kcodes_off() { return 0; }
+__host__ __device__ constexpr int row_vcodes_off(int G) { return 32 * G; }
+__host__ __device__ constexpr int row_kscale_off(int G) { return 64 * G; }
+__host__ __device__ constexpr int row_kzero_off(int G) { return 64 * G + 256; }
+__host__ __device__ constexpr int row_vsz_off(int G) { return 64 * G + 512; }
+// bit of element e (0..15) inside a code word
+__host__ __device__ constexpr int row_code_bit(int e) { return 16 * (e & 1) + 8 * (e >> 3) + 2 * ((e >> 1) & 3); }
+
+// ---- layout-generic element addressing (overflow, ingestion, export and scalar kernels) ----
+// bytes between the K row and the V row of a slot
+__host__ __device__ inline int fp_v_delta(int layout) { return layout == kLayoutRow ? kFpUnitVOffset : kFpTileVOffset; }
+__host__ __device__ inline int64_t fp_store_bytes(int layout, int slots) {
+  return layout == kLayoutRow ? static_cast<int64_t>((slots + kFpUnitSlots - 1) / kFpUnitSlots) * kFpUnitBytes
+                              : static_cast<int64_t>((slots + kFpTileSlots - 1) / kFpTileSlots) * kFpTileBytes;
+}
+__host__ __device__ inline int64_t fp_chunk_off(int layout, int slot, int c) {
+  if (layout == kLayoutRow)
+    return static_cast<int64_t>(slot >> 5) * kFpUnitBytes + ((slot & 31) >> 3) * 2048 + c * 128 + (slot & 7) * 16;
+  return fp_chunk_off(slot, c);
+}
+__host__ __device__ inline int64_t fp_elem_off(int layout, int slot, int d) {
+  return layout == kLayoutRow ? fp_chunk_off(layout, slot, d >> 3) + (d & 7) * 2 : fp_elem_off(slot, d);
+}
+// byte offset (in the tile) of the 32-bit word and the bit position of the K / V code of (token t, channel d)
+__host__ __device__ inline void kcode_pos(int layout, int G, int P, int pl, int t, int d, int& byte_off, int& bit) {
+  if (layout == kLayoutRow) {
+    const int ks = d >> 4;
+    byte_off = row_kcodes_off() + 4 * ((ks >> 2) * (G * 4) + t * 4 + (ks & 3));
+    bit = row_code_bit(d & 15);
+  } else {
+    int word;
+    kcode_pos(t, d, word, bit);
+    byte_off = qt_kcodes_off() + pl * qt_plane_bytes(G) + 4 * word;
+  }
+}
+__host__ __device__ inline void vcode_pos(int layout, int G, int P, int pl, int t, int d, int& byte_off, int& bit) {
+  if (layout == kLayoutRow) {
+    byte_off = row_vcodes_off(G) + 4 * (d * (G / 16) + (t >> 4));
+    bit = row_code_bit(t & 15);
+  } else {
+    int word;
+    vcode_pos(t, d, word, bit);
+    byte_off = qt_vcodes_off(G, P) + pl * qt_plane_bytes(G) + 4 * word;
+  }
+}
+// byte offsets (in the tile) of the bf16 scale / zero of key channel d, and of value (token t, group g)
+__host__ __device__ inline int kscale_off(int layout, int G, int d) {
+  return layout == kLayoutRow ? row_kscale_off(G) + 2 * d : qt_kscale_off() + 2 * kparam_index(d);
+}
+__host__ __device__ inline int kzero_off(int layout, int G, int d) {
+  return layout == kLayoutRow ? row_kzero_off(G) + 2 * d : qt_kzero_off() + 2 * d;
+}
+__host__ __device__ inline int vscale_off(int layout, int G, int P, int t, int g) {
+  return layout == kLayoutRow ? row_vsz_off(G) + 2 * (t * (2 * (kD / G)) + g) : qt_vscale_off(G, P) + 2 * vscale_index(t, g, G);
+}
+__host__ __device__ inline int vzero_off(int layout, int G, int P, int t, int g) {
+  return layout == kLayoutRow ? row_vsz_off(G) + 2 * (t * (2 * (kD / G)) + kD / G + g)
+                              : qt_vzero_off(G, P) + 2 * vzero_index(t, g, G);
+}
+
 }  // namespace lq

@@ -33,7 +33,7 @@ lq_append_kernel(CacheView cv, int layer, const uint4* __restrict__ k, const uin
   const int64_t pair = row / n;
   const uint4* src = (which ? v : k) + ((pair * n_src + src0 + t) * 16 + c);
   uint8_t* base = cv.fp + layer * cv.fp_layer_stride + pair * cv.fp_head_stride;
-  const int64_t off = fp_chunk_off(slot0 + t, c) + (which ? kFpTileVOffset : 0);
+  const int64_t off = fp_chunk_off(cv.layout, slot0 + t, c) + (which ? fp_v_delta(cv.layout) : 0);
   *reinterpret_cast<uint4*>(base + off) = *src;
 }
 
@@ -100,7 +100,8 @@ __device__ __forceinline__ void group_params(float mn, float mx, float top, uint
 // Steps 3 and 4 of the overflow step for one key group whose G rows sit in shared memory
 // (sK, sV: [G][128] bf16 bits; overwritten by the codes).  256 threads.
 template <int G, int P>
-__device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kD], uint16_t (&sV)[G][kD], uint8_t* tile, int tid) {
+__device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kD], uint16_t (&sV)[G][kD], uint8_t* tile, int tid,
+                                                   int layout) {
   constexpr int NS = G / 16;
   constexpr float kTop = P == 1 ? 3.0f : 15.0f;
   // 3. quantise
@@ -116,8 +117,8 @@ __device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kD], uint16
     uint16_t sb, zb;
     float mnc, scale;
     group_params(mn, mx, kTop, sb, zb, mnc, scale);
-    reinterpret_cast<uint16_t*>(tile + qt_kscale_off())[kparam_index(d)] = sb;
-    reinterpret_cast<uint16_t*>(tile + qt_kzero_off())[d] = zb;
+    *reinterpret_cast<uint16_t*>(tile + kscale_off(layout, G, d)) = sb;
+    *reinterpret_cast<uint16_t*>(tile + kzero_off(layout, G, d)) = zb;
 #pragma unroll 4
     for (int e = 0; e < G; ++e)
       sK[e][d] = static_cast<uint16_t>(quant_code(bf16_bits_to_float(sK[e][d]), mnc, scale, kTop));
@@ -140,8 +141,8 @@ __device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kD], uint16
       group_params(mn, mx, kTop, sb, zb, mnc, scale);
       if ((lane % LPG) == 0) {
         const int g = lane / LPG;
-        reinterpret_cast<uint16_t*>(tile + qt_vscale_off(G, P))[vscale_index(e, g, G)] = sb;
-        reinterpret_cast<uint16_t*>(tile + qt_vzero_off(G, P))[vzero_index(e, g, G)] = zb;
+        *reinterpret_cast<uint16_t*>(tile + vscale_off(layout, G, P, e, g)) = sb;
+        *reinterpret_cast<uint16_t*>(tile + vzero_off(layout, G, P, e, g)) = zb;
       }
 #pragma unroll
       for (int i = 0; i < 4; ++i)
@@ -150,7 +151,26 @@ __device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kD], uint16
   }
   __syncthreads();
 
-  // 4. pack into fragment order, one 2-bit plane after the other
+  // 4. pack
+  if (layout == kLayoutRow) {
+    // one word = 16 codes of one row: K words [half][token][4], V words [channel][G/16]
+    for (int idx = tid; idx < 2 * G * 8; idx += 256) {
+      uint32_t word = 0;
+      if (idx < G * 8) {
+        const int hf = idx / (G * 4), t = (idx >> 2) % G, ks = 4 * hf + (idx & 3);
+#pragma unroll
+        for (int e = 0; e < 16; ++e) word |= static_cast<uint32_t>(sK[t][16 * ks + e] & 3u) << row_code_bit(e);
+        reinterpret_cast<uint32_t*>(tile + row_kcodes_off())[idx] = word;
+      } else {
+        const int wd = idx - G * 8, d = wd / (G / 16), j = wd % (G / 16);
+#pragma unroll
+        for (int e = 0; e < 16; ++e) word |= static_cast<uint32_t>(sV[16 * j + e][d] & 3u) << row_code_bit(e);
+        reinterpret_cast<uint32_t*>(tile + row_vcodes_off(G))[wd] = word;
+      }
+    }
+    return;
+  }
+  // fragment order, one 2-bit plane after the other
   for (int idx = tid; idx < 2 * P * NS * 128; idx += 256) {
     const int which = idx / (P * NS * 128);
     const int pl = (idx / (NS * 128)) % P;
@@ -199,8 +219,8 @@ lq_compress_kernel(CacheView cv, LayerList layers, EvictList ev, int64_t tile0) 
   for (int idx = tid; idx < G * 32; idx += 256) {
     const int c = idx & 15, which = (idx >> 4) & 1, e = idx >> 5;
     const int slot = ev.slot[tau * G + e];
-    const uint4 val = *reinterpret_cast<const uint4*>(fpbase + fp_chunk_off(slot, c) +
-                                                      (which ? kFpTileVOffset : 0));
+    const uint4 val = *reinterpret_cast<const uint4*>(fpbase + fp_chunk_off(cv.layout, slot, c) +
+                                                      (which ? fp_v_delta(cv.layout) : 0));
     *reinterpret_cast<uint4*>(which ? &sV[e][c * 8] : &sK[e][c * 8]) = val;
   }
   __syncthreads();
@@ -211,12 +231,12 @@ lq_compress_kernel(CacheView cv, LayerList layers, EvictList ev, int64_t tile0) 
     const int dst = ev.slot[tau * G + e];
     const int src = ev.src[tau * G + e];
     if (src == kNoMove) continue;
-    const int vo = which ? kFpTileVOffset : 0;
-    const uint4 val = *reinterpret_cast<const uint4*>(fpbase + fp_chunk_off(src, c) + vo);
-    *reinterpret_cast<uint4*>(fpbase + fp_chunk_off(dst, c) + vo) = val;
+    const int vo = which ? fp_v_delta(cv.layout) : 0;
+    const uint4 val = *reinterpret_cast<const uint4*>(fpbase + fp_chunk_off(cv.layout, src, c) + vo);
+    *reinterpret_cast<uint4*>(fpbase + fp_chunk_off(cv.layout, dst, c) + vo) = val;
   }
 
-  quantise_pack_tile<G, P>(sK, sV, tile, tid);
+  quantise_pack_tile<G, P>(sK, sV, tile, tid, cv.layout);
 }
 
 cudaError_t launch_compress(const CacheView& cv, const LayerList& layers, const EvictList& ev,
@@ -261,14 +281,14 @@ lq_ingest_kernel(CacheView cv, int layer, const uint4* __restrict__ k, const uin
       *reinterpret_cast<uint4*>(which ? &sV[e][c * 8] : &sK[e][c * 8]) = val;
     }
     __syncthreads();
-    quantise_pack_tile<G, P>(sK, sV, tile, tid);
+    quantise_pack_tile<G, P>(sK, sV, tile, tid, cv.layout);
   } else {
     const int i = (static_cast<int>(blockIdx.x) - n_tiles) * 256 + tid;
     if (i >= n_fp * 32) return;
     const int c = i & 15, which = (i >> 4) & 1, slot = i >> 5;
     const int64_t t = idx[n_tiles * G + slot];
     uint8_t* base = cv.fp + layer * cv.fp_layer_stride + pair * cv.fp_head_stride;
-    *reinterpret_cast<uint4*>(base + fp_chunk_off(slot, c) + (which ? kFpTileVOffset : 0)) =
+    *reinterpret_cast<uint4*>(base + fp_chunk_off(cv.layout, slot, c) + (which ? fp_v_delta(cv.layout) : 0)) =
         (which ? v : k)[(pair * n_src + t) * 16 + c];
   }
 }
@@ -311,13 +331,11 @@ __global__ void lq_export_codes_kernel(CacheView cv, int layer, int64_t n_quant,
     for (int i = 0; i < cpb; ++i) {
       uint32_t kcode = 0, vcode = 0;
       for (int pl = 0; pl < P; ++pl) {
-        const uint32_t* kw = reinterpret_cast<const uint32_t*>(tile + qt_kcodes_off() + pl * qt_plane_bytes(cv.G));
-        const uint32_t* vw = reinterpret_cast<const uint32_t*>(tile + qt_vcodes_off(cv.G, P) + pl * qt_plane_bytes(cv.G));
-        int word, bit;
-        kcode_pos(t, cpb * jb + i, word, bit);
-        kcode |= ((kw[word] >> bit) & 3u) << (2 * pl);
-        vcode_pos(t, cpb * jb + i, word, bit);
-        vcode |= ((vw[word] >> bit) & 3u) << (2 * pl);
+        int off, bit;
+        kcode_pos(cv.layout, cv.G, P, pl, t, cpb * jb + i, off, bit);
+        kcode |= ((*reinterpret_cast<const uint32_t*>(tile + off) >> bit) & 3u) << (2 * pl);
+        vcode_pos(cv.layout, cv.G, P, pl, t, cpb * jb + i, off, bit);
+        vcode |= ((*reinterpret_cast<const uint32_t*>(tile + off) >> bit) & 3u) << (2 * pl);
       }
       kb |= kcode << (2 * P * i);
       vb |= vcode << (2 * P * i);
@@ -341,8 +359,8 @@ __global__ void lq_export_params_kernel(CacheView cv, int layer, int64_t n_quant
       const int64_t pair = idx / kD / (n_quant / G);
       const uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
                             grp * quant_tile_bytes(G, cv.planes);
-      if (k_scale) k_scale[idx] = reinterpret_cast<const uint16_t*>(tile + qt_kscale_off())[kparam_index(d)];
-      if (k_zero) k_zero[idx] = reinterpret_cast<const uint16_t*>(tile + qt_kzero_off())[d];
+      if (k_scale) k_scale[idx] = *reinterpret_cast<const uint16_t*>(tile + kscale_off(cv.layout, G, d));
+      if (k_zero) k_zero[idx] = *reinterpret_cast<const uint16_t*>(tile + kzero_off(cv.layout, G, d));
     } else {
       const int64_t i2 = idx - nk;
       const int g = static_cast<int>(i2 % NG);
@@ -351,8 +369,8 @@ __global__ void lq_export_params_kernel(CacheView cv, int layer, int64_t n_quant
       const uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
                             (tq / G) * quant_tile_bytes(G, cv.planes);
       const int t = static_cast<int>(tq % G);
-      if (v_scale) v_scale[i2] = reinterpret_cast<const uint16_t*>(tile + qt_vscale_off(G, cv.planes))[vscale_index(t, g, G)];
-      if (v_zero) v_zero[i2] = reinterpret_cast<const uint16_t*>(tile + qt_vzero_off(G, cv.planes))[vzero_index(t, g, G)];
+      if (v_scale) v_scale[i2] = *reinterpret_cast<const uint16_t*>(tile + vscale_off(cv.layout, G, cv.planes, t, g));
+      if (v_zero) v_zero[i2] = *reinterpret_cast<const uint16_t*>(tile + vzero_off(cv.layout, G, cv.planes, t, g));
     }
   }
 }
@@ -366,9 +384,9 @@ __global__ void lq_export_fp_kernel(CacheView cv, int layer, int n_fp, const int
     const int rank = static_cast<int>((idx >> 4) % n_fp);
     const int64_t pair = (idx >> 4) / n_fp;
     const uint8_t* base = cv.fp + layer * cv.fp_layer_stride + pair * cv.fp_head_stride;
-    const int64_t off = fp_chunk_off(slot_of_rank[rank], c);
+    const int64_t off = fp_chunk_off(cv.layout, slot_of_rank[rank], c);
     if (fp_k) fp_k[idx] = *reinterpret_cast<const uint4*>(base + off);
-    if (fp_v) fp_v[idx] = *reinterpret_cast<const uint4*>(base + off + kFpTileVOffset);
+    if (fp_v) fp_v[idx] = *reinterpret_cast<const uint4*>(base + off + fp_v_delta(cv.layout));
   }
 }
 
