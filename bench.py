@@ -52,6 +52,7 @@ WORKLOADS = {
     "tiny": dict(L=1, B=1, Hq=8, Hkv=2, W=128, G=32, ctx=1024, n_outliers=4, seed=1),
 }
 D = 128
+KERNELS = {"auto": 0, "scalar": 1, "mma": 2, "umma": 3}  # LQ_KERNEL_* of include/lq.h
 Q_ROTATE = 16  # distinct query/new-token sets cycled through the steps
 
 
@@ -171,7 +172,7 @@ def run_ours(args, wl, rank, world, device):
     total_steps = 2 * (steps + warmup) + steps + warmup + 8  # device-timed, profiled and host-buffer passes
     bits = wl.get("bits", 2)
     cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=ctx + total_steps + 8, device=device.index or 0, bits=bits,
-                          n_splits=args.n_splits)
+                          n_splits=args.n_splits, kernel=KERNELS[args.kernel])
     pad = wl.get("pad")
     n_pad = sum(pad) if pad else 0
     if pad:
@@ -353,7 +354,7 @@ def run_ours(args, wl, rank, world, device):
                 "api": "lq_decode_step_host (pinned host buffers, one stream sync per step)"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": None, "peak_kind": peak_kind,
-                     "kernel": "lq_decode_mma_kernel", "bytes_per_launch": bytes_per_launch,
+                     "kernel": "lq_decode_umma_kernel" if args.kernel == "umma" else "lq_decode_mma_kernel", "bytes_per_launch": bytes_per_launch,
                      "us_per_launch": b2b_us, "us_per_launch_best": b2b_best_us,
                      "timing": "median over %d rounds of %d back-to-back launches, one per layer cache" % (len(round_us), L),
                      "us_per_launch_isolated": isolated_us,
@@ -373,7 +374,7 @@ def run_ours(args, wl, rank, world, device):
     return line, cache
 
 
-def roofline_only(name, device, layers, rounds=24, n_splits=0):
+def roofline_only(name, device, layers, rounds=24, n_splits=0, kernel=0):
     """Back-to-back timing of the attention kernel on another workload (a few layer caches, a few seconds):
     the same measurement as the `roofline` object of the main line."""
     from paper_2503_19950_b200 import LogQuantCache
@@ -381,7 +382,7 @@ def roofline_only(name, device, layers, rounds=24, n_splits=0):
     wl["_outliers"] = synth.outlier_channels(wl["seed"], wl["Hkv"], D, wl["n_outliers"]) if wl["n_outliers"] else None
     L, B, Hq, Hkv, W, G, ctx = (wl[k] for k in ("L", "B", "Hq", "Hkv", "W", "G", "ctx"))
     cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=ctx + 64, device=device.index or 0, bits=wl.get("bits", 2),
-                          n_splits=n_splits)
+                          n_splits=n_splits, kernel=kernel)
     prefill(cache, wl, device)
     ks, vs, qs = make_step_inputs(wl, device, 4)
     outs = [torch.empty(B, Hq, D, device=device) for _ in range(L)]
@@ -544,6 +545,7 @@ def main():
     ap.add_argument("--shorten-prefill", type=int, default=0,
                     help="prefill this many tokens fewer than the workload's context (e.g. W/2: the overflow step then "
                          "falls in the middle of the timed steps instead of on the first decode step)")
+    ap.add_argument("--kernel", default="auto", choices=sorted(KERNELS), help="decode-attention kernel (LQ_KERNEL_*)")
     ap.add_argument("--also", default=None,
                     help="comma-separated workloads whose attention kernel is timed back to back as well and reported "
                          "under roofline_<workload> (default: gqa7-32k and llama3-8b-4k-b64 beside the default workload)")
@@ -602,7 +604,8 @@ def main():
     if rank == 0:
         for name in [n for n in args.also.split(",") if n]:
             try:
-                line["roofline_" + name.replace("-", "_")] = roofline_only(name, device, args.also_layers)
+                line["roofline_" + name.replace("-", "_")] = roofline_only(name, device, args.also_layers,
+                                                                           kernel=KERNELS[args.kernel])
             except Exception as exc:  # the main line stands without it
                 line["roofline_" + name.replace("-", "_")] = {"error": str(exc)}
         if not args.no_cpu_baseline:

@@ -302,6 +302,8 @@ lq_status_t run_events(lq_cache* c, const std::vector<int>& full_layers, cudaStr
 }
 
 bool use_mma(const lq_cache* c) { return c->cfg.kernel == LQ_KERNEL_AUTO || c->cfg.kernel == LQ_KERNEL_MMA; }
+// the tcgen05 kernel serves a call unless the batch is padded (that goes through the plain kernel on the same layout)
+bool use_umma(const lq_cache* c) { return c->cfg.kernel == LQ_KERNEL_UMMA && !c->has_pad; }
 
 // Padding masks of one layer from the host mirror of its stores (which token id sits in which fp slot and at
 // which place of the quantised store) and upload.  Rows appended later lie beyond the rebuilt prefix of the fp
@@ -437,6 +439,8 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
     c->max_splits = 1 + (cfg->n_splits > 0
                         ? cfg->n_splits
                         : static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(256, (8LL * c->sm_count + pairs - 1) / pairs))));
+    if (cfg->kernel == LQ_KERNEL_UMMA)  // the tcgen05 kernel cuts one cost line over all pairs: a few more slots per pair
+      c->max_splits = std::max(c->max_splits, static_cast<int>(std::min<int64_t>(128, (2LL * c->sm_count + pairs - 1) / pairs + 3)));
     const int r = ratio(c);
     bool ok = dev_alloc(c, reinterpret_cast<void**>(&cv.quant), cv.quant_layer_stride * cfg->n_layers) &&
               dev_alloc(c, reinterpret_cast<void**>(&cv.fp), cv.fp_layer_stride * cfg->n_layers) &&
@@ -737,6 +741,11 @@ lq_status_t decode_impl(lq_cache_t* c, int32_t layer, const void* q, float sm_sc
     a.acc = c->acc;
     e = launch_decode_mma(a, st);
     if (e != cudaSuccess) return cuda_fail(c, e, "lq_decode_mma_kernel");
+  } else if (use_umma(c)) {
+    plan_decode_umma(a, c->sm_count, c->max_splits, c->cfg.n_splits);
+    a.tickets = c->tickets;
+    e = launch_decode_umma(a, st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "lq_decode_umma_kernel");
   } else {
     a.S = choose_splits(c, L);
     e = launch_decode_scalar(a, st);
@@ -874,6 +883,14 @@ lq_status_t lq_cache_info(const lq_cache_t* c, int32_t layer, lq_info_t* info) {
     plan_decode_mma(a, c->sm_count, c->max_splits, c->cfg.n_splits);
     info->n_splits = a.S - 1;
     info->n_ctas = (a.S - 1) * c->cfg.batch * c->cfg.n_kv_heads + a.n_extra;
+  } else if (use_umma(c)) {
+    DecodeArgs a;
+    a.cv = c->cv;
+    a.n_fp = L.n_fp;
+    a.n_quant = L.n_quant;
+    plan_decode_umma(a, c->sm_count, c->max_splits, c->cfg.n_splits);
+    info->n_splits = a.S;
+    info->n_ctas = a.n_ctas;
   } else
     info->n_splits = choose_splits(c, L);
   return LQ_OK;

@@ -105,6 +105,10 @@ struct DecodeArgs {
   // completes the pair only has to read one sum: acc[pair * kAccStride + h * 128 + d] and, for the
   // denominators, acc[pair * kAccStride + kMaxRatio * 128 + h]; all zero at rest.  null: records only.
   float* acc;
+  // tcgen05 kernel (row layout): per (b, kv) pair u_fp_units fp units of 32 slots, then u_supertiles super-tiles of
+  // 128 quantised tokens: u_items items of total cost u_cost (in units of 2 KB); the pairs' items lie on one cost
+  // line that is cut into n_ctas equal ranges; S = record slots per pair
+  int u_items, u_fp_units, u_supertiles, u_cost;
 };
 
 constexpr int kAccStride = kMaxRatio * 128 + 32;  // floats per (b, kv) pair in DecodeArgs::acc
@@ -120,6 +124,9 @@ int max_ctas_decode_mma(int sm_count);
 int plan_decode_mma_padded(const DecodeArgs& a, int sm_count, int max_records, const int32_t* rowinfo_host,
                            int32_t* cta_map, int32_t* pair_ctas, int* stride);
 cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st);
+// tcgen05 kernel: fills tiles_fp (fp units), tiles_quant, the u_* fields, n_ctas and S (<= max_records, <= 128)
+void plan_decode_umma(DecodeArgs& a, int sm_count, int max_records, int s_override);
+cudaError_t launch_decode_umma(const DecodeArgs& a, cudaStream_t st);
 cudaError_t launch_merge(const DecodeArgs& a, cudaStream_t st);
 
 }  // namespace lq

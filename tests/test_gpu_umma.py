@@ -39,6 +39,19 @@ def test_shapes_and_edge_cases(B, Hq, Hkv, W, G, n_prefill, n_steps, chunk):
     assert worst <= 1.0
 
 
+@pytest.mark.parametrize("B,Hq,Hkv,W,G,n_prefill,n_splits", [
+    (1, 8, 2, 64, 32, 64 * 40 + 3, 1),     # one CTA per pair: ~27 items per CTA through the whole pipeline
+    (2, 14, 2, 64, 64, 64 * 30 + 9, 1),    # the same at G = 64, GQA-7
+    (1, 16, 2, 64, 32, 64 * 25 + 1, 1),    # r = 8: one buffer of key codes
+    (40, 32, 8, 64, 32, 64 * 9 + 5, 0),    # 320 pairs on 296 CTAs: CTAs that work for two pairs
+    (75, 8, 8, 32, 32, 32 * 5 + 7, 0),     # 600 pairs: up to four pairs per CTA, MHA
+])
+def test_many_items_and_several_pairs_per_cta(B, Hq, Hkv, W, G, n_prefill, n_splits):
+    worst = run_case(B, Hq, Hkv, W, G, n_prefill, 3, seed=23, kernel=LQ_KERNEL_UMMA, n_splits=n_splits,
+                     check_image_every=0)
+    assert worst <= 1.0
+
+
 def test_four_bit_codes_are_refused():
     with pytest.raises(LogQuantError):
         LogQuantCache(1, 1, 8, 2, 64, 32, max_tokens=512, bits=4, kernel=LQ_KERNEL_UMMA)
