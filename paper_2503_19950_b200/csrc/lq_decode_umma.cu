@@ -17,13 +17,16 @@
 //   bf16 rows of the full-precision store: A straight from shared memory (no unpacking): K rows as a
 //        K-major operand, V rows as an MN-major operand, units of 32 tokens.
 //
-// One CTA = 4 "unpack" warps (q*s, q.zero, key and value codes into tensor memory; thread = token / channel =
-// TMEM lane), 4 "softmax" warps (scores, online softmax, B of p.v, partial and merge), one warp that issues
-// the q.k MMAs and one that issues the p.v MMAs and the bulk copies (an issuing thread manages one
-// tcgen05.mma per ~62 cycles whatever the tile width, so the two streams get a thread each).  The unpack
-// warps run up to two items ahead of the softmax warps (two buffers of key codes).  Everything is ordered
-// by mbarriers with bounded waits; a wait that runs out sets bit 0 of the status word, the CTA stops
-// working, frees its tensor memory and returns.
+// One CTA = 4 worker warps (thread = token for q.k = channel for p.v = TMEM lane), one warp that issues the q.k
+// MMAs, one that issues the p.v MMAs and one that issues the bulk copies.  Per item j the workers read the scores
+// of item j, prepare the q.k operands of item j + 1 (q*s, q.zero, key codes) so that its MMAs run during the
+// softmax of item j, then build B of p.v and unpack the value codes of item j (two buffers, so that the p.v MMAs
+// of item j - 1 may still be running).  Workers wake the issuing warps through named barriers (bar.arrive /
+// bar.sync: hardware barriers, ~36 cycles, nobody polls); MMA completion comes back through tcgen05.commit on
+// mbarriers, which by then have normally completed (an issuing thread manages one tcgen05.mma per ~62 cycles
+// whatever the tile width, so the two streams get a thread each).  Every mbarrier wait is bounded; a warp whose
+// wait ran out sets bit 0 of the status word, attempts no further wait and keeps taking part in every barrier,
+// so that the CTA runs to its end, frees its tensor memory and returns.
 //
 // Work partition: all (b, kv) pairs lie on one cost line (fp units, then 128-token super-tiles, weighted
 // by their bytes) that is cut into equal ranges, one per CTA (2 CTAs per SM); a CTA whose range spans
@@ -53,8 +56,11 @@ namespace {
 
 constexpr int kGroup = 128;            // threads of a worker group = TMEM lanes
 constexpr int kGroupWarps = 4;         // barriers count one arrival per warp
-constexpr int kThreads = 320;          // unpack warps 0-3, softmax warps 4-7, q.k issuer warp, p.v issuer / producer warp
-constexpr int kWarpQK = 8, kWarpPV = 9;
+constexpr int kThreads = 224;          // worker warps 0-3, q.k issuer warp, p.v issuer warp, producer warp
+constexpr int kWarpQK = 4, kWarpPV = 5, kWarpLoad = 6;
+constexpr int kBarQK = 1;              // named barriers: q.k operands of an item are in place (workers -> q.k issuer),
+constexpr int kBarPV0 = 2;             // p.v operands of an even / odd item are in place (workers -> p.v issuer; 2 and 3),
+constexpr int kBarW = 4;               // rendezvous of the worker warps
 constexpr int kStages = 4;
 constexpr int kStageBytes = 16384;     // one fp unit, or one super-tile (12 KB at G = 32, 10 KB at G = 64)
 constexpr int kSpin = 1 << 22;
@@ -92,22 +98,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
   }
   return false;
 }
-// the same for a whole (converged) warp: every lane gets the same answer, so that the warp stays converged for the
-// .sync.aligned tensor-memory instructions that follow
-// Lane 0 polls; once it has seen the phase complete the other lanes take one look of their own (their acquire).
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity) {
-  bool ok = true;
-  if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity);
-  ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
-  if (ok) ok = mbar_wait(bar, parity);
-  return __all_sync(0xFFFFFFFFu, ok);
-}
 // One arrival per warp (128 arrivals on one barrier word serialise): the warp's lanes have done their fences,
 // __syncwarp orders their writes before lane 0's releasing arrival.
 __device__ __forceinline__ void warp_arrive(uint32_t bar) {
   __syncwarp();
   if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
 }
+// named barriers (hardware barriers: the waiting warp sleeps, nobody polls)
+template <int ID, int COUNT>
+__device__ __forceinline__ void named_sync() { asm volatile("bar.sync %0, %1;" ::"n"(ID), "n"(COUNT) : "memory"); }
+template <int ID, int COUNT>
+__device__ __forceinline__ void named_arrive() { asm volatile("bar.arrive %0, %1;" ::"n"(ID), "n"(COUNT) : "memory"); }
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                "l"(src), "r"(bytes), "r"(bar)
@@ -255,15 +256,15 @@ struct Geo {
   static constexpr int NR = 2 * HP;              // columns per group: (hi, lo) of every head
   static constexpr int NRAW = NGS * NR;
   static constexpr int N = NRAW < 16 ? 16 : NRAW;  // MMA width of q.k and of p.v
-  static constexpr int KBUF = N <= 32 ? 2 : 1;   // buffers for the unpacked key codes (and for q*s)
+  static constexpr int VBUF = N <= 32 ? 2 : 1;   // buffers for the unpacked value codes and for B of p.v
   static constexpr int TILE = 1024 + 64 * G;     // bytes of one key group in the store
   static constexpr int WQ = NGS * TILE / 2048;   // cost of a super-tile in units of 2 KB
   static constexpr int BITEMS = NGS * 8 * HP;    // work items of the B build: (group, 8-channel chunk, head pair)
   static constexpr int BROUNDS = (BITEMS + kGroup - 1) / kGroup;
   // TMEM columns
   static constexpr int COL_AK = 0;
-  static constexpr int COL_AV = 64 * KBUF;
-  static constexpr int COL_S = COL_AV + 64;
+  static constexpr int COL_AV = 64;
+  static constexpr int COL_S = COL_AV + 64 * VBUF;
   static constexpr int COL_O = COL_S + N;
   static constexpr int COLS = 256;
   static_assert(COL_O + N <= COLS, "tensor memory");
@@ -275,19 +276,20 @@ struct Geo {
   static constexpr int BPV_BYTES = (N / 8) * 2048;    // B(p.v), N-contiguous: [8-column block][token / 8][token % 8][8 columns]
   static constexpr int OFF_STAGES = 0;
   static constexpr int OFF_BQK = kStages * kStageBytes;
-  static constexpr int OFF_BPV = OFF_BQK + KBUF * BQK_BYTES;
-  static constexpr int OFF_BQFP = OFF_BPV + BPV_BYTES;
+  static constexpr int OFF_BPV = OFF_BQK + BQK_BYTES;
+  static constexpr int OFF_BQFP = OFF_BPV + VBUF * BPV_BYTES;
   static constexpr int OFF_Q = OFF_BQFP + BQFP_BYTES;           // 2 x (8 heads x 256 B)
-  static constexpr int OFF_BIAS = OFF_Q + 2 * kMaxRatio * kD * 2;  // [KBUF][NGS][HP] floats
-  static constexpr int OFF_MAX = OFF_BIAS + 2 * 4 * 8 * 4;         // [8] ints (ordered floats) + flag
-  static constexpr int OFF_RED = OFF_MAX + 64;                    // [4 warps][NGS*HP + HP] floats of the segment reduction
+  static constexpr int OFF_BIAS = OFF_Q + 2 * kMaxRatio * kD * 2;  // [2][NGS][8] floats
+  static constexpr int OFF_MAX = OFF_BIAS + 2 * 4 * 8 * 4;         // [2][16] ints: 8 ordered floats + flag, one set per item parity
+  static constexpr int OFF_RED = OFF_MAX + 128;                    // [4 warps][NGS*HP + HP] floats of the segment reduction
   static constexpr int OFF_BARS = OFF_RED + 4 * 48 * 4;
-  static constexpr int N_BARS = 2 * kStages + 8 + 6;
+  static constexpr int N_BARS = 2 * kStages + 7;
   static constexpr int OFF_MISC = OFF_BARS + N_BARS * 8;          // tmem base, is_last
   static constexpr int SMEM = OFF_MISC + 32 + 128;  // + one byte per record slot of a pair (contributors)
   // the tensor core reads 128 rows behind the start of an fp unit (rows past the unit are never used): they must
   // lie inside the allocation
   static_assert(OFF_STAGES + (kStages - 1) * kStageBytes + 32768 <= SMEM, "A window of the last stage");
+  static_assert(2 * (SMEM + 1024) <= 233472, "two CTAs per SM");
 };
 
 // order-preserving map between floats and ints (for atomicMax on scores)
@@ -316,31 +318,25 @@ struct Cut {
 template <int G, int HP>
 __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs a) {
   using GE = Geo<G, HP>;
-  constexpr int NGS = GE::NGS, NR = GE::NR, N = GE::N, KBUF = GE::KBUF, TILE = GE::TILE;
+  constexpr int NGS = GE::NGS, NR = GE::NR, N = GE::N, VBUF = GE::VBUF, TILE = GE::TILE;
   extern __shared__ __align__(1024) uint8_t smem[];
 #ifdef LQ_UMMA_TRACE
-  __shared__ uint32_t trace[4][12][8];
-  for (int i = threadIdx.x; i < 4 * 12 * 8; i += kThreads) (&trace[0][0][0])[i] = 0;
+  __shared__ uint32_t trace[4][12][12];
+  for (int i = threadIdx.x; i < 4 * 12 * 12; i += kThreads) (&trace[0][0][0])[i] = 0;
 #endif
   const CacheView& cv = a.cv;
   const int r = cv.Hq / cv.Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t sbase = smem_u32(smem);
 
-  // barriers
+  // mbarriers
   const uint32_t bar0 = sbase + GE::OFF_BARS;
   auto bar_full = [&](int s) { return bar0 + 8 * s; };
   auto bar_empty = [&](int s) { return bar0 + 8 * (kStages + s); };
   const uint32_t bar_qfull0 = bar0 + 8 * (2 * kStages);       // [2] query rows of a segment have landed
   const uint32_t bar_qfree0 = bar_qfull0 + 16;                // [2] ... have been taken into registers
-  const uint32_t bar_qk_ready0 = bar_qfree0 + 16;             // [2] q.k operands of an item are in place
-  const uint32_t bar_x_done0 = bar_qk_ready0 + 16;            // [2] scores and bias of an item have been read
-  const uint32_t bar_s_ready = bar_x_done0 + 16;              // q.k MMAs of an item are complete
-  const uint32_t bar_s_free = bar_s_ready + 8;                // the score accumulator may be overwritten
-  const uint32_t bar_av_ready = bar_s_free + 8;               // value codes of an item are in tensor memory
-  const uint32_t bar_bpv_ready = bar_av_ready + 8;            // B of p.v of an item is in shared memory
-  const uint32_t bar_pv_done = bar_bpv_ready + 8;             // p.v MMAs of an item are complete
-  const uint32_t bar_smx = bar_pv_done + 8;                   // rendezvous of the softmax warps
+  const uint32_t bar_s_ready = bar_qfree0 + 16;               // q.k MMAs of an item are complete
+  const uint32_t bar_pv_done0 = bar_s_ready + 8;              // [2] p.v MMAs of an even / odd item are complete
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + GE::OFF_MISC);
   int* is_last_s = reinterpret_cast<int*>(smem + GE::OFF_MISC + 8);
 
@@ -355,25 +351,21 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(bar_full(s), 1);
-      mbar_init(bar_empty(s), 2 * kGroupWarps + 1);
+      mbar_init(bar_empty(s), kGroupWarps + 1);   // the worker warps and the commit behind the item's p.v MMAs
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar_qfull0 + 8 * i, 1);
       mbar_init(bar_qfree0 + 8 * i, kGroupWarps);
-      mbar_init(bar_qk_ready0 + 8 * i, kGroupWarps);
-      mbar_init(bar_x_done0 + 8 * i, kGroupWarps);
+      mbar_init(bar_pv_done0 + 8 * i, 1);
     }
     mbar_init(bar_s_ready, 1);
-    mbar_init(bar_s_free, kGroupWarps);
-    mbar_init(bar_av_ready, kGroupWarps);
-    mbar_init(bar_bpv_ready, kGroupWarps);
-    mbar_init(bar_pv_done, 1);
-    mbar_init(bar_smx, kGroupWarps);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
     int* mx = reinterpret_cast<int*>(smem + GE::OFF_MAX);
-    for (int h = 0; h < 8; ++h) mx[h] = ord_f2i(-INFINITY);
-    mx[8] = 0;
+    for (int i = 0; i < 2; ++i) {
+      for (int h = 0; h < 8; ++h) mx[16 * i + h] = ord_f2i(-INFINITY);
+      mx[16 * i + 8] = 0;
+    }
   }
   if (warp == kWarpQK && n_items > 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(GE::COLS)
@@ -389,24 +381,23 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
 
   const uint8_t* fp_layer = cv.fp + a.layer * cv.fp_layer_stride;
   const uint8_t* quant_layer = cv.quant + a.layer * cv.quant_layer_stride;
-  bool failed = false;
   const int wt = tid & (kGroup - 1);                       // token / channel / TMEM lane of a worker thread
   const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
 
-  if (n_items > 0 && warp == kWarpPV) {
-    // ================= p.v issuer + producer of the bulk copies (one thread) =================
+  if (n_items > 0 && warp == kWarpLoad) {
+    // ================= producer of the bulk copies (one thread) =================
     if (lane == 0) {
-      constexpr uint32_t idesc_q = instr_desc(N, 0, 1);   // A (value codes) from TMEM, B N-contiguous
-      constexpr uint32_t idesc_f = instr_desc(N, 1, 1);   // A = bf16 V rows from shared memory, MN-major
+      bool failed = false;
       int seg = 0;
-      int64_t lpair = pair0;   // position of the next item to load
+      int64_t lpair = pair0;
       int lli = li0;
-      auto load_next = [&](int j) {
+      for (int j = 0; j < n_items && !failed; ++j) {
         const int s = j % kStages;
+        if (j >= kStages && !mbar_wait(bar_empty(s), ((j / kStages) - 1) & 1)) { failed = true; break; }
         if (j == 0 || lli == 0) {
           // first item of a segment: its query rows (double-buffered by segment)
           const int qb = seg & 1;
-          if (seg >= 2 && !mbar_wait(bar_qfree0 + 8 * qb, ((seg >> 1) - 1) & 1)) { failed = true; return; }
+          if (seg >= 2 && !mbar_wait(bar_qfree0 + 8 * qb, ((seg >> 1) - 1) & 1)) { failed = true; break; }
           const int b = static_cast<int>(lpair / cv.Hkv), kv = static_cast<int>(lpair % cv.Hkv);
           mbar_expect_tx(bar_qfull0 + 8 * qb, r * kD * 2);
           bulk_load(sbase + GE::OFF_Q + qb * (kMaxRatio * kD * 2),
@@ -427,57 +418,53 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
         mbar_expect_tx(bar_full(s), bytes);
         bulk_load(sbase + GE::OFF_STAGES + s * kStageBytes, src, bytes, bar_full(s));
         if (++lli == cut.I) { lli = 0; ++lpair; }
-      };
-      for (int j = 0; j < min(n_items, kStages) && !failed; ++j) load_next(j);
-      int li = li0;
-      for (int j = 0; j < n_items && !failed; ++j) {
-        const int s = j % kStages;
+      }
+      if (failed) atomicOr(a.status, 1);
+    }
+  } else if (n_items > 0 && warp == kWarpPV) {
+    // ================= p.v issuer: woken by the workers through a named barrier, never polls =================
+    constexpr uint32_t idesc_q = instr_desc(N, 0, 1);   // A (value codes) from TMEM, B N-contiguous
+    constexpr uint32_t idesc_f = instr_desc(N, 1, 1);   // A = bf16 V rows from shared memory, MN-major
+    int li = li0;
+    for (int j = 0; j < n_items; ++j) {
+      const int s = j % kStages;
+      const int vb = j % VBUF;
+      if (j & 1) named_sync<kBarPV0 + 1, kGroup + 32>(); else named_sync<kBarPV0, kGroup + 32>();
+      tc_fence_after();
+      if (lane == 0) {
         TR(3, j, 0);
-        if (!mbar_wait(bar_av_ready, j & 1)) { failed = true; break; }
-        if (!mbar_wait(bar_bpv_ready, j & 1)) { failed = true; break; }
-        TR(3, j, 1);
-        tc_fence_after();
         const uint32_t acc0 = (j == 0 || li == 0) ? 0u : 1u;  // the first item of a segment overwrites O
+        const uint32_t bpv = sbase + GE::OFF_BPV + vb * GE::BPV_BYTES;
         if (li < cut.F) {
           const int nv = min(kFpUnitSlots, a.n_fp - li * kFpUnitSlots);
           const uint32_t vrows = sbase + GE::OFF_STAGES + s * kStageBytes + kFpUnitVOffset;
           for (int ks = 0; ks < (nv + 15) / 16; ++ks)
-            mma_ss(tmem + GE::COL_O, smem_desc(vrows + ks * 4096, 2048, 128),
-                   smem_desc(sbase + GE::OFF_BPV + ks * 256, 128, 2048), idesc_f, ks ? 1u : acc0);
+            mma_ss(tmem + GE::COL_O, smem_desc(vrows + ks * 4096, 2048, 128), smem_desc(bpv + ks * 256, 128, 2048),
+                   idesc_f, ks ? 1u : acc0);
         } else {
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks)
-            mma_ts(tmem + GE::COL_O, tmem + GE::COL_AV + 8 * ks, smem_desc(sbase + GE::OFF_BPV + ks * 256, 128, 2048),
+            mma_ts(tmem + GE::COL_O, tmem + GE::COL_AV + 64 * vb + 8 * ks, smem_desc(bpv + ks * 256, 128, 2048),
                    idesc_q, ks ? 1u : acc0);
         }
-        tc_commit(bar_pv_done);
+        tc_commit(bar_pv_done0 + 8 * (j & 1));
         tc_commit(bar_empty(s));
-        TR(3, j, 2);
-        if (j + kStages < n_items) {
-          // refill this stage once the workers and the MMAs above are done with it
-          if (!mbar_wait(bar_empty(s), (j / kStages) & 1)) { failed = true; break; }
-          TR(3, j, 3);
-          load_next(j + kStages);
-        }
-        if (++li == cut.I) li = 0;
+        TR(3, j, 1);
       }
-      if (failed) atomicOr(a.status, 1);
+      __syncwarp();
+      if (++li == cut.I) li = 0;
     }
   } else if (n_items > 0 && warp == kWarpQK) {
-    // ================= q.k issuer (one thread) =================
-    if (lane == 0) {
-      constexpr uint32_t idesc_q = instr_desc(N, 0, 0);    // A (key codes) from TMEM, B = q*s K-major
-      constexpr uint32_t idesc_f = instr_desc(16, 0, 0);   // A = bf16 K rows from shared memory, B = q K-major
-      int li = li0;
-      for (int j = 0; j < n_items; ++j) {
-        const int s = j % kStages;
-        const int kb = j % KBUF;
+    // ================= q.k issuer =================
+    constexpr uint32_t idesc_q = instr_desc(N, 0, 0);    // A (key codes) from TMEM, B = q*s K-major
+    constexpr uint32_t idesc_f = instr_desc(16, 0, 0);   // A = bf16 K rows from shared memory, B = q K-major
+    int li = li0;
+    for (int j = 0; j < n_items; ++j) {
+      const int s = j % kStages;
+      named_sync<kBarQK, kGroup + 32>();
+      tc_fence_after();
+      if (lane == 0) {
         TR(2, j, 0);
-        if (!mbar_wait(bar_qk_ready0 + 8 * kb, (j / KBUF) & 1)) { failed = true; break; }
-        TR(2, j, 1);
-        if (j > 0 && !mbar_wait(bar_s_free, (j - 1) & 1)) { failed = true; break; }
-        TR(2, j, 2);
-        tc_fence_after();
         if (li < cut.F) {
           const uint32_t krows = sbase + GE::OFF_STAGES + s * kStageBytes;
 #pragma unroll
@@ -485,41 +472,43 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
             mma_ss(tmem + GE::COL_S, smem_desc(krows + ks * 256, 128, 2048),
                    smem_desc(sbase + GE::OFF_BQFP + ks * 2 * GE::LBO_QFP, GE::LBO_QFP, 128), idesc_f, ks ? 1u : 0u);
         } else {
-          const uint32_t bq = sbase + GE::OFF_BQK + kb * GE::BQK_BYTES;
+          const uint32_t bq = sbase + GE::OFF_BQK;
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks)
-            mma_ts(tmem + GE::COL_S, tmem + GE::COL_AK + 64 * kb + 8 * ks,
-                   smem_desc(bq + ks * 2 * GE::LBO_QK, GE::LBO_QK, 128), idesc_q, ks ? 1u : 0u);
+            mma_ts(tmem + GE::COL_S, tmem + GE::COL_AK + 8 * ks, smem_desc(bq + ks * 2 * GE::LBO_QK, GE::LBO_QK, 128),
+                   idesc_q, ks ? 1u : 0u);
         }
         tc_commit(bar_s_ready);
-        TR(2, j, 3);
-        if (++li == cut.I) li = 0;
+        TR(2, j, 1);
       }
-      if (failed) atomicOr(a.status, 1);
+      __syncwarp();
+      if (++li == cut.I) li = 0;
     }
-  } else if (n_items > 0 && warp < 4) {
-    // ================= unpack warps: q*s and q.zero, key codes and value codes into tensor memory =================
-    // thread = token (key codes) = channel (value codes) = TMEM lane.  The q.k operands of item j + 1 are prepared
-    // before the value codes of item j (which have to wait for the p.v MMAs of item j - 1), so that the q.k MMAs
-    // run one item ahead of the softmax warps.
+  } else if (n_items > 0 && warp < kGroupWarps) {
+    // ================= worker warps: thread = token (q.k) = channel (p.v) = TMEM lane =================
+    // Per item j, in this order: read the scores of item j; prepare the q.k operands of item j + 1 (q*s and the
+    // q.zero bias into shared memory, the key codes into tensor memory) and hand them to the q.k issuer; online
+    // softmax of item j; B of p.v and the value codes of item j; hand them to the p.v issuer.  The MMAs of item
+    // j + 1 (q.k) and of item j (p.v) run while the workers go on, so the waits below are normally satisfied.
+    bool failed = false;   // warp-uniform: after a wait that ran out no wait is attempted any more; the warp keeps
+                           // taking part in every barrier so that nobody is left waiting for it
+    auto wait = [&](uint32_t bar, uint32_t parity) {
+      if (!failed) failed = !__all_sync(kFullMask, mbar_wait(bar, parity) ? 1 : 0);
+    };
     uint32_t qpk[GE::BROUNDS][2][4];   // query of the B build: item (group g, chunk c, head pair hp) per round
     float qf[GE::BROUNDS][2][8];
     int kli = li0, kseg = -1;          // position of the next item whose q.k operands are prepared
     int64_t kpair = pair0;
 
     // ---- q.k operands of item j: B = q*s and the bias in shared memory, key codes in tensor memory ----
-    auto kprep = [&](int j) {
+    auto prep = [&](int j) {
       const int s = j % kStages;
-      const int kb = j % KBUF;
       const uint32_t stage = sbase + GE::OFF_STAGES + s * kStageBytes;
-      if (tid == 0) TR(0, j, 0);
       if (j == 0 || kli == 0) {
         // segment start: the query rows of the pair into registers; B of the bf16 keys
         ++kseg;
         const int qb = kseg & 1;
-        if (!mbar_wait_warp(bar_qfull0 + 8 * qb, (kseg >> 1) & 1)) { failed = true; return; }
-        // the q.k MMAs of the previous item (another pair) may still be reading B of the bf16 keys
-        if (j > 0 && !mbar_wait_warp(bar_x_done0 + 8 * ((j - 1) % KBUF), ((j - 1) / KBUF) & 1)) { failed = true; return; }
+        wait(bar_qfull0 + 8 * qb, (kseg >> 1) & 1);
         const uint32_t qs = sbase + GE::OFF_Q + qb * (kMaxRatio * kD * 2);
 #pragma unroll
         for (int rd = 0; rd < GE::BROUNDS; ++rd) {
@@ -551,12 +540,8 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
         warp_arrive(bar_qfree0 + 8 * qb);
         fence_async_smem();
       }
-      if (!mbar_wait_warp(bar_full(s), (j / kStages) & 1)) { failed = true; return; }
-      // buffer kb (key codes, q*s, bias) is free once item j - KBUF has had its scores read
-      if (j >= KBUF && !mbar_wait_warp(bar_x_done0 + 8 * kb, ((j - KBUF) / KBUF) & 1)) { failed = true; return; }
-      if (tid == 0) TR(0, j, 1);
+      wait(bar_full(s), (j / kStages) & 1);
       if (kli >= cut.F) {
-        tc_fence_after();
         // key codes first (loads in flight while B is built): thread = token
         uint4 kw4[2];
         {
@@ -566,8 +551,8 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
           kw4[1] = lds128(kc + G * 16);
         }
         // B(q.k): rows n = g*NR + 2*head + {hi, lo}, K-major; bias = q . zero per (group, head)
-        const uint32_t bq = sbase + GE::OFF_BQK + kb * GE::BQK_BYTES;
-        float* bias = reinterpret_cast<float*>(smem + GE::OFF_BIAS) + kb * (4 * 8);
+        const uint32_t bq = sbase + GE::OFF_BQK;
+        float* bias = reinterpret_cast<float*>(smem + GE::OFF_BIAS) + (j & 1) * (4 * 8);
 #pragma unroll
         for (int rd = 0; rd < GE::BROUNDS; ++rd) {
           const int it = tid + rd * kGroup;
@@ -617,7 +602,7 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
               regs[8 * jj + 4 + i] = ws & (0x00030003u << (2 * i));
             }
           }
-          tmem_st<32>(tmem + lane_base + GE::COL_AK + 64 * kb + 32 * hf, regs);
+          tmem_st<32>(tmem + lane_base + GE::COL_AK + 32 * hf, regs);
         }
         tc_wait_st();
         fence_async_smem();
@@ -637,88 +622,20 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
         fence_async_smem();
       }
       tc_fence_before();
-      warp_arrive(bar_qk_ready0 + 8 * kb);
-      if (tid == 0) TR(0, j, 2);
       if (++kli == cut.I) { kli = 0; ++kpair; }
     };
 
-    kprep(0);
-    int li = li0;
-    for (int j = 0; j < n_items && !failed; ++j) {
-      const int s = j % kStages;
-      const uint32_t stage = sbase + GE::OFF_STAGES + s * kStageBytes;
-      if (KBUF == 2 && j + 1 < n_items) {
-        kprep(j + 1);
-        if (failed) break;
-      }
-      // ---- value codes of item j: thread = channel; its 128 tokens = 8 words (G/16 per tile) ----
-      const bool is_fp = li < cut.F;
-      uint32_t w[8];
-      if (!is_fp) {
-#pragma unroll
-        for (int tl = 0; tl < NGS; ++tl) {
-          const uint32_t vc = stage + tl * TILE + row_vcodes_off(G) + tid * (G / 4);
-          if (G == 32) {
-            const uint2 x = lds64(vc);
-            w[2 * tl] = x.x; w[2 * tl + 1] = x.y;
-          } else {
-            const uint4 x = lds128(vc);
-            w[4 * tl] = x.x; w[4 * tl + 1] = x.y; w[4 * tl + 2] = x.z; w[4 * tl + 3] = x.w;
-          }
-        }
-      }
-      // the previous p.v MMAs may still be reading the value codes (waited for at every item, so that no phase of
-      // the barrier is skipped)
-      if (j > 0 && !mbar_wait_warp(bar_pv_done, (j - 1) & 1)) { failed = true; break; }
-      if (tid == 0) TR(0, j, 3);
-      if (!is_fp) {
-        tc_fence_after();
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          uint32_t regs[32];
-#pragma unroll
-          for (int jj = 0; jj < 4; ++jj) {
-            const uint32_t wv = w[4 * hf + jj], ws = wv >> 8;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              regs[8 * jj + i] = wv & (0x00030003u << (2 * i));
-              regs[8 * jj + 4 + i] = ws & (0x00030003u << (2 * i));
-            }
-          }
-          tmem_st<32>(tmem + lane_base + GE::COL_AV + 32 * hf, regs);
-        }
-        tc_wait_st();
-        tc_fence_before();
-      }
-      warp_arrive(bar_av_ready);
-      warp_arrive(bar_empty(s));
-      if (tid == 0) TR(0, j, 4);
-      if (KBUF == 1 && j + 1 < n_items) {
-        kprep(j + 1);
-        if (failed) break;
-      }
-      if (++li == cut.I) li = 0;
-    }
-    if (failed && lane == 0) atomicOr(a.status, 1);
-  } else if (n_items > 0) {
-    // ================= softmax warps: scores, online softmax, B of p.v, partial and merge =================
-    // thread = token (scores) = channel (output) = TMEM lane
     const float kq = a.scale_log2 * pow2i(69);
     float m_run[HP], l_run[HP], zacc[NGS][HP];
     int li = li0;
     int64_t pair = pair0;
     int items_in_seg = 0, first_j_of_seg = 0;
-    uint32_t smx_phase = 0;
-    // rendezvous of the 128 softmax threads (bounded); every one of them takes the same sequence of them
-    auto smx_sync = [&]() {
-      warp_arrive(bar_smx);
-      const bool ok = mbar_wait_warp(bar_smx, smx_phase & 1);
-      ++smx_phase;
-      return ok;
-    };
-    for (int j = 0; j < n_items && !failed; ++j) {
+
+    prep(0);
+    named_arrive<kBarQK, kGroup + 32>();
+    for (int j = 0; j < n_items; ++j) {
       const int s = j % kStages;
-      const int kb = j % KBUF;
+      const int vb = j % VBUF;
       const bool is_fp = li < cut.F;
       const uint32_t stage = sbase + GE::OFF_STAGES + s * kStageBytes;
       if (j == 0 || li == 0) {
@@ -736,9 +653,8 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
       const bool o_started = j > first_j_of_seg;   // a p.v MMA of this segment has been issued
       if (wt == 0) TR(1, j, 0);
 
-      // ---------------- scores ----------------
-      if (!mbar_wait_warp(bar_full(s), (j / kStages) & 1)) { failed = true; break; }
-      if (!mbar_wait_warp(bar_s_ready, j & 1)) { failed = true; break; }
+      // ---------------- scores of item j ----------------
+      wait(bar_s_ready, j & 1);
       tc_fence_after();
       if (wt == 0) TR(1, j, 1);
       float sc[HP];
@@ -754,7 +670,7 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
         const int g_tok = wt / G;   // key group of this thread's token inside the super-tile
         uint32_t d[NR];
         tmem_ld<NR>(tmem + lane_base + GE::COL_S + g_tok * NR, d);
-        const float* bias = reinterpret_cast<const float*>(smem + GE::OFF_BIAS) + kb * (4 * 8) + g_tok * 8;
+        const float* bias = reinterpret_cast<const float*>(smem + GE::OFF_BIAS) + (j & 1) * (4 * 8) + g_tok * 8;
         float bs[HP];
 #pragma unroll
         for (int h = 0; h < HP; ++h) bs[h] = bias[h];
@@ -765,11 +681,17 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
           sc[h] = fmaf(__uint_as_float(d[2 * h]) + __uint_as_float(d[2 * h + 1]), kq, bs[h]);
       }
       tc_fence_before();
-      warp_arrive(bar_s_free);
-      warp_arrive(bar_x_done0 + 8 * kb);
+
+      // ---------------- q.k operands of item j + 1 (the score accumulator and the key codes are free now) ----------------
+      if (j + 1 < n_items) {
+        prep(j + 1);
+        named_arrive<kBarQK, kGroup + 32>();
+      }
+      if (wt == 0) TR(1, j, 2);
 
       // ---------------- online softmax with a CTA-wide, lazily moved reference maximum ----------------
-      int* mx = reinterpret_cast<int*>(smem + GE::OFF_MAX);
+      // (exchange words per item parity: a warp that is already at the next item touches the other set)
+      int* mx = reinterpret_cast<int*>(smem + GE::OFF_MAX) + 16 * (j & 1);
       {
         bool need = false;
 #pragma unroll
@@ -784,9 +706,8 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
           }
           if (lane == 0) atomicOr(mx + 8, 1);
         }
-        warp_arrive(bar_smx);
       }
-      // (independent work between the arrival and the wait) value scale and zero of this thread's token
+      // value scale and zero of this thread's token
       float vs[NGS], vz[NGS];
       if (!is_fp) {
         const int tl = wt / G, tt = wt % G;
@@ -807,11 +728,7 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
           vz[g] = valid ? vz[g] : 0.f;
         }
       }
-      {
-        const bool ok = mbar_wait_warp(bar_smx, smx_phase & 1);
-        ++smx_phase;
-        if (!ok) { failed = true; break; }
-      }
+      named_sync<kBarW, kGroup>();
       if (*reinterpret_cast<volatile int*>(mx + 8)) {
         // rare: some score exceeds the reference by more than 2^8 (or the segment has just begun)
         float corr[HP];
@@ -827,7 +744,7 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
         }
         if (o_started) {
           // rescale the output accumulator: no p.v MMA may be in flight
-          if (!mbar_wait_warp(bar_pv_done, (j - 1) & 1)) { failed = true; break; }
+          wait(bar_pv_done0 + 8 * ((j - 1) & 1), ((j - 1) >> 1) & 1);
           tc_fence_after();
           uint32_t o[N];
           tmem_ld<N>(tmem + lane_base + GE::COL_O, o);
@@ -844,20 +761,20 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
           tc_fence_before();
         }
         // everybody has read the exchange words: thread 0 puts them back to rest before anybody goes on
-        if (!smx_sync()) { failed = true; break; }
+        named_sync<kBarW, kGroup>();
         if (wt == 0) {
           for (int h = 0; h < 8; ++h) mx[h] = ord_f2i(-INFINITY);
           mx[8] = 0;
         }
-        if (!smx_sync()) { failed = true; break; }
+        named_sync<kBarW, kGroup>();
       }
-      if (wt == 0) TR(1, j, 2);
       float p[HP];
 #pragma unroll
       for (int h = 0; h < HP; ++h) {
         p[h] = valid && h < r ? ex2(sc[h] - m_run[h]) : 0.f;
         l_run[h] += p[h];
       }
+      if (wt == 0) TR(1, j, 3);
 
       // ---------------- B of p.v ----------------
       uint32_t w[NGS][HP];
@@ -879,11 +796,26 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
             zacc[g][h] = fmaf(p[h], vz[g], zacc[g][h]);
           }
       }
-      // the previous p.v MMAs (of this or the previous segment) may still be reading B
-      if (j > 0 && !mbar_wait_warp(bar_pv_done, (j - 1) & 1)) { failed = true; break; }
-      if (wt == 0) TR(1, j, 3);
+      // value codes of item j: thread = channel; its 128 tokens = 8 words (G/16 per tile)
+      uint32_t vw[8];
+      if (!is_fp) {
+#pragma unroll
+        for (int tl = 0; tl < NGS; ++tl) {
+          const uint32_t vc = stage + tl * TILE + row_vcodes_off(G) + tid * (G / 4);
+          if (G == 32) {
+            const uint2 x = lds64(vc);
+            vw[2 * tl] = x.x; vw[2 * tl + 1] = x.y;
+          } else {
+            const uint4 x = lds128(vc);
+            vw[4 * tl] = x.x; vw[4 * tl + 1] = x.y; vw[4 * tl + 2] = x.z; vw[4 * tl + 3] = x.w;
+          }
+        }
+      }
+      // buffer vb (value codes in tensor memory, B in shared memory) is free once the p.v MMAs of item j - VBUF are complete
+      if (j >= VBUF) wait(bar_pv_done0 + 8 * ((j - VBUF) & 1), ((j - VBUF) >> 1) & 1);
+      if (wt == 0) TR(1, j, 4);
       if (!is_fp || wt < 32) {
-        const uint32_t row = sbase + GE::OFF_BPV + wt * 16;
+        const uint32_t row = sbase + GE::OFF_BPV + vb * GE::BPV_BYTES + wt * 16;
         if (NR >= 8) {
 #pragma unroll
           for (int g = 0; g < NGS; ++g)
@@ -899,14 +831,33 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
                    w[(2 * nb + 1) % NGS][1 % HP]);
         }
       }
+      if (!is_fp) {
+        tc_fence_after();
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          uint32_t regs[32];
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj) {
+            const uint32_t wv = vw[4 * hf + jj], ws = wv >> 8;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              regs[8 * jj + i] = wv & (0x00030003u << (2 * i));
+              regs[8 * jj + 4 + i] = ws & (0x00030003u << (2 * i));
+            }
+          }
+          tmem_st<32>(tmem + lane_base + GE::COL_AV + 64 * vb + 32 * hf, regs);
+        }
+        tc_wait_st();
+      }
       fence_async_smem();
-      warp_arrive(bar_bpv_ready);
+      tc_fence_before();
       warp_arrive(bar_empty(s));
-      if (wt == 0) TR(1, j, 4);
+      if (j & 1) named_arrive<kBarPV0 + 1, kGroup + 32>(); else named_arrive<kBarPV0, kGroup + 32>();
+      if (wt == 0) TR(1, j, 5);
 
       if (!more) {
         // ---------------- segment end: reduce l and the zero term, read O, write the partial ----------------
-        if (!mbar_wait_warp(bar_pv_done, j & 1)) { failed = true; break; }
+        wait(bar_pv_done0 + 8 * (j & 1), (j >> 1) & 1);
         tc_fence_after();
         float* red = reinterpret_cast<float*>(smem + GE::OFF_RED);
         const int xw = warp & 3;
@@ -930,7 +881,7 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
             }
           }
         }
-        if (!smx_sync()) { failed = true; break; }
+        named_sync<kBarW, kGroup>();
         const int vg = wt / G;   // value group of this thread's channel
         uint32_t o[NR];
         tmem_ld<NR>(tmem + lane_base + GE::COL_O + vg * NR, o);
@@ -966,7 +917,7 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
           }
           contrib[wt] = yes ? 1 : 0;
         }
-        if (!smx_sync()) { failed = true; break; }
+        named_sync<kBarW, kGroup>();
         if (wt == 0) {
           int* ticket = a.tickets + 32 * pair + 1;
           const int old = atomicAdd(ticket, items_in_seg);
@@ -975,7 +926,7 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
           __threadfence();
           *is_last_s = last;
         }
-        if (!smx_sync()) { failed = true; break; }
+        named_sync<kBarW, kGroup>();
         if (*reinterpret_cast<volatile int*>(is_last_s)) {
           __threadfence();
           for (int h = 0; h < r; ++h) {
@@ -1006,7 +957,7 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
           }
         }
         // the exchange areas (red, contrib, is_last) are rewritten by the next segment only after its own rendezvous
-        if (!smx_sync()) { failed = true; break; }
+        named_sync<kBarW, kGroup>();
       }
       if (++li == cut.I) { li = 0; ++pair; }
     }
@@ -1018,17 +969,15 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
   __syncthreads();
 #ifdef LQ_UMMA_TRACE
   if (blockIdx.x == LQ_UMMA_TRACE && threadIdx.x == 0) {
-    const uint32_t t0 = trace[0][0][0];
+    const uint32_t t0 = trace[1][0][0];
     printf("cta %d items %d F %d Q %d\n", blockIdx.x, n_items, a.u_fp_units, a.u_supertiles);
     for (int j = 0; j < 12 && j < n_items; ++j) {
-      printf("item %2d U:", j);
-      for (int k = 0; k < 5; ++k) printf(" %6d", static_cast<int>(trace[0][j][k] - t0));
-      printf(" | X:");
-      for (int k = 0; k < 5; ++k) printf(" %6d", static_cast<int>(trace[1][j][k] - t0));
+      printf("item %2d W:", j);
+      for (int k = 0; k < 6; ++k) printf(" %6d", static_cast<int>(trace[1][j][k] - t0));
       printf(" | QK:");
-      for (int k = 0; k < 4; ++k) printf(" %6d", static_cast<int>(trace[2][j][k] - t0));
+      for (int k = 0; k < 2; ++k) printf(" %6d", static_cast<int>(trace[2][j][k] - t0));
       printf(" | PV:");
-      for (int k = 0; k < 4; ++k) printf(" %6d", static_cast<int>(trace[3][j][k] - t0));
+      for (int k = 0; k < 2; ++k) printf(" %6d", static_cast<int>(trace[3][j][k] - t0));
       printf("\n");
     }
   }
