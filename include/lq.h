@@ -77,7 +77,7 @@ typedef struct {
   int32_t window;        /* W of Algorithm 1, <= 512.  W % G != 0 (the paper's W = 42 or 85 with G = 64): removed
                             tokens wait at full precision, in removal order, until G of them form a key group */
   int32_t group;         /* G: quantisation group size, 32 or 64                                 */
-  int32_t bits;          /* 2, or 4 (the paper's second precision; needs group == 32)             */
+  int32_t bits;          /* 2, or 4 (the paper's second precision, Table 3; not with LQ_KERNEL_UMMA) */
   int64_t max_tokens;    /* capacity per sequence (tokens ever appended)                         */
   int32_t auto_compress; /* 1: lq_append runs the overflow step itself when the window is full   */
   int32_t device;        /* CUDA device ordinal, or LQ_DEVICE_NONE for bookkeeping only          */

@@ -402,7 +402,6 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
   if ((cfg->dev_alloc == nullptr) != (cfg->dev_free == nullptr)) return LQ_ERR_INVALID_ARG;
   if (cfg->head_dim != kD || (cfg->bits != 2 && cfg->bits != 4)) return LQ_ERR_UNSUPPORTED;
   if (cfg->group != 32 && cfg->group != 64) return LQ_ERR_UNSUPPORTED;
-  if (cfg->bits == 4 && cfg->group != 32) return LQ_ERR_UNSUPPORTED;  // a 4-bit tile of G = 64 exceeds a stage
   if (cfg->window > kMaxW) return LQ_ERR_UNSUPPORTED;
   if (cfg->n_q_heads / cfg->n_kv_heads > kMaxRatio || cfg->n_layers > 128) return LQ_ERR_UNSUPPORTED;
   if (cfg->kernel < LQ_KERNEL_AUTO || cfg->kernel > LQ_KERNEL_UMMA) return LQ_ERR_INVALID_ARG;

@@ -43,9 +43,12 @@ constexpr int kWarps = 4;
 // every warp owns 12 KB of stages: 2 x 6 KB, each holding two G = 32 tiles (3 KB), one G = 64 tile
 // (5 KB) or half an fp tile (K rows or V rows, 4 KB).  Loads of two tiles measured faster than
 // single tiles (1.55 vs 1.9 us per tile and warp): the per-load bookkeeping is not free.
-constexpr int kWarpStageBytes = 12288;
-__host__ __device__ constexpr int stage_bytes(int) { return 6144; }
-__host__ __device__ constexpr int n_stages(int G) { return kWarpStageBytes / stage_bytes(G); }
+// (4-bit codes at G = 64: one tile is 9 KB, so that variant's stages are 9 KB and a CTA's shared memory allows
+// three CTAs per SM instead of four.)
+__host__ __device__ constexpr int stage_bytes(int G, int PL = 1) { return G == 64 && PL == 2 ? 9216 : 6144; }
+__host__ __device__ constexpr int n_stages(int) { return 2; }
+__host__ __device__ constexpr int warp_stage_bytes(int G, int PL = 1) { return n_stages(G) * stage_bytes(G, PL); }
+constexpr int kWarpStageBytes = warp_stage_bytes(32);
 constexpr int kMaxStages = 3;
 constexpr int kCtasPerSm = 4;  // at 128 registers and 51 KB of shared memory; 3 and 5 both measured slower
 constexpr uint32_t kFull = 0xFFFFFFFFu;
@@ -610,10 +613,11 @@ __device__ __forceinline__ void process_quant_tile(WarpState<NCB>& st, const uin
 }
 
 // shared memory: [per-warp stages][query rows of the pair][mbarriers][flags]
-constexpr int kSmemStages = kWarps * kWarpStageBytes;
+constexpr int kSmemStages = kWarps * kWarpStageBytes;   // the smallest variant: the merge areas below must fit into it
+__host__ __device__ constexpr int smem_stages(int G, int PL) { return kWarps * warp_stage_bytes(G, PL); }
 constexpr int kSmemQ = kMaxRatio * kD * 2;
 constexpr int kSmemBars = (kWarps * kMaxStages + 1) * 8;
-constexpr int kSmemBytes = kSmemStages + kSmemQ + kSmemBars + 16;
+__host__ __device__ constexpr int smem_bytes(int G, int PL) { return smem_stages(G, PL) + kSmemQ + kSmemBars + 16; }
 constexpr int kMergeMax = 2048;  // S * r records the fused second pass can stage
 constexpr int kMergeOneBatch = 12;  // CTA records the fused second pass loads in one batch (kSB per warp)
 
@@ -634,7 +638,8 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   const int n = lane >> 2, j = lane & 3;
   const uint32_t oddmask = (n & 1) ? 0xFFFFFFFFu : 0u;
   constexpr int TILE = quant_tile_bytes(G, PL);
-  constexpr int kStages = n_stages(G), kStageBytes = stage_bytes(G);
+  constexpr int kStages = n_stages(G), kStageBytes = stage_bytes(G, PL);
+  constexpr int kWarpStage = warp_stage_bytes(G, PL), kStagesAll = smem_stages(G, PL);
   static_assert(TILE <= kStageBytes && kFpTileVOffset <= kStageBytes && kStages <= kMaxStages, "stage geometry");
   // CTA c works for pair c % P in slot c / P: pairs [0, n_extra) have S CTAs, the others S - 1 (a.S
   // is also the record stride).  Interleaving gives every pair CTAs from every launch rank of the
@@ -678,11 +683,11 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   }
   int* ticket = a.tickets + 32 * pair + 1;  // one 128-byte line per pair; word 1 is the arrival ticket
 
-  const uint32_t stage0 = smem_u32(smem + warp * kWarpStageBytes);
-  const uint32_t qsm = smem_u32(smem + kSmemStages);
-  const uint32_t bar0 = smem_u32(smem + kSmemStages + kSmemQ) + warp * kMaxStages * 8;
-  const uint32_t qbar = smem_u32(smem + kSmemStages + kSmemQ) + kWarps * kMaxStages * 8;
-  int* is_last = reinterpret_cast<int*>(smem + kSmemStages + kSmemQ + kSmemBars);
+  const uint32_t stage0 = smem_u32(smem + warp * kWarpStage);
+  const uint32_t qsm = smem_u32(smem + kStagesAll);
+  const uint32_t bar0 = smem_u32(smem + kStagesAll + kSmemQ) + warp * kMaxStages * 8;
+  const uint32_t qbar = smem_u32(smem + kStagesAll + kSmemQ) + kWarps * kMaxStages * 8;
+  int* is_last = reinterpret_cast<int*>(smem + kStagesAll + kSmemQ + kSmemBars);
 
   if (lane == 0) {
 #pragma unroll
@@ -1197,10 +1202,11 @@ void plan_decode_mma(DecodeArgs& a, int sm_count, int max_records, int s_overrid
   const int r = a.cv.Hq / a.cv.Hkv;
   a.tiles_fp = (a.n_fp + kFpTileSlots - 1) / kFpTileSlots;
   a.tiles_quant = static_cast<int>(a.n_quant / a.cv.G);
-  const int items = a.tiles_fp + a.tiles_quant / (stage_bytes(a.cv.G) / quant_tile_bytes(a.cv.G, a.cv.planes));
+  const int items = a.tiles_fp + a.tiles_quant / (stage_bytes(a.cv.G, a.cv.planes) / quant_tile_bytes(a.cv.G, a.cv.planes));
   // at most one resident wave of CTAs in total: a CTA that had to wait for a free slot would start
   // when the others finish, and its pair's merge would wait for it
-  const int ctas_per_sm = r <= 4 ? kCtasPerSm : kCtasPerSm - 1;  // the two-column-block variant needs more registers
+  // the two-column-block variant needs more registers, the 9 KB stages of 4-bit codes at G = 64 more shared memory
+  const int ctas_per_sm = r <= 4 && !(a.cv.G == 64 && a.cv.planes == 2) ? kCtasPerSm : kCtasPerSm - 1;
   int S = s_override > 0 ? s_override : (ctas_per_sm * sm_count) / pairs;
   S = std::min(S, (items + kWarps - 1) / kWarps);  // at least one item per warp
   S = std::min(S, max_records - 1);
@@ -1226,8 +1232,8 @@ int plan_decode_mma_padded(const DecodeArgs& a, int sm_count, int max_records, c
   const int r = a.cv.Hq / a.cv.Hkv;
   const int tiles_fp = (a.n_fp + kFpTileSlots - 1) / kFpTileSlots;
   const int tiles_quant = static_cast<int>(a.n_quant / a.cv.G);
-  const int tps = stage_bytes(a.cv.G) / quant_tile_bytes(a.cv.G, a.cv.planes);
-  const int wave = (r <= 4 ? kCtasPerSm : kCtasPerSm - 1) * sm_count;
+  const int tps = stage_bytes(a.cv.G, a.cv.planes) / quant_tile_bytes(a.cv.G, a.cv.planes);
+  const int wave = (r <= 4 && !(a.cv.G == 64 && a.cv.planes == 2) ? kCtasPerSm : kCtasPerSm - 1) * sm_count;
   const int cap_records = std::max(1, std::min(max_records, kMergeMax / r));
   std::vector<int64_t> work(pairs);
   std::vector<int> cap(pairs);
@@ -1292,6 +1298,7 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
   if (a.cv.G == 32 && a.cv.planes == 1) LQ_PICK(32, 1);
   else if (a.cv.G == 32 && a.cv.planes == 2) LQ_PICK(32, 2);
   else if (a.cv.G == 64 && a.cv.planes == 1) LQ_PICK(64, 1);
+  else if (a.cv.G == 64 && a.cv.planes == 2) LQ_PICK(64, 2);
   else return cudaErrorInvalidValue;
 #undef LQ_PICK
 #undef LQ_PICK2
@@ -1305,14 +1312,14 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
   if (e != cudaSuccess) return e;
   const int variant = (padded ? 16 : 0) + (fused ? 8 : 0) + (a.cv.planes == 2 ? 4 : 0) + (a.cv.G == 64 ? 2 : 0) + (r <= 4 ? 0 : 1);
   if (dev < 0 || dev >= 64 || !configured[dev][variant]) {
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(a.cv.G, a.cv.planes));
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) configured[dev][variant] = true;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(padded ? a.n_ctas : a.cv.B * a.cv.Hkv * (a.S - 1) + a.n_extra);
   cfg.blockDim = dim3(kWarps * 32);
-  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.dynamicSmemBytes = smem_bytes(a.cv.G, a.cv.planes);
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

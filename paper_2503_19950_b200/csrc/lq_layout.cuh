@@ -20,9 +20,9 @@
 //     512 + 64 G             V scale, G/16 sub-tiles x (4096/G) B
 //     512 + 64 G + 256       V zero,  G/16 sub-tiles x (4096/G) B
 //     tile bytes = 1024 + 64 G   (3072 at G = 32, 5120 at G = 64; 96 / 80 B per token)
-//   4-bit codes (G = 32 only): every code is split into two 2-bit planes; the K codes area holds
+//   4-bit codes: every code is split into two 2-bit planes; the K codes area holds
 //   plane 0 then plane 1 (32 G bytes each), likewise the V codes area, and the offsets after the
-//   codes move accordingly: tile bytes = 1024 + 128 G = 5120 (160 B per token).
+//   codes move accordingly: tile bytes = 1024 + 128 G (5120 at G = 32, 9216 at G = 64; 160 / 144 B per token).
 //
 //   Fragment coordinates use lane = 4*(lane/4) + j of a warp, as in mma.sync.m16n8k16:
 //   K codes of sub-tile u: 32-bit word 4*lane + 2*nt + w  (lane = 4*n + j), bits

@@ -248,6 +248,8 @@ cudaError_t launch_compress(const CacheView& cv, const LayerList& layers, const 
     lq_compress_kernel<32, 2><<<grid, 256, 0, st>>>(cv, layers, ev, tile0);
   else if (cv.G == 64 && cv.planes == 1)
     lq_compress_kernel<64, 1><<<grid, 256, 0, st>>>(cv, layers, ev, tile0);
+  else if (cv.G == 64 && cv.planes == 2)
+    lq_compress_kernel<64, 2><<<grid, 256, 0, st>>>(cv, layers, ev, tile0);
   else
     return cudaErrorInvalidValue;
   return cudaGetLastError();
@@ -304,6 +306,8 @@ cudaError_t launch_ingest(const CacheView& cv, int layer, const void* k, const v
     lq_ingest_kernel<32, 2><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, n_fp, tile0);
   else if (cv.G == 64 && cv.planes == 1)
     lq_ingest_kernel<64, 1><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, n_fp, tile0);
+  else if (cv.G == 64 && cv.planes == 2)
+    lq_ingest_kernel<64, 2><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, n_fp, tile0);
   else
     return cudaErrorInvalidValue;
   return cudaGetLastError();

@@ -92,6 +92,12 @@ def test_config5_mha_128k_one_layer():
     assert (inf.n_quant, inf.n_fp) == (130560, 513)
 
 
+def test_config4_with_four_bit_codes_at_group_64():
+    # config 4 (GQA-7, W = 256, G = 64) at the paper's second precision and its own group size (Sec. 3.1, Table 3)
+    inf = _run(B=4, Hq=28, Hkv=4, W=256, G=64, ctx=32768, seed=4, n_steps=2, bits=4)
+    assert inf.bytes_quant_per_token == 144
+
+
 def test_config2_with_four_bit_codes():
     # the llama3-8b-8k-int4 workload of bench.py: config 2 at the paper's second precision
     inf = _run(B=8, Hq=32, Hkv=8, W=128, G=32, ctx=8192, seed=2, n_steps=2, bits=4)

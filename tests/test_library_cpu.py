@@ -43,7 +43,7 @@ def _dry(W=4, G=4, **kw):
 
 
 @pytest.mark.parametrize("bad", [dict(group=16), dict(group=48, window=96), dict(head_dim=64),
-                                 dict(bits=3), dict(bits=8), dict(bits=4, group=64, window=128),
+                                 dict(bits=3), dict(bits=8),
                                  dict(n_q_heads=18, n_kv_heads=2), dict(window=1024)])
 def test_unsupported_configurations(bad):
     with pytest.raises(LogQuantError) as e:
