@@ -24,6 +24,11 @@
  *     cache unchanged; every length is a function of the number of appended tokens, so the
  *     host never has to read one back from the device.
  *   - No call throws, aborts or traps.  One cache must not be used from two threads at once.
+ *   - All layers of a cache share one split-K workspace (partial records, arrival counters, sums), and
+ *     the kernels rely on stream order to hand it from one launch to the next: every call on one
+ *     cache must be enqueued on the same stream, or the caller must order the streams with events.
+ *     Calls for different layers on different, unordered streams race on that workspace and give
+ *     wrong results without any error.  Different caches are independent.
  *   - There is no CPU implementation: without a CUDA device lq_cache_create fails, except for
  *     the bookkeeping-only mode device == LQ_DEVICE_NONE in which the compute calls return
  *     LQ_ERR_UNSUPPORTED.
@@ -231,6 +236,21 @@ lq_status_t lq_profile_read(lq_cache_t* cache, double* total_ms, int64_t* n_laun
  * (its output is then invalid).  Kernels never trap or spin for ever; they record the failure
  * here.  Synchronises the device. */
 lq_status_t lq_kernel_status(lq_cache_t* cache, int32_t* status_word);
+
+/* Set the status word back to 0 (after the caller has dealt with a failure).  Synchronises the device. */
+lq_status_t lq_reset_kernel_status(lq_cache_t* cache);
+
+/* Test hook for the failure path (no counterpart in the paper): the next decode-attention launch of this cache
+ * on a tensor-core kernel arms the barrier of its query copy, issues no copy and polls a few hundred times only,
+ * so that its bounded wait runs out.  That launch must set bit 0 of the status word, write nothing to `out` and
+ * return normally; the cache and the CUDA context stay usable.  Nothing on the GPU faults, traps or hangs. */
+lq_status_t lq_debug_stall_next_decode(lq_cache_t* cache);
+
+/* Guard words: every device block a cache allocates (through cudaMalloc or the caller's allocator) is
+ * followed by 256 guard bytes of a fixed pattern that no kernel may touch.  lq_check_guards synchronises the
+ * device, reads them back and stores the number of blocks whose guard was overwritten in *n_damaged
+ * (0 = intact): a cheap stand-in for a memory checker that the tests call on every cache they close. */
+lq_status_t lq_check_guards(lq_cache_t* cache, int32_t* n_damaged);
 
 /* Introspection (host-side bookkeeping only; never synchronises). */
 lq_status_t lq_cache_info(const lq_cache_t* cache, int32_t layer, lq_info_t* info);

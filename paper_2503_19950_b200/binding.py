@@ -3,6 +3,7 @@ from __future__ import annotations
 
 import ctypes as C
 import os
+import weakref
 
 import numpy as np
 
@@ -50,7 +51,8 @@ class lq_device_image_t(C.Structure):
 SYMBOLS = ["lq_cache_create", "lq_destroy", "lq_append", "lq_compress", "lq_decode_attn", "lq_append_decode_attn",
            "lq_decode_attn_fp_only", "lq_set_padding",
            "lq_decode_step_host", "lq_profile_enable", "lq_profile_read", "lq_kernel_status", "lq_cache_info", "lq_export",
-           "lq_next_evicted_ids", "lq_decode_attn_image_static", "lq_status_str", "lq_last_error"]
+           "lq_next_evicted_ids", "lq_decode_attn_image_static", "lq_status_str", "lq_last_error", "lq_check_guards",
+           "lq_reset_kernel_status", "lq_debug_stall_next_decode"]
 
 _lib = None
 
@@ -80,6 +82,9 @@ def load_library():
         L.lq_set_padding.argtypes = [vp, vp]
         L.lq_decode_step_host.argtypes = [vp, i32, vp, vp, vp, C.c_float, vp, i32, vp]
         L.lq_kernel_status.argtypes = [vp, C.POINTER(C.c_int32)]
+        L.lq_check_guards.argtypes = [vp, C.POINTER(C.c_int32)]
+        L.lq_reset_kernel_status.argtypes = [vp]
+        L.lq_debug_stall_next_decode.argtypes = [vp]
         L.lq_profile_enable.argtypes = [vp, i32]
         L.lq_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         L.lq_cache_info.argtypes = [vp, i32, C.POINTER(lq_info_t)]
@@ -135,6 +140,9 @@ def decode_attn_image_static(image: dict, n_q_heads: int, group: int, q, out, sm
 class LogQuantCache:
     """Owner of one lq_cache_t.  Methods mirror the C entry points one to one."""
 
+    live = weakref.WeakSet()   # caches that have not been collected yet (the tests check their guard bytes)
+    guards_on_close = False    # True: close() checks the guard bytes behind every device block and raises if one changed
+
     def __init__(self, n_layers, batch, n_q_heads, n_kv_heads, window, group, max_tokens, head_dim=128, bits=2,
                  auto_compress=True, device=0, kernel=LQ_KERNEL_AUTO, n_splits=0, filter=0, allocator=None):
         """allocator: None (cudaMalloc / cudaFree), "torch" (every device block of the cache is a uint8 tensor from
@@ -142,6 +150,7 @@ class LogQuantCache:
         (alloc(bytes) -> device address or 0, free(address))."""
         self._lib = load_library()
         self._blocks = {}
+        LogQuantCache.live.add(self)
         alloc_cb, free_cb = ALLOC_FN(0), FREE_FN(0)
         if allocator == "torch":
             import torch
@@ -177,8 +186,11 @@ class LogQuantCache:
 
     def close(self):
         if getattr(self, "_h", None):
+            damaged = self.check_guards() if LogQuantCache.guards_on_close else 0
             self._lib.lq_destroy(self._h)
             self._h = None
+            if damaged:
+                raise LogQuantError(LQ_ERR_CUDA, "%d device block(s) of the cache were written past their end" % damaged)
 
     def __del__(self):
         try:
@@ -240,6 +252,18 @@ class LogQuantCache:
         return ms.value, n.value
 
     # -- introspection --------------------------------------------------------------------
+    def check_guards(self) -> int:
+        """Number of device blocks whose guard bytes were overwritten (lq_check_guards; synchronises)."""
+        n = C.c_int32(0)
+        self._check(self._lib.lq_check_guards(self._h, C.byref(n)))
+        return n.value
+
+    def reset_kernel_status(self):
+        self._check(self._lib.lq_reset_kernel_status(self._h))
+
+    def debug_stall_next_decode(self):
+        self._check(self._lib.lq_debug_stall_next_decode(self._h))
+
     def kernel_status(self) -> int:
         w = C.c_int32(0)
         self._check(self._lib.lq_kernel_status(self._h, C.byref(w)))

@@ -54,6 +54,7 @@ struct lq_cache {
   uint8_t* stage_q = nullptr;
   uint8_t* stage_out = nullptr;
   int64_t n_launches = 0;
+  bool stall_next = false;  // lq_debug_stall_next_decode
   // left padding of a ragged batch (lq_set_padding): pad[b] leading positions of sequence b that attention
   // leaves out.  Device copy per layer: [B][4] row info, [B][fp_words] slot mask, [B][q_words] store mask,
   // rebuilt (mask_dirty) when the layer's stores changed.
@@ -70,6 +71,7 @@ struct lq_cache {
   std::vector<cudaEvent_t> ev_pool;  // 2 events per timed launch
   size_t ev_used = 0;
   std::string last_error;
+  std::vector<std::pair<uint8_t*, int64_t>> blocks;  // device blocks (address, payload bytes): guard bytes follow the payload
 };
 
 namespace {
@@ -81,23 +83,45 @@ lq_status_t cuda_fail(lq_cache* c, cudaError_t e, const char* what) {
   return LQ_ERR_CUDA;
 }
 
-bool dev_alloc(lq_cache* c, void** p, int64_t bytes) {
+constexpr int kGuardBytes = 256;       // after every device block; checked by lq_check_guards
+constexpr int kGuardPattern = 0xA5;
+
+// Every device block of a cache -- long-lived or temporary -- comes from here: the caller's allocator when one
+// is set, else cudaMalloc.  `bytes` is rounded up to 256 so that the guard starts on an aligned address.
+bool dev_alloc(lq_cache* c, void** p, int64_t bytes, bool temporary = false) {
+  const int64_t payload = (bytes + 255) / 256 * 256, total = payload + kGuardBytes;
   if (c->cfg.dev_alloc) {  // the caller's allocator
-    *p = c->cfg.dev_alloc(static_cast<size_t>(bytes), c->cfg.alloc_ctx);
+    *p = c->cfg.dev_alloc(static_cast<size_t>(total), c->cfg.alloc_ctx);
     if (*p == nullptr) return false;
-  } else if (cudaMalloc(p, static_cast<size_t>(bytes)) != cudaSuccess) {
+  } else if (cudaMalloc(p, static_cast<size_t>(total)) != cudaSuccess) {
     cudaGetLastError();
     *p = nullptr;
     return false;
   }
-  c->bytes_device += bytes;
+  if (cudaMemset(static_cast<uint8_t*>(*p) + payload, kGuardPattern, kGuardBytes) != cudaSuccess) cudaGetLastError();
+  c->blocks.emplace_back(static_cast<uint8_t*>(*p), payload);
+  if (!temporary) c->bytes_device += total;
   return true;
 }
 
 void dev_release(lq_cache* c, void* p) {
   if (p == nullptr) return;
+  for (size_t i = 0; i < c->blocks.size(); ++i)
+    if (c->blocks[i].first == p) { c->blocks.erase(c->blocks.begin() + i); break; }
   if (c->cfg.dev_free) c->cfg.dev_free(p, c->cfg.alloc_ctx);
   else cudaFree(p);
+}
+
+// number of blocks whose guard bytes no longer hold the pattern (the device must be idle)
+int damaged_guards(const lq_cache* c) {
+  int bad = 0;
+  uint8_t host[kGuardBytes];
+  for (const auto& b : c->blocks) {
+    if (cudaMemcpy(host, b.first + b.second, kGuardBytes, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); ++bad; continue; }
+    for (int i = 0; i < kGuardBytes; ++i)
+      if (host[i] != kGuardPattern) { ++bad; break; }
+  }
+  return bad;
 }
 
 void free_all(lq_cache* c) {
@@ -723,6 +747,8 @@ lq_status_t decode_impl(lq_cache_t* c, int32_t layer, const void* q, float sm_sc
   a.new_slot = new_slot;
   a.tickets = nullptr;
   a.acc = nullptr;
+  a.debug_stall = c->stall_next ? 1 : 0;
+  c->stall_next = false;
   cudaError_t e;
   const bool timed = c->profiling && c->ev_used + 2 <= c->ev_pool.size();
   if (timed) cudaEventRecord(c->ev_pool[c->ev_used], st);
@@ -859,6 +885,21 @@ lq_status_t lq_kernel_status(lq_cache_t* c, int32_t* word) {
   return LQ_OK;
 }
 
+lq_status_t lq_reset_kernel_status(lq_cache_t* c) {
+  if (!c) return LQ_ERR_INVALID_ARG;
+  if (c->dry) return LQ_OK;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemset(c->status, 0, sizeof(int32_t));
+  if (e != cudaSuccess) return cuda_fail(c, e, "status reset");
+  return LQ_OK;
+}
+
+lq_status_t lq_debug_stall_next_decode(lq_cache_t* c) {
+  if (!c) return LQ_ERR_INVALID_ARG;
+  c->stall_next = true;
+  return LQ_OK;
+}
+
 lq_status_t lq_cache_info(const lq_cache_t* c, int32_t layer, lq_info_t* info) {
   if (!c || !info || layer < 0 || layer >= c->cfg.n_layers) return LQ_ERR_INVALID_ARG;
   const LayerState& L = c->layers[layer];
@@ -937,11 +978,11 @@ lq_status_t lq_export(const lq_cache_t* cc, int32_t layer, lq_image_t* img) {
   cudaError_t e = cudaDeviceSynchronize();
   if (e != cudaSuccess) return cuda_fail(c, e, "cudaDeviceSynchronize");
   for (auto& b : bufs)
-    if (b.host && b.bytes > 0 && cudaMalloc(&b.dev, static_cast<size_t>(b.bytes)) != cudaSuccess) status = LQ_ERR_OOM;
+    if (b.host && b.bytes > 0 && !dev_alloc(c, &b.dev, b.bytes, true)) status = LQ_ERR_OOM;
   if (status == LQ_OK && nf > 0) {
     std::vector<int> slots(nf);
     for (int i = 0; i < nf; ++i) slots[i] = rows[i].second;
-    if (cudaMalloc(&slots_dev, nf * sizeof(int)) != cudaSuccess) status = LQ_ERR_OOM;
+    if (!dev_alloc(c, reinterpret_cast<void**>(&slots_dev), nf * sizeof(int), true)) status = LQ_ERR_OOM;
     else cudaMemcpy(slots_dev, slots.data(), nf * sizeof(int), cudaMemcpyHostToDevice);
   }
   if (status == LQ_OK) {
@@ -959,10 +1000,21 @@ lq_status_t lq_export(const lq_cache_t* cc, int32_t layer, lq_image_t* img) {
         e = cudaMemcpy(b.host, b.dev, static_cast<size_t>(b.bytes), cudaMemcpyDeviceToHost);
         if (e != cudaSuccess) { status = cuda_fail(c, e, "export copy"); break; }
       }
-  for (auto& b : bufs) cudaFree(b.dev);
-  cudaFree(slots_dev);
+  // (the device is idle here: a caller's allocator may hand the blocks out again at once)
+  for (auto& b : bufs) dev_release(c, b.dev);
+  dev_release(c, slots_dev);
   if (status == LQ_ERR_OOM) cudaGetLastError();
   return status;
+}
+
+lq_status_t lq_check_guards(lq_cache_t* c, int32_t* n_damaged) {
+  if (!c || !n_damaged) return LQ_ERR_INVALID_ARG;
+  *n_damaged = 0;
+  if (c->dry) return LQ_OK;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(c, e, "cudaDeviceSynchronize");
+  *n_damaged = damaged_guards(c);
+  return LQ_OK;
 }
 
 }  // extern "C"

@@ -704,8 +704,9 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   if (threadIdx.x == 0) {
     // the r query rows of this pair are contiguous: one bulk copy
     mbar_expect_tx(qbar, r * kD * 2);
-    bulk_load(qsm, static_cast<const uint8_t*>(a.q) + (static_cast<int64_t>(b) * cv.Hq + kv * r) * kD * 2, r * kD * 2,
-              qbar);
+    if (!a.debug_stall)
+      bulk_load(qsm, static_cast<const uint8_t*>(a.q) + (static_cast<int64_t>(b) * cv.Hq + kv * r) * kD * 2, r * kD * 2,
+                qbar);
   }
 
   float kc[4];
@@ -772,8 +773,9 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   if (use_acc && warp == 0) k0row = __ldcg(reinterpret_cast<const uint2*>(fpbase) + lane);  // row 0: lane = 4 channels
   {
     int spins = 0;
+    const int limit = a.debug_stall ? 256 : kSpinLimit;
     while (!mbar_try_wait(qbar, 0)) {
-      if (++spins > kSpinLimit) { failed = true; break; }
+      if (++spins > limit) { failed = true; break; }
     }
     failed = __any_sync(kFull, failed);
     if (use_acc && warp == 0) {
@@ -991,7 +993,8 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
 #pragma unroll
       for (int w = 0; w < kWarps; ++w) o = fmaf(wout[(w * 8 + h) * kRow + d], wf[w * 8 + h], o);
       if (n_ctas_pair == 1) {
-        // the only CTA of its pair: this is the final result
+        // the only CTA of its pair: this is the final result (nothing is written after a wait that gave up)
+        if (failed) continue;
         const int64_t oi = (static_cast<int64_t>(b) * cv.Hq + kv * r + h) * kD + d;
         const float res = o / cml[2 * h + 1];
         if (a.out_bf16)
@@ -1022,6 +1025,8 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     __syncthreads();
     if (*is_last) {
       __threadfence();
+      // a CTA of the pair whose wait gave up has set the status word before its ticket: the output stays untouched
+      const bool healthy = (__ldcg(a.status) & 1) == 0;
       // Fast path: the partials have already been summed on arrival (DecodeArgs::acc); one round trip
       // fetches the sums.  It is taken unless a CTA flagged the pair (partial too far above the
       // reference score) or a denominator is not a positive finite number (everything far below it).
@@ -1037,7 +1042,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
           sl[h] = h < r ? __ldcg(accp + kMaxRatio * kD + h) : 1.f;
           so[h] = h < r ? __ldcg(accp + h * kD + d) : 0.f;
         }
-        fast = flagged == 0;
+        fast = flagged == 0 && healthy;
 #pragma unroll
         for (int h = 0; h < RALL; ++h) fast = fast && sl[h] > 0.f && sl[h] < INFINITY;
       }
@@ -1053,6 +1058,8 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
               static_cast<float*>(a.out)[oi] = res;
           }
         }
+      } else if (!healthy) {
+        // nothing is written
       } else if (NCB == 1 && n_ctas_pair <= kMergeOneBatch) {
         // Up to 4 heads and few records: warp w merges head w on its own -- every record of the head in one
         // batch of loads, the weights spread over the lanes and handed round by shuffles -- and writes the

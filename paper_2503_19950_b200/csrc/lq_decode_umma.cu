@@ -92,8 +92,8 @@ __device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity
   return ok;
 }
 // bounded wait: false when the phase did not complete within the poll limit
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (int spin = 0; spin < kSpin; ++spin) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int limit = kSpin) {
+  for (int spin = 0; spin < limit; ++spin) {
     if (mbar_test_wait(bar, parity)) return true;
   }
   return false;
@@ -400,9 +400,10 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
           if (seg >= 2 && !mbar_wait(bar_qfree0 + 8 * qb, ((seg >> 1) - 1) & 1)) { failed = true; break; }
           const int b = static_cast<int>(lpair / cv.Hkv), kv = static_cast<int>(lpair % cv.Hkv);
           mbar_expect_tx(bar_qfull0 + 8 * qb, r * kD * 2);
-          bulk_load(sbase + GE::OFF_Q + qb * (kMaxRatio * kD * 2),
-                    static_cast<const uint8_t*>(a.q) + (static_cast<int64_t>(b) * cv.Hq + kv * r) * kD * 2, r * kD * 2,
-                    bar_qfull0 + 8 * qb);
+          if (!a.debug_stall)
+            bulk_load(sbase + GE::OFF_Q + qb * (kMaxRatio * kD * 2),
+                      static_cast<const uint8_t*>(a.q) + (static_cast<int64_t>(b) * cv.Hq + kv * r) * kD * 2, r * kD * 2,
+                      bar_qfull0 + 8 * qb);
           ++seg;
         }
         const uint8_t* src;
@@ -492,8 +493,9 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
     // j + 1 (q.k) and of item j (p.v) run while the workers go on, so the waits below are normally satisfied.
     bool failed = false;   // warp-uniform: after a wait that ran out no wait is attempted any more; the warp keeps
                            // taking part in every barrier so that nobody is left waiting for it
+    const int spin_limit = a.debug_stall ? 256 : kSpin;
     auto wait = [&](uint32_t bar, uint32_t parity) {
-      if (!failed) failed = !__all_sync(kFullMask, mbar_wait(bar, parity) ? 1 : 0);
+      if (!failed) failed = !__all_sync(kFullMask, mbar_wait(bar, parity, spin_limit) ? 1 : 0);
     };
     uint32_t qpk[GE::BROUNDS][2][4];   // query of the B build: item (group g, chunk c, head pair hp) per round
     float qf[GE::BROUNDS][2][8];
@@ -904,6 +906,7 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
           }
         }
         // ---- arrival: the CTA that brings the pair's item count to I merges its partials ----
+        if (failed && lane == 0) atomicOr(a.status, 1);   // before the ticket: the merging CTA then writes nothing
         __threadfence();
         // which CTAs hold a partial of this pair (their item range meets the pair's): one candidate per thread
         uint8_t* contrib = smem + GE::OFF_MISC + 32;
@@ -929,7 +932,8 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
         named_sync<kBarW, kGroup>();
         if (*reinterpret_cast<volatile int*>(is_last_s)) {
           __threadfence();
-          for (int h = 0; h < r; ++h) {
+          const bool healthy = (__ldcg(a.status) & 1) == 0;   // after a wait that gave up the output stays untouched
+          for (int h = 0; h < r && healthy; ++h) {
             float M = -INFINITY;
             for (int sl = 0; sl < a.S; ++sl) {
               if (!contrib[sl]) continue;

@@ -109,6 +109,9 @@ struct DecodeArgs {
   // 128 quantised tokens: u_items items of total cost u_cost (in units of 2 KB); the pairs' items lie on one cost
   // line that is cut into n_ctas equal ranges; S = record slots per pair
   int u_items, u_fp_units, u_supertiles, u_cost;
+  // test hook (lq_debug_stall_next_decode): the tensor-core kernels arm the barrier of the query copy but issue
+  // no copy and poll with a short limit, so that the bounded wait runs out and the failure path is taken
+  int debug_stall;
 };
 
 constexpr int kAccStride = kMaxRatio * 128 + 32;  // floats per (b, kv) pair in DecodeArgs::acc

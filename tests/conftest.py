@@ -24,3 +24,18 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _guard_bytes_intact(request):
+    """After every GPU test: no kernel wrote past the end of a device block (256 guard bytes follow each block of
+    every cache; lq_check_guards).  Caches closed inside the test are checked by close() itself."""
+    if "gpu" not in request.keywords:
+        yield
+        return
+    from paper_2503_19950_b200 import LogQuantCache
+    LogQuantCache.guards_on_close = True
+    yield
+    for cache in list(LogQuantCache.live):
+        if getattr(cache, "_h", None) and cache.cfg.device >= 0:
+            assert cache.check_guards() == 0, "a kernel wrote past the end of a device block"
