@@ -246,6 +246,14 @@ lq_status_t lq_reset_kernel_status(lq_cache_t* cache);
  * return normally; the cache and the CUDA context stay usable.  Nothing on the GPU faults, traps or hangs. */
 lq_status_t lq_debug_stall_next_decode(lq_cache_t* cache);
 
+/* Test hook of the index-check build (library compiled with -DLQ_DEBUG_BOUNDS, where every index that comes from
+ * the host's bookkeeping is checked in the kernels; no counterpart in the paper): the next lq_append launches
+ * its kernel with a first slot beyond the full-precision store.  The checks must refuse every row, set bit 2
+ * of the status word and write nothing.  The normal build returns LQ_ERR_UNSUPPORTED and changes nothing.
+ * The cache's contents are undefined after the hooked append (its bookkeeping counts rows that were not
+ * written): destroy it. */
+lq_status_t lq_debug_bad_slot_next_append(lq_cache_t* cache);
+
 /* Guard words: every device block a cache allocates (through cudaMalloc or the caller's allocator) is
  * followed by 256 guard bytes of a fixed pattern that no kernel may touch.  lq_check_guards synchronises the
  * device, reads them back and stores the number of blocks whose guard was overwritten in *n_damaged

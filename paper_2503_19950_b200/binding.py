@@ -8,7 +8,8 @@ import weakref
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "liblogquant.so")
+# LOGQUANT_LIBRARY: another build of the same library (e.g. liblogquant_bounds.so, the build with index checks)
+_LIB_PATH = os.environ.get("LOGQUANT_LIBRARY") or os.path.join(_HERE, "liblogquant.so")
 
 LQ_DEVICE_NONE = -1
 LQ_KERNEL_AUTO, LQ_KERNEL_SCALAR, LQ_KERNEL_MMA, LQ_KERNEL_UMMA = 0, 1, 2, 3
@@ -52,7 +53,7 @@ SYMBOLS = ["lq_cache_create", "lq_destroy", "lq_append", "lq_compress", "lq_deco
            "lq_decode_attn_fp_only", "lq_set_padding",
            "lq_decode_step_host", "lq_profile_enable", "lq_profile_read", "lq_kernel_status", "lq_cache_info", "lq_export",
            "lq_next_evicted_ids", "lq_decode_attn_image_static", "lq_status_str", "lq_last_error", "lq_check_guards",
-           "lq_reset_kernel_status", "lq_debug_stall_next_decode"]
+           "lq_reset_kernel_status", "lq_debug_stall_next_decode", "lq_debug_bad_slot_next_append"]
 
 _lib = None
 
@@ -85,6 +86,7 @@ def load_library():
         L.lq_check_guards.argtypes = [vp, C.POINTER(C.c_int32)]
         L.lq_reset_kernel_status.argtypes = [vp]
         L.lq_debug_stall_next_decode.argtypes = [vp]
+        L.lq_debug_bad_slot_next_append.argtypes = [vp]
         L.lq_profile_enable.argtypes = [vp, i32]
         L.lq_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         L.lq_cache_info.argtypes = [vp, i32, C.POINTER(lq_info_t)]
@@ -260,6 +262,9 @@ class LogQuantCache:
 
     def reset_kernel_status(self):
         self._check(self._lib.lq_reset_kernel_status(self._h))
+
+    def debug_bad_slot_next_append(self):
+        self._check(self._lib.lq_debug_bad_slot_next_append(self._h))
 
     def debug_stall_next_decode(self):
         self._check(self._lib.lq_debug_stall_next_decode(self._h))

@@ -55,6 +55,7 @@ struct lq_cache {
   uint8_t* stage_out = nullptr;
   int64_t n_launches = 0;
   bool stall_next = false;  // lq_debug_stall_next_decode
+  bool bad_slot_next = false;  // lq_debug_bad_slot_next_append (index-check build only)
   // left padding of a ragged batch (lq_set_padding): pad[b] leading positions of sequence b that attention
   // leaves out.  Device copy per layer: [B][4] row info, [B][fp_words] slot mask, [B][q_words] store mask,
   // rebuilt (mask_dirty) when the layer's stores changed.
@@ -480,6 +481,7 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_out),
                         static_cast<int64_t>(cfg->n_layers) * cfg->batch * cfg->n_q_heads * kD * 4);
     if (ok) ok = cudaMemset(c->status, 0, 256) == cudaSuccess;
+    cv.status = c->status;
     if (ok) ok = cudaMemset(c->tickets, 0, pairs * 128) == cudaSuccess;
     if (ok) ok = cudaMemset(c->acc, 0, static_cast<size_t>(pairs) * kAccStride * 4) == cudaSuccess;
     // the fp store must never hold non-finite garbage in unused slots of a partly filled tile
@@ -586,7 +588,10 @@ lq_status_t append_impl(lq_cache_t* c, int32_t layer, const void* k, const void*
     const int take = std::min(n - done, 3 * W - kept(L));
     if (!c->dry) {
       const bool last = done + take == n;
-      cudaError_t e = launch_append(c->cv, layer, k, v, n, done, take, L.n_fp, st, last ? extra_src : nullptr,
+      // (test hook of the index-check build: a first slot beyond the store, which the kernel's check must refuse)
+      const int slot0 = L.n_fp + (c->bad_slot_next ? static_cast<int>(fp_slots_cap(c->cv)) : 0);
+      c->bad_slot_next = false;
+      cudaError_t e = launch_append(c->cv, layer, k, v, n, done, take, slot0, st, last ? extra_src : nullptr,
                                     last ? extra_dst : nullptr, last ? extra_bytes : 0);
       if (e != cudaSuccess) return cuda_fail(c, e, "lq_append_kernel");
       c->n_launches++;
@@ -892,6 +897,16 @@ lq_status_t lq_reset_kernel_status(lq_cache_t* c) {
   if (e == cudaSuccess) e = cudaMemset(c->status, 0, sizeof(int32_t));
   if (e != cudaSuccess) return cuda_fail(c, e, "status reset");
   return LQ_OK;
+}
+
+lq_status_t lq_debug_bad_slot_next_append(lq_cache_t* c) {
+  if (!c) return LQ_ERR_INVALID_ARG;
+#ifdef LQ_DEBUG_BOUNDS
+  c->bad_slot_next = true;
+  return LQ_OK;
+#else
+  return LQ_ERR_UNSUPPORTED;  // without the checks the rows would really be written out of range
+#endif
 }
 
 lq_status_t lq_debug_stall_next_decode(lq_cache_t* c) {

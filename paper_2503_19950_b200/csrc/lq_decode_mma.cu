@@ -749,8 +749,12 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     const uint32_t s = issued % kStages;
     if (s == 0) desc0 = desc; else if (s == 1) desc1 = desc; else desc2 = desc;
     if (lane == 0) {
+      // (debug build: the copy must lie inside this pair's part of the store it reads; a copy that does not is
+      // not issued, its barrier never completes and the bounded wait reports it as well)
+      const bool inside = desc < a.tiles_fp ? src >= fpbase && src + bytes <= fpbase + cv.fp_head_stride
+                                            : src >= qbase && src + bytes <= qbase + cv.quant_head_stride;
       mbar_expect_tx(bar0 + 8 * s, bytes);
-      bulk_load(stage0 + s * kStageBytes, src, bytes, bar0 + 8 * s);
+      if (LQ_IN_BOUNDS(cv, inside)) bulk_load(stage0 + s * kStageBytes, src, bytes, bar0 + 8 * s);
     }
     ++issued;
   };
@@ -1001,7 +1005,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
           static_cast<__nv_bfloat16*>(a.out)[oi] = __float2bfloat16_rn(res);
         else
           static_cast<float*>(a.out)[oi] = res;
-      } else {
+      } else if (LQ_IN_BOUNDS(cv, slot < a.S)) {
         a.part_o[(rec + h) * kD + d] = o;
         if (use_acc && wsc[h] > 0.f) atomicAdd(a.acc + static_cast<int64_t>(pair) * kAccStride + h * kD + d, o * wsc[h]);
         if (d == 0) {

@@ -416,8 +416,12 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
           src = quant_layer + lpair * cv.quant_head_stride + static_cast<int64_t>(st) * NGS * TILE;
           bytes = min(NGS, a.tiles_quant - st * NGS) * TILE;
         }
+        // (debug build: the copy must lie inside this pair's part of the store it reads)
+        const uint8_t* lo = lli < cut.F ? fp_layer + lpair * cv.fp_head_stride : quant_layer + lpair * cv.quant_head_stride;
+        const int64_t extent = lli < cut.F ? cv.fp_head_stride : cv.quant_head_stride;
         mbar_expect_tx(bar_full(s), bytes);
-        bulk_load(sbase + GE::OFF_STAGES + s * kStageBytes, src, bytes, bar_full(s));
+        if (LQ_IN_BOUNDS(cv, lpair < cut.P && src >= lo && src + bytes <= lo + extent))
+          bulk_load(sbase + GE::OFF_STAGES + s * kStageBytes, src, bytes, bar_full(s));
         if (++lli == cut.I) { lli = 0; ++lpair; }
       }
       if (failed) atomicOr(a.status, 1);
@@ -895,7 +899,7 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
         const int64_t rec = (pair * a.S + slot) * r;
 #pragma unroll
         for (int h = 0; h < HP; ++h) {
-          if (h < r) {
+          if (h < r && LQ_IN_BOUNDS(cv, slot >= 0 && slot < a.S)) {
             const float zsum = red[8 + vg * 8 + h] + red[48 + 8 + vg * 8 + h] + red[96 + 8 + vg * 8 + h] + red[144 + 8 + vg * 8 + h];
             const float val = fmaf(__uint_as_float(o[2 * h]) + __uint_as_float(o[2 * h + 1]), 0x1p69f, zsum);
             a.part_o[(rec + h) * kD + d] = val;

@@ -19,7 +19,23 @@ struct CacheView {
   int64_t fp_layer_stride;
   uint8_t* quant;  // 2-bit store base
   uint8_t* fp;     // full-precision store base
+  int* status;     // the cache's device status word (bit 0: a bounded wait gave up; bit 2: an index check of
+                   // the LQ_DEBUG_BOUNDS build failed)
 };
+
+// Index checks of the debug build (-DLQ_DEBUG_BOUNDS, python -m paper_2503_19950_b200.build --bounds): every
+// access whose index comes from the host's bookkeeping or from a launch argument is checked against the extent
+// of the store it goes to; a failing check sets bit 2 of the status word and the access is skipped -- nothing
+// traps.  In the normal build the checks compile to nothing.
+#ifdef LQ_DEBUG_BOUNDS
+#define LQ_IN_BOUNDS(cv, cond) ((cond) ? true : (atomicOr((cv).status, 4), false))
+#else
+#define LQ_IN_BOUNDS(cv, cond) true
+#endif
+// slots of the full-precision store of one (layer, b, kv); tiles of the 2-bit store
+__host__ __device__ inline int64_t fp_slots_cap(const CacheView& cv) {
+  return cv.fp_head_stride / (2 * kD * 2);
+}
 
 struct EvictList {
   uint16_t slot[kMaxW];  // physical fp slots of the tokens to quantise, in removal order

@@ -34,6 +34,7 @@ lq_append_kernel(CacheView cv, int layer, const uint4* __restrict__ k, const uin
   const uint4* src = (which ? v : k) + ((pair * n_src + src0 + t) * 16 + c);
   uint8_t* base = cv.fp + layer * cv.fp_layer_stride + pair * cv.fp_head_stride;
   const int64_t off = fp_chunk_off(cv.layout, slot0 + t, c) + (which ? fp_v_delta(cv.layout) : 0);
+  if (!LQ_IN_BOUNDS(cv, slot0 + t >= 0 && slot0 + t < fp_slots_cap(cv) && src0 + t < n_src)) return;
   *reinterpret_cast<uint4*>(base + off) = *src;
 }
 
@@ -215,10 +216,12 @@ lq_compress_kernel(CacheView cv, LayerList layers, EvictList ev, int64_t tile0) 
   uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
                   (tile0 + tau) * quant_tile_bytes(G, P);
 
+  if (!LQ_IN_BOUNDS(cv, tile0 + tau >= 0 && tile0 + tau < cv.quant_tiles_cap)) return;
   // 1. gather the removed rows
   for (int idx = tid; idx < G * 32; idx += 256) {
     const int c = idx & 15, which = (idx >> 4) & 1, e = idx >> 5;
     const int slot = ev.slot[tau * G + e];
+    if (!LQ_IN_BOUNDS(cv, slot < fp_slots_cap(cv))) continue;
     const uint4 val = *reinterpret_cast<const uint4*>(fpbase + fp_chunk_off(cv.layout, slot, c) +
                                                       (which ? fp_v_delta(cv.layout) : 0));
     *reinterpret_cast<uint4*>(which ? &sV[e][c * 8] : &sK[e][c * 8]) = val;
@@ -231,6 +234,7 @@ lq_compress_kernel(CacheView cv, LayerList layers, EvictList ev, int64_t tile0) 
     const int dst = ev.slot[tau * G + e];
     const int src = ev.src[tau * G + e];
     if (src == kNoMove) continue;
+    if (!LQ_IN_BOUNDS(cv, src < fp_slots_cap(cv) && dst < fp_slots_cap(cv))) continue;
     const int vo = which ? fp_v_delta(cv.layout) : 0;
     const uint4 val = *reinterpret_cast<const uint4*>(fpbase + fp_chunk_off(cv.layout, src, c) + vo);
     *reinterpret_cast<uint4*>(fpbase + fp_chunk_off(cv.layout, dst, c) + vo) = val;
@@ -276,9 +280,11 @@ lq_ingest_kernel(CacheView cv, int layer, const uint4* __restrict__ k, const uin
     const int tau = blockIdx.x;
     uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
                     (tile0 + tau) * quant_tile_bytes(G, P);
+    if (!LQ_IN_BOUNDS(cv, tile0 + tau >= 0 && tile0 + tau < cv.quant_tiles_cap)) return;
     for (int i = tid; i < G * 32; i += 256) {
       const int c = i & 15, which = (i >> 4) & 1, e = i >> 5;
-      const int64_t t = idx[tau * G + e];
+      int64_t t = idx[tau * G + e];
+      if (!LQ_IN_BOUNDS(cv, t >= 0 && t < n_src)) t = 0;
       const uint4 val = (which ? v : k)[(pair * n_src + t) * 16 + c];
       *reinterpret_cast<uint4*>(which ? &sV[e][c * 8] : &sK[e][c * 8]) = val;
     }
@@ -289,6 +295,7 @@ lq_ingest_kernel(CacheView cv, int layer, const uint4* __restrict__ k, const uin
     if (i >= n_fp * 32) return;
     const int c = i & 15, which = (i >> 4) & 1, slot = i >> 5;
     const int64_t t = idx[n_tiles * G + slot];
+    if (!LQ_IN_BOUNDS(cv, t >= 0 && t < n_src && slot < fp_slots_cap(cv))) return;
     uint8_t* base = cv.fp + layer * cv.fp_layer_stride + pair * cv.fp_head_stride;
     *reinterpret_cast<uint4*>(base + fp_chunk_off(cv.layout, slot, c) + (which ? fp_v_delta(cv.layout) : 0)) =
         (which ? v : k)[(pair * n_src + t) * 16 + c];
