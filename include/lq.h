@@ -266,6 +266,18 @@ lq_status_t lq_cache_info(const lq_cache_t* cache, int32_t layer, lq_info_t* inf
 /* Copy the canonical image of one layer into the caller's HOST buffers.  Synchronises the device. */
 lq_status_t lq_export(const lq_cache_t* cache, int32_t layer, lq_image_t* image_host);
 
+/* Load a canonical image (as lq_export wrote it; HOST buffers) into a layer that is still EMPTY: the inverse of
+ * lq_export, for checkpoint / resume (no counterpart in the paper).  n_seen = tokens the exported layer had seen
+ * (lq_info_t.n_seen), n_fp and n_quant = its sizes.  Algorithm 1 never looks at the data, so the library
+ * rebuilds its bookkeeping by replaying n_seen appends on token ids and then writes both stores from the image
+ * in its private layout; decode and further appends continue exactly as on the exported cache.  The cache must
+ * have the exporting cache's batch, heads, window, group, bits and filter (its kernel, hence its device layout,
+ * may differ); image->kept_ids and image->quant_ids, when not NULL, are compared with the replayed lists.
+ * LQ_ERR_INVALID_ARG: layer not empty, sizes or id lists that are not those of this configuration after n_seen
+ * tokens, or a missing array; nothing changes then.  Synchronises the device. */
+lq_status_t lq_import(lq_cache_t* cache, int32_t layer, const lq_image_t* image_host, int64_t n_seen, int64_t n_fp,
+                      int64_t n_quant);
+
 /* Host-side bookkeeping only (works in LQ_DEVICE_NONE mode): ids of the tokens the next
  * lq_compress on `layer` would remove, in removal order (W entries; LQ_ERR_NOT_FULL if the
  * layer holds fewer than 3W full-precision tokens). */

@@ -53,7 +53,7 @@ SYMBOLS = ["lq_cache_create", "lq_destroy", "lq_append", "lq_compress", "lq_deco
            "lq_decode_attn_fp_only", "lq_set_padding",
            "lq_decode_step_host", "lq_profile_enable", "lq_profile_read", "lq_kernel_status", "lq_cache_info", "lq_export",
            "lq_next_evicted_ids", "lq_decode_attn_image_static", "lq_status_str", "lq_last_error", "lq_check_guards",
-           "lq_reset_kernel_status", "lq_debug_stall_next_decode", "lq_debug_bad_slot_next_append"]
+           "lq_reset_kernel_status", "lq_debug_stall_next_decode", "lq_debug_bad_slot_next_append", "lq_import"]
 
 _lib = None
 
@@ -91,6 +91,7 @@ def load_library():
         L.lq_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         L.lq_cache_info.argtypes = [vp, i32, C.POINTER(lq_info_t)]
         L.lq_export.argtypes = [vp, i32, C.POINTER(lq_image_t)]
+        L.lq_import.argtypes = [vp, i32, C.POINTER(lq_image_t), C.c_int64, C.c_int64, C.c_int64]
         L.lq_next_evicted_ids.argtypes = [vp, i32, vp]
         L.lq_decode_attn_image_static.argtypes = [C.POINTER(lq_device_image_t), vp, C.c_float, vp, vp]
         L.lq_status_str.argtypes = [i32]
@@ -304,3 +305,10 @@ class LogQuantCache:
         st = lq_image_t(**{k: (v.ctypes.data if v.size else None) for k, v in img.items()})
         self._check(self._lib.lq_export(self._h, layer, C.byref(st)))
         return img
+
+    def import_image(self, layer, img: dict, n_seen: int):
+        """lq_import: load an image made by export() into an empty layer (sizes are taken from the arrays)."""
+        arrs = {k: np.ascontiguousarray(v) for k, v in img.items()}
+        st = lq_image_t(**{k: (v.ctypes.data if v.size else None) for k, v in arrs.items()})
+        self._check(self._lib.lq_import(self._h, layer, C.byref(st), int(n_seen), int(arrs["kept_ids"].size),
+                                        int(arrs["quant_ids"].size)))

@@ -511,30 +511,32 @@ namespace {
 // A prompt appended to an empty layer: the host plays Algorithm 1 token by token on its mirror of
 // the filter (which never looks at the data), collects the removed token ids of every overflow
 // step and the final slot map, and one kernel writes both stores.
-lq_status_t ingest_prompt(lq_cache* c, int layer, const void* k, const void* v, int n, cudaStream_t st) {
-  LayerState& L = c->layers[layer];
-  if (!c->mask_dirty.empty()) c->mask_dirty[layer] = 1;
+// host bookkeeping of one overflow of layer L (no device work); idx, when given, collects the ids of the tokens that
+// enter the 2-bit store, in store order
+void host_event(const lq_cache* c, LayerState& L, std::vector<int32_t>* idx) {
   const int W = c->cfg.window, G = c->cfg.group;
-  std::vector<int32_t> idx;
-  idx.reserve(static_cast<size_t>(n) + 3 * W);
   std::vector<int32_t> ids(std::max(W, G));
-  int done = 0;
-  while (done < n) {
-    if (kept(L) == 3 * W) {
-      if (residual_mode(c)) {
-        apply_event_residual(c, L);
-        while (static_cast<int>(L.pend_slot.size()) >= G) {
-          EvictList unused;
-          plan_group_residual(c, L, &unused, ids.data());
-          idx.insert(idx.end(), ids.begin(), ids.begin() + G);
-        }
-      } else {
-        next_evicted(c, L, nullptr, ids.data());
-        idx.insert(idx.end(), ids.begin(), ids.end());
-        apply_event(c, L);
-      }
+  if (residual_mode(c)) {
+    apply_event_residual(c, L);
+    while (static_cast<int>(L.pend_slot.size()) >= G) {
+      EvictList unused;
+      plan_group_residual(c, L, &unused, ids.data());
+      if (idx) idx->insert(idx->end(), ids.begin(), ids.begin() + G);
     }
-    const int take = std::min(n - done, 3 * W - kept(L));
+  } else {
+    next_evicted(c, L, nullptr, ids.data());
+    if (idx) idx->insert(idx->end(), ids.begin(), ids.end());
+    apply_event(c, L);
+  }
+}
+
+// host bookkeeping of n tokens appended one by one with the overflow step run whenever the window is full
+void replay_appends(const lq_cache* c, LayerState& L, int64_t n, std::vector<int32_t>* idx) {
+  const int W = c->cfg.window;
+  int64_t done = 0;
+  while (done < n) {
+    if (kept(L) == 3 * W) host_event(c, L, idx);
+    const int take = static_cast<int>(std::min<int64_t>(n - done, 3 * W - kept(L)));
     for (int t = 0; t < take; ++t) {
       L.age_slot.push_back(L.n_fp + t);
       L.slot_token[L.n_fp + t] = static_cast<int32_t>(L.n_seen + t);
@@ -543,6 +545,15 @@ lq_status_t ingest_prompt(lq_cache* c, int layer, const void* k, const void* v, 
     L.n_seen += take;
     done += take;
   }
+}
+
+lq_status_t ingest_prompt(lq_cache* c, int layer, const void* k, const void* v, int n, cudaStream_t st) {
+  LayerState& L = c->layers[layer];
+  if (!c->mask_dirty.empty()) c->mask_dirty[layer] = 1;
+  const int W = c->cfg.window, G = c->cfg.group;
+  std::vector<int32_t> idx;
+  idx.reserve(static_cast<size_t>(n) + 3 * W);
+  replay_appends(c, L, n, &idx);
   const int n_tiles = static_cast<int>(idx.size()) / G;
   for (int s = 0; s < L.n_fp; ++s) idx.push_back(L.slot_token[s]);
   // pageable source: the runtime stages it before the call returns, so `idx` may die here
@@ -1019,6 +1030,76 @@ lq_status_t lq_export(const lq_cache_t* cc, int32_t layer, lq_image_t* img) {
   for (auto& b : bufs) dev_release(c, b.dev);
   dev_release(c, slots_dev);
   if (status == LQ_ERR_OOM) cudaGetLastError();
+  return status;
+}
+
+lq_status_t lq_import(lq_cache_t* c, int32_t layer, const lq_image_t* img, int64_t n_seen, int64_t n_fp, int64_t n_quant) {
+  if (!c || !img || layer < 0 || layer >= c->cfg.n_layers) return LQ_ERR_INVALID_ARG;
+  if (c->dry) return LQ_ERR_UNSUPPORTED;
+  LayerState& L = c->layers[layer];
+  if (L.n_seen != 0 || n_seen <= 0 || n_fp < 0 || n_quant < 0) return LQ_ERR_INVALID_ARG;
+  if (n_seen > c->cfg.max_tokens) return LQ_ERR_CAPACITY;
+  const bool have_q = img->k_codes && img->v_codes && img->k_scale && img->k_zero && img->v_scale && img->v_zero;
+  if ((n_quant > 0 && !have_q) || (n_fp > 0 && (!img->fp_k || !img->fp_v))) return LQ_ERR_INVALID_ARG;
+  // The filter never looks at the data: the layer's bookkeeping is that of n_seen single appends.  A layer that was
+  // full when it was exported may or may not have had its overflow step run (lq_compress with auto_compress = 0):
+  // the sizes tell.
+  const LayerState saved = L;
+  replay_appends(c, L, n_seen, nullptr);
+  if ((L.n_fp != n_fp || L.n_quant != n_quant) && kept(L) == 3 * c->cfg.window) host_event(c, L, nullptr);
+  std::vector<std::pair<int32_t, int32_t>> rows;  // (token id, slot), ascending ids as in the image
+  for (int slot : L.age_slot) rows.emplace_back(L.slot_token[slot], slot);
+  for (int slot : L.pend_slot) rows.emplace_back(L.slot_token[slot], slot);
+  std::sort(rows.begin(), rows.end());
+  bool match = L.n_fp == n_fp && L.n_quant == n_quant;
+  if (match && img->kept_ids)
+    for (int64_t i = 0; i < n_fp && match; ++i) match = img->kept_ids[i] == rows[i].first;
+  if (match && img->quant_ids)
+    for (int64_t i = 0; i < n_quant && match; ++i) match = img->quant_ids[i] == L.quant_ids[i];
+  if (!match) {  // not an image of this configuration after n_seen tokens
+    L = saved;
+    return LQ_ERR_INVALID_ARG;
+  }
+  const int64_t pairs = static_cast<int64_t>(c->cfg.batch) * c->cfg.n_kv_heads;
+  const int G = c->cfg.group;
+  const int64_t sz_codes = pairs * n_quant * (kD * c->cfg.bits / 8), sz_kp = pairs * (n_quant / G) * kD * 2,
+                sz_vp = pairs * n_quant * (kD / G) * 2, sz_fp = pairs * n_fp * kD * 2;
+  struct Buf { const void* host; int64_t bytes; void* dev; };
+  Buf bufs[8] = {{img->k_codes, sz_codes, nullptr}, {img->v_codes, sz_codes, nullptr},
+                 {img->k_scale, sz_kp, nullptr},    {img->k_zero, sz_kp, nullptr},
+                 {img->v_scale, sz_vp, nullptr},    {img->v_zero, sz_vp, nullptr},
+                 {img->fp_k, sz_fp, nullptr},       {img->fp_v, sz_fp, nullptr}};
+  int* slots_dev = nullptr;
+  lq_status_t status = LQ_OK;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) status = cuda_fail(c, e, "cudaDeviceSynchronize");
+  for (auto& b : bufs) {
+    if (status != LQ_OK || b.bytes == 0) continue;
+    if (!dev_alloc(c, &b.dev, b.bytes, true)) status = LQ_ERR_OOM;
+    else if ((e = cudaMemcpy(b.dev, b.host, static_cast<size_t>(b.bytes), cudaMemcpyHostToDevice)) != cudaSuccess)
+      status = cuda_fail(c, e, "import copy");
+  }
+  if (status == LQ_OK && n_fp > 0) {
+    std::vector<int> slots(n_fp);
+    for (int64_t i = 0; i < n_fp; ++i) slots[i] = rows[i].second;
+    if (!dev_alloc(c, reinterpret_cast<void**>(&slots_dev), n_fp * sizeof(int), true)) status = LQ_ERR_OOM;
+    else cudaMemcpy(slots_dev, slots.data(), n_fp * sizeof(int), cudaMemcpyHostToDevice);
+  }
+  if (status == LQ_OK) {
+    e = launch_import(c->cv, layer, static_cast<int>(n_fp), n_quant, slots_dev,
+                      static_cast<const uint8_t*>(bufs[0].dev), static_cast<const uint8_t*>(bufs[1].dev),
+                      static_cast<const uint16_t*>(bufs[2].dev), static_cast<const uint16_t*>(bufs[3].dev),
+                      static_cast<const uint16_t*>(bufs[4].dev), static_cast<const uint16_t*>(bufs[5].dev),
+                      static_cast<const uint16_t*>(bufs[6].dev), static_cast<const uint16_t*>(bufs[7].dev), nullptr);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) status = cuda_fail(c, e, "import kernels");
+    c->n_launches += (n_quant > 0) + (n_fp > 0);
+  }
+  for (auto& b : bufs) dev_release(c, b.dev);
+  dev_release(c, slots_dev);
+  if (status == LQ_ERR_OOM) cudaGetLastError();
+  if (status != LQ_OK) L = saved;
+  else if (!c->mask_dirty.empty()) c->mask_dirty[layer] = 1;
   return status;
 }
 

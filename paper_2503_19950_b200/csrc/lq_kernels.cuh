@@ -72,6 +72,12 @@ cudaError_t launch_export(const CacheView& cv, int layer, int n_fp, int64_t n_qu
                           uint16_t* k_scale, uint16_t* k_zero, uint16_t* v_scale, uint16_t* v_zero,
                           uint16_t* fp_k, uint16_t* fp_v, cudaStream_t st);
 
+// Canonical import of one (empty) layer from device copies of the image arrays: the inverse of launch_export.
+cudaError_t launch_import(const CacheView& cv, int layer, int n_fp, int64_t n_quant, const int* slot_of_rank_dev,
+                          const uint8_t* k_codes, const uint8_t* v_codes, const uint16_t* k_scale,
+                          const uint16_t* k_zero, const uint16_t* v_scale, const uint16_t* v_zero,
+                          const uint16_t* fp_k, const uint16_t* fp_v, cudaStream_t st);
+
 // Split-K partial state: for partition s of head pair p = b*Hkv + kv and query head j of the
 // group (j < r): o[128] unnormalised, m (in log2 units), l.
 //   part_o : [(p*S + s)*r + j][128] float,  part_ml : [(p*S + s)*r + j][2] float

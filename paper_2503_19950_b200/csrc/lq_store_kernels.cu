@@ -415,4 +415,85 @@ cudaError_t launch_export(const CacheView& cv, int layer, int n_fp, int64_t n_qu
   return cudaGetLastError();
 }
 
+
+// ---------------------------------------------------------------------------------------
+// Canonical import (checkpoint / resume; the inverse of the export above; not on the hot path).
+// One CTA per (key group, pair) builds the tile in shared memory -- codes by atomicOr into the words the
+// layout assigns them, scale and zero by plain 16-bit stores -- and writes it out with 16-byte stores.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+lq_import_tile_kernel(CacheView cv, int layer, int64_t n_quant, const uint8_t* __restrict__ k_codes,
+                      const uint8_t* __restrict__ v_codes, const uint16_t* __restrict__ k_scale,
+                      const uint16_t* __restrict__ k_zero, const uint16_t* __restrict__ v_scale,
+                      const uint16_t* __restrict__ v_zero) {
+  __shared__ __align__(16) uint32_t sm[quant_tile_bytes(64, 2) / 4];
+  const int G = cv.G, P = cv.planes, NG = kD / G, cpb = 4 / P;
+  const int tile_bytes = quant_tile_bytes(G, P);
+  const int64_t grp = blockIdx.x, pair = blockIdx.y;
+  const int tid = threadIdx.x;
+  if (!LQ_IN_BOUNDS(cv, grp < cv.quant_tiles_cap)) return;
+  for (int i = tid; i < tile_bytes / 4; i += 256) sm[i] = 0u;
+  __syncthreads();
+  uint16_t* sm16 = reinterpret_cast<uint16_t*>(sm);
+  for (int idx = tid; idx < G * kD; idx += 256) {
+    const int t = idx / kD, d = idx % kD;
+    const int64_t byte = (pair * n_quant + grp * G + t) * (kD / cpb) + d / cpb;
+    const uint32_t kcode = (k_codes[byte] >> (2 * P * (d % cpb))) & ((1u << (2 * P)) - 1u);
+    const uint32_t vcode = (v_codes[byte] >> (2 * P * (d % cpb))) & ((1u << (2 * P)) - 1u);
+    for (int pl = 0; pl < P; ++pl) {
+      int off, bit;
+      kcode_pos(cv.layout, G, P, pl, t, d, off, bit);
+      atomicOr(&sm[off >> 2], ((kcode >> (2 * pl)) & 3u) << bit);
+      vcode_pos(cv.layout, G, P, pl, t, d, off, bit);
+      atomicOr(&sm[off >> 2], ((vcode >> (2 * pl)) & 3u) << bit);
+    }
+  }
+  for (int d = tid; d < kD; d += 256) {
+    const int64_t i = (pair * (n_quant / G) + grp) * kD + d;
+    sm16[kscale_off(cv.layout, G, d) >> 1] = k_scale[i];
+    sm16[kzero_off(cv.layout, G, d) >> 1] = k_zero[i];
+  }
+  for (int idx = tid; idx < G * NG; idx += 256) {
+    const int t = idx / NG, g = idx % NG;
+    const int64_t i = (pair * n_quant + grp * G + t) * NG + g;
+    sm16[vscale_off(cv.layout, G, P, t, g) >> 1] = v_scale[i];
+    sm16[vzero_off(cv.layout, G, P, t, g) >> 1] = v_zero[i];
+  }
+  __syncthreads();
+  uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride + grp * tile_bytes;
+  for (int i = tid; i < tile_bytes / 16; i += 256)
+    reinterpret_cast<uint4*>(tile)[i] = reinterpret_cast<const uint4*>(sm)[i];
+}
+
+__global__ void lq_import_fp_kernel(CacheView cv, int layer, int n_fp, const int* __restrict__ slot_of_rank,
+                                    const uint4* __restrict__ fp_k, const uint4* __restrict__ fp_v) {
+  const int64_t total = static_cast<int64_t>(cv.B) * cv.Hkv * n_fp * 16;
+  for (int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; idx < total;
+       idx += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int c = static_cast<int>(idx & 15);
+    const int rank = static_cast<int>((idx >> 4) % n_fp);
+    const int64_t pair = (idx >> 4) / n_fp;
+    const int slot = slot_of_rank[rank];
+    if (!LQ_IN_BOUNDS(cv, slot >= 0 && slot < fp_slots_cap(cv))) continue;
+    uint8_t* base = cv.fp + layer * cv.fp_layer_stride + pair * cv.fp_head_stride;
+    const int64_t off = fp_chunk_off(cv.layout, slot, c);
+    *reinterpret_cast<uint4*>(base + off) = fp_k[idx];
+    *reinterpret_cast<uint4*>(base + off + fp_v_delta(cv.layout)) = fp_v[idx];
+  }
+}
+
+cudaError_t launch_import(const CacheView& cv, int layer, int n_fp, int64_t n_quant, const int* slot_of_rank_dev,
+                          const uint8_t* k_codes, const uint8_t* v_codes, const uint16_t* k_scale,
+                          const uint16_t* k_zero, const uint16_t* v_scale, const uint16_t* v_zero,
+                          const uint16_t* fp_k, const uint16_t* fp_v, cudaStream_t st) {
+  if (n_quant > 0) {
+    dim3 grid(static_cast<unsigned>(n_quant / cv.G), cv.B * cv.Hkv);
+    lq_import_tile_kernel<<<grid, 256, 0, st>>>(cv, layer, n_quant, k_codes, v_codes, k_scale, k_zero, v_scale, v_zero);
+  }
+  if (n_fp > 0)
+    lq_import_fp_kernel<<<1184, 256, 0, st>>>(cv, layer, n_fp, slot_of_rank_dev, reinterpret_cast<const uint4*>(fp_k),
+                                              reinterpret_cast<const uint4*>(fp_v));
+  return cudaGetLastError();
+}
+
 }  // namespace lq
