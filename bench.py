@@ -172,7 +172,7 @@ def run_ours(args, wl, rank, world, device):
     total_steps = 2 * (steps + warmup) + steps + warmup + 8  # device-timed, profiled and host-buffer passes
     bits = wl.get("bits", 2)
     cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=ctx + total_steps + 8, device=device.index or 0, bits=bits,
-                          n_splits=args.n_splits, kernel=KERNELS[args.kernel])
+                          n_splits=args.n_splits, kernel=KERNELS[args.kernel], flags=0 if args.no_overlap else 1)
     pad = wl.get("pad")
     n_pad = sum(pad) if pad else 0
     if pad:
@@ -336,6 +336,10 @@ def run_ours(args, wl, rank, world, device):
                    "merge": ("partials summed on arrival with global atomics (more than 12 CTAs per (b, kv) pair; not "
                              "bit-reproducible), records as fallback" if int(inf.n_splits) >= 12 else
                              "ordered merge of the CTA records by the last CTA of a pair (bit-reproducible)"),
+                   "launch_overlap": ("every launch waits for the one before it" if args.no_overlap else
+                                      "LQ_FLAG_OVERLAP_DECODE: attention launches of consecutive layers overlap (a launch streams its "
+                                      "own layer's stores while the previous one merges, and waits for it before the shared "
+                                      "workspace); roofline.serialized is the same kernel without it"),
                    "replicas": "independent per GPU, no collective on the data path"},
         "per_layer_us": ms_max / steps / L * 1e3,
         "algorithmic_gbs_whole_step": bytes_step_last / (ms_max / steps * 1e-3) / 1e9,
@@ -374,7 +378,7 @@ def run_ours(args, wl, rank, world, device):
     return line, cache
 
 
-def roofline_only(name, device, layers, rounds=24, n_splits=0, kernel=0):
+def roofline_only(name, device, layers, rounds=24, n_splits=0, kernel=0, flags=1):
     """Back-to-back timing of the attention kernel on another workload (a few layer caches, a few seconds):
     the same measurement as the `roofline` object of the main line."""
     from paper_2503_19950_b200 import LogQuantCache
@@ -382,7 +386,7 @@ def roofline_only(name, device, layers, rounds=24, n_splits=0, kernel=0):
     wl["_outliers"] = synth.outlier_channels(wl["seed"], wl["Hkv"], D, wl["n_outliers"]) if wl["n_outliers"] else None
     L, B, Hq, Hkv, W, G, ctx = (wl[k] for k in ("L", "B", "Hq", "Hkv", "W", "G", "ctx"))
     cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=ctx + 64, device=device.index or 0, bits=wl.get("bits", 2),
-                          n_splits=n_splits, kernel=kernel)
+                          n_splits=n_splits, kernel=kernel, flags=flags)
     prefill(cache, wl, device)
     ks, vs, qs = make_step_inputs(wl, device, 4)
     outs = [torch.empty(B, Hq, D, device=device) for _ in range(L)]
@@ -546,6 +550,8 @@ def main():
                     help="prefill this many tokens fewer than the workload's context (e.g. W/2: the overflow step then "
                          "falls in the middle of the timed steps instead of on the first decode step)")
     ap.add_argument("--kernel", default="auto", choices=sorted(KERNELS), help="decode-attention kernel (LQ_KERNEL_*)")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="create the caches without LQ_FLAG_OVERLAP_DECODE: every attention launch waits for the one before it")
     ap.add_argument("--also", default=None,
                     help="comma-separated workloads whose attention kernel is timed back to back as well and reported "
                          "under roofline_<workload> (default: gqa7-32k and llama3-8b-4k-b64 beside the default workload)")
@@ -605,9 +611,17 @@ def main():
         for name in [n for n in args.also.split(",") if n]:
             try:
                 line["roofline_" + name.replace("-", "_")] = roofline_only(name, device, args.also_layers,
-                                                                           kernel=KERNELS[args.kernel])
+                                                                           kernel=KERNELS[args.kernel],
+                                                                           flags=0 if args.no_overlap else 1)
             except Exception as exc:  # the main line stands without it
                 line["roofline_" + name.replace("-", "_")] = {"error": str(exc)}
+        if not args.no_overlap:
+            # the same kernel with every launch waiting for the one before it (LQ_FLAG_OVERLAP_DECODE off)
+            try:
+                ser = roofline_only(args.workload, device, max(8, args.also_layers), kernel=KERNELS[args.kernel], flags=0)
+                line["roofline"]["serialized"] = {k: ser[k] for k in ("us_per_launch", "achieved", "frac", "layers")}
+            except Exception as exc:
+                line["roofline"]["serialized"] = {"error": str(exc)}
         if not args.no_cpu_baseline:
             import oracle
             oracle.build()

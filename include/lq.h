@@ -73,6 +73,19 @@ typedef enum {
 #define LQ_FILTER_LOG 0
 #define LQ_FILTER_RECENT 1
 
+/* lq_config_t.flags.
+ *   LQ_FLAG_OVERLAP_DECODE  Decode-attention launches of DIFFERENT layers of this cache that follow one another
+ *     on a stream may overlap: the later launch streams its own layer's stores while the earlier one is still
+ *     merging its partials, and waits for it only before it touches the shared split-K workspace (programmatic
+ *     dependent launch with the dependency wait moved behind the main loop).  The library applies this only when
+ *     its own previous call on the cache was a decode call for another layer on the same stream; what it cannot
+ *     see is work the CALLER enqueues in between.  The flag is therefore a promise: between two lq decode calls
+ *     for different layers the caller enqueues on that stream either nothing, or only kernels that were launched
+ *     without the programmatic-stream-serialization attribute and do not trigger dependents early (plain launches,
+ *     which is what frameworks issue by default): then q, k and v are complete before the decode launch starts.
+ *     Without the flag every launch waits for its predecessor before it reads anything. */
+#define LQ_FLAG_OVERLAP_DECODE 1
+
 typedef struct {
   int32_t n_layers;      /* independent stacked layer caches, >= 1                               */
   int32_t batch;         /* B: sequences; all share one length                                   */
@@ -89,6 +102,7 @@ typedef struct {
   int32_t kernel;        /* LQ_KERNEL_*                                                          */
   int32_t n_splits;      /* split-K CTAs per (batch row, KV head); 0 = chosen by the library     */
   int32_t filter;        /* LQ_FILTER_*: which W tokens leave the full-precision store on overflow */
+  int32_t flags;         /* LQ_FLAG_* bits, 0 = none                                             */
   /* Optional device allocator (all three NULL / 0: cudaMalloc and cudaFree).  dev_alloc returns device memory of
      at least `bytes` bytes, 256-byte aligned, on `device`, or NULL on failure (the call that needed it then gives
      LQ_ERR_OOM); every block is handed back to dev_free by lq_destroy (or at once when creation fails).  Both

@@ -14,6 +14,7 @@ _LIB_PATH = os.environ.get("LOGQUANT_LIBRARY") or os.path.join(_HERE, "liblogqua
 LQ_DEVICE_NONE = -1
 LQ_KERNEL_AUTO, LQ_KERNEL_SCALAR, LQ_KERNEL_MMA, LQ_KERNEL_UMMA = 0, 1, 2, 3
 LQ_FILTER_LOG, LQ_FILTER_RECENT = 0, 1
+LQ_FLAG_OVERLAP_DECODE = 1
 LQ_OK, LQ_ERR_INVALID_ARG, LQ_ERR_UNSUPPORTED, LQ_ERR_OOM, LQ_ERR_WINDOW_FULL, LQ_ERR_NOT_FULL, \
     LQ_ERR_CAPACITY, LQ_ERR_CUDA = range(8)
 
@@ -27,7 +28,7 @@ class lq_config_t(C.Structure):
                 ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("window", C.c_int32),
                 ("group", C.c_int32), ("bits", C.c_int32), ("max_tokens", C.c_int64),
                 ("auto_compress", C.c_int32), ("device", C.c_int32), ("kernel", C.c_int32),
-                ("n_splits", C.c_int32), ("filter", C.c_int32),
+                ("n_splits", C.c_int32), ("filter", C.c_int32), ("flags", C.c_int32),
                 ("dev_alloc", ALLOC_FN), ("dev_free", FREE_FN), ("alloc_ctx", C.c_void_p)]
 
 
@@ -147,7 +148,7 @@ class LogQuantCache:
     guards_on_close = False    # True: close() checks the guard bytes behind every device block and raises if one changed
 
     def __init__(self, n_layers, batch, n_q_heads, n_kv_heads, window, group, max_tokens, head_dim=128, bits=2,
-                 auto_compress=True, device=0, kernel=LQ_KERNEL_AUTO, n_splits=0, filter=0, allocator=None):
+                 auto_compress=True, device=0, kernel=LQ_KERNEL_AUTO, n_splits=0, filter=0, allocator=None, flags=0):
         """allocator: None (cudaMalloc / cudaFree), "torch" (every device block of the cache is a uint8 tensor from
         torch's caching allocator, kept alive until the cache is closed), or a pair of callables
         (alloc(bytes) -> device address or 0, free(address))."""
@@ -176,7 +177,7 @@ class LogQuantCache:
             free_cb = FREE_FN(lambda ptr, _ctx: user_free(ptr))
         self._callbacks = (alloc_cb, free_cb)  # keep the trampolines alive as long as the cache
         self.cfg = lq_config_t(n_layers, batch, n_q_heads, n_kv_heads, head_dim, window, group, bits, max_tokens,
-                               int(auto_compress), device, kernel, n_splits, filter, alloc_cb, free_cb, None)
+                               int(auto_compress), device, kernel, n_splits, filter, flags, alloc_cb, free_cb, None)
         self._h = C.c_void_p()
         self._check(self._lib.lq_cache_create(C.byref(self.cfg), C.byref(self._h)), create=True)
 

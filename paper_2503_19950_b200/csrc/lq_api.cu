@@ -55,6 +55,14 @@ struct lq_cache {
   uint8_t* stage_out = nullptr;
   int64_t n_launches = 0;
   bool stall_next = false;  // lq_debug_stall_next_decode
+  // LQ_FLAG_OVERLAP_DECODE: layer and stream of the decode launch that was this cache's last enqueued work (-1: the
+  // last work was something else)
+  int last_decode_layer = -1;
+  cudaStream_t last_decode_stream = nullptr;
+  // layers whose full-precision store got a row from a fused append+attention launch that no later launch has
+  // waited for yet: a launch for such a layer takes the dependency wait first (which, through the chain of waits,
+  // covers every earlier launch) and clears the list
+  std::vector<char> row_in_flight;
   bool bad_slot_next = false;  // lq_debug_bad_slot_next_append (index-check build only)
   // left padding of a ragged batch (lq_set_padding): pad[b] leading positions of sequence b that attention
   // leaves out.  Device copy per layer: [B][4] row info, [B][fp_words] slot mask, [B][q_words] store mask,
@@ -281,7 +289,7 @@ lq_status_t run_events_residual(lq_cache* c, const std::vector<int>& full_layers
       if (!c->dry) {
         cudaError_t e = launch_compress(c->cv, ll, plans[i].ev, plans[i].tile0, 1, st);
         if (e != cudaSuccess) return cuda_fail(c, e, "lq_compress_kernel");
-        c->n_launches++;
+        { c->n_launches++; c->last_decode_layer = -1; }
       }
     }
   }
@@ -316,7 +324,7 @@ lq_status_t run_events(lq_cache* c, const std::vector<int>& full_layers, cudaStr
     if (!c->dry) {
       cudaError_t e = launch_compress(c->cv, ll, ev, Li.n_quant / c->cfg.group, c->cfg.window / c->cfg.group, st);
       if (e != cudaSuccess) return cuda_fail(c, e, "lq_compress_kernel");
-      c->n_launches++;
+      { c->n_launches++; c->last_decode_layer = -1; }
     }
     for (int k : members) {
       done[k] = 1;
@@ -380,6 +388,7 @@ lq_status_t upload_masks(lq_cache* c, int layer, cudaStream_t st) {
                                                 &c->pad_stride[layer]);
   }
   // pageable source: staged by the runtime before the call returns
+  c->last_decode_layer = -1;
   cudaError_t e = cudaMemcpyAsync(c->masks + layer * c->mask_layer_words, c->mask_host.data(),
                                   c->mask_host.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, st);
   if (e != cudaSuccess) return cuda_fail(c, e, "padding mask upload");
@@ -561,7 +570,7 @@ lq_status_t ingest_prompt(lq_cache* c, int layer, const void* k, const void* v, 
   if (e != cudaSuccess) return cuda_fail(c, e, "prompt index upload");
   e = launch_ingest(c->cv, layer, k, v, n, c->ingest_idx, n_tiles, L.n_fp, 0, st);
   if (e != cudaSuccess) return cuda_fail(c, e, "lq_ingest_kernel");
-  c->n_launches++;
+  { c->n_launches++; c->last_decode_layer = -1; }
   return LQ_OK;
 }
 
@@ -605,7 +614,7 @@ lq_status_t append_impl(lq_cache_t* c, int32_t layer, const void* k, const void*
       cudaError_t e = launch_append(c->cv, layer, k, v, n, done, take, slot0, st, last ? extra_src : nullptr,
                                     last ? extra_dst : nullptr, last ? extra_bytes : 0);
       if (e != cudaSuccess) return cuda_fail(c, e, "lq_append_kernel");
-      c->n_launches++;
+      { c->n_launches++; c->last_decode_layer = -1; }
     }
     for (int t = 0; t < take; ++t) {
       L.age_slot.push_back(L.n_fp + t);
@@ -771,7 +780,13 @@ lq_status_t decode_impl(lq_cache_t* c, int32_t layer, const void* q, float sm_sc
   a.tiles_fp = a.tiles_quant = 0;
   a.zero = 0;
   a.n_extra = 0;
+  a.early = 0;
   if (use_mma(c)) {
+    if (c->row_in_flight.empty()) c->row_in_flight.assign(c->cfg.n_layers, 0);
+    a.early = (c->cfg.flags & LQ_FLAG_OVERLAP_DECODE) && !timed && c->last_decode_layer >= 0 &&
+              c->last_decode_layer != layer && c->last_decode_stream == st && !c->row_in_flight[layer];
+    if (!a.early) std::fill(c->row_in_flight.begin(), c->row_in_flight.end(), 0);
+    if (new_k != nullptr) c->row_in_flight[layer] = 1;
     plan_decode_mma(a, c->sm_count, c->max_splits, c->cfg.n_splits);
     if (a.rowinfo) {
       a.S = c->pad_stride[layer];
@@ -802,6 +817,8 @@ lq_status_t decode_impl(lq_cache_t* c, int32_t layer, const void* q, float sm_sc
     c->n_launches++;
   }
   c->n_launches++;
+  c->last_decode_layer = use_mma(c) && !timed ? layer : -1;
+  c->last_decode_stream = st;
   return LQ_OK;
 }
 }  // namespace

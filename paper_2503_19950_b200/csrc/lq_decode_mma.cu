@@ -700,7 +700,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   // Programmatic dependent launch: everything above touches only this CTA's shared memory and the
   // launch arguments; nothing an earlier kernel may still be writing is read before it has finished
   // (the matching launch_dependents comes after the main loop).
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (!a.early) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (threadIdx.x == 0) {
     // the r query rows of this pair are contiguous: one bulk copy
     mbar_expect_tx(qbar, r * kD * 2);
@@ -894,6 +894,9 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   // the main loop is over: from here on the next kernel of the stream may start launching into
   // the slots that free up (earlier, its waiting CTAs would only take issue slots from this loop)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // an overlapped launch (DecodeArgs::early) has read only its own layer's stores so far; the workspace below is
+  // shared with the launch before it
+  if (a.early) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (failed) {
     // a bulk copy never completed: flag it and contribute nothing (checked again at the end)
     if (lane == 0) atomicOr(a.status, 1);

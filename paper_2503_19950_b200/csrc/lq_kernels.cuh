@@ -134,6 +134,10 @@ struct DecodeArgs {
   // test hook (lq_debug_stall_next_decode): the tensor-core kernels arm the barrier of the query copy but issue
   // no copy and poll with a short limit, so that the bounded wait runs out and the failure path is taken
   int debug_stall;
+  // tensor-core (mma.sync) kernel: 1 = the launch before this one on the stream is a decode launch of another layer
+  // of the same cache (LQ_FLAG_OVERLAP_DECODE): nothing the main loop reads is written by it, so the dependency
+  // wait of the programmatic launch moves behind the main loop, in front of the first use of the shared workspace
+  int early;
 };
 
 constexpr int kAccStride = kMaxRatio * 128 + 32;  // floats per (b, kv) pair in DecodeArgs::acc

@@ -587,3 +587,51 @@ def test_seeded_random_padded_configurations(B, Hq, Hkv, W, G, bits, n_prefill, 
     worst = run_case(B, Hq, Hkv, W, G, n_prefill, 3, seed=200 + n_prefill, kernel=kernel, bits=bits, prefill_chunk=chunk,
                      recent_only=recent, pad=pad, auto_compress=auto, check_image_every=1)
     assert worst <= 1.0
+
+
+@pytest.mark.parametrize("L,fused,r", [(4, True, 4), (4, False, 4), (2, True, 7), (3, False, 1)])
+def test_overlapped_decode_launches_of_different_layers(L, fused, r):
+    """LQ_FLAG_OVERLAP_DECODE: back-to-back decode launches of different layers start streaming before the launch
+    in front of them has finished (and wait for it only before the shared workspace); every layer's output and
+    image must still be the oracle's, step after step, also when a layer is visited twice in a row and when
+    appends and an overflow step fall between the launches."""
+    from paper_2503_19950_b200 import LQ_FLAG_OVERLAP_DECODE
+    B, Hkv, W, G, D, n0, n_steps = 2, 2, 64, 32, 128, 64 * 10 + 50, 20
+    Hq = Hkv * r
+    cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=n0 + n_steps + 8, kernel=LQ_KERNEL_MMA,
+                          flags=LQ_FLAG_OVERLAP_DECODE)
+    ocs = [oracle.OracleCache(B, Hq, Hkv, D, W, G) for _ in range(L)]
+    ks, vs = [], []
+    for l in range(L):
+        k, v = synth.keys_values(300 + l, B, Hkv, n0 + n_steps, D, "cuda", outliers=synth.outlier_channels(300 + l, Hkv, D, 3))
+        ks.append(k); vs.append(v)
+        cache.append(l, k[:, :, :n0].contiguous(), v[:, :, :n0].contiguous())
+        ocs[l].append(synth.bf16_bits(k[:, :, :n0]), synth.bf16_bits(v[:, :, :n0]))
+    outs = [torch.empty(B, Hq, D, device="cuda") for _ in range(L)]
+    twice = torch.empty(B, Hq, D, device="cuda")
+    for step in range(n_steps):   # the 14th step overflows the window of every layer
+        t = n0 + step
+        qs = [synth.queries(300 + l, B, Hq, D, step, "cuda") for l in range(L)]
+        for l in range(L):        # all launches of a step are enqueued before anything is checked
+            kt, vt = ks[l][:, :, t:t + 1].contiguous(), vs[l][:, :, t:t + 1].contiguous()
+            if fused:
+                cache.append_decode_attn(l, kt, vt, qs[l], outs[l])
+            else:
+                cache.append(l, kt, vt)
+                cache.decode_attn(l, qs[l], outs[l])
+                if l == L - 1:
+                    cache.decode_attn(l, qs[l], twice)   # the same layer twice in a row
+            ocs[l].append(synth.bf16_bits(kt), synth.bf16_bits(vt))
+        if not fused:             # attention only, layer after layer: every launch but the first overlaps
+            for l in range(L):
+                cache.decode_attn(l, qs[l], outs[l])
+        torch.cuda.synchronize()
+        for l in range(L):
+            ref = ocs[l].attention(synth.bf16_bits(qs[l]), 1 / np.sqrt(D))
+            assert np.abs(outs[l].cpu().numpy() - ref).max() <= attn_tolerance(ref), (step, l)
+        if not fused:
+            assert torch.equal(twice, outs[L - 1])
+    for l in range(L):
+        assert_images_equal(cache.export(l), ocs[l].export())
+    assert cache.kernel_status() == 0
+    cache.close()
