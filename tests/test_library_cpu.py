@@ -73,7 +73,7 @@ def test_no_gpu_means_no_compute():
 
 
 def test_allocator_hooks_come_in_pairs():
-    cfg = binding.lq_config_t(1, 1, 4, 2, 128, 128, 32, 2, 1024, 1, LQ_DEVICE_NONE, 0, 0, 0,
+    cfg = binding.lq_config_t(1, 1, 4, 2, 128, 128, 32, 2, 1024, 1, LQ_DEVICE_NONE, 0, 0, 0, 0,
                               binding.ALLOC_FN(lambda n, ctx: 0), binding.FREE_FN(0), None)
     import ctypes
     h = ctypes.c_void_p()
