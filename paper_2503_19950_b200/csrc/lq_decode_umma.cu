@@ -937,23 +937,36 @@ __global__ void __launch_bounds__(kThreads, 2) lq_decode_umma_kernel(DecodeArgs 
         if (*reinterpret_cast<volatile int*>(is_last_s)) {
           __threadfence();
           const bool healthy = (__ldcg(a.status) & 1) == 0;   // after a wait that gave up the output stays untouched
+          // (m, l) of every record of the pair into shared memory with one round of loads (B of p.v is free: the
+          // p.v MMAs of this item are complete and nobody writes the next item's before the rendezvous below)
+          float2* sml = reinterpret_cast<float2*>(smem + GE::OFF_BPV);
+          const int R = a.S * r;
+          for (int i = wt; i < R; i += kGroup) {
+            const int sl = i / r;
+            sml[i] = contrib[sl] ? __ldcg(reinterpret_cast<const float2*>(a.part_ml) + (pair * a.S + sl) * r + (i - sl * r))
+                                 : make_float2(-INFINITY, 0.f);
+          }
+          named_sync<kBarW, kGroup>();
           for (int h = 0; h < r && healthy; ++h) {
             float M = -INFINITY;
             for (int sl = 0; sl < a.S; ++sl) {
-              if (!contrib[sl]) continue;
-              const int64_t rr = (pair * a.S + sl) * r + h;
-              if (__ldcg(a.part_ml + rr * 2 + 1) > 0.f) M = fmaxf(M, __ldcg(a.part_ml + rr * 2));
+              const float2 ml = sml[sl * r + h];
+              if (ml.y > 0.f) M = fmaxf(M, ml.x);
             }
             float L = 0.f, acc = 0.f;
-            for (int sl = 0; sl < a.S; ++sl) {
-              if (!contrib[sl]) continue;
-              const int64_t rr = (pair * a.S + sl) * r + h;
-              const float ls = __ldcg(a.part_ml + rr * 2 + 1);
-              if (ls > 0.f) {
-                const float wgt = ex2(__ldcg(a.part_ml + rr * 2) - M);
-                L = fmaf(ls, wgt, L);
-                acc = fmaf(__ldcg(a.part_o + rr * kD + d), wgt, acc);
+            for (int sl0 = 0; sl0 < a.S; sl0 += 8) {
+              float v[8], wgt[8];
+#pragma unroll
+              for (int u = 0; u < 8; ++u) {   // eight independent loads in flight
+                const int sl = sl0 + u;
+                const float2 ml = sl < a.S ? sml[sl * r + h] : make_float2(-INFINITY, 0.f);
+                const bool on = ml.y > 0.f;
+                wgt[u] = on ? ex2(ml.x - M) : 0.f;
+                v[u] = on ? __ldcg(a.part_o + ((pair * a.S + sl) * r + h) * kD + d) : 0.f;
+                L = fmaf(ml.y, wgt[u], L);
               }
+#pragma unroll
+              for (int u = 0; u < 8; ++u) acc = fmaf(v[u], wgt[u], acc);
             }
             const int b = static_cast<int>(pair / cv.Hkv), kv = static_cast<int>(pair % cv.Hkv);
             const int64_t oi = (static_cast<int64_t>(b) * cv.Hq + kv * r + h) * kD + d;
