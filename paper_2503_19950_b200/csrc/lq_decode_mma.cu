@@ -701,6 +701,10 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   // launch arguments; nothing an earlier kernel may still be writing is read before it has finished
   // (the matching launch_dependents comes after the main loop).
   if (!a.early) asm volatile("griddepcontrol.wait;" ::: "memory");
+  // In a chain of overlapped launches the next launch may take the slots of this one as soon as they free up (its
+  // CTAs stream their own layer and wait for this grid only before the workspace); otherwise the trigger comes
+  // after the main loop, so that CTAs that could only wait do not take the slots earlier.
+  if (a.early) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (threadIdx.x == 0) {
     // the r query rows of this pair are contiguous: one bulk copy
     mbar_expect_tx(qbar, r * kD * 2);
@@ -893,7 +897,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   }
   // the main loop is over: from here on the next kernel of the stream may start launching into
   // the slots that free up (earlier, its waiting CTAs would only take issue slots from this loop)
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (!a.early) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // an overlapped launch (DecodeArgs::early) has read only its own layer's stores so far; the workspace below is
   // shared with the launch before it
   if (a.early) asm volatile("griddepcontrol.wait;" ::: "memory");
