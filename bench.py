@@ -393,15 +393,17 @@ def roofline_only(name, device, layers, rounds=24, n_splits=0, kernel=0, flags=1
     for l in range(L):  # first decode step: the overflow step runs here, the timed launches see the state after it
         cache.append_decode_attn(l, ks[l][0], vs[l][0], qs[l][0], outs[l])
     evs = []
+    passes = max(1, 32 // L)  # launches between two event records: as many as the main workload's 32 layers
     for rep in range(rounds + 3):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        for l in range(L):
-            cache.decode_attn(l, qs[l][rep % 4], outs[l])
+        for p in range(passes):
+            for l in range(L):
+                cache.decode_attn(l, qs[l][(rep + p) % 4], outs[l])
         e1.record()
         evs.append((e0, e1))
     torch.cuda.synchronize()
-    us = sorted(e0.elapsed_time(e1) * 1e3 for e0, e1 in evs[3:])
+    us = sorted(e0.elapsed_time(e1) * 1e3 / passes for e0, e1 in evs[3:])
     b2b_us = us[len(us) // 2] / L
     inf = cache.info(0)
     nbytes = int(inf.bytes_decode_step)
@@ -414,7 +416,8 @@ def roofline_only(name, device, layers, rounds=24, n_splits=0, kernel=0, flags=1
             "kv_tokens_per_s": B * (int(inf.n_quant) + int(inf.n_fp)) / (b2b_us * 1e-6),
             "n_quant": int(inf.n_quant), "n_fp": int(inf.n_fp), "n_ctas": int(inf.n_ctas), "finite_and_status_ok": ok,
             "frac_of_8tbs_nominal": nbytes / (b2b_us * 1e-6) / 1e9 / 8000.0,
-            "timing": "median over %d rounds of %d back-to-back launches, one per layer cache" % (len(us), L)}
+            "timing": "median over %d rounds of %d back-to-back launches (%d passes over %d layer caches)" % (
+                len(us), passes * L, passes, L)}
 
 
 def parity_against_oracle(cache, wl, device, replay):
@@ -555,7 +558,7 @@ def main():
     ap.add_argument("--also", default=None,
                     help="comma-separated workloads whose attention kernel is timed back to back as well and reported "
                          "under roofline_<workload> (default: gqa7-32k and llama3-8b-4k-b64 beside the default workload)")
-    ap.add_argument("--also-layers", type=int, default=4, help="layer caches of the --also workloads")
+    ap.add_argument("--also-layers", type=int, default=8, help="layer caches of the --also workloads")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.also is None:
