@@ -765,7 +765,12 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   bool failed = false;
   // Only one small load per warp before the query fragments are built: all warps start at the same
   // time, and the first bytes every warp needs should not queue behind everybody's second load.
-  issue_next(1);
+  // (an overlapped launch starts while other CTAs of the SM are in mid-stream: it fills all its stages at once)
+  if (a.early) {
+    for (int s = 0; s < kStages; ++s) issue_next(TPS);
+  } else {
+    issue_next(1);
+  }
 
   // query fragments: B operand, column n -> head 4cb + n/2 (even column = hi, odd = lo of q*s);
   // k-step ks carries the factor 2^(64 - 2*(ks&3)) that cancels the code-position factor
@@ -813,7 +818,8 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
         }
     }
   }
-  for (int s = 1; s < kStages; ++s) issue_next(TPS);
+  if (!a.early)
+    for (int s = 1; s < kStages; ++s) issue_next(TPS);
   WarpState<NCB> st;
 #pragma unroll
   for (int mt = 0; mt < 8; ++mt) st.out[mt][0] = st.out[mt][1] = st.out[mt][2] = st.out[mt][3] = 0.f;
