@@ -629,8 +629,9 @@ def test_overlapped_decode_launches_of_different_layers(L, fused, r):
         for l in range(L):
             ref = ocs[l].attention(synth.bf16_bits(qs[l]), 1 / np.sqrt(D))
             assert np.abs(outs[l].cpu().numpy() - ref).max() <= attn_tolerance(ref), (step, l)
-        if not fused:
-            assert torch.equal(twice, outs[L - 1])
+        if not fused:   # (a launch that overlaps shares its pair's work out differently: equal up to summation order)
+            ref = ocs[L - 1].attention(synth.bf16_bits(qs[L - 1]), 1 / np.sqrt(D))
+            assert np.abs(twice.cpu().numpy() - ref).max() <= attn_tolerance(ref), step
     for l in range(L):
         assert_images_equal(cache.export(l), ocs[l].export())
     assert cache.kernel_status() == 0
