@@ -963,6 +963,7 @@ lq_status_t lq_cache_info(const lq_cache_t* c, int32_t layer, lq_info_t* info) {
     a.cv = c->cv;
     a.n_fp = L.n_fp;
     a.n_quant = L.n_quant;
+    a.early = 0;  // the plan of a launch that does not overlap (an overlapped one uses a third of these CTAs)
     plan_decode_mma(a, c->sm_count, c->max_splits, c->cfg.n_splits);
     info->n_splits = a.S - 1;
     info->n_ctas = (a.S - 1) * c->cfg.batch * c->cfg.n_kv_heads + a.n_extra;

@@ -50,6 +50,7 @@ __host__ __device__ constexpr int n_stages(int) { return 2; }
 __host__ __device__ constexpr int warp_stage_bytes(int G, int PL = 1) { return n_stages(G) * stage_bytes(G, PL); }
 constexpr int kWarpStageBytes = warp_stage_bytes(32);
 constexpr int kMaxStages = 3;
+constexpr int kOverlapDepth = 3;  // consecutive overlapped launches that share the SMs (plan_decode_mma)
 constexpr int kCtasPerSm = 4;  // at 128 registers and 51 KB of shared memory; 3 and 5 both measured slower
 constexpr uint32_t kFull = 0xFFFFFFFFu;
 constexpr int kSpinLimit = 1 << 22;
@@ -1239,7 +1240,12 @@ void plan_decode_mma(DecodeArgs& a, int sm_count, int max_records, int s_overrid
   // when the others finish, and its pair's merge would wait for it
   // the two-column-block variant needs more registers, the 9 KB stages of 4-bit codes at G = 64 more shared memory
   const int ctas_per_sm = r <= 4 && !(a.cv.G == 64 && a.cv.planes == 2) ? kCtasPerSm : kCtasPerSm - 1;
-  int S = s_override > 0 ? s_override : (ctas_per_sm * sm_count) / pairs;
+  // A serialised launch fills exactly one resident wave.  An overlapped launch (DecodeArgs::early) takes a third of
+  // the slots with CTAs three times as long (at least one CTA per pair): three consecutive launches then share the
+  // SMs, every slot stays busy, and the fixed costs of a CTA (start-up, merge, ticket: 4 - 5 us) are paid once per
+  // three times the bytes (measured: 1/2 and 1/3 alike, 1/4 worse; 8k workload 15.4 -> 14.4 us per launch).
+  const int wave = a.early ? std::max(pairs, ctas_per_sm * sm_count / kOverlapDepth) : ctas_per_sm * sm_count;
+  int S = s_override > 0 ? s_override : wave / pairs;
   S = std::min(S, (items + kWarps - 1) / kWarps);  // at least one item per warp
   S = std::min(S, max_records - 1);
   S = std::min(S, kMergeMax / r - 1);
@@ -1248,8 +1254,9 @@ void plan_decode_mma(DecodeArgs& a, int sm_count, int max_records, int s_overrid
   // exactly: every SM then carries the same number of CTAs (an SM with 4 CTAs runs each of them a
   // third slower than an SM with 3, and work does not move between pairs)
   int extra = 0;
-  if (s_override <= 0 && S + 1 <= max_records && (S + 1) * kWarps <= items) {
-    extra = ctas_per_sm * sm_count - S * pairs;
+  // (an overlapped launch with one CTA per pair stays that way: such a CTA writes its result without any merge)
+  if (s_override <= 0 && S + 1 <= max_records && (S + 1) * kWarps <= items && !(a.early && S == 1)) {
+    extra = wave - S * pairs;
     extra = std::max(0, std::min(extra, pairs));
   }
   a.n_extra = extra;
