@@ -675,16 +675,16 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   int it, it_end;
   {
     const int F8 = a.tiles_fp * kFpCost8, C8 = F8 + (a.tiles_quant - qskip) * 8;
-    // Overlapped launches (DecodeArgs::early): the CTAs of a launch take over the slots of the launch before it
-    // in launch order, and the last slots to free up are those of its merging CTAs -- one per pair, and the last
-    // CTA of every pair is launched last.  That CTA therefore starts a merge later than the others; with a full
-    // share it would finish last, merge last and hand its slot on late again.  It gets half a share (measured:
-    // 3/8 to 5/8 alike, +4 to +7 % on every workload; a serialised launch keeps equal shares).
+    // Overlapped launches (DecodeArgs::early): the CTAs of a launch take over the slots of earlier launches in
+    // launch order, and the last slots to free up are those of merging CTAs -- one per pair, and the last CTA of
+    // every pair is launched last.  That CTA starts later than the others; it gets 3/4 of a share (measured with a
+    // third of a wave per launch: 3/4 and 1 alike on the 8k workload, 3/4 better by 2 % on GQA-7, 1/2 and 1/4 worse;
+    // a serialised launch keeps equal shares).
     const int64_t full_warps = static_cast<int64_t>(n_warps) - (a.early && n_ctas_pair > 1 ? kWarps : 0);
-    const int64_t total_w2 = 2 * full_warps + (n_warps - full_warps);
+    const int64_t total_w4 = 4 * full_warps + 3 * (n_warps - full_warps);
     auto cut = [&](int k) {
-      const int64_t cw2 = k <= full_warps ? 2LL * k : 2 * full_warps + (k - full_warps);
-      const int pos8 = static_cast<int>(cw2 * C8 / total_w2);
+      const int64_t cw4 = k <= full_warps ? 4LL * k : 4 * full_warps + 3 * (k - full_warps);
+      const int pos8 = static_cast<int>(cw4 * C8 / total_w4);
       return pos8 < F8 ? (pos8 + kFpCost8 / 2) / kFpCost8 : a.tiles_fp + (pos8 - F8 + 4) / 8;
     };
     it = cut(gw);
