@@ -706,9 +706,10 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
-  // Programmatic dependent launch: everything above touches only this CTA's shared memory and the
-  // launch arguments; nothing an earlier kernel may still be writing is read before it has finished
-  // (the matching launch_dependents comes after the main loop).
+  // Programmatic dependent launch: everything above touches only this CTA's shared memory, the launch
+  // arguments and, in the padded variant, the CTA map and row info of the mask block -- which only a host copy
+  // enqueued by the same call writes (upload_masks), never a kernel that could still be running.  Nothing an
+  // earlier kernel may still be writing is read before it has finished.
   if (!a.early) asm volatile("griddepcontrol.wait;" ::: "memory");
   // In a chain of overlapped launches the next launch may take the slots of this one as soon as they free up (its
   // CTAs stream their own layer and wait for this grid only before the workspace); otherwise the trigger comes
