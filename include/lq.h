@@ -233,8 +233,9 @@ lq_status_t lq_append_decode_attn(lq_cache_t* cache, int32_t layer, const void* 
  * so steps of different layers may be enqueued back to back.  When k_host, v_host and out_host are
  * page-locked, device-addressable (cudaHostAlloc / cudaHostRegister, as reported by
  * cudaPointerGetAttributes) and 16-byte aligned -- all four buffers --, the kernels read the inputs
- * from and write the result to host memory directly (the append launch also stages the query in
- * device memory); otherwise every buffer is copied through device staging memory. */
+ * from and write the result to host memory directly, in the single launch of lq_append_decode_attn (every CTA
+ * fetches the query rows of its pair from host memory, about 1 KB; consecutive layers overlap under
+ * LQ_FLAG_OVERLAP_DECODE); otherwise every buffer is copied through device staging memory. */
 lq_status_t lq_decode_step_host(lq_cache_t* cache, int32_t layer, const void* k_host,
                                 const void* v_host, const void* q_host, float sm_scale,
                                 float* out_host, int32_t sync, void* stream);

@@ -838,11 +838,11 @@ lq_status_t lq_decode_step_host(lq_cache_t* c, int32_t layer, const void* k_host
   uint8_t* sq = c->stage_q + layer * qb;
   uint8_t* so = c->stage_out + layer * qb * 2;
   cudaError_t e;
-  // Page-locked host buffers that the device can address are used in place: the append kernel reads
-  // the new k and v rows straight from host memory and the attention kernel writes its result
-  // straight into out_host; the query, which every CTA of a pair reads, is moved to device memory
-  // by the append launch.  No separate copy is left.  Anything else goes through the staging
-  // buffers with one copy each.
+  // Page-locked host buffers that the device can address are used in place, by the same single launch as the
+  // device-buffer step (lq_append_decode_attn): the attention kernel takes the new k and v rows and the query
+  // rows straight from host memory (the query once per CTA: about 1 KB each) and writes its result straight into
+  // out_host; consecutive layers overlap like device-resident steps.  No separate copy is left.  Anything else
+  // goes through the staging buffers with one copy each.
   auto mapped = [](const void* p) -> void* {
     cudaPointerAttributes at;
     if ((reinterpret_cast<uintptr_t>(p) & 15) != 0) return nullptr;
@@ -861,16 +861,20 @@ lq_status_t lq_decode_step_host(lq_cache_t* c, int32_t layer, const void* k_host
     if ((e = cudaMemcpyAsync(sq, q_host, qb, cudaMemcpyHostToDevice, st)) != cudaSuccess)
       return cuda_fail(c, e, "host-to-device copy");
   }
-  if (kept(L) == 3 * c->cfg.window) {
-    lq_status_t s = run_events(c, std::vector<int>{layer}, st);
+  lq_status_t s;
+  if (kept(L) == 3 * c->cfg.window) {  // the overflow step of this layer is due
+    s = run_events(c, std::vector<int>{layer}, st);
     if (s != LQ_OK) return s;
   }
-  // in place: the append launch also moves the query into device memory (every CTA of a pair reads it)
-  lq_status_t s = direct ? append_impl(c, layer, dk, dv, 1, stream, dq, sq, static_cast<int>(qb))
-                         : lq_append(c, layer, sk, sv, 1, stream);
-  if (s != LQ_OK) return s;
-  s = lq_decode_attn(c, layer, sq, sm_scale, direct ? dout : so, 0, stream);
-  if (s != LQ_OK) return s;
+  if (direct) {
+    s = lq_append_decode_attn(c, layer, dk, dv, dq, sm_scale, dout, 0, stream);
+    if (s != LQ_OK) return s;
+  } else {
+    s = lq_append(c, layer, sk, sv, 1, stream);
+    if (s != LQ_OK) return s;
+    s = lq_decode_attn(c, layer, sq, sm_scale, so, 0, stream);
+    if (s != LQ_OK) return s;
+  }
   if (!direct && (e = cudaMemcpyAsync(out_host, so, qb * 2, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
     return cuda_fail(c, e, "device-to-host copy");
   if (sync && (e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(c, e, "cudaStreamSynchronize");
