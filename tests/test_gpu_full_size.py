@@ -193,3 +193,66 @@ def test_config4_timed_entry_points_across_an_overflow(entry):
     events = _run_timed_entry(entry, B=4, Hq=28, Hkv=4, W=256, G=64, ctx=32768 - 128, seed=4,
                               check_steps=[1, 2, 64, 128, 129, 130], n_outliers=0, planted=True)
     assert events == 1
+
+
+# ---- overlapped launches (LQ_FLAG_OVERLAP_DECODE), the configuration bench.py times ------------------
+@pytest.mark.parametrize("entry", ["fused", "host_pinned"])
+@pytest.mark.parametrize("cfg", [dict(B=8, Hq=32, Hkv=8, W=128, G=32, ctx=8192 - 3, seed=2, n_outliers=3),
+                                 dict(B=4, Hq=28, Hkv=4, W=256, G=64, ctx=32768 - 3, seed=4, n_outliers=0)])
+def test_overlapped_launches_of_stacked_layers_at_full_size(entry, cfg):
+    """Three layer caches with different contents, six decode steps enqueued layer after layer without any
+    synchronisation in between (the fourth step overflows every window): every launch but the first of a chain
+    overlaps the one before it, with a third of a wave per launch.  Every layer's output of every step and the
+    final images must be the oracle's."""
+    from paper_2503_19950_b200 import LQ_FLAG_OVERLAP_DECODE
+    B, Hq, Hkv, W, G, ctx, seed = (cfg[k] for k in ("B", "Hq", "Hkv", "W", "G", "ctx", "seed"))
+    L, n_steps, dev = 3, 6, "cuda"
+    total = ctx + n_steps
+    cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=total + 8, flags=LQ_FLAG_OVERLAP_DECODE)
+    ocs = [oracle.OracleCache(B, Hq, Hkv, D, W, G) for _ in range(L)]
+    outl = [synth.outlier_channels(seed + 10 * l, Hkv, D, cfg["n_outliers"]) if cfg["n_outliers"] else None for l in range(L)]
+    for l in range(L):
+        for t0 in range(0, ctx, 4096):
+            n = min(4096, ctx - t0)
+            k, v = synth.keys_values(seed + 10 * l, B, Hkv, n, D, dev, token_start=t0, token_total=total, outliers=outl[l])
+            cache.append(l, k, v)
+            ocs[l].append(synth.bf16_bits(k), synth.bf16_bits(v))
+    pin = lambda t: t.cpu().pin_memory()
+    outs = [[(torch.full((B, Hq, D), float("nan")).pin_memory() if entry == "host_pinned"
+              else torch.full((B, Hq, D), float("nan"), device=dev)) for _ in range(L)] for _ in range(n_steps)]
+    qs, keep = [], []
+    for step in range(n_steps):          # everything is enqueued first ...
+        qs.append([])
+        for l in range(L):
+            k, v = synth.keys_values(seed + 10 * l, B, Hkv, 1, D, dev, token_start=ctx + step, token_total=total,
+                                     outliers=outl[l])
+            q = synth.queries(seed + 10 * l, B, Hq, D, step, dev)
+            qs[step].append(q)
+            if entry == "host_pinned":
+                hk, hv, hq = pin(k), pin(v), pin(q)
+                keep.append((hk, hv, hq))
+                cache.decode_step_host(l, hk, hv, hq, outs[step][l], sync=False)
+            else:
+                cache.append_decode_attn(l, k, v, q, outs[step][l])
+            ocs[l].append(synth.bf16_bits(k), synth.bf16_bits(v))
+    torch.cuda.synchronize()             # ... and checked afterwards, against oracles replayed step by step
+    assert cache.kernel_status() == 0
+    replay = [oracle.OracleCache(B, Hq, Hkv, D, W, G) for _ in range(L)]
+    for l in range(L):
+        for t0 in range(0, ctx, 4096):
+            n = min(4096, ctx - t0)
+            k, v = synth.keys_values(seed + 10 * l, B, Hkv, n, D, dev, token_start=t0, token_total=total, outliers=outl[l])
+            replay[l].append(synth.bf16_bits(k), synth.bf16_bits(v))
+    for step in range(n_steps):
+        for l in range(L):
+            k, v = synth.keys_values(seed + 10 * l, B, Hkv, 1, D, dev, token_start=ctx + step, token_total=total,
+                                     outliers=outl[l])
+            replay[l].append(synth.bf16_bits(k), synth.bf16_bits(v))
+            ref = replay[l].attention(synth.bf16_bits(qs[step][l]), 1 / np.sqrt(D), n_threads=16)
+            got = outs[step][l].cpu().numpy().astype(np.float64)
+            err, tol = float(np.abs(got - ref).max()), attn_tolerance(ref)
+            assert np.isfinite(got).all() and err <= tol, f"step {step} layer {l}: max|delta| {err:.3e} > {tol:.3e}"
+    for l in range(L):
+        assert replay[l].n_events == ocs[l].n_events and ocs[l].n_events >= 1
+        assert_images_equal(cache.export(l), ocs[l].export())
+    cache.close()
