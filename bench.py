@@ -336,6 +336,7 @@ def run_ours(args, wl, rank, world, device):
                    "merge": ("partials summed on arrival with global atomics (more than 12 CTAs per (b, kv) pair; not "
                              "bit-reproducible), records as fallback" if int(inf.n_splits) >= 12 else
                              "ordered merge of the CTA records by the last CTA of a pair (bit-reproducible)"),
+                   "n_ctas_overlapped": int(getattr(inf, "n_ctas_overlapped", 0)),
                    "launch_overlap": ("every launch waits for the one before it" if args.no_overlap else
                                       "LQ_FLAG_OVERLAP_DECODE: attention launches of consecutive layers overlap (a launch streams its "
                                       "own layer's stores while the previous one merges, and waits for it before the shared "

@@ -126,6 +126,9 @@ typedef struct {
                                   lq_decode_attn would use                                        */
   int32_t n_ctas;              /* CTAs of its attention kernel (tensor-core kernel; else 0)      */
   int64_t n_kernel_launches;   /* kernels this cache has launched so far (all layers)            */
+  int32_t n_ctas_overlapped;   /* CTAs of an attention launch that overlaps the launch before it
+                                  (LQ_FLAG_OVERLAP_DECODE: a third of the resident wave; else 0)  */
+  int32_t reserved;
 } lq_info_t;
 
 /*

@@ -971,6 +971,11 @@ lq_status_t lq_cache_info(const lq_cache_t* c, int32_t layer, lq_info_t* info) {
     plan_decode_mma(a, c->sm_count, c->max_splits, c->cfg.n_splits);
     info->n_splits = a.S - 1;
     info->n_ctas = (a.S - 1) * c->cfg.batch * c->cfg.n_kv_heads + a.n_extra;
+    if ((c->cfg.flags & LQ_FLAG_OVERLAP_DECODE) && !c->has_pad) {
+      a.early = 1;
+      plan_decode_mma(a, c->sm_count, c->max_splits, c->cfg.n_splits);
+      info->n_ctas_overlapped = (a.S - 1) * c->cfg.batch * c->cfg.n_kv_heads + a.n_extra;
+    }
   } else if (use_umma(c)) {
     DecodeArgs a;
     a.cv = c->cv;
