@@ -75,6 +75,7 @@ struct lq_cache {
   int64_t mask_layer_words = 0;
   std::vector<uint32_t> mask_host;
   std::vector<int> pad_grid, pad_stride;  // per layer: CTAs and record stride of the padded tensor-core launch
+  std::vector<int> pad_grid_ov, pad_stride_ov;  // the same for a launch that overlaps the one before it
   // optional timing of the split-K attention kernel
   bool profiling = false;
   std::vector<cudaEvent_t> ev_pool;  // 2 events per timed launch
@@ -386,6 +387,10 @@ lq_status_t upload_masks(lq_cache* c, int layer, cudaStream_t st) {
     a.n_quant = L.n_quant;
     c->pad_grid[layer] = plan_decode_mma_padded(a, c->sm_count, c->max_splits, rowinfo, cta_map, pair_ctas,
                                                 &c->pad_stride[layer]);
+    // second plan, behind the first: a third of the wave for launches that overlap (LQ_FLAG_OVERLAP_DECODE)
+    int32_t* pair_ctas_ov = cta_map + c->map_words;
+    c->pad_grid_ov[layer] = plan_decode_mma_padded(a, c->sm_count, c->max_splits, rowinfo, pair_ctas_ov + B * c->cfg.n_kv_heads,
+                                                   pair_ctas_ov, &c->pad_stride_ov[layer], true);
   }
   // pageable source: staged by the runtime before the call returns
   c->last_decode_layer = -1;
@@ -673,7 +678,7 @@ lq_status_t lq_set_padding(lq_cache_t* c, const int32_t* pad_host) {
     c->fp_words = (slots + 31) / 32;
     c->q_words = static_cast<int>((c->cfg.max_tokens + 31) / 32);
     c->map_words = std::max(max_ctas_decode_mma(c->sm_count), B * c->cfg.n_kv_heads);  // at least one CTA per pair
-    c->mask_layer_words = static_cast<int64_t>(B) * (4 + c->fp_words + c->q_words) + B * c->cfg.n_kv_heads + c->map_words;
+    c->mask_layer_words = static_cast<int64_t>(B) * (4 + c->fp_words + c->q_words) + 2 * (B * c->cfg.n_kv_heads + c->map_words);
     if (!dev_alloc(c, reinterpret_cast<void**>(&c->masks), c->mask_layer_words * c->cfg.n_layers * 4)) return LQ_ERR_OOM;
   }
   c->pad.assign(pad_host, pad_host + B);
@@ -682,6 +687,8 @@ lq_status_t lq_set_padding(lq_cache_t* c, const int32_t* pad_host) {
   c->mask_dirty.assign(c->cfg.n_layers, 1);
   c->pad_grid.assign(c->cfg.n_layers, 0);
   c->pad_stride.assign(c->cfg.n_layers, 1);
+  c->pad_grid_ov.assign(c->cfg.n_layers, 0);
+  c->pad_stride_ov.assign(c->cfg.n_layers, 1);
   return LQ_OK;
 }
 
@@ -789,8 +796,12 @@ lq_status_t decode_impl(lq_cache_t* c, int32_t layer, const void* q, float sm_sc
     if (new_k != nullptr) c->row_in_flight[layer] = 1;
     plan_decode_mma(a, c->sm_count, c->max_splits, c->cfg.n_splits);
     if (a.rowinfo) {
-      a.S = c->pad_stride[layer];
-      a.n_ctas = c->pad_grid[layer];
+      a.S = a.early ? c->pad_stride_ov[layer] : c->pad_stride[layer];
+      a.n_ctas = a.early ? c->pad_grid_ov[layer] : c->pad_grid[layer];
+      if (a.early) {  // the second plan lies behind the first in the mask block
+        a.pair_ctas = a.cta_map + c->map_words;
+        a.cta_map = a.pair_ctas + c->cfg.batch * c->cfg.n_kv_heads;
+      }
       a.n_extra = 0;
     }
     a.tickets = c->tickets;  // the CTA that completes a (b, kv) pair merges it: no second launch

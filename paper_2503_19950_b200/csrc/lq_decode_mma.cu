@@ -1267,13 +1267,14 @@ void plan_decode_mma(DecodeArgs& a, int sm_count, int max_records, int s_overrid
 int max_ctas_decode_mma(int sm_count) { return kCtasPerSm * sm_count; }
 
 int plan_decode_mma_padded(const DecodeArgs& a, int sm_count, int max_records, const int32_t* rowinfo_host,
-                           int32_t* cta_map, int32_t* pair_ctas, int* stride) {
+                           int32_t* cta_map, int32_t* pair_ctas, int* stride, bool overlapped) {
   const int pairs = a.cv.B * a.cv.Hkv;
   const int r = a.cv.Hq / a.cv.Hkv;
   const int tiles_fp = (a.n_fp + kFpTileSlots - 1) / kFpTileSlots;
   const int tiles_quant = static_cast<int>(a.n_quant / a.cv.G);
   const int tps = stage_bytes(a.cv.G, a.cv.planes) / quant_tile_bytes(a.cv.G, a.cv.planes);
-  const int wave = (r <= 4 && !(a.cv.G == 64 && a.cv.planes == 2) ? kCtasPerSm : kCtasPerSm - 1) * sm_count;
+  const int slots = (r <= 4 && !(a.cv.G == 64 && a.cv.planes == 2) ? kCtasPerSm : kCtasPerSm - 1) * sm_count;
+  const int wave = overlapped ? std::max(pairs, slots / kOverlapDepth) : slots;  // as in plan_decode_mma
   const int cap_records = std::max(1, std::min(max_records, kMergeMax / r));
   std::vector<int64_t> work(pairs);
   std::vector<int> cap(pairs);

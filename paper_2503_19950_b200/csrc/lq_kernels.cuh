@@ -150,8 +150,9 @@ void plan_decode_mma(DecodeArgs& a, int sm_count, int max_records, int s_overrid
 // max_ctas_decode_mma(sm_count) entries) and pair_ctas (B * Hkv entries); returns the grid size and sets
 // *stride to the record stride (the largest CTA count of a pair, <= max_records).
 int max_ctas_decode_mma(int sm_count);
+// overlapped: the plan of a launch that overlaps the one before it (a third of the wave, DecodeArgs::early).
 int plan_decode_mma_padded(const DecodeArgs& a, int sm_count, int max_records, const int32_t* rowinfo_host,
-                           int32_t* cta_map, int32_t* pair_ctas, int* stride);
+                           int32_t* cta_map, int32_t* pair_ctas, int* stride, bool overlapped = false);
 cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st);
 // tcgen05 kernel: fills tiles_fp (fp units), tiles_quant, the u_* fields, n_ctas and S (<= max_records, <= 128)
 void plan_decode_umma(DecodeArgs& a, int sm_count, int max_records, int s_override);

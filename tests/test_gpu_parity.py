@@ -589,8 +589,15 @@ def test_seeded_random_padded_configurations(B, Hq, Hkv, W, G, bits, n_prefill, 
     assert worst <= 1.0
 
 
-@pytest.mark.parametrize("L,fused,r", [(4, True, 4), (4, False, 4), (2, True, 7), (3, False, 1)])
-def test_overlapped_decode_launches_of_different_layers(L, fused, r):
+def _overlap_ref(oc, q, D, pad):
+    if pad is None:
+        return oc.attention(synth.bf16_bits(q), 1 / np.sqrt(D))
+    return oc.attention_subset(synth.bf16_bits(q), 1 / np.sqrt(D), pad=pad)
+
+
+@pytest.mark.parametrize("L,fused,r,pad", [(4, True, 4, None), (4, False, 4, None), (2, True, 7, None), (3, False, 1, None),
+                                           (4, True, 4, [0, 333]), (3, False, 7, [650, 17])])
+def test_overlapped_decode_launches_of_different_layers(L, fused, r, pad):
     """LQ_FLAG_OVERLAP_DECODE: back-to-back decode launches of different layers start streaming before the launch
     in front of them has finished (and wait for it only before the shared workspace); every layer's output and
     image must still be the oracle's, step after step, also when a layer is visited twice in a row and when
@@ -600,6 +607,8 @@ def test_overlapped_decode_launches_of_different_layers(L, fused, r):
     Hq = Hkv * r
     cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=n0 + n_steps + 8, kernel=LQ_KERNEL_MMA,
                           flags=LQ_FLAG_OVERLAP_DECODE)
+    if pad is not None:   # a left-padded batch: the padded kernel variant and its own third-of-a-wave plan
+        cache.set_padding(pad)
     ocs = [oracle.OracleCache(B, Hq, Hkv, D, W, G) for _ in range(L)]
     ks, vs = [], []
     for l in range(L):
@@ -627,10 +636,10 @@ def test_overlapped_decode_launches_of_different_layers(L, fused, r):
                 cache.decode_attn(l, qs[l], outs[l])
         torch.cuda.synchronize()
         for l in range(L):
-            ref = ocs[l].attention(synth.bf16_bits(qs[l]), 1 / np.sqrt(D))
+            ref = _overlap_ref(ocs[l], qs[l], D, pad)
             assert np.abs(outs[l].cpu().numpy() - ref).max() <= attn_tolerance(ref), (step, l)
         if not fused:   # (a launch that overlaps shares its pair's work out differently: equal up to summation order)
-            ref = ocs[L - 1].attention(synth.bf16_bits(qs[L - 1]), 1 / np.sqrt(D))
+            ref = _overlap_ref(ocs[L - 1], qs[L - 1], D, pad)
             assert np.abs(twice.cpu().numpy() - ref).max() <= attn_tolerance(ref), step
     for l in range(L):
         assert_images_equal(cache.export(l), ocs[l].export())
