@@ -204,3 +204,27 @@ def test_info_byte_accounting():
     inf = c4.info(0)
     assert (inf.n_quant, inf.n_fp, inf.bytes_quant_per_token) == (7936, 257, 160)
     assert inf.bytes_decode_step == 64 * (7936 * 160 + 257 * 512)
+
+
+def test_new_entry_points_without_a_device():
+    """Bookkeeping-only caches: guard check and status reset succeed trivially, the test hooks and lq_import refuse
+    or do nothing; null handles are argument errors."""
+    import numpy as np
+    c = _dry(W=128, G=32)
+    assert c.check_guards() == 0
+    c.reset_kernel_status()
+    c.debug_stall_next_decode()
+    with pytest.raises(LogQuantError) as e:
+        c.debug_bad_slot_next_append()   # only the index-check build of the library takes this hook
+    assert e.value.status == binding.LQ_ERR_UNSUPPORTED
+    img = dict(kept_ids=np.zeros(4, np.int32), quant_ids=np.zeros(0, np.int32))
+    with pytest.raises(LogQuantError) as e:
+        c.import_image(0, img, 4)
+    assert e.value.status == binding.LQ_ERR_UNSUPPORTED
+    lib = c._lib
+    n = binding.C.c_int32(0)
+    assert lib.lq_check_guards(None, binding.C.byref(n)) == binding.LQ_ERR_INVALID_ARG
+    assert lib.lq_reset_kernel_status(None) == binding.LQ_ERR_INVALID_ARG
+    assert lib.lq_debug_stall_next_decode(None) == binding.LQ_ERR_INVALID_ARG
+    assert lib.lq_import(None, 0, None, 1, 0, 0) == binding.LQ_ERR_INVALID_ARG
+    assert c.info(0).n_ctas_overlapped == 0
