@@ -11,7 +11,7 @@ LIB = os.path.join(_HERE, "liblogquant.so")
 LIB_BOUNDS = os.path.join(_HERE, "liblogquant_bounds.so")  # the same library with the index checks compiled in
 SOURCES = ["lq_api.cu", "lq_store_kernels.cu", "lq_decode_scalar.cu", "lq_decode_mma.cu", "lq_decode_umma.cu", "lq_decode_static.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-              "-Xcompiler", "-fPIC", "-shared", "--expt-relaxed-constexpr"]
+              "-Xcompiler", "-fPIC", "-shared", "--expt-relaxed-constexpr", "--threads", "0"]
 
 
 def _stale(lib=LIB) -> bool:
