@@ -1132,6 +1132,7 @@ lq_status_t lq_import(lq_cache_t* c, int32_t layer, const lq_image_t* img, int64
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) status = cuda_fail(c, e, "import kernels");
     c->n_launches += (n_quant > 0) + (n_fp > 0);
+    c->last_decode_layer = -1;
   }
   for (auto& b : bufs) dev_release(c, b.dev);
   dev_release(c, slots_dev);
