@@ -30,7 +30,7 @@ struct CacheView {
 #ifdef LQ_DEBUG_BOUNDS
 #define LQ_IN_BOUNDS(cv, cond) ((cond) ? true : (atomicOr((cv).status, 4), false))
 #else
-#define LQ_IN_BOUNDS(cv, cond) true
+#define LQ_IN_BOUNDS(cv, cond) ((void)sizeof(cond), true)
 #endif
 // slots of the full-precision store of one (layer, b, kv); tiles of the 2-bit store
 __host__ __device__ inline int64_t fp_slots_cap(const CacheView& cv) {
