@@ -57,6 +57,9 @@ constexpr int kSpinLimit = 1 << 22;
 // cost of one fp tile (16 bf16 tokens, two loads) in eighths of a quant tile: 4 to 12 measured alike,
 // 2 and 16 slower
 constexpr int kFpCost8 = 8;
+// (with two column blocks -- five to eight query heads per KV head -- a quant tile costs more and the bf16 tile
+// relatively less: 4, measured 2.5 % better than 8 on the GQA-7 workload)
+__host__ __device__ constexpr int fp_cost8(int ncb) { return ncb == 2 ? 4 : kFpCost8; }
 
 // ---- PTX wrappers ----------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -674,7 +677,8 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
   const uint32_t* fpmask = PADDED ? a.fpmask + static_cast<int64_t>(b) * a.fpmask_words : nullptr;
   int it, it_end;
   {
-    const int F8 = a.tiles_fp * kFpCost8, C8 = F8 + (a.tiles_quant - qskip) * 8;
+    constexpr int kCost = fp_cost8(NCB);
+    const int F8 = a.tiles_fp * kCost, C8 = F8 + (a.tiles_quant - qskip) * 8;
     // Overlapped launches (DecodeArgs::early): the CTAs of a launch take over the slots of earlier launches in
     // launch order, and the last slots to free up are those of merging CTAs -- one per pair, and the last CTA of
     // every pair is launched last.  That CTA starts later than the others; it gets 3/4 of a share (measured with a
@@ -685,7 +689,7 @@ __global__ void __launch_bounds__(kWarps * 32, NCB == 1 ? kCtasPerSm : kCtasPerS
     auto cut = [&](int k) {
       const int64_t cw4 = k <= full_warps ? 4LL * k : 4 * full_warps + 3 * (k - full_warps);
       const int pos8 = static_cast<int>(cw4 * C8 / total_w4);
-      return pos8 < F8 ? (pos8 + kFpCost8 / 2) / kFpCost8 : a.tiles_fp + (pos8 - F8 + 4) / 8;
+      return pos8 < F8 ? (pos8 + kCost / 2) / kCost : a.tiles_fp + (pos8 - F8 + 4) / 8;
     };
     it = cut(gw);
     it_end = cut(gw + 1);
@@ -1281,7 +1285,7 @@ int plan_decode_mma_padded(const DecodeArgs& a, int sm_count, int max_records, c
   int64_t total = 0;
   for (int p = 0; p < pairs; ++p) {
     const int tq = std::max(0, tiles_quant - rowinfo_host[4 * (p / a.cv.Hkv) + 0]);
-    work[p] = static_cast<int64_t>(tiles_fp) * kFpCost8 + 8LL * tq;  // the kernel's cost line
+    work[p] = static_cast<int64_t>(tiles_fp) * fp_cost8(r <= 4 ? 1 : 2) + 8LL * tq;  // the kernel's cost line
     const int items = tiles_fp + tq / tps;
     cap[p] = std::max(1, std::min(cap_records, items / kWarps));  // at least one item per warp
     total += work[p];
