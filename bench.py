@@ -558,12 +558,13 @@ def main():
                     help="create the caches without LQ_FLAG_OVERLAP_DECODE: every attention launch waits for the one before it")
     ap.add_argument("--also", default=None,
                     help="comma-separated workloads whose attention kernel is timed back to back as well and reported "
-                         "under roofline_<workload> (default: gqa7-32k and llama3-8b-4k-b64 beside the default workload)")
+                         "under roofline_<workload> (default: the other configurations -- gqa7-32k, the batch sweep, mha-128k -- beside the default workload)")
     ap.add_argument("--also-layers", type=int, default=8, help="layer caches of the --also workloads")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.also is None:
-        args.also = "gqa7-32k,llama3-8b-4k-b64" if args.workload == "llama3-8b-8k" and args.layers == 0 else ""
+        args.also = ("gqa7-32k,llama3-8b-4k-b16,llama3-8b-4k-b32,llama3-8b-4k-b64,mha-128k"
+                     if args.workload == "llama3-8b-8k" and args.layers == 0 else "")
 
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         # replicas only: --gpus N without a launcher starts N ranks of this script (one per GPU), which time N
