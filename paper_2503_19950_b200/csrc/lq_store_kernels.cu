@@ -74,17 +74,32 @@ cudaError_t launch_append(const CacheView& cv, int layer, const void* k, const v
 //   all codes 0 when scale == 0.  A zero-valued min or max is taken as +0.  The 4-bit cache uses 15
 //   in place of 3 and stores every code as two 2-bit planes (low bits, high bits).
 // ---------------------------------------------------------------------------------------
+// rows of the staged K / V rows in shared memory: 8 elements of padding (a multiple of 16 bytes) so that the packing
+// step, which reads one element of 8 rows per code position, meets 8 different banks
+constexpr int kSRow = kD + 8;
+
 __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) {
   return __uint_as_float(static_cast<uint32_t>(b) << 16);
 }
 
-// top = highest code: 3 (2 bits) or 15 (4 bits)
-__device__ __forceinline__ uint32_t quant_code(float x, float mn, float scale, float top) {
-  if (scale == 0.0f) return 0u;
-  float q = __fdiv_rn(__fsub_rn(x, mn), scale);
-  float r = rintf(q);
+// top = highest code: 3 (2 bits) or 15 (4 bits).  inv = an approximation of 1 / scale (rcp.approx, computed once
+// per group).  The code is rint(fdiv(fsub(x, mn), scale)) in IEEE arithmetic, exactly: the quotient lies in
+// [0, top + 1/2], so d * inv differs from it by less than 16 * 2^-21 = 2^-17; unless d * inv comes that close to a
+// rounding boundary k + 1/2 (ties included), rounding it gives the same integer as rounding the exact quotient,
+// and only then is the division carried out.
+// scale == 0 (all codes 0): the caller passes inv = 0, so that d * inv = 0 without a branch.
+__device__ __forceinline__ uint32_t quant_code(float x, float mn, float scale, float inv, float top) {
+  const float d = __fsub_rn(x, mn);
+  const float t = __fmul_rn(d, inv);
+  float r = rintf(t);
+  if (!(fabsf(fabsf(__fsub_rn(t, r)) - 0.5f) > 0x1p-16f)) r = rintf(__fdiv_rn(d, scale));  // also catches NaN / inf
   r = fminf(fmaxf(r, 0.0f), top);
   return static_cast<uint32_t>(r);
+}
+__device__ __forceinline__ float approx_rcp(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 
 __device__ __forceinline__ void group_params(float mn, float mx, float top, uint16_t& scale_bits,
@@ -101,7 +116,7 @@ __device__ __forceinline__ void group_params(float mn, float mx, float top, uint
 // Steps 3 and 4 of the overflow step for one key group whose G rows sit in shared memory
 // (sK, sV: [G][128] bf16 bits; overwritten by the codes).  256 threads.
 template <int G, int P>
-__device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kD], uint16_t (&sV)[G][kD], uint8_t* tile, int tid,
+__device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kSRow], uint16_t (&sV)[G][kSRow], uint8_t* tile, int tid,
                                                    int layout) {
   constexpr int NS = G / 16;
   constexpr float kTop = P == 1 ? 3.0f : 15.0f;
@@ -120,9 +135,10 @@ __device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kD], uint16
     group_params(mn, mx, kTop, sb, zb, mnc, scale);
     *reinterpret_cast<uint16_t*>(tile + kscale_off(layout, G, d)) = sb;
     *reinterpret_cast<uint16_t*>(tile + kzero_off(layout, G, d)) = zb;
+    const float inv = scale == 0.0f ? 0.0f : approx_rcp(scale);
 #pragma unroll 4
     for (int e = 0; e < G; ++e)
-      sK[e][d] = static_cast<uint16_t>(quant_code(bf16_bits_to_float(sK[e][d]), mnc, scale, kTop));
+      sK[e][d] = static_cast<uint16_t>(quant_code(bf16_bits_to_float(sK[e][d]), mnc, scale, inv, kTop));
   } else {
     const int warp = (tid >> 5) - 4, lane = tid & 31;
     constexpr int LPG = G / 4;  // lanes per value group
@@ -140,6 +156,7 @@ __device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kD], uint16
       uint16_t sb, zb;
       float mnc, scale;
       group_params(mn, mx, kTop, sb, zb, mnc, scale);
+      const float inv = scale == 0.0f ? 0.0f : approx_rcp(scale);
       if ((lane % LPG) == 0) {
         const int g = lane / LPG;
         *reinterpret_cast<uint16_t*>(tile + vscale_off(layout, G, P, e, g)) = sb;
@@ -147,7 +164,7 @@ __device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kD], uint16
       }
 #pragma unroll
       for (int i = 0; i < 4; ++i)
-        sV[e][4 * lane + i] = static_cast<uint16_t>(quant_code(x[i], mnc, scale, kTop));
+        sV[e][4 * lane + i] = static_cast<uint16_t>(quant_code(x[i], mnc, scale, inv, kTop));
     }
   }
   __syncthreads();
@@ -206,8 +223,8 @@ __device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kD], uint16
 template <int G, int P>
 __global__ void __launch_bounds__(256)
 lq_compress_kernel(CacheView cv, LayerList layers, EvictList ev, int64_t tile0) {
-  __shared__ __align__(16) uint16_t sK[G][kD];
-  __shared__ __align__(16) uint16_t sV[G][kD];
+  __shared__ __align__(16) uint16_t sK[G][kSRow];
+  __shared__ __align__(16) uint16_t sV[G][kSRow];
   const int tau = blockIdx.x;
   const int64_t pair = blockIdx.y;
   const int layer = layers.layer[blockIdx.z];
@@ -272,8 +289,8 @@ template <int G, int P>
 __global__ void __launch_bounds__(256)
 lq_ingest_kernel(CacheView cv, int layer, const uint4* __restrict__ k, const uint4* __restrict__ v, int n_src,
                  const int* __restrict__ idx, int n_tiles, int n_fp, int64_t tile0) {
-  __shared__ __align__(16) uint16_t sK[G][kD];
-  __shared__ __align__(16) uint16_t sV[G][kD];
+  __shared__ __align__(16) uint16_t sK[G][kSRow];
+  __shared__ __align__(16) uint16_t sV[G][kSRow];
   const int64_t pair = blockIdx.y;
   const int tid = threadIdx.x;
   if (static_cast<int>(blockIdx.x) < n_tiles) {
