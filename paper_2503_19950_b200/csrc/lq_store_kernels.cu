@@ -113,63 +113,113 @@ __device__ __forceinline__ void group_params(float mn, float mx, float top, uint
   zero_bits = __bfloat16_as_ushort(__float2bfloat16_rn(mn_c));  // exact: mn is a bf16 value
 }
 
+// What the code phase needs of one group, as a float4:
+//   2-bit codes: {min, T1, T2, T3} with T_i = (i - 1/2) * scale.  scale is a bf16 value, so every T_i is an exact
+//     binary32 number, and for d = fsub(x, min) >= 0
+//         rint(fdiv(d, scale)) = [d > T1] + [d >= T2] + [d > T3]          (clamped at 3 by construction)
+//     holds exactly: at d = T_i the quotient is i - 1/2 and the tie goes to the even neighbour (0, 2, 2); a float
+//     d above (below) T_i differs from it by at least one unit in the last place of T_i, i.e. by more than
+//     2^-24 T_i, which is more than the half unit in the last place of the quotient's neighbourhood of i - 1/2
+//     (at most 2^-24 (i - 1/2)), so the rounded quotient lies strictly on the same side of i - 1/2 as d of T_i.
+//     scale == 0 (every code 0) is encoded as T_i = +inf.
+//   4-bit codes: {min, scale, inv, unused}, see quant_code.
+template <int P>
+__device__ __forceinline__ float4 make_group(float mn, float mx, uint16_t& scale_bits, uint16_t& zero_bits) {
+  constexpr float kTop = P == 1 ? 3.0f : 15.0f;
+  float mnc, scale;
+  group_params(mn, mx, kTop, scale_bits, zero_bits, mnc, scale);
+  if (P == 1) {
+    const bool flat = scale == 0.0f;
+    return make_float4(mnc, flat ? INFINITY : 0.5f * scale, flat ? INFINITY : 1.5f * scale,
+                       flat ? INFINITY : 2.5f * scale);
+  }
+  return make_float4(mnc, scale, scale == 0.0f ? 0.0f : approx_rcp(scale), 0.0f);
+}
+template <int P>
+__device__ __forceinline__ uint32_t group_code(float x, const float4& p) {
+  if (P == 1) {
+    const float d = __fsub_rn(x, p.x);
+    return static_cast<uint32_t>(d > p.y) + static_cast<uint32_t>(d >= p.z) + static_cast<uint32_t>(d > p.w);
+  }
+  return quant_code(x, p.x, p.y, p.z, 15.0f);
+}
+__device__ __forceinline__ float lo_bf16(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float hi_bf16(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+__device__ __forceinline__ uint32_t min_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("min.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+
 // Steps 3 and 4 of the overflow step for one key group whose G rows sit in shared memory
-// (sK, sV: [G][128] bf16 bits; overwritten by the codes).  256 threads.
+// (sK, sV: [G][128] bf16 bits, read only).  256 threads.
+//   A. group parameters: keys, two threads per channel pair (packed bf16 min / max down half of the tokens each);
+//      values, LPG = G/4 lanes per group and LPG rows per warp: the rows' (min, -max) pairs are reduced with a
+//      folding exchange, after which every lane owns one (row, group) and the parameters are computed once each.
+//   B. every thread builds whole words of the tile: it quantises exactly the 16 elements a word holds (two words
+//      that share their parameters at a time), so the codes never pass through shared memory.
 template <int G, int P>
 __device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kSRow], uint16_t (&sV)[G][kSRow], uint8_t* tile, int tid,
                                                    int layout) {
   constexpr int NS = G / 16;
-  constexpr float kTop = P == 1 ? 3.0f : 15.0f;
-  // 3. quantise
+  constexpr int NG = kD / G;
+  __shared__ float4 pK[kD];      // per key channel
+  __shared__ float4 pV[NG * G];  // per (value group, token): [g][t]
+  const int lane = tid & 31;
+  // ---- A. parameters ----
   if (tid < kD) {
-    const int d = tid;
-    float mn = bf16_bits_to_float(sK[0][d]), mx = mn;
-#pragma unroll 4
-    for (int e = 1; e < G; ++e) {
-      const float x = bf16_bits_to_float(sK[e][d]);
-      mn = fminf(mn, x);
-      mx = fmaxf(mx, x);
+    const int cp = tid >> 1, half = tid & 1;
+    uint32_t mn2 = *reinterpret_cast<const uint32_t*>(&sK[half * (G / 2)][2 * cp]), mx2 = mn2;
+#pragma unroll
+    for (int i = 1; i < G / 2; ++i) {
+      const uint32_t w = *reinterpret_cast<const uint32_t*>(&sK[half * (G / 2) + i][2 * cp]);
+      mn2 = min_bf16x2(mn2, w);
+      mx2 = max_bf16x2(mx2, w);
     }
+    mn2 = min_bf16x2(mn2, __shfl_xor_sync(0xFFFFFFFFu, mn2, 1));
+    mx2 = max_bf16x2(mx2, __shfl_xor_sync(0xFFFFFFFFu, mx2, 1));
+    const int d = tid;  // = 2 * cp + half
     uint16_t sb, zb;
-    float mnc, scale;
-    group_params(mn, mx, kTop, sb, zb, mnc, scale);
+    pK[d] = make_group<P>(half ? hi_bf16(mn2) : lo_bf16(mn2), half ? hi_bf16(mx2) : lo_bf16(mx2), sb, zb);
     *reinterpret_cast<uint16_t*>(tile + kscale_off(layout, G, d)) = sb;
     *reinterpret_cast<uint16_t*>(tile + kzero_off(layout, G, d)) = zb;
-    const float inv = scale == 0.0f ? 0.0f : approx_rcp(scale);
-#pragma unroll 4
-    for (int e = 0; e < G; ++e)
-      sK[e][d] = static_cast<uint16_t>(quant_code(bf16_bits_to_float(sK[e][d]), mnc, scale, inv, kTop));
   } else {
-    const int warp = (tid >> 5) - 4, lane = tid & 31;
-    constexpr int LPG = G / 4;  // lanes per value group
-    for (int e = warp; e < G; e += 4) {
-      const uint2 raw = *reinterpret_cast<const uint2*>(&sV[e][4 * lane]);
-      float x[4] = {bf16_bits_to_float(raw.x & 0xFFFFu), bf16_bits_to_float(raw.x >> 16),
-                    bf16_bits_to_float(raw.y & 0xFFFFu), bf16_bits_to_float(raw.y >> 16)};
-      float mn = fminf(fminf(x[0], x[1]), fminf(x[2], x[3]));
-      float mx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3]));
+    constexpr int LPG = G / 4;  // lanes per value group = rows per warp
+    const int wv = (tid >> 5) - 4;
+    uint32_t m2[LPG];           // (min, -max) of this lane's four channels, row by row
 #pragma unroll
-      for (int o = 1; o < LPG; o <<= 1) {
-        mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, o));
-        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-      }
-      uint16_t sb, zb;
-      float mnc, scale;
-      group_params(mn, mx, kTop, sb, zb, mnc, scale);
-      const float inv = scale == 0.0f ? 0.0f : approx_rcp(scale);
-      if ((lane % LPG) == 0) {
-        const int g = lane / LPG;
-        *reinterpret_cast<uint16_t*>(tile + vscale_off(layout, G, P, e, g)) = sb;
-        *reinterpret_cast<uint16_t*>(tile + vzero_off(layout, G, P, e, g)) = zb;
-      }
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-        sV[e][4 * lane + i] = static_cast<uint16_t>(quant_code(x[i], mnc, scale, inv, kTop));
+    for (int i = 0; i < LPG; ++i) {
+      const uint2 raw = *reinterpret_cast<const uint2*>(&sV[wv * LPG + i][4 * lane]);
+      const uint32_t lo = min_bf16x2(raw.x, raw.y), hi = max_bf16x2(raw.x, raw.y);
+      const uint32_t a = __byte_perm(lo, hi, 0x5410) ^ 0x80000000u;  // (min of channels 0 and 2, -max of the same)
+      const uint32_t b = __byte_perm(lo, hi, 0x7632) ^ 0x80000000u;  // channels 1 and 3
+      m2[i] = min_bf16x2(a, b);
     }
+#pragma unroll
+    for (int lvl = LPG / 2; lvl >= 1; lvl >>= 1) {
+      const bool upper = (lane & lvl) != 0;
+#pragma unroll
+      for (int i = 0; i < lvl; ++i) {
+        const uint32_t send = upper ? m2[i] : m2[i + lvl];
+        const uint32_t keep = upper ? m2[i + lvl] : m2[i];
+        m2[i] = min_bf16x2(keep, __shfl_xor_sync(0xFFFFFFFFu, send, lvl));
+      }
+    }
+    // m2[0] now covers the whole group of row (lane % LPG) of this warp's rows
+    const int e = wv * LPG + (lane % LPG), g = lane / LPG;
+    uint16_t sb, zb;
+    pV[g * G + e] = make_group<P>(lo_bf16(m2[0]), hi_bf16(m2[0] ^ 0x80000000u), sb, zb);
+    *reinterpret_cast<uint16_t*>(tile + vscale_off(layout, G, P, e, g)) = sb;
+    *reinterpret_cast<uint16_t*>(tile + vzero_off(layout, G, P, e, g)) = zb;
   }
   __syncthreads();
 
-  // 4. pack
+  // ---- B. codes, word by word ----
   if (layout == kLayoutRow) {
     // one word = 16 codes of one row: K words [half][token][4], V words [channel][G/16]
     for (int idx = tid; idx < 2 * G * 8; idx += 256) {
@@ -177,45 +227,74 @@ __device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kSRow], uin
       if (idx < G * 8) {
         const int hf = idx / (G * 4), t = (idx >> 2) % G, ks = 4 * hf + (idx & 3);
 #pragma unroll
-        for (int e = 0; e < 16; ++e) word |= static_cast<uint32_t>(sK[t][16 * ks + e] & 3u) << row_code_bit(e);
+        for (int e = 0; e < 16; ++e)
+          word |= (group_code<P>(bf16_bits_to_float(sK[t][16 * ks + e]), pK[16 * ks + e]) & 3u) << row_code_bit(e);
         reinterpret_cast<uint32_t*>(tile + row_kcodes_off())[idx] = word;
       } else {
         const int wd = idx - G * 8, d = wd / (G / 16), j = wd % (G / 16);
 #pragma unroll
-        for (int e = 0; e < 16; ++e) word |= static_cast<uint32_t>(sV[16 * j + e][d] & 3u) << row_code_bit(e);
+        for (int e = 0; e < 16; ++e)
+          word |= (group_code<P>(bf16_bits_to_float(sV[16 * j + e][d]), pV[(d / G) * G + 16 * j + e]) & 3u)
+                  << row_code_bit(e);
         reinterpret_cast<uint32_t*>(tile + row_vcodes_off(G))[wd] = word;
       }
     }
     return;
   }
   // fragment order, one 2-bit plane after the other
-  for (int idx = tid; idx < 2 * P * NS * 128; idx += 256) {
-    const int which = idx / (P * NS * 128);
-    const int pl = (idx / (NS * 128)) % P;
-    const int wd = idx % (NS * 128);
-    uint32_t* kw = reinterpret_cast<uint32_t*>(tile + qt_kcodes_off() + pl * qt_plane_bytes(G));
-    uint32_t* vw = reinterpret_cast<uint32_t*>(tile + qt_vcodes_off(G, P) + pl * qt_plane_bytes(G));
-    const int u = wd >> 7, lane = (wd >> 2) & 31, sub = wd & 3;
-    const int hi = lane >> 2, j = lane & 3;
-    uint32_t word = 0;
-    if (which == 0) {
-      const int nt = sub >> 1, w = sub & 1;
-      const int t = 16 * u + 8 * nt + hi;
+  for (int item = tid; item < NS * 128; item += 256) {
+    uint32_t word[2][P] = {};
+    if (item < NS * 64) {
+      // keys: tokens t0 and t0 + 8 (n-tiles 0 and 1) at the 16 channels 16 ks + 8 w + 2 j + h
+      const int hi = (item >> 2) & 7, j = item & 3, w = (item >> 5) & 1, u = item >> 6;
+      const int t0 = 16 * u + hi;
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks)
+      for (int ks = 0; ks < 8; ++ks) {
+        const int ch = 16 * ks + 8 * w + 2 * j;
+        const float4 pa = pK[ch], pb = pK[ch + 1];
 #pragma unroll
-        for (int h = 0; h < 2; ++h)
-          word |= static_cast<uint32_t>((sK[t][16 * ks + 8 * w + 2 * j + h] >> (2 * pl)) & 3u) << (16 * h + 2 * ks);
-      kw[wd] = word;
+        for (int nt = 0; nt < 2; ++nt) {
+          const uint32_t x = *reinterpret_cast<const uint32_t*>(&sK[t0 + 8 * nt][ch]);
+          const uint32_t ca = group_code<P>(lo_bf16(x), pa), cb = group_code<P>(hi_bf16(x), pb);
+#pragma unroll
+          for (int pl = 0; pl < P; ++pl)
+            word[nt][pl] |= (((ca >> (2 * pl)) & 3u) << (2 * ks)) | (((cb >> (2 * pl)) & 3u) << (16 + 2 * ks));
+        }
+      }
+#pragma unroll
+      for (int pl = 0; pl < P; ++pl) {
+        uint32_t* kw = reinterpret_cast<uint32_t*>(tile + qt_kcodes_off() + pl * qt_plane_bytes(G));
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) kw[u * 128 + 4 * (4 * hi + j) + 2 * nt + w] = word[nt][pl];
+      }
     } else {
-      const int dh = sub & 1, th = sub >> 1;
+      // values: tokens tt and tt + 1 at the channels 16 mt + 8 dh + r for r = 2 p and 2 p + 1 (one word each)
+      const int vi = item - NS * 64;
+      const int j = vi & 3, p = (vi >> 2) & 3, dh = (vi >> 4) & 1, th = (vi >> 5) & 1, u = vi >> 6;
+      const int tt = 16 * u + 8 * th + 2 * j;
 #pragma unroll
-      for (int mt = 0; mt < 8; ++mt)
+      for (int mt = 0; mt < 8; ++mt) {
+        const int ch = 16 * mt + 8 * dh + 2 * p;
+        constexpr int kShift = G == 32 ? 1 : 2;  // value group of m-tile mt: 16 mt / G
+        const int g = mt >> kShift;
 #pragma unroll
-        for (int h = 0; h < 2; ++h)
-          word |= static_cast<uint32_t>((sV[16 * u + 8 * th + 2 * j + h][16 * mt + 8 * dh + hi] >> (2 * pl)) & 3u)
-                  << (16 * h + 2 * mt);
-      vw[wd] = word;
+        for (int h = 0; h < 2; ++h) {
+          const float4 pv = pV[g * G + tt + h];
+          const uint32_t x = *reinterpret_cast<const uint32_t*>(&sV[tt + h][ch]);
+          const uint32_t ca = group_code<P>(lo_bf16(x), pv), cb = group_code<P>(hi_bf16(x), pv);
+#pragma unroll
+          for (int pl = 0; pl < P; ++pl) {
+            word[0][pl] |= ((ca >> (2 * pl)) & 3u) << (16 * h + 2 * mt);
+            word[1][pl] |= ((cb >> (2 * pl)) & 3u) << (16 * h + 2 * mt);
+          }
+        }
+      }
+#pragma unroll
+      for (int pl = 0; pl < P; ++pl) {
+        uint32_t* vw = reinterpret_cast<uint32_t*>(tile + qt_vcodes_off(G, P) + pl * qt_plane_bytes(G));
+#pragma unroll
+        for (int b = 0; b < 2; ++b) vw[u * 128 + 4 * (4 * (2 * p + b) + j) + dh + 2 * th] = word[b][pl];
+      }
     }
   }
 }
