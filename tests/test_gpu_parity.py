@@ -645,3 +645,51 @@ def test_overlapped_decode_launches_of_different_layers(L, fused, r, pad):
         assert_images_equal(cache.export(l), ocs[l].export())
     assert cache.kernel_status() == 0
     cache.close()
+
+
+@pytest.mark.parametrize("W,G,bits", [(32, 32, 2), (64, 64, 2), (32, 32, 4), (64, 64, 4)])
+def test_codes_at_the_rounding_boundaries(W, G, bits):
+    """Groups whose quotients (x - min) / scale sit exactly on k + 1/2 (ties) and one bf16 step beside it, at
+    exponents from the bf16 subnormal range up: the codes must be the oracle's, bit for bit.  Every group draws from
+    {0 .. 2 top} * 2^e and the bf16 neighbours of the odd members, so that scale = 2 * 2^e whenever 0 and
+    2 top are both drawn, and other nearby scales otherwise."""
+    B, Hq, Hkv, D = 2, 4, 2, 128
+    N = 5 * W + 1
+    top = (1 << bits) - 1
+    rng = np.random.default_rng(1234 + W + bits)
+    base = np.arange(0, 2 * top + 1, dtype=np.float64)
+    odd = base[1::2]
+    ulp = 2.0 ** (np.floor(np.log2(odd)) - 7)            # bf16 spacing at the odd members
+    cand = np.concatenate([base, odd + ulp, odd - ulp / np.where(odd == 2.0 ** np.floor(np.log2(odd)), 2, 1)])
+    exps = np.array([-130.0, -40.0, -3.0, 0.0, 3.0])
+
+    def draw(shape_groups, axis_len, axis):
+        e = rng.choice(exps, size=shape_groups)
+        idx = rng.integers(0, len(cand), size=shape_groups[:axis] + (axis_len,) + shape_groups[axis:])
+        # bf16 subnormals (multiples of 2^-133) hold the integer members only
+        idx = np.where(np.expand_dims(e, axis) < -126, idx % len(base), idx)
+        vals = cand[idx] * np.expand_dims(2.0 ** e, axis)
+        sign = rng.choice([1.0, -1.0], size=shape_groups)   # mirrored groups: the minimum is the negative end
+        return (vals * np.expand_dims(sign, axis)).astype(np.float32)
+
+    k = draw((B, Hkv, D), N, 2)                               # one exponent per channel: key groups run over tokens
+    v = draw((B, Hkv, N, D // G), G, 4).reshape(B, Hkv, N, D)  # one exponent per (token, channel group)
+    kt = torch.from_numpy(k).to(torch.bfloat16).cuda()
+    vt = torch.from_numpy(v).to(torch.bfloat16).cuda()
+    assert (kt.float().cpu().numpy() == k).all() and (vt.float().cpu().numpy() == v).all()  # representable
+    for chunk in (N, 1):                                       # one ingestion launch, then token by token
+        cache = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=N + 4, bits=bits)
+        oc = oracle.OracleCache(B, Hq, Hkv, D, W, G, bits=bits)
+        for s in range(0, N, chunk):
+            cache.append(0, kt[:, :, s:s + chunk].contiguous(), vt[:, :, s:s + chunk].contiguous())
+        oc.append(synth.bf16_bits(kt), synth.bf16_bits(vt))
+        want = oc.export()
+        assert_images_equal(cache.export(0), want)
+        for key in ("k_codes", "v_codes"):                      # every code value occurs (packed low bits first)
+            seen = set()
+            for sh in range(0, 8, bits):
+                seen |= set(np.unique((want[key] >> sh) & top).tolist())
+            assert seen == set(range(top + 1)), key
+        assert cache.kernel_status() == 0
+        cache.close()
+        oc.close()
