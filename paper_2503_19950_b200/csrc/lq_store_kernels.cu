@@ -138,8 +138,10 @@ __device__ __forceinline__ float4 make_group(float mn, float mx, uint16_t& scale
 template <int P>
 __device__ __forceinline__ uint32_t group_code(float x, const float4& p) {
   if (P == 1) {
+    // the thresholds are nested: the high bit is [d >= T2], the low bit compares with T3 or T1 accordingly
     const float d = __fsub_rn(x, p.x);
-    return static_cast<uint32_t>(d > p.y) + static_cast<uint32_t>(d >= p.z) + static_cast<uint32_t>(d > p.w);
+    const bool high = d >= p.z;
+    return (high ? 2u : 0u) + (d > (high ? p.w : p.y) ? 1u : 0u);
   }
   return quant_code(x, p.x, p.y, p.z, 15.0f);
 }
