@@ -65,9 +65,9 @@ cudaError_t launch_append(const CacheView& cv, int layer, const void* k, const v
 //   2. back-fills the G holes with rows the host names (the top rows of the dense prefix: slots
 //      2W + tau*G + e when W is a multiple of G), so the valid slots stay a dense prefix -- legal
 //      because the order of the cache is free (Eq. 3) -- and only this CTA ever touches these 2G slots,
-//   3. quantises: keys per channel down the G tokens (one thread per channel), values per token
-//      across G channels (one warp per token, group min/max by __shfl_xor_sync),
-//   4. packs the codes into the fragment order of the tile and stores the tile.
+//   3. finds min, scale and zero of every group: keys per channel down the G tokens, values per token
+//      across G channels,
+//   4. quantises and stores the tile word by word, in the fragment order (quantise_pack_tile below).
 //
 // Quantiser arithmetic (IEEE binary32, one rounding per operation, ties to even):
 //   zero = min, scale = bf16(fdiv(fsub(max, min), 3)), code = clamp(rint(fdiv(fsub(x, min), scale)), 0, 3),
