@@ -12,6 +12,7 @@
 #include <cstring>
 #include <new>
 #include <string>
+#include <unordered_map>
 #include <vector>
 
 #include "../../include/lq.h"
@@ -45,7 +46,7 @@ struct lq_cache {
   float* part_o = nullptr;
   float* part_ml = nullptr;
   int* status = nullptr;
-  int* ingest_idx = nullptr;  // index list of the one-launch prompt ingestion (max_tokens ints)
+  int* ingest_idx = nullptr;  // index lists of the one-launch ingestion (3 max_tokens + 16 W + 3 G ints)
   int* tickets = nullptr;  // per (b, kv) arrival counters of the fused split-K merge
   float* acc = nullptr;    // per (b, kv) sums of the partials added on arrival (DecodeArgs::acc)
   // staging for the host-buffer entry point, one slice per layer
@@ -487,7 +488,7 @@ lq_status_t lq_cache_create(const lq_config_t* cfg, lq_cache_t** out) {
               dev_alloc(c, reinterpret_cast<void**>(&c->status), 256) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->tickets), pairs * 128) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->acc), static_cast<int64_t>(pairs) * kAccStride * 4) &&
-              dev_alloc(c, reinterpret_cast<void**>(&c->ingest_idx), (cfg->max_tokens + 3 * cfg->window + cfg->group) * 4) &&
+              dev_alloc(c, reinterpret_cast<void**>(&c->ingest_idx), (3 * cfg->max_tokens + 16 * cfg->window + 3 * cfg->group) * 4) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_k), cfg->n_layers * pairs * kD * 2) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_v), cfg->n_layers * pairs * kD * 2) &&
               dev_alloc(c, reinterpret_cast<void**>(&c->stage_q),
@@ -522,8 +523,8 @@ lq_status_t lq_destroy(lq_cache_t* c) {
 
 namespace {
 
-// A prompt appended to an empty layer: the host plays Algorithm 1 token by token on its mirror of
-// the filter (which never looks at the data), collects the removed token ids of every overflow
+// A prompt (or a chunk of one) appended in one launch: the host plays Algorithm 1 token by token on its mirror
+// of the filter (which never looks at the data), collects the removed token ids of every overflow
 // step and the final slot map, and one kernel writes both stores.
 // host bookkeeping of one overflow of layer L (no device work); idx, when given, collects the ids of the tokens that
 // enter the 2-bit store, in store order
@@ -561,19 +562,184 @@ void replay_appends(const lq_cache* c, LayerState& L, int64_t n, std::vector<int
   }
 }
 
+// Plays an ingestion plan on token ids instead of rows (host only, no device work) and checks what the kernel
+// relies on: every key group gathers its tokens in store order; no fp slot is written twice or read twice; a slot
+// that is both read and written has its reader and its writer in the same list entry (one thread of one CTA, the read
+// first); copied slots held nothing before; the store ends as the host maps say; and (top_in_place: W a multiple of
+// G) age positions from 2W on sit in the slot of the same number, as the overflow step expects.  old_tok: slot ->
+// token before the call.  Used by the device-less mode, so that the CPU tests cover the planner.
+bool ingest_plan_is_sound(const LayerState& L, int W, bool top_in_place, const std::vector<int32_t>& old_tok, int64_t seen_old,
+                          const std::vector<int32_t>& ids, const std::vector<int32_t>& idx, bool has_fill, int n_copy) {
+  const int NQ = static_cast<int>(ids.size()), n_old = static_cast<int>(old_tok.size());
+  const int cap = static_cast<int>(L.slot_token.size());
+  std::vector<int32_t> content(cap, -1), reader(cap, -1), writer(cap, -1);
+  for (int s = 0; s < n_old; ++s) content[s] = old_tok[s];
+  std::vector<int32_t> final_tok(content);
+  auto read = [&](int slot, int who) {
+    if (slot < 0 || slot >= n_old || reader[slot] != -1) return false;
+    reader[slot] = who;
+    return true;
+  };
+  auto write = [&](int slot, int who, int32_t tok) {
+    if (slot < 0 || slot >= cap || writer[slot] != -1) return false;
+    writer[slot] = who;
+    final_tok[slot] = tok;
+    return true;
+  };
+  for (int i = 0; i < NQ; ++i) {
+    const int32_t src = idx[i];
+    if (src == -1) return false;
+    if (src >= 0) {
+      if (seen_old + src != ids[i]) return false;
+      if (has_fill && (idx[NQ + i] != -1 || idx[2 * NQ + i] != -1)) return false;
+      continue;
+    }
+    const int s = -2 - src;
+    if (!has_fill || !read(s, i) || content[s] != ids[i]) return false;
+    const int32_t f1 = idx[NQ + i], f2 = idx[2 * NQ + i];
+    if (f1 >= 0) {
+      if (!write(s, i, static_cast<int32_t>(seen_old + f1)) || f2 != -1) return false;
+    } else if (f1 <= -2) {
+      const int m = -2 - f1;
+      if (!read(m, i) || !write(s, i, content[m])) return false;
+      if (f2 >= 0 && !write(m, i, static_cast<int32_t>(seen_old + f2))) return false;
+    } else if (f2 != -1) {
+      return false;
+    }
+  }
+  const size_t copy0 = static_cast<size_t>(has_fill ? 3 : 1) * NQ;
+  for (int j = 0; j < n_copy; ++j) {
+    const int slot = idx[copy0 + 2 * j];
+    if (slot < n_old || idx[copy0 + 2 * j + 1] < 0) return false;
+    if (!write(slot, -2, static_cast<int32_t>(seen_old + idx[copy0 + 2 * j + 1]))) return false;
+  }
+  for (int s = 0; s < cap; ++s)
+    if (reader[s] != -1 && writer[s] != -1 && reader[s] != writer[s]) return false;
+  for (int s = 0; s < L.n_fp; ++s)
+    if (final_tok[s] != L.slot_token[s]) return false;
+  std::vector<char> used(cap, 0);
+  for (size_t a = 0; a < L.age_slot.size(); ++a) {
+    const int s = L.age_slot[a];
+    if (s < 0 || s >= L.n_fp || used[s]) return false;
+    used[s] = 1;
+    if (top_in_place && static_cast<int>(a) >= 2 * W && s != static_cast<int>(a)) return false;
+  }
+  return L.pend_slot.size() + L.age_slot.size() == static_cast<size_t>(L.n_fp);
+}
+
 lq_status_t ingest_prompt(lq_cache* c, int layer, const void* k, const void* v, int n, cudaStream_t st) {
   LayerState& L = c->layers[layer];
   if (!c->mask_dirty.empty()) c->mask_dirty[layer] = 1;
   const int W = c->cfg.window, G = c->cfg.group;
-  std::vector<int32_t> idx;
-  idx.reserve(static_cast<size_t>(n) + 3 * W);
-  replay_appends(c, L, n, &idx);
-  const int n_tiles = static_cast<int>(idx.size()) / G;
-  for (int s = 0; s < L.n_fp; ++s) idx.push_back(L.slot_token[s]);
+  // the layer as it is now: token -> slot of its full-precision rows
+  const int n_fp_old = L.n_fp;
+  const int64_t seen_old = L.n_seen, tile0 = L.n_quant / G;
+  const std::vector<int32_t> old_tok(L.slot_token.begin(), L.slot_token.begin() + n_fp_old);
+  std::unordered_map<int32_t, int> old_slots;
+  for (int s = 0; s < n_fp_old; ++s) old_slots[old_tok[s]] = s;
+  auto old_slot_of = [&](int32_t tok) {
+    auto it = old_slots.find(tok);
+    return it == old_slots.end() ? -1 : it->second;
+  };
+  std::vector<int32_t> ids;  // tokens that enter the 2-bit store, in store order
+  ids.reserve(static_cast<size_t>(n) + 3 * W);
+  replay_appends(c, L, n, &ids);
+  const int n_tiles = static_cast<int>(ids.size()) / G, NQ = n_tiles * G;
+  const bool has_fill = n_fp_old > 0;
+  std::vector<int32_t> idx(static_cast<size_t>(has_fill ? 3 : 1) * NQ, -1);
+  std::vector<int32_t> copy;  // (slot, new-tensor row)
+  if (!has_fill) {
+    for (int i = 0; i < NQ; ++i) idx[i] = ids[i];
+    for (int s = 0; s < L.n_fp; ++s) {
+      copy.push_back(s);
+      copy.push_back(L.slot_token[s]);
+    }
+  } else {
+    // The replay above moved rows the way the token-by-token path does; the slots are private, so this launch is
+    // free to place them otherwise, and it places them so that no slot is read by one thread and written by another:
+    // old rows that stay below 2W keep their slot; age positions >= 2W (new tokens all: an overflow step has run)
+    // sit in the slot of the same number, as the overflow step expects; the slots below 2W that lost their token
+    // take first the old rows that sat at 2W or above, then new tokens.
+    const int kept_now = kept(L), n_fp_new = L.n_fp;
+    std::vector<int32_t> tok_at_age(kept_now), new_slot(kept_now, -1);
+    for (int a = 0; a < kept_now; ++a) tok_at_age[a] = L.slot_token[L.age_slot[a]];
+    const int low = std::min(2 * W, n_fp_old);
+    std::vector<char> stays(low, 0);
+    std::vector<int> movers, fresh_tokens;  // age positions below 2W that still need a slot
+    for (int a = 0; a < kept_now; ++a) {
+      if (a >= 2 * W) {
+        new_slot[a] = a;
+        continue;
+      }
+      const int so = tok_at_age[a] < seen_old ? old_slot_of(tok_at_age[a]) : -1;
+      if (so >= 0 && so < 2 * W) {
+        new_slot[a] = so;
+        stays[so] = 1;
+      } else if (so >= 0) {
+        movers.push_back(a);
+      } else {
+        fresh_tokens.push_back(a);
+      }
+    }
+    std::vector<int32_t> fill1_of(std::max(n_fp_old, 1), -1), fill2_of(std::max(n_fp_old, 1), -1);
+    std::vector<int> free_slots;  // below 2W: first the slots that lost their token, then those never used
+    for (int s = 0; s < low; ++s)
+      if (!stays[s]) free_slots.push_back(s);
+    for (int s = n_fp_old; s < 2 * W; ++s) free_slots.push_back(s);
+    size_t next = 0;
+    for (int a : movers) {
+      const int s = free_slots[next++], m = old_slot_of(tok_at_age[a]);
+      new_slot[a] = s;
+      fill1_of[s] = -2 - m;
+      // slot m itself goes to the new token of age position m, if the store reaches that far
+      if (m < n_fp_new) fill2_of[m] = static_cast<int32_t>(tok_at_age[m] - seen_old);
+    }
+    for (int a : fresh_tokens) {
+      const int s = free_slots[next++];
+      new_slot[a] = s;
+      const int32_t row = static_cast<int32_t>(tok_at_age[a] - seen_old);
+      if (s < n_fp_old) {
+        fill1_of[s] = row;
+      } else {
+        copy.push_back(s);
+        copy.push_back(row);
+      }
+    }
+    for (int a = 2 * W; a < n_fp_new; ++a) {
+      const int32_t row = static_cast<int32_t>(tok_at_age[a] - seen_old);
+      if (a >= n_fp_old) {
+        copy.push_back(a);
+        copy.push_back(row);
+      } else if (fill2_of[a] == -1) {
+        fill1_of[a] = row;  // its old token leaves through a key group (or it would be a mover with fill2 set)
+      }
+    }
+    for (int i = 0; i < NQ; ++i) {
+      if (ids[i] >= seen_old) {
+        idx[i] = static_cast<int32_t>(ids[i] - seen_old);
+        continue;
+      }
+      const int s = old_slot_of(ids[i]);
+      idx[i] = -2 - s;
+      idx[NQ + i] = fill1_of[s];
+      if (fill1_of[s] <= -2) idx[2 * NQ + i] = fill2_of[-2 - fill1_of[s]];
+    }
+    for (int a = 0; a < kept_now; ++a) {
+      L.age_slot[a] = new_slot[a];
+      L.slot_token[new_slot[a]] = tok_at_age[a];
+    }
+  }
+  const int n_copy = static_cast<int>(copy.size()) / 2;
+  idx.insert(idx.end(), copy.begin(), copy.end());
+  if (c->dry) {
+    if (ingest_plan_is_sound(L, W, !residual_mode(c), old_tok, seen_old, ids, idx, has_fill, n_copy)) return LQ_OK;
+    c->last_error = "ingestion plan failed its self-check";
+    return LQ_ERR_CUDA;
+  }
   // pageable source: the runtime stages it before the call returns, so `idx` may die here
   cudaError_t e = cudaMemcpyAsync(c->ingest_idx, idx.data(), idx.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st);
   if (e != cudaSuccess) return cuda_fail(c, e, "prompt index upload");
-  e = launch_ingest(c->cv, layer, k, v, n, c->ingest_idx, n_tiles, L.n_fp, 0, st);
+  e = launch_ingest(c->cv, layer, k, v, n, c->ingest_idx, n_tiles, has_fill, n_copy, tile0, st);
   if (e != cudaSuccess) return cuda_fail(c, e, "lq_ingest_kernel");
   { c->n_launches++; c->last_decode_layer = -1; }
   return LQ_OK;
@@ -602,7 +768,11 @@ lq_status_t append_impl(lq_cache_t* c, int32_t layer, const void* k, const void*
   if (L.n_seen + n > c->cfg.max_tokens) return LQ_ERR_CAPACITY;
   if (!c->cfg.auto_compress && kept(L) + n > 3 * W) return LQ_ERR_WINDOW_FULL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (!c->dry && c->cfg.auto_compress && L.n_seen == 0 && n > 3 * W && extra_bytes == 0)
+  // more than one launch's worth of work: a prompt for an empty layer, or a chunk of at least two windows that makes
+  // a layer already in use overflow (not when removed tokens wait for a full key group, W % G != 0).  Below two
+  // windows the index upload of the one-launch path costs more than the launches it saves.
+  if (c->cfg.auto_compress && extra_bytes == 0 &&
+      (L.n_seen == 0 ? n > 3 * W : (n >= 2 * W && kept(L) + n > 3 * W && !residual_mode(c))))
     return ingest_prompt(c, layer, k, v, n, st);
   int done = 0;
   while (done < n) {

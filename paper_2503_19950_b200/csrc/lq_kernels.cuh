@@ -60,10 +60,11 @@ cudaError_t launch_append(const CacheView& cv, int layer, const void* k, const v
 cudaError_t launch_compress(const CacheView& cv, const LayerList& layers, const EvictList& ev,
                             int64_t tile0, int n_groups, cudaStream_t st);
 
-// Prompt ingestion into an empty layer in one launch: idx_dev = [n_tiles*G removed prompt positions in store
-// order][n_fp: final fp slot -> prompt position]; k, v = [B, Hkv, n_src, 128] bf16.
+// Ingestion of n_src new tokens in one launch (lq_ingest_kernel): idx_dev = [n_tiles*G sources of the new key
+// groups in store order][with has_fill: 2 x n_tiles*G take-over sources][n_copy x (fp slot, new-tensor row)];
+// k, v = [B, Hkv, n_src, 128] bf16.
 cudaError_t launch_ingest(const CacheView& cv, int layer, const void* k, const void* v, int n_src, const int* idx_dev,
-                          int n_tiles, int n_fp, int64_t tile0, cudaStream_t st);
+                          int n_tiles, bool has_fill, int n_copy, int64_t tile0, cudaStream_t st);
 
 // Canonical export of one layer into device buffers (any pointer may be null).
 // slot_of_rank[i] = fp slot of the i-th kept id (ascending ids); device array of n_fp ints.

@@ -358,22 +358,32 @@ cudaError_t launch_compress(const CacheView& cv, const LayerList& layers, const 
 }
 
 // ---------------------------------------------------------------------------------------
-// Prompt ingestion in one launch.  Appending an n-token prompt to an empty layer one token at a
-// time (Algorithm 1) ends in a state the host knows in advance, because the filter never looks at
-// the data: the removed tokens of every overflow step, in store order, and the token that ends up
-// in every fp slot.  idx = [n_tiles * G removed prompt positions][n_fp final slot -> prompt
-// position].  CTAs [0, n_tiles) each quantise one key group straight from the prompt tensors, the
-// remaining CTAs write the surviving rows to their final slots; the result is bit-identical to
-// the token-by-token path.
+// Prompt (or prompt chunk) ingestion in one launch.  Appending n tokens one at a time (Algorithm 1)
+// ends in a state the host knows in advance, because the filter never looks at the data: the removed
+// tokens of every overflow step, in store order, and the token that ends up in every fp slot.
+//
+// A source is a row of the new tensors (value >= 0: position in [0, n_src)) or a row the fp store held
+// before the call (value <= -2: slot -2 - value); -1 = none.  idx holds
+//   src   [n_tiles * G]  the rows of every new key group, in store order
+//   fill1 [n_tiles * G]  (only with has_fill) for a group row that came from fp slot s: the source of the row
+//                        that takes slot s over, if any
+//   fill2 [n_tiles * G]  (only with has_fill) when fill1 names an old slot m: the new-tensor row that takes slot m over
+//   copy  [n_copy][2]    (slot, new-tensor row) for the fp slots nobody held before
+// CTAs [0, n_tiles) each gather and quantise one key group; only after its gather does a CTA overwrite the slots it
+// gathered from, and the thread that moves an old row m into such a slot is the one that then overwrites slot m:
+// every slot that is both read and written has its reader and its writer in one thread, in that order.  The
+// remaining CTAs write the copy list.  The stores end up bit-identical to the token-by-token path.
 // ---------------------------------------------------------------------------------------
 template <int G, int P>
 __global__ void __launch_bounds__(256)
 lq_ingest_kernel(CacheView cv, int layer, const uint4* __restrict__ k, const uint4* __restrict__ v, int n_src,
-                 const int* __restrict__ idx, int n_tiles, int n_fp, int64_t tile0) {
+                 const int* __restrict__ idx, int n_tiles, int has_fill, int n_copy, int64_t tile0) {
   __shared__ __align__(16) uint16_t sK[G][kSRow];
   __shared__ __align__(16) uint16_t sV[G][kSRow];
   const int64_t pair = blockIdx.y;
   const int tid = threadIdx.x;
+  uint8_t* fpbase = cv.fp + layer * cv.fp_layer_stride + pair * cv.fp_head_stride;
+  const int vdelta = fp_v_delta(cv.layout);
   if (static_cast<int>(blockIdx.x) < n_tiles) {
     const int tau = blockIdx.x;
     uint8_t* tile = cv.quant + layer * cv.quant_layer_stride + pair * cv.quant_head_stride +
@@ -382,37 +392,67 @@ lq_ingest_kernel(CacheView cv, int layer, const uint4* __restrict__ k, const uin
     for (int i = tid; i < G * 32; i += 256) {
       const int c = i & 15, which = (i >> 4) & 1, e = i >> 5;
       int64_t t = idx[tau * G + e];
-      if (!LQ_IN_BOUNDS(cv, t >= 0 && t < n_src)) t = 0;
-      const uint4 val = (which ? v : k)[(pair * n_src + t) * 16 + c];
+      uint4 val;
+      if (t >= 0) {
+        if (!LQ_IN_BOUNDS(cv, t < n_src)) t = 0;
+        val = (which ? v : k)[(pair * n_src + t) * 16 + c];
+      } else {
+        int slot = static_cast<int>(-2 - t);
+        if (!LQ_IN_BOUNDS(cv, slot >= 0 && slot < fp_slots_cap(cv))) slot = 0;
+        val = *reinterpret_cast<const uint4*>(fpbase + fp_chunk_off(cv.layout, slot, c) + (which ? vdelta : 0));
+      }
       *reinterpret_cast<uint4*>(which ? &sV[e][c * 8] : &sK[e][c * 8]) = val;
     }
     __syncthreads();
+    if (has_fill) {
+      const int* fill1 = idx + n_tiles * G;
+      const int* fill2 = fill1 + n_tiles * G;
+      for (int i = tid; i < G * 32; i += 256) {
+        const int c = i & 15, which = (i >> 4) & 1, e = i >> 5;
+        const int t = idx[tau * G + e], f1 = fill1[tau * G + e];
+        if (t >= 0 || f1 == -1) continue;
+        const int s = -2 - t, vo = which ? vdelta : 0;
+        if (!LQ_IN_BOUNDS(cv, s >= 0 && s < fp_slots_cap(cv) && f1 < n_src && -2 - f1 < fp_slots_cap(cv))) continue;
+        uint4* dst = reinterpret_cast<uint4*>(fpbase + fp_chunk_off(cv.layout, s, c) + vo);
+        if (f1 >= 0) {
+          *dst = (which ? v : k)[(pair * n_src + f1) * 16 + c];
+        } else {
+          const int m = -2 - f1, f2 = fill2[tau * G + e];
+          uint4* old = reinterpret_cast<uint4*>(fpbase + fp_chunk_off(cv.layout, m, c) + vo);
+          *dst = *old;
+          if (f2 >= 0 && LQ_IN_BOUNDS(cv, f2 < n_src)) *old = (which ? v : k)[(pair * n_src + f2) * 16 + c];
+        }
+      }
+    }
     quantise_pack_tile<G, P>(sK, sV, tile, tid, cv.layout);
   } else {
     const int i = (static_cast<int>(blockIdx.x) - n_tiles) * 256 + tid;
-    if (i >= n_fp * 32) return;
-    const int c = i & 15, which = (i >> 4) & 1, slot = i >> 5;
-    const int64_t t = idx[n_tiles * G + slot];
-    if (!LQ_IN_BOUNDS(cv, t >= 0 && t < n_src && slot < fp_slots_cap(cv))) return;
-    uint8_t* base = cv.fp + layer * cv.fp_layer_stride + pair * cv.fp_head_stride;
-    *reinterpret_cast<uint4*>(base + fp_chunk_off(cv.layout, slot, c) + (which ? fp_v_delta(cv.layout) : 0)) =
+    if (i >= n_copy * 32) return;
+    const int c = i & 15, which = (i >> 4) & 1, j = i >> 5;
+    const int* copy = idx + (has_fill ? 3 : 1) * n_tiles * G;
+    const int slot = copy[2 * j];
+    const int64_t t = copy[2 * j + 1];
+    if (!LQ_IN_BOUNDS(cv, t >= 0 && t < n_src && slot >= 0 && slot < fp_slots_cap(cv))) return;
+    *reinterpret_cast<uint4*>(fpbase + fp_chunk_off(cv.layout, slot, c) + (which ? vdelta : 0)) =
         (which ? v : k)[(pair * n_src + t) * 16 + c];
   }
 }
 
 cudaError_t launch_ingest(const CacheView& cv, int layer, const void* k, const void* v, int n_src, const int* idx_dev,
-                          int n_tiles, int n_fp, int64_t tile0, cudaStream_t st) {
-  dim3 grid(n_tiles + (n_fp * 32 + 255) / 256, cv.B * cv.Hkv);
+                          int n_tiles, bool has_fill, int n_copy, int64_t tile0, cudaStream_t st) {
+  dim3 grid(n_tiles + (n_copy * 32 + 255) / 256, cv.B * cv.Hkv);
+  if (grid.x == 0) return cudaSuccess;
   const uint4* k4 = static_cast<const uint4*>(k);
   const uint4* v4 = static_cast<const uint4*>(v);
+  const int hf = has_fill ? 1 : 0;
   if (cv.G == 32 && cv.planes == 1)
-    lq_ingest_kernel<32, 1><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, n_fp, tile0);
+    lq_ingest_kernel<32, 1><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, hf, n_copy, tile0);
   else if (cv.G == 32 && cv.planes == 2)
-    lq_ingest_kernel<32, 2><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, n_fp, tile0);
+    lq_ingest_kernel<32, 2><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, hf, n_copy, tile0);
   else if (cv.G == 64 && cv.planes == 1)
-    lq_ingest_kernel<64, 1><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, n_fp, tile0);
+    lq_ingest_kernel<64, 1><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, hf, n_copy, tile0);
   else if (cv.G == 64 && cv.planes == 2)
-    lq_ingest_kernel<64, 2><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, n_fp, tile0);
+    lq_ingest_kernel<64, 2><<<grid, 256, 0, st>>>(cv, layer, k4, v4, n_src, idx_dev, n_tiles, hf, n_copy, tile0);
   else
     return cudaErrorInvalidValue;
   return cudaGetLastError();

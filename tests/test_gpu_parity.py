@@ -271,8 +271,8 @@ def test_prompt_ingestion_in_one_launch_equals_token_by_token(W, G, n):
     one.append(1, k, v)
     assert one.info(1).n_kernel_launches == before + 1
     seq.append(0, k[:, :, :1].contiguous(), v[:, :, :1].contiguous())
-    for t0 in range(1, n, 97):
-        seq.append(0, k[:, :, t0:t0 + 97].contiguous(), v[:, :, t0:t0 + 97].contiguous())
+    for t0 in range(1, n, 31):   # fewer than W tokens per call: the append and overflow kernels
+        seq.append(0, k[:, :, t0:t0 + 31].contiguous(), v[:, :, t0:t0 + 31].contiguous())
     assert seq.info(0).n_kernel_launches > 2
     oc = oracle.OracleCache(B, Hq, Hkv, D, W, G)
     oc.append(synth.bf16_bits(k), synth.bf16_bits(v))
@@ -295,6 +295,61 @@ def test_prompt_ingestion_in_one_launch_equals_token_by_token(W, G, n):
     assert_images_equal(one.export(1), seq.export(0))
     assert one.kernel_status() == 0 and seq.kernel_status() == 0
     one.close(); seq.close(); oc.close()
+
+
+@pytest.mark.parametrize("W,G,bits,recent,chunks", [
+    (32, 32, 2, False, [1, 32, 100, 33, 64, 250, 32]),          # first call leaves 1 token: every later slot is new
+    (32, 32, 2, False, [95, 97, 1, 1, 40, 500]),                # store almost full, then chunks and single tokens
+    (64, 32, 2, False, [130, 64, 700, 65, 191]),                # two key groups per step; old rows above 2W move down
+    (64, 64, 4, False, [3 * 64, 64, 3 * 64 + 7, 128]),          # full store first, 4-bit codes
+    (128, 64, 2, False, [300, 1000, 129, 2048]),
+    (32, 32, 2, True, [50, 60, 200, 32, 33]),                   # recent-window comparator
+])
+def test_chunks_appended_to_a_layer_in_use_take_one_launch_each(W, G, bits, recent, chunks):
+    """Chunked prefill: a chunk of at least 2 W tokens that makes a layer in use overflow goes through ONE launch,
+    which gathers key groups from the old full-precision rows and from the chunk, lets rows take over the slots
+    that lose their token, and writes the rest of the chunk.  After every chunk the image must be the oracle's bit
+    for bit and attention must agree; single decode steps afterwards (overflow kernel, fused append) must find the
+    store as they expect it."""
+    B, Hq, Hkv, D = 2, 8, 2, 128
+    total = sum(chunks) + 2 * W + 3
+    k, v = synth.keys_values(91, B, Hkv, total, D, "cuda", outliers=synth.outlier_channels(91, Hkv, D, 3))
+    cache = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=total + 8, bits=bits, filter=1 if recent else 0)
+    oc = oracle.OracleCache(B, Hq, Hkv, D, W, G, bits=bits, recent_only=recent)
+    done = 0
+
+    def check(step):
+        inf = cache.info(0)
+        assert (inf.n_seen, inf.n_fp, inf.n_quant, inf.n_events) == (oc.n_seen, oc.n_fp, oc.n_quant, oc.n_events)
+        assert_images_equal(cache.export(0), oc.export())
+        q = synth.queries(91, B, Hq, D, step, "cuda")
+        out = torch.empty(B, Hq, D, device="cuda")
+        cache.decode_attn(0, q, out)
+        ref = oc.attention(synth.bf16_bits(q), 1 / np.sqrt(D))
+        assert np.abs(out.cpu().numpy() - ref).max() <= attn_tolerance(ref)
+
+    for i, n in enumerate(chunks):
+        before = cache.info(0).n_kernel_launches
+        in_use, kept = done > 0, cache.info(0).n_fp
+        cache.append(0, k[:, :, done:done + n].contiguous(), v[:, :, done:done + n].contiguous())
+        if in_use and n >= 2 * W and kept + n > 3 * W:
+            assert cache.info(0).n_kernel_launches == before + 1, (i, n)
+        oc.append(synth.bf16_bits(k[:, :, done:done + n]), synth.bf16_bits(v[:, :, done:done + n]))
+        done += n
+        check(i)
+    for t in range(2 * W + 3):   # token by token across the next overflow steps
+        kn, vn = k[:, :, done:done + 1].contiguous(), v[:, :, done:done + 1].contiguous()
+        q = synth.queries(91, B, Hq, D, 100 + t, "cuda")
+        out = torch.empty(B, Hq, D, device="cuda")
+        cache.append_decode_attn(0, kn, vn, q, out)
+        oc.append(synth.bf16_bits(kn), synth.bf16_bits(vn))
+        done += 1
+        if t % 16 == 0 or t == 2 * W + 2:
+            ref = oc.attention(synth.bf16_bits(q), 1 / np.sqrt(D))
+            assert np.abs(out.cpu().numpy() - ref).max() <= attn_tolerance(ref)
+            assert_images_equal(cache.export(0), oc.export())
+    assert cache.kernel_status() == 0
+    cache.close(); oc.close()
 
 
 @pytest.mark.parametrize("B,Hq,Hkv,W,G,bits,n0,pad", [

@@ -228,3 +228,30 @@ def test_new_entry_points_without_a_device():
     assert lib.lq_debug_stall_next_decode(None) == binding.LQ_ERR_INVALID_ARG
     assert lib.lq_import(None, 0, None, 1, 0, 0) == binding.LQ_ERR_INVALID_ARG
     assert c.info(0).n_ctas_overlapped == 0
+
+
+@pytest.mark.parametrize("W,G,recent", [(32, 32, False), (64, 32, False), (128, 64, False), (64, 64, True)])
+def test_chunks_appended_to_a_layer_in_use_go_through_the_one_launch_plan(W, G, recent):
+    """A chunk of at least 2 W tokens that makes a layer in use overflow is planned as ONE launch (sources of the new
+    key groups, take-over lists, copy list).  Without a device the library plays that plan on token ids and checks
+    that no slot is read by one thread and written by another, that each key group gathers its tokens in store
+    order and that the store ends as its maps say (a failed check is an error status); here the counts and both id
+    lists must also follow the oracle through every mix of first-chunk sizes and chunk lengths, with
+    token-by-token steps (the overflow step's own slot rules) in between."""
+    rng = np.random.default_rng(W + G + recent)
+    for first in (1, W - 1, 2 * W - 3, 2 * W, 2 * W + 1, 3 * W - 1, 3 * W):
+        c = _dry(W=W, G=G, max_tokens=80 * W, filter=binding.LQ_FILTER_RECENT if recent else 0)
+        oc = oracle.OracleCache(1, 4, 2, 128, W, G, recent_only=recent)
+        n = 0
+        for step in [first] + [int(x) for x in rng.choice([1, 2, W, W + 1, 2 * W - 1, 2 * W, 3 * W, 3 * W + 5, 7 * W + 3],
+                                                         size=14)]:
+            c.append(0, None, None, n_tokens=step)
+            oc.append(np.zeros((1, 2, step, 128), np.uint16), np.zeros((1, 2, step, 128), np.uint16))
+            n += step
+            inf = c.info(0)
+            assert (inf.n_seen, inf.n_fp, inf.n_quant, inf.n_events) == (n, oc.n_fp, oc.n_quant, oc.n_events)
+            img, oimg = c.export(0, ids_only=True), oc.export()
+            assert img["kept_ids"].tolist() == oimg["kept_ids"].tolist()
+            assert img["quant_ids"].tolist() == oimg["quant_ids"].tolist()
+        c.close()
+        oc.close()
