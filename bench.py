@@ -559,7 +559,7 @@ def main():
     ap.add_argument("--also", default=None,
                     help="comma-separated workloads whose attention kernel is timed back to back as well and reported "
                          "under roofline_<workload> (default: the other configurations -- gqa7-32k, the batch sweep, mha-128k -- beside the default workload)")
-    ap.add_argument("--also-layers", type=int, default=8, help="layer caches of the --also workloads")
+    ap.add_argument("--also-layers", type=int, default=32, help="layer caches of the --also workloads")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.also is None:

@@ -12,7 +12,6 @@
 #include <cstring>
 #include <new>
 #include <string>
-#include <unordered_map>
 #include <vector>
 
 #include "../../include/lq.h"
@@ -635,11 +634,12 @@ lq_status_t ingest_prompt(lq_cache* c, int layer, const void* k, const void* v, 
   const int n_fp_old = L.n_fp;
   const int64_t seen_old = L.n_seen, tile0 = L.n_quant / G;
   const std::vector<int32_t> old_tok(L.slot_token.begin(), L.slot_token.begin() + n_fp_old);
-  std::unordered_map<int32_t, int> old_slots;
-  for (int s = 0; s < n_fp_old; ++s) old_slots[old_tok[s]] = s;
+  std::vector<std::pair<int32_t, int32_t>> old_slots(n_fp_old);  // (token, slot), sorted by token
+  for (int s = 0; s < n_fp_old; ++s) old_slots[s] = {old_tok[s], s};
+  std::sort(old_slots.begin(), old_slots.end());
   auto old_slot_of = [&](int32_t tok) {
-    auto it = old_slots.find(tok);
-    return it == old_slots.end() ? -1 : it->second;
+    auto it = std::lower_bound(old_slots.begin(), old_slots.end(), std::make_pair(tok, static_cast<int32_t>(-1)));
+    return it != old_slots.end() && it->first == tok ? it->second : -1;
   };
   std::vector<int32_t> ids;  // tokens that enter the 2-bit store, in store order
   ids.reserve(static_cast<size_t>(n) + 3 * W);
