@@ -171,7 +171,7 @@ lq_status_t lq_destroy(lq_cache_t* cache);
  * appends.  auto_compress = 0: LQ_ERR_WINDOW_FULL if the tokens do not fit below 3W (nothing is
  * appended).  auto_compress = 1: the call is split into fill-to-3W / overflow step / continue;
  * when the layer is still empty and n_tokens > 3W (a prompt), or the layer is in use, n_tokens >= 2W
- * and the window overflows on the way (a chunk of a prompt; W a multiple of the group size), the same
+ * and the window overflows on the way (a chunk of a prompt), the same
  * result -- the same image -- is produced by one kernel launch from the kept/removed sets that
  * Algorithm 1 fixes in advance (the index lists of that launch are copied from pageable host memory
  * on `stream`; calls that ingest prompts must share one stream or be ordered by the caller). */

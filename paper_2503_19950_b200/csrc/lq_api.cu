@@ -623,6 +623,10 @@ bool ingest_plan_is_sound(const LayerState& L, int W, bool top_in_place, const s
     used[s] = 1;
     if (top_in_place && static_cast<int>(a) >= 2 * W && s != static_cast<int>(a)) return false;
   }
+  for (int s : L.pend_slot) {
+    if (s < 0 || s >= L.n_fp || used[s]) return false;
+    used[s] = 1;
+  }
   return L.pend_slot.size() + L.age_slot.size() == static_cast<size_t>(L.n_fp);
 }
 
@@ -656,23 +660,29 @@ lq_status_t ingest_prompt(lq_cache* c, int layer, const void* k, const void* v, 
     }
   } else {
     // The replay above moved rows the way the token-by-token path does; the slots are private, so this launch is
-    // free to place them otherwise, and it places them so that no slot is read by one thread and written by another:
-    // old rows that stay below 2W keep their slot; age positions >= 2W (new tokens all: an overflow step has run)
-    // sit in the slot of the same number, as the overflow step expects; the slots below 2W that lost their token
-    // take first the old rows that sat at 2W or above, then new tokens.
-    const int kept_now = kept(L), n_fp_new = L.n_fp;
-    std::vector<int32_t> tok_at_age(kept_now), new_slot(kept_now, -1);
-    for (int a = 0; a < kept_now; ++a) tok_at_age[a] = L.slot_token[L.age_slot[a]];
-    const int low = std::min(2 * W, n_fp_old);
-    std::vector<char> stays(low, 0);
-    std::vector<int> movers, fresh_tokens;  // age positions below 2W that still need a slot
-    for (int a = 0; a < kept_now; ++a) {
-      if (a >= 2 * W) {
+    // free to place them otherwise, and it places them so that no slot is read by one thread and written by another.
+    // W a multiple of G: old rows that stay below 2W keep their slot; age positions >= 2W (new tokens all: an
+    // overflow step has run) sit in the slot of the same number, as the overflow step expects; the slots below 2W
+    // that lost their token take first the old rows that sat at 2W or above, then new tokens.  Otherwise (removed
+    // tokens may wait in the store, and the step path expects nothing but a dense prefix): the same with the end of
+    // the store in place of 2W.
+    const bool residual = residual_mode(c);
+    const int kept_now = kept(L), n_pend = static_cast<int>(L.pend_slot.size()), n_fp_new = L.n_fp;
+    const int n_live = kept_now + n_pend;  // survivors: list A in age order, then the waiting tokens
+    const int limit = residual ? n_fp_new : 2 * W;
+    std::vector<int32_t> tok_of(n_live), new_slot(n_live, -1);
+    for (int a = 0; a < kept_now; ++a) tok_of[a] = L.slot_token[L.age_slot[a]];
+    for (int p = 0; p < n_pend; ++p) tok_of[kept_now + p] = L.slot_token[L.pend_slot[p]];
+    const int low = std::min(limit, n_fp_old);
+    std::vector<char> stays(std::max(low, 1), 0);
+    std::vector<int> movers, fresh_tokens;  // survivors that still need a slot below `limit`
+    for (int a = 0; a < n_live; ++a) {
+      if (a >= limit) {  // (only when W is a multiple of G: there is no waiting list then)
         new_slot[a] = a;
         continue;
       }
-      const int so = tok_at_age[a] < seen_old ? old_slot_of(tok_at_age[a]) : -1;
-      if (so >= 0 && so < 2 * W) {
+      const int so = tok_of[a] < seen_old ? old_slot_of(tok_of[a]) : -1;
+      if (so >= 0 && so < limit) {
         new_slot[a] = so;
         stays[so] = 1;
       } else if (so >= 0) {
@@ -682,22 +692,22 @@ lq_status_t ingest_prompt(lq_cache* c, int layer, const void* k, const void* v, 
       }
     }
     std::vector<int32_t> fill1_of(std::max(n_fp_old, 1), -1), fill2_of(std::max(n_fp_old, 1), -1);
-    std::vector<int> free_slots;  // below 2W: first the slots that lost their token, then those never used
+    std::vector<int> free_slots;  // below `limit`: first the slots that lost their token, then those never used
     for (int s = 0; s < low; ++s)
       if (!stays[s]) free_slots.push_back(s);
-    for (int s = n_fp_old; s < 2 * W; ++s) free_slots.push_back(s);
+    for (int s = n_fp_old; s < limit; ++s) free_slots.push_back(s);
     size_t next = 0;
     for (int a : movers) {
-      const int s = free_slots[next++], m = old_slot_of(tok_at_age[a]);
+      const int s = free_slots[next++], m = old_slot_of(tok_of[a]);
       new_slot[a] = s;
       fill1_of[s] = -2 - m;
       // slot m itself goes to the new token of age position m, if the store reaches that far
-      if (m < n_fp_new) fill2_of[m] = static_cast<int32_t>(tok_at_age[m] - seen_old);
+      if (m < n_fp_new) fill2_of[m] = static_cast<int32_t>(tok_of[m] - seen_old);
     }
     for (int a : fresh_tokens) {
       const int s = free_slots[next++];
       new_slot[a] = s;
-      const int32_t row = static_cast<int32_t>(tok_at_age[a] - seen_old);
+      const int32_t row = static_cast<int32_t>(tok_of[a] - seen_old);
       if (s < n_fp_old) {
         fill1_of[s] = row;
       } else {
@@ -705,8 +715,8 @@ lq_status_t ingest_prompt(lq_cache* c, int layer, const void* k, const void* v, 
         copy.push_back(row);
       }
     }
-    for (int a = 2 * W; a < n_fp_new; ++a) {
-      const int32_t row = static_cast<int32_t>(tok_at_age[a] - seen_old);
+    for (int a = limit; a < n_fp_new; ++a) {
+      const int32_t row = static_cast<int32_t>(tok_of[a] - seen_old);
       if (a >= n_fp_old) {
         copy.push_back(a);
         copy.push_back(row);
@@ -724,9 +734,9 @@ lq_status_t ingest_prompt(lq_cache* c, int layer, const void* k, const void* v, 
       idx[NQ + i] = fill1_of[s];
       if (fill1_of[s] <= -2) idx[2 * NQ + i] = fill2_of[-2 - fill1_of[s]];
     }
-    for (int a = 0; a < kept_now; ++a) {
-      L.age_slot[a] = new_slot[a];
-      L.slot_token[new_slot[a]] = tok_at_age[a];
+    for (int a = 0; a < n_live; ++a) {
+      (a < kept_now ? L.age_slot[a] : L.pend_slot[a - kept_now]) = new_slot[a];
+      L.slot_token[new_slot[a]] = tok_of[a];
     }
   }
   const int n_copy = static_cast<int>(copy.size()) / 2;
@@ -769,10 +779,10 @@ lq_status_t append_impl(lq_cache_t* c, int32_t layer, const void* k, const void*
   if (!c->cfg.auto_compress && kept(L) + n > 3 * W) return LQ_ERR_WINDOW_FULL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // more than one launch's worth of work: a prompt for an empty layer, or a chunk of at least two windows that makes
-  // a layer already in use overflow (not when removed tokens wait for a full key group, W % G != 0).  Below two
-  // windows the index upload of the one-launch path costs more than the launches it saves.
+  // a layer already in use overflow.  Below two windows the index upload of the one-launch path costs more than the
+  // launches it saves.
   if (c->cfg.auto_compress && extra_bytes == 0 &&
-      (L.n_seen == 0 ? n > 3 * W : (n >= 2 * W && kept(L) + n > 3 * W && !residual_mode(c))))
+      (L.n_seen == 0 ? n > 3 * W : (n >= 2 * W && kept(L) + n > 3 * W)))
     return ingest_prompt(c, layer, k, v, n, st);
   int done = 0;
   while (done < n) {

@@ -304,6 +304,9 @@ def test_prompt_ingestion_in_one_launch_equals_token_by_token(W, G, n):
     (64, 64, 4, False, [3 * 64, 64, 3 * 64 + 7, 128]),          # full store first, 4-bit codes
     (128, 64, 2, False, [300, 1000, 129, 2048]),
     (32, 32, 2, True, [50, 60, 200, 32, 33]),                   # recent-window comparator
+    (42, 64, 2, False, [100, 90, 300, 84, 1, 500]),             # W not a multiple of G: waiting tokens in the store
+    (48, 32, 4, False, [140, 96, 97, 400]),                     # the same with 4-bit codes
+    (21, 32, 2, True, [60, 42, 43, 200]),                       # W < G, recent-window comparator
 ])
 def test_chunks_appended_to_a_layer_in_use_take_one_launch_each(W, G, bits, recent, chunks):
     """Chunked prefill: a chunk of at least 2 W tokens that makes a layer in use overflow goes through ONE launch,

@@ -230,7 +230,8 @@ def test_new_entry_points_without_a_device():
     assert c.info(0).n_ctas_overlapped == 0
 
 
-@pytest.mark.parametrize("W,G,recent", [(32, 32, False), (64, 32, False), (128, 64, False), (64, 64, True)])
+@pytest.mark.parametrize("W,G,recent", [(32, 32, False), (64, 32, False), (128, 64, False), (64, 64, True),
+                                        (42, 64, False), (48, 32, False), (100, 64, True), (21, 32, False)])
 def test_chunks_appended_to_a_layer_in_use_go_through_the_one_launch_plan(W, G, recent):
     """A chunk of at least 2 W tokens that makes a layer in use overflow is planned as ONE launch (sources of the new
     key groups, take-over lists, copy list).  Without a device the library plays that plan on token ids and checks
