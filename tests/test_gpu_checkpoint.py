@@ -27,7 +27,7 @@ def _built():
 def test_export_import_round_trip_and_resume(kernel_out, kernel_in, W, G, bits, recent, n_tokens):
     """Checkpoint / resume: an exported image loaded into a fresh cache (lq_import) gives the same image, the same
     attention as the oracle, and the same stores as the oracle after further decode steps."""
-    B, Hq, Hkv, D, n_more = 2, 8, 2, 128, W + 7
+    B, Hq, Hkv, D, n_more, n_chunk = 2, 8, 2, 128, W + 7, 3 * W + 5
     filt = 1 if recent else 0
     src = LogQuantCache(1, B, Hq, Hkv, W, G, max_tokens=n_tokens + n_more + 8, bits=bits, kernel=kernel_out, filter=filt)
     oc = oracle.OracleCache(B, Hq, Hkv, D, W, G, bits=bits, recent_only=recent)
@@ -37,7 +37,7 @@ def test_export_import_round_trip_and_resume(kernel_out, kernel_in, W, G, bits, 
     oc.append(synth.bf16_bits(k0), synth.bf16_bits(v0))
     image = src.export(0)
     src.close()
-    dst = LogQuantCache(2, B, Hq, Hkv, W, G, max_tokens=n_tokens + n_more + 8, bits=bits, kernel=kernel_in, filter=filt)
+    dst = LogQuantCache(2, B, Hq, Hkv, W, G, max_tokens=n_tokens + n_more + n_chunk + 8, bits=bits, kernel=kernel_in, filter=filt)
     dst.import_image(1, image, n_tokens)
     inf = dst.info(1)
     assert (inf.n_seen, inf.n_fp, inf.n_quant) == (n_tokens, image["kept_ids"].size, image["quant_ids"].size)
@@ -58,6 +58,18 @@ def test_export_import_round_trip_and_resume(kernel_out, kernel_in, W, G, bits, 
     dst.decode_attn(1, q, out)
     ref = oc.attention(synth.bf16_bits(q), 1 / np.sqrt(D))
     assert np.abs(out.cpu().numpy() - ref).max() <= attn_tolerance(ref)
+    # a chunk of a prompt on top of the resumed layer: one launch that gathers from the imported rows and the chunk
+    kc, vc = synth.keys_values(48, B, Hkv, n_chunk, D, "cuda", outliers=synth.outlier_channels(47, Hkv, D, 3))
+    before = dst.info(1).n_kernel_launches
+    dst.append(1, kc, vc)
+    assert dst.info(1).n_kernel_launches == before + 1
+    oc.append(synth.bf16_bits(kc), synth.bf16_bits(vc))
+    want, got = oc.export(), dst.export(1)
+    assert all(np.array_equal(got[key], want[key]) for key in want)
+    dst.decode_attn(1, q, out)
+    ref = oc.attention(synth.bf16_bits(q), 1 / np.sqrt(D))
+    assert np.abs(out.cpu().numpy() - ref).max() <= attn_tolerance(ref)
+    assert dst.kernel_status() == 0
     assert dst.kernel_status() == 0
     # a layer that is not empty, or sizes that do not belong to n_seen tokens, are refused and change nothing
     with pytest.raises(LogQuantError):

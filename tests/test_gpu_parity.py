@@ -751,3 +751,37 @@ def test_codes_at_the_rounding_boundaries(W, G, bits):
         assert cache.kernel_status() == 0
         cache.close()
         oc.close()
+
+
+def test_chunks_at_the_largest_window_with_padding_and_stacked_layers():
+    """Chunk ingestion at W = 512 (the largest window), G = 64, on a left-padded batch, on two layers of one cache
+    in turn with overlapped decode launches in between: images bit-exact, attention (which leaves the padding out)
+    within tolerance."""
+    from paper_2503_19950_b200 import LQ_FLAG_OVERLAP_DECODE
+    B, Hq, Hkv, D, W, G, L = 2, 8, 2, 128, 512, 64, 2
+    pad = [700, 0]
+    chunks = [900, 1024, 2 * W, 1500]
+    total = sum(chunks)
+    cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=total + 8, flags=LQ_FLAG_OVERLAP_DECODE)
+    cache.set_padding(pad)
+    ocs = [oracle.OracleCache(B, Hq, Hkv, D, W, G) for _ in range(L)]
+    done = 0
+    for i, n in enumerate(chunks):
+        outs = []
+        for l in range(L):
+            k, v = synth.keys_values(5, B, Hkv, n, D, "cuda", token_start=done, token_total=total, layer=l)
+            cache.append(l, k, v)
+            ocs[l].append(synth.bf16_bits(k), synth.bf16_bits(v))
+        qs = [synth.queries(5, B, Hq, D, i, "cuda", layer=l) for l in range(L)]
+        for l in range(L):   # back to back: the second launch overlaps the first
+            outs.append(torch.empty(B, Hq, D, device="cuda"))
+            cache.decode_attn(l, qs[l], outs[l])
+        done += n
+        for l in range(L):
+            assert_images_equal(cache.export(l), ocs[l].export())
+            ref = ocs[l].attention_subset(synth.bf16_bits(qs[l]), 1 / np.sqrt(D), pad=pad)
+            assert np.abs(outs[l].cpu().numpy() - ref).max() <= attn_tolerance(ref), (i, l)
+    assert cache.kernel_status() == 0
+    cache.close()
+    for oc in ocs:
+        oc.close()
