@@ -128,7 +128,8 @@ typedef struct {
   int64_t n_kernel_launches;   /* kernels this cache has launched so far (all layers)            */
   int32_t n_ctas_overlapped;   /* CTAs of an attention launch that overlaps the launch before it
                                   (LQ_FLAG_OVERLAP_DECODE: a third of the resident wave; else 0)  */
-  int32_t reserved;
+  int32_t n_launches_overlapped; /* attention launches of this cache so far (all layers) that did overlap the
+                                    launch before them                                               */
 } lq_info_t;
 
 /*

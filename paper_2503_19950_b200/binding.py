@@ -36,7 +36,7 @@ class lq_info_t(C.Structure):
     _fields_ = [("n_seen", C.c_int64), ("n_fp", C.c_int64), ("n_quant", C.c_int64), ("n_events", C.c_int64),
                 ("bytes_device", C.c_int64), ("bytes_decode_step", C.c_int64),
                 ("bytes_quant_per_token", C.c_int64), ("n_splits", C.c_int32), ("n_ctas", C.c_int32),
-                ("n_kernel_launches", C.c_int64), ("n_ctas_overlapped", C.c_int32), ("reserved", C.c_int32)]
+                ("n_kernel_launches", C.c_int64), ("n_ctas_overlapped", C.c_int32), ("n_launches_overlapped", C.c_int32)]
 
 
 class lq_image_t(C.Structure):

@@ -59,10 +59,18 @@ struct lq_cache {
   // last work was something else)
   int last_decode_layer = -1;
   cudaStream_t last_decode_stream = nullptr;
-  // layers whose full-precision store got a row from a fused append+attention launch that no later launch has
-  // waited for yet: a launch for such a layer takes the dependency wait first (which, through the chain of waits,
-  // covers every earlier launch) and clears the list
-  std::vector<char> row_in_flight;
+  // Rows written by fused append+attention launches that may still be running.  An overlapped launch of the same
+  // layer reads that row in its main loop, before its dependency wait, so it may overlap only when the writing
+  // launch A is known to be complete.  Known without asking the device: a CTA of these kernels leaves only after
+  // the launch before its own has completed, and a launch starts only when every CTA of the one before it has
+  // started; so while A is incomplete every launch after A has all of its CTAs resident at once, and their CTA
+  // counts cannot add up to more than the device holds.  ctas_since_wait = CTAs of the launches since the last one
+  // that took its dependency wait first (which, through the chain of waits, covers everything before it);
+  // row_mark[layer] = that count right after the layer's last fused launch, -1 = no row in doubt.  Once the
+  // launches after A hold resident_bound CTAs or more, A is complete.
+  std::vector<int64_t> row_mark;
+  int64_t ctas_since_wait = 0;
+  int32_t n_overlapped = 0;  // launches that took the overlapped form (lq_info_t::n_launches_overlapped)
   bool bad_slot_next = false;  // lq_debug_bad_slot_next_append (index-check build only)
   // left padding of a ragged batch (lq_set_padding): pad[b] leading positions of sequence b that attention
   // leaves out.  Device copy per layer: [B][4] row info, [B][fp_words] slot mask, [B][q_words] store mask,
@@ -969,11 +977,16 @@ lq_status_t decode_impl(lq_cache_t* c, int32_t layer, const void* q, float sm_sc
   a.n_extra = 0;
   a.early = 0;
   if (use_mma(c)) {
-    if (c->row_in_flight.empty()) c->row_in_flight.assign(c->cfg.n_layers, 0);
+    if (c->row_mark.empty()) c->row_mark.assign(c->cfg.n_layers, -1);
+    // twice the CTAs of these kernels the device can hold (51 KB of shared memory each: at most four per SM)
+    const int64_t resident_bound = 2LL * max_ctas_decode_mma(c->sm_count);
+    const bool row_safe = c->row_mark[layer] < 0 || c->ctas_since_wait - c->row_mark[layer] >= resident_bound;
     a.early = (c->cfg.flags & LQ_FLAG_OVERLAP_DECODE) && !timed && c->last_decode_layer >= 0 &&
-              c->last_decode_layer != layer && c->last_decode_stream == st && !c->row_in_flight[layer];
-    if (!a.early) std::fill(c->row_in_flight.begin(), c->row_in_flight.end(), 0);
-    if (new_k != nullptr) c->row_in_flight[layer] = 1;
+              c->last_decode_layer != layer && c->last_decode_stream == st && row_safe;
+    if (!a.early) {
+      std::fill(c->row_mark.begin(), c->row_mark.end(), -1);
+      c->ctas_since_wait = 0;
+    }
     plan_decode_mma(a, c->sm_count, c->max_splits, c->cfg.n_splits);
     if (a.rowinfo) {
       a.S = a.early ? c->pad_stride_ov[layer] : c->pad_stride[layer];
@@ -984,6 +997,9 @@ lq_status_t decode_impl(lq_cache_t* c, int32_t layer, const void* q, float sm_sc
       }
       a.n_extra = 0;
     }
+    c->ctas_since_wait += a.rowinfo ? a.n_ctas : c->cfg.batch * c->cfg.n_kv_heads * (a.S - 1) + a.n_extra;  // the grid
+    if (a.early) c->n_overlapped++;
+    c->row_mark[layer] = new_k != nullptr ? c->ctas_since_wait : -1;
     a.tickets = c->tickets;  // the CTA that completes a (b, kv) pair merges it: no second launch
     a.acc = c->acc;
     e = launch_decode_mma(a, st);
@@ -1148,6 +1164,7 @@ lq_status_t lq_cache_info(const lq_cache_t* c, int32_t layer, lq_info_t* info) {
   info->n_events = L.n_events;
   info->bytes_device = c->bytes_device;
   info->n_kernel_launches = c->n_launches;
+  info->n_launches_overlapped = c->n_overlapped;
   info->bytes_quant_per_token = quant_tile_bytes(c->cfg.group, c->cfg.bits / 2) / c->cfg.group;
   info->bytes_decode_step = static_cast<int64_t>(c->cfg.batch) * c->cfg.n_kv_heads *
                             (L.n_quant * info->bytes_quant_per_token + static_cast<int64_t>(L.n_fp) * 4 * kD);

@@ -785,3 +785,53 @@ def test_chunks_at_the_largest_window_with_padding_and_stacked_layers():
     cache.close()
     for oc in ocs:
         oc.close()
+
+
+@pytest.mark.parametrize("L,expect_all", [(16, True), (3, False)])
+def test_fused_steps_of_many_layers_overlap_without_a_wait_per_step(L, expect_all):
+    """Steps of fused append+attention launches over the layers of one cache, back to back on one stream with
+    LQ_FLAG_OVERLAP_DECODE.  The launch of layer l in step t+1 reads the row that the launch of layer l in step t
+    wrote; it may overlap its predecessor only if that earlier launch is known to be complete, which the library
+    derives from the CTAs launched in between (16 layers: enough, every launch after the first overlaps; 3 layers:
+    not enough, the first launch of a step waits).  Outputs of every layer and step against the oracle, images at
+    the end."""
+    from paper_2503_19950_b200 import LQ_FLAG_OVERLAP_DECODE
+    B, Hq, Hkv, D, W, G = 8, 32, 8, 128, 32, 32
+    n0, steps = 128 * W + 5, 6
+    cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=n0 + steps + 8, flags=LQ_FLAG_OVERLAP_DECODE)
+    ocs = [oracle.OracleCache(B, Hq, Hkv, D, W, G) for _ in range(L)]
+    for l in range(L):
+        k, v = synth.keys_values(61, B, Hkv, n0, D, "cuda", layer=l)
+        cache.append(l, k, v)
+        ocs[l].append(synth.bf16_bits(k), synth.bf16_bits(v))
+    ins = [[(synth.keys_values(62 + t, B, Hkv, 1, D, "cuda", layer=l), synth.queries(62 + t, B, Hq, D, t, "cuda", layer=l))
+            for l in range(L)] for t in range(steps)]
+    outs = [[torch.empty(B, Hq, D, device="cuda") for _ in range(L)] for _ in range(steps)]
+    torch.cuda.synchronize()
+    before = cache.info(0).n_launches_overlapped
+    for t in range(steps):          # nothing between the launches: this is the pattern bench.py times
+        for l in range(L):
+            (kn, vn), q = ins[t][l]
+            cache.append_decode_attn(l, kn, vn, q, outs[t][l])
+    torch.cuda.synchronize()
+    inf = cache.info(0)
+    overlapped = inf.n_launches_overlapped - before
+    # CTAs of the L - 1 launches between two launches of a layer, against twice what the device can hold (4 per SM)
+    grid = B * Hkv + inf.n_ctas_overlapped
+    enough = (L - 1) * grid >= 2 * 4 * torch.cuda.get_device_properties(0).multi_processor_count
+    assert enough == expect_all, (grid, L)
+    assert overlapped == (steps * L - 1 if expect_all else steps * (L - 1))
+    for t in range(steps):
+        for l in range(L):
+            (kn, vn), q = ins[t][l]
+            ocs[l].append(synth.bf16_bits(kn), synth.bf16_bits(vn))
+            if l % 5 == 0 or t == steps - 1:
+                ref = ocs[l].attention(synth.bf16_bits(q), 1 / np.sqrt(D), n_threads=8)
+                err = np.abs(outs[t][l].cpu().numpy() - ref).max()
+                assert err <= attn_tolerance(ref), (t, l, err)
+    for l in range(0, L, 5):
+        assert_images_equal(cache.export(l), ocs[l].export())
+    assert cache.kernel_status() == 0
+    cache.close()
+    for oc in ocs:
+        oc.close()
