@@ -83,6 +83,8 @@ typedef enum {
  *     for different layers the caller enqueues on that stream either nothing, or only kernels that were launched
  *     without the programmatic-stream-serialization attribute and do not trigger dependents early (plain launches,
  *     which is what frameworks issue by default): then q, k and v are complete before the decode launch starts.
+ *     (A launch whose layer got a row from an earlier fused lq_append_decode_attn launch overlaps only once that
+ *     launch is known to be complete, which the library derives from the launches enqueued since.)
  *     Without the flag every launch waits for its predecessor before it reads anything. */
 #define LQ_FLAG_OVERLAP_DECODE 1
 
