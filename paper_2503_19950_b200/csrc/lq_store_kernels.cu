@@ -145,6 +145,22 @@ __device__ __forceinline__ uint32_t group_code(float x, const float4& p) {
   }
   return quant_code(x, p.x, p.y, p.z, 15.0f);
 }
+// ORs the code of x into the words of its planes at bit `pos` (a compile-time constant where it matters).  2-bit
+// codes: one predicated OR of a constant per code bit, no integer code in between.
+template <int P>
+__device__ __forceinline__ void add_code(uint32_t (&word)[P], int pos, float x, const float4& p) {
+  if (P == 1) {
+    const float d = __fsub_rn(x, p.x);
+    const bool high = d >= p.z;
+    const bool low = d > (high ? p.w : p.y);
+    if (high) word[0] |= 2u << pos;
+    if (low) word[0] |= 1u << pos;
+  } else {
+    const uint32_t c = quant_code(x, p.x, p.y, p.z, 15.0f);
+#pragma unroll
+    for (int pl = 0; pl < P; ++pl) word[pl] |= ((c >> (2 * pl)) & 3u) << pos;
+  }
+}
 __device__ __forceinline__ float lo_bf16(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float hi_bf16(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 __device__ __forceinline__ uint32_t min_bf16x2(uint32_t a, uint32_t b) {
@@ -257,10 +273,8 @@ __device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kSRow], uin
 #pragma unroll
         for (int nt = 0; nt < 2; ++nt) {
           const uint32_t x = *reinterpret_cast<const uint32_t*>(&sK[t0 + 8 * nt][ch]);
-          const uint32_t ca = group_code<P>(lo_bf16(x), pa), cb = group_code<P>(hi_bf16(x), pb);
-#pragma unroll
-          for (int pl = 0; pl < P; ++pl)
-            word[nt][pl] |= (((ca >> (2 * pl)) & 3u) << (2 * ks)) | (((cb >> (2 * pl)) & 3u) << (16 + 2 * ks));
+          add_code<P>(word[nt], 2 * ks, lo_bf16(x), pa);
+          add_code<P>(word[nt], 16 + 2 * ks, hi_bf16(x), pb);
         }
       }
 #pragma unroll
@@ -283,12 +297,8 @@ __device__ __forceinline__ void quantise_pack_tile(uint16_t (&sK)[G][kSRow], uin
         for (int h = 0; h < 2; ++h) {
           const float4 pv = pV[g * G + tt + h];
           const uint32_t x = *reinterpret_cast<const uint32_t*>(&sV[tt + h][ch]);
-          const uint32_t ca = group_code<P>(lo_bf16(x), pv), cb = group_code<P>(hi_bf16(x), pv);
-#pragma unroll
-          for (int pl = 0; pl < P; ++pl) {
-            word[0][pl] |= ((ca >> (2 * pl)) & 3u) << (16 * h + 2 * mt);
-            word[1][pl] |= ((cb >> (2 * pl)) & 3u) << (16 * h + 2 * mt);
-          }
+          add_code<P>(word[0], 16 * h + 2 * mt, lo_bf16(x), pv);
+          add_code<P>(word[1], 16 * h + 2 * mt, hi_bf16(x), pv);
         }
       }
 #pragma unroll
