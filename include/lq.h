@@ -225,7 +225,8 @@ lq_status_t lq_set_padding(lq_cache_t* cache, const int32_t* pad);
  * writes it to the full-precision store on the way (Algorithm 1's append and Eq. 2 of the same
  * step; the result is the one of the two separate calls).  When the window is full (the overflow
  * step has to run in between; auto_compress = 0 then gives LQ_ERR_WINDOW_FULL), the plain kernel
- * is selected, or the cache is so large that the saved launch no longer pays, the call simply makes
+ * is selected, or the cache is so large that the saved launch no longer pays (only without
+ * LQ_FLAG_OVERLAP_DECODE: with it a separate append would cost the overlap), the call simply makes
  * the two calls.  Errors leave the cache unchanged. */
 lq_status_t lq_append_decode_attn(lq_cache_t* cache, int32_t layer, const void* k, const void* v,
                                   const void* q, float sm_scale, void* out, int32_t out_dtype,

@@ -891,11 +891,14 @@ lq_status_t lq_append_decode_attn(lq_cache_t* c, int32_t layer, const void* k, c
   const int W = c->cfg.window;
   if (L.n_seen + 1 > c->cfg.max_tokens) return LQ_ERR_CAPACITY;
   // The fused instantiation of the kernel runs its main loop about 2 % slower than the plain one
-  // and saves a 2 us launch: it pays below roughly 200 MB per launch.
+  // and saves a 2 us launch: it pays below roughly 200 MB per launch -- unless launches overlap
+  // (LQ_FLAG_OVERLAP_DECODE): a separate append kernel between two attention launches would make the second one
+  // wait for the first, which costs far more than 2 %.
   const int64_t step_bytes = static_cast<int64_t>(c->cfg.batch) * c->cfg.n_kv_heads *
                              (L.n_quant * (quant_tile_bytes(c->cfg.group, c->cfg.bits / 2) / c->cfg.group) +
                               static_cast<int64_t>(L.n_fp) * 4 * kD);
-  if (kept(L) == 3 * W || !use_mma(c) || step_bytes > (192LL << 20)) {
+  const bool overlap = (c->cfg.flags & LQ_FLAG_OVERLAP_DECODE) != 0;
+  if (kept(L) == 3 * W || !use_mma(c) || (!overlap && step_bytes > (192LL << 20))) {
     // the window is full (the overflow step has to run between the two), the plain kernel is
     // selected, or the launch is long: the two separate calls
     lq_status_t s = lq_append(c, layer, k, v, 1, stream);

@@ -198,13 +198,20 @@ def test_config4_timed_entry_points_across_an_overflow(entry):
 # ---- overlapped launches (LQ_FLAG_OVERLAP_DECODE), the configuration bench.py times ------------------
 @pytest.mark.parametrize("entry", ["fused", "host_pinned"])
 @pytest.mark.parametrize("cfg", [dict(B=8, Hq=32, Hkv=8, W=128, G=32, ctx=8192 - 3, seed=2, n_outliers=3),
-                                 dict(B=4, Hq=28, Hkv=4, W=256, G=64, ctx=32768 - 3, seed=4, n_outliers=0)])
+                                 dict(B=4, Hq=28, Hkv=4, W=256, G=64, ctx=32768 - 3, seed=4, n_outliers=0),
+                                 # launches of more than 192 MB: fused only because launches overlap
+                                 dict(B=64, Hq=32, Hkv=8, W=128, G=32, ctx=4096 - 3, seed=3, n_outliers=3),
+                                 dict(B=1, Hq=32, Hkv=32, W=256, G=32, ctx=131072 - 3, seed=5, n_outliers=3,
+                                      entries=("fused",))],
+                         ids=["llama3-8b-8k", "gqa7-32k", "llama3-8b-4k-b64", "mha-128k"])
 def test_overlapped_launches_of_stacked_layers_at_full_size(entry, cfg):
     """Three layer caches with different contents, six decode steps enqueued layer after layer without any
     synchronisation in between (the fourth step overflows every window): every launch but the first of a chain
     overlaps the one before it, with a third of a wave per launch.  Every layer's output of every step and the
     final images must be the oracle's."""
     from paper_2503_19950_b200 import LQ_FLAG_OVERLAP_DECODE
+    if entry not in cfg.get("entries", ("fused", "host_pinned")):
+        pytest.skip("one entry point is enough at this size")
     B, Hq, Hkv, W, G, ctx, seed = (cfg[k] for k in ("B", "Hq", "Hkv", "W", "G", "ctx", "seed"))
     L, n_steps, dev = 3, 6, "cuda"
     total = ctx + n_steps
@@ -217,6 +224,7 @@ def test_overlapped_launches_of_stacked_layers_at_full_size(entry, cfg):
             k, v = synth.keys_values(seed + 10 * l, B, Hkv, n, D, dev, token_start=t0, token_total=total, outliers=outl[l])
             cache.append(l, k, v)
             ocs[l].append(synth.bf16_bits(k), synth.bf16_bits(v))
+    launches0 = cache.info(0).n_kernel_launches
     pin = lambda t: t.cpu().pin_memory()
     outs = [[(torch.full((B, Hq, D), float("nan")).pin_memory() if entry == "host_pinned"
               else torch.full((B, Hq, D), float("nan"), device=dev)) for _ in range(L)] for _ in range(n_steps)]
@@ -237,6 +245,9 @@ def test_overlapped_launches_of_stacked_layers_at_full_size(entry, cfg):
             ocs[l].append(synth.bf16_bits(k), synth.bf16_bits(v))
     torch.cuda.synchronize()             # ... and checked afterwards, against oracles replayed step by step
     assert cache.kernel_status() == 0
+    # one launch per layer and step, except in the step that overflows (overflow kernel, append, attention)
+    if entry == "fused":
+        assert cache.info(0).n_kernel_launches - launches0 == L * (n_steps - 1) + 3 * L
     replay = [oracle.OracleCache(B, Hq, Hkv, D, W, G) for _ in range(L)]
     for l in range(L):
         for t0 in range(0, ctx, 4096):
