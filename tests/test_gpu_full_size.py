@@ -267,3 +267,57 @@ def test_overlapped_launches_of_stacked_layers_at_full_size(entry, cfg):
         assert replay[l].n_events == ocs[l].n_events and ocs[l].n_events >= 1
         assert_images_equal(cache.export(l), ocs[l].export())
     cache.close()
+
+
+def test_long_run_of_overlapped_fused_steps_over_32_layers():
+    """The pattern bench.py times, for longer: 32 layer caches of configuration 2, 260 decode steps of fused
+    append+attention launches enqueued without a pause (three overflow steps per layer on the way), every launch
+    overlapping its predecessor except around the overflow steps.  Four of the layers are replayed in the oracle:
+    their outputs of the last step and their final images must be the oracle's; every layer's output is finite."""
+    from paper_2503_19950_b200 import LQ_FLAG_OVERLAP_DECODE
+    B, Hq, Hkv, W, G, ctx, seed, L, n_steps, dev = 8, 32, 8, 128, 32, 8192, 2, 32, 260, "cuda"
+    checked = (0, 1, 15, 31)
+    total = ctx + n_steps
+    cache = LogQuantCache(L, B, Hq, Hkv, W, G, max_tokens=total + 8, flags=LQ_FLAG_OVERLAP_DECODE)
+    ocs = {l: oracle.OracleCache(B, Hq, Hkv, D, W, G) for l in checked}
+    outl = [synth.outlier_channels(seed + 10 * l, Hkv, D, 3) for l in range(L)]
+    for l in range(L):
+        for t0 in range(0, ctx, 4096):
+            k, v = synth.keys_values(seed + 10 * l, B, Hkv, 4096, D, dev, token_start=t0, token_total=total, outliers=outl[l])
+            cache.append(l, k, v)
+            if l in ocs:
+                ocs[l].append(synth.bf16_bits(k), synth.bf16_bits(v))
+    # a small rotation of inputs per layer (as in the benchmark), generated before the run
+    R = 4
+    kvq = [[(synth.keys_values(seed + 10 * l + 1000 * i, B, Hkv, 1, D, dev, outliers=outl[l]),
+             synth.queries(seed + 10 * l, B, Hq, D, i, dev)) for i in range(R)] for l in range(L)]
+    outs = [torch.full((B, Hq, D), float("nan"), device=dev) for _ in range(L)]
+    torch.cuda.synchronize()
+    before = cache.info(0)
+    for step in range(n_steps):
+        for l in range(L):
+            (k, v), q = kvq[l][step % R]
+            cache.append_decode_attn(l, k, v, q, outs[l])
+    torch.cuda.synchronize()
+    after = cache.info(0)
+    assert cache.kernel_status() == 0
+    # an overflow step takes three launches per layer (overflow kernel, append, attention), none of them overlapped
+    n_ovf = after.n_events - before.n_events
+    assert n_ovf >= 2
+    assert after.n_kernel_launches - before.n_kernel_launches == L * n_steps + 2 * n_ovf * L
+    assert after.n_launches_overlapped - before.n_launches_overlapped >= L * (n_steps - n_ovf) - 1 - n_ovf
+    for l in range(L):
+        assert bool(torch.isfinite(outs[l]).all()), l
+    for l in checked:
+        for step in range(n_steps):
+            (k, v), q = kvq[l][step % R]
+            ocs[l].append(synth.bf16_bits(k), synth.bf16_bits(v))
+        (k, v), q = kvq[l][(n_steps - 1) % R]
+        ref = ocs[l].attention(synth.bf16_bits(q), 1 / np.sqrt(D), n_threads=16)
+        got = outs[l].cpu().numpy().astype(np.float64)
+        err, tol = float(np.abs(got - ref).max()), attn_tolerance(ref)
+        assert err <= tol, f"layer {l}: max|delta| {err:.3e} > {tol:.3e}"
+        assert_images_equal(cache.export(l), ocs[l].export())
+    cache.close()
+    for oc in ocs.values():
+        oc.close()
